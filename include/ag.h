@@ -1,0 +1,206 @@
+/*
+ * ag.h — C boundary of the Attention-Gate (AG) gated attention layer for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The layer is the inference hot path of "In-context KV-Cache Eviction for
+ * LLMs via Attention-Gate" (arXiv 2410.12876):
+ *
+ *   ag_gate_forward   AG(X) = G(MHA'(X), tau)                 Sec. 3.3, Eq. 3, Eq. 4
+ *   ag_compact_kv     keep k_i^(t), v_i^(t) iff AG(X)_i^(t)=1  Sec. 3.3 (after Eq. 4)
+ *   ag_prefill_attn   Softmax(QK^T/sqrt(d_k) - INF(1-M_i))V    Eq. 2 with M_i of Eq. 5
+ *   ag_decode_attn    one query over the retained cache + self Sec. 3.1 (decoding stage), Eq. 5 (j = t)
+ *   ag_cache_append   concatenate the new k, v to the cache    Sec. 3.1 (decoding stage)
+ *
+ * Conventions common to every call
+ * --------------------------------
+ *  - Every data pointer is a DEVICE pointer unless the comment says "host".
+ *    `desc` and the `ag_cache` struct itself live in HOST memory; the arrays
+ *    the cache struct points to are device memory.
+ *  - All tensors are dense, row-major, innermost dimension last, and every
+ *    base pointer is 16-byte aligned.
+ *  - Element type of X, the weights, Q, K, V, O, q, k_new, v_new, o and the
+ *    cache rows is `desc->dtype` (float32 or bfloat16).  Accumulation is
+ *    float32; outputs are rounded to nearest even.
+ *  - Flags are one byte per (sequence, head, token): 1 = retain, 0 = evict.
+ *  - The library allocates no memory and keeps no state between calls.  All
+ *    buffers, the workspace and the stream belong to the caller.  Calls are
+ *    asynchronous on `cuda_stream` (a cudaStream_t passed as void*; NULL is
+ *    the legacy default stream).
+ *  - Return value: AG_OK (0) or a negative ag_status.  Argument errors are
+ *    found on the host before anything is launched.  A condition only the
+ *    device can see (cache slab full on append) sets a bit in a caller-owned
+ *    status word and skips the write; kernels never trap.
+ */
+#ifndef AG_H_
+#define AG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  AG_OK = 0,
+  AG_ERR_INVALID_ARG = -1, /* null / misaligned pointer, non-positive size, h' >= h */
+  AG_ERR_UNSUPPORTED = -2, /* shape or dtype combination without a kernel */
+  AG_ERR_WORKSPACE = -3,   /* workspace missing or smaller than ag_workspace_bytes() */
+  AG_ERR_CAPACITY = -4,    /* a host-known capacity bound is exceeded */
+  AG_ERR_CUDA = -5         /* a CUDA runtime / driver call failed; see ag_last_cuda_error() */
+} ag_status;
+
+typedef enum { AG_F32 = 0, AG_BF16 = 1 } ag_dtype;
+
+/* Which call a workspace query refers to. */
+typedef enum {
+  AG_CALL_GATE = 0,
+  AG_CALL_COMPACT = 1,
+  AG_CALL_PREFILL = 2,
+  AG_CALL_DECODE = 3,
+  AG_CALL_APPEND = 4
+} ag_call;
+
+/* Shape of one AG-gated attention layer (host memory, plain data).
+ * Notation of Sec. 3.1 / 3.3: X in R^{n x d}; h heads of width d_k = d_v;
+ * MHA' has h' < h heads of width d'_k and W^{O'} in R^{h' d'_k x h}. */
+typedef struct {
+  int32_t batch;         /* B  independent sequences                       */
+  int32_t seq;           /* n  prompt length (all sequences share it)      */
+  int32_t hidden;        /* d  width of X (used by ag_gate_forward only)   */
+  int32_t heads;         /* h                                              */
+  int32_t head_dim;      /* d_k = d_v, 64 or 128                           */
+  int32_t gate_heads;    /* h' (must be < h)                               */
+  int32_t gate_head_dim; /* d'_k = d'_v, 64 or 128                         */
+  float tau;             /* threshold of Eq. 4, in (0, 1)                  */
+  int32_t gate_causal;   /* 1: MHA' uses the lower-triangular decoder mask;
+                            0: every token of MHA' sees the whole sequence  */
+  int32_t dtype;         /* ag_dtype                                       */
+} ag_layer_desc;
+
+/* Ragged per-(sequence, head) cache of retained keys and values.  The struct
+ * is host memory; every pointer in it is device memory owned by the caller.
+ * Slab s = b * h + i occupies rows [row_off[s], row_off[s] + cap[s]) of both
+ * row pools; its first len[s] rows are valid, in ascending token order.
+ * Slabs must not overlap.  Rows of a slab beyond len[s] may hold anything. */
+typedef struct {
+  void *k_rows;      /* [pool_rows, head_dim] keys                          */
+  void *v_rows;      /* [pool_rows, head_dim] values                        */
+  int64_t pool_rows; /* rows in each pool                                   */
+  int64_t *row_off;  /* [B*h] first row of each slab                        */
+  int32_t *cap;      /* [B*h] rows reserved for each slab                   */
+  int32_t *len;      /* [B*h] rows in use (written by compact, append)      */
+  int32_t max_cap;   /* host-known upper bound of every cap[s] (sizes the
+                        decode grid; must be >= max_s cap[s])               */
+} ag_cache;
+
+/* Bits of the device status word written by ag_compact_kv / ag_cache_append. */
+#define AG_DEV_OVERFLOW 1 /* a slab had no free row; the write was skipped */
+
+/* Bytes of workspace `which` needs for this layer shape (0 = none needed).
+ * Host-only; returns 0 for an invalid descriptor.  The workspace must be
+ * 256-byte aligned device memory; its contents are scratch. */
+size_t ag_workspace_bytes(const ag_layer_desc *desc, int which);
+
+/*
+ * Step 1 — the gate (Sec. 3.3, Eq. 3 and Eq. 4; gamma: Sec. 3.5).
+ *   Q' = X Wq_g, K' = X Wk_g, V' = X Wv_g, split into h' heads of width d'_k;
+ *   H'_g = Softmax(Q'_g K'_g^T / sqrt(d'_k) [causal if gate_causal]) V'_g;
+ *   s = [H'_1 .. H'_h'] Wo_g                         (n x h);
+ *   flag[t, i] = 1 iff Sigmoid(s[t, i] + gamma[i]) > tau   (strict).
+ * The comparison is done as s + gamma > log(tau / (1 - tau)) in float32.
+ *
+ *   X      [B, n, d]                 in
+ *   Wq_g, Wk_g, Wv_g  [d, h' d'_k]   in   ("in x out", so X W matches Eq. 2)
+ *   Wo_g   [h' d'_k, h]              in
+ *   gamma  [h] float32 or NULL (= 0) in
+ *   scores [B, h, n] float32 or NULL out  s, head-major
+ *   flags  [B, h, n] uint8           out
+ */
+int ag_gate_forward(const ag_layer_desc *desc, const void *X, const void *Wq_g,
+                    const void *Wk_g, const void *Wv_g, const void *Wo_g,
+                    const float *gamma, float *scores, uint8_t *flags, void *ws,
+                    size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Step 2 — selective caching (Sec. 3.3: k_i^(t), v_i^(t) are retained iff
+ * AG(X)_i^(t) = 1).  For every slab s = (b, i):
+ *   prefix[s, j] = #{t < j : flags[s, t] = 1}, j = 0..n  (prefix[s, n] = L_s);
+ *   idx[s, r]    = r-th retained position (ascending), r < L_s;
+ *   cache rows row_off[s] + r  <-  K[s, idx[s, r]], V[s, idx[s, r]] (bit copies);
+ *   cache.len[s] = L_s.
+ * If L_s > cap[s] nothing is copied for that slab, len[s] is set to 0 and
+ * AG_DEV_OVERFLOW is or-ed into *dev_status.
+ * With K = V = NULL only prefix, idx and len are produced (a count pass that
+ * lets the caller lay out tight slabs before the copying pass).
+ *
+ *   K, V    [B, h, n, D]          in (or both NULL)
+ *   flags   [B, h, n] uint8       in
+ *   cache   host struct           in/out (len; k_rows, v_rows)
+ *   prefix  [B, h, n + 1] int32   out
+ *   idx     [B, h, n] int32 or NULL  out (entries r >= L_s are left untouched)
+ *   dev_status  int32 or NULL     in/out (bits are or-ed in)
+ */
+int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
+                  const uint8_t *flags, ag_cache *cache, int32_t *prefix,
+                  int32_t *idx, int32_t *dev_status, void *ws, size_t ws_bytes,
+                  void *cuda_stream);
+
+/*
+ * Step 3 — prefill attention under the eviction mask (Eq. 2 with Eq. 5):
+ *   O_i[j] = sum_t A_i[j, t] V_i[t],
+ *   A_i = row-Softmax(Q_i K_i^T * scale - INF (1 - M_i)),
+ *   M_i[j, t] = 1 if t = j;  flags_i[t] if t < j;  0 if t > j.
+ * The kernel reads the retained keys from the compacted cache (rows
+ * r < prefix[s, j] are exactly the retained t < j) and the self term from
+ * the dense K, V, so `cache` and `prefix` must be those ag_compact_kv wrote
+ * for the same K, V, flags.
+ *
+ *   Q, K, V [B, h, n, D]  in      softmax_scale: 0 means 1/sqrt(D)
+ *   O       [B, h, n, D]  out
+ */
+int ag_prefill_attn(const ag_layer_desc *desc, const void *Q, const void *K,
+                    const void *V, const uint8_t *flags, const ag_cache *cache,
+                    const int32_t *prefix, float softmax_scale, void *O,
+                    void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Step 4a — one decode query per (sequence, head) (Sec. 3.1 decoding stage;
+ * the cache holds only retained tokens, Sec. 3.3; the token always sees its
+ * own key, Eq. 5 case j = t):
+ *   o[s] = Softmax([q[s] . Kc_s^T, q[s] . k_new[s]] * scale) [Vc_s; v_new[s]]
+ * over the len[s] valid rows of slab s.  len[s] = 0 gives o[s] = v_new[s].
+ * Does not modify the cache.
+ *
+ *   q, k_new, v_new [B, h, D]  in      o [B, h, D]  out
+ */
+int ag_decode_attn(const ag_layer_desc *desc, const void *q, const void *k_new,
+                   const void *v_new, const ag_cache *cache,
+                   float softmax_scale, void *o, void *ws, size_t ws_bytes,
+                   void *cuda_stream);
+
+/*
+ * Step 4b — conditional append (Sec. 3.1: the new k, v are concatenated to
+ * the cache; here only when the token's flag retains it):
+ *   if flag_new[s]: rows row_off[s] + len[s] <- k_new[s], v_new[s]; len[s] += 1.
+ * A full slab (len[s] = cap[s]) skips the write and or-s AG_DEV_OVERFLOW into
+ * *dev_status.
+ *
+ *   k_new, v_new [B, h, D]   in      flag_new [B, h] uint8  in
+ *   dev_status   int32 or NULL  in/out
+ */
+int ag_cache_append(const ag_layer_desc *desc, const void *k_new,
+                    const void *v_new, const uint8_t *flag_new, ag_cache *cache,
+                    int32_t *dev_status, void *cuda_stream);
+
+/* Text for an ag_status (static storage, never NULL). */
+const char *ag_status_string(int status);
+
+/* cudaError_t value of the most recent failed CUDA call made by this library
+ * on the calling thread (0 if none). */
+int ag_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AG_H_ */

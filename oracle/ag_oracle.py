@@ -1,0 +1,237 @@
+"""fp64 CPU oracle for the Attention-Gate (AG) gated attention layer.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, dense, obviously-correct
+statement of what the layer computes.  It is imported by the tests, by the
+smoke check and by the benchmark's CPU-baseline leg, and by nothing else: the
+product path (the CUDA library and its Python binding) never calls it and
+shares no code, table or helper with it.
+
+Every function evaluates the paper's definition on the ORIGINAL, uncompacted
+tensors in float64.  There is no compaction, no prefix-sum shortcut, no
+tiling, no online softmax: those are the devices of the GPU path and are what
+this oracle checks.
+
+Layouts (same as the C boundary):
+    X               [B, n, d]        hidden states
+    Wq_g/Wk_g/Wv_g  [d, h' * D']     AG projections, row-major "in x out"
+    Wo_g            [h' * D', h]     AG output projection (Sec. 3.3, W^{O'})
+    Q, K, V, O      [B, h, n, D]
+    scores          [B, h, n]        MHA'(X) transposed to head-major
+    flags           [B, h, n] uint8  1 = retain, 0 = evict
+
+Pins (see tests/test_oracle_*.py): all-keep == textbook causal attention,
+all-evict == O[j] = V[j], brute force over explicit visible-key sets for all
+2^n flag patterns at tiny n, uniform-attention closed forms, gate closed
+forms (Wo'=0, identical rows, n=1), causality of MHA', prefill/decode
+consistency.  What remains unpinned: the paper prints no worked numeric
+example and does not say whether MHA' is causal; "parity unpinned" applies to
+that choice of reading only (both readings are implemented).
+"""
+import math
+
+import numpy as np
+
+F64 = np.float64
+
+
+def _as_f64(a):
+    return np.asarray(a, dtype=F64)
+
+
+def softmax_rows(S):
+    """Row softmax of a matrix whose masked entries are -inf (Eq. 2 with the
+    additive term -INF(1-M) taken in the INF -> infinity limit).  Every row
+    must have at least one finite entry; Eq. 5 guarantees it (the diagonal)."""
+    m = np.max(S, axis=-1, keepdims=True)
+    E = np.exp(S - m)
+    return E / np.sum(E, axis=-1, keepdims=True)
+
+
+# --------------------------------------------------------------------------
+# Step 1: the gate.  Sec. 3.3 "Main architecture", Eq. 3, Eq. 4; gamma from
+# Sec. 3.5 "Initialization".
+# --------------------------------------------------------------------------
+def mha_prime(X, Wq_g, Wk_g, Wv_g, Wo_g, gate_heads, causal=True):
+    """MHA'(X) for one sequence: Eq. 1 / Eq. 2 with h' heads of width D' and
+    the output projection W^{O'} in R^{h'D' x h}.  X [n, d] -> [n, h].
+
+    `causal=True` applies the ordinary lower-triangular decoder mask inside
+    MHA'; `causal=False` lets every token see the whole sequence.  The paper
+    does not say which; causal is the default reading here."""
+    X = _as_f64(X)
+    Wq_g, Wk_g, Wv_g, Wo_g = map(_as_f64, (Wq_g, Wk_g, Wv_g, Wo_g))
+    n = X.shape[0]
+    width = Wq_g.shape[1]
+    assert width % gate_heads == 0
+    Dg = width // gate_heads
+    Qg = X @ Wq_g
+    Kg = X @ Wk_g
+    Vg = X @ Wv_g
+    heads = []
+    for g in range(gate_heads):
+        c = slice(g * Dg, (g + 1) * Dg)
+        S = (Qg[:, c] @ Kg[:, c].T) / math.sqrt(Dg)
+        if causal:
+            j = np.arange(n)[:, None]
+            t = np.arange(n)[None, :]
+            S = np.where(t <= j, S, -np.inf)
+        A = softmax_rows(S)
+        heads.append(A @ Vg[:, c])
+    H = np.concatenate(heads, axis=1)          # [n, h' D']
+    return H @ Wo_g                            # [n, h]
+
+
+def gate_scores(X, Wq_g, Wk_g, Wv_g, Wo_g, gate_heads, causal=True):
+    """scores[b, i, t] = MHA'(X_b)[t, i] for every sequence of the batch."""
+    X = _as_f64(X)
+    out = [mha_prime(X[b], Wq_g, Wk_g, Wv_g, Wo_g, gate_heads, causal).T
+           for b in range(X.shape[0])]
+    return np.stack(out, axis=0)
+
+
+def sigmoid(z):
+    return 1.0 / (1.0 + np.exp(-_as_f64(z)))
+
+
+def gate_flags(scores, gamma, tau):
+    """Eq. 4 with the optional constant inside the Sigmoid:
+    flag = 1 iff Sigmoid(s + gamma_i) > tau (strict).  gamma: scalar, [h] or
+    None.  scores [B, h, n] -> uint8 [B, h, n]."""
+    s = _as_f64(scores)
+    if gamma is None:
+        g = np.zeros(s.shape[1], dtype=F64)
+    else:
+        g = np.broadcast_to(_as_f64(gamma), (s.shape[1],))
+    p = sigmoid(s + g[None, :, None])
+    return (p > tau).astype(np.uint8)
+
+
+def attention_gate(X, Wq_g, Wk_g, Wv_g, Wo_g, gate_heads, gamma, tau, causal=True):
+    """AG(X) = G(MHA'(X), tau), Eq. 3.  Returns (scores, flags)."""
+    s = gate_scores(X, Wq_g, Wk_g, Wv_g, Wo_g, gate_heads, causal)
+    return s, gate_flags(s, gamma, tau)
+
+
+# --------------------------------------------------------------------------
+# Step 2: selective caching.  Sec. 3.3, sentence after Eq. 4: k_i^(t), v_i^(t)
+# are retained iff AG(X)_i^(t) = 1.
+# --------------------------------------------------------------------------
+def retained_indices(flags_i):
+    """Ascending list of token positions whose flag is 1, for one head."""
+    return np.asarray([t for t in range(len(flags_i)) if flags_i[t] == 1],
+                      dtype=np.int64)
+
+
+def exclusive_counts(flags_i):
+    """P[j] = #{t < j : flag[t] = 1} for j = 0..n (so P[n] is the retained
+    length).  Written as the definition, one count per j."""
+    n = len(flags_i)
+    f = np.asarray(flags_i, dtype=np.int64)
+    return np.asarray([int(f[:j].sum()) for j in range(n + 1)], dtype=np.int64)
+
+
+def compact_kv(K, V, flags):
+    """Ragged cache after prefill: cache[b][i] = dict(k=[L, D], v=[L, D],
+    idx=[L]) holding exactly the retained tokens in ascending position.
+    K, V [B, h, n, D] are copied bit-for-bit (dtype preserved)."""
+    K = np.asarray(K)
+    V = np.asarray(V)
+    B, h = flags.shape[0], flags.shape[1]
+    cache = []
+    for b in range(B):
+        row = []
+        for i in range(h):
+            idx = retained_indices(flags[b, i])
+            row.append({"k": K[b, i][idx].copy(), "v": V[b, i][idx].copy(), "idx": idx})
+        cache.append(row)
+    return cache
+
+
+# --------------------------------------------------------------------------
+# Step 3: prefill attention under the eviction mask.  Eq. 2 and Eq. 5.
+# --------------------------------------------------------------------------
+def eviction_mask(flags_i, rows=None):
+    """M_i[j, t] of Eq. 5 for one head: 0 above the diagonal (j < t), 1 on it,
+    AG(X)_i^(t) below it.  j indexes queries (rows), t keys (columns).
+    `rows` selects a subset of query positions; default all."""
+    f = np.asarray(flags_i).astype(np.int64)
+    n = f.shape[0]
+    j = (np.arange(n) if rows is None else np.asarray(rows, dtype=np.int64))[:, None]
+    t = np.arange(n)[None, :]
+    below = np.broadcast_to(f[None, :], (j.shape[0], n))
+    return np.where(j < t, 0, np.where(j == t, 1, below))
+
+
+def prefill_head(Q_i, K_i, V_i, flags_i, scale=None, rows=None):
+    """H_i = Softmax(Q K^T / sqrt(d_k) - INF (1 - M_i)) V for one head
+    (Eq. 2) with M_i from Eq. 5.  Q_i, K_i, V_i [n, D] -> [len(rows), D]."""
+    Q_i, K_i, V_i = map(_as_f64, (Q_i, K_i, V_i))
+    D = Q_i.shape[1]
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    Qs = Q_i if rows is None else Q_i[np.asarray(rows, dtype=np.int64)]
+    S = (Qs @ K_i.T) * scale
+    M = eviction_mask(flags_i, rows)
+    S = np.where(M == 1, S, -np.inf)
+    A = softmax_rows(S)
+    return A @ V_i
+
+
+def prefill_attention(Q, K, V, flags, scale=None):
+    """All heads of all sequences: [B, h, n, D] -> [B, h, n, D] float64."""
+    B, h, n, D = np.asarray(Q).shape
+    O = np.empty((B, h, n, D), dtype=F64)
+    for b in range(B):
+        for i in range(h):
+            O[b, i] = prefill_head(Q[b, i], K[b, i], V[b, i], flags[b, i], scale)
+    return O
+
+
+# --------------------------------------------------------------------------
+# Step 4: decode over the retained cache + conditional append.  Sec. 3.1
+# "decoding stage" (concatenate the new k, v with the cache, attend, update
+# the cache), with the cache holding only retained tokens (Sec. 3.3) and the
+# j = t case of Eq. 5 (a token always attends to itself).
+# --------------------------------------------------------------------------
+def decode_head(q, k_new, v_new, k_cache, v_cache, scale=None):
+    """One query against the retained rows followed by its own (k, v)."""
+    q, k_new, v_new = map(_as_f64, (q, k_new, v_new))
+    D = q.shape[0]
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    Kall = np.concatenate([_as_f64(k_cache).reshape(-1, D), k_new[None, :]], axis=0)
+    Vall = np.concatenate([_as_f64(v_cache).reshape(-1, D), v_new[None, :]], axis=0)
+    s = (Kall @ q) * scale
+    a = softmax_rows(s[None, :])[0]
+    return a @ Vall
+
+
+def decode_attention(q, k_new, v_new, cache, scale=None):
+    """q, k_new, v_new [B, h, D]; cache as returned by compact_kv -> [B, h, D]."""
+    q = np.asarray(q)
+    B, h, D = q.shape
+    o = np.empty((B, h, D), dtype=F64)
+    for b in range(B):
+        for i in range(h):
+            c = cache[b][i]
+            o[b, i] = decode_head(q[b, i], k_new[b, i], v_new[b, i], c["k"], c["v"], scale)
+    return o
+
+
+def cache_append(cache, k_new, v_new, flag_new):
+    """Append (k_new, v_new)[b, i] to slab (b, i) iff flag_new[b, i] = 1.
+    Bit-for-bit copy; mutates and returns `cache`."""
+    k_new = np.asarray(k_new)
+    v_new = np.asarray(v_new)
+    B, h = flag_new.shape
+    for b in range(B):
+        for i in range(h):
+            if flag_new[b, i] == 1:
+                c = cache[b][i]
+                c["k"] = np.concatenate([c["k"], k_new[b, i][None, :]], axis=0)
+                c["v"] = np.concatenate([c["v"], v_new[b, i][None, :]], axis=0)
+    return cache
+
+
+def cache_lengths(cache):
+    return np.asarray([[c["k"].shape[0] for c in row] for row in cache], dtype=np.int64)

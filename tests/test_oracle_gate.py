@@ -1,0 +1,114 @@
+"""Pins for the oracle's gate: MHA' (Sec. 3.3), Eq. 3, Eq. 4, gamma (Sec. 3.5)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ag_oracle as orc
+
+
+def _w(shape, seed, std=1.0):
+    return np.random.default_rng(seed).standard_normal(shape) * std
+
+
+def _gate_inputs(n=11, d=6, hg=2, Dg=4, h=3, seed=0):
+    X = _w((n, d), seed)
+    Wq, Wk, Wv = (_w((d, hg * Dg), seed + 1 + k, 0.5) for k in range(3))
+    Wo = _w((hg * Dg, h), seed + 4, 0.5)
+    return X, Wq, Wk, Wv, Wo
+
+
+def test_zero_output_projection_gives_sigmoid_of_gamma():
+    X, Wq, Wk, Wv, Wo = _gate_inputs()
+    s, f = orc.attention_gate(X[None], Wq, Wk, Wv, 0 * Wo, 2, gamma=2.0, tau=0.5)
+    assert np.all(s == 0)
+    assert np.all(f == 1)          # Sigmoid(2) = 0.88 > 0.5: everything retained at init
+    _, f0 = orc.attention_gate(X[None], Wq, Wk, Wv, 0 * Wo, 2, gamma=0.0, tau=0.5)
+    assert np.all(f0 == 0)         # Sigmoid(0) = 0.5 is not > 0.5 (strict)
+    _, f1 = orc.attention_gate(X[None], Wq, Wk, Wv, 0 * Wo, 2, gamma=None, tau=0.3)
+    assert np.all(f1 == 1)         # 0.5 > 0.3
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_identical_tokens_closed_form(causal):
+    # If every row of X equals x then every value row equals x Wv, attention
+    # averages identical rows, and s = x Wv Wo regardless of the mask.
+    X, Wq, Wk, Wv, Wo = _gate_inputs(seed=3)
+    X = np.tile(X[:1], (X.shape[0], 1))
+    s = orc.mha_prime(X, Wq, Wk, Wv, Wo, 2, causal=causal)
+    want = X[:1] @ Wv @ Wo
+    assert np.max(np.abs(s - want)) < 1e-12
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_single_token(causal):
+    X, Wq, Wk, Wv, Wo = _gate_inputs(n=1, seed=5)
+    s = orc.mha_prime(X, Wq, Wk, Wv, Wo, 2, causal=causal)
+    assert np.max(np.abs(s - X @ Wv @ Wo)) < 1e-13
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_against_library_attention(causal):
+    n, d, hg, Dg, h = 23, 10, 3, 4, 5
+    X, Wq, Wk, Wv, Wo = _gate_inputs(n, d, hg, Dg, h, seed=7)
+    s = orc.mha_prime(X, Wq, Wk, Wv, Wo, hg, causal=causal)
+    tX = torch.from_numpy(X)
+    split = lambda W: (tX @ torch.from_numpy(W)).view(n, hg, Dg).transpose(0, 1)
+    H = torch.nn.functional.scaled_dot_product_attention(split(Wq), split(Wk), split(Wv), is_causal=causal)
+    want = (H.transpose(0, 1).reshape(n, hg * Dg) @ torch.from_numpy(Wo)).numpy()
+    assert np.max(np.abs(s - want)) < 1e-12
+
+
+def test_python_loops_tiny():
+    n, d, hg, Dg, h = 5, 3, 2, 2, 3
+    X, Wq, Wk, Wv, Wo = _gate_inputs(n, d, hg, Dg, h, seed=9)
+    s = orc.mha_prime(X, Wq, Wk, Wv, Wo, hg, causal=True)
+    proj = lambda W, t, c: sum(X[t, a] * W[a, c] for a in range(d))
+    for j in range(n):
+        Hrow = []
+        for g in range(hg):
+            cols = range(g * Dg, (g + 1) * Dg)
+            w = [math.exp(sum(proj(Wq, j, c) * proj(Wk, t, c) for c in cols) / math.sqrt(Dg))
+                 for t in range(j + 1)]
+            z = sum(w)
+            Hrow += [sum(w[t] * proj(Wv, t, c) for t in range(j + 1)) / z for c in cols]
+        for i in range(h):
+            assert abs(s[j, i] - sum(Hrow[c] * Wo[c, i] for c in range(hg * Dg))) < 1e-12
+
+
+def test_causal_reading_ignores_the_future_and_global_does_not():
+    X, Wq, Wk, Wv, Wo = _gate_inputs(n=12, seed=11)
+    X2 = X.copy()
+    X2[8:] += 1.0
+    a = orc.mha_prime(X, Wq, Wk, Wv, Wo, 2, causal=True)
+    b = orc.mha_prime(X2, Wq, Wk, Wv, Wo, 2, causal=True)
+    assert np.array_equal(a[:8], b[:8]) and not np.allclose(a[8:], b[8:])
+    a = orc.mha_prime(X, Wq, Wk, Wv, Wo, 2, causal=False)
+    b = orc.mha_prime(X2, Wq, Wk, Wv, Wo, 2, causal=False)
+    assert not np.allclose(a[:8], b[:8])
+
+
+def test_threshold_rule_and_layout():
+    s = np.asarray([[[-3.0, -0.1, 0.0, 0.1, 3.0], [0.0, 0.0, 0.0, 0.0, 0.0]]])   # [1, 2, 5]
+    f = orc.gate_flags(s, gamma=None, tau=0.5)
+    assert f.dtype == np.uint8 and f.shape == (1, 2, 5)
+    assert f[0, 0].tolist() == [0, 0, 0, 1, 1]
+    f = orc.gate_flags(s, gamma=np.asarray([0.0, 1e-9]), tau=0.5)
+    assert f[0, 1].tolist() == [1, 1, 1, 1, 1]
+    # tau = 0.3: keep iff s > logit(0.3) = -0.8473
+    f = orc.gate_flags(s, gamma=None, tau=0.3)
+    assert f[0, 0].tolist() == [0, 1, 1, 1, 1]
+    # batch / head-major layout of gate_scores
+    X, Wq, Wk, Wv, Wo = _gate_inputs(seed=13)
+    Xb = np.stack([X, X[::-1]])
+    sc = orc.gate_scores(Xb, Wq, Wk, Wv, Wo, 2)
+    assert sc.shape == (2, 3, 11)
+    assert np.array_equal(sc[1], orc.mha_prime(X[::-1], Wq, Wk, Wv, Wo, 2).T)
+
+
+def test_keep_count_grows_with_gamma():
+    X, Wq, Wk, Wv, Wo = _gate_inputs(n=64, seed=15)
+    s = orc.gate_scores(X[None], Wq, Wk, Wv, Wo, 2)
+    counts = [int(orc.gate_flags(s, g, 0.5).sum()) for g in (-5.0, -0.5, 0.0, 0.5, 5.0)]
+    assert counts == sorted(counts) and counts[0] == 0 and counts[-1] == s.size
