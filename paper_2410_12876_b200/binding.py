@@ -1,0 +1,197 @@
+"""ctypes binding of libag.so: argument marshalling only.
+
+Each function has the name and argument order of its C counterpart in
+include/ag.h and does nothing but turn torch tensors into device pointers.
+Every step of the layer runs inside the CUDA library; there is no Python or
+CPU fallback, and loading fails loudly when the library has not been built.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libag.so")
+
+AG_F32, AG_BF16 = 0, 1
+AG_CALL_GATE, AG_CALL_COMPACT, AG_CALL_PREFILL, AG_CALL_DECODE, AG_CALL_APPEND = range(5)
+AG_OK, AG_ERR_INVALID_ARG, AG_ERR_UNSUPPORTED, AG_ERR_WORKSPACE, AG_ERR_CAPACITY, AG_ERR_CUDA = 0, -1, -2, -3, -4, -5
+AG_DEV_OVERFLOW = 1
+
+EXPORTS = (
+    "ag_workspace_bytes", "ag_gate_forward", "ag_compact_kv", "ag_prefill_attn",
+    "ag_decode_attn", "ag_cache_append", "ag_status_string", "ag_last_cuda_error",
+)
+
+
+class AgError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {ag_status_string(status)} ({status})")
+
+
+class ag_layer_desc(ctypes.Structure):
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("seq", ctypes.c_int32), ("hidden", ctypes.c_int32),
+        ("heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+        ("gate_heads", ctypes.c_int32), ("gate_head_dim", ctypes.c_int32),
+        ("tau", ctypes.c_float), ("gate_causal", ctypes.c_int32), ("dtype", ctypes.c_int32),
+    ]
+
+
+class ag_cache(ctypes.Structure):
+    _fields_ = [
+        ("k_rows", ctypes.c_void_p), ("v_rows", ctypes.c_void_p), ("pool_rows", ctypes.c_int64),
+        ("row_off", ctypes.c_void_p), ("cap", ctypes.c_void_p), ("len", ctypes.c_void_p),
+        ("max_cap", ctypes.c_int32),
+    ]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded CUDA library; raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2410_12876_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, f32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        dp, cp = ctypes.POINTER(ag_layer_desc), ctypes.POINTER(ag_cache)
+        L.ag_workspace_bytes.restype = sz
+        L.ag_workspace_bytes.argtypes = [dp, i32]
+        L.ag_gate_forward.restype = i32
+        L.ag_gate_forward.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.ag_compact_kv.restype = i32
+        L.ag_compact_kv.argtypes = [dp, vp, vp, vp, cp, vp, vp, vp, vp, sz, vp]
+        L.ag_prefill_attn.restype = i32
+        L.ag_prefill_attn.argtypes = [dp, vp, vp, vp, vp, cp, vp, f32, vp, vp, sz, vp]
+        L.ag_decode_attn.restype = i32
+        L.ag_decode_attn.argtypes = [dp, vp, vp, vp, cp, f32, vp, vp, sz, vp]
+        L.ag_cache_append.restype = i32
+        L.ag_cache_append.argtypes = [dp, vp, vp, vp, cp, vp, vp]
+        L.ag_status_string.restype = ctypes.c_char_p
+        L.ag_status_string.argtypes = [i32]
+        L.ag_last_cuda_error.restype = i32
+        L.ag_last_cuda_error.argtypes = []
+        _lib = L
+    return _lib
+
+
+def make_desc(shape):
+    """ag_layer_desc from an object with the LayerShape fields."""
+    return ag_layer_desc(shape.batch, shape.seq, shape.hidden, shape.heads, shape.head_dim,
+                         shape.gate_heads, shape.gate_head_dim, float(shape.tau),
+                         int(shape.gate_causal), AG_F32 if shape.dtype == "f32" else AG_BF16)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def _ws(ws):
+    if ws is None:
+        return None, 0
+    return ws.data_ptr(), ws.numel() * ws.element_size()
+
+
+class RaggedCache:
+    """Device buffers of a ragged retained-KV cache plus the host struct the
+    C calls take.  Holds references so the tensors outlive the struct."""
+
+    def __init__(self, k_rows, v_rows, row_off, cap, length, max_cap):
+        self.k_rows, self.v_rows, self.row_off, self.cap, self.len = k_rows, v_rows, row_off, cap, length
+        self.max_cap = int(max_cap)
+        self.struct = ag_cache(_ptr(k_rows), _ptr(v_rows), int(k_rows.shape[0]), _ptr(row_off),
+                               _ptr(cap), _ptr(length), self.max_cap)
+
+    @classmethod
+    def allocate(cls, shape, cap, device="cuda"):
+        """Back-to-back slabs with the given per-slab capacities (int array [B*h])."""
+        import numpy as np
+        cap = np.asarray(cap, dtype=np.int64)
+        off = np.zeros(cap.size, dtype=np.int64)
+        off[1:] = np.cumsum(cap[:-1])
+        pool = int(cap.sum())
+        k = torch.zeros(max(pool, 1), shape.head_dim, dtype=shape.torch_dtype, device=device)
+        v = torch.zeros_like(k)
+        return cls(k[:pool], v[:pool],
+                   torch.from_numpy(off).to(device),
+                   torch.from_numpy(cap.astype("int32")).to(device),
+                   torch.zeros(cap.size, dtype=torch.int32, device=device),
+                   int(cap.max()) if cap.size else 0)
+
+
+def ag_status_string(status):
+    return lib().ag_status_string(int(status)).decode()
+
+
+def ag_last_cuda_error():
+    return lib().ag_last_cuda_error()
+
+
+def ag_workspace_bytes(desc, which):
+    return int(lib().ag_workspace_bytes(ctypes.byref(desc), int(which)))
+
+
+def _check(st, where):
+    if st != AG_OK:
+        raise AgError(st, where)
+    return st
+
+
+def ag_gate_forward(desc, X, Wq_g, Wk_g, Wv_g, Wo_g, gamma, scores, flags, ws, stream=None):
+    p, nbytes = _ws(ws)
+    return _check(lib().ag_gate_forward(ctypes.byref(desc), _ptr(X), _ptr(Wq_g), _ptr(Wk_g), _ptr(Wv_g),
+                                        _ptr(Wo_g), _ptr(gamma), _ptr(scores), _ptr(flags), p, nbytes,
+                                        _stream(stream)), "ag_gate_forward")
+
+
+def ag_compact_kv(desc, K, V, flags, cache, prefix, idx, dev_status, ws, stream=None):
+    p, nbytes = _ws(ws)
+    return _check(lib().ag_compact_kv(ctypes.byref(desc), _ptr(K), _ptr(V), _ptr(flags),
+                                      ctypes.byref(cache.struct), _ptr(prefix), _ptr(idx),
+                                      _ptr(dev_status), p, nbytes, _stream(stream)), "ag_compact_kv")
+
+
+def ag_prefill_attn(desc, Q, K, V, flags, cache, prefix, softmax_scale, O, ws, stream=None):
+    p, nbytes = _ws(ws)
+    return _check(lib().ag_prefill_attn(ctypes.byref(desc), _ptr(Q), _ptr(K), _ptr(V), _ptr(flags),
+                                        ctypes.byref(cache.struct), _ptr(prefix), float(softmax_scale),
+                                        _ptr(O), p, nbytes, _stream(stream)), "ag_prefill_attn")
+
+
+def ag_decode_attn(desc, q, k_new, v_new, cache, softmax_scale, o, ws, stream=None):
+    p, nbytes = _ws(ws)
+    return _check(lib().ag_decode_attn(ctypes.byref(desc), _ptr(q), _ptr(k_new), _ptr(v_new),
+                                       ctypes.byref(cache.struct), float(softmax_scale), _ptr(o), p, nbytes,
+                                       _stream(stream)), "ag_decode_attn")
+
+
+def ag_cache_append(desc, k_new, v_new, flag_new, cache, dev_status, stream=None):
+    return _check(lib().ag_cache_append(ctypes.byref(desc), _ptr(k_new), _ptr(v_new), _ptr(flag_new),
+                                        ctypes.byref(cache.struct), _ptr(dev_status), _stream(stream)),
+                  "ag_cache_append")
+
+
+def workspace(desc, which, device="cuda"):
+    """A device buffer of ag_workspace_bytes(desc, which) bytes (None if 0)."""
+    n = ag_workspace_bytes(desc, which)
+    if n == 0:
+        return None
+    return torch.empty(n, dtype=torch.uint8, device=device)

@@ -1,0 +1,89 @@
+// Shared device/host helpers for the AG-gated attention kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ag.h"
+
+namespace ag {
+
+// ---------------------------------------------------------------- host side
+void set_last_cuda_error(int e);
+
+#define AG_CUDA_TRY(expr)                                 \
+  do {                                                    \
+    cudaError_t _e = (expr);                              \
+    if (_e != cudaSuccess) {                              \
+      ::ag::set_last_cuda_error((int)_e);                 \
+      return AG_ERR_CUDA;                                 \
+    }                                                     \
+  } while (0)
+
+#define AG_LAUNCH_CHECK() AG_CUDA_TRY(cudaGetLastError())
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+// Per-step launchers (defined in the kernel files, called from ag_api.cu).
+size_t gate_workspace_bytes(const ag_layer_desc &d);
+int launch_gate(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk,
+                const void *Wv, const void *Wo, const float *gamma, float *scores,
+                uint8_t *flags, void *ws, cudaStream_t st);
+
+size_t compact_workspace_bytes(const ag_layer_desc &d);
+int launch_compact(const ag_layer_desc &d, const void *K, const void *V, const uint8_t *flags,
+                   const ag_cache &c, int32_t *prefix, int32_t *idx, int32_t *dev_status,
+                   void *ws, cudaStream_t st);
+
+size_t prefill_workspace_bytes(const ag_layer_desc &d);
+int launch_prefill(const ag_layer_desc &d, const void *Q, const void *K, const void *V,
+                   const uint8_t *flags, const ag_cache &c, const int32_t *prefix, float scale,
+                   void *O, void *ws, cudaStream_t st);
+
+size_t decode_workspace_bytes(const ag_layer_desc &d);
+int launch_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
+                  const ag_cache &c, float scale, void *o, void *ws, size_t ws_bytes,
+                  cudaStream_t st);
+int launch_append(const ag_layer_desc &d, const void *k_new, const void *v_new,
+                  const uint8_t *flag_new, const ag_cache &c, int32_t *dev_status,
+                  cudaStream_t st);
+
+// -------------------------------------------------------------- device side
+#ifdef __CUDACC__
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static constexpr int kPerVec = 4;  // elements in a 16-byte vector
+  __device__ static inline void unpack(const uint4 &v, float *f) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+    f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
+  __device__ static inline float load(const float *p) { return *p; }
+  __device__ static inline void store(float *p, float v) { *p = v; }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static constexpr int kPerVec = 8;
+  __device__ static inline void unpack(const uint4 &v, float *f) {
+    // bf16 -> f32 is a 16-bit left shift
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+    f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+    f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+  __device__ static inline float load(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+  __device__ static inline void store(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+__device__ __forceinline__ uint4 ldg128(const void *p) {
+  return __ldg(reinterpret_cast<const uint4 *>(p));
+}
+// Streaming 16-byte load that does not allocate in L1 (data used once).
+__device__ __forceinline__ uint4 ldg128_stream(const void *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+#endif  // __CUDACC__
+
+}  // namespace ag

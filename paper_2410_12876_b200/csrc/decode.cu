@@ -1,0 +1,186 @@
+// Single-query decode attention over the ragged retained cache (Sec. 3.1
+// decoding stage; cache = retained tokens only, Sec. 3.3; the new token always
+// sees its own key, Eq. 5 case j = t).
+//
+// Split-K: slab s = (sequence, head) is cut into chunks of `chunk_rows` rows.
+// decode_partial_kernel reduces one chunk to an un-normalised (o, m, l)
+// triple; decode_combine_kernel merges the chunks of a slab with the self
+// term (q . k_new, v_new) and normalises.  The work is HBM-bound: every cache
+// row is read exactly once with 16-byte vector loads, one row per group of
+// kLanes consecutive lanes, several rows in flight per lane.
+#include "ag_common.cuh"
+
+namespace ag {
+
+constexpr int kMaxSplits = 32;     // chunks per slab the workspace is sized for
+constexpr int kPartThreads = 128;
+constexpr int kUnroll = 4;         // rows in flight per lane group (x2: K and V)
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kPartThreads)
+decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
+                      const T *__restrict__ v_rows, const int64_t *__restrict__ row_off,
+                      const int32_t *__restrict__ len, float scale_log2, int chunk_rows,
+                      float *__restrict__ part_o, float *__restrict__ part_ml) {
+  constexpr int kEpl = Elem<T>::kPerVec;        // elements per lane
+  constexpr int kLanes = D / kEpl;              // lanes per row
+  constexpr int kGroups = kPartThreads / kLanes;
+  const int slab = blockIdx.y, chunk = blockIdx.x;
+  const int L = len[slab];
+  const int r_begin = chunk * chunk_rows;
+  if (r_begin >= L) return;
+  const int r_end = min(L, r_begin + chunk_rows);
+  const int g = threadIdx.x / kLanes, v = threadIdx.x % kLanes;
+
+  float qf[kEpl];
+  Elem<T>::unpack(ldg128(q + (size_t)slab * D + v * kEpl), qf);
+#pragma unroll
+  for (int e = 0; e < kEpl; ++e) qf[e] *= scale_log2;
+
+  const T *Kb = k_rows + (size_t)row_off[slab] * D + v * kEpl;
+  const T *Vb = v_rows + (size_t)row_off[slab] * D + v * kEpl;
+
+  float m = -INFINITY, l = 0.f, o[kEpl];
+#pragma unroll
+  for (int e = 0; e < kEpl; ++e) o[e] = 0.f;
+
+  for (int r = r_begin + g; r < r_end; r += kUnroll * kGroups) {
+    uint4 kv[kUnroll], vv[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int ru = min(r + u * kGroups, r_end - 1);   // clamped rows get weight 0 below
+      kv[u] = ldg128_stream(Kb + (size_t)ru * D);
+      vv[u] = ldg128_stream(Vb + (size_t)ru * D);
+    }
+    float s[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      float kf[kEpl];
+      Elem<T>::unpack(kv[u], kf);
+      float a = 0.f;
+#pragma unroll
+      for (int e = 0; e < kEpl; ++e) a = fmaf(qf[e], kf[e], a);
+#pragma unroll
+      for (int off = kLanes / 2; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+      s[u] = (r + u * kGroups < r_end) ? a : -INFINITY;
+    }
+    float m_new = m;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) m_new = fmaxf(m_new, s[u]);
+    const float alpha = exp2f(m - m_new);   // first pass: exp2(-inf) = 0
+    l *= alpha;
+#pragma unroll
+    for (int e = 0; e < kEpl; ++e) o[e] *= alpha;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const float p = exp2f(s[u] - m_new);
+      l += p;
+      float vf[kEpl];
+      Elem<T>::unpack(vv[u], vf);
+#pragma unroll
+      for (int e = 0; e < kEpl; ++e) o[e] = fmaf(p, vf[e], o[e]);
+    }
+    m = m_new;
+  }
+
+  __shared__ float sm_m[kGroups], sm_l[kGroups];
+  __shared__ float sm_o[kGroups][D];
+  if (v == 0) { sm_m[g] = m; sm_l[g] = l; }
+#pragma unroll
+  for (int e = 0; e < kEpl; ++e) sm_o[g][v * kEpl + e] = o[e];
+  __syncthreads();
+  float mc = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < kGroups; ++i) mc = fmaxf(mc, sm_m[i]);
+  float *po = part_o + ((size_t)slab * kMaxSplits + chunk) * D;
+  for (int d = threadIdx.x; d < D; d += kPartThreads) {
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < kGroups; ++i) acc = fmaf(exp2f(sm_m[i] - mc), sm_o[i][d], acc);
+    po[d] = acc;
+  }
+  if (threadIdx.x == 0) {
+    float lc = 0.f;
+#pragma unroll
+    for (int i = 0; i < kGroups; ++i) lc = fmaf(exp2f(sm_m[i] - mc), sm_l[i], lc);
+    part_ml[((size_t)slab * kMaxSplits + chunk) * 2 + 0] = mc;
+    part_ml[((size_t)slab * kMaxSplits + chunk) * 2 + 1] = lc;
+  }
+}
+
+// One CTA of D threads per slab: thread d owns output dimension d.
+template <typename T, int D>
+__global__ void __launch_bounds__(D)
+decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
+                      const T *__restrict__ v_new, const int32_t *__restrict__ len,
+                      float scale_log2, int chunk_rows, const float *__restrict__ part_o,
+                      const float *__restrict__ part_ml, T *__restrict__ o) {
+  const int slab = blockIdx.x, d = threadIdx.x;
+  const int L = len[slab];
+  const int n_chunks = (L + chunk_rows - 1) / chunk_rows;
+  __shared__ float red[D / 32];
+  float a = Elem<T>::load(q + (size_t)slab * D + d) * Elem<T>::load(k_new + (size_t)slab * D + d);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+  if ((d & 31) == 0) red[d >> 5] = a;
+  __syncthreads();
+  float s_self = 0.f;
+#pragma unroll
+  for (int i = 0; i < D / 32; ++i) s_self += red[i];
+  s_self *= scale_log2;
+  const float *pml = part_ml + (size_t)slab * kMaxSplits * 2;
+  float m = s_self;
+  for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, pml[2 * c]);
+  const float w_self = exp2f(s_self - m);
+  float acc = w_self * Elem<T>::load(v_new + (size_t)slab * D + d);
+  float l = w_self;
+  const float *po = part_o + (size_t)slab * kMaxSplits * D + d;
+  for (int c = 0; c < n_chunks; ++c) {
+    const float w = exp2f(pml[2 * c] - m);
+    acc = fmaf(w, po[(size_t)c * D], acc);
+    l = fmaf(w, pml[2 * c + 1], l);
+  }
+  Elem<T>::store(o + (size_t)slab * D + d, acc / l);
+}
+
+size_t decode_workspace_bytes(const ag_layer_desc &d) {
+  const size_t slabs = (size_t)d.batch * d.heads;
+  return align_up(slabs * kMaxSplits * (d.head_dim + 2) * sizeof(float), 256);
+}
+
+template <typename T, int D>
+static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
+                      const ag_cache &c, float scale, void *o, void *ws, cudaStream_t st) {
+  const int slabs = d.batch * d.heads;
+  int chunk_rows = (c.max_cap + kMaxSplits - 1) / kMaxSplits;
+  chunk_rows = (chunk_rows + 63) / 64 * 64;
+  if (chunk_rows < 256) chunk_rows = 256;
+  const int n_chunks = c.max_cap > 0 ? (c.max_cap + chunk_rows - 1) / chunk_rows : 0;
+  float *part_o = static_cast<float *>(ws);
+  float *part_ml = part_o + (size_t)slabs * kMaxSplits * D;
+  const float scale_log2 = scale * 1.4426950408889634f;
+  if (n_chunks > 0) {
+    dim3 grid(n_chunks, slabs);
+    decode_partial_kernel<T, D><<<grid, kPartThreads, 0, st>>>(
+        static_cast<const T *>(q), static_cast<const T *>(c.k_rows),
+        static_cast<const T *>(c.v_rows), c.row_off, c.len, scale_log2, chunk_rows, part_o, part_ml);
+    AG_LAUNCH_CHECK();
+  }
+  decode_combine_kernel<T, D><<<slabs, D, 0, st>>>(
+      static_cast<const T *>(q), static_cast<const T *>(k_new), static_cast<const T *>(v_new),
+      c.len, scale_log2, chunk_rows, part_o, part_ml, static_cast<T *>(o));
+  AG_LAUNCH_CHECK();
+  return AG_OK;
+}
+
+int launch_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
+                  const ag_cache &c, float scale, void *o, void *ws, size_t, cudaStream_t st) {
+  if (d.dtype == AG_F32) {
+    if (d.head_dim == 64) return run_decode<float, 64>(d, q, k_new, v_new, c, scale, o, ws, st);
+    return run_decode<float, 128>(d, q, k_new, v_new, c, scale, o, ws, st);
+  }
+  if (d.head_dim == 64) return run_decode<__nv_bfloat16, 64>(d, q, k_new, v_new, c, scale, o, ws, st);
+  return run_decode<__nv_bfloat16, 128>(d, q, k_new, v_new, c, scale, o, ws, st);
+}
+
+}  // namespace ag
