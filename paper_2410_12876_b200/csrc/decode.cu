@@ -44,11 +44,14 @@ decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
 #pragma unroll
   for (int e = 0; e < kEpl; ++e) o[e] = 0.f;
 
-  for (int r = r_begin + g; r < r_end; r += kUnroll * kGroups) {
+  // The trip count is the same for every thread of the CTA (the shuffles below
+  // need whole warps); rows past r_end are clamped for the load and get weight 0.
+  for (int r0 = r_begin; r0 < r_end; r0 += kUnroll * kGroups) {
+    const int r = r0 + g;
     uint4 kv[kUnroll], vv[kUnroll];
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
-      const int ru = min(r + u * kGroups, r_end - 1);   // clamped rows get weight 0 below
+      const int ru = min(r + u * kGroups, r_end - 1);
       kv[u] = ldg128_stream(Kb + (size_t)ru * D);
       vv[u] = ldg128_stream(Vb + (size_t)ru * D);
     }
@@ -67,13 +70,14 @@ decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
     float m_new = m;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) m_new = fmaxf(m_new, s[u]);
-    const float alpha = exp2f(m - m_new);   // first pass: exp2(-inf) = 0
+    // a group may not have seen a valid row yet: keep everything at zero then
+    const float alpha = (m_new == -INFINITY) ? 1.f : exp2f(m - m_new);
     l *= alpha;
 #pragma unroll
     for (int e = 0; e < kEpl; ++e) o[e] *= alpha;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
-      const float p = exp2f(s[u] - m_new);
+      const float p = (s[u] == -INFINITY) ? 0.f : exp2f(s[u] - m_new);
       l += p;
       float vf[kEpl];
       Elem<T>::unpack(vv[u], vf);
@@ -96,13 +100,13 @@ decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
   for (int d = threadIdx.x; d < D; d += kPartThreads) {
     float acc = 0.f;
 #pragma unroll
-    for (int i = 0; i < kGroups; ++i) acc = fmaf(exp2f(sm_m[i] - mc), sm_o[i][d], acc);
+    for (int i = 0; i < kGroups; ++i) acc = fmaf(sm_m[i] == -INFINITY ? 0.f : exp2f(sm_m[i] - mc), sm_o[i][d], acc);
     po[d] = acc;
   }
   if (threadIdx.x == 0) {
     float lc = 0.f;
 #pragma unroll
-    for (int i = 0; i < kGroups; ++i) lc = fmaf(exp2f(sm_m[i] - mc), sm_l[i], lc);
+    for (int i = 0; i < kGroups; ++i) lc = fmaf(sm_m[i] == -INFINITY ? 0.f : exp2f(sm_m[i] - mc), sm_l[i], lc);
     part_ml[((size_t)slab * kMaxSplits + chunk) * 2 + 0] = mc;
     part_ml[((size_t)slab * kMaxSplits + chunk) * 2 + 1] = lc;
   }
