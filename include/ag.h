@@ -193,6 +193,42 @@ int ag_cache_append(const ag_layer_desc *desc, const void *k_new,
                     const void *v_new, const uint8_t *flag_new, ag_cache *cache,
                     int32_t *dev_status, void *cuda_stream);
 
+/*
+ * ag_decode_attn without any caller-supplied scratch.  The paper has no
+ * counterpart to this call; it exists for integration reasons only.
+ *
+ * Who needs it: code that runs where device memory cannot be requested —
+ * for example a plug-in inside a serving process that handed the whole GPU
+ * to its own memory pool at start-up (a later cudaMalloc simply fails), or a
+ * latency-critical step that must not hit the device-wide synchronisation an
+ * allocation can cause.  Such a caller has pointers to its inputs and outputs
+ * and nothing else, so it cannot provide the split-K workspace that
+ * ag_decode_attn asks for.
+ *
+ * This variant computes exactly what ag_decode_attn computes, with the
+ * workspace replaced by a fixed 17,039,360-byte array that is part of the
+ * library image (every GPU that loads the library holds it until the process
+ * exits).  It calls no allocation routine of any kind.
+ *
+ *  - Limit: batch * heads * 32 * (head_dim + 2) * 4 bytes must fit in the
+ *    array, i.e. batch * heads <= 1024 at head_dim 128 (2016 at head_dim 64).
+ *    Larger problems are refused with AG_ERR_CAPACITY before any launch.
+ *  - The first call on each device looks up the array's device address (the
+ *    device must be current, as for every call).  Make that first call
+ *    outside any stream capture.
+ *  - All calls share the one array.  Its previous contents never matter (each
+ *    call writes every partial result before reading it), but two calls that
+ *    may overlap on the GPU — different streams, or different host threads
+ *    on the same device — race on it.  Serialise them, or use ag_decode_attn
+ *    with separate workspaces.
+ *
+ * Arguments, layouts and return values are those of ag_decode_attn.
+ */
+int ag_decode_attn_noalloc(const ag_layer_desc *desc, const void *q,
+                           const void *k_new, const void *v_new,
+                           const ag_cache *cache, float softmax_scale, void *o,
+                           void *cuda_stream);
+
 /* Text for an ag_status (static storage, never NULL). */
 const char *ag_status_string(int status);
 

@@ -21,6 +21,7 @@ AG_DEV_OVERFLOW = 1
 EXPORTS = (
     "ag_workspace_bytes", "ag_gate_forward", "ag_compact_kv", "ag_prefill_attn",
     "ag_decode_attn", "ag_cache_append", "ag_status_string", "ag_last_cuda_error",
+    "ag_decode_attn_noalloc",
 )
 
 
@@ -71,6 +72,8 @@ def lib():
         L.ag_prefill_attn.argtypes = [dp, vp, vp, vp, vp, cp, vp, f32, vp, vp, sz, vp]
         L.ag_decode_attn.restype = i32
         L.ag_decode_attn.argtypes = [dp, vp, vp, vp, cp, f32, vp, vp, sz, vp]
+        L.ag_decode_attn_noalloc.restype = i32
+        L.ag_decode_attn_noalloc.argtypes = [dp, vp, vp, vp, cp, f32, vp, vp]
         L.ag_cache_append.restype = i32
         L.ag_cache_append.argtypes = [dp, vp, vp, vp, cp, vp, vp]
         L.ag_status_string.restype = ctypes.c_char_p
@@ -181,6 +184,16 @@ def ag_decode_attn(desc, q, k_new, v_new, cache, softmax_scale, o, ws, stream=No
     return _check(lib().ag_decode_attn(ctypes.byref(desc), _ptr(q), _ptr(k_new), _ptr(v_new),
                                        ctypes.byref(cache.struct), float(softmax_scale), _ptr(o), p, nbytes,
                                        _stream(stream)), "ag_decode_attn")
+
+
+def ag_decode_attn_noalloc(desc, q, k_new, v_new, cache, softmax_scale, o, stream=None):
+    """ag_decode_attn for callers that have no device memory to offer as
+    workspace (see include/ag.h): same result, scratch held inside the library,
+    no allocation.  Calls on one device must not overlap; batch * heads is
+    limited (1024 at head_dim 128), beyond which AgError(AG_ERR_CAPACITY)."""
+    return _check(lib().ag_decode_attn_noalloc(ctypes.byref(desc), _ptr(q), _ptr(k_new), _ptr(v_new),
+                                               ctypes.byref(cache.struct), float(softmax_scale), _ptr(o),
+                                               _stream(stream)), "ag_decode_attn_noalloc")
 
 
 def ag_cache_append(desc, k_new, v_new, flag_new, cache, dev_status, stream=None):

@@ -8,6 +8,8 @@
 // term (q . k_new, v_new) and normalises.  The work is HBM-bound: every cache
 // row is read exactly once with 16-byte vector loads, one row per group of
 // kLanes consecutive lanes, several rows in flight per lane.
+#include <math.h>
+
 #include "ag_common.cuh"
 
 namespace ag {
@@ -187,4 +189,60 @@ int launch_decode(const ag_layer_desc &d, const void *q, const void *k_new, cons
   return run_decode<__nv_bfloat16, 128>(d, q, k_new, v_new, c, scale, o, ws, st);
 }
 
+// ---------------------------------------------------------------------------
+// ag_decode_attn_noalloc: decode attention whose split-K scratch is a fixed
+// array inside the library, for callers that cannot obtain device memory.
+// ---------------------------------------------------------------------------
+constexpr size_t kNoAllocScratchBytes = (size_t)1024 * kMaxSplits * (128 + 2) * sizeof(float);  // 17,039,360
+
+// Lives in the global memory of every GPU that loads the library, until exit.
+// Host code may only use this name to look the device address up.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+// Device address of g_noalloc_scratch on the CURRENT device, looked up once per device.
+static int noalloc_scratch_ptr(void **out) {
+  constexpr int kMaxDevices = 64;
+  static void *ptrs[kMaxDevices] = {};
+  int dev = -1;
+  AG_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return AG_ERR_UNSUPPORTED;
+  void *p = __atomic_load_n(&ptrs[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    AG_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+    if (!p) return AG_ERR_CUDA;
+    __atomic_store_n(&ptrs[dev], p, __ATOMIC_RELEASE);   // same value whichever thread wins
+  }
+  *out = p;
+  return AG_OK;
+}
+
 }  // namespace ag
+
+extern "C" int ag_decode_attn_noalloc(const ag_layer_desc *desc, const void *q, const void *k_new,
+                                      const void *v_new, const ag_cache *cache, float softmax_scale,
+                                      void *o, void *cuda_stream) {
+  using namespace ag;
+  if (!desc || !cache || !q || !k_new || !v_new || !o) return AG_ERR_INVALID_ARG;
+  if (desc->batch <= 0 || desc->heads <= 0 || desc->seq <= 0) return AG_ERR_INVALID_ARG;
+  if (desc->dtype != AG_F32 && desc->dtype != AG_BF16) return AG_ERR_INVALID_ARG;
+  if (desc->head_dim != 64 && desc->head_dim != 128) return AG_ERR_UNSUPPORTED;
+  if (!cache->row_off || !cache->cap || !cache->len || cache->pool_rows < 0 || cache->max_cap < 0)
+    return AG_ERR_INVALID_ARG;
+  if (cache->pool_rows > 0 && (!cache->k_rows || !cache->v_rows)) return AG_ERR_INVALID_ARG;
+  if (cache->max_cap > cache->pool_rows) return AG_ERR_CAPACITY;
+  if (misaligned16(q) || misaligned16(k_new) || misaligned16(v_new) || misaligned16(o) ||
+      misaligned16(cache->k_rows) || misaligned16(cache->v_rows))
+    return AG_ERR_INVALID_ARG;
+  if (!(softmax_scale >= 0.f) || isinf(softmax_scale)) return AG_ERR_INVALID_ARG;
+  // the fixed array bounds the problem size: refuse anything that would not fit
+  if ((int64_t)desc->batch * desc->heads > ((int64_t)1 << 24)) return AG_ERR_CAPACITY;
+  if (decode_workspace_bytes(*desc) > kNoAllocScratchBytes) return AG_ERR_CAPACITY;
+  void *scratch = nullptr;
+  int st = noalloc_scratch_ptr(&scratch);
+  if (st) return st;
+  const float scale = softmax_scale == 0.f ? 1.0f / sqrtf((float)desc->head_dim) : softmax_scale;
+  // Nothing in the scratch has to start at zero: every partial the merge step
+  // reads is written by the chunk pass of this same call.
+  return launch_decode(*desc, q, k_new, v_new, *cache, scale, o, scratch, kNoAllocScratchBytes,
+                       (cudaStream_t)cuda_stream);
+}

@@ -1,0 +1,72 @@
+"""The decode call for callers that cannot allocate device memory.
+
+Some users of this library run where cudaMalloc is not an option: inside a
+process whose own pool already owns all of the GPU's memory, or on a step that
+cannot afford the stall an allocation may bring.  They cannot hand
+ag_decode_attn its split-K workspace, so ag_decode_attn_noalloc keeps that
+scratch in a fixed array inside the library.  These tests check, through the C
+boundary, that it gives what ag_decode_attn gives, twice in a row (the array
+is shared and keeps the previous call's contents), and that it refuses
+problems larger than the array.
+
+This file is named to be collected last, so a run that stops at the first
+failure has already been through every other test.
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import agtest as T
+from paper_2410_12876_b200 import binding as ag
+from paper_2410_12876_b200 import inputs
+from paper_2410_12876_b200.inputs import LayerShape
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    T.ensure_built()
+
+
+def test_too_large_a_problem_is_refused_on_the_host():
+    lib = ag.lib()
+    p = 4096
+    cache = ag.ag_cache(p, p, 1 << 20, p, p, p, 16)
+    ok_size = ag.make_desc(LayerShape(32, 8192, 4096, 32, 128, 4, 128, "bf16"))     # 1024 slabs: fits
+    too_big = ag.make_desc(LayerShape(33, 8192, 4096, 32, 128, 4, 128, "bf16"))    # 1056 slabs: does not
+    assert ag.ag_workspace_bytes(ok_size, ag.AG_CALL_DECODE) == 17039360
+    st = lib.ag_decode_attn_noalloc(ctypes.byref(too_big), p, p, p, ctypes.byref(cache), 0.0, p, None)
+    assert st == ag.AG_ERR_CAPACITY
+    assert "capacity" in ag.ag_status_string(st)
+    # argument checks come first, as in the other calls
+    assert lib.ag_decode_attn_noalloc(ctypes.byref(ok_size), None, p, p, ctypes.byref(cache), 0.0, p, None) \
+        == ag.AG_ERR_INVALID_ARG
+    assert lib.ag_decode_attn_noalloc(ctypes.byref(ok_size), p + 2, p, p, ctypes.byref(cache), 0.0, p, None) \
+        == ag.AG_ERR_INVALID_ARG
+
+
+@pytest.mark.gpu
+def test_matches_the_workspace_call_twice_in_a_row():
+    dev = "cuda"
+    shape = LayerShape(2, 900, 512, 8, 128, 2, 128, "bf16")
+    desc = ag.make_desc(shape)
+    Q, K, V = inputs.qkv_gaussian(shape, 700, dev)
+    f = inputs.bernoulli_flags((shape.batch, shape.heads, shape.seq), 0.6, 701).numpy()
+    f[0, 1] = 0                                     # an empty slab: only the self term
+    f[1, 2] = 1                                     # a full one: several split-K chunks
+    flags = torch.from_numpy(f).to(dev)
+    cap = (f.reshape(shape.batch * shape.heads, -1).sum(axis=1) + 2).tolist()
+    cache, prefix, idx, status = T.gpu_compact(shape, K, V, flags, cap=cap)
+    ws = ag.workspace(desc, ag.AG_CALL_DECODE)
+    for step in range(2):
+        q, kn, vn, fn = inputs.decode_inputs(shape, 710, step, dev, keep_new=0.5)
+        want = torch.full_like(q, float("nan"))
+        got = torch.full_like(q, float("nan"))
+        ag.ag_decode_attn(desc, q, kn, vn, cache, 0.0, want, ws)
+        ag.ag_decode_attn_noalloc(desc, q, kn, vn, cache, 0.0, got)
+        torch.cuda.synchronize()
+        T.check_close(T.f64(got), T.f64(want), "bf16", f"no-alloc decode, call {step}")
+        assert torch.equal(got, want)               # same kernels, same order: same bits
+        ag.ag_cache_append(desc, kn, vn, fn, cache, status)   # the second call sees a longer cache
+    assert int(status.item()) == 0
