@@ -236,6 +236,13 @@ const char *ag_status_string(int status);
  * on the calling thread (0 if none). */
 int ag_last_cuda_error(void);
 
+/* Diagnostic: number of bounded device-side waits (on a TMA load or a tensor-core
+ * completion) that expired in this library's kernels on the current device since
+ * the library was loaded.  0 in a healthy run; a kernel whose wait expired
+ * unwound cleanly but its output is not valid.  Returns -1 if the counter
+ * cannot be read.  Synchronises the device. */
+int ag_device_wait_timeouts(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,7 @@ AG_DEV_OVERFLOW = 1
 EXPORTS = (
     "ag_workspace_bytes", "ag_gate_forward", "ag_compact_kv", "ag_prefill_attn",
     "ag_decode_attn", "ag_cache_append", "ag_status_string", "ag_last_cuda_error",
-    "ag_decode_attn_noalloc",
+    "ag_decode_attn_noalloc", "ag_device_wait_timeouts",
 )
 
 
@@ -80,6 +80,8 @@ def lib():
         L.ag_status_string.argtypes = [i32]
         L.ag_last_cuda_error.restype = i32
         L.ag_last_cuda_error.argtypes = []
+        L.ag_device_wait_timeouts.restype = i32
+        L.ag_device_wait_timeouts.argtypes = []
         _lib = L
     return _lib
 
@@ -146,6 +148,10 @@ def ag_status_string(status):
 
 def ag_last_cuda_error():
     return lib().ag_last_cuda_error()
+
+
+def ag_device_wait_timeouts():
+    return lib().ag_device_wait_timeouts()
 
 
 def ag_workspace_bytes(desc, which):

@@ -172,4 +172,10 @@ const char *ag_status_string(int status) {
 
 int ag_last_cuda_error(void) { return ag::g_last_cuda_error; }
 
+int ag_device_wait_timeouts(void) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+  const int a = gemm_tc_wait_timeouts();
+  return a < 0 ? -1 : a;
+}
+
 }  // extern "C"

@@ -31,6 +31,12 @@ int launch_gate(const ag_layer_desc &d, const void *X, const void *Wq, const voi
                 const void *Wv, const void *Wo, const float *gamma, float *scores,
                 uint8_t *flags, void *ws, cudaStream_t st);
 
+// Tensor-core (tcgen05) projection GEMM for bf16 inputs: C[M, 3*GD] f32 = X [W0 | W1 | W2].
+bool gate_proj_tc_supported(int K, int GD);
+int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, int M,
+                        int K, int GD, cudaStream_t st);
+int gemm_tc_wait_timeouts();
+
 size_t compact_workspace_bytes(const ag_layer_desc &d);
 int launch_compact(const ag_layer_desc &d, const void *K, const void *V, const uint8_t *flags,
                    const ag_cache &c, int32_t *prefix, int32_t *idx, int32_t *dev_status,

@@ -105,11 +105,16 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
   float *qkv = static_cast<float *>(ws);
   float *hcat = reinterpret_cast<float *>(static_cast<char *>(ws) +
                                           align_up((size_t)M * 3 * GD * sizeof(float), 256));
-  dim3 grid(3 * GD / kGemmBN, (M + kGemmBM - 1) / kGemmBM);
-  gate_proj_kernel<T><<<grid, 256, 0, st>>>(static_cast<const T *>(X), static_cast<const T *>(Wq),
-                                            static_cast<const T *>(Wk), static_cast<const T *>(Wv),
-                                            qkv, M, d.hidden, GD);
-  AG_LAUNCH_CHECK();
+  if (sizeof(T) == 2 && gate_proj_tc_supported(d.hidden, GD)) {
+    int rc = launch_gate_proj_tc(X, Wq, Wk, Wv, qkv, M, d.hidden, GD, st);
+    if (rc) return rc;
+  } else {
+    dim3 grid(3 * GD / kGemmBN, (M + kGemmBM - 1) / kGemmBM);
+    gate_proj_kernel<T><<<grid, 256, 0, st>>>(static_cast<const T *>(X), static_cast<const T *>(Wq),
+                                              static_cast<const T *>(Wk), static_cast<const T *>(Wv),
+                                              qkv, M, d.hidden, GD);
+    AG_LAUNCH_CHECK();
+  }
 
   SimtAttnArgs a{};
   a.Q = qkv; a.K = qkv + GD; a.V = qkv + 2 * GD; a.O = hcat;

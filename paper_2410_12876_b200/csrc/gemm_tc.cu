@@ -1,0 +1,209 @@
+// bf16 x bf16 -> f32 GEMM on the 5th-generation tensor cores (tcgen05.mma with
+// the accumulator in tensor memory, operands staged by TMA), used for the gate's
+// projection [Q' | K' | V'] = X [Wq_g | Wk_g | Wv_g] (Sec. 3.3, MHA').
+//
+// One CTA computes a 128 x BN tile of the packed output.  Warp 0 drives TMA,
+// warp 1 owns TMEM and issues the MMAs, warps 2..5 drain the accumulator.
+//   A = X   [M, K]  row-major  -> K-major operand, 128-byte swizzled rows
+//   B = W   [K, GD] row-major  -> MN-major operand: panels of [64 k][64 n]
+// Products of bf16 inputs are exact in the f32 accumulator, so the result
+// differs from an exact evaluation only by f32 summation error.
+#include "ag_common.cuh"
+#include "umma.cuh"
+
+namespace ag {
+
+using namespace umma;
+
+constexpr int kTcBM = 128, kTcBK = 64, kTcThreads = 192;
+
+template <int BN> struct GemmTcCfg {
+  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static constexpr int kABytes = kTcBM * kTcBK * 2;          // 16 KB
+  static constexpr int kPanelBytes = kTcBK * 64 * 2;         // [64 k][64 n] = 8 KB
+  static constexpr int kBBytes = (BN / 64) * kPanelBytes;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+                    const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
+                    float *__restrict__ C, int M, int K, int GD) {
+  using Cfg = GemmTcCfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + Cfg::kStages * Cfg::kStageBytes);
+  uint64_t *empty = full + Cfg::kStages;
+  uint64_t *acc_full = empty + Cfg::kStages;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.y * kTcBM;
+  const int n0 = blockIdx.x * BN;              // column in the packed [3 * GD] output
+  const int which = n0 / GD, nw = n0 % GD;     // BN divides GD: a tile never straddles two weights
+  const CUtensorMap *tmB = which == 0 ? &tmB0 : (which == 1 ? &tmB1 : &tmB2);
+  const int num_kb = (K + kTcBK - 1) / kTcBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    fence_barrier_init();
+    prefetch_tensormap(&tmA);
+    prefetch_tensormap(tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, BN);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_acc = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % Cfg::kStages;
+        const uint32_t ph = (kb / Cfg::kStages) & 1;
+        if (!mbar_wait(&empty[s], ph ^ 1)) break;
+        uint8_t *a = smem + s * Cfg::kStageBytes, *b = a + Cfg::kABytes;
+        mbar_arrive_expect_tx(&full[s], Cfg::kStageBytes);
+        tma_load_2d(a, &tmA, &full[s], kb * kTcBK, m0);
+#pragma unroll
+        for (int p = 0; p < BN / 64; ++p)
+          tma_load_2d(b + p * Cfg::kPanelBytes, tmB, &full[s], nw + p * 64, kb * kTcBK);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16_f32(kTcBM, BN, false, true);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb && ok; ++kb) {
+        const int s = kb % Cfg::kStages;
+        const uint32_t ph = (kb / Cfg::kStages) & 1;
+        ok = mbar_wait(&full[s], ph);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t a = smem_u32(smem + s * Cfg::kStageBytes), b = a + Cfg::kABytes;
+#pragma unroll
+        for (int k = 0; k < kTcBK / 16; ++k) {
+          // 16 elements of K: 32 bytes along a K-major row; 16 k-rows (2048 B) of an MN-major panel
+          mma_ss(tmem_acc, desc_kmajor_sw128(a + k * 32), desc_mnmajor_sw128(b + k * 2048, Cfg::kPanelBytes),
+                 idesc, (kb | k) != 0);
+        }
+        mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
+      }
+      mma_commit(acc_full);        // accumulator complete (or unwinding)
+    }
+  } else {
+    // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32)
+    const int quad = warp & 3;
+    const int row = m0 + quad * 32 + lane;
+    const bool ok = mbar_wait(acc_full, 0);
+    tc_fence_after_sync();
+    if (ok && num_kb > 0) {
+      float *crow = C + (size_t)row * 3 * GD + n0;
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 32) {
+        uint32_t r[32];
+        tmem_ld_x32(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
+        tmem_ld_wait();
+        if (row < M) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 4)
+            *reinterpret_cast<uint4 *>(crow + c + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+        }
+      }
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_acc, BN);
+}
+
+// ------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+int make_tmap_2d_bf16(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t pitch_bytes,
+                      uint32_t box_rows, uint32_t box_cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { set_last_cuda_error((int)cudaErrorNotSupported); return AG_ERR_CUDA; }
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { set_last_cuda_error(1000 + (int)r); return AG_ERR_CUDA; }
+  return AG_OK;
+}
+
+int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t planes, uint64_t rows, uint64_t cols,
+                      uint32_t box_rows, uint32_t box_cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { set_last_cuda_error((int)cudaErrorNotSupported); return AG_ERR_CUDA; }
+  cuuint64_t dims[3] = {cols, rows, planes};
+  cuuint64_t strides[2] = {cols * 2, rows * cols * 2};
+  cuuint32_t box[3] = {box_cols, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { set_last_cuda_error(1000 + (int)r); return AG_ERR_CUDA; }
+  return AG_OK;
+}
+
+// ----------------------------------------------------------------- launch
+template <int BN>
+static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, int M, int K,
+                       int GD, cudaStream_t st) {
+  using Cfg = GemmTcCfg<BN>;
+  CUtensorMap tmA, tmB[3];
+  int rc = make_tmap_2d_bf16(&tmA, X, M, K, (uint64_t)K * 2, kTcBM, kTcBK);
+  if (rc) return rc;
+  const void *Ws[3] = {W0, W1, W2};
+  for (int i = 0; i < 3; ++i) {
+    rc = make_tmap_2d_bf16(&tmB[i], Ws[i], K, GD, (uint64_t)GD * 2, kTcBK, 64);
+    if (rc) return rc;
+  }
+  auto kern = gemm_bf16_tc_kernel<BN>;
+  AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+  dim3 grid(3 * GD / BN, (M + kTcBM - 1) / kTcBM);
+  kern<<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(tmA, tmB[0], tmB[1], tmB[2], C, M, K, GD);
+  AG_LAUNCH_CHECK();
+  return AG_OK;
+}
+
+bool gate_proj_tc_supported(int K, int GD) { return GD % 128 == 0 && K % 8 == 0; }
+
+int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, int M, int K,
+                        int GD, cudaStream_t st) {
+  if (GD % 256 == 0) return run_gemm_tc<256>(X, W0, W1, W2, C, M, K, GD, st);
+  return run_gemm_tc<128>(X, W0, W1, W2, C, M, K, GD, st);
+}
+
+int gemm_tc_wait_timeouts() {
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, umma::g_wait_expired, sizeof(int)) != cudaSuccess) return -1;
+  return v;
+}
+
+}  // namespace ag

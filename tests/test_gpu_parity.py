@@ -284,3 +284,8 @@ def test_results_are_bitwise_repeatable():
         runs.append([scores, flags, prefix, O, o, cache.len.clone(), cache.k_rows.clone()])
     for a, b in zip(*runs):
         assert torch.equal(a, b)
+
+
+def test_no_device_wait_expired():
+    """Runs after the other tests of this file: no bounded wait inside a kernel gave up."""
+    assert ag.ag_device_wait_timeouts() == 0
