@@ -47,6 +47,12 @@ int launch_prefill(const ag_layer_desc &d, const void *Q, const void *K, const v
                    const uint8_t *flags, const ag_cache &c, const int32_t *prefix, float scale,
                    void *O, void *ws, cudaStream_t st);
 
+// Tensor-core (tcgen05) prefill attention for bf16, head_dim 128.
+bool prefill_tc_supported(const ag_layer_desc &d, const ag_cache &c);
+int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, const void *V, const ag_cache &c,
+                      const int32_t *prefix, float scale, void *O, cudaStream_t st);
+int prefill_tc_wait_timeouts();
+
 size_t decode_workspace_bytes(const ag_layer_desc &d);
 int launch_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
                   const ag_cache &c, float scale, void *o, void *ws, size_t ws_bytes,

@@ -108,8 +108,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
         uint32_t r[32];
-        tmem_ld_x32(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
-        tmem_ld_wait();
+        tmem_ld_x32_sync(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
         if (row < M) {
 #pragma unroll
           for (int e = 0; e < 32; e += 4)

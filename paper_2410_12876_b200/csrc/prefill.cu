@@ -30,6 +30,7 @@ static int run_prefill_simt(const ag_layer_desc &d, const void *Q, const void *K
 int launch_prefill(const ag_layer_desc &d, const void *Q, const void *K, const void *V,
                    const uint8_t *, const ag_cache &c, const int32_t *prefix, float scale,
                    void *O, void *, cudaStream_t st) {
+  if (prefill_tc_supported(d, c)) return launch_prefill_tc(d, Q, K, V, c, prefix, scale, O, st);
   if (d.dtype == AG_F32) {
     if (d.head_dim == 64) return run_prefill_simt<float, 64>(d, Q, K, V, c, prefix, scale, O, st);
     return run_prefill_simt<float, 128>(d, Q, K, V, c, prefix, scale, O, st);
