@@ -174,8 +174,8 @@ int ag_last_cuda_error(void) { return ag::g_last_cuda_error; }
 
 int ag_device_wait_timeouts(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return -1;
-  const int a = gemm_tc_wait_timeouts(), b = prefill_tc_wait_timeouts();
-  return (a < 0 || b < 0) ? -1 : a + b;
+  const int a = gemm_tc_wait_timeouts(), b = prefill_tc_wait_timeouts(), c = gate_attn_tc_wait_timeouts();
+  return (a < 0 || b < 0 || c < 0) ? -1 : a + b + c;
 }
 
 }  // extern "C"

@@ -31,10 +31,16 @@ int launch_gate(const ag_layer_desc &d, const void *X, const void *Wq, const voi
                 const void *Wv, const void *Wo, const float *gamma, float *scores,
                 uint8_t *flags, void *ws, cudaStream_t st);
 
-// Tensor-core (tcgen05) projection GEMM for bf16 inputs: C[M, 3*GD] f32 = X [W0 | W1 | W2].
+// Tensor-core (tcgen05) projection GEMM for bf16 inputs: [M, 3*GD] = X [W0 | W1 | W2], written
+// either as float32 (C) or, when Chi / Clo are given, as the bf16 pair hi + lo of each float32 value.
 bool gate_proj_tc_supported(int K, int GD);
-int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, int M,
-                        int K, int GD, cudaStream_t st);
+int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, void *Chi,
+                        void *Clo, int M, int K, int GD, cudaStream_t st);
+// Tensor-core MHA' (Sec. 3.3) on the hi / lo pairs: H' [B*n, GD] float32.
+bool gate_attn_tc_supported(const ag_layer_desc &d);
+int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *qkv_lo, float *hcat,
+                        cudaStream_t st);
+int gate_attn_tc_wait_timeouts();
 int gemm_tc_wait_timeouts();
 
 size_t compact_workspace_bytes(const ag_layer_desc &d);

@@ -1,8 +1,9 @@
 // The Attention-Gate pass (Sec. 3.3): AG(X) = G(MHA'(X), tau), Eq. 3 / Eq. 4,
 // with the optional constant gamma inside the Sigmoid (Sec. 3.5).
 //
-//   1. gate_proj_kernel    [Q' | K' | V'] = X [Wq_g | Wk_g | Wv_g]   -> float32
-//   2. simt_attn_kernel    H'_g = Softmax(Q'_g K'_g^T / sqrt(d'_k)) V'_g, float32
+//   1. projection   [Q' | K' | V'] = X [Wq_g | Wk_g | Wv_g]   (tcgen05 GEMM for bf16, else CUDA cores)
+//   2. MHA'         H'_g = Softmax(Q'_g K'_g^T / sqrt(d'_k)) V'_g  (tcgen05 on bf16 hi/lo pairs for
+//                   bf16 layers with d'_k = 128, else float32 on CUDA cores)
 //   3. gate_out_kernel     s = [H'_1 .. H'_h'] Wo_g;  flag = s + gamma > logit(tau)
 //
 // The scores decide a hard threshold, so everything after the (exact) products
@@ -105,34 +106,43 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
   float *qkv = static_cast<float *>(ws);
   float *hcat = reinterpret_cast<float *>(static_cast<char *>(ws) +
                                           align_up((size_t)M * 3 * GD * sizeof(float), 256));
-  if (sizeof(T) == 2 && gate_proj_tc_supported(d.hidden, GD)) {
-    int rc = launch_gate_proj_tc(X, Wq, Wk, Wv, qkv, M, d.hidden, GD, st);
+  if (sizeof(T) == 2 && gate_attn_tc_supported(d)) {
+    // tensor-core path: projections as bf16 hi/lo pairs, MHA' on tcgen05 with three products per term
+    void *hi = ws;
+    void *lo = static_cast<char *>(ws) + (size_t)M * 3 * GD * sizeof(__nv_bfloat16);
+    int rc = launch_gate_proj_tc(X, Wq, Wk, Wv, nullptr, hi, lo, M, d.hidden, GD, st);
+    if (rc) return rc;
+    rc = launch_gate_attn_tc(d, hi, lo, hcat, st);
     if (rc) return rc;
   } else {
-    dim3 grid(3 * GD / kGemmBN, (M + kGemmBM - 1) / kGemmBM);
-    gate_proj_kernel<T><<<grid, 256, 0, st>>>(static_cast<const T *>(X), static_cast<const T *>(Wq),
-                                              static_cast<const T *>(Wk), static_cast<const T *>(Wv),
-                                              qkv, M, d.hidden, GD);
-    AG_LAUNCH_CHECK();
+    if (sizeof(T) == 2 && gate_proj_tc_supported(d.hidden, GD)) {
+      int rc = launch_gate_proj_tc(X, Wq, Wk, Wv, qkv, nullptr, nullptr, M, d.hidden, GD, st);
+      if (rc) return rc;
+    } else {
+      dim3 grid(3 * GD / kGemmBN, (M + kGemmBM - 1) / kGemmBM);
+      gate_proj_kernel<T><<<grid, 256, 0, st>>>(static_cast<const T *>(X), static_cast<const T *>(Wq),
+                                                static_cast<const T *>(Wk), static_cast<const T *>(Wv),
+                                                qkv, M, d.hidden, GD);
+      AG_LAUNCH_CHECK();
+    }
+    SimtAttnArgs a{};
+    a.Q = qkv; a.K = qkv + GD; a.V = qkv + 2 * GD; a.O = hcat;
+    a.n = d.seq; a.inner = d.gate_heads;
+    a.q_batch = a.k_batch = a.v_batch = (long long)d.seq * 3 * GD;
+    a.q_inner = a.k_inner = a.v_inner = Dg;
+    a.q_row = a.k_row = a.v_row = 3 * GD;
+    a.o_batch = (long long)d.seq * GD; a.o_inner = Dg; a.o_row = GD;
+    a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)Dg));
+    const int problems = d.batch * d.gate_heads;
+    int rc;
+    if (Dg == 64)
+      rc = d.gate_causal ? launch_simt_attn<float, float, 64, kGateCausal>(a, problems, st)
+                         : launch_simt_attn<float, float, 64, kGateFull>(a, problems, st);
+    else
+      rc = d.gate_causal ? launch_simt_attn<float, float, 128, kGateCausal>(a, problems, st)
+                         : launch_simt_attn<float, float, 128, kGateFull>(a, problems, st);
+    if (rc) return rc;
   }
-
-  SimtAttnArgs a{};
-  a.Q = qkv; a.K = qkv + GD; a.V = qkv + 2 * GD; a.O = hcat;
-  a.n = d.seq; a.inner = d.gate_heads;
-  a.q_batch = a.k_batch = a.v_batch = (long long)d.seq * 3 * GD;
-  a.q_inner = a.k_inner = a.v_inner = Dg;
-  a.q_row = a.k_row = a.v_row = 3 * GD;
-  a.o_batch = (long long)d.seq * GD; a.o_inner = Dg; a.o_row = GD;
-  a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)Dg));
-  const int problems = d.batch * d.gate_heads;
-  int rc;
-  if (Dg == 64)
-    rc = d.gate_causal ? launch_simt_attn<float, float, 64, kGateCausal>(a, problems, st)
-                       : launch_simt_attn<float, float, 64, kGateFull>(a, problems, st);
-  else
-    rc = d.gate_causal ? launch_simt_attn<float, float, 128, kGateCausal>(a, problems, st)
-                       : launch_simt_attn<float, float, 128, kGateFull>(a, problems, st);
-  if (rc) return rc;
 
   const float logit_tau = (float)log((double)d.tau / (1.0 - (double)d.tau));
   const int warps = M, blocks = (warps * 32 + 255) / 256;

@@ -30,7 +30,8 @@ template <int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                     const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
-                    float *__restrict__ C, int M, int K, int GD) {
+                    float *__restrict__ C, __nv_bfloat16 *__restrict__ Chi, __nv_bfloat16 *__restrict__ Clo,
+                    int M, int K, int GD) {
   using Cfg = GemmTcCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -104,15 +105,33 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const bool ok = mbar_wait(acc_full, 0);
     tc_fence_after_sync();
     if (ok && num_kb > 0) {
-      float *crow = C + (size_t)row * 3 * GD + n0;
+      const size_t crow = (size_t)row * 3 * GD + n0;
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
         uint32_t r[32];
         tmem_ld_x32_sync(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
         if (row < M) {
+          if (Chi) {
+            // x = hi + lo in bf16 pairs, for consumers that rebuild float32 precision from three products
 #pragma unroll
-          for (int e = 0; e < 32; e += 4)
-            *reinterpret_cast<uint4 *>(crow + c + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+            for (int e = 0; e < 32; e += 8) {
+              uint32_t h[4], l[4];
+#pragma unroll
+              for (int q = 0; q < 8; q += 2) {
+                float h0, l0, h1, l1;
+                split_bf16(__uint_as_float(r[e + q]), h0, l0);
+                split_bf16(__uint_as_float(r[e + q + 1]), h1, l1);
+                h[q >> 1] = pack_bf16x2(h0, h1);
+                l[q >> 1] = pack_bf16x2(l0, l1);
+              }
+              *reinterpret_cast<uint4 *>(Chi + crow + c + e) = make_uint4(h[0], h[1], h[2], h[3]);
+              *reinterpret_cast<uint4 *>(Clo + crow + c + e) = make_uint4(l[0], l[1], l[2], l[3]);
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; e += 4)
+              *reinterpret_cast<uint4 *>(C + crow + c + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+          }
         }
       }
     }
@@ -172,8 +191,8 @@ int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t planes, uint6
 
 // ----------------------------------------------------------------- launch
 template <int BN>
-static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, int M, int K,
-                       int GD, cudaStream_t st) {
+static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C,
+                       __nv_bfloat16 *Chi, __nv_bfloat16 *Clo, int M, int K, int GD, cudaStream_t st) {
   using Cfg = GemmTcCfg<BN>;
   CUtensorMap tmA, tmB[3];
   int rc = make_tmap_2d_bf16(&tmA, X, M, K, (uint64_t)K * 2, kTcBM, kTcBK);
@@ -186,17 +205,18 @@ static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void
   auto kern = gemm_bf16_tc_kernel<BN>;
   AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
   dim3 grid(3 * GD / BN, (M + kTcBM - 1) / kTcBM);
-  kern<<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(tmA, tmB[0], tmB[1], tmB[2], C, M, K, GD);
+  kern<<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(tmA, tmB[0], tmB[1], tmB[2], C, Chi, Clo, M, K, GD);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
 
 bool gate_proj_tc_supported(int K, int GD) { return GD % 128 == 0 && K % 8 == 0; }
 
-int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, int M, int K,
-                        int GD, cudaStream_t st) {
-  if (GD % 256 == 0) return run_gemm_tc<256>(X, W0, W1, W2, C, M, K, GD, st);
-  return run_gemm_tc<128>(X, W0, W1, W2, C, M, K, GD, st);
+int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, void *Chi,
+                        void *Clo, int M, int K, int GD, cudaStream_t st) {
+  auto hi = static_cast<__nv_bfloat16 *>(Chi), lo = static_cast<__nv_bfloat16 *>(Clo);
+  if (GD % 256 == 0) return run_gemm_tc<256>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
+  return run_gemm_tc<128>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
 }
 
 int gemm_tc_wait_timeouts() {

@@ -7,6 +7,7 @@
 // return) instead of spinning forever.
 #pragma once
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -223,6 +224,22 @@ __device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint32_t *r) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi): |x - hi - lo| <= 2^-17 |x|.
+__device__ __forceinline__ void split_bf16(float x, float &hi, float &lo) {
+  hi = __uint_as_float(__float_as_uint(__bfloat162float(__float2bfloat16_rn(x))));
+  lo = x - hi;
+}
 
 }  // namespace umma
 
