@@ -33,6 +33,8 @@ WORKLOADS = {
     # name: (shape, decode steps per step, description)
     "prefill7b": (inputs.PREFILL7B, 16, "Llama-2-7B-shaped AG-gated layer, batch 1 x seq 4096, keep rates U[0.3,0.8] per head"),
     "tiny": (inputs.TINY, 16, "fp32 correctness layer, batch 1 x seq 128, ~50% keep"),
+    "deep_layer": (inputs.DEEP_LAYER, 16, "deep-layer pattern, batch 1 x seq 16384: 24 heads keep ~10%, 8 heads keep nothing"),
+    "decode_ragged": (inputs.DECODE_RAGGED, 16, "ragged decode, batch 32 x 32 heads, retained lengths U[0.2,0.9] x 8192, keep-new Bernoulli(0.5)"),
 }
 # kernels launched per call of the library
 LAUNCHES = {"gate": 3, "compact": 2, "prefill": 1, "decode": 2, "append": 1}
@@ -106,26 +108,53 @@ class LayerRun:
         self.dev = dev
         self.desc = ag.make_desc(sh)
         B, h, n, D = sh.batch, sh.heads, sh.seq, sh.head_dim
-        self.X = inputs.hidden_states(sh, seed, dev)
-        self.W = inputs.layer_weights(sh, seed + 10, dev)
-        self.Q, self.K, self.V = inputs.project_qkv(sh, self.X, self.W)
-        self.scores = torch.empty(B, h, n, dtype=torch.float32, device=dev)
-        self.flags = torch.empty(B, h, n, dtype=torch.uint8, device=dev)
-        self.prefix = torch.empty(B, h, n + 1, dtype=torch.int32, device=dev)
-        self.O = torch.empty_like(self.Q)
+        self.name = name
+        self.has_gate = name in ("prefill7b", "tiny")
+        self.has_prefill = name != "decode_ragged"
+        if self.has_gate:
+            self.X = inputs.hidden_states(sh, seed, dev)
+            self.W = inputs.layer_weights(sh, seed + 10, dev)
+            self.Q, self.K, self.V = inputs.project_qkv(sh, self.X, self.W)
+        elif self.has_prefill:
+            self.Q, self.K, self.V = inputs.qkv_gaussian(sh, seed, dev)
+        else:
+            self.Q = torch.empty(0, dtype=sh.torch_dtype, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.ws = {c: ag.workspace(self.desc, c, dev) for c in
-                   (ag.AG_CALL_GATE, ag.AG_CALL_COMPACT, ag.AG_CALL_PREFILL, ag.AG_CALL_DECODE)}
-        # dense-capacity slabs: n rows + the decode steps of one pass
-        self.cache = ag.RaggedCache.allocate(sh, [n + self.decode_steps] * (B * h), dev)
-        self.dq = [inputs.decode_inputs(sh, seed + 500, s, dev, keep_new=0.5) for s in range(self.decode_steps)]
+        calls = [ag.AG_CALL_DECODE] + ([ag.AG_CALL_COMPACT, ag.AG_CALL_PREFILL] if self.has_prefill else []) \
+            + ([ag.AG_CALL_GATE] if self.has_gate else [])
+        self.ws = {c: ag.workspace(self.desc, c, dev) for c in calls}
+        if self.has_prefill:
+            self.scores = torch.empty(B, h, n, dtype=torch.float32, device=dev)
+            self.flags = torch.empty(B, h, n, dtype=torch.uint8, device=dev)
+            self.prefix = torch.empty(B, h, n + 1, dtype=torch.int32, device=dev)
+            self.O = torch.empty_like(self.Q)
+            # dense-capacity slabs: n rows + the decode steps of one pass
+            self.cache = ag.RaggedCache.allocate(sh, [n + self.decode_steps] * (B * h), dev)
+        else:
+            # the cache is the input: tight slabs of seeded random length, filled with N(0, 1)
+            self.L0 = inputs.ragged_lengths(B * h, n, seed + 30)
+            self.cache = ag.RaggedCache.allocate(sh, (self.L0.astype(np.int64) + 256).tolist(), dev)
+            for t, sd in ((self.cache.k_rows, seed + 31), (self.cache.v_rows, seed + 32)):
+                step_rows = 1 << 20
+                for r0 in range(0, t.shape[0], step_rows):
+                    r1 = min(t.shape[0], r0 + step_rows)
+                    t[r0:r1] = inputs.randn((r1 - r0, D), sd + r0, dev, sh.torch_dtype)
+            self.len0 = torch.from_numpy(self.L0).to(dev)
+            self.cache.len.copy_(self.len0)
+        self.dq = [inputs.decode_inputs(sh, seed + 500, s, dev, keep_new=0.1 if name == "deep_layer" else 0.5)
+                   for s in range(self.decode_steps)]
         self.o = torch.empty(B, h, D, dtype=sh.torch_dtype, device=dev)
         # gamma: per-head keep rate ~ U[0.3, 0.8], calibrated on the scores at gamma = 0
         self.gamma = None
-        self.gate()
-        keep = inputs.keep_targets_uniform(h, seed + 20) if name != "tiny" else [0.5] * h
-        self.gamma = inputs.calibrate_gamma(self.scores, keep, sh.tau).to(dev)
-        self.keep_target = np.asarray(keep)
+        if self.has_gate:
+            self.gate()
+            keep = inputs.keep_targets_uniform(h, seed + 20) if name != "tiny" else [0.5] * h
+            self.gamma = inputs.calibrate_gamma(self.scores, keep, sh.tau).to(dev)
+        elif self.has_prefill:
+            f, empty = inputs.deep_layer_flags(sh, seed + 20)
+            self.flags.copy_(f.to(dev))
+            for q in self.dq:
+                q[3][:, torch.from_numpy(empty).to(dev)] = 0     # fully evicted heads stay empty
 
     def gate(self):
         W, ag = self.W, self.ag
@@ -158,17 +187,32 @@ class LayerRun:
             fn(*a)
             e.record()
             ev[key].append((s, e))
-        timed("gate", self.gate)
-        timed("compact", self.compact)
-        timed("prefill", self.prefill)
+        if self.has_gate:
+            timed("gate", self.gate)
+        if self.has_prefill:
+            timed("compact", self.compact)
+            timed("prefill", self.prefill)
+        else:
+            self.cache.len.copy_(self.len0)      # every pass starts from the same cache
         timed("decode", lambda: [self.decode(s) for s in range(self.decode_steps)])
 
     def tokens_per_step(self):
-        return self.shape.batch * (self.shape.seq + self.decode_steps)
+        return self.shape.batch * ((self.shape.seq if self.has_prefill else 0) + self.decode_steps)
 
     def launches_per_step(self):
-        return (LAUNCHES["gate"] + LAUNCHES["compact"] + LAUNCHES["prefill"] +
+        return ((LAUNCHES["gate"] if self.has_gate else 0) +
+                (LAUNCHES["compact"] + LAUNCHES["prefill"] if self.has_prefill else 0) +
                 self.decode_steps * (LAUNCHES["decode"] + LAUNCHES["append"]))
+
+    def decode_bytes_per_decode_step(self):
+        """Bytes one decode step must move: every valid cache row once (K and V) plus
+        q, k_new, v_new, o.  Lengths grow linearly over the pass, so the mean of the
+        lengths before the first and after the last step is the per-step average."""
+        e = 2 if self.shape.dtype == "bf16" else 4
+        D = self.shape.head_dim
+        before = (self.prefix[:, :, -1] if self.has_prefill else self.len0).to(torch.float64).sum().item()
+        after = self.cache.len.to(torch.float64).sum().item()
+        return 2.0 * 0.5 * (before + after) * D * e + 4.0 * self.shape.batch * self.shape.heads * D * e
 
     def effective_prefill_flops(self):
         """4 D sum_j (1 + P[j]): QK^T and PV over the visible (query, key) pairs only."""
@@ -220,18 +264,25 @@ def run_ours(args, rank, world, dev):
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     total_ms = sum(s.elapsed_time(e) for s, e in step_ev)
-    per_call_ms = {k: float(np.mean([s.elapsed_time(e) for s, e in v])) for k, v in ev.items()}
+    per_call_ms = {k: float(np.mean([s.elapsed_time(e) for s, e in v])) for k, v in ev.items() if v}
     assert int(run.status.item()) == 0, "device reported a cache overflow"
+    timeouts = run.ag.ag_device_wait_timeouts()
+    assert timeouts == 0, f"{timeouts} bounded device waits expired"
 
     # end to end: pinned host inputs in, results out, through the same calls
     sh = run.shape
-    host_in = [t.detach().cpu().pin_memory() for t in (run.X, run.Q, run.K, run.V)]
-    dev_in = [run.X, run.Q, run.K, run.V]
-    host_O = torch.empty(run.O.shape, dtype=run.O.dtype).pin_memory()
-    host_flags = torch.empty(run.flags.shape, dtype=torch.uint8).pin_memory()
-    host_o = torch.empty(run.o.shape, dtype=run.o.dtype).pin_memory()
+    if run.has_gate:
+        dev_in = [run.X, run.Q, run.K, run.V]
+    elif run.has_prefill:
+        dev_in = [run.Q, run.K, run.V, run.flags]
+    else:
+        dev_in = []
+    dev_in += [t for q in run.dq for t in q]
+    dev_out = ([run.O, run.flags] if run.has_prefill else []) + [run.o]
+    host_in = [t.detach().cpu().pin_memory() for t in dev_in]
+    host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in dev_out]
     h2d = sum(t.numel() * t.element_size() for t in host_in)
-    d2h = sum(t.numel() * t.element_size() for t in (host_O, host_flags, host_o))
+    d2h = sum(t.numel() * t.element_size() for t in host_out)
     e2e_steps = max(1, min(args.steps, 10))
     barrier()
     t_e2e = 0.0
@@ -242,9 +293,8 @@ def run_ours(args, rank, world, dev):
         for d, hsrc in zip(dev_in, host_in):
             d.copy_(hsrc, non_blocking=True)
         run.step()
-        host_O.copy_(run.O, non_blocking=True)
-        host_flags.copy_(run.flags, non_blocking=True)
-        host_o.copy_(run.o, non_blocking=True)
+        for hdst, d in zip(host_out, dev_out):
+            hdst.copy_(d, non_blocking=True)
         e.record()
         e.synchronize()
         t_e2e += s.elapsed_time(e)
@@ -258,13 +308,35 @@ def run_ours(args, rank, world, dev):
         return None
     tokens = run.tokens_per_step() * world
     peaks = _peaks()
-    f_eff = run.effective_prefill_flops()
-    dom = max(per_call_ms, key=per_call_ms.get)
-    prefill_tflops = f_eff / (per_call_ms["prefill"] * 1e-3) / 1e12
-    gate_tflops = run.gate_flops() / (per_call_ms["gate"] * 1e-3) / 1e12
-    roof = {"bound": "tensor", "kernel": "ag_prefill_attn", "achieved": prefill_tflops, "peak": peaks["bf16_tflops"],
-            "unit": "TFLOP/s", "frac": prefill_tflops / peaks["bf16_tflops"], "traffic": None,
-            "peak_source": peaks["source"], "algorithmic_flops": f_eff, "ms": per_call_ms["prefill"]}
+    rooflines = {}
+    dec_bytes = run.decode_bytes_per_decode_step()
+    dec_ms = per_call_ms["decode"] / run.decode_steps
+    dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
+    rooflines["decode"] = {"bound": "hbm", "kernel": "ag_decode_attn + ag_cache_append", "achieved": dec_gbs,
+                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"],
+                           "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": dec_bytes,
+                           "ms": dec_ms}
+    if run.has_prefill:
+        f_eff = run.effective_prefill_flops()
+        tf = f_eff / (per_call_ms["prefill"] * 1e-3) / 1e12
+        rooflines["prefill"] = {"bound": "tensor", "kernel": "ag_prefill_attn", "achieved": tf,
+                                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
+                                "traffic": None, "peak_source": peaks["source"], "algorithmic_flops": f_eff,
+                                "ms": per_call_ms["prefill"]}
+        e = 2 if sh.dtype == "bf16" else 4
+        kept = float(run.prefix[:, :, -1].to(torch.float64).sum().item())
+        cb = 2.0 * (2.0 * kept * sh.head_dim * e) + sh.batch * sh.heads * sh.seq * 9.0
+        gbs = cb / (per_call_ms["compact"] * 1e-3) / 1e9
+        rooflines["compact"] = {"bound": "hbm", "kernel": "ag_compact_kv", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                                "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                                "peak_source": peaks["source"], "algorithmic_bytes": cb, "ms": per_call_ms["compact"]}
+    if run.has_gate:
+        gf = run.gate_flops()
+        tf = gf / (per_call_ms["gate"] * 1e-3) / 1e12
+        rooflines["gate"] = {"bound": "tensor", "kernel": "ag_gate_forward", "achieved": tf, "peak": peaks["bf16_tflops"],
+                             "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "traffic": None,
+                             "peak_source": peaks["source"], "algorithmic_flops": gf, "ms": per_call_ms["gate"]}
+    head = "prefill" if run.has_prefill else "decode"
     ms_step = total_ms / args.steps
     out = {
         "metric": METRIC, "value": tokens * args.steps / (total_ms * 1e-3), "unit": UNIT,
@@ -274,19 +346,21 @@ def run_ours(args, rank, world, dev):
         "config": {"workload": args.workload, "description": run.desc_text, "batch": sh.batch, "seq": sh.seq,
                    "hidden": sh.hidden, "heads": sh.heads, "head_dim": sh.head_dim, "gate_heads": sh.gate_heads,
                    "gate_head_dim": sh.gate_head_dim, "decode_steps_per_step": run.decode_steps,
-                   "mean_keep": float(run.flags.float().mean().item()), "l2": "flushed between steps (256 MiB write)",
-                   "replicas": world},
+                   "mean_keep": float(run.flags.float().mean().item()) if run.has_prefill else None,
+                   "l2": "flushed between steps (256 MiB write)", "replicas": world},
         "clocks": clocks,
         "e2e": {"value": tokens * e2e_steps / (t_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": run.launches_per_step() * args.steps,
-        "roofline": roof,
+        "roofline": rooflines[head],
+        "rooflines": rooflines,
         "per_call_ms": per_call_ms,
-        "dominant_call": dom,
-        "prefill_tokens_per_s": sh.batch * sh.seq / ((per_call_ms["gate"] + per_call_ms["compact"] + per_call_ms["prefill"]) * 1e-3),
+        "dominant_call": max(per_call_ms, key=per_call_ms.get),
         "decode_tokens_per_s": sh.batch * run.decode_steps / (per_call_ms["decode"] * 1e-3),
-        "gate_tflops": gate_tflops,
     }
+    if run.has_prefill:
+        pre_ms = sum(per_call_ms.get(k, 0.0) for k in ("gate", "compact", "prefill"))
+        out["prefill_tokens_per_s"] = sh.batch * sh.seq / (pre_ms * 1e-3)
     return out, run
 
 
@@ -400,7 +474,7 @@ def main():
     res = run_ours(args, rank, world, torch.device("cuda", local))
     if rank == 0:
         out, run = res
-        if not args.no_cpu_baseline and world == 1:
+        if not args.no_cpu_baseline and world == 1 and args.workload in ("prefill7b", "tiny"):
             cb = oracle_sample(args.workload, 2000)
             cb.pop("est_step_s", None)
             out["cpu_baseline"] = cb

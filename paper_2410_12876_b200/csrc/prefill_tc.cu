@@ -7,14 +7,14 @@
 // the compacted rows the mask is a staircase, so only the tiles that touch it
 // need per-element masking and evicted keys are never loaded.
 //
-//   warp 0      TMA: Q tile once, then K / V tiles of 128 cache rows (2 stages)
+//   warp 0      TMA: Q tile once, then K / V tiles of 128 cache rows
 //   warp 1      owns tensor memory, issues S = Q K^T (tcgen05.mma, operands in
 //               shared memory) and O += P V (P read from tensor memory)
 //   warps 2..5  one query row per thread: online softmax on S read from TMEM,
 //               P written back to TMEM as bf16, O rescaled only when the running
 //               maximum grows by more than 2^8, final normalisation and store
 //
-// TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P [384,448) (bf16 pairs).
+// TMEM columns: S [0,128), overwritten in place by P [0,64) (bf16 pairs); O [128,256).
 // The self term seeds the running softmax (m = s_jj, l = 1) and its value row
 // is added in the epilogue: O_j = (sum_r p_r v_r + w_self v_j) / l.
 #include "ag_common.cuh"
@@ -28,9 +28,8 @@ constexpr int kPfThreads = 192;
 constexpr int kPfBM = 128, kPfBN = 128, kPfD = 128;
 constexpr int kPfPanel = 128 * 128;                   // [128 rows][64 bf16] = 16 KB
 constexpr int kPfTile = 2 * kPfPanel;                 // 32 KB
-constexpr int kPfStages = 2;
-constexpr int kPfSmemBytes = kPfTile * (1 + 2 * kPfStages) + 1024 + 256;
-constexpr uint32_t kColS = 0, kColO = 256, kColP = 384, kTmemCols = 512;
+constexpr int kPfSmemBytes = 3 * kPfTile + 1024 + 256;
+constexpr uint32_t kColS = 0, kColP = 0, kColO = 128, kTmemCols = 256;
 constexpr float kRescaleThreshold = 8.f;              // log2 units
 
 struct PrefillTcArgs {
@@ -43,20 +42,21 @@ struct PrefillTcArgs {
   float scale_log2;
 };
 
-__global__ void __launch_bounds__(kPfThreads, 1)
+// Two CTAs share an SM (256 TMEM columns, 97 KB of shared memory each): inside a
+// CTA the chain S = Q K^T -> softmax -> O += P V is serial, and the tensor core
+// works on one CTA's tile while the other CTA is in its softmax.
+__global__ void __launch_bounds__(kPfThreads, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const PrefillTcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sQ = smem;
-  uint8_t *sK = sQ + kPfTile;                      // [stage][tile]
-  uint8_t *sV = sK + kPfStages * kPfTile;
-  uint64_t *bars = reinterpret_cast<uint64_t *>(sV + kPfStages * kPfTile);
-  uint64_t *q_full = bars;
-  uint64_t *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;
-  uint64_t *s_full = bars + 9;                     // [2]
-  uint64_t *p_ready = bars + 11, *pv_done = bars + 12;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 13);
+  uint8_t *sK = sQ + kPfTile;
+  uint8_t *sV = sK + kPfTile;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(sV + kPfTile);
+  uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 2, *v_full = bars + 3, *v_empty = bars + 4;
+  uint64_t *s_full = bars + 5, *p_ready = bars + 6, *pv_done = bars + 7;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // heaviest query tiles first
@@ -71,11 +71,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
-      mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
-      mbar_init(&s_full[s], 1);
-    }
+    mbar_init(k_full, 1); mbar_init(k_empty, 1);
+    mbar_init(v_full, 1); mbar_init(v_empty, 1);
+    mbar_init(s_full, 1);
     mbar_init(p_ready, 128);
     mbar_init(pv_done, 1);
     fence_barrier_init();
@@ -97,56 +95,49 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       tma_load_3d(sQ, &tmQ, q_full, 0, j0, slab);
       tma_load_3d(sQ + kPfPanel, &tmQ, q_full, 64, j0, slab);
       for (int i = 0; i < n_kv; ++i) {
-        const int st = i & 1;
-        const uint32_t ph = (i >> 1) & 1;
+        const uint32_t ph = i & 1;
         const int y = row0 + i * kPfBN;
-        if (!mbar_wait(&k_empty[st], ph ^ 1)) break;
-        mbar_arrive_expect_tx(&k_full[st], kPfTile);
-        tma_load_2d(sK + st * kPfTile, &tmK, &k_full[st], 0, y);
-        tma_load_2d(sK + st * kPfTile + kPfPanel, &tmK, &k_full[st], 64, y);
-        if (!mbar_wait(&v_empty[st], ph ^ 1)) break;
-        mbar_arrive_expect_tx(&v_full[st], kPfTile);
-        tma_load_2d(sV + st * kPfTile, &tmV, &v_full[st], 0, y);
-        tma_load_2d(sV + st * kPfTile + kPfPanel, &tmV, &v_full[st], 64, y);
+        if (!mbar_wait(k_empty, ph ^ 1)) break;
+        mbar_arrive_expect_tx(k_full, kPfTile);
+        tma_load_2d(sK, &tmK, k_full, 0, y);
+        tma_load_2d(sK + kPfPanel, &tmK, k_full, 64, y);
+        if (!mbar_wait(v_empty, ph ^ 1)) break;
+        mbar_arrive_expect_tx(v_full, kPfTile);
+        tma_load_2d(sV, &tmV, v_full, 0, y);
+        tma_load_2d(sV + kPfPanel, &tmV, v_full, 64, y);
       }
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0 && n_kv > 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(kPfBM, kPfBN, false, false);
-      constexpr uint32_t idesc_pv = idesc_bf16_f32(kPfBM, kPfD, false, true);
-      const uint32_t q_addr = smem_u32(sQ);
-      auto issue_qk = [&](int i) -> bool {
-        const int st = i & 1;
-        if (!mbar_wait(&k_full[st], (i >> 1) & 1)) return false;
+      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+      bool ok = mbar_wait(q_full, 0);
+      for (int i = 0; i < n_kv && ok; ++i) {
+        const uint32_t ph = i & 1;
+        // keys of this tile any row can see, rounded up to the MMA's N / K granularity
+        const int keys = min(kPfBN, (max_bound - i * kPfBN + 15) & ~15);
+        const uint32_t idesc_qk = idesc_bf16_f32(kPfBM, keys, false, false);
+        constexpr uint32_t idesc_pv = idesc_bf16_f32(kPfBM, kPfD, false, true);
+        if (!mbar_wait(k_full, ph)) { ok = false; break; }
         tc_fence_after_sync();
-        const uint32_t k_addr = smem_u32(sK + st * kPfTile);
 #pragma unroll
         for (int k = 0; k < kPfD / 16; ++k) {
           const uint32_t off = (k >> 2) * kPfPanel + (k & 3) * 32;
-          mma_ss(tmem + kColS + st * 128, desc_kmajor_sw128(q_addr + off), desc_kmajor_sw128(k_addr + off),
-                 idesc_qk, k != 0);
+          mma_ss(tmem + kColS, desc_kmajor_sw128(q_addr + off), desc_kmajor_sw128(k_addr + off), idesc_qk, k != 0);
         }
-        mma_commit(&k_empty[st]);
-        mma_commit(&s_full[st]);
-        return true;
-      };
-      bool ok = mbar_wait(q_full, 0);
-      ok = ok && issue_qk(0);
-      for (int i = 0; i < n_kv && ok; ++i) {
-        if (i + 1 < n_kv) ok = issue_qk(i + 1);
-        if (!ok) break;
-        const int st = i & 1;
-        if (!mbar_wait(p_ready, i & 1)) { ok = false; break; }
-        if (!mbar_wait(&v_full[st], (i >> 1) & 1)) { ok = false; break; }
+        mma_commit(k_empty);
+        mma_commit(s_full);
+        if (!mbar_wait(p_ready, ph)) { ok = false; break; }
+        if (!mbar_wait(v_full, ph)) { ok = false; break; }
         tc_fence_after_sync();
-        const uint32_t v_addr = smem_u32(sV + st * kPfTile);
-#pragma unroll
-        for (int k = 0; k < kPfBN / 16; ++k)
+        for (int k = 0; k < keys / 16; ++k)
           mma_ts(tmem + kColO, tmem + kColP + k * 8, desc_mnmajor_sw128(v_addr + k * 2048, kPfPanel), idesc_pv,
                  (i | k) != 0);
-        mma_commit(&v_empty[st]);
+        mma_commit(v_empty);
         mma_commit(pv_done);
+        // P lives in the columns the next Q K^T overwrites, and the softmax threads
+        // rescale O between tiles: let this P V finish first
+        if (i + 1 < n_kv && !mbar_wait(pv_done, ph)) { ok = false; break; }
       }
     }
   } else {
@@ -179,27 +170,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     bool ok = true;
 
     for (int i = 0; i < n_kv && ok; ++i) {
-      const int st = i & 1;
-      ok = mbar_wait(&s_full[st], (i >> 1) & 1);
+      const uint32_t ph = i & 1;
+      ok = mbar_wait(s_full, ph);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t tS = tm_lane + kColS + st * 128;
       const int nvalid = min(max(bound - i * kPfBN, 0), kPfBN);
       const bool full = nvalid >= kPfBN;
 
-      // pass 1: row maximum over the visible columns
+      uint32_t r[128];
+      tmem_ld_x128_sync(tm_lane + kColS, r);
       float tmax = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld_x32_sync(tS + c * 32, r);
-        if (full) {
+      if (full) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(r[e]));
-        } else {
+        for (int e = 0; e < 128; ++e) tmax = fmaxf(tmax, __uint_as_float(r[e]));
+      } else {
 #pragma unroll
-          for (int e = 0; e < 32; ++e)
-            tmax = fmaxf(tmax, (c * 32 + e < nvalid) ? __uint_as_float(r[e]) : -INFINITY);
+        for (int e = 0; e < 128; ++e) {
+          if (e >= nvalid) r[e] = 0xff800000u;        // -inf: weight 0 below
+          tmax = fmaxf(tmax, __uint_as_float(r[e]));
         }
       }
       tmax *= a.scale_log2;                           // scale > 0: max commutes; -inf stays -inf
@@ -210,41 +198,31 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const float alpha = fast_exp2(m - m_new);
       l *= alpha;
 
-      // P buffer free and O stable once the previous P V has completed
-      if (i > 0) {
-        ok = mbar_wait(pv_done, (i - 1) & 1);
-        if (!ok) break;
-        tc_fence_after_sync();
-        if (rescale) {
+      // O is stable here: the previous P V completed before this tile's Q K^T was issued
+      if (rescale) {
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            uint32_t r[32];
-            tmem_ld_x32_sync(tm_lane + kColO + c * 32, r);
+        for (int c = 0; c < 4; ++c) {
+          uint32_t o[32];
+          tmem_ld_x32_sync(tm_lane + kColO + c * 32, o);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-            tmem_st_x32(tm_lane + kColO + c * 32, r);
-          }
+          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+          tmem_st_x32(tm_lane + kColO + c * 32, o);
         }
       }
 
-      // pass 2: p = 2^(s - m), written to TMEM as bf16 pairs
+      // p = 2^(s - m) as bf16 pairs, written over the columns S occupied
       float rowsum = 0.f;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32], pk[16];
-        tmem_ld_x32_sync(tS + c * 32, r);
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(r[e]), a.scale_log2, -m_new));
-          float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, -m_new));
-          if (!full) {
-            p0 = (c * 32 + e < nvalid) ? p0 : 0.f;
-            p1 = (c * 32 + e + 1 < nvalid) ? p1 : 0.f;
-          }
+      for (int c = 0; c < 8; ++c) {
+        uint32_t pk[8];
+#pragma unroll
+        for (int e = 0; e < 16; e += 2) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e]), a.scale_log2, -m_new));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e + 1]), a.scale_log2, -m_new));
           rowsum += p0 + p1;
           pk[e >> 1] = pack_bf16x2(p0, p1);
         }
-        tmem_st_x16(tm_lane + kColP + c * 16, pk);
+        tmem_st_x8(tm_lane + kColP + c * 8, pk);
       }
       l += rowsum;
       m = m_new;
@@ -253,11 +231,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       // holds (possibly NaN bit patterns): their weight is 0, but 0 * NaN is NaN
       // in the tensor core, so zero them in shared memory before P V reads them.
       if ((i + 1) * kPfBN > L) {
-        ok = mbar_wait(&v_full[st], (i >> 1) & 1);
+        ok = mbar_wait(v_full, ph);
         if (!ok) break;
         if (i * kPfBN + row >= L) {
           uint4 z = make_uint4(0, 0, 0, 0);
-          uint8_t *v0 = sV + st * kPfTile + row * 128;
+          uint8_t *v0 = sV + row * 128;
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             *reinterpret_cast<uint4 *>(v0 + c * 16) = z;
