@@ -16,7 +16,8 @@
 //
 // TMEM columns: S [0,128), overwritten in place by P [0,64) (bf16 pairs); O [128,256).
 // The self term seeds the running softmax (m = s_jj, l = 1) and its value row
-// is added in the epilogue: O_j = (sum_r p_r v_r + w_self v_j) / l.
+// is added in the epilogue: O_j = (sum_r p_r v_r + w_self v_j) / l.  Every byte
+// that enters or leaves the CTA travels by TMA.
 #include "ag_common.cuh"
 #include "umma.cuh"
 
@@ -33,8 +34,6 @@ constexpr uint32_t kColS = 0, kColP = 0, kColO = 128, kTmemCols = 256;
 constexpr float kRescaleThreshold = 8.f;              // log2 units
 
 struct PrefillTcArgs {
-  const __nv_bfloat16 *Q, *K, *V;   // dense [slabs, n, 128]
-  __nv_bfloat16 *O;
   const int32_t *prefix;            // [slabs, n + 1]
   const int64_t *row_off;
   const int32_t *len;
@@ -42,12 +41,25 @@ struct PrefillTcArgs {
   float scale_log2;
 };
 
+// Byte offset of 16-byte chunk `chunk` (0..15) of row `row` inside a [128 x 128] bf16 tile stored
+// as two 128-byte-swizzled panels of 64 columns (the layout TMA writes and tcgen05.mma reads).
+__device__ __forceinline__ uint32_t tile_chunk_offset(int row, int chunk) {
+  return (uint32_t)((chunk >> 3) * kPfPanel + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
+
 // Two CTAs share an SM (256 TMEM columns, 97 KB of shared memory each): inside a
 // CTA the chain S = Q K^T -> softmax -> O += P V is serial, and the tensor core
 // works on one CTA's tile while the other CTA is in its softmax.
+//
+// MMA tile 0 is the "self tile": S = Q_tile Kdense_tile^T, of which only the
+// diagonal (q_j . k_j) is read.  Tiles 1..n_kv run over the compacted cache.
+// Last, the dense V tile is brought in for the self term of the output, and
+// the O tile leaves through shared memory with one TMA store.
 __global__ void __launch_bounds__(kPfThreads, 2)
-prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                  const __grid_constant__ CUtensorMap tmV, const PrefillTcArgs a) {
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKd,
+                  const __grid_constant__ CUtensorMap tmVd, const __grid_constant__ CUtensorMap tmO,
+                  const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                  const PrefillTcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sQ = smem;
@@ -67,6 +79,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int32_t *pre = a.prefix + (size_t)slab * (a.n + 1);
   const int max_bound = pre[j_last];               // keys any row of this tile may see
   const int n_kv = (max_bound + kPfBN - 1) / kPfBN;
+  const int n_self = n_kv > 0 ? 1 : 0;             // a lone diagonal needs no score
   const int row0 = (int)a.row_off[slab];
 
   if (threadIdx.x == 0) {
@@ -77,7 +90,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     mbar_init(p_ready, 128);
     mbar_init(pv_done, 1);
     fence_barrier_init();
-    prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
+    prefetch_tensormap(&tmQ); prefetch_tensormap(&tmKd); prefetch_tensormap(&tmVd);
+    prefetch_tensormap(&tmK); prefetch_tensormap(&tmV); prefetch_tensormap(&tmO);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, kTmemCols);
@@ -90,35 +104,51 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0 && n_kv > 0) {
-      mbar_arrive_expect_tx(q_full, kPfTile);
-      tma_load_3d(sQ, &tmQ, q_full, 0, j0, slab);
-      tma_load_3d(sQ + kPfPanel, &tmQ, q_full, 64, j0, slab);
-      for (int i = 0; i < n_kv; ++i) {
-        const uint32_t ph = i & 1;
-        const int y = row0 + i * kPfBN;
-        if (!mbar_wait(k_empty, ph ^ 1)) break;
+    if (lane == 0) {
+      bool ok = true;
+      if (n_kv > 0) {
+        mbar_arrive_expect_tx(q_full, kPfTile);
+        tma_load_3d(sQ, &tmQ, q_full, 0, j0, slab);
+        tma_load_3d(sQ + kPfPanel, &tmQ, q_full, 64, j0, slab);
+        // self tile: dense K rows j0 .. j0 + 127 (k_empty is fresh: no wait)
         mbar_arrive_expect_tx(k_full, kPfTile);
-        tma_load_2d(sK, &tmK, k_full, 0, y);
-        tma_load_2d(sK + kPfPanel, &tmK, k_full, 64, y);
-        if (!mbar_wait(v_empty, ph ^ 1)) break;
-        mbar_arrive_expect_tx(v_full, kPfTile);
-        tma_load_2d(sV, &tmV, v_full, 0, y);
-        tma_load_2d(sV + kPfPanel, &tmV, v_full, 64, y);
+        tma_load_3d(sK, &tmKd, k_full, 0, j0, slab);
+        tma_load_3d(sK + kPfPanel, &tmKd, k_full, 64, j0, slab);
+        for (int i = 0; i < n_kv && ok; ++i) {
+          const int t = i + 1;
+          const int y = row0 + i * kPfBN;
+          ok = mbar_wait(k_empty, (t & 1) ^ 1);
+          if (!ok) break;
+          mbar_arrive_expect_tx(k_full, kPfTile);
+          tma_load_2d(sK, &tmK, k_full, 0, y);
+          tma_load_2d(sK + kPfPanel, &tmK, k_full, 64, y);
+          ok = mbar_wait(v_empty, (i & 1) ^ 1);
+          if (!ok) break;
+          mbar_arrive_expect_tx(v_full, kPfTile);
+          tma_load_2d(sV, &tmV, v_full, 0, y);
+          tma_load_2d(sV + kPfPanel, &tmV, v_full, 64, y);
+        }
+      }
+      // dense V rows for the self term of the output, into the K buffer once it is free
+      const int t_last = n_kv + n_self;
+      if (ok && (t_last == 0 || mbar_wait(k_empty, (t_last & 1) ^ 1))) {
+        mbar_arrive_expect_tx(k_full, kPfTile);
+        tma_load_3d(sK, &tmVd, k_full, 0, j0, slab);
+        tma_load_3d(sK + kPfPanel, &tmVd, k_full, 64, j0, slab);
       }
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0 && n_kv > 0) {
       const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+      constexpr uint32_t idesc_pv = idesc_bf16_f32(kPfBM, kPfD, false, true);
       bool ok = mbar_wait(q_full, 0);
-      for (int i = 0; i < n_kv && ok; ++i) {
-        const uint32_t ph = i & 1;
+      for (int t = 0; t <= n_kv && ok; ++t) {
+        const int i = t - 1;                         // cache tile index; -1 = self tile
         // keys of this tile any row can see, rounded up to the MMA's N / K granularity
-        const int keys = min(kPfBN, (max_bound - i * kPfBN + 15) & ~15);
+        const int keys = t == 0 ? kPfBN : min(kPfBN, (max_bound - i * kPfBN + 15) & ~15);
         const uint32_t idesc_qk = idesc_bf16_f32(kPfBM, keys, false, false);
-        constexpr uint32_t idesc_pv = idesc_bf16_f32(kPfBM, kPfD, false, true);
-        if (!mbar_wait(k_full, ph)) { ok = false; break; }
+        if (!mbar_wait(k_full, t & 1)) { ok = false; break; }
         tc_fence_after_sync();
 #pragma unroll
         for (int k = 0; k < kPfD / 16; ++k) {
@@ -127,8 +157,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         mma_commit(k_empty);
         mma_commit(s_full);
-        if (!mbar_wait(p_ready, ph)) { ok = false; break; }
-        if (!mbar_wait(v_full, ph)) { ok = false; break; }
+        if (!mbar_wait(p_ready, t & 1)) { ok = false; break; }
+        if (t == 0) continue;                        // the self tile has no P V
+        if (!mbar_wait(v_full, i & 1)) { ok = false; break; }
         tc_fence_after_sync();
         for (int k = 0; k < keys / 16; ++k)
           mma_ts(tmem + kColO, tmem + kColP + k * 8, desc_mnmajor_sw128(v_addr + k * 2048, kPfPanel), idesc_pv,
@@ -137,7 +168,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mma_commit(pv_done);
         // P lives in the columns the next Q K^T overwrites, and the softmax threads
         // rescale O between tiles: let this P V finish first
-        if (i + 1 < n_kv && !mbar_wait(pv_done, ph)) { ok = false; break; }
+        if (i + 1 < n_kv && !mbar_wait(pv_done, i & 1)) { ok = false; break; }
       }
     }
   } else {
@@ -146,32 +177,30 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int row = quad * 32 + lane;
     const int j = j0 + row;
     const bool valid = j < a.n;
-    const int jc = min(j, a.n - 1);
-    const int bound = valid ? pre[jc] : 0;
+    const int bound = valid ? pre[j] : 0;
     const int L = a.len[slab];
     const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
-    const size_t row_elem = ((size_t)slab * a.n + jc) * kPfD;
-
-    // self term: q_j . k_j
-    float s_self = 0.f;
-    {
-      const __nv_bfloat16 *qp = a.Q + row_elem, *kp = a.K + row_elem;
-#pragma unroll 4
-      for (int c = 0; c < kPfD / 8; ++c) {
-        float qf[8], kf[8];
-        Elem<__nv_bfloat16>::unpack(ldg128(qp + c * 8), qf);
-        Elem<__nv_bfloat16>::unpack(ldg128(kp + c * 8), kf);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) s_self = fmaf(qf[e], kf[e], s_self);
-      }
-    }
-    const float self2 = s_self * a.scale_log2;
-    float m = self2, l = 1.f;
+    float m = 0.f, self2 = 0.f, l = 1.f;
     bool ok = true;
 
+    if (n_kv > 0) {
+      // self tile: this thread's diagonal element S[row][row] = q_j . k_j
+      ok = mbar_wait(s_full, 0);
+      tc_fence_after_sync();
+      uint32_t d[32];
+      tmem_ld_x32_sync(tm_lane + kColS + quad * 32, d);
+      float s_self = 0.f;
+#pragma unroll
+      for (int e = 0; e < 32; ++e) s_self = (e == lane) ? __uint_as_float(d[e]) : s_self;
+      self2 = s_self * a.scale_log2;
+      m = self2;
+      tc_fence_before_sync();
+      mbar_arrive(p_ready);
+    }
+
     for (int i = 0; i < n_kv && ok; ++i) {
-      const uint32_t ph = i & 1;
-      ok = mbar_wait(s_full, ph);
+      const int t = i + 1;
+      ok = mbar_wait(s_full, t & 1);
       if (!ok) break;
       tc_fence_after_sync();
       const int nvalid = min(max(bound - i * kPfBN, 0), kPfBN);
@@ -179,17 +208,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
       uint32_t r[128];
       tmem_ld_x128_sync(tm_lane + kColS, r);
-      float tmax = -INFINITY;
-      if (full) {
+      if (!full) {
 #pragma unroll
-        for (int e = 0; e < 128; ++e) tmax = fmaxf(tmax, __uint_as_float(r[e]));
-      } else {
-#pragma unroll
-        for (int e = 0; e < 128; ++e) {
+        for (int e = 0; e < 128; ++e)
           if (e >= nvalid) r[e] = 0xff800000u;        // -inf: weight 0 below
-          tmax = fmaxf(tmax, __uint_as_float(r[e]));
-        }
       }
+      // eight independent chains instead of one 128-long dependency
+      float mx[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) mx[q] = __uint_as_float(r[q]);
+#pragma unroll
+      for (int e = 8; e < 128; e += 8)
+#pragma unroll
+        for (int q = 0; q < 8; ++q) mx[q] = fmaxf(mx[q], __uint_as_float(r[e + q]));
+      float tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
       tmax *= a.scale_log2;                           // scale > 0: max commutes; -inf stays -inf
       float m_new;
       if (i == 0) m_new = fmaxf(m, tmax);
@@ -211,7 +244,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       }
 
       // p = 2^(s - m) as bf16 pairs, written over the columns S occupied
-      float rowsum = 0.f;
+      float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         uint32_t pk[8];
@@ -219,11 +252,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int e = 0; e < 16; e += 2) {
           const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e]), a.scale_log2, -m_new));
           const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e + 1]), a.scale_log2, -m_new));
-          rowsum += p0 + p1;
+          rs[(e >> 1) & 3] += p0 + p1;
           pk[e >> 1] = pack_bf16x2(p0, p1);
         }
         tmem_st_x8(tm_lane + kColP + c * 8, pk);
       }
+      const float rowsum = (rs[0] + rs[1]) + (rs[2] + rs[3]);
       l += rowsum;
       m = m_new;
 
@@ -231,7 +265,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       // holds (possibly NaN bit patterns): their weight is 0, but 0 * NaN is NaN
       // in the tensor core, so zero them in shared memory before P V reads them.
       if ((i + 1) * kPfBN > L) {
-        ok = mbar_wait(v_full, ph);
+        ok = mbar_wait(v_full, i & 1);
         if (!ok) break;
         if (i * kPfBN + row >= L) {
           uint4 z = make_uint4(0, 0, 0, 0);
@@ -249,16 +283,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       mbar_arrive(p_ready);
     }
 
-    // epilogue
+    // epilogue: O_j = (sum_r p_r v_r + w_self v_j) / l, staged in the V buffer, one TMA store
     if (ok && n_kv > 0) {
       ok = mbar_wait(pv_done, (n_kv - 1) & 1);
       tc_fence_after_sync();
     }
+    if (ok) ok = mbar_wait(k_full, (n_kv + n_self) & 1);      // dense V tile has landed in sK
     if (ok) {
       const float w_self = fast_exp2(self2 - m);
       const float inv = 1.f / l;
-      const __nv_bfloat16 *vp = a.V + row_elem;
-      __nv_bfloat16 *op = a.O + row_elem;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         uint32_t r[32];
@@ -268,22 +301,29 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
           for (int e = 0; e < 32; ++e) r[e] = 0u;
         }
-        if (valid) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            float vf[8];
-            Elem<__nv_bfloat16>::unpack(ldg128(vp + c * 32 + g * 8), vf);
-            uint32_t o[4];
+        for (int g = 0; g < 4; ++g) {
+          const uint32_t off = tile_chunk_offset(row, c * 4 + g);
+          float vf[8];
+          Elem<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4 *>(sK + off), vf);
+          uint32_t o[4];
 #pragma unroll
-            for (int e = 0; e < 8; e += 2) {
-              const float x0 = fmaf(w_self, vf[e], __uint_as_float(r[g * 8 + e])) * inv;
-              const float x1 = fmaf(w_self, vf[e + 1], __uint_as_float(r[g * 8 + e + 1])) * inv;
-              o[e >> 1] = pack_bf16x2(x0, x1);
-            }
-            *reinterpret_cast<uint4 *>(op + c * 32 + g * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+          for (int e = 0; e < 8; e += 2) {
+            const float x0 = fmaf(w_self, vf[e], __uint_as_float(r[g * 8 + e])) * inv;
+            const float x1 = fmaf(w_self, vf[e + 1], __uint_as_float(r[g * 8 + e + 1])) * inv;
+            o[e >> 1] = pack_bf16x2(x0, x1);
           }
+          *reinterpret_cast<uint4 *>(sV + off) = make_uint4(o[0], o[1], o[2], o[3]);
         }
       }
+      fence_proxy_async_smem();
+    }
+    named_barrier_sync(1, 128);
+    if (ok && threadIdx.x == 64) {
+      tma_store_3d(&tmO, sV, 0, j0, slab);           // rows past n are dropped by the tensor map
+      tma_store_3d(&tmO, sV + kPfPanel, 64, j0, slab);
+      tma_store_commit();
+      tma_store_wait_read();
     }
   }
   tc_fence_before_sync();
@@ -299,9 +339,12 @@ bool prefill_tc_supported(const ag_layer_desc &d, const ag_cache &c) {
 int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, const void *V, const ag_cache &c,
                       const int32_t *prefix, float scale, void *O, cudaStream_t st) {
   const int slabs = d.batch * d.heads;
-  CUtensorMap tmQ, tmK, tmV;
-  int rc = make_tmap_3d_bf16(&tmQ, Q, slabs, d.seq, kPfD, kPfBM, 64);
-  if (rc) return rc;
+  CUtensorMap tmQ, tmKd, tmVd, tmO, tmK, tmV;
+  int rc;
+  if ((rc = make_tmap_3d_bf16(&tmQ, Q, slabs, d.seq, kPfD, kPfBM, 64))) return rc;
+  if ((rc = make_tmap_3d_bf16(&tmKd, K, slabs, d.seq, kPfD, kPfBM, 64))) return rc;
+  if ((rc = make_tmap_3d_bf16(&tmVd, V, slabs, d.seq, kPfD, kPfBM, 64))) return rc;
+  if ((rc = make_tmap_3d_bf16(&tmO, O, slabs, d.seq, kPfD, kPfBM, 64))) return rc;
   // an empty pool still needs a valid map: describe one row of the dense K / V instead (never read)
   const bool empty = c.pool_rows == 0;
   rc = make_tmap_2d_bf16(&tmK, empty ? K : c.k_rows, empty ? 1 : (uint64_t)c.pool_rows, kPfD, kPfD * 2, kPfBN, 64);
@@ -309,15 +352,11 @@ int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, cons
   rc = make_tmap_2d_bf16(&tmV, empty ? V : c.v_rows, empty ? 1 : (uint64_t)c.pool_rows, kPfD, kPfD * 2, kPfBN, 64);
   if (rc) return rc;
   PrefillTcArgs a;
-  a.Q = static_cast<const __nv_bfloat16 *>(Q);
-  a.K = static_cast<const __nv_bfloat16 *>(K);
-  a.V = static_cast<const __nv_bfloat16 *>(V);
-  a.O = static_cast<__nv_bfloat16 *>(O);
   a.prefix = prefix; a.row_off = c.row_off; a.len = c.len;
   a.n = d.seq; a.n_qtiles = (d.seq + kPfBM - 1) / kPfBM; a.slabs = slabs;
   a.scale_log2 = scale * 1.4426950408889634f;
   AG_CUDA_TRY(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes));
-  prefill_tc_kernel<<<a.n_qtiles * slabs, kPfThreads, kPfSmemBytes, st>>>(tmQ, tmK, tmV, a);
+  prefill_tc_kernel<<<a.n_qtiles * slabs, kPfThreads, kPfSmemBytes, st>>>(tmQ, tmKd, tmVd, tmO, tmK, tmV, a);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }

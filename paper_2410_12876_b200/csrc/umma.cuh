@@ -59,17 +59,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait for the phase with the given parity to complete.  Once any wait
-// of this translation unit has expired, every later wait that would block gives
-// up at once, so that a stuck launch drains quickly instead of CTA by CTA.
+// Bounded wait for the phase with the given parity to complete.  The poll loop
+// touches nothing but the barrier; the clock and the give-up flag are looked at
+// once every 1024 polls.  Once any wait of this translation unit has expired,
+// every later wait that blocks that long gives up too, so that a stuck launch
+// drains quickly instead of CTA by CTA.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
+  uint32_t polls = 0;
+  long long t0 = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if (*reinterpret_cast<volatile int *>(&g_wait_expired) != 0) return false;
-    if (clock64() - t0 > kWaitCycles) {
-      atomicAdd(&g_wait_expired, 1);
-      return false;
+    if ((++polls & 1023u) == 0) {
+      if (*reinterpret_cast<volatile int *>(&g_wait_expired) != 0) return false;
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitCycles) {
+        atomicAdd(&g_wait_expired, 1);
+        return false;
+      }
     }
   }
   return true;
@@ -96,6 +103,20 @@ __device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *m
       "cp.async.bulk.tensor.3d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(smem_dst)), "l"(m), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
       : "memory");
+}
+
+// Tile store shared -> global (bulk async group); rows / planes outside the tensor are dropped.
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *m, const void *smem_src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(m), "r"(smem_u32(smem_src)), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Wait until the committed stores have finished READING shared memory.
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// Barrier among a subset of the CTA's warps (id 1..15, count a multiple of 32).
+__device__ __forceinline__ void named_barrier_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
 // ----------------------------------------------------------------- TMEM
