@@ -7,14 +7,14 @@
 // the compacted rows the mask is a staircase, so only the tiles that touch it
 // need per-element masking and evicted keys are never loaded.
 //
-//   warp 0      TMA: Q tile once, then K / V tiles of 128 cache rows
+//   warp 0      TMA: Q tile once, then K / V tiles of 64 cache rows (2 stages)
 //   warp 1      owns tensor memory, issues S = Q K^T (tcgen05.mma, operands in
 //               shared memory) and O += P V (P read from tensor memory)
 //   warps 2..5  one query row per thread: online softmax on S read from TMEM,
 //               P written back to TMEM as bf16, O rescaled only when the running
 //               maximum grows by more than 2^8, final normalisation and store
 //
-// TMEM columns: S [0,128), overwritten in place by P [0,64) (bf16 pairs); O [128,256).
+// TMEM columns: S0 [0,64) S1 [64,128), each overwritten in place by its P (bf16 pairs); O [128,256).
 // The self term seeds the running softmax (m = s_jj, l = 1) and its value row
 // is added in the epilogue: O_j = (sum_r p_r v_r + w_self v_j) / l.  Every byte
 // that enters or leaves the CTA travels by TMA.
@@ -26,11 +26,13 @@ namespace ag {
 using namespace umma;
 
 constexpr int kPfThreads = 192;
-constexpr int kPfBM = 128, kPfBN = 128, kPfD = 128;
-constexpr int kPfPanel = 128 * 128;                   // [128 rows][64 bf16] = 16 KB
+constexpr int kPfBM = 128, kPfBN = 64, kPfD = 128;
+constexpr int kPfPanel = 128 * 128;                   // [128 rows][64 bf16] = 16 KB (Q, dense K / V, O)
 constexpr int kPfTile = 2 * kPfPanel;                 // 32 KB
+constexpr int kPfKvPanel = kPfBN * 128;               // [64 rows][64 bf16] = 8 KB (cache tiles)
+constexpr int kPfKvTile = 2 * kPfKvPanel;             // 16 KB; two stages fill one 32 KB buffer
 constexpr int kPfSmemBytes = 3 * kPfTile + 1024 + 256;
-constexpr uint32_t kColS = 0, kColP = 0, kColO = 128, kTmemCols = 256;
+constexpr uint32_t kColS = 0, kColO = 128, kTmemCols = 256;   // S0 [0,64) S1 [64,128), P in place
 constexpr float kRescaleThreshold = 8.f;              // log2 units
 
 struct PrefillTcArgs {
@@ -47,14 +49,16 @@ __device__ __forceinline__ uint32_t tile_chunk_offset(int row, int chunk) {
   return (uint32_t)((chunk >> 3) * kPfPanel + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
-// Two CTAs share an SM (256 TMEM columns, 97 KB of shared memory each): inside a
-// CTA the chain S = Q K^T -> softmax -> O += P V is serial, and the tensor core
-// works on one CTA's tile while the other CTA is in its softmax.
+// Two CTAs share an SM (256 TMEM columns, 97 KB of shared memory each).  Keys
+// are visited in tiles of 64 with S double-buffered, so S = Q K^T of tile i + 1
+// runs while the softmax threads work on tile i and O += P V of tile i runs
+// while they work on tile i + 1: the softmax threads never wait for the tensor
+// core in steady state, and the tensor core interleaves the two CTAs.
 //
-// MMA tile 0 is the "self tile": S = Q_tile Kdense_tile^T, of which only the
-// diagonal (q_j . k_j) is read.  Tiles 1..n_kv run over the compacted cache.
-// Last, the dense V tile is brought in for the self term of the output, and
-// the O tile leaves through shared memory with one TMA store.
+// The first MMA tile is the "self tile": S = Q_tile Kdense_tile^T over the
+// CTA's own 128 rows, of which only the diagonal (q_j . k_j) is read.  Last,
+// the dense V tile is brought in for the self term of the output, and the O
+// tile leaves through shared memory with one TMA store.
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKd,
                   const __grid_constant__ CUtensorMap tmVd, const __grid_constant__ CUtensorMap tmO,
@@ -63,12 +67,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sQ = smem;
-  uint8_t *sK = sQ + kPfTile;
+  uint8_t *sK = sQ + kPfTile;                      // two 16 KB stages, or one 128-row dense tile
   uint8_t *sV = sK + kPfTile;
   uint64_t *bars = reinterpret_cast<uint64_t *>(sV + kPfTile);
-  uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 2, *v_full = bars + 3, *v_empty = bars + 4;
-  uint64_t *s_full = bars + 5, *p_ready = bars + 6, *pv_done = bars + 7;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 8);
+  uint64_t *q_full = bars;
+  uint64_t *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;   // [2] each
+  uint64_t *s_full = bars + 9;                     // [2]
+  uint64_t *p_ready = bars + 11, *pv_done = bars + 12;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 13);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // heaviest query tiles first
@@ -81,12 +87,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int n_kv = (max_bound + kPfBN - 1) / kPfBN;
   const int n_self = n_kv > 0 ? 1 : 0;             // a lone diagonal needs no score
   const int row0 = (int)a.row_off[slab];
+  // completions of k_full[0] / s_full[0] before the dense V tile: self tile + even cache tiles
+  const int k0_uses = n_self + (n_kv + 1) / 2, k1_uses = n_self + n_kv / 2;
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    mbar_init(k_full, 1); mbar_init(k_empty, 1);
-    mbar_init(v_full, 1); mbar_init(v_empty, 1);
-    mbar_init(s_full, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
+      mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
+      mbar_init(&s_full[s], 1);
+    }
     mbar_init(p_ready, 128);
     mbar_init(pv_done, 1);
     fence_barrier_init();
@@ -110,31 +120,33 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mbar_arrive_expect_tx(q_full, kPfTile);
         tma_load_3d(sQ, &tmQ, q_full, 0, j0, slab);
         tma_load_3d(sQ + kPfPanel, &tmQ, q_full, 64, j0, slab);
-        // self tile: dense K rows j0 .. j0 + 127 (k_empty is fresh: no wait)
-        mbar_arrive_expect_tx(k_full, kPfTile);
-        tma_load_3d(sK, &tmKd, k_full, 0, j0, slab);
-        tma_load_3d(sK + kPfPanel, &tmKd, k_full, 64, j0, slab);
+        // self tile: dense K rows j0 .. j0 + 127 across both K stages (fresh: no wait)
+        mbar_arrive_expect_tx(&k_full[0], kPfTile);
+        tma_load_3d(sK, &tmKd, &k_full[0], 0, j0, slab);
+        tma_load_3d(sK + kPfPanel, &tmKd, &k_full[0], 64, j0, slab);
         for (int i = 0; i < n_kv && ok; ++i) {
-          const int t = i + 1;
+          const int st = i & 1;
           const int y = row0 + i * kPfBN;
-          ok = mbar_wait(k_empty, (t & 1) ^ 1);
+          // the self tile was use 0 of both K stages; V stages start fresh
+          ok = mbar_wait(&k_empty[st], (((i >> 1) + 1) & 1) ^ 1);
           if (!ok) break;
-          mbar_arrive_expect_tx(k_full, kPfTile);
-          tma_load_2d(sK, &tmK, k_full, 0, y);
-          tma_load_2d(sK + kPfPanel, &tmK, k_full, 64, y);
-          ok = mbar_wait(v_empty, (i & 1) ^ 1);
+          mbar_arrive_expect_tx(&k_full[st], kPfKvTile);
+          tma_load_2d(sK + st * kPfKvTile, &tmK, &k_full[st], 0, y);
+          tma_load_2d(sK + st * kPfKvTile + kPfKvPanel, &tmK, &k_full[st], 64, y);
+          ok = mbar_wait(&v_empty[st], ((i >> 1) & 1) ^ 1);
           if (!ok) break;
-          mbar_arrive_expect_tx(v_full, kPfTile);
-          tma_load_2d(sV, &tmV, v_full, 0, y);
-          tma_load_2d(sV + kPfPanel, &tmV, v_full, 64, y);
+          mbar_arrive_expect_tx(&v_full[st], kPfKvTile);
+          tma_load_2d(sV + st * kPfKvTile, &tmV, &v_full[st], 0, y);
+          tma_load_2d(sV + st * kPfKvTile + kPfKvPanel, &tmV, &v_full[st], 64, y);
         }
       }
-      // dense V rows for the self term of the output, into the K buffer once it is free
-      const int t_last = n_kv + n_self;
-      if (ok && (t_last == 0 || mbar_wait(k_empty, (t_last & 1) ^ 1))) {
-        mbar_arrive_expect_tx(k_full, kPfTile);
-        tma_load_3d(sK, &tmVd, k_full, 0, j0, slab);
-        tma_load_3d(sK + kPfPanel, &tmVd, k_full, 64, j0, slab);
+      // dense V rows for the self term of the output, into the K buffer once both stages are free
+      if (ok && k0_uses > 0) ok = mbar_wait(&k_empty[0], (k0_uses & 1) ^ 1);
+      if (ok && k1_uses > 0) ok = mbar_wait(&k_empty[1], (k1_uses & 1) ^ 1);
+      if (ok) {
+        mbar_arrive_expect_tx(&k_full[0], kPfTile);
+        tma_load_3d(sK, &tmVd, &k_full[0], 0, j0, slab);
+        tma_load_3d(sK + kPfPanel, &tmVd, &k_full[0], 64, j0, slab);
       }
     }
   } else if (warp == 1) {
@@ -142,39 +154,63 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (lane == 0 && n_kv > 0) {
       const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kPfBM, kPfD, false, true);
-      bool ok = mbar_wait(q_full, 0);
-      for (int t = 0; t <= n_kv && ok; ++t) {
-        const int i = t - 1;                         // cache tile index; -1 = self tile
-        // keys of this tile any row can see, rounded up to the MMA's N / K granularity
-        const int keys = t == 0 ? kPfBN : min(kPfBN, (max_bound - i * kPfBN + 15) & ~15);
-        const uint32_t idesc_qk = idesc_bf16_f32(kPfBM, keys, false, false);
-        if (!mbar_wait(k_full, t & 1)) { ok = false; break; }
+      // keys of cache tile i any row can see, rounded up to the MMA's N / K granularity
+      auto tile_keys = [&](int i) { return min(kPfBN, (max_bound - i * kPfBN + 15) & ~15); };
+      auto issue_qk = [&](int i) -> bool {
+        const int st = i & 1;
+        if (!mbar_wait(&k_full[st], ((i >> 1) + (st == 0 ? 1 : 0)) & 1)) return false;
         tc_fence_after_sync();
+        const uint32_t idesc_qk = idesc_bf16_f32(kPfBM, tile_keys(i), false, false);
+        const uint32_t kb = k_addr + st * kPfKvTile;
+#pragma unroll
+        for (int k = 0; k < kPfD / 16; ++k)
+          mma_ss(tmem + kColS + st * kPfBN, desc_kmajor_sw128(q_addr + (k >> 2) * kPfPanel + (k & 3) * 32),
+                 desc_kmajor_sw128(kb + (k >> 2) * kPfKvPanel + (k & 3) * 32), idesc_qk, k != 0);
+        mma_commit(&k_empty[st]);
+        mma_commit(&s_full[st]);
+        return true;
+      };
+      bool ok = mbar_wait(q_full, 0);
+      // self tile: 128 dense K rows, S over both buffers
+      ok = ok && mbar_wait(&k_full[0], 0);
+      if (ok) {
+        tc_fence_after_sync();
+        constexpr uint32_t idesc_self = idesc_bf16_f32(kPfBM, 128, false, false);
 #pragma unroll
         for (int k = 0; k < kPfD / 16; ++k) {
           const uint32_t off = (k >> 2) * kPfPanel + (k & 3) * 32;
-          mma_ss(tmem + kColS, desc_kmajor_sw128(q_addr + off), desc_kmajor_sw128(k_addr + off), idesc_qk, k != 0);
+          mma_ss(tmem + kColS, desc_kmajor_sw128(q_addr + off), desc_kmajor_sw128(k_addr + off), idesc_self, k != 0);
         }
-        mma_commit(k_empty);
-        mma_commit(s_full);
-        if (!mbar_wait(p_ready, t & 1)) { ok = false; break; }
-        if (t == 0) continue;                        // the self tile has no P V
-        if (!mbar_wait(v_full, i & 1)) { ok = false; break; }
+        mma_commit(&k_empty[0]);
+        mma_commit(&k_empty[1]);
+        mma_commit(&s_full[0]);
+        ok = mbar_wait(p_ready, 0);                  // diagonal extracted: S may be overwritten
+      }
+      ok = ok && issue_qk(0);
+      for (int i = 0; i < n_kv && ok; ++i) {
+        if (i + 1 < n_kv) {
+          // S[(i+1)&1] still holds P of tile i - 1 until that P V has completed
+          if (i >= 1 && !mbar_wait(pv_done, (i - 1) & 1)) { ok = false; break; }
+          if (!issue_qk(i + 1)) { ok = false; break; }
+        }
+        const int st = i & 1;
+        if (!mbar_wait(p_ready, (i + 1) & 1)) { ok = false; break; }
+        if (!mbar_wait(&v_full[st], (i >> 1) & 1)) { ok = false; break; }
         tc_fence_after_sync();
-        for (int k = 0; k < keys / 16; ++k)
-          mma_ts(tmem + kColO, tmem + kColP + k * 8, desc_mnmajor_sw128(v_addr + k * 2048, kPfPanel), idesc_pv,
-                 (i | k) != 0);
-        mma_commit(v_empty);
+        const int ksteps = tile_keys(i) / 16;
+        const uint32_t vb = v_addr + st * kPfKvTile;
+        for (int k = 0; k < ksteps; ++k)
+          mma_ts(tmem + kColO, tmem + kColS + st * kPfBN + k * 8, desc_mnmajor_sw128(vb + k * 2048, kPfKvPanel),
+                 idesc_pv, (i | k) != 0);
+        mma_commit(&v_empty[st]);
         mma_commit(pv_done);
-        // P lives in the columns the next Q K^T overwrites, and the softmax threads
-        // rescale O between tiles: let this P V finish first
-        if (i + 1 < n_kv && !mbar_wait(pv_done, i & 1)) { ok = false; break; }
       }
     }
   } else {
     // ------------------------------------------- softmax / correction / epilogue
     const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
     const int row = quad * 32 + lane;
+    const int tid = threadIdx.x - 64;                // 0..127
     const int j = j0 + row;
     const bool valid = j < a.n;
     const int bound = valid ? pre[j] : 0;
@@ -185,7 +221,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
     if (n_kv > 0) {
       // self tile: this thread's diagonal element S[row][row] = q_j . k_j
-      ok = mbar_wait(s_full, 0);
+      ok = mbar_wait(&s_full[0], 0);
       tc_fence_after_sync();
       uint32_t d[32];
       tmem_ld_x32_sync(tm_lane + kColS + quad * 32, d);
@@ -199,26 +235,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
 
     for (int i = 0; i < n_kv && ok; ++i) {
-      const int t = i + 1;
-      ok = mbar_wait(s_full, t & 1);
+      const int st = i & 1;
+      ok = mbar_wait(&s_full[st], ((i >> 1) + (st == 0 ? 1 : 0)) & 1);
       if (!ok) break;
       tc_fence_after_sync();
       const int nvalid = min(max(bound - i * kPfBN, 0), kPfBN);
-      const bool full = nvalid >= kPfBN;
+      const uint32_t tS = tm_lane + kColS + st * kPfBN;
 
-      uint32_t r[128];
-      tmem_ld_x128_sync(tm_lane + kColS, r);
-      if (!full) {
+      uint32_t r[64];
+      tmem_ld_x64_sync(tS, r);
+      if (nvalid < kPfBN) {
 #pragma unroll
-        for (int e = 0; e < 128; ++e)
+        for (int e = 0; e < 64; ++e)
           if (e >= nvalid) r[e] = 0xff800000u;        // -inf: weight 0 below
       }
-      // eight independent chains instead of one 128-long dependency
+      // eight independent chains instead of one long dependency
       float mx[8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) mx[q] = __uint_as_float(r[q]);
 #pragma unroll
-      for (int e = 8; e < 128; e += 8)
+      for (int e = 8; e < 64; e += 8)
 #pragma unroll
         for (int q = 0; q < 8; ++q) mx[q] = fmaxf(mx[q], __uint_as_float(r[e + q]));
       float tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
@@ -229,24 +265,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       else m_new = (tmax > m + kRescaleThreshold) ? tmax : m;
       const bool rescale = (i > 0) && __any_sync(0xffffffffu, m_new != m);
       const float alpha = fast_exp2(m - m_new);
-      l *= alpha;
-
-      // O is stable here: the previous P V completed before this tile's Q K^T was issued
-      if (rescale) {
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t o[32];
-          tmem_ld_x32_sync(tm_lane + kColO + c * 32, o);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st_x32(tm_lane + kColO + c * 32, o);
-        }
-      }
 
       // p = 2^(s - m) as bf16 pairs, written over the columns S occupied
       float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
+      for (int c = 0; c < 4; ++c) {
         uint32_t pk[8];
 #pragma unroll
         for (int e = 0; e < 16; e += 2) {
@@ -255,26 +278,41 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           rs[(e >> 1) & 3] += p0 + p1;
           pk[e >> 1] = pack_bf16x2(p0, p1);
         }
-        tmem_st_x8(tm_lane + kColP + c * 8, pk);
+        tmem_st_x8(tS + c * 8, pk);
       }
-      const float rowsum = (rs[0] + rs[1]) + (rs[2] + rs[3]);
-      l += rowsum;
+      l = l * alpha + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
       m = m_new;
+
+      // The previous P V must be complete before O is rescaled; waiting for it on
+      // every tile also keeps this thread in step with the barrier's phases.
+      if (i > 0) {
+        ok = mbar_wait(pv_done, (i - 1) & 1);
+        if (!ok) break;
+        if (rescale) {
+          tc_fence_after_sync();
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld_x32_sync(tm_lane + kColO + c * 32, o);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st_x32(tm_lane + kColO + c * 32, o);
+          }
+        }
+      }
 
       // Rows of the V tile past the slab's valid length hold whatever the pool
       // holds (possibly NaN bit patterns): their weight is 0, but 0 * NaN is NaN
       // in the tensor core, so zero them in shared memory before P V reads them.
       if ((i + 1) * kPfBN > L) {
-        ok = mbar_wait(v_full, i & 1);
+        ok = mbar_wait(&v_full[st], (i >> 1) & 1);
         if (!ok) break;
-        if (i * kPfBN + row >= L) {
+        const int vr = tid >> 1;                      // two threads per row, one panel each
+        if (i * kPfBN + vr >= L) {
           uint4 z = make_uint4(0, 0, 0, 0);
-          uint8_t *v0 = sV + row * 128;
+          uint8_t *v0 = sV + st * kPfKvTile + (tid & 1) * kPfKvPanel + vr * 128;
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            *reinterpret_cast<uint4 *>(v0 + c * 16) = z;
-            *reinterpret_cast<uint4 *>(v0 + kPfPanel + c * 16) = z;
-          }
+          for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4 *>(v0 + c * 16) = z;
         }
         fence_proxy_async_smem();
       }
@@ -288,7 +326,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       ok = mbar_wait(pv_done, (n_kv - 1) & 1);
       tc_fence_after_sync();
     }
-    if (ok) ok = mbar_wait(k_full, (n_kv + n_self) & 1);      // dense V tile has landed in sK
+    if (ok) ok = mbar_wait(&k_full[0], k0_uses & 1);          // dense V tile has landed in sK
     if (ok) {
       const float w_self = fast_exp2(self2 - m);
       const float inv = 1.f / l;
