@@ -151,8 +151,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0 && n_kv > 0) {
-      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+    // Every lane runs the control flow so that operands stay warp-uniform (the tensor-core
+    // instructions take uniform registers); one elected lane issues.
+    if (n_kv > 0) {
+      // descriptors as (low, high) words: the high words are fixed per operand kind, the low
+      // words are a base plus a compile-time offset per K step
+      const uint64_t dq = desc_kmajor_sw128(smem_u32(sQ)), dk = desc_kmajor_sw128(smem_u32(sK));
+      const uint64_t dv = desc_mnmajor_sw128(smem_u32(sV), kPfKvPanel);
+      const uint32_t q_lo = (uint32_t)dq, q_hi = (uint32_t)(dq >> 32);
+      const uint32_t k_lo = (uint32_t)dk, k_hi = (uint32_t)(dk >> 32);
+      const uint32_t v_lo = (uint32_t)dv, v_hi = (uint32_t)(dv >> 32);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kPfBM, kPfD, false, true);
       // keys of cache tile i any row can see, rounded up to the MMA's N / K granularity
       auto tile_keys = [&](int i) { return min(kPfBN, (max_bound - i * kPfBN + 15) & ~15); };
@@ -161,13 +169,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (!mbar_wait(&k_full[st], ((i >> 1) + (st == 0 ? 1 : 0)) & 1)) return false;
         tc_fence_after_sync();
         const uint32_t idesc_qk = idesc_bf16_f32(kPfBM, tile_keys(i), false, false);
-        const uint32_t kb = k_addr + st * kPfKvTile;
+        const uint32_t kb = k_lo + ((st * kPfKvTile) >> 4);
+        const uint32_t d = tmem + kColS + st * kPfBN;
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < kPfD / 16; ++k)
-          mma_ss(tmem + kColS + st * kPfBN, desc_kmajor_sw128(q_addr + (k >> 2) * kPfPanel + (k & 3) * 32),
-                 desc_kmajor_sw128(kb + (k >> 2) * kPfKvPanel + (k & 3) * 32), idesc_qk, k != 0);
-        mma_commit(&k_empty[st]);
-        mma_commit(&s_full[st]);
+          for (int k = 0; k < kPfD / 16; ++k)
+            mma_ss_lohi(d, q_lo + (((k >> 2) * kPfPanel + (k & 3) * 32) >> 4), q_hi,
+                        kb + (((k >> 2) * kPfKvPanel + (k & 3) * 32) >> 4), k_hi, idesc_qk, k != 0);
+          mma_commit(&k_empty[st]);
+          mma_commit(&s_full[st]);
+        }
+        __syncwarp();
         return true;
       };
       bool ok = mbar_wait(q_full, 0);
@@ -176,14 +188,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       if (ok) {
         tc_fence_after_sync();
         constexpr uint32_t idesc_self = idesc_bf16_f32(kPfBM, 128, false, false);
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < kPfD / 16; ++k) {
-          const uint32_t off = (k >> 2) * kPfPanel + (k & 3) * 32;
-          mma_ss(tmem + kColS, desc_kmajor_sw128(q_addr + off), desc_kmajor_sw128(k_addr + off), idesc_self, k != 0);
+          for (int k = 0; k < kPfD / 16; ++k) {
+            const uint32_t off = ((k >> 2) * kPfPanel + (k & 3) * 32) >> 4;
+            mma_ss_lohi(tmem + kColS, q_lo + off, q_hi, k_lo + off, k_hi, idesc_self, k != 0);
+          }
+          mma_commit(&k_empty[0]);
+          mma_commit(&k_empty[1]);
+          mma_commit(&s_full[0]);
         }
-        mma_commit(&k_empty[0]);
-        mma_commit(&k_empty[1]);
-        mma_commit(&s_full[0]);
+        __syncwarp();
         ok = mbar_wait(p_ready, 0);                  // diagonal extracted: S may be overwritten
       }
       ok = ok && issue_qk(0);
@@ -198,12 +213,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (!mbar_wait(&v_full[st], (i >> 1) & 1)) { ok = false; break; }
         tc_fence_after_sync();
         const int ksteps = tile_keys(i) / 16;
-        const uint32_t vb = v_addr + st * kPfKvTile;
-        for (int k = 0; k < ksteps; ++k)
-          mma_ts(tmem + kColO, tmem + kColS + st * kPfBN + k * 8, desc_mnmajor_sw128(vb + k * 2048, kPfKvPanel),
-                 idesc_pv, (i | k) != 0);
-        mma_commit(&v_empty[st]);
-        mma_commit(pv_done);
+        const uint32_t vb = v_lo + ((st * kPfKvTile) >> 4);
+        const uint32_t pa = tmem + kColS + st * kPfBN;
+        if (elect_one()) {
+#pragma unroll
+          for (int k = 0; k < kPfBN / 16; ++k)
+            if (k < ksteps) mma_ts_lohi(tmem + kColO, pa + k * 8, vb + ((k * 2048) >> 4), v_hi, idesc_pv, (i | k) != 0);
+          mma_commit(&v_empty[st]);
+          mma_commit(pv_done);
+        }
+        __syncwarp();
       }
     }
   } else {
