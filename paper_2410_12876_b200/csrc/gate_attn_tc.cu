@@ -95,48 +95,56 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(kGaBM, kGaBN, false, false);
-      constexpr uint32_t idesc_pv = idesc_bf16_f32(kGaBM, kGaD, false, true);
-      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
-      auto issue_qk = [&](int i) -> bool {
-        if (!mbar_wait(k_full, i & 1)) return false;
-        tc_fence_after_sync();
-        const uint32_t d = tmem + kGaColS + (i & 1) * 128;
+    // every lane runs the control flow (operands stay warp-uniform); one elected lane issues
+    constexpr uint32_t idesc_qk = idesc_bf16_f32(kGaBM, kGaBN, false, false);
+    constexpr uint32_t idesc_pv = idesc_bf16_f32(kGaBM, kGaD, false, true);
+    const uint64_t dq = desc_kmajor_sw128(smem_u32(sQ)), dk = desc_kmajor_sw128(smem_u32(sK));
+    const uint64_t dv = desc_mnmajor_sw128(smem_u32(sV), kGaPanel);
+    const uint32_t q_lo = (uint32_t)dq, q_hi = (uint32_t)(dq >> 32);
+    const uint32_t k_lo = (uint32_t)dk, k_hi = (uint32_t)(dk >> 32);
+    const uint32_t v_lo = (uint32_t)dv, v_hi = (uint32_t)(dv >> 32);
+    auto issue_qk = [&](int i) -> bool {
+      if (!mbar_wait(k_full, i & 1)) return false;
+      tc_fence_after_sync();
+      const uint32_t d = tmem + kGaColS + (i & 1) * 128;
+      if (elect_one()) {
         // Qhi Khi + Qhi Klo + Qlo Khi
 #pragma unroll
         for (int t = 0; t < 3; ++t) {
-          const uint32_t qa = q_addr + (t == 2 ? kGaTile : 0), ka = k_addr + (t == 1 ? kGaTile : 0);
+          const uint32_t qa = q_lo + ((t == 2 ? kGaTile : 0) >> 4), ka = k_lo + ((t == 1 ? kGaTile : 0) >> 4);
 #pragma unroll
           for (int k = 0; k < kGaD / 16; ++k) {
-            const uint32_t off = (k >> 2) * kGaPanel + (k & 3) * 32;
-            mma_ss(d, desc_kmajor_sw128(qa + off), desc_kmajor_sw128(ka + off), idesc_qk, (t | k) != 0);
+            const uint32_t off = ((k >> 2) * kGaPanel + (k & 3) * 32) >> 4;
+            mma_ss_lohi(d, qa + off, q_hi, ka + off, k_hi, idesc_qk, (t | k) != 0);
           }
         }
         mma_commit(k_empty);
         mma_commit(&s_full[i & 1]);
-        return true;
-      };
-      bool ok = mbar_wait(q_full, 0);
-      ok = ok && issue_qk(0);
-      for (int i = 0; i < n_kv && ok; ++i) {
-        if (i + 1 < n_kv) ok = issue_qk(i + 1);
-        if (!ok) break;
-        if (!mbar_wait(p_ready, i & 1)) { ok = false; break; }
-        if (!mbar_wait(v_full, i & 1)) { ok = false; break; }
-        tc_fence_after_sync();
+      }
+      __syncwarp();
+      return true;
+    };
+    bool ok = mbar_wait(q_full, 0);
+    ok = ok && issue_qk(0);
+    for (int i = 0; i < n_kv && ok; ++i) {
+      if (i + 1 < n_kv) ok = issue_qk(i + 1);
+      if (!ok) break;
+      if (!mbar_wait(p_ready, i & 1)) { ok = false; break; }
+      if (!mbar_wait(v_full, i & 1)) { ok = false; break; }
+      tc_fence_after_sync();
+      if (elect_one()) {
         // Phi Vhi + Phi Vlo + Plo Vhi
 #pragma unroll
         for (int t = 0; t < 3; ++t) {
-          const uint32_t pa = tmem + (t == 2 ? kGaColPlo : kGaColPhi), va = v_addr + (t == 1 ? kGaTile : 0);
+          const uint32_t pa = tmem + (t == 2 ? kGaColPlo : kGaColPhi), va = v_lo + ((t == 1 ? kGaTile : 0) >> 4);
 #pragma unroll
           for (int k = 0; k < kGaBN / 16; ++k)
-            mma_ts(tmem + kGaColO, pa + k * 8, desc_mnmajor_sw128(va + k * 2048, kGaPanel), idesc_pv,
-                   (i | t | k) != 0);
+            mma_ts_lohi(tmem + kGaColO, pa + k * 8, va + ((k * 2048) >> 4), v_hi, idesc_pv, (i | t | k) != 0);
         }
         mma_commit(v_empty);
         mma_commit(pv_done);
       }
+      __syncwarp();
     }
   } else {
     const int quad = warp & 3;
@@ -157,20 +165,22 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
       const int nvalid = min(max(bound - i * kGaBN, 0), kGaBN);
       const bool full = nvalid >= kGaBN;
 
-      float tmax = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld_x32_sync(tS + c * 32, r);
-        if (full) {
+      uint32_t r[128];
+      tmem_ld_x128_sync(tS, r);
+      if (!full) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(r[e]));
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            tmax = fmaxf(tmax, (c * 32 + e < nvalid) ? __uint_as_float(r[e]) : -INFINITY);
-        }
+        for (int e = 0; e < 128; ++e)
+          if (e >= nvalid) r[e] = 0xff800000u;        // -inf: weight 0 below
       }
+      float mx[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) mx[q] = __uint_as_float(r[q]);
+#pragma unroll
+      for (int e = 8; e < 128; e += 8)
+#pragma unroll
+        for (int q = 0; q < 8; ++q) mx[q] = fmaxf(mx[q], __uint_as_float(r[e + q]));
+      float tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
       tmax *= a.scale_log2;
       // tile 0 always holds key 0, visible to every row, so m is finite from here on
       float m_new;
@@ -196,29 +206,25 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
         }
       }
 
-      float rowsum = 0.f;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32], ph[16], pl[16];
-        tmem_ld_x32_sync(tS + c * 32, r);
+      float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(r[e]), a.scale_log2, -m_new));
-          float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, -m_new));
-          if (!full) {
-            p0 = (c * 32 + e < nvalid) ? p0 : 0.f;
-            p1 = (c * 32 + e + 1 < nvalid) ? p1 : 0.f;
-          }
-          rowsum += p0 + p1;
+      for (int c = 0; c < 8; ++c) {
+        uint32_t ph[8], pl[8];
+#pragma unroll
+        for (int e = 0; e < 16; e += 2) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e]), a.scale_log2, -m_new));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e + 1]), a.scale_log2, -m_new));
+          rs[(e >> 1) & 3] += p0 + p1;
           float h0, l0, h1, l1;
           split_bf16(p0, h0, l0);
           split_bf16(p1, h1, l1);
           ph[e >> 1] = pack_bf16x2(h0, h1);
           pl[e >> 1] = pack_bf16x2(l0, l1);
         }
-        tmem_st_x16(tm_lane + kGaColPhi + c * 16, ph);
-        tmem_st_x16(tm_lane + kGaColPlo + c * 16, pl);
+        tmem_st_x8(tm_lane + kGaColPhi + c * 8, ph);
+        tmem_st_x8(tm_lane + kGaColPlo + c * 8, pl);
       }
+      const float rowsum = (rs[0] + rs[1]) + (rs[2] + rs[3]);
       l += rowsum;
       m = m_new;
       tmem_st_wait();

@@ -78,26 +78,32 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16_f32(kTcBM, BN, false, true);
-      bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % Cfg::kStages;
-        const uint32_t ph = (kb / Cfg::kStages) & 1;
-        ok = mbar_wait(&full[s], ph);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint32_t a = smem_u32(smem + s * Cfg::kStageBytes), b = a + Cfg::kABytes;
+    // every lane runs the control flow (operands stay warp-uniform); one elected lane issues
+    constexpr uint32_t idesc = idesc_bf16_f32(kTcBM, BN, false, true);
+    const uint64_t da0 = desc_kmajor_sw128(smem_u32(smem));
+    const uint64_t db0 = desc_mnmajor_sw128(smem_u32(smem) + Cfg::kABytes, Cfg::kPanelBytes);
+    const uint32_t a_lo0 = (uint32_t)da0, a_hi = (uint32_t)(da0 >> 32);
+    const uint32_t b_lo0 = (uint32_t)db0, b_hi = (uint32_t)(db0 >> 32);
+    bool ok = true;
+    for (int kb = 0; kb < num_kb && ok; ++kb) {
+      const int s = kb % Cfg::kStages;
+      const uint32_t ph = (kb / Cfg::kStages) & 1;
+      ok = mbar_wait(&full[s], ph);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t a_lo = a_lo0 + ((s * Cfg::kStageBytes) >> 4), b_lo = b_lo0 + ((s * Cfg::kStageBytes) >> 4);
+      if (elect_one()) {
 #pragma unroll
         for (int k = 0; k < kTcBK / 16; ++k) {
           // 16 elements of K: 32 bytes along a K-major row; 16 k-rows (2048 B) of an MN-major panel
-          mma_ss(tmem_acc, desc_kmajor_sw128(a + k * 32), desc_mnmajor_sw128(b + k * 2048, Cfg::kPanelBytes),
-                 idesc, (kb | k) != 0);
+          mma_ss_lohi(tmem_acc, a_lo + ((k * 32) >> 4), a_hi, b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
         }
         mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
       }
-      mma_commit(acc_full);        // accumulator complete (or unwinding)
+      __syncwarp();
     }
+    if (elect_one()) mma_commit(acc_full);   // accumulator complete (or unwinding)
+    __syncwarp();
   } else {
     // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32)
     const int quad = warp & 3;
