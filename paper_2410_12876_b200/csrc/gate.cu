@@ -73,23 +73,53 @@ gate_proj_kernel(const T *__restrict__ A, const T *__restrict__ W0, const T *__r
   }
 }
 
-// One warp per token: s[i] = sum_c H[t, c] Wo[c, i]; lane i (+32, ...) owns head i.
+// s = [H'_1 .. H'_h'] Wo_g and the threshold of Eq. 4.  One CTA = 16 tokens, one
+// warp = 4 of them, lane = head (in rounds of 32 heads).  The 16 rows of H and a
+// [GD][32] slice of Wo are staged in shared memory: per step of the reduction a
+// warp reads one conflict-free row of Wo and four broadcast values of H.
+constexpr int kOutTokens = 16, kOutThreads = 128;
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kOutThreads)
 gate_out_kernel(const float *__restrict__ H, const T *__restrict__ Wo,
                 const float *__restrict__ gamma, float logit_tau, int B, int n, int GD, int h,
                 float *__restrict__ scores, uint8_t *__restrict__ flags) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (warp >= B * n) return;
-  const int b = warp / n, t = warp % n;
-  const float *Hr = H + (size_t)warp * GD;
-  for (int i = lane; i < h; i += 32) {
-    float acc = 0.f;
-    for (int c = 0; c < GD; ++c) acc = fmaf(Hr[c], Elem<T>::load(Wo + (size_t)c * h + i), acc);
-    const size_t o = ((size_t)b * h + i) * n + t;
-    if (scores) scores[o] = acc;
-    const float z = acc + (gamma ? gamma[i] : 0.f);
-    flags[o] = z > logit_tau ? 1 : 0;
+  extern __shared__ __align__(16) unsigned char sh_raw[];
+  float *Hs = reinterpret_cast<float *>(sh_raw);                       // [16][GD]
+  T *Ws = reinterpret_cast<T *>(sh_raw + sizeof(float) * kOutTokens * GD);   // [GD][32]
+  const int tiles_per_seq = (n + kOutTokens - 1) / kOutTokens;
+  const int b = blockIdx.x / tiles_per_seq, t0 = (blockIdx.x % tiles_per_seq) * kOutTokens;
+  const int nt = min(kOutTokens, n - t0);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float *Hg = H + ((size_t)b * n + t0) * GD;                     // rows are contiguous
+  for (int x = threadIdx.x; x < kOutTokens * GD; x += kOutThreads) Hs[x] = x < nt * GD ? Hg[x] : 0.f;
+  for (int i0 = 0; i0 < h; i0 += 32) {
+    __syncthreads();
+    for (int x = threadIdx.x; x < GD * 32; x += kOutThreads) {
+      const int c = x >> 5, i = i0 + (x & 31);
+      Ws[x] = i < h ? Wo[(size_t)c * h + i] : T(0.f);
+    }
+    __syncthreads();
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const float *hr = Hs + warp * 4 * GD;
+#pragma unroll 8
+    for (int c = 0; c < GD; ++c) {
+      const float w = Elem<T>::load(Ws + c * 32 + lane);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) acc[q] = fmaf(hr[q * GD + c], w, acc[q]);
+    }
+    const int i = i0 + lane;
+    if (i < h) {
+      const float gm = gamma ? gamma[i] : 0.f;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int tt = warp * 4 + q;
+        if (tt < nt) {
+          const size_t o = ((size_t)b * h + i) * n + t0 + tt;
+          if (scores) scores[o] = acc[q];
+          flags[o] = (acc[q] + gm) > logit_tau ? 1 : 0;
+        }
+      }
+    }
   }
 }
 
@@ -145,9 +175,12 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
   }
 
   const float logit_tau = (float)log((double)d.tau / (1.0 - (double)d.tau));
-  const int warps = M, blocks = (warps * 32 + 255) / 256;
-  gate_out_kernel<T><<<blocks, 256, 0, st>>>(hcat, static_cast<const T *>(Wo), gamma, logit_tau,
-                                             d.batch, d.seq, GD, d.heads, scores, flags);
+  const size_t out_smem = sizeof(float) * (size_t)kOutTokens * GD + sizeof(T) * (size_t)GD * 32;
+  auto out_kern = gate_out_kernel<T>;
+  AG_CUDA_TRY(cudaFuncSetAttribute(out_kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)out_smem));
+  const int blocks = d.batch * ((d.seq + kOutTokens - 1) / kOutTokens);
+  out_kern<<<blocks, kOutThreads, out_smem, st>>>(hcat, static_cast<const T *>(Wo), gamma, logit_tau,
+                                                 d.batch, d.seq, GD, d.heads, scores, flags);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
