@@ -1,0 +1,160 @@
+"""Parity at the full workload sizes, in the launch configuration bench.py times.
+
+The oracle cannot evaluate every output at these sizes in reasonable time, so
+attention outputs are compared on sampled query rows / slabs (each computed by
+the oracle one by one from the dense definition), while everything integer
+(flags outside the threshold band, prefix, idx, lengths, cache rows) is compared
+in full.  The GPU's compaction and attention are driven by the ORACLE's flags,
+so the oracle never depends on a GPU result."""
+import numpy as np
+import pytest
+import torch
+
+import agtest as T
+from oracle import ag_oracle as orc
+from paper_2410_12876_b200 import binding as ag
+from paper_2410_12876_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    T.ensure_built()
+
+
+def _sample_rows(n, k, seed):
+    rng = np.random.default_rng(seed)
+    rows = np.unique(np.concatenate([[0, 1, 63, 64, 127, 128, n - 129, n - 128, n - 1],
+                                     rng.integers(0, n, size=k)]))
+    return rows[(rows >= 0) & (rows < n)]
+
+
+def _check_prefill_rows(shape, Q, K, V, flags_np, O, heads, rows_per_head, seed):
+    worst = (0.0, 0.0)
+    for b in range(shape.batch):
+        for i in heads:
+            rows = _sample_rows(shape.seq, rows_per_head, seed + 31 * i + b)
+            ref = orc.prefill_head(T.f64(Q[b, i]), T.f64(K[b, i]), T.f64(V[b, i]), flags_np[b, i], rows=rows)
+            got = T.f64(O[b, i][torch.from_numpy(rows).to(O.device)])
+            e = T.check_close(got, ref, shape.dtype, f"prefill b={b} head={i}")
+            worst = (max(worst[0], e[0]), max(worst[1], e[1]))
+    return worst
+
+
+def test_prefill7b_layer():
+    """Llama-2-7B-shaped layer: gate, compaction, prefill attention, decode + append."""
+    shape = inputs.PREFILL7B
+    seed = 2000
+    X = inputs.hidden_states(shape, seed, DEV)
+    W = inputs.layer_weights(shape, seed + 10, DEV)
+    Q, K, V = inputs.project_qkv(shape, X, W)
+    keep = inputs.keep_targets_uniform(shape.heads, seed + 20)
+    # gate: oracle scores at gamma = 0 give gamma (an input); then both sides run with it
+    s0, _ = T.oracle_gate(shape, X, W, None)
+    gamma = inputs.calibrate_gamma(torch.from_numpy(s0), keep, shape.tau).to(DEV)
+    s_ref, f_ref = T.oracle_gate(shape, X, W, gamma)
+    scores, flags = T.gpu_gate(shape, X, W, gamma)
+    err = np.max(np.abs(T.f64(scores) - s_ref))
+    assert err < 1e-4, err
+    excluded = T.check_flags(shape, flags, s_ref, f_ref, gamma)
+    assert excluded < 0.1, excluded
+    assert np.max(np.abs(f_ref.mean(axis=(0, 2)) - keep)) < 0.01
+    # downstream calls run on the oracle's flags
+    fl = torch.from_numpy(f_ref).to(DEV)
+    steps = 4
+    cap = [shape.seq + steps] * (shape.batch * shape.heads)
+    cache, prefix, idx, status = T.gpu_compact(shape, K, V, fl, cap=cap)
+    T.check_compaction(shape, K, V, fl, cache, prefix, idx)
+    O = T.gpu_prefill(shape, Q, K, V, fl, cache, prefix)
+    assert torch.isfinite(O.float()).all()
+    _check_prefill_rows(shape, Q, K, V, f_ref, O, range(shape.heads), 192, 7)
+    # decode over the cache just built, all slabs
+    ocache = orc.compact_kv(T.f64(K), T.f64(V), f_ref)
+    for step in range(steps):
+        q, kn, vn, fn = inputs.decode_inputs(shape, seed + 500, step, DEV, keep_new=0.5)
+        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status)
+        T.check_close(T.f64(o), orc.decode_attention(T.f64(q), T.f64(kn), T.f64(vn), ocache), "bf16", f"decode {step}")
+        orc.cache_append(ocache, T.f64(kn), T.f64(vn), fn.cpu().numpy())
+    assert np.array_equal(cache.len.cpu().numpy(), orc.cache_lengths(ocache).reshape(-1))
+    assert int(status.item()) == 0 and ag.ag_device_wait_timeouts() == 0
+
+
+def test_deep_layer_pattern():
+    """Sequence 16384, 24 heads at ~90 % eviction and 8 heads fully evicted."""
+    shape = inputs.DEEP_LAYER
+    seed = 4000
+    Q, K, V = inputs.qkv_gaussian(shape, seed, DEV)
+    flags_cpu, empty = inputs.deep_layer_flags(shape, seed + 20)
+    f_np = flags_cpu.numpy()
+    fl = flags_cpu.to(DEV)
+    steps = 4
+    L = f_np.reshape(shape.heads, -1).sum(axis=1)
+    cache, prefix, idx, status = T.gpu_compact(shape, K, V, fl, cap=(L + steps).tolist())     # tight slabs
+    T.check_compaction(shape, K, V, fl, cache, prefix, idx)
+    O = T.gpu_prefill(shape, Q, K, V, fl, cache, prefix)
+    assert torch.isfinite(O.float()).all()
+    # fully evicted heads: only the diagonal survives (Sec. 3.3), O = V exactly
+    for i in empty:
+        assert torch.equal(O[0, i], V[0, i])
+    sparse = [i for i in range(shape.heads) if i not in set(empty.tolist())]
+    _check_prefill_rows(shape, Q, K, V, f_np, O, sparse, 96, 11)
+    # decode: sparse heads keep new tokens with probability 0.1, empty heads never do
+    ocache = orc.compact_kv(T.f64(K), T.f64(V), f_np)
+    for step in range(steps):
+        q, kn, vn, fn = inputs.decode_inputs(shape, seed + 500, step, DEV, keep_new=0.1)
+        fn[:, torch.from_numpy(empty).to(DEV)] = 0
+        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status)
+        T.check_close(T.f64(o), orc.decode_attention(T.f64(q), T.f64(kn), T.f64(vn), ocache), "bf16", f"decode {step}")
+        for i in empty:
+            assert torch.equal(o[0, i], vn[0, i])                      # empty slab: o = v_new
+        orc.cache_append(ocache, T.f64(kn), T.f64(vn), fn.cpu().numpy())
+    assert np.array_equal(cache.len.cpu().numpy(), orc.cache_lengths(ocache).reshape(-1))
+    assert int(status.item()) == 0 and ag.ag_device_wait_timeouts() == 0
+
+
+def test_ragged_decode():
+    """Batch 32 x 32 heads, retained lengths U[0.2, 0.9] x 8192, keep-new Bernoulli(0.5)."""
+    shape = inputs.DECODE_RAGGED
+    seed = 3000
+    B, h, D = shape.batch, shape.heads, shape.head_dim
+    steps = 3
+    L0 = inputs.ragged_lengths(B * h, shape.seq, seed + 30)
+    cache = ag.RaggedCache.allocate(shape, (L0.astype(np.int64) + 256).tolist(), DEV)
+    for t, sd in ((cache.k_rows, seed + 31), (cache.v_rows, seed + 32)):
+        for r0 in range(0, t.shape[0], 1 << 20):
+            r1 = min(t.shape[0], r0 + (1 << 20))
+            t[r0:r1] = inputs.randn((r1 - r0, D), sd + r0, DEV, shape.torch_dtype)
+    cache.len.copy_(torch.from_numpy(L0).to(DEV))
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    off = cache.row_off.cpu().numpy()
+    slabs = np.unique(np.concatenate([[0, 1, B * h - 1, int(np.argmin(L0)), int(np.argmax(L0))],
+                                      np.random.default_rng(5).integers(0, B * h, size=59)]))
+    # the oracle's view of the sampled slabs: input rows, widened exactly
+    ocache = {int(s): {"k": T.f64(cache.k_rows[off[s]:off[s] + L0[s]]), "v": T.f64(cache.v_rows[off[s]:off[s] + L0[s]])}
+              for s in slabs}
+    want_len = L0.astype(np.int64).copy()
+    ws = ag.workspace(ag.make_desc(shape), ag.AG_CALL_DECODE)
+    for step in range(steps):
+        q, kn, vn, fn = inputs.decode_inputs(shape, seed + 500, step, DEV, keep_new=0.5)
+        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status, ws=ws)
+        assert torch.isfinite(o.float()).all()
+        qf, kf, vf, fnp = T.f64(q).reshape(B * h, D), T.f64(kn).reshape(B * h, D), T.f64(vn).reshape(B * h, D), \
+            fn.cpu().numpy().reshape(-1)
+        of = T.f64(o).reshape(B * h, D)
+        for s in slabs:
+            c = ocache[int(s)]
+            ref = orc.decode_head(qf[s], kf[s], vf[s], c["k"], c["v"])
+            T.check_close(of[s], ref, "bf16", f"step {step} slab {s}")
+            if fnp[s]:
+                c["k"] = np.concatenate([c["k"], kf[s][None]])
+                c["v"] = np.concatenate([c["v"], vf[s][None]])
+        want_len += fnp
+    assert np.array_equal(cache.len.cpu().numpy(), want_len)
+    # appended rows of the sampled slabs are bit copies, in order
+    for s in slabs:
+        n_s = int(want_len[s])
+        assert np.array_equal(T.f64(cache.k_rows[off[s]:off[s] + n_s]), ocache[int(s)]["k"])
+        assert np.array_equal(T.f64(cache.v_rows[off[s]:off[s] + n_s]), ocache[int(s)]["v"])
+    assert int(status.item()) == 0
