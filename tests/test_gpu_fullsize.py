@@ -55,6 +55,7 @@ def test_prefill7b_layer():
     s0, _ = T.oracle_gate(shape, X, W, None)
     gamma = inputs.calibrate_gamma(torch.from_numpy(s0), keep, shape.tau).to(DEV)
     s_ref, f_ref = T.oracle_gate(shape, X, W, gamma)
+    f_ref = np.ascontiguousarray(f_ref)
     scores, flags = T.gpu_gate(shape, X, W, gamma)
     err = np.max(np.abs(T.f64(scores) - s_ref))
     assert err < 1e-4, err
