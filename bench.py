@@ -109,6 +109,7 @@ class LayerRun:
         self.desc = ag.make_desc(sh)
         B, h, n, D = sh.batch, sh.heads, sh.seq, sh.head_dim
         self.name = name
+        self.use_graph, self.graph = True, None
         self.has_gate = name in ("prefill7b", "tiny")
         self.has_prefill = name != "decode_ragged"
         if self.has_gate:
@@ -194,7 +195,28 @@ class LayerRun:
             timed("prefill", self.prefill)
         else:
             self.cache.len.copy_(self.len0)      # every pass starts from the same cache
-        timed("decode", lambda: [self.decode(s) for s in range(self.decode_steps)])
+        timed("decode", self.decode_all)
+
+    def decode_all(self):
+        """All decode steps of a pass.  They are dozens of small launches, so they are
+        replayed from one CUDA graph (captured once, on first use) unless disabled."""
+        if not self.use_graph:
+            for s in range(self.decode_steps):
+                self.decode(s)
+            return
+        if self.graph is None:
+            len_before = self.cache.len.clone()
+            for s in range(self.decode_steps):       # warm-up outside capture
+                self.decode(s)
+            self.cache.len.copy_(len_before)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for s in range(self.decode_steps):
+                    self.decode(s)
+            self.cache.len.copy_(len_before)         # capture does not run the kernels
+            self.graph = g
+        self.graph.replay()
 
     def tokens_per_step(self):
         return self.shape.batch * ((self.shape.seq if self.has_prefill else 0) + self.decode_steps)
@@ -234,6 +256,7 @@ def flush_l2(buf):
 def run_ours(args, rank, world, dev):
     torch.cuda.set_device(dev)
     run = LayerRun(args.workload, 2000 + 100 * rank, dev)
+    run.use_graph = not args.no_graph
     l2buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     dist = None
     if world > 1:
@@ -347,7 +370,8 @@ def run_ours(args, rank, world, dev):
                    "hidden": sh.hidden, "heads": sh.heads, "head_dim": sh.head_dim, "gate_heads": sh.gate_heads,
                    "gate_head_dim": sh.gate_head_dim, "decode_steps_per_step": run.decode_steps,
                    "mean_keep": float(run.flags.float().mean().item()) if run.has_prefill else None,
-                   "l2": "flushed between steps (256 MiB write)", "replicas": world},
+                   "l2": "flushed between steps (256 MiB write)", "replicas": world,
+                   "decode_launch": "one CUDA graph per pass" if run.use_graph else "individual launches"},
         "clocks": clocks,
         "e2e": {"value": tokens * e2e_steps / (t_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
@@ -448,6 +472,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="prefill7b", choices=list(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch the decode steps one by one instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
