@@ -15,8 +15,8 @@
 namespace ag {
 
 constexpr int kMaxSplits = 32;     // chunks per slab the workspace is sized for
-constexpr int kPartThreads = 128;
-constexpr int kUnroll = 4;         // rows in flight per lane group (x2: K and V)
+constexpr int kPartThreads = 256;
+constexpr int kUnroll = 8;         // rows in flight per lane group (x2: K and V)
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kPartThreads)
@@ -159,8 +159,7 @@ static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, 
                       const ag_cache &c, float scale, void *o, void *ws, cudaStream_t st) {
   const int slabs = d.batch * d.heads;
   int chunk_rows = (c.max_cap + kMaxSplits - 1) / kMaxSplits;
-  chunk_rows = (chunk_rows + 63) / 64 * 64;
-  if (chunk_rows < 256) chunk_rows = 256;
+  chunk_rows = (chunk_rows + 127) / 128 * 128;   // whole iterations of the partial kernel (bf16, D = 128)
   const int n_chunks = c.max_cap > 0 ? (c.max_cap + chunk_rows - 1) / chunk_rows : 0;
   float *part_o = static_cast<float *>(ws);
   float *part_ml = part_o + (size_t)slabs * kMaxSplits * D;
