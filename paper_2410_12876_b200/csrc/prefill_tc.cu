@@ -73,8 +73,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   uint64_t *q_full = bars;
   uint64_t *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;   // [2] each
   uint64_t *s_full = bars + 9;                     // [2]
-  uint64_t *p_ready = bars + 11, *pv_done = bars + 12;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 13);
+  uint64_t *p_ready = bars + 11, *pv_done = bars + 12;   // pv_done[2]: even / odd cache tiles
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 14);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // heaviest query tiles first
@@ -98,7 +98,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       mbar_init(&s_full[s], 1);
     }
     mbar_init(p_ready, 128);
-    mbar_init(pv_done, 1);
+    mbar_init(&pv_done[0], 1); mbar_init(&pv_done[1], 1);
     fence_barrier_init();
     prefetch_tensormap(&tmQ); prefetch_tensormap(&tmKd); prefetch_tensormap(&tmVd);
     prefetch_tensormap(&tmK); prefetch_tensormap(&tmV); prefetch_tensormap(&tmO);
@@ -205,7 +205,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       for (int i = 0; i < n_kv && ok; ++i) {
         if (i + 1 < n_kv) {
           // S[(i+1)&1] still holds P of tile i - 1 until that P V has completed
-          if (i >= 1 && !mbar_wait(pv_done, (i - 1) & 1)) { ok = false; break; }
+          if (i >= 1 && !mbar_wait(&pv_done[(i - 1) & 1], ((i - 1) >> 1) & 1)) { ok = false; break; }
           if (!issue_qk(i + 1)) { ok = false; break; }
         }
         const int st = i & 1;
@@ -220,7 +220,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           for (int k = 0; k < kPfBN / 16; ++k)
             if (k < ksteps) mma_ts_lohi(tmem + kColO, pa + k * 8, vb + ((k * 2048) >> 4), v_hi, idesc_pv, (i | k) != 0);
           mma_commit(&v_empty[st]);
-          mma_commit(pv_done);
+          mma_commit(&pv_done[st]);
         }
         __syncwarp();
       }
@@ -302,21 +302,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       l = l * alpha + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
       m = m_new;
 
-      // The previous P V must be complete before O is rescaled; waiting for it on
-      // every tile also keeps this thread in step with the barrier's phases.
-      if (i > 0) {
-        ok = mbar_wait(pv_done, (i - 1) & 1);
+      // P V completions alternate between two barriers, so the wait that keeps this
+      // thread in step with their phases is for tile i - 2, long finished; only a
+      // rescale of O has to wait for the P V of tile i - 1 itself.
+      if (i >= 2) {
+        ok = mbar_wait(&pv_done[st], ((i - 2) >> 1) & 1);
         if (!ok) break;
-        if (rescale) {
-          tc_fence_after_sync();
+      }
+      if (rescale) {
+        ok = mbar_wait(&pv_done[(i - 1) & 1], ((i - 1) >> 1) & 1);
+        if (!ok) break;
+        tc_fence_after_sync();
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            uint32_t o[32];
-            tmem_ld_x32_sync(tm_lane + kColO + c * 32, o);
+        for (int c = 0; c < 4; ++c) {
+          uint32_t o[32];
+          tmem_ld_x32_sync(tm_lane + kColO + c * 32, o);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st_x32(tm_lane + kColO + c * 32, o);
-          }
+          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+          tmem_st_x32(tm_lane + kColO + c * 32, o);
         }
       }
 
@@ -341,8 +344,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
 
     // epilogue: O_j = (sum_r p_r v_r + w_self v_j) / l, staged in the V buffer, one TMA store
+    if (ok && n_kv > 1) ok = mbar_wait(&pv_done[(n_kv - 2) & 1], ((n_kv - 2) >> 1) & 1);
     if (ok && n_kv > 0) {
-      ok = mbar_wait(pv_done, (n_kv - 1) & 1);
+      ok = mbar_wait(&pv_done[(n_kv - 1) & 1], ((n_kv - 1) >> 1) & 1);
       tc_fence_after_sync();
     }
     if (ok) ok = mbar_wait(&k_full[0], k0_uses & 1);          // dense V tile has landed in sK
