@@ -26,14 +26,23 @@ namespace ag {
 using namespace umma;
 
 constexpr int kPfThreads = 192;
-constexpr int kPfBM = 128, kPfBN = 64, kPfD = 128;
+constexpr int kPfBM = 128, kPfD = 128;
 constexpr int kPfPanel = 128 * 128;                   // [128 rows][64 bf16] = 16 KB (Q, dense K / V, O)
 constexpr int kPfTile = 2 * kPfPanel;                 // 32 KB
-constexpr int kPfKvPanel = kPfBN * 128;               // [64 rows][64 bf16] = 8 KB (cache tiles)
-constexpr int kPfKvTile = 2 * kPfKvPanel;             // 16 KB; two stages fill one 32 KB buffer
-constexpr int kPfSmemBytes = 3 * kPfTile + 1024 + 256;
-constexpr uint32_t kColS = 0, kColO = 128, kTmemCols = 256;   // S0 [0,64) S1 [64,128), P in place
 constexpr float kRescaleThreshold = 8.f;              // log2 units
+
+// Geometry for key tiles of BN cache rows.  BN = 64: two CTAs per SM (256 TMEM columns each);
+// BN = 128: one CTA per SM (384 of 512 columns used).  TMEM: S0 [0,BN) S1 [BN,2BN), each
+// overwritten in place by its P (bf16 pairs); O [2BN, 2BN+128).
+template <int BN> struct PfCfg {
+  static constexpr int kKvPanel = BN * 128;           // [BN rows][64 bf16]
+  static constexpr int kKvTile = 2 * kKvPanel;
+  static constexpr int kKvBuf = 2 * kKvTile;          // two stages; >= one 32 KB dense tile
+  static constexpr int kSelfStages = 128 / BN;        // K stages the 128-row self tile covers
+  static constexpr int kSmemBytes = kPfTile + 2 * kKvBuf + 1024 + 256;
+  static constexpr uint32_t kColO = 2 * BN, kTmemCols = BN == 64 ? 256 : 512;
+  static constexpr int kCtasPerSm = BN == 64 ? 2 : 1;
+};
 
 struct PrefillTcArgs {
   const int32_t *prefix;            // [slabs, n + 1]
@@ -59,17 +68,21 @@ __device__ __forceinline__ uint32_t tile_chunk_offset(int row, int chunk) {
 // CTA's own 128 rows, of which only the diagonal (q_j . k_j) is read.  Last,
 // the dense V tile is brought in for the self term of the output, and the O
 // tile leaves through shared memory with one TMA store.
-__global__ void __launch_bounds__(kPfThreads, 2)
+template <int BN>
+__global__ void __launch_bounds__(kPfThreads, PfCfg<BN>::kCtasPerSm)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKd,
                   const __grid_constant__ CUtensorMap tmVd, const __grid_constant__ CUtensorMap tmO,
                   const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const PrefillTcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  using Cfg = PfCfg<BN>;
+  constexpr int kPfBN = BN, kPfKvPanel = Cfg::kKvPanel, kPfKvTile = Cfg::kKvTile;
+  constexpr uint32_t kColS = 0, kColO = Cfg::kColO, kTmemCols = Cfg::kTmemCols;
   uint8_t *sQ = smem;
-  uint8_t *sK = sQ + kPfTile;                      // two 16 KB stages, or one 128-row dense tile
-  uint8_t *sV = sK + kPfTile;
-  uint64_t *bars = reinterpret_cast<uint64_t *>(sV + kPfTile);
+  uint8_t *sK = sQ + kPfTile;                      // two stages, or one 128-row dense tile
+  uint8_t *sV = sK + Cfg::kKvBuf;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(sV + Cfg::kKvBuf);
   uint64_t *q_full = bars;
   uint64_t *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;   // [2] each
   uint64_t *s_full = bars + 9;                     // [2]
@@ -87,8 +100,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int n_kv = (max_bound + kPfBN - 1) / kPfBN;
   const int n_self = n_kv > 0 ? 1 : 0;             // a lone diagonal needs no score
   const int row0 = (int)a.row_off[slab];
-  // completions of k_full[0] / s_full[0] before the dense V tile: self tile + even cache tiles
-  const int k0_uses = n_self + (n_kv + 1) / 2, k1_uses = n_self + n_kv / 2;
+  // uses of K stage 0 / 1 before the dense V tile: self tile (stage 0, and stage 1 when the
+  // 128-row tile spans both) + even / odd cache tiles
+  const int self1 = Cfg::kSelfStages == 2 ? n_self : 0;
+  const int k0_uses = n_self + (n_kv + 1) / 2, k1_uses = self1 + n_kv / 2;
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
@@ -127,8 +142,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int i = 0; i < n_kv && ok; ++i) {
           const int st = i & 1;
           const int y = row0 + i * kPfBN;
-          // the self tile was use 0 of both K stages; V stages start fresh
-          ok = mbar_wait(&k_empty[st], (((i >> 1) + 1) & 1) ^ 1);
+          // uses of this K stage so far: the self tile (where it covers the stage) + earlier tiles
+          const int k_used = (st == 0 ? n_self : self1) + (i >> 1);
+          ok = mbar_wait(&k_empty[st], (k_used & 1) ^ 1);
           if (!ok) break;
           mbar_arrive_expect_tx(&k_full[st], kPfKvTile);
           tma_load_2d(sK + st * kPfKvTile, &tmK, &k_full[st], 0, y);
@@ -142,7 +158,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       }
       // dense V rows for the self term of the output, into the K buffer once both stages are free
       if (ok && k0_uses > 0) ok = mbar_wait(&k_empty[0], (k0_uses & 1) ^ 1);
-      if (ok && k1_uses > 0) ok = mbar_wait(&k_empty[1], (k1_uses & 1) ^ 1);
+      if (ok && Cfg::kSelfStages == 2 && k1_uses > 0) ok = mbar_wait(&k_empty[1], (k1_uses & 1) ^ 1);
       if (ok) {
         mbar_arrive_expect_tx(&k_full[0], kPfTile);
         tma_load_3d(sK, &tmVd, &k_full[0], 0, j0, slab);
@@ -195,7 +211,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             mma_ss_lohi(tmem + kColS, q_lo + off, q_hi, k_lo + off, k_hi, idesc_self, k != 0);
           }
           mma_commit(&k_empty[0]);
-          mma_commit(&k_empty[1]);
+          if (Cfg::kSelfStages == 2) mma_commit(&k_empty[1]);
           mma_commit(&s_full[0]);
         }
         __syncwarp();
@@ -261,11 +277,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const int nvalid = min(max(bound - i * kPfBN, 0), kPfBN);
       const uint32_t tS = tm_lane + kColS + st * kPfBN;
 
-      uint32_t r[64];
-      tmem_ld_x64_sync(tS, r);
+      uint32_t r[BN];
+      if (BN == 64) tmem_ld_x64_sync(tS, r); else tmem_ld_x128_sync(tS, r);
       if (nvalid < kPfBN) {
 #pragma unroll
-        for (int e = 0; e < 64; ++e)
+        for (int e = 0; e < BN; ++e)
           if (e >= nvalid) r[e] = 0xff800000u;        // -inf: weight 0 below
       }
       // eight independent chains instead of one long dependency
@@ -273,7 +289,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
       for (int q = 0; q < 8; ++q) mx[q] = __uint_as_float(r[q]);
 #pragma unroll
-      for (int e = 8; e < 64; e += 8)
+      for (int e = 8; e < BN; e += 8)
 #pragma unroll
         for (int q = 0; q < 8; ++q) mx[q] = fmaxf(mx[q], __uint_as_float(r[e + q]));
       float tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
@@ -288,7 +304,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       // p = 2^(s - m) as bf16 pairs, written over the columns S occupied
       float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < BN / 16; ++c) {
         uint32_t pk[8];
 #pragma unroll
         for (int e = 0; e < 16; e += 2) {
@@ -329,12 +345,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       if ((i + 1) * kPfBN > L) {
         ok = mbar_wait(&v_full[st], (i >> 1) & 1);
         if (!ok) break;
-        const int vr = tid >> 1;                      // two threads per row, one panel each
+        // BN = 64: two threads per row, one panel each; BN = 128: one thread per row, both panels
+        const int vr = BN == 64 ? tid >> 1 : tid;
         if (i * kPfBN + vr >= L) {
           uint4 z = make_uint4(0, 0, 0, 0);
-          uint8_t *v0 = sV + st * kPfKvTile + (tid & 1) * kPfKvPanel + vr * 128;
+          uint8_t *v0 = sV + st * kPfKvTile + (BN == 64 ? (tid & 1) * kPfKvPanel : 0) + vr * 128;
 #pragma unroll
-          for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4 *>(v0 + c * 16) = z;
+          for (int c = 0; c < 8; ++c) {
+            *reinterpret_cast<uint4 *>(v0 + c * 16) = z;
+            if (BN == 128) *reinterpret_cast<uint4 *>(v0 + kPfKvPanel + c * 16) = z;
+          }
         }
         fence_proxy_async_smem();
       }
@@ -392,6 +412,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
+// Cache rows per key tile.  64 (two CTAs per SM) measured faster than 128 (one CTA per SM) on
+// 4096-token heads: 100 us against 131 us; the softmax threads, not the tensor core, set the pace.
+constexpr int kPrefillKeyTile = 64;
+
 bool prefill_tc_supported(const ag_layer_desc &d, const ag_cache &c) {
   return d.dtype == AG_BF16 && d.head_dim == 128 && c.pool_rows < ((int64_t)1 << 31) &&
          (int64_t)d.batch * d.heads * ((d.seq + kPfBM - 1) / kPfBM) < ((int64_t)1 << 31);
@@ -408,16 +432,18 @@ int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, cons
   if ((rc = make_tmap_3d_bf16(&tmO, O, slabs, d.seq, kPfD, kPfBM, 64))) return rc;
   // an empty pool still needs a valid map: describe one row of the dense K / V instead (never read)
   const bool empty = c.pool_rows == 0;
-  rc = make_tmap_2d_bf16(&tmK, empty ? K : c.k_rows, empty ? 1 : (uint64_t)c.pool_rows, kPfD, kPfD * 2, kPfBN, 64);
+  constexpr int BN = kPrefillKeyTile;
+  rc = make_tmap_2d_bf16(&tmK, empty ? K : c.k_rows, empty ? 1 : (uint64_t)c.pool_rows, kPfD, kPfD * 2, BN, 64);
   if (rc) return rc;
-  rc = make_tmap_2d_bf16(&tmV, empty ? V : c.v_rows, empty ? 1 : (uint64_t)c.pool_rows, kPfD, kPfD * 2, kPfBN, 64);
+  rc = make_tmap_2d_bf16(&tmV, empty ? V : c.v_rows, empty ? 1 : (uint64_t)c.pool_rows, kPfD, kPfD * 2, BN, 64);
   if (rc) return rc;
   PrefillTcArgs a;
   a.prefix = prefix; a.row_off = c.row_off; a.len = c.len;
   a.n = d.seq; a.n_qtiles = (d.seq + kPfBM - 1) / kPfBM; a.slabs = slabs;
   a.scale_log2 = scale * 1.4426950408889634f;
-  AG_CUDA_TRY(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes));
-  prefill_tc_kernel<<<a.n_qtiles * slabs, kPfThreads, kPfSmemBytes, st>>>(tmQ, tmKd, tmVd, tmO, tmK, tmV, a);
+  auto kern = prefill_tc_kernel<BN>;
+  AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PfCfg<BN>::kSmemBytes));
+  kern<<<a.n_qtiles * slabs, kPfThreads, PfCfg<BN>::kSmemBytes, st>>>(tmQ, tmKd, tmVd, tmO, tmK, tmV, a);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
