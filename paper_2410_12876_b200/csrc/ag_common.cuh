@@ -38,8 +38,9 @@ int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const voi
                         void *Clo, int M, int K, int GD, cudaStream_t st);
 // Tensor-core MHA' (Sec. 3.3) on the hi / lo pairs: H' [B*n, GD] float32.
 bool gate_attn_tc_supported(const ag_layer_desc &d);
+size_t gate_attn_partial_bytes(const ag_layer_desc &d);   // split-K partials (workspace)
 int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *qkv_lo, float *hcat,
-                        cudaStream_t st);
+                        void *partials, cudaStream_t st);
 int gate_attn_tc_wait_timeouts();
 int gemm_tc_wait_timeouts();
 

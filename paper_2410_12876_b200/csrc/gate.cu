@@ -125,7 +125,9 @@ gate_out_kernel(const float *__restrict__ H, const T *__restrict__ Wo,
 
 size_t gate_workspace_bytes(const ag_layer_desc &d) {
   const size_t rows = (size_t)d.batch * d.seq, GD = (size_t)d.gate_heads * d.gate_head_dim;
-  return align_up(rows * 3 * GD * sizeof(float), 256) + align_up(rows * GD * sizeof(float), 256);
+  size_t bytes = align_up(rows * 3 * GD * sizeof(float), 256) + align_up(rows * GD * sizeof(float), 256);
+  if (gate_attn_tc_supported(d)) bytes += gate_attn_partial_bytes(d);
+  return bytes;
 }
 
 template <typename T>
@@ -142,7 +144,8 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
     void *lo = static_cast<char *>(ws) + (size_t)M * 3 * GD * sizeof(__nv_bfloat16);
     int rc = launch_gate_proj_tc(X, Wq, Wk, Wv, nullptr, hi, lo, M, d.hidden, GD, st);
     if (rc) return rc;
-    rc = launch_gate_attn_tc(d, hi, lo, hcat, st);
+    void *partials = reinterpret_cast<char *>(hcat) + align_up((size_t)M * GD * sizeof(float), 256);
+    rc = launch_gate_attn_tc(d, hi, lo, hcat, partials, st);
     if (rc) return rc;
   } else {
     if (sizeof(T) == 2 && gate_proj_tc_supported(d.hidden, GD)) {

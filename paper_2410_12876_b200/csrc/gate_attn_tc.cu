@@ -9,9 +9,12 @@
 //
 // One CTA = 128 queries of one (sequence, gate head).  Structure as in the
 // prefill kernel: warp 0 TMA, warp 1 tcgen05.mma issue, warps 2..5 softmax with
-// one row per thread.  K and V tiles are single-buffered: the K load of tile
-// i + 2 overlaps P V of tile i and the V load of tile i + 1 overlaps Q K^T of
-// tile i + 2.
+// one row per thread.  Key tiles hold 64 keys (32 KB per K or V stage with the
+// hi and lo halves), two stages each, so loads run a tile ahead of the MMAs.
+//
+// A (query tile, head) pair with many key tiles is cut into work items of at most
+// `chunk` key tiles so that the causal triangle spreads evenly over the SMs; every
+// item leaves an un-normalised partial (O, m, l) and gate_merge_kernel combines them.
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O [256,384) Phi [384,448) Plo [448,512).
 #include "ag_common.cuh"
@@ -22,50 +25,85 @@ namespace ag {
 using namespace umma;
 
 constexpr int kGaThreads = 192;
-constexpr int kGaBM = 128, kGaBN = 128, kGaD = 128;
-constexpr int kGaPanel = 128 * 128;                  // [128 rows][64 bf16]
-constexpr int kGaTile = 2 * kGaPanel;                // 32 KB: one of hi / lo
-constexpr int kGaSmemBytes = 6 * kGaTile + 1024 + 256;
+constexpr int kGaBM = 128, kGaBN = 64, kGaD = 128;
+constexpr int kGaPanel = 128 * 128;                  // Q: [128 rows][64 bf16]
+constexpr int kGaTile = 2 * kGaPanel;                // 32 KB: Q hi or Q lo
+constexpr int kGaKvPanel = kGaBN * 128;              // K / V: [64 rows][64 bf16] = 8 KB
+constexpr int kGaKvTile = 2 * kGaKvPanel;            // 16 KB: one of hi / lo
+constexpr int kGaKvStage = 2 * kGaKvTile;            // 32 KB: hi + lo
+constexpr int kGaSmemBytes = 2 * kGaTile + 4 * kGaKvStage + 1024 + 256;   // Q + 2 K stages + 2 V stages
 constexpr uint32_t kGaColS = 0, kGaColO = 256, kGaColPhi = 384, kGaColPlo = 448, kGaTmemCols = 512;
 constexpr float kGaRescaleThreshold = 8.f;
 
 struct GateAttnArgs {
-  float *H;                 // [B * n, GD]
+  float *H;                 // [B * n, GD]                     (merge output)
+  float *part_o;            // [items, 128, 128] un-normalised partial outputs
+  float *part_ml;           // [items, 128, 2]   running max (log2 units) and sum per row
   int n, n_qtiles, gate_heads, problems, GD, causal;
+  int chunk;                // key tiles per work item
+  int items_per_prob;       // work items of one (sequence, head)
   float scale_log2;
 };
 
+// Key tiles query tile qt attends to, and the work items they are cut into.
+// (key tiles hold 64 keys, query tiles 128 queries)
+__host__ __device__ inline int ga_key_tiles(int qt, int n_qtiles, int causal) {
+  return (kGaBM / kGaBN) * (causal ? qt + 1 : n_qtiles);
+}
+__host__ __device__ inline int ga_splits(int qt, int n_qtiles, int causal, int chunk) {
+  return (ga_key_tiles(qt, n_qtiles, causal) + chunk - 1) / chunk;
+}
+// Work item k of a problem -> (query tile, split); items are numbered by ascending query tile.
+__device__ inline void ga_locate(int k, int n_qtiles, int causal, int chunk, int &qt, int &split) {
+  qt = 0;
+  for (;;) {
+    const int ns = ga_splits(qt, n_qtiles, causal, chunk);
+    if (k < ns || qt == n_qtiles - 1) break;
+    k -= ns;
+    ++qt;
+  }
+  split = k;
+}
+
 __global__ void __launch_bounds__(kGaThreads, 1)
 gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_constant__ CUtensorMap tmLo,
+                    const __grid_constant__ CUtensorMap tmHiKv, const __grid_constant__ CUtensorMap tmLoKv,
                     const GateAttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sQ = smem;                    // [hi | lo]
-  uint8_t *sK = sQ + 2 * kGaTile;
-  uint8_t *sV = sK + 2 * kGaTile;
-  uint64_t *bars = reinterpret_cast<uint64_t *>(sV + 2 * kGaTile);
-  uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 2, *v_full = bars + 3, *v_empty = bars + 4;
-  uint64_t *s_full = bars + 5;           // [2]
-  uint64_t *p_ready = bars + 7, *pv_done = bars + 8;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 9);
+  uint8_t *sK = sQ + 2 * kGaTile;        // [stage][hi | lo]
+  uint8_t *sV = sK + 2 * kGaKvStage;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(sV + 2 * kGaKvStage);
+  uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;  // [2]
+  uint64_t *s_full = bars + 9;           // [2]
+  uint64_t *p_ready = bars + 11, *pv_done = bars + 12;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 13);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int qt = a.n_qtiles - 1 - (int)(blockIdx.x / a.problems);
+  // items of the last (longest) query tiles first
   const int prob = blockIdx.x % a.problems;
+  const int item = a.items_per_prob - 1 - (int)(blockIdx.x / a.problems);
+  int qt, split;
+  ga_locate(item, a.n_qtiles, a.causal, a.chunk, qt, split);
   const int b = prob / a.gate_heads, g = prob % a.gate_heads;
   const int j0 = qt * kGaBM;
-  const int n_kv = a.causal ? qt + 1 : a.n_qtiles;
+  const int kv_begin = split * a.chunk;            // first key tile of this item
+  const int n_kv = min(a.chunk, ga_key_tiles(qt, a.n_qtiles, a.causal) - kv_begin);   // tiles of this item
   const int xq = g * kGaD, xk = a.GD + g * kGaD, xv = 2 * a.GD + g * kGaD;   // columns in [Q' | K' | V']
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    mbar_init(k_full, 1); mbar_init(k_empty, 1);
-    mbar_init(v_full, 1); mbar_init(v_empty, 1);
-    mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
+      mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
+      mbar_init(&s_full[s], 1);
+    }
     mbar_init(p_ready, 128);
     mbar_init(pv_done, 1);
     fence_barrier_init();
     prefetch_tensormap(&tmHi); prefetch_tensormap(&tmLo);
+    prefetch_tensormap(&tmHiKv); prefetch_tensormap(&tmLoKv);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, kGaTmemCols);
@@ -78,20 +116,26 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
 
   if (warp == 0) {
     if (lane == 0) {
-      auto load_tile = [&](uint8_t *dst, uint64_t *bar, int x, int y) {
-        mbar_arrive_expect_tx(bar, 2 * kGaTile);
-        tma_load_3d(dst, &tmHi, bar, x, y, b);
-        tma_load_3d(dst + kGaPanel, &tmHi, bar, x + 64, y, b);
-        tma_load_3d(dst + kGaTile, &tmLo, bar, x, y, b);
-        tma_load_3d(dst + kGaTile + kGaPanel, &tmLo, bar, x + 64, y, b);
+      mbar_arrive_expect_tx(q_full, 2 * kGaTile);
+      tma_load_3d(sQ, &tmHi, q_full, xq, j0, b);
+      tma_load_3d(sQ + kGaPanel, &tmHi, q_full, xq + 64, j0, b);
+      tma_load_3d(sQ + kGaTile, &tmLo, q_full, xq, j0, b);
+      tma_load_3d(sQ + kGaTile + kGaPanel, &tmLo, q_full, xq + 64, j0, b);
+      auto load_kv = [&](uint8_t *dst, uint64_t *bar, int x, int y) {
+        mbar_arrive_expect_tx(bar, kGaKvStage);
+        tma_load_3d(dst, &tmHiKv, bar, x, y, b);
+        tma_load_3d(dst + kGaKvPanel, &tmHiKv, bar, x + 64, y, b);
+        tma_load_3d(dst + kGaKvTile, &tmLoKv, bar, x, y, b);
+        tma_load_3d(dst + kGaKvTile + kGaKvPanel, &tmLoKv, bar, x + 64, y, b);
       };
-      load_tile(sQ, q_full, xq, j0);
       for (int i = 0; i < n_kv; ++i) {
-        const uint32_t ph = i & 1;
-        if (!mbar_wait(k_empty, ph ^ 1)) break;
-        load_tile(sK, k_full, xk, i * kGaBN);
-        if (!mbar_wait(v_empty, ph ^ 1)) break;
-        load_tile(sV, v_full, xv, i * kGaBN);
+        const int st = i & 1;
+        const uint32_t ph = (i >> 1) & 1;
+        const int y = (kv_begin + i) * kGaBN;
+        if (!mbar_wait(&k_empty[st], ph ^ 1)) break;
+        load_kv(sK + st * kGaKvStage, &k_full[st], xk, y);
+        if (!mbar_wait(&v_empty[st], ph ^ 1)) break;
+        load_kv(sV + st * kGaKvStage, &v_full[st], xv, y);
       }
     }
   } else if (warp == 1) {
@@ -99,27 +143,28 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
     constexpr uint32_t idesc_qk = idesc_bf16_f32(kGaBM, kGaBN, false, false);
     constexpr uint32_t idesc_pv = idesc_bf16_f32(kGaBM, kGaD, false, true);
     const uint64_t dq = desc_kmajor_sw128(smem_u32(sQ)), dk = desc_kmajor_sw128(smem_u32(sK));
-    const uint64_t dv = desc_mnmajor_sw128(smem_u32(sV), kGaPanel);
+    const uint64_t dv = desc_mnmajor_sw128(smem_u32(sV), kGaKvPanel);
     const uint32_t q_lo = (uint32_t)dq, q_hi = (uint32_t)(dq >> 32);
     const uint32_t k_lo = (uint32_t)dk, k_hi = (uint32_t)(dk >> 32);
     const uint32_t v_lo = (uint32_t)dv, v_hi = (uint32_t)(dv >> 32);
     auto issue_qk = [&](int i) -> bool {
-      if (!mbar_wait(k_full, i & 1)) return false;
+      const int st = i & 1;
+      if (!mbar_wait(&k_full[st], (i >> 1) & 1)) return false;
       tc_fence_after_sync();
-      const uint32_t d = tmem + kGaColS + (i & 1) * 128;
+      const uint32_t d = tmem + kGaColS + st * 128;
+      const uint32_t kb = k_lo + ((st * kGaKvStage) >> 4);
       if (elect_one()) {
         // Qhi Khi + Qhi Klo + Qlo Khi
 #pragma unroll
         for (int t = 0; t < 3; ++t) {
-          const uint32_t qa = q_lo + ((t == 2 ? kGaTile : 0) >> 4), ka = k_lo + ((t == 1 ? kGaTile : 0) >> 4);
+          const uint32_t qa = q_lo + ((t == 2 ? kGaTile : 0) >> 4), ka = kb + ((t == 1 ? kGaKvTile : 0) >> 4);
 #pragma unroll
-          for (int k = 0; k < kGaD / 16; ++k) {
-            const uint32_t off = ((k >> 2) * kGaPanel + (k & 3) * 32) >> 4;
-            mma_ss_lohi(d, qa + off, q_hi, ka + off, k_hi, idesc_qk, (t | k) != 0);
-          }
+          for (int k = 0; k < kGaD / 16; ++k)
+            mma_ss_lohi(d, qa + (((k >> 2) * kGaPanel + (k & 3) * 32) >> 4), q_hi,
+                        ka + (((k >> 2) * kGaKvPanel + (k & 3) * 32) >> 4), k_hi, idesc_qk, (t | k) != 0);
         }
-        mma_commit(k_empty);
-        mma_commit(&s_full[i & 1]);
+        mma_commit(&k_empty[st]);
+        mma_commit(&s_full[st]);
       }
       __syncwarp();
       return true;
@@ -129,19 +174,21 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
     for (int i = 0; i < n_kv && ok; ++i) {
       if (i + 1 < n_kv) ok = issue_qk(i + 1);
       if (!ok) break;
+      const int st = i & 1;
       if (!mbar_wait(p_ready, i & 1)) { ok = false; break; }
-      if (!mbar_wait(v_full, i & 1)) { ok = false; break; }
+      if (!mbar_wait(&v_full[st], (i >> 1) & 1)) { ok = false; break; }
       tc_fence_after_sync();
+      const uint32_t vb = v_lo + ((st * kGaKvStage) >> 4);
       if (elect_one()) {
         // Phi Vhi + Phi Vlo + Plo Vhi
 #pragma unroll
         for (int t = 0; t < 3; ++t) {
-          const uint32_t pa = tmem + (t == 2 ? kGaColPlo : kGaColPhi), va = v_lo + ((t == 1 ? kGaTile : 0) >> 4);
+          const uint32_t pa = tmem + (t == 2 ? kGaColPlo : kGaColPhi), va = vb + ((t == 1 ? kGaKvTile : 0) >> 4);
 #pragma unroll
           for (int k = 0; k < kGaBN / 16; ++k)
             mma_ts_lohi(tmem + kGaColO, pa + k * 8, va + ((k * 2048) >> 4), v_hi, idesc_pv, (i | t | k) != 0);
         }
-        mma_commit(v_empty);
+        mma_commit(&v_empty[st]);
         mma_commit(pv_done);
       }
       __syncwarp();
@@ -162,27 +209,28 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t tS = tm_lane + kGaColS + (i & 1) * 128;
-      const int nvalid = min(max(bound - i * kGaBN, 0), kGaBN);
+      const int nvalid = min(max(bound - (kv_begin + i) * kGaBN, 0), kGaBN);
       const bool full = nvalid >= kGaBN;
 
-      uint32_t r[128];
-      tmem_ld_x128_sync(tS, r);
+      uint32_t r[kGaBN];
+      tmem_ld_x64_sync(tS, r);
       if (!full) {
 #pragma unroll
-        for (int e = 0; e < 128; ++e)
+        for (int e = 0; e < kGaBN; ++e)
           if (e >= nvalid) r[e] = 0xff800000u;        // -inf: weight 0 below
       }
       float mx[8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) mx[q] = __uint_as_float(r[q]);
 #pragma unroll
-      for (int e = 8; e < 128; e += 8)
+      for (int e = 8; e < kGaBN; e += 8)
 #pragma unroll
         for (int q = 0; q < 8; ++q) mx[q] = fmaxf(mx[q], __uint_as_float(r[e + q]));
       float tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
                          fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
       tmax *= a.scale_log2;
-      // tile 0 always holds key 0, visible to every row, so m is finite from here on
+      // the first tile of an item always holds a key visible to every row (key 0, or a tile
+      // wholly before the query tile), so m is finite from here on
       float m_new;
       if (i == 0) m_new = tmax;
       else m_new = (tmax > m + kGaRescaleThreshold) ? tmax : m;
@@ -208,7 +256,7 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
 
       float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
+      for (int c = 0; c < kGaBN / 16; ++c) {
         uint32_t ph[8], pl[8];
 #pragma unroll
         for (int e = 0; e < 16; e += 2) {
@@ -237,8 +285,8 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
       tc_fence_after_sync();
     }
     if (ok) {
-      const float inv = 1.f / l;
-      float *hp = a.H + ((size_t)b * a.n + jc) * a.GD + g * kGaD;
+      const size_t it = (size_t)prob * a.items_per_prob + item;
+      float *op = a.part_o + (it * kGaBM + row) * kGaD;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         uint32_t r[32];
@@ -246,11 +294,10 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
         if (valid) {
 #pragma unroll
           for (int e = 0; e < 32; e += 4)
-            *reinterpret_cast<float4 *>(hp + c * 32 + e) =
-                make_float4(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv,
-                            __uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+            *reinterpret_cast<uint4 *>(op + c * 32 + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
         }
       }
+      if (valid) *reinterpret_cast<float2 *>(a.part_ml + (it * kGaBM + row) * 2) = make_float2(m, l);
     }
   }
   tc_fence_before_sync();
@@ -263,21 +310,91 @@ bool gate_attn_tc_supported(const ag_layer_desc &d) {
   return d.dtype == AG_BF16 && d.gate_head_dim == 128 && gate_proj_tc_supported(d.hidden, GD);
 }
 
+// H'[t, g * 128 + c] = sum_s w_s O_s[r, c] / sum_s w_s l_s with w_s = 2^(m_s - max_s m_s): the
+// split-K merge of an online softmax.  One warp per query row (8 rows per CTA), a lane per
+// four columns: every access of a warp is one 512-byte row.
+constexpr int kMergeRows = 8;
+__global__ void __launch_bounds__(kMergeRows * 32)
+gate_merge_kernel(const GateAttnArgs a) {
+  constexpr int kBlocksPerTile = kGaBM / kMergeRows;
+  const int tile = blockIdx.x / kBlocksPerTile;                    // (problem, query tile)
+  const int prob = tile / a.n_qtiles, qt = tile % a.n_qtiles;
+  const int b = prob / a.gate_heads, g = prob % a.gate_heads;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = (blockIdx.x % kBlocksPerTile) * kMergeRows + warp;
+  const int t = qt * kGaBM + r;
+  if (t >= a.n) return;
+  int first = 0;
+  for (int q = 0; q < qt; ++q) first += ga_splits(q, a.n_qtiles, a.causal, a.chunk);
+  const int ns = ga_splits(qt, a.n_qtiles, a.causal, a.chunk);
+  const size_t row0 = ((size_t)prob * a.items_per_prob + first) * kGaBM + r;   // + s * 128 per split
+  float mmax = -INFINITY;
+  for (int s = lane; s < ns; s += 32) mmax = fmaxf(mmax, a.part_ml[(row0 + (size_t)s * kGaBM) * 2]);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float lsum = 0.f;
+#pragma unroll 4
+  for (int s = 0; s < ns; ++s) {
+    const float2 ml = *reinterpret_cast<const float2 *>(a.part_ml + (row0 + (size_t)s * kGaBM) * 2);
+    const float4 o = *reinterpret_cast<const float4 *>(a.part_o + (row0 + (size_t)s * kGaBM) * kGaD + lane * 4);
+    const float w = fast_exp2(ml.x - mmax);
+    acc.x = fmaf(w, o.x, acc.x); acc.y = fmaf(w, o.y, acc.y);
+    acc.z = fmaf(w, o.z, acc.z); acc.w = fmaf(w, o.w, acc.w);
+    lsum = fmaf(w, ml.y, lsum);
+  }
+  const float inv = 1.f / lsum;
+  *reinterpret_cast<float4 *>(a.H + ((size_t)b * a.n + t) * a.GD + g * kGaD + lane * 4) =
+      make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+}
+
+// Key tiles per work item: small enough for about three waves of items over the SMs.
+static void gate_attn_plan(const ag_layer_desc &d, int &chunk, int &items_per_prob) {
+  const int nq = (d.seq + kGaBM - 1) / kGaBM, problems = d.batch * d.gate_heads;
+  long long tiles = 0;
+  for (int q = 0; q < nq; ++q) tiles += ga_key_tiles(q, nq, d.gate_causal);
+  tiles *= problems;
+  chunk = (int)((tiles + 3 * 148 - 1) / (3 * 148));
+  // even, so that an item starts on a 128-key boundary: its first tile then holds a key every
+  // row of the query tile may see (the kernel seeds the running maximum from it)
+  chunk = (chunk + 1) & ~1;
+  chunk = chunk < 2 ? 2 : (chunk > 32 ? 32 : chunk);
+  items_per_prob = 0;
+  for (int q = 0; q < nq; ++q) items_per_prob += ga_splits(q, nq, d.gate_causal, chunk);
+}
+
+size_t gate_attn_partial_bytes(const ag_layer_desc &d) {
+  int chunk, ipp;
+  gate_attn_plan(d, chunk, ipp);
+  const size_t items = (size_t)d.batch * d.gate_heads * ipp;
+  return align_up(items * kGaBM * kGaD * sizeof(float), 256) + align_up(items * kGaBM * 2 * sizeof(float), 256);
+}
+
 int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *qkv_lo, float *hcat,
-                        cudaStream_t st) {
+                        void *partials, cudaStream_t st) {
   const int GD = d.gate_heads * d.gate_head_dim;
   CUtensorMap tmHi, tmLo;
   int rc = make_tmap_3d_bf16(&tmHi, qkv_hi, d.batch, d.seq, 3 * GD, kGaBM, 64);
   if (rc) return rc;
   rc = make_tmap_3d_bf16(&tmLo, qkv_lo, d.batch, d.seq, 3 * GD, kGaBM, 64);
   if (rc) return rc;
+  CUtensorMap tmHiKv, tmLoKv;
+  if ((rc = make_tmap_3d_bf16(&tmHiKv, qkv_hi, d.batch, d.seq, 3 * GD, kGaBN, 64))) return rc;
+  if ((rc = make_tmap_3d_bf16(&tmLoKv, qkv_lo, d.batch, d.seq, 3 * GD, kGaBN, 64))) return rc;
   GateAttnArgs a;
   a.H = hcat;
   a.n = d.seq; a.n_qtiles = (d.seq + kGaBM - 1) / kGaBM;
   a.gate_heads = d.gate_heads; a.problems = d.batch * d.gate_heads; a.GD = GD; a.causal = d.gate_causal;
+  gate_attn_plan(d, a.chunk, a.items_per_prob);
+  const size_t items = (size_t)a.problems * a.items_per_prob;
+  a.part_o = static_cast<float *>(partials);
+  a.part_ml = reinterpret_cast<float *>(static_cast<char *>(partials) +
+                                        align_up(items * kGaBM * kGaD * sizeof(float), 256));
   a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kGaD));
   AG_CUDA_TRY(cudaFuncSetAttribute(gate_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGaSmemBytes));
-  gate_attn_tc_kernel<<<a.n_qtiles * a.problems, kGaThreads, kGaSmemBytes, st>>>(tmHi, tmLo, a);
+  gate_attn_tc_kernel<<<(unsigned)items, kGaThreads, kGaSmemBytes, st>>>(tmHi, tmLo, tmHiKv, tmLoKv, a);
+  AG_LAUNCH_CHECK();
+  gate_merge_kernel<<<a.problems * a.n_qtiles * (kGaBM / kMergeRows), kMergeRows * 32, 0, st>>>(a);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
