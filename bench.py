@@ -34,10 +34,11 @@ WORKLOADS = {
     "prefill7b": (inputs.PREFILL7B, 16, "Llama-2-7B-shaped AG-gated layer, batch 1 x seq 4096, keep rates U[0.3,0.8] per head"),
     "tiny": (inputs.TINY, 16, "fp32 correctness layer, batch 1 x seq 128, ~50% keep"),
     "deep_layer": (inputs.DEEP_LAYER, 16, "deep-layer pattern, batch 1 x seq 16384: 24 heads keep ~10%, 8 heads keep nothing"),
+    "stack7b": (inputs.STACK7B, 16, "32 AG-gated layers back to back, batch 8 x seq 4096; per-layer mean eviction rising from 10% to 90%"),
     "decode_ragged": (inputs.DECODE_RAGGED, 16, "ragged decode, batch 32 x 32 heads, retained lengths U[0.2,0.9] x 8192, keep-new Bernoulli(0.5)"),
 }
 # kernels launched per call of the library
-LAUNCHES = {"gate": 3, "compact": 2, "prefill": 1, "decode": 2, "append": 1}
+LAUNCHES = {"gate": 4, "compact": 2, "prefill": 1, "decode": 2, "append": 1}
 
 
 def _peaks():
@@ -49,48 +50,86 @@ def _peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """SM clock and throttle reasons sampled through NVML (read-only) every few milliseconds
+    while the timed region runs; falls back to polling nvidia-smi when NVML is not importable."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, gpu_index):
-        self.gpu, self.proc, self.path = gpu_index, None, None
+        import threading
+        self.gpu, self.samples, self.stop_flag = gpu_index, [], threading.Event()
+        self.thread, self.max_mhz, self.proc, self.path = None, None, None, None
+
+    def _nvml_index(self):
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+        if vis:
+            ids = [v.strip() for v in vis.split(",") if v.strip()]
+            if self.gpu < len(ids) and ids[self.gpu].isdigit():
+                return int(ids[self.gpu])
+        return self.gpu
 
     def start(self):
+        import threading
         try:
-            fd, self.path = tempfile.mkstemp(suffix=".csv")
-            os.close(fd)
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
-                 "-i", str(self.gpu)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            import pynvml
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(self._nvml_index())
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+
+            def loop():
+                while not self.stop_flag.is_set():
+                    try:
+                        self.samples.append((float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)),
+                                             int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)),
+                                             pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0))
+                    except Exception:
+                        pass
+                    time.sleep(0.004)
+            self.thread = threading.Thread(target=loop, daemon=True)
+            self.thread.start()
         except Exception:
-            self.proc = None
+            self.thread = None
+            try:
+                fd, self.path = tempfile.mkstemp(suffix=".csv")
+                os.close(fd)
+                q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active"
+                self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits",
+                                              "-lms", "20", "-i", str(self._nvml_index())],
+                                             stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            except Exception:
+                self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
-        if self.proc is None:
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        if self.thread is not None:
+            self.stop_flag.set()
+            self.thread.join(timeout=2)
+            if self.samples:
+                sm = np.asarray([x[0] for x in self.samples])
+                pw = np.asarray([x[2] for x in self.samples])
+                busy = sm[pw >= 0.5 * pw.max()] if pw.max() > 0 else sm
+                bits = 0
+                for x in self.samples:
+                    bits |= x[1]
+                out.update(sm_mhz=float(np.median(busy)), samples=len(self.samples), power_w_max=float(pw.max()),
+                           reasons=[n for b, n in self.REASONS.items() if bits & b])
             return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        rows = [r.split(",") for r in open(self.path).read().strip().splitlines() if r.count(",") >= 8]
-        os.unlink(self.path)
-        if not rows:
-            return out
-        try:
-            sm = np.asarray([float(r[1]) for r in rows])
-            power = np.asarray([float(r[3]) for r in rows])
-            busy = sm[power >= 0.5 * power.max()] if power.max() > 0 else sm
-            out["sm_mhz"] = float(np.median(busy))
-            out["sm_max_mhz"] = float(rows[0][2])
-            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-            out["reasons"] = [n for k, n in enumerate(names) if any("Active" in r[5 + k] and "Not" not in r[5 + k] for r in rows)]
-            out["samples"] = len(rows)
-        except Exception:
-            pass
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+            rows = [r.split(",") for r in open(self.path).read().strip().splitlines() if r.count(",") >= 3]
+            os.unlink(self.path)
+            try:
+                sm = np.asarray([float(r[0]) for r in rows])
+                bits = 0
+                for r in rows:
+                    bits |= int(r[3].strip(), 16)
+                out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(rows[0][1]), samples=len(rows),
+                           reasons=[n for b, n in self.REASONS.items() if bits & b])
+            except Exception:
+                pass
         return out
 
 
@@ -110,7 +149,8 @@ class LayerRun:
         B, h, n, D = sh.batch, sh.heads, sh.seq, sh.head_dim
         self.name = name
         self.use_graph, self.graph = True, None
-        self.has_gate = name in ("prefill7b", "tiny")
+        self.has_gate = name in ("prefill7b", "tiny", "stack7b")
+        self.layers = 32 if name == "stack7b" else 1
         self.has_prefill = name != "decode_ragged"
         if self.has_gate:
             self.X = inputs.hidden_states(sh, seed, dev)
@@ -149,8 +189,15 @@ class LayerRun:
         self.gamma = None
         if self.has_gate:
             self.gate()
-            keep = inputs.keep_targets_uniform(h, seed + 20) if name != "tiny" else [0.5] * h
-            self.gamma = inputs.calibrate_gamma(self.scores, keep, sh.tau).to(dev)
+            if name == "stack7b":
+                # the layers share X and the weights (inputs, not the timed work); what differs per
+                # layer is the keep rate, i.e. gamma: mean eviction 10 % (first) ... 90 % (last)
+                self.gammas = [inputs.calibrate_gamma(self.scores, inputs.keep_targets_layer(h, seed + 20, l), sh.tau).to(dev)
+                               for l in range(self.layers)]
+            else:
+                keep = inputs.keep_targets_uniform(h, seed + 20) if name != "tiny" else [0.5] * h
+                self.gammas = [inputs.calibrate_gamma(self.scores, keep, sh.tau).to(dev)]
+            self.gamma = self.gammas[0]
         elif self.has_prefill:
             f, empty = inputs.deep_layer_flags(sh, seed + 20)
             self.flags.copy_(f.to(dev))
@@ -188,14 +235,16 @@ class LayerRun:
             fn(*a)
             e.record()
             ev[key].append((s, e))
-        if self.has_gate:
-            timed("gate", self.gate)
-        if self.has_prefill:
-            timed("compact", self.compact)
-            timed("prefill", self.prefill)
-        else:
-            self.cache.len.copy_(self.len0)      # every pass starts from the same cache
-        timed("decode", self.decode_all)
+        for layer in range(self.layers):
+            if self.has_gate:
+                self.gamma = self.gammas[layer]
+                timed("gate", self.gate)
+            if self.has_prefill:
+                timed("compact", self.compact)
+                timed("prefill", self.prefill)
+            else:
+                self.cache.len.copy_(self.len0)      # every pass starts from the same cache
+            timed("decode", self.decode_all)
 
     def decode_all(self):
         """All decode steps of a pass.  They are dozens of small launches, so they are
@@ -219,27 +268,37 @@ class LayerRun:
         self.graph.replay()
 
     def tokens_per_step(self):
-        return self.shape.batch * ((self.shape.seq if self.has_prefill else 0) + self.decode_steps)
+        return self.shape.batch * ((self.shape.seq if self.has_prefill else 0) + self.decode_steps) * self.layers
 
     def launches_per_step(self):
-        return ((LAUNCHES["gate"] if self.has_gate else 0) +
-                (LAUNCHES["compact"] + LAUNCHES["prefill"] if self.has_prefill else 0) +
-                self.decode_steps * (LAUNCHES["decode"] + LAUNCHES["append"]))
+        return self.layers * ((LAUNCHES["gate"] if self.has_gate else 0) +
+                              (LAUNCHES["compact"] + LAUNCHES["prefill"] if self.has_prefill else 0) +
+                              self.decode_steps * (LAUNCHES["decode"] + LAUNCHES["append"]))
 
-    def decode_bytes_per_decode_step(self):
-        """Bytes one decode step must move: every valid cache row once (K and V) plus
-        q, k_new, v_new, o.  Lengths grow linearly over the pass, so the mean of the
-        lengths before the first and after the last step is the per-step average."""
+    def work_per_call(self):
+        """Algorithmic work of one call, averaged over the layers of a pass (untimed extra pass):
+        effective prefill FLOPs 4 D sum_j (1 + P[j]) (QK^T and PV over visible (query, key) pairs
+        only), retained rows, and the bytes one decode step must move (every valid cache row once,
+        K and V, plus q, k_new, v_new, o; lengths grow linearly over the decode steps)."""
         e = 2 if self.shape.dtype == "bf16" else 4
-        D = self.shape.head_dim
-        before = (self.prefix[:, :, -1] if self.has_prefill else self.len0).to(torch.float64).sum().item()
-        after = self.cache.len.to(torch.float64).sum().item()
-        return 2.0 * 0.5 * (before + after) * D * e + 4.0 * self.shape.batch * self.shape.heads * D * e
-
-    def effective_prefill_flops(self):
-        """4 D sum_j (1 + P[j]): QK^T and PV over the visible (query, key) pairs only."""
-        P = self.prefix[:, :, :-1].to(torch.float64)
-        return float(4.0 * self.shape.head_dim * (P.sum() + P.numel()))
+        D, slabs = self.shape.head_dim, self.shape.batch * self.shape.heads
+        appended = float(sum(q[3].to(torch.float64).sum().item() for q in self.dq))
+        f_eff, kept = [], []
+        for layer in range(self.layers):
+            if self.has_gate:
+                self.gamma = self.gammas[layer]
+                self.gate()
+            if self.has_prefill:
+                self.compact()
+                P = self.prefix[:, :, :-1].to(torch.float64)
+                f_eff.append(float(4.0 * D * (P.sum() + P.numel())))
+                kept.append(float(self.prefix[:, :, -1].to(torch.float64).sum().item()))
+            else:
+                kept.append(float(self.len0.to(torch.float64).sum().item()))
+        mean_kept = float(np.mean(kept))
+        mean_len = mean_kept + appended * (self.decode_steps - 1) / (2.0 * self.decode_steps)
+        return {"prefill_flops": float(np.mean(f_eff)) if f_eff else 0.0, "kept_rows": mean_kept,
+                "decode_bytes": 2.0 * mean_len * D * e + 4.0 * slabs * D * e}
 
     def gate_flops(self):
         sh = self.shape
@@ -332,7 +391,8 @@ def run_ours(args, rank, world, dev):
     tokens = run.tokens_per_step() * world
     peaks = _peaks()
     rooflines = {}
-    dec_bytes = run.decode_bytes_per_decode_step()
+    work = run.work_per_call()
+    dec_bytes = work["decode_bytes"]
     dec_ms = per_call_ms["decode"] / run.decode_steps
     dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
     rooflines["decode"] = {"bound": "hbm", "kernel": "ag_decode_attn + ag_cache_append", "achieved": dec_gbs,
@@ -340,14 +400,14 @@ def run_ours(args, rank, world, dev):
                            "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": dec_bytes,
                            "ms": dec_ms}
     if run.has_prefill:
-        f_eff = run.effective_prefill_flops()
+        f_eff = work["prefill_flops"]
         tf = f_eff / (per_call_ms["prefill"] * 1e-3) / 1e12
         rooflines["prefill"] = {"bound": "tensor", "kernel": "ag_prefill_attn", "achieved": tf,
                                 "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
                                 "traffic": None, "peak_source": peaks["source"], "algorithmic_flops": f_eff,
                                 "ms": per_call_ms["prefill"]}
         e = 2 if sh.dtype == "bf16" else 4
-        kept = float(run.prefix[:, :, -1].to(torch.float64).sum().item())
+        kept = work["kept_rows"]
         cb = 2.0 * (2.0 * kept * sh.head_dim * e) + sh.batch * sh.heads * sh.seq * 9.0
         gbs = cb / (per_call_ms["compact"] * 1e-3) / 1e9
         rooflines["compact"] = {"bound": "hbm", "kernel": "ag_compact_kv", "achieved": gbs, "peak": peaks["hbm_gbs"],
@@ -467,7 +527,7 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="prefill7b", choices=list(WORKLOADS))
@@ -500,7 +560,7 @@ def main():
     if rank == 0:
         out, run = res
         if not args.no_cpu_baseline and world == 1 and args.workload in ("prefill7b", "tiny"):
-            cb = oracle_sample(args.workload, 2000)
+            cb = oracle_sample(args.workload, 2000, n_heads_sample=WORKLOADS[args.workload][0].heads, decode_steps=16)
             cb.pop("est_step_s", None)
             out["cpu_baseline"] = cb
         print(json.dumps(out))
