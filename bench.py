@@ -308,6 +308,20 @@ class LayerRun:
                 + 2.0 * rows * GD * sh.heads)
 
 
+def max_over_ranks(values, dist, device):
+    """Replicas share nothing on the data path; the only exchange of a multi-GPU run is this
+    max-reduction of the per-rank timings (the job is as slow as its slowest rank)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def aggregate_value(tokens_per_rank_step, world, steps, total_ms):
+    """Whole-job tokens/s of `world` weak-scaled replicas timed as max over ranks."""
+    return tokens_per_rank_step * world * steps / (total_ms * 1e-3)
+
+
 def flush_l2(buf):
     buf.zero_()
 
@@ -382,10 +396,7 @@ def run_ours(args, rank, world, dev):
         t_e2e += s.elapsed_time(e)
     barrier()
 
-    times = torch.tensor([total_ms, t_e2e], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, t_e2e = times.tolist()
+    total_ms, t_e2e = max_over_ranks([total_ms, t_e2e], dist, dev)
     if rank != 0:
         return None
     tokens = run.tokens_per_step() * world
@@ -422,7 +433,7 @@ def run_ours(args, rank, world, dev):
     head = "prefill" if run.has_prefill else "decode"
     ms_step = total_ms / args.steps
     out = {
-        "metric": METRIC, "value": tokens * args.steps / (total_ms * 1e-3), "unit": UNIT,
+        "metric": METRIC, "value": aggregate_value(run.tokens_per_step(), world, args.steps, total_ms), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if sh.dtype == "bf16" else "f32", "data": "synthetic",
