@@ -37,6 +37,13 @@ WORKLOADS = {
     "stack7b": (inputs.STACK7B, 16, "32 AG-gated layers back to back, batch 8 x seq 4096; per-layer mean eviction rising from 10% to 90%"),
     "decode_ragged": (inputs.DECODE_RAGGED, 16, "ragged decode, batch 32 x 32 heads, retained lengths U[0.2,0.9] x 8192, keep-new Bernoulli(0.5)"),
 }
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (None for workloads that were not captured).  To be reset to
+# None whenever the kernel changes after the capture.
+TRAFFIC = {
+    ("prefill7b", "prefill"): 155.06e6 + 17.77e6,        # prefill_tc_kernel<64>
+    ("decode_ragged", "decode"): 2.3529e9 + 6.9e6,       # decode_partial_kernel<bf16,128>
+}
 # kernels launched per call of the library
 LAUNCHES = {"gate": 4, "compact": 2, "prefill": 1, "decode": 2, "append": 1}
 
@@ -430,6 +437,8 @@ def run_ours(args, rank, world, dev):
         rooflines["gate"] = {"bound": "tensor", "kernel": "ag_gate_forward", "achieved": tf, "peak": peaks["bf16_tflops"],
                              "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "traffic": None,
                              "peak_source": peaks["source"], "algorithmic_flops": gf, "ms": per_call_ms["gate"]}
+    for k, r in rooflines.items():
+        r["traffic"] = TRAFFIC.get((args.workload, k))
     head = "prefill" if run.has_prefill else "decode"
     ms_step = total_ms / args.steps
     out = {
