@@ -38,7 +38,6 @@ template <int BN> struct PfCfg {
   static constexpr int kKvPanel = BN * 128;           // [BN rows][64 bf16]
   static constexpr int kKvTile = 2 * kKvPanel;
   static constexpr int kKvBuf = 2 * kKvTile;          // two stages; >= one 32 KB dense tile
-  static constexpr int kSelfStages = 128 / BN;        // K stages the 128-row self tile covers
   static constexpr int kSmemBytes = kPfTile + 2 * kKvBuf + 1024 + 256;
   static constexpr uint32_t kColO = 2 * BN, kTmemCols = BN == 64 ? 256 : 512;
   static constexpr int kCtasPerSm = BN == 64 ? 2 : 1;
@@ -86,8 +85,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   uint64_t *q_full = bars;
   uint64_t *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;   // [2] each
   uint64_t *s_full = bars + 9;                     // [2]
-  uint64_t *p_ready = bars + 11, *pv_done = bars + 12;   // pv_done[2]: even / odd cache tiles
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 14);
+  // p_ready[2], pv_done[2]: even / odd cache tiles.  Two p_ready barriers because a softmax warp
+  // may finish tile i + 1 before a slower one has finished tile i; it cannot get further ahead,
+  // since S of tile i + 2 waits for the P V of tile i.
+  uint64_t *p_ready = bars + 11, *pv_done = bars + 13, *self_full = bars + 15;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 16);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // heaviest query tiles first
@@ -98,12 +100,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int32_t *pre = a.prefix + (size_t)slab * (a.n + 1);
   const int max_bound = pre[j_last];               // keys any row of this tile may see
   const int n_kv = (max_bound + kPfBN - 1) / kPfBN;
-  const int n_self = n_kv > 0 ? 1 : 0;             // a lone diagonal needs no score
   const int row0 = (int)a.row_off[slab];
-  // uses of K stage 0 / 1 before the dense V tile: self tile (stage 0, and stage 1 when the
-  // 128-row tile spans both) + even / odd cache tiles
-  const int self1 = Cfg::kSelfStages == 2 ? n_self : 0;
-  const int k0_uses = n_self + (n_kv + 1) / 2, k1_uses = self1 + n_kv / 2;
+  static_assert(BN == 64, "the self tile below spans exactly the two V stages");
+  // uses of K stage 0 / 1 before the dense V tile: even / odd cache tiles
+  const int k0_uses = (n_kv + 1) / 2, k1_uses = n_kv / 2;
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
@@ -112,8 +112,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
       mbar_init(&s_full[s], 1);
     }
-    mbar_init(p_ready, 128);
+    mbar_init(&p_ready[0], 128); mbar_init(&p_ready[1], 128);
     mbar_init(&pv_done[0], 1); mbar_init(&pv_done[1], 1);
+    mbar_init(self_full, 1);
     fence_barrier_init();
     prefetch_tensormap(&tmQ); prefetch_tensormap(&tmKd); prefetch_tensormap(&tmVd);
     prefetch_tensormap(&tmK); prefetch_tensormap(&tmV); prefetch_tensormap(&tmO);
@@ -135,21 +136,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mbar_arrive_expect_tx(q_full, kPfTile);
         tma_load_3d(sQ, &tmQ, q_full, 0, j0, slab);
         tma_load_3d(sQ + kPfPanel, &tmQ, q_full, 64, j0, slab);
-        // self tile: dense K rows j0 .. j0 + 127 across both K stages (fresh: no wait)
-        mbar_arrive_expect_tx(&k_full[0], kPfTile);
-        tma_load_3d(sK, &tmKd, &k_full[0], 0, j0, slab);
-        tma_load_3d(sK + kPfPanel, &tmKd, &k_full[0], 64, j0, slab);
+        // self tile: dense K rows j0 .. j0 + 127 across both V stages, which no P V needs before
+        // the first softmax is done; the first cache tiles of K load alongside it
+        mbar_arrive_expect_tx(&v_full[0], kPfTile);
+        tma_load_3d(sV, &tmKd, &v_full[0], 0, j0, slab);
+        tma_load_3d(sV + kPfPanel, &tmKd, &v_full[0], 64, j0, slab);
         for (int i = 0; i < n_kv && ok; ++i) {
           const int st = i & 1;
           const int y = row0 + i * kPfBN;
-          // uses of this K stage so far: the self tile (where it covers the stage) + earlier tiles
-          const int k_used = (st == 0 ? n_self : self1) + (i >> 1);
-          ok = mbar_wait(&k_empty[st], (k_used & 1) ^ 1);
+          ok = mbar_wait(&k_empty[st], ((i >> 1) & 1) ^ 1);     // earlier uses of the stage: i >> 1
           if (!ok) break;
           mbar_arrive_expect_tx(&k_full[st], kPfKvTile);
           tma_load_2d(sK + st * kPfKvTile, &tmK, &k_full[st], 0, y);
           tma_load_2d(sK + st * kPfKvTile + kPfKvPanel, &tmK, &k_full[st], 64, y);
-          ok = mbar_wait(&v_empty[st], ((i >> 1) & 1) ^ 1);
+          ok = mbar_wait(&v_empty[st], (i >> 1) & 1);           // the self tile + i >> 1 earlier tiles
           if (!ok) break;
           mbar_arrive_expect_tx(&v_full[st], kPfKvTile);
           tma_load_2d(sV + st * kPfKvTile, &tmV, &v_full[st], 0, y);
@@ -158,7 +158,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       }
       // dense V rows for the self term of the output, into the K buffer once both stages are free
       if (ok && k0_uses > 0) ok = mbar_wait(&k_empty[0], (k0_uses & 1) ^ 1);
-      if (ok && Cfg::kSelfStages == 2 && k1_uses > 0) ok = mbar_wait(&k_empty[1], (k1_uses & 1) ^ 1);
+      if (ok && k1_uses > 0) ok = mbar_wait(&k_empty[1], (k1_uses & 1) ^ 1);
       if (ok) {
         mbar_arrive_expect_tx(&k_full[0], kPfTile);
         tma_load_3d(sK, &tmVd, &k_full[0], 0, j0, slab);
@@ -173,6 +173,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       // descriptors as (low, high) words: the high words are fixed per operand kind, the low
       // words are a base plus a compile-time offset per K step
       const uint64_t dq = desc_kmajor_sw128(smem_u32(sQ)), dk = desc_kmajor_sw128(smem_u32(sK));
+      const uint64_t dself = desc_kmajor_sw128(smem_u32(sV));
       const uint64_t dv = desc_mnmajor_sw128(smem_u32(sV), kPfKvPanel);
       const uint32_t q_lo = (uint32_t)dq, q_hi = (uint32_t)(dq >> 32);
       const uint32_t k_lo = (uint32_t)dk, k_hi = (uint32_t)(dk >> 32);
@@ -182,7 +183,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       auto tile_keys = [&](int i) { return min(kPfBN, (max_bound - i * kPfBN + 15) & ~15); };
       auto issue_qk = [&](int i) -> bool {
         const int st = i & 1;
-        if (!mbar_wait(&k_full[st], ((i >> 1) + (st == 0 ? 1 : 0)) & 1)) return false;
+        if (!mbar_wait(&k_full[st], (i >> 1) & 1)) return false;
         tc_fence_after_sync();
         const uint32_t idesc_qk = idesc_bf16_f32(kPfBM, tile_keys(i), false, false);
         const uint32_t kb = k_lo + ((st * kPfKvTile) >> 4);
@@ -199,23 +200,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         return true;
       };
       bool ok = mbar_wait(q_full, 0);
-      // self tile: 128 dense K rows, S over both buffers
-      ok = ok && mbar_wait(&k_full[0], 0);
+      // self tile: 128 dense K rows (in the V stages); its scores land in the columns of O,
+      // which are free until the first P V - that one starts a fresh accumulation, and it cannot
+      // be issued before the softmax threads, who read the diagonal first, are done with tile 0
+      ok = ok && mbar_wait(&v_full[0], 0);
       if (ok) {
         tc_fence_after_sync();
         constexpr uint32_t idesc_self = idesc_bf16_f32(kPfBM, 128, false, false);
+        const uint32_t s_lo = (uint32_t)dself, s_hi = (uint32_t)(dself >> 32);
         if (elect_one()) {
 #pragma unroll
           for (int k = 0; k < kPfD / 16; ++k) {
             const uint32_t off = ((k >> 2) * kPfPanel + (k & 3) * 32) >> 4;
-            mma_ss_lohi(tmem + kColS, q_lo + off, q_hi, k_lo + off, k_hi, idesc_self, k != 0);
+            mma_ss_lohi(tmem + kColO, q_lo + off, q_hi, s_lo + off, s_hi, idesc_self, k != 0);
           }
-          mma_commit(&k_empty[0]);
-          if (Cfg::kSelfStages == 2) mma_commit(&k_empty[1]);
-          mma_commit(&s_full[0]);
+          mma_commit(&v_empty[0]);
+          mma_commit(&v_empty[1]);
+          mma_commit(self_full);
         }
         __syncwarp();
-        ok = mbar_wait(p_ready, 0);                  // diagonal extracted: S may be overwritten
       }
       ok = ok && issue_qk(0);
       for (int i = 0; i < n_kv && ok; ++i) {
@@ -225,8 +228,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           if (!issue_qk(i + 1)) { ok = false; break; }
         }
         const int st = i & 1;
-        if (!mbar_wait(p_ready, (i + 1) & 1)) { ok = false; break; }
-        if (!mbar_wait(&v_full[st], (i >> 1) & 1)) { ok = false; break; }
+        if (!mbar_wait(&p_ready[st], (i >> 1) & 1)) { ok = false; break; }
+        // V stage 0 has held the self tile before (stage 1 shared that load's barrier)
+        if (!mbar_wait(&v_full[st], ((i >> 1) + (st == 0 ? 1 : 0)) & 1)) { ok = false; break; }
         tc_fence_after_sync();
         const int ksteps = tile_keys(i) / 16;
         const uint32_t vb = v_lo + ((st * kPfKvTile) >> 4);
@@ -256,22 +260,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
     if (n_kv > 0) {
       // self tile: this thread's diagonal element S[row][row] = q_j . k_j
-      ok = mbar_wait(&s_full[0], 0);
+      ok = mbar_wait(self_full, 0);
       tc_fence_after_sync();
       uint32_t d[32];
-      tmem_ld_x32_sync(tm_lane + kColS + quad * 32, d);
+      tmem_ld_x32_sync(tm_lane + kColO + quad * 32, d);
       float s_self = 0.f;
 #pragma unroll
       for (int e = 0; e < 32; ++e) s_self = (e == lane) ? __uint_as_float(d[e]) : s_self;
       self2 = s_self * a.scale_log2;
       m = self2;
-      tc_fence_before_sync();
-      mbar_arrive(p_ready);
     }
 
     for (int i = 0; i < n_kv && ok; ++i) {
       const int st = i & 1;
-      ok = mbar_wait(&s_full[st], ((i >> 1) + (st == 0 ? 1 : 0)) & 1);
+      ok = mbar_wait(&s_full[st], (i >> 1) & 1);
       if (!ok) break;
       tc_fence_after_sync();
       const int nvalid = min(max(bound - i * kPfBN, 0), kPfBN);
@@ -343,7 +345,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       // holds (possibly NaN bit patterns): their weight is 0, but 0 * NaN is NaN
       // in the tensor core, so zero them in shared memory before P V reads them.
       if ((i + 1) * kPfBN > L) {
-        ok = mbar_wait(&v_full[st], (i >> 1) & 1);
+        ok = mbar_wait(&v_full[st], ((i >> 1) + (st == 0 ? 1 : 0)) & 1);
         if (!ok) break;
         // BN = 64: two threads per row, one panel each; BN = 128: one thread per row, both panels
         const int vr = BN == 64 ? tid >> 1 : tid;
@@ -360,7 +362,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       }
       tmem_st_wait();
       tc_fence_before_sync();
-      mbar_arrive(p_ready);
+      mbar_arrive(&p_ready[st]);
     }
 
     // epilogue: O_j = (sum_r p_r v_r + w_self v_j) / l, staged in the V buffer, one TMA store
