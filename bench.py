@@ -45,7 +45,9 @@ TRAFFIC = {
     ("decode_ragged", "decode"): 2.3529e9 + 6.9e6,       # decode_partial_kernel<bf16,128>
 }
 # kernels launched per call of the library
+# (decode: one cluster kernel up to DECODE_CLUSTER_MAX_SLABS slabs, else chunk pass + merge)
 LAUNCHES = {"gate": 4, "compact": 2, "prefill": 1, "decode": 2, "append": 1}
+DECODE_CLUSTER_MAX_SLABS = 64
 
 
 def _peaks():
@@ -280,7 +282,11 @@ class LayerRun:
     def launches_per_step(self):
         return self.layers * ((LAUNCHES["gate"] if self.has_gate else 0) +
                               (LAUNCHES["compact"] + LAUNCHES["prefill"] if self.has_prefill else 0) +
-                              self.decode_steps * (LAUNCHES["decode"] + LAUNCHES["append"]))
+                              self.decode_steps * (self.decode_launches() + LAUNCHES["append"]))
+
+    def decode_launches(self):
+        slabs = self.shape.batch * self.shape.heads
+        return 1 if slabs <= DECODE_CLUSTER_MAX_SLABS else LAUNCHES["decode"]
 
     def work_per_call(self):
         """Algorithmic work of one call, averaged over the layers of a pass (untimed extra pass):

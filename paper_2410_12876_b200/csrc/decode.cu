@@ -2,12 +2,18 @@
 // decoding stage; cache = retained tokens only, Sec. 3.3; the new token always
 // sees its own key, Eq. 5 case j = t).
 //
-// Split-K: slab s = (sequence, head) is cut into chunks of `chunk_rows` rows.
-// decode_partial_kernel reduces one chunk to an un-normalised (o, m, l)
-// triple; decode_combine_kernel merges the chunks of a slab with the self
-// term (q . k_new, v_new) and normalises.  The work is HBM-bound: every cache
-// row is read exactly once with 16-byte vector loads, one row per group of
-// kLanes consecutive lanes, several rows in flight per lane.
+// Split-K: slab s = (sequence, head) is cut into chunks of rows; a chunk is
+// reduced to an un-normalised (o, m, l) triple, and the chunks of a slab are
+// merged with the self term (q . k_new, v_new) and normalised.  The work is
+// HBM-bound: every cache row is read exactly once with 16-byte vector loads,
+// one row per group of kLanes consecutive lanes, several rows in flight per lane.
+//
+// Two forms.  Few slabs (a launch is latency-bound): one thread-block cluster
+// per slab, one chunk per CTA, the triples merged through distributed shared
+// memory by the cluster's first CTA - one kernel, no scratch.  Many slabs:
+// decode_partial_kernel writes the triples of up to kMaxSplits chunks per slab
+// to the workspace and decode_combine_kernel merges them.
+#include <cooperative_groups.h>
 #include <math.h>
 
 #include "ag_common.cuh"
@@ -17,21 +23,20 @@ namespace ag {
 constexpr int kMaxSplits = 32;     // chunks per slab the workspace is sized for
 constexpr int kPartThreads = 256;
 constexpr int kUnroll = 8;         // rows in flight per lane group (x2: K and V)
+constexpr int kClusterMaxSlabs = 64;    // up to here one cluster per slab; beyond, split-K through the workspace
+constexpr int kClusterThreads = 512;    // 256 rows in flight per CTA of a cluster (bf16, D = 128)
 
-template <typename T, int D>
-__global__ void __launch_bounds__(kPartThreads)
-decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
-                      const T *__restrict__ v_rows, const int64_t *__restrict__ row_off,
-                      const int32_t *__restrict__ len, float scale_log2, int chunk_rows,
-                      float *__restrict__ part_o, float *__restrict__ part_ml) {
+// Rows [r_begin, r_end) of one slab, streamed by a whole CTA of kThreads threads: thread (g, v) =
+// (row group, 16-byte slice of the row) ends with its group's running maximum m, sum l and slice
+// of o (log2 domain).
+template <typename T, int D, int kThreads>
+__device__ __forceinline__ void decode_stream_rows(const T *__restrict__ q, const T *__restrict__ k_rows,
+                                                   const T *__restrict__ v_rows, int64_t row0, int slab,
+                                                   int r_begin, int r_end, float scale_log2, float &m,
+                                                   float &l, float (&o)[Elem<T>::kPerVec]) {
   constexpr int kEpl = Elem<T>::kPerVec;        // elements per lane
   constexpr int kLanes = D / kEpl;              // lanes per row
-  constexpr int kGroups = kPartThreads / kLanes;
-  const int slab = blockIdx.y, chunk = blockIdx.x;
-  const int L = len[slab];
-  const int r_begin = chunk * chunk_rows;
-  if (r_begin >= L) return;
-  const int r_end = min(L, r_begin + chunk_rows);
+  constexpr int kGroups = kThreads / kLanes;
   const int g = threadIdx.x / kLanes, v = threadIdx.x % kLanes;
 
   float qf[kEpl];
@@ -39,10 +44,10 @@ decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
 #pragma unroll
   for (int e = 0; e < kEpl; ++e) qf[e] *= scale_log2;
 
-  const T *Kb = k_rows + (size_t)row_off[slab] * D + v * kEpl;
-  const T *Vb = v_rows + (size_t)row_off[slab] * D + v * kEpl;
+  const T *Kb = k_rows + (size_t)row0 * D + v * kEpl;
+  const T *Vb = v_rows + (size_t)row0 * D + v * kEpl;
 
-  float m = -INFINITY, l = 0.f, o[kEpl];
+  m = -INFINITY; l = 0.f;
 #pragma unroll
   for (int e = 0; e < kEpl; ++e) o[e] = 0.f;
 
@@ -88,6 +93,25 @@ decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
     }
     m = m_new;
   }
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kPartThreads)
+decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
+                      const T *__restrict__ v_rows, const int64_t *__restrict__ row_off,
+                      const int32_t *__restrict__ len, float scale_log2, int chunk_rows,
+                      float *__restrict__ part_o, float *__restrict__ part_ml) {
+  constexpr int kEpl = Elem<T>::kPerVec;
+  constexpr int kLanes = D / kEpl;
+  constexpr int kGroups = kPartThreads / kLanes;
+  const int slab = blockIdx.y, chunk = blockIdx.x;
+  const int L = len[slab];
+  const int r_begin = chunk * chunk_rows;
+  if (r_begin >= L) return;
+  const int r_end = min(L, r_begin + chunk_rows);
+  const int g = threadIdx.x / kLanes, v = threadIdx.x % kLanes;
+  float m, l, o[kEpl];
+  decode_stream_rows<T, D, kPartThreads>(q, k_rows, v_rows, row_off[slab], slab, r_begin, r_end, scale_log2, m, l, o);
 
   __shared__ float sm_m[kGroups], sm_l[kGroups];
   __shared__ float sm_o[kGroups][D];
@@ -149,6 +173,120 @@ decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
   Elem<T>::store(o + (size_t)slab * D + d, acc / l);
 }
 
+// One cluster of kClusterSize CTAs per slab.  CTA `rank` reduces rows [rank, rank + 1) * per of
+// the slab to a triple in its own shared memory; after a cluster barrier the first CTA reads all
+// triples through distributed shared memory, adds the self term and writes the output.  The
+// second barrier keeps every CTA's shared memory alive until it has been read.  No CTA leaves
+// early: the cluster barriers need all of them.
+constexpr int kClusterSize = 8;
+template <typename T, int D, int kThreads>
+__global__ void __launch_bounds__(kThreads)
+decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, const T *__restrict__ v_new,
+                      const T *__restrict__ k_rows, const T *__restrict__ v_rows,
+                      const int64_t *__restrict__ row_off, const int32_t *__restrict__ len,
+                      float scale_log2, T *__restrict__ out) {
+  namespace cg = cooperative_groups;
+  constexpr int kEpl = Elem<T>::kPerVec;
+  constexpr int kLanes = D / kEpl;
+  constexpr int kGroups = kThreads / kLanes;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int slab = blockIdx.y, rank = (int)cluster.block_rank();
+  const int L = len[slab];
+  const int per = ((L + kClusterSize - 1) / kClusterSize + kGroups - 1) / kGroups * kGroups;
+  const int r_begin = min(L, rank * per), r_end = min(L, r_begin + per);
+  const int g = threadIdx.x / kLanes, v = threadIdx.x % kLanes;
+
+  __shared__ float sm_m[kGroups], sm_l[kGroups];
+  __shared__ float sm_o[kGroups][D];
+  __shared__ float cta_o[D];          // this CTA's triple, read by the first CTA of the cluster
+  __shared__ float cta_ml[2];
+  __shared__ float red[D / 32];
+
+  // self score q . k_new: only the first CTA needs it; its loads are in flight with the stream's
+  float prod = 0.f;
+  if (rank == 0 && threadIdx.x < D)
+    prod = Elem<T>::load(q + (size_t)slab * D + threadIdx.x) * Elem<T>::load(k_new + (size_t)slab * D + threadIdx.x);
+
+  float m, l, o[kEpl];
+  decode_stream_rows<T, D, kThreads>(q, k_rows, v_rows, row_off[slab], slab, r_begin, r_end, scale_log2, m, l, o);
+
+  if (v == 0) { sm_m[g] = m; sm_l[g] = l; }
+#pragma unroll
+  for (int e = 0; e < kEpl; ++e) sm_o[g][v * kEpl + e] = o[e];
+  if (threadIdx.x < D) {              // whole warps: D is a multiple of 32
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) prod += __shfl_xor_sync(0xffffffffu, prod, off);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = prod;
+  }
+  __syncthreads();
+  float mc = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < kGroups; ++i) mc = fmaxf(mc, sm_m[i]);
+  if (threadIdx.x < D) {
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < kGroups; ++i)
+      acc = fmaf(sm_m[i] == -INFINITY ? 0.f : exp2f(sm_m[i] - mc), sm_o[i][threadIdx.x], acc);
+    cta_o[threadIdx.x] = acc;
+  }
+  if (threadIdx.x == 0) {
+    float lc = 0.f;
+#pragma unroll
+    for (int i = 0; i < kGroups; ++i) lc = fmaf(sm_m[i] == -INFINITY ? 0.f : exp2f(sm_m[i] - mc), sm_l[i], lc);
+    cta_ml[0] = mc;
+    cta_ml[1] = lc;
+  }
+  cluster.sync();
+  if (rank == 0 && threadIdx.x < D) {
+    const int d = threadIdx.x;
+    float s_self = 0.f;
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) s_self += red[i];
+    s_self *= scale_log2;
+    float mr[kClusterSize], lr[kClusterSize], orr[kClusterSize];
+#pragma unroll
+    for (int r = 0; r < kClusterSize; ++r) {
+      const float *ml = cluster.map_shared_rank(cta_ml, r);
+      mr[r] = ml[0];
+      lr[r] = ml[1];
+      orr[r] = cluster.map_shared_rank(cta_o, r)[d];
+    }
+    float mm = s_self;
+#pragma unroll
+    for (int r = 0; r < kClusterSize; ++r) mm = fmaxf(mm, mr[r]);
+    const float w_self = exp2f(s_self - mm);
+    float acc = w_self * Elem<T>::load(v_new + (size_t)slab * D + d);
+    float lsum = w_self;
+#pragma unroll
+    for (int r = 0; r < kClusterSize; ++r) {
+      const float w = mr[r] == -INFINITY ? 0.f : exp2f(mr[r] - mm);
+      acc = fmaf(w, orr[r], acc);
+      lsum = fmaf(w, lr[r], lsum);
+    }
+    Elem<T>::store(out + (size_t)slab * D + d, acc / lsum);
+  }
+  cluster.sync();
+}
+
+template <typename T, int D, int kThreads>
+static int launch_decode_cluster(int slabs, const void *q, const void *k_new, const void *v_new,
+                                 const ag_cache &c, float scale_log2, void *o, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kClusterSize, slabs);
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = kClusterSize; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_cluster_kernel<T, D, kThreads>, static_cast<const T *>(q),
+                                 static_cast<const T *>(k_new), static_cast<const T *>(v_new),
+                                 static_cast<const T *>(c.k_rows), static_cast<const T *>(c.v_rows),
+                                 c.row_off, c.len, scale_log2, static_cast<T *>(o)));
+  return AG_OK;
+}
+
 size_t decode_workspace_bytes(const ag_layer_desc &d) {
   const size_t slabs = (size_t)d.batch * d.heads;
   return align_up(slabs * kMaxSplits * (d.head_dim + 2) * sizeof(float), 256);
@@ -158,12 +296,14 @@ template <typename T, int D>
 static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
                       const ag_cache &c, float scale, void *o, void *ws, cudaStream_t st) {
   const int slabs = d.batch * d.heads;
+  const float scale_log2 = scale * 1.4426950408889634f;
+  if (slabs <= kClusterMaxSlabs)
+    return launch_decode_cluster<T, D, kClusterThreads>(slabs, q, k_new, v_new, c, scale_log2, o, st);
   int chunk_rows = (c.max_cap + kMaxSplits - 1) / kMaxSplits;
   chunk_rows = (chunk_rows + 127) / 128 * 128;   // whole iterations of the partial kernel (bf16, D = 128)
   const int n_chunks = c.max_cap > 0 ? (c.max_cap + chunk_rows - 1) / chunk_rows : 0;
   float *part_o = static_cast<float *>(ws);
   float *part_ml = part_o + (size_t)slabs * kMaxSplits * D;
-  const float scale_log2 = scale * 1.4426950408889634f;
   if (n_chunks > 0) {
     dim3 grid(n_chunks, slabs);
     decode_partial_kernel<T, D><<<grid, kPartThreads, 0, st>>>(

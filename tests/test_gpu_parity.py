@@ -249,6 +249,32 @@ def test_decode_long_slabs_many_chunks():
     T.check_close(T.f64(o), orc.decode_attention(T.f64(q), T.f64(kn), T.f64(vn), ocache), "bf16", "long slabs")
 
 
+@pytest.mark.parametrize("shape", [LayerShape(9, 300, 256, 8, 128, 2, 128, "bf16"),
+                                   LayerShape(17, 150, 128, 4, 64, 1, 64, "f32")],
+                         ids=["bf16_72slabs", "f32_d64_68slabs"])
+def test_decode_many_slabs_takes_the_workspace_form(shape):
+    """More slabs than the one-cluster-per-slab form serves: chunk pass + merge through the
+    workspace, at a size the oracle checks in full; ragged and empty slabs included."""
+    Q, K, V = inputs.qkv_gaussian(shape, 470, DEV)
+    f = inputs.bernoulli_flags((shape.batch, shape.heads, shape.seq), 0.6, 471).numpy()
+    f[0, 0] = 1
+    f[1, 1] = 0
+    f[2, 2, 5:] = 0
+    flags = torch.from_numpy(f).to(DEV)
+    steps = 3
+    cap = [shape.seq + steps] * (shape.batch * shape.heads)
+    cache, prefix, idx, status = T.gpu_compact(shape, K, V, flags, cap=cap)
+    ocache = orc.compact_kv(T.f64(K), T.f64(V), f)
+    for step in range(steps):
+        q, kn, vn, fn = inputs.decode_inputs(shape, 472, step, DEV, keep_new=0.5)
+        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status)
+        o_ref = orc.decode_attention(T.f64(q), T.f64(kn), T.f64(vn), ocache)
+        T.check_close(T.f64(o), o_ref, shape.dtype, f"decode step {step}")
+        orc.cache_append(ocache, T.f64(kn), T.f64(vn), fn.cpu().numpy())
+    assert np.array_equal(cache.len.cpu().numpy(), orc.cache_lengths(ocache).reshape(-1))
+    assert int(status.item()) == 0
+
+
 def test_decode_empty_cache_returns_own_value_and_full_slab_reports_overflow():
     shape = SMALL_BF16.with_(seq=64)
     Q, K, V = inputs.qkv_gaussian(shape, 500, DEV)
