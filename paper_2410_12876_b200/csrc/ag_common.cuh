@@ -36,11 +36,13 @@ int launch_gate(const ag_layer_desc &d, const void *X, const void *Wq, const voi
 bool gate_proj_tc_supported(int K, int GD);
 int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, void *Chi,
                         void *Clo, int M, int K, int GD, cudaStream_t st);
-// Tensor-core MHA' (Sec. 3.3) on the hi / lo pairs: H' [B*n, GD] float32.
+// Tensor-core MHA' (Sec. 3.3) on the hi / lo pairs, then the split-K merge fused with the gate's
+// output layer and threshold (Eq. 3, Eq. 4): scores (optional) and flags [B, h, n].
 bool gate_attn_tc_supported(const ag_layer_desc &d);
 size_t gate_attn_partial_bytes(const ag_layer_desc &d);   // split-K partials (workspace)
-int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *qkv_lo, float *hcat,
-                        void *partials, cudaStream_t st);
+int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *qkv_lo, void *partials,
+                        const void *Wo, const float *gamma, float logit_tau, float *scores, uint8_t *flags,
+                        cudaStream_t st);
 int gate_attn_tc_wait_timeouts();
 int gemm_tc_wait_timeouts();
 

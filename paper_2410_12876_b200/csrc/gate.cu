@@ -4,7 +4,8 @@
 //   1. projection   [Q' | K' | V'] = X [Wq_g | Wk_g | Wv_g]   (tcgen05 GEMM for bf16, else CUDA cores)
 //   2. MHA'         H'_g = Softmax(Q'_g K'_g^T / sqrt(d'_k)) V'_g  (tcgen05 on bf16 hi/lo pairs for
 //                   bf16 layers with d'_k = 128, else float32 on CUDA cores)
-//   3. gate_out_kernel     s = [H'_1 .. H'_h'] Wo_g;  flag = s + gamma > logit(tau)
+//   3. output layer    s = [H'_1 .. H'_h'] Wo_g;  flag = s + gamma > logit(tau)
+//                   (gate_out_kernel; on the tensor-core path fused into the merge of MHA's split-K partials)
 //
 // The scores decide a hard threshold, so everything after the (exact) products
 // of the input elements is kept in float32: a flag can then differ from an
@@ -138,6 +139,7 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
   float *qkv = static_cast<float *>(ws);
   float *hcat = reinterpret_cast<float *>(static_cast<char *>(ws) +
                                           align_up((size_t)M * 3 * GD * sizeof(float), 256));
+  const float logit_tau = (float)log((double)d.tau / (1.0 - (double)d.tau));
   if (sizeof(T) == 2 && gate_attn_tc_supported(d)) {
     // tensor-core path: projections as bf16 hi/lo pairs, MHA' on tcgen05 with three products per term
     void *hi = ws;
@@ -145,8 +147,8 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
     int rc = launch_gate_proj_tc(X, Wq, Wk, Wv, nullptr, hi, lo, M, d.hidden, GD, st);
     if (rc) return rc;
     void *partials = reinterpret_cast<char *>(hcat) + align_up((size_t)M * GD * sizeof(float), 256);
-    rc = launch_gate_attn_tc(d, hi, lo, hcat, partials, st);
-    if (rc) return rc;
+    // the merge of the split-K partials carries the output layer and the threshold with it
+    return launch_gate_attn_tc(d, hi, lo, partials, Wo, gamma, logit_tau, scores, flags, st);
   } else {
     if (sizeof(T) == 2 && gate_proj_tc_supported(d.hidden, GD)) {
       int rc = launch_gate_proj_tc(X, Wq, Wk, Wv, qkv, nullptr, nullptr, M, d.hidden, GD, st);
@@ -177,7 +179,6 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
     if (rc) return rc;
   }
 
-  const float logit_tau = (float)log((double)d.tau / (1.0 - (double)d.tau));
   const size_t out_smem = sizeof(float) * (size_t)kOutTokens * GD + sizeof(T) * (size_t)GD * 32;
   auto out_kern = gate_out_kernel<T>;
   AG_CUDA_TRY(cudaFuncSetAttribute(out_kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)out_smem));

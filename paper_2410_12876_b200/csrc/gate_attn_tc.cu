@@ -14,7 +14,8 @@
 //
 // A (query tile, head) pair with many key tiles is cut into work items of at most
 // `chunk` key tiles so that the causal triangle spreads evenly over the SMs; every
-// item leaves an un-normalised partial (O, m, l) and gate_merge_kernel combines them.
+// item leaves an un-normalised partial (O, m, l); gate_merge_out_kernel combines them and applies
+// the gate's output layer and threshold.
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O [256,384) Phi [384,448) Plo [448,512).
 #include "ag_common.cuh"
@@ -36,7 +37,6 @@ constexpr uint32_t kGaColS = 0, kGaColO = 256, kGaColPhi = 384, kGaColPlo = 448,
 constexpr float kGaRescaleThreshold = 8.f;
 
 struct GateAttnArgs {
-  float *H;                 // [B * n, GD]                     (merge output)
   float *part_o;            // [items, 128, 128] un-normalised partial outputs
   float *part_ml;           // [items, 128, 2]   running max (log2 units) and sum per row
   int n, n_qtiles, gate_heads, problems, GD, causal;
@@ -310,42 +310,72 @@ bool gate_attn_tc_supported(const ag_layer_desc &d) {
   return d.dtype == AG_BF16 && d.gate_head_dim == 128 && gate_proj_tc_supported(d.hidden, GD);
 }
 
-// H'[t, g * 128 + c] = sum_s w_s O_s[r, c] / sum_s w_s l_s with w_s = 2^(m_s - max_s m_s): the
-// split-K merge of an online softmax.  One warp per query row (8 rows per CTA), a lane per
-// four columns: every access of a warp is one 512-byte row.
-constexpr int kMergeRows = 8;
-__global__ void __launch_bounds__(kMergeRows * 32)
-gate_merge_kernel(const GateAttnArgs a) {
-  constexpr int kBlocksPerTile = kGaBM / kMergeRows;
-  const int tile = blockIdx.x / kBlocksPerTile;                    // (problem, query tile)
-  const int prob = tile / a.n_qtiles, qt = tile % a.n_qtiles;
-  const int b = prob / a.gate_heads, g = prob % a.gate_heads;
+// The split-K merge of MHA' and the gate's output layer in one pass (Eq. 3, Eq. 4):
+//   H'[t, g * 128 + c] = sum_s w_s O_s[r, c] / sum_s w_s l_s,  w_s = 2^(m_s - max_s m_s)
+//   s[t, i] = H'[t, :] Wo_g[:, i];  flag = s + gamma_i > logit(tau)
+// One CTA = 16 tokens, one warp per token.  A warp merges the token's row of every gate head
+// (a lane per four columns: every access is one 512-byte row) into shared memory; then thread
+// (token, lane) owns head `lane` of that token, in rounds of 32 heads, against a [GD][32]
+// slice of Wo staged in shared memory (a conflict-free row of Wo and a broadcast value of H'
+// per step).  H' never goes to global memory.
+constexpr int kMoTokens = 16, kMoThreads = kMoTokens * 32;
+template <typename T>
+__global__ void __launch_bounds__(kMoThreads)
+gate_merge_out_kernel(const GateAttnArgs a, const T *__restrict__ Wo, const float *__restrict__ gamma,
+                      float logit_tau, int h, float *__restrict__ scores, uint8_t *__restrict__ flags) {
+  extern __shared__ __align__(16) unsigned char mo_smem[];
+  float *Hs = reinterpret_cast<float *>(mo_smem);                                   // [16][GD]
+  T *Ws = reinterpret_cast<T *>(mo_smem + sizeof(float) * kMoTokens * a.GD);       // [GD][32]
+  const int tiles_per_seq = (a.n + kMoTokens - 1) / kMoTokens;
+  const int b = blockIdx.x / tiles_per_seq, t0 = (blockIdx.x % tiles_per_seq) * kMoTokens;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r = (blockIdx.x % kBlocksPerTile) * kMergeRows + warp;
-  const int t = qt * kGaBM + r;
-  if (t >= a.n) return;
-  int first = 0;
-  for (int q = 0; q < qt; ++q) first += ga_splits(q, a.n_qtiles, a.causal, a.chunk);
-  const int ns = ga_splits(qt, a.n_qtiles, a.causal, a.chunk);
-  const size_t row0 = ((size_t)prob * a.items_per_prob + first) * kGaBM + r;   // + s * 128 per split
-  float mmax = -INFINITY;
-  for (int s = lane; s < ns; s += 32) mmax = fmaxf(mmax, a.part_ml[(row0 + (size_t)s * kGaBM) * 2]);
+  const int t = t0 + warp;
+  float *hrow = Hs + warp * a.GD;
+  if (t < a.n) {
+    const int qt = t / kGaBM, r = t % kGaBM;
+    int first = 0;
+    for (int q = 0; q < qt; ++q) first += ga_splits(q, a.n_qtiles, a.causal, a.chunk);
+    const int ns = ga_splits(qt, a.n_qtiles, a.causal, a.chunk);
+    for (int g = 0; g < a.gate_heads; ++g) {
+      const int prob = b * a.gate_heads + g;
+      const size_t row0 = ((size_t)prob * a.items_per_prob + first) * kGaBM + r;   // + s * 128 per split
+      float mmax = -INFINITY;
+      for (int s = lane; s < ns; s += 32) mmax = fmaxf(mmax, a.part_ml[(row0 + (size_t)s * kGaBM) * 2]);
 #pragma unroll
-  for (int off = 16; off > 0; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  float lsum = 0.f;
+      for (int off = 16; off > 0; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float lsum = 0.f;
 #pragma unroll 4
-  for (int s = 0; s < ns; ++s) {
-    const float2 ml = *reinterpret_cast<const float2 *>(a.part_ml + (row0 + (size_t)s * kGaBM) * 2);
-    const float4 o = *reinterpret_cast<const float4 *>(a.part_o + (row0 + (size_t)s * kGaBM) * kGaD + lane * 4);
-    const float w = fast_exp2(ml.x - mmax);
-    acc.x = fmaf(w, o.x, acc.x); acc.y = fmaf(w, o.y, acc.y);
-    acc.z = fmaf(w, o.z, acc.z); acc.w = fmaf(w, o.w, acc.w);
-    lsum = fmaf(w, ml.y, lsum);
+      for (int s = 0; s < ns; ++s) {
+        const float2 ml = *reinterpret_cast<const float2 *>(a.part_ml + (row0 + (size_t)s * kGaBM) * 2);
+        const float4 o = *reinterpret_cast<const float4 *>(a.part_o + (row0 + (size_t)s * kGaBM) * kGaD + lane * 4);
+        const float w = fast_exp2(ml.x - mmax);
+        acc.x = fmaf(w, o.x, acc.x); acc.y = fmaf(w, o.y, acc.y);
+        acc.z = fmaf(w, o.z, acc.z); acc.w = fmaf(w, o.w, acc.w);
+        lsum = fmaf(w, ml.y, lsum);
+      }
+      const float inv = 1.f / lsum;
+      *reinterpret_cast<float4 *>(hrow + g * kGaD + lane * 4) =
+          make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+    }
   }
-  const float inv = 1.f / lsum;
-  *reinterpret_cast<float4 *>(a.H + ((size_t)b * a.n + t) * a.GD + g * kGaD + lane * 4) =
-      make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+  for (int i0 = 0; i0 < h; i0 += 32) {
+    __syncthreads();                                 // H' rows complete; previous slice of Wo consumed
+    for (int x = threadIdx.x; x < a.GD * 32; x += kMoThreads) {
+      const int c = x >> 5, i = i0 + (x & 31);
+      Ws[x] = i < h ? Wo[(size_t)c * h + i] : T(0.f);
+    }
+    __syncthreads();
+    float acc = 0.f;
+#pragma unroll 8
+    for (int c = 0; c < a.GD; ++c) acc = fmaf(hrow[c], Elem<T>::load(Ws + c * 32 + lane), acc);
+    const int i = i0 + lane;
+    if (i < h && t < a.n) {
+      const size_t o = ((size_t)b * h + i) * a.n + t;
+      if (scores) scores[o] = acc;
+      flags[o] = (acc + (gamma ? gamma[i] : 0.f)) > logit_tau ? 1 : 0;
+    }
+  }
 }
 
 // Key tiles per work item: small enough for about three waves of items over the SMs.
@@ -370,8 +400,9 @@ size_t gate_attn_partial_bytes(const ag_layer_desc &d) {
   return align_up(items * kGaBM * kGaD * sizeof(float), 256) + align_up(items * kGaBM * 2 * sizeof(float), 256);
 }
 
-int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *qkv_lo, float *hcat,
-                        void *partials, cudaStream_t st) {
+int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *qkv_lo, void *partials,
+                        const void *Wo, const float *gamma, float logit_tau, float *scores, uint8_t *flags,
+                        cudaStream_t st) {
   const int GD = d.gate_heads * d.gate_head_dim;
   CUtensorMap tmHi, tmLo;
   int rc = make_tmap_3d_bf16(&tmHi, qkv_hi, d.batch, d.seq, 3 * GD, kGaBM, 64);
@@ -382,7 +413,6 @@ int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *
   if ((rc = make_tmap_3d_bf16(&tmHiKv, qkv_hi, d.batch, d.seq, 3 * GD, kGaBN, 64))) return rc;
   if ((rc = make_tmap_3d_bf16(&tmLoKv, qkv_lo, d.batch, d.seq, 3 * GD, kGaBN, 64))) return rc;
   GateAttnArgs a;
-  a.H = hcat;
   a.n = d.seq; a.n_qtiles = (d.seq + kGaBM - 1) / kGaBM;
   a.gate_heads = d.gate_heads; a.problems = d.batch * d.gate_heads; a.GD = GD; a.causal = d.gate_causal;
   gate_attn_plan(d, a.chunk, a.items_per_prob);
@@ -394,7 +424,12 @@ int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *
   AG_CUDA_TRY(cudaFuncSetAttribute(gate_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGaSmemBytes));
   gate_attn_tc_kernel<<<(unsigned)items, kGaThreads, kGaSmemBytes, st>>>(tmHi, tmLo, tmHiKv, tmLoKv, a);
   AG_LAUNCH_CHECK();
-  gate_merge_kernel<<<a.problems * a.n_qtiles * (kGaBM / kMergeRows), kMergeRows * 32, 0, st>>>(a);
+  const size_t mo_smem = sizeof(float) * kMoTokens * GD + sizeof(__nv_bfloat16) * GD * 32;
+  auto mo = gate_merge_out_kernel<__nv_bfloat16>;
+  AG_CUDA_TRY(cudaFuncSetAttribute(mo, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mo_smem));
+  const int blocks = d.batch * ((d.seq + kMoTokens - 1) / kMoTokens);
+  mo<<<blocks, kMoThreads, mo_smem, st>>>(a, static_cast<const __nv_bfloat16 *>(Wo), gamma, logit_tau, d.heads,
+                                          scores, flags);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
