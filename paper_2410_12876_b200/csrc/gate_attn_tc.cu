@@ -7,15 +7,19 @@
 // each product A B is evaluated as  Ahi Bhi + Ahi Blo + Alo Bhi  in the float32
 // accumulator (the dropped lo*lo term is 2^-16 relative).
 //
-// One CTA = 128 queries of one (sequence, gate head).  Structure as in the
-// prefill kernel: warp 0 TMA, warp 1 tcgen05.mma issue, warps 2..5 softmax with
-// one row per thread.  Key tiles hold 64 keys (32 KB per K or V stage with the
-// hi and lo halves), two stages each, so loads run a tile ahead of the MMAs.
+// Structure as in the prefill kernel: warp 0 TMA, warp 1 tcgen05.mma issue,
+// warps 2..5 softmax with one row per thread.  A query tile is 128 queries of
+// one (sequence, gate head); key tiles hold 64 keys (32 KB per K or V stage with
+// the hi and lo halves), two stages each, so loads run a tile ahead of the MMAs.
 //
-// A (query tile, head) pair with many key tiles is cut into work items of at most
-// `chunk` key tiles so that the causal triangle spreads evenly over the SMs; every
-// item leaves an un-normalised partial (O, m, l); gate_merge_out_kernel combines them and applies
-// the gate's output layer and threshold.
+// Work is the list of all (query tile, key tile) steps, query tiles in order
+// and each one's key tiles in order.  The list is cut into equal segments, one
+// CTA (one SM) each, so every SM gets the same number of steps whatever the
+// shape of the causal triangle.  A segment crosses query tiles: the CTA handles
+// its pieces one after the other, the loads of the next piece running under the
+// tail of the current one.  Every piece leaves an un-normalised partial
+// (O, m, l); gate_merge_out_kernel combines the pieces of a query tile and
+// applies the gate's output layer and threshold.
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O [256,384) Phi [384,448) Plo [448,512).
 #include "ag_common.cuh"
@@ -40,8 +44,10 @@ struct GateAttnArgs {
   float *part_o;            // [items, 128, 128] un-normalised partial outputs
   float *part_ml;           // [items, 128, 2]   running max (log2 units) and sum per row
   int n, n_qtiles, gate_heads, problems, GD, causal;
-  int chunk;                // key tiles per work item
-  int items_per_prob;       // work items of one (sequence, head)
+  int steps_per_prob;       // (query tile, key tile) steps of one (sequence, head)
+  int total_steps;          // over all problems
+  int seg_steps;            // steps per segment (even: a piece starts on a 128-key boundary, so its
+                            // first tile holds a key every row of the query tile may see)
   float scale_log2;
 };
 
@@ -50,19 +56,35 @@ struct GateAttnArgs {
 __host__ __device__ inline int ga_key_tiles(int qt, int n_qtiles, int causal) {
   return (kGaBM / kGaBN) * (causal ? qt + 1 : n_qtiles);
 }
-__host__ __device__ inline int ga_splits(int qt, int n_qtiles, int causal, int chunk) {
-  return (ga_key_tiles(qt, n_qtiles, causal) + chunk - 1) / chunk;
+// First step of query tile qt within its problem's list.
+__host__ __device__ inline int ga_first_step(int qt, int n_qtiles, int causal) {
+  return causal ? qt * (qt + 1) : qt * 2 * n_qtiles;
 }
-// Work item k of a problem -> (query tile, split); items are numbered by ascending query tile.
-__device__ inline void ga_locate(int k, int n_qtiles, int causal, int chunk, int &qt, int &split) {
-  qt = 0;
-  for (;;) {
-    const int ns = ga_splits(qt, n_qtiles, causal, chunk);
-    if (k < ns || qt == n_qtiles - 1) break;
-    k -= ns;
-    ++qt;
+// The piece of a segment that starts at global step x (x < x_end, the segment's end).
+struct GaPiece {
+  int prob, qt, kv_begin, n_kv;
+};
+__device__ inline GaPiece ga_piece(const GateAttnArgs &a, int x, int x_end) {
+  GaPiece p;
+  p.prob = x / a.steps_per_prob;
+  const int y = x - p.prob * a.steps_per_prob;
+  if (a.causal) {
+    int qt = (int)((sqrtf(4.f * (float)y + 1.f) - 1.f) * 0.5f);
+    while (qt > 0 && qt * (qt + 1) > y) --qt;
+    while ((qt + 1) * (qt + 2) <= y) ++qt;
+    p.qt = qt;
+  } else {
+    p.qt = y / (2 * a.n_qtiles);
   }
-  split = k;
+  p.kv_begin = y - ga_first_step(p.qt, a.n_qtiles, a.causal);
+  const int tile_end = x - p.kv_begin + ga_key_tiles(p.qt, a.n_qtiles, a.causal);   // global end of the query tile
+  p.n_kv = min(x_end, tile_end) - x;
+  return p;
+}
+// Partial slot of the piece of query tile (prob, qt) that lies in segment seg: consecutive pieces
+// differ in the query tile, the segment or both, so the sum is unique and grows along the list.
+__host__ __device__ inline int ga_slot(int prob, int qt, int n_qtiles, int seg) {
+  return prob * n_qtiles + qt + seg;
 }
 
 __global__ void __launch_bounds__(kGaThreads, 1)
@@ -78,19 +100,15 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
   uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;  // [2]
   uint64_t *s_full = bars + 9;           // [2]
   uint64_t *p_ready = bars + 11, *pv_done = bars + 12;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 13);
+  uint64_t *q_empty = bars + 13, *o_free = bars + 14;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 15);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // items of the last (longest) query tiles first
-  const int prob = blockIdx.x % a.problems;
-  const int item = a.items_per_prob - 1 - (int)(blockIdx.x / a.problems);
-  int qt, split;
-  ga_locate(item, a.n_qtiles, a.causal, a.chunk, qt, split);
-  const int b = prob / a.gate_heads, g = prob % a.gate_heads;
-  const int j0 = qt * kGaBM;
-  const int kv_begin = split * a.chunk;            // first key tile of this item
-  const int n_kv = min(a.chunk, ga_key_tiles(qt, a.n_qtiles, a.causal) - kv_begin);   // tiles of this item
-  const int xq = g * kGaD, xk = a.GD + g * kGaD, xv = 2 * a.GD + g * kGaD;   // columns in [Q' | K' | V']
+  // This CTA's segment of the step list.  Every role walks its pieces with the same arithmetic;
+  // tiles are numbered t = 0, 1, ... across the pieces (stage and S buffer t & 1, in their use
+  // number t >> 1; P and the P V barrier in their use number t), pieces pc = 0, 1, ...
+  const int x_begin = blockIdx.x * a.seg_steps;
+  const int x_end = min(a.total_steps, x_begin + a.seg_steps);
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
@@ -101,6 +119,8 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
     }
     mbar_init(p_ready, 128);
     mbar_init(pv_done, 1);
+    mbar_init(q_empty, 1);
+    mbar_init(o_free, 128);
     fence_barrier_init();
     prefetch_tensormap(&tmHi); prefetch_tensormap(&tmLo);
     prefetch_tensormap(&tmHiKv); prefetch_tensormap(&tmLoKv);
@@ -116,26 +136,36 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
 
   if (warp == 0) {
     if (lane == 0) {
-      mbar_arrive_expect_tx(q_full, 2 * kGaTile);
-      tma_load_3d(sQ, &tmHi, q_full, xq, j0, b);
-      tma_load_3d(sQ + kGaPanel, &tmHi, q_full, xq + 64, j0, b);
-      tma_load_3d(sQ + kGaTile, &tmLo, q_full, xq, j0, b);
-      tma_load_3d(sQ + kGaTile + kGaPanel, &tmLo, q_full, xq + 64, j0, b);
-      auto load_kv = [&](uint8_t *dst, uint64_t *bar, int x, int y) {
-        mbar_arrive_expect_tx(bar, kGaKvStage);
-        tma_load_3d(dst, &tmHiKv, bar, x, y, b);
-        tma_load_3d(dst + kGaKvPanel, &tmHiKv, bar, x + 64, y, b);
-        tma_load_3d(dst + kGaKvTile, &tmLoKv, bar, x, y, b);
-        tma_load_3d(dst + kGaKvTile + kGaKvPanel, &tmLoKv, bar, x + 64, y, b);
-      };
-      for (int i = 0; i < n_kv; ++i) {
-        const int st = i & 1;
-        const uint32_t ph = (i >> 1) & 1;
-        const int y = (kv_begin + i) * kGaBN;
-        if (!mbar_wait(&k_empty[st], ph ^ 1)) break;
-        load_kv(sK + st * kGaKvStage, &k_full[st], xk, y);
-        if (!mbar_wait(&v_empty[st], ph ^ 1)) break;
-        load_kv(sV + st * kGaKvStage, &v_full[st], xv, y);
+      bool ok = true;
+      int t = 0;
+      for (int x = x_begin, pc = 0; x < x_end && ok; ++pc) {
+        const GaPiece pz = ga_piece(a, x, x_end);
+        const int b = pz.prob / a.gate_heads, g = pz.prob % a.gate_heads, j0 = pz.qt * kGaBM;
+        const int xq = g * kGaD, xk = a.GD + g * kGaD, xv = 2 * a.GD + g * kGaD;   // columns in [Q' | K' | V']
+        ok = mbar_wait(q_empty, (pc & 1) ^ 1);       // the previous piece's last Q K^T has read Q
+        if (!ok) break;
+        mbar_arrive_expect_tx(q_full, 2 * kGaTile);
+        tma_load_3d(sQ, &tmHi, q_full, xq, j0, b);
+        tma_load_3d(sQ + kGaPanel, &tmHi, q_full, xq + 64, j0, b);
+        tma_load_3d(sQ + kGaTile, &tmLo, q_full, xq, j0, b);
+        tma_load_3d(sQ + kGaTile + kGaPanel, &tmLo, q_full, xq + 64, j0, b);
+        auto load_kv = [&](uint8_t *dst, uint64_t *bar, int xc, int y) {
+          mbar_arrive_expect_tx(bar, kGaKvStage);
+          tma_load_3d(dst, &tmHiKv, bar, xc, y, b);
+          tma_load_3d(dst + kGaKvPanel, &tmHiKv, bar, xc + 64, y, b);
+          tma_load_3d(dst + kGaKvTile, &tmLoKv, bar, xc, y, b);
+          tma_load_3d(dst + kGaKvTile + kGaKvPanel, &tmLoKv, bar, xc + 64, y, b);
+        };
+        for (int i = 0; i < pz.n_kv; ++i, ++t) {
+          const int st = t & 1;
+          const uint32_t ph = (t >> 1) & 1;
+          const int y = (pz.kv_begin + i) * kGaBN;
+          if (!mbar_wait(&k_empty[st], ph ^ 1)) { ok = false; break; }
+          load_kv(sK + st * kGaKvStage, &k_full[st], xk, y);
+          if (!mbar_wait(&v_empty[st], ph ^ 1)) { ok = false; break; }
+          load_kv(sV + st * kGaKvStage, &v_full[st], xv, y);
+        }
+        x += pz.n_kv;
       }
     }
   } else if (warp == 1) {
@@ -147,9 +177,9 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
     const uint32_t q_lo = (uint32_t)dq, q_hi = (uint32_t)(dq >> 32);
     const uint32_t k_lo = (uint32_t)dk, k_hi = (uint32_t)(dk >> 32);
     const uint32_t v_lo = (uint32_t)dv, v_hi = (uint32_t)(dv >> 32);
-    auto issue_qk = [&](int i) -> bool {
-      const int st = i & 1;
-      if (!mbar_wait(&k_full[st], (i >> 1) & 1)) return false;
+    auto issue_qk = [&](int t, bool last) -> bool {   // t: tile number across the pieces
+      const int st = t & 1;
+      if (!mbar_wait(&k_full[st], (t >> 1) & 1)) return false;
       tc_fence_after_sync();
       const uint32_t d = tmem + kGaColS + st * 128;
       const uint32_t kb = k_lo + ((st * kGaKvStage) >> 4);
@@ -165,18 +195,26 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
         }
         mma_commit(&k_empty[st]);
         mma_commit(&s_full[st]);
+        if (last) mma_commit(q_empty);               // Q may be replaced by the next piece's
       }
       __syncwarp();
       return true;
     };
-    bool ok = mbar_wait(q_full, 0);
-    ok = ok && issue_qk(0);
-    for (int i = 0; i < n_kv && ok; ++i) {
-      if (i + 1 < n_kv) ok = issue_qk(i + 1);
+    bool ok = true;
+    int t0 = 0;                                      // tile number of the piece's first tile
+    for (int x = x_begin, pc = 0; x < x_end && ok; ++pc) {
+      const int n_kv = ga_piece(a, x, x_end).n_kv;
+      ok = mbar_wait(q_full, pc & 1);
+      ok = ok && issue_qk(t0, n_kv == 1);
+      for (int i = 0; i < n_kv && ok; ++i) {
+      const int t = t0 + i;
+      if (i + 1 < n_kv) ok = issue_qk(t + 1, i + 2 == n_kv);
       if (!ok) break;
-      const int st = i & 1;
-      if (!mbar_wait(p_ready, i & 1)) { ok = false; break; }
-      if (!mbar_wait(&v_full[st], (i >> 1) & 1)) { ok = false; break; }
+      const int st = t & 1;
+      if (!mbar_wait(p_ready, t & 1)) { ok = false; break; }
+      if (!mbar_wait(&v_full[st], (t >> 1) & 1)) { ok = false; break; }
+      // the first P V of a piece overwrites O: the previous piece's epilogue must have read it
+      if (i == 0 && pc > 0 && !mbar_wait(o_free, (pc - 1) & 1)) { ok = false; break; }
       tc_fence_after_sync();
       const uint32_t vb = v_lo + ((st * kGaKvStage) >> 4);
       if (elect_one()) {
@@ -192,23 +230,32 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
         mma_commit(pv_done);
       }
       __syncwarp();
+      }
+      t0 += n_kv;
+      x += n_kv;
     }
   } else {
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
-    const int j = j0 + row;
+    const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
+    bool ok = true;
+    int t0 = 0;                                      // tile number of the piece's first tile
+
+    for (int x = x_begin; x < x_end && ok;) {
+    const GaPiece pz = ga_piece(a, x, x_end);
+    const int n_kv = pz.n_kv, kv_begin = pz.kv_begin;
+    const int j = pz.qt * kGaBM + row;
     const bool valid = j < a.n;
     const int jc = min(j, a.n - 1);
-    const int bound = a.causal ? jc + 1 : a.n;       // keys t < bound are visible
-    const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
+    const int bound = a.causal ? jc + 1 : a.n;       // keys below bound are visible
     float m = -INFINITY, l = 0.f;
-    bool ok = true;
 
     for (int i = 0; i < n_kv && ok; ++i) {
-      ok = mbar_wait(&s_full[i & 1], (i >> 1) & 1);
+      const int t = t0 + i;
+      ok = mbar_wait(&s_full[t & 1], (t >> 1) & 1);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t tS = tm_lane + kGaColS + (i & 1) * 128;
+      const uint32_t tS = tm_lane + kGaColS + (t & 1) * 128;
       const int nvalid = min(max(bound - (kv_begin + i) * kGaBN, 0), kGaBN);
       const bool full = nvalid >= kGaBN;
 
@@ -239,7 +286,7 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
       l *= alpha;
 
       if (i > 0) {
-        ok = mbar_wait(pv_done, (i - 1) & 1);
+        ok = mbar_wait(pv_done, (t - 1) & 1);
         if (!ok) break;
         tc_fence_after_sync();
         if (rescale) {
@@ -281,16 +328,20 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
     }
 
     if (ok) {
-      ok = mbar_wait(pv_done, (n_kv - 1) & 1);
+      ok = mbar_wait(pv_done, (t0 + n_kv - 1) & 1);
       tc_fence_after_sync();
     }
     if (ok) {
-      const size_t it = (size_t)prob * a.items_per_prob + item;
+      const size_t it = (size_t)ga_slot(pz.prob, pz.qt, a.n_qtiles, (int)blockIdx.x);
       float *op = a.part_o + (it * kGaBM + row) * kGaD;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         uint32_t r[32];
         tmem_ld_x32_sync(tm_lane + kGaColO + c * 32, r);
+        if (c == 3) {                                // O is in registers: the next piece may overwrite it
+          tc_fence_before_sync();
+          mbar_arrive(o_free);
+        }
         if (valid) {
 #pragma unroll
           for (int e = 0; e < 32; e += 4)
@@ -298,6 +349,9 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
         }
       }
       if (valid) *reinterpret_cast<float2 *>(a.part_ml + (it * kGaBM + row) * 2) = make_float2(m, l);
+    }
+    t0 += n_kv;
+    x += n_kv;
     }
   }
   tc_fence_before_sync();
@@ -333,12 +387,13 @@ gate_merge_out_kernel(const GateAttnArgs a, const T *__restrict__ Wo, const floa
   float *hrow = Hs + warp * a.GD;
   if (t < a.n) {
     const int qt = t / kGaBM, r = t % kGaBM;
-    int first = 0;
-    for (int q = 0; q < qt; ++q) first += ga_splits(q, a.n_qtiles, a.causal, a.chunk);
-    const int ns = ga_splits(qt, a.n_qtiles, a.causal, a.chunk);
+    const int y0 = ga_first_step(qt, a.n_qtiles, a.causal), y1 = y0 + ga_key_tiles(qt, a.n_qtiles, a.causal);
     for (int g = 0; g < a.gate_heads; ++g) {
       const int prob = b * a.gate_heads + g;
-      const size_t row0 = ((size_t)prob * a.items_per_prob + first) * kGaBM + r;   // + s * 128 per split
+      // the query tile's steps [x0, x1) of the list lie in segments seg0 .. seg1, one piece in each
+      const int x0 = prob * a.steps_per_prob + y0, x1 = prob * a.steps_per_prob + y1;
+      const int seg0 = x0 / a.seg_steps, ns = (x1 - 1) / a.seg_steps - seg0 + 1;
+      const size_t row0 = (size_t)ga_slot(prob, qt, a.n_qtiles, seg0) * kGaBM + r;   // + s * 128 per piece
       float mmax = -INFINITY;
       for (int s = lane; s < ns; s += 32) mmax = fmaxf(mmax, a.part_ml[(row0 + (size_t)s * kGaBM) * 2]);
 #pragma unroll
@@ -378,26 +433,41 @@ gate_merge_out_kernel(const GateAttnArgs a, const T *__restrict__ Wo, const floa
   }
 }
 
-// Key tiles per work item: small enough for about three waves of items over the SMs.
-static void gate_attn_plan(const ag_layer_desc &d, int &chunk, int &items_per_prob) {
+// Segments: one per SM (at most kGaMaxSeg) when there is that much work, of an even number of steps.
+constexpr int kGaMaxSeg = 256;
+struct GateAttnPlan {
+  int steps_per_prob, total_steps, seg_steps, n_seg;
+  size_t slots;
+};
+static int gate_attn_plan(const ag_layer_desc &d, GateAttnPlan &p) {
+  static int sm_count[64] = {0};                     // per device, read once
+  int dev = 0;
+  AG_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return AG_ERR_UNSUPPORTED;
+  if (sm_count[dev] == 0) {
+    int v = 0;
+    AG_CUDA_TRY(cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev));
+    sm_count[dev] = v < 1 ? 1 : (v > kGaMaxSeg ? kGaMaxSeg : v);
+  }
   const int nq = (d.seq + kGaBM - 1) / kGaBM, problems = d.batch * d.gate_heads;
-  long long tiles = 0;
-  for (int q = 0; q < nq; ++q) tiles += ga_key_tiles(q, nq, d.gate_causal);
-  tiles *= problems;
-  chunk = (int)((tiles + 3 * 148 - 1) / (3 * 148));
-  // even, so that an item starts on a 128-key boundary: its first tile then holds a key every
-  // row of the query tile may see (the kernel seeds the running maximum from it)
-  chunk = (chunk + 1) & ~1;
-  chunk = chunk < 2 ? 2 : (chunk > 32 ? 32 : chunk);
-  items_per_prob = 0;
-  for (int q = 0; q < nq; ++q) items_per_prob += ga_splits(q, nq, d.gate_causal, chunk);
+  const long long per = d.gate_causal ? (long long)nq * (nq + 1) : 2LL * nq * nq;
+  const long long total = per * problems;
+  if (total >= (1LL << 30)) return AG_ERR_UNSUPPORTED;
+  long long seg = (total + sm_count[dev] - 1) / sm_count[dev];
+  seg = (seg + 1) & ~1LL;
+  p.steps_per_prob = (int)per;
+  p.total_steps = (int)total;
+  p.seg_steps = (int)seg;
+  p.n_seg = (int)((total + seg - 1) / seg);
+  p.slots = (size_t)problems * nq + p.n_seg;
+  return AG_OK;
 }
 
 size_t gate_attn_partial_bytes(const ag_layer_desc &d) {
-  int chunk, ipp;
-  gate_attn_plan(d, chunk, ipp);
-  const size_t items = (size_t)d.batch * d.gate_heads * ipp;
-  return align_up(items * kGaBM * kGaD * sizeof(float), 256) + align_up(items * kGaBM * 2 * sizeof(float), 256);
+  // one slot per piece: query tiles + segments, whatever the device (no device is asked here)
+  const size_t nq = (d.seq + kGaBM - 1) / kGaBM;
+  const size_t slots = (size_t)d.batch * d.gate_heads * nq + kGaMaxSeg;
+  return align_up(slots * kGaBM * kGaD * sizeof(float), 256) + align_up(slots * kGaBM * 2 * sizeof(float), 256);
 }
 
 int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *qkv_lo, void *partials,
@@ -415,14 +485,16 @@ int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *
   GateAttnArgs a;
   a.n = d.seq; a.n_qtiles = (d.seq + kGaBM - 1) / kGaBM;
   a.gate_heads = d.gate_heads; a.problems = d.batch * d.gate_heads; a.GD = GD; a.causal = d.gate_causal;
-  gate_attn_plan(d, a.chunk, a.items_per_prob);
-  const size_t items = (size_t)a.problems * a.items_per_prob;
+  GateAttnPlan plan;
+  if ((rc = gate_attn_plan(d, plan))) return rc;
+  a.steps_per_prob = plan.steps_per_prob; a.total_steps = plan.total_steps; a.seg_steps = plan.seg_steps;
+  const size_t slots = (size_t)a.problems * a.n_qtiles + kGaMaxSeg;
   a.part_o = static_cast<float *>(partials);
   a.part_ml = reinterpret_cast<float *>(static_cast<char *>(partials) +
-                                        align_up(items * kGaBM * kGaD * sizeof(float), 256));
+                                        align_up(slots * kGaBM * kGaD * sizeof(float), 256));
   a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kGaD));
   AG_CUDA_TRY(cudaFuncSetAttribute(gate_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGaSmemBytes));
-  gate_attn_tc_kernel<<<(unsigned)items, kGaThreads, kGaSmemBytes, st>>>(tmHi, tmLo, tmHiKv, tmLoKv, a);
+  gate_attn_tc_kernel<<<(unsigned)plan.n_seg, kGaThreads, kGaSmemBytes, st>>>(tmHi, tmLo, tmHiKv, tmLoKv, a);
   AG_LAUNCH_CHECK();
   const size_t mo_smem = sizeof(float) * kMoTokens * GD + sizeof(__nv_bfloat16) * GD * 32;
   auto mo = gate_merge_out_kernel<__nv_bfloat16>;
