@@ -23,6 +23,14 @@ void set_last_cuda_error(int e);
 #define AG_LAUNCH_CHECK() AG_CUDA_TRY(cudaGetLastError())
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+// Launch attribute that lets a kernel overlap its set-up with the tail of its predecessor (the
+// kernel itself starts with pdl_wait()).
+inline cudaLaunchAttribute pdl_attribute() {
+  cudaLaunchAttribute at = {};
+  at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at.val.programmaticStreamSerializationAllowed = 1;
+  return at;
+}
 inline bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
 // Per-step launchers (defined in the kernel files, called from ag_api.cu).
@@ -94,6 +102,14 @@ template <> struct Elem<__nv_bfloat16> {
   __device__ static inline float load(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
   __device__ static inline void store(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
 };
+
+// Programmatic dependent launch, for the small kernels of a decode step that run back to back:
+// a kernel launched with the stream-serialization attribute may be set up while its predecessor
+// in the stream is still running.  It must call pdl_wait() before it touches global memory (the
+// predecessor has then completed, its writes visible); pdl_launch_dependents() lets the successor's
+// set-up begin.  Both are no-ops in a launch without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ uint4 ldg128(const void *p) {
   return __ldg(reinterpret_cast<const uint4 *>(p));

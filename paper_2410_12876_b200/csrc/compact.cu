@@ -113,6 +113,8 @@ append_rows_kernel(const uint8_t *__restrict__ k_new, const uint8_t *__restrict_
   constexpr int kGroups = 256 / kVecs;
   const int slab = blockIdx.x * kGroups + threadIdx.x / kVecs;
   const int v = threadIdx.x % kVecs;
+  pdl_launch_dependents();
+  pdl_wait();
   const bool want = slab < n_slabs && flag_new[slab] != 0;
   // every lane of a group reads the length before lane 0 of the group bumps it
   const int L = want ? len[slab] : 0;
@@ -181,15 +183,22 @@ int launch_append(const ag_layer_desc &d, const void *k_new, const void *v_new,
   auto vr = static_cast<uint8_t *>(c.v_rows);
   const int groups = 256 / (rb / 16);
   const int grid = (slabs + groups - 1) / groups;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr = pdl_attribute();
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
   switch (rb) {
     case 128:
-      append_rows_kernel<128><<<grid, 256, 0, st>>>(kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status);
+      AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, append_rows_kernel<128>, kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status));
       break;
     case 256:
-      append_rows_kernel<256><<<grid, 256, 0, st>>>(kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status);
+      AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, append_rows_kernel<256>, kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status));
       break;
     case 512:
-      append_rows_kernel<512><<<grid, 256, 0, st>>>(kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status);
+      AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, append_rows_kernel<512>, kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status));
       break;
     default:
       return AG_ERR_UNSUPPORTED;

@@ -191,6 +191,8 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
   constexpr int kGroups = kThreads / kLanes;
   cg::cluster_group cluster = cg::this_cluster();
   const int slab = blockIdx.y, rank = (int)cluster.block_rank();
+  pdl_launch_dependents();
+  pdl_wait();
   const int L = len[slab];
   const int per = ((L + kClusterSize - 1) / kClusterSize + kGroups - 1) / kGroups * kGroups;
   const int r_begin = min(L, rank * per), r_end = min(L, r_begin + per);
@@ -275,11 +277,12 @@ static int launch_decode_cluster(int slabs, const void *q, const void *k_new, co
   cfg.gridDim = dim3(kClusterSize, slabs);
   cfg.blockDim = dim3(kThreads);
   cfg.stream = st;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = kClusterSize; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kClusterSize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1] = pdl_attribute();
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
   AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_cluster_kernel<T, D, kThreads>, static_cast<const T *>(q),
                                  static_cast<const T *>(k_new), static_cast<const T *>(v_new),
                                  static_cast<const T *>(c.k_rows), static_cast<const T *>(c.v_rows),
