@@ -368,10 +368,9 @@ bool gate_attn_tc_supported(const ag_layer_desc &d) {
 //   H'[t, g * 128 + c] = sum_s w_s O_s[r, c] / sum_s w_s l_s,  w_s = 2^(m_s - max_s m_s)
 //   s[t, i] = H'[t, :] Wo_g[:, i];  flag = s + gamma_i > logit(tau)
 // One CTA = 16 tokens, one warp per token.  A warp merges the token's row of every gate head
-// (a lane per four columns: every access is one 512-byte row) into shared memory; then thread
-// (token, lane) owns head `lane` of that token, in rounds of 32 heads, against a [GD][32]
-// slice of Wo staged in shared memory (a conflict-free row of Wo and a broadcast value of H'
-// per step).  H' never goes to global memory.
+// (a lane per four columns: every access is one 512-byte row) into shared memory; then four
+// warps take four tokens each, a lane per head, in rounds of 32 heads, against a [GD][32]
+// slice of Wo staged in shared memory.  H' never goes to global memory.
 constexpr int kMoTokens = 16, kMoThreads = kMoTokens * 32;
 template <typename T>
 __global__ void __launch_bounds__(kMoThreads)
@@ -421,14 +420,38 @@ gate_merge_out_kernel(const GateAttnArgs a, const T *__restrict__ Wo, const floa
       Ws[x] = i < h ? Wo[(size_t)c * h + i] : T(0.f);
     }
     __syncthreads();
-    float acc = 0.f;
-#pragma unroll 8
-    for (int c = 0; c < a.GD; ++c) acc = fmaf(hrow[c], Elem<T>::load(Ws + c * 32 + lane), acc);
-    const int i = i0 + lane;
-    if (i < h && t < a.n) {
-      const size_t o = ((size_t)b * h + i) * a.n + t;
-      if (scores) scores[o] = acc;
-      flags[o] = (acc + (gamma ? gamma[i] : 0.f)) > logit_tau ? 1 : 0;
+    if (warp < kMoTokens / 4) {
+      // warp w: tokens 4 w .. 4 w + 3 against head `lane`; per four steps of the reduction four
+      // broadcast float4 of H' and four values of Wo feed sixteen FMAs
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      const float *h4 = Hs + warp * 4 * a.GD;
+#pragma unroll 2
+      for (int c = 0; c < a.GD; c += 4) {
+        float w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) w[k] = Elem<T>::load(Ws + (c + k) * 32 + lane);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 x = *reinterpret_cast<const float4 *>(h4 + q * a.GD + c);
+          acc[q] = fmaf(x.x, w[0], acc[q]);
+          acc[q] = fmaf(x.y, w[1], acc[q]);
+          acc[q] = fmaf(x.z, w[2], acc[q]);
+          acc[q] = fmaf(x.w, w[3], acc[q]);
+        }
+      }
+      const int i = i0 + lane;
+      if (i < h) {
+        const float gm = gamma ? gamma[i] : 0.f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int tt = t0 + warp * 4 + q;
+          if (tt < a.n) {
+            const size_t o = ((size_t)b * h + i) * a.n + tt;
+            if (scores) scores[o] = acc[q];
+            flags[o] = (acc[q] + gm) > logit_tau ? 1 : 0;
+          }
+        }
+      }
     }
   }
 }
