@@ -3,7 +3,9 @@
 // projection [Q' | K' | V'] = X [Wq_g | Wk_g | Wv_g] (Sec. 3.3, MHA').
 //
 // One CTA computes a 128 x BN tile of the packed output.  Warp 0 drives TMA,
-// warp 1 owns TMEM and issues the MMAs, warps 2..5 drain the accumulator.
+// warp 1 owns TMEM and issues the MMAs, warps 2..5 drain the accumulator: the
+// float32 form straight to global memory, the hi / lo bf16 form through the
+// (by then free) operand stages and TMA stores, which write whole 128-byte lines.
 //   A = X   [M, K]  row-major  -> K-major operand, 128-byte swizzled rows
 //   B = W   [K, GD] row-major  -> MN-major operand: panels of [64 k][64 n]
 // Products of bf16 inputs are exact in the f32 accumulator, so the result
@@ -30,8 +32,8 @@ template <int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                     const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
-                    float *__restrict__ C, __nv_bfloat16 *__restrict__ Chi, __nv_bfloat16 *__restrict__ Clo,
-                    int M, int K, int GD) {
+                    const __grid_constant__ CUtensorMap tmChi, const __grid_constant__ CUtensorMap tmClo,
+                    float *__restrict__ C, bool split, int M, int K, int GD) {
   using Cfg = GemmTcCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -110,34 +112,57 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int row = m0 + quad * 32 + lane;
     const bool ok = mbar_wait(acc_full, 0);
     tc_fence_after_sync();
-    if (ok && num_kb > 0) {
+    if (ok && num_kb > 0 && split) {
+      // x = hi + lo in bf16 pairs, for consumers that rebuild float32 precision from three
+      // products.  Every MMA has completed, so every stage has been read: the tile is staged
+      // over them as panels of [128 rows][64 bf16] (128-byte rows, 16-byte chunks XOR-swizzled by
+      // the row, the layout of a swizzled TMA store): hi panels first, then lo panels.
+      static_assert(2 * (BN / 64) * kTcBM * 128 <= Cfg::kStages * Cfg::kStageBytes, "staging fits the stages");
+      const int r_in = quad * 32 + lane;
+      uint8_t *stage_lo = smem + (BN / 64) * kTcBM * 128;
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 32) {
+        uint32_t r[32];
+        tmem_ld_x32_sync(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
+        const uint32_t panel = (uint32_t)(c >> 6) * kTcBM * 128 + r_in * 128;
+#pragma unroll
+        for (int e = 0; e < 32; e += 8) {
+          uint32_t h[4], l[4];
+#pragma unroll
+          for (int q = 0; q < 8; q += 2) {
+            float h0, l0, h1, l1;
+            split_bf16(__uint_as_float(r[e + q]), h0, l0);
+            split_bf16(__uint_as_float(r[e + q + 1]), h1, l1);
+            h[q >> 1] = pack_bf16x2(h0, h1);
+            l[q >> 1] = pack_bf16x2(l0, l1);
+          }
+          const uint32_t chunk = (uint32_t)(((c & 32) >> 3) + (e >> 3));          // 16-byte chunk within the 128-byte row
+          const uint32_t off = panel + ((chunk ^ (r_in & 7)) << 4);
+          *reinterpret_cast<uint4 *>(smem + off) = make_uint4(h[0], h[1], h[2], h[3]);
+          *reinterpret_cast<uint4 *>(stage_lo + off) = make_uint4(l[0], l[1], l[2], l[3]);
+        }
+      }
+      fence_proxy_async_smem();
+      named_barrier_sync(1, 128);
+      if (threadIdx.x == 64) {
+#pragma unroll
+        for (int p = 0; p < BN / 64; ++p) {            // rows past M are dropped by the tensor map
+          tma_store_2d(&tmChi, smem + p * kTcBM * 128, n0 + p * 64, m0);
+          tma_store_2d(&tmClo, stage_lo + p * kTcBM * 128, n0 + p * 64, m0);
+        }
+        tma_store_commit();
+        tma_store_wait_read();
+      }
+    } else if (ok && num_kb > 0) {
       const size_t crow = (size_t)row * 3 * GD + n0;
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
         uint32_t r[32];
         tmem_ld_x32_sync(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
         if (row < M) {
-          if (Chi) {
-            // x = hi + lo in bf16 pairs, for consumers that rebuild float32 precision from three products
 #pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-              uint32_t h[4], l[4];
-#pragma unroll
-              for (int q = 0; q < 8; q += 2) {
-                float h0, l0, h1, l1;
-                split_bf16(__uint_as_float(r[e + q]), h0, l0);
-                split_bf16(__uint_as_float(r[e + q + 1]), h1, l1);
-                h[q >> 1] = pack_bf16x2(h0, h1);
-                l[q >> 1] = pack_bf16x2(l0, l1);
-              }
-              *reinterpret_cast<uint4 *>(Chi + crow + c + e) = make_uint4(h[0], h[1], h[2], h[3]);
-              *reinterpret_cast<uint4 *>(Clo + crow + c + e) = make_uint4(l[0], l[1], l[2], l[3]);
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < 32; e += 4)
-              *reinterpret_cast<uint4 *>(C + crow + c + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
-          }
+          for (int e = 0; e < 32; e += 4)
+            *reinterpret_cast<uint4 *>(C + crow + c + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
         }
       }
     }
@@ -208,10 +233,18 @@ static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void
     rc = make_tmap_2d_bf16(&tmB[i], Ws[i], K, GD, (uint64_t)GD * 2, kTcBK, 64);
     if (rc) return rc;
   }
+  // output maps of the hi / lo form (one row of a weight stands in when that form is not asked for)
+  CUtensorMap tmC[2];
+  const void *outs[2] = {Chi ? (const void *)Chi : W0, Clo ? (const void *)Clo : W0};
+  for (int i = 0; i < 2; ++i) {
+    rc = Chi ? make_tmap_2d_bf16(&tmC[i], outs[i], M, 3 * (uint64_t)GD, 3 * (uint64_t)GD * 2, kTcBM, 64)
+             : make_tmap_2d_bf16(&tmC[i], outs[i], 1, GD, (uint64_t)GD * 2, 1, 64);
+    if (rc) return rc;
+  }
   auto kern = gemm_bf16_tc_kernel<BN>;
   AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
   dim3 grid(3 * GD / BN, (M + kTcBM - 1) / kTcBM);
-  kern<<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(tmA, tmB[0], tmB[1], tmB[2], C, Chi, Clo, M, K, GD);
+  kern<<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(tmA, tmB[0], tmB[1], tmB[2], tmC[0], tmC[1], C, Chi != nullptr, M, K, GD);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
