@@ -41,8 +41,9 @@ WORKLOADS = {
 # captures summarised under profiles/ (None for workloads that were not captured).  To be reset to
 # None whenever the kernel changes after the capture.
 TRAFFIC = {
-    ("prefill7b", "prefill"): 155.06e6 + 17.77e6,        # prefill_tc_kernel<64>
-    ("decode_ragged", "decode"): 2.3529e9 + 6.9e6,       # decode_partial_kernel<bf16,128>
+    ("prefill7b", "prefill"): 154.94e6 + 17.27e6,        # prefill_tc_kernel<64>
+    ("prefill7b", "decode"): 41.21e6 + 0.02e6,           # decode_cluster_kernel<bf16,128,512>
+    ("decode_ragged", "decode"): 2.3530e9 + 7.1e6,       # decode_partial_kernel<bf16,128>
 }
 # kernels launched per call of the library
 # (decode: one cluster kernel up to DECODE_CLUSTER_MAX_SLABS slabs, else chunk pass + merge)

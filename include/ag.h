@@ -208,7 +208,9 @@ int ag_cache_append(const ag_layer_desc *desc, const void *k_new,
  * This variant computes exactly what ag_decode_attn computes, with the
  * workspace replaced by a fixed 17,039,360-byte array that is part of the
  * library image (every GPU that loads the library holds it until the process
- * exits).  It calls no allocation routine of any kind.
+ * exits).  It calls no allocation routine of any kind.  (Up to 64 slabs
+ * neither the workspace nor the array is touched: that form of the kernel
+ * keeps its partial results on chip.)
  *
  *  - Limit: batch * heads * 32 * (head_dim + 2) * 4 bytes must fit in the
  *    array, i.e. batch * heads <= 1024 at head_dim 128 (2016 at head_dim 64).
