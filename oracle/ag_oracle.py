@@ -106,6 +106,22 @@ def gate_flags(scores, gamma, tau):
     return (p > tau).astype(np.uint8)
 
 
+def linear_gate_scores(X, W_lin):
+    """The local gate of Sec. 3.4 ("Local or global?"; ablation setting (5)):
+    MHA' is replaced by one linear layer, so a token's score depends on its own
+    hidden state only: s[b, i, t] = X[b, t, :] . W_lin[:, i].
+    X [B, n, d], W_lin [d, h] -> scores [B, h, n]."""
+    X = _as_f64(X)
+    W = _as_f64(W_lin)
+    return np.stack([(X[b] @ W).T for b in range(X.shape[0])], axis=0)
+
+
+def linear_gate(X, W_lin, gamma, tau):
+    """Flags of the local gate: the threshold of Eq. 4 on linear_gate_scores."""
+    s = linear_gate_scores(X, W_lin)
+    return s, gate_flags(s, gamma, tau)
+
+
 def attention_gate(X, Wq_g, Wk_g, Wv_g, Wo_g, gate_heads, gamma, tau, causal=True):
     """AG(X) = G(MHA'(X), tau), Eq. 3.  Returns (scores, flags)."""
     s = gate_scores(X, Wq_g, Wk_g, Wv_g, Wo_g, gate_heads, causal)

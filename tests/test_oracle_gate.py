@@ -112,3 +112,49 @@ def test_keep_count_grows_with_gamma():
     s = orc.gate_scores(X[None], Wq, Wk, Wv, Wo, 2)
     counts = [int(orc.gate_flags(s, g, 0.5).sum()) for g in (-5.0, -0.5, 0.0, 0.5, 5.0)]
     assert counts == sorted(counts) and counts[0] == 0 and counts[-1] == s.size
+
+
+# ---- the local (linear) gate of Sec. 3.4, "Local or global?" / ablation setting (5)
+
+def test_linear_gate_unit_rows_pick_rows_of_the_weight():
+    """A token whose hidden state is the unit vector e_k scores W_lin[k, :] exactly."""
+    d, h = 7, 3
+    W = _w((d, h), 40)
+    s = orc.linear_gate_scores(np.eye(d)[None], W)            # token t = e_t
+    assert s.shape == (1, h, d)
+    assert np.array_equal(s[0], W.T)
+
+
+def test_linear_gate_python_loops_tiny():
+    B, n, d, h = 2, 5, 4, 3
+    X, W = _w((B, n, d), 41), _w((d, h), 42)
+    ref = np.zeros((B, h, n))
+    for b in range(B):
+        for t in range(n):
+            for i in range(h):
+                acc = 0.0
+                for k in range(d):
+                    acc += X[b, t, k] * W[k, i]
+                ref[b, i, t] = acc
+    assert np.allclose(orc.linear_gate_scores(X, W), ref, rtol=0, atol=1e-14)
+
+
+def test_linear_gate_is_local_and_linear():
+    """A token's score ignores every other token (the opposite of MHA'), and scores add over inputs."""
+    n, d, h = 9, 6, 4
+    X, Y, W = _w((1, n, d), 43), _w((1, n, d), 44), _w((d, h), 45)
+    s = orc.linear_gate_scores(X, W)
+    X2 = X.copy()
+    X2[0, 3] += 10.0
+    s2 = orc.linear_gate_scores(X2, W)
+    keep = np.arange(n) != 3
+    assert np.array_equal(s[:, :, keep], s2[:, :, keep]) and not np.allclose(s[:, :, 3], s2[:, :, 3])
+    assert np.allclose(orc.linear_gate_scores(X + 2 * Y, W), s + 2 * orc.linear_gate_scores(Y, W), atol=1e-12)
+
+
+def test_linear_gate_flags_follow_eq4():
+    X, W = _w((1, 6, 3), 46), _w((3, 2), 47)
+    gamma, tau = np.array([0.3, -0.2]), 0.6
+    s, f = orc.linear_gate(X, W, gamma, tau)
+    want = 1.0 / (1.0 + np.exp(-(s + gamma[None, :, None]))) > tau
+    assert np.array_equal(f, want.astype(np.uint8)) and f.dtype == np.uint8
