@@ -219,6 +219,13 @@ class LayerRun:
         ag.ag_gate_forward(self.desc, self.X, W["Wq_g"], W["Wk_g"], W["Wv_g"], W["Wo_g"], self.gamma,
                            self.scores, self.flags, self.ws[ag.AG_CALL_GATE])
 
+    def gate_linear(self):
+        """The local gate (Sec. 3.4): same X, one [d, h] weight; timed on its own, not part of a step."""
+        if not hasattr(self, "W_lin"):
+            self.W_lin = inputs.linear_gate_weight(self.shape, 2900, self.X.device)
+            self.flags_lin = torch.empty_like(self.flags)
+        self.ag.ag_gate_linear_forward(self.desc, self.X, self.W_lin, None, self.scores, self.flags_lin)
+
     def compact(self):
         ag = self.ag
         ag.ag_compact_kv(self.desc, self.K, self.V, self.flags, self.cache, self.prefix, None, self.status,
@@ -444,6 +451,25 @@ def run_ours(args, rank, world, dev):
         rooflines["gate"] = {"bound": "tensor", "kernel": "ag_gate_forward", "achieved": tf, "peak": peaks["bf16_tflops"],
                              "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "traffic": None,
                              "peak_source": peaks["source"], "algorithmic_flops": gf, "ms": per_call_ms["gate"]}
+        # the local gate variant, timed apart from the step (L2 flushed before each call)
+        lin_ev = []
+        for i in range(3 + min(args.steps, 20)):
+            flush_l2(l2buf)
+            s_, e_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s_.record()
+            run.gate_linear()
+            e_.record()
+            if i >= 3:
+                lin_ev.append((s_, e_))
+        torch.cuda.synchronize()
+        lin_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in lin_ev]))
+        e = 2 if sh.dtype == "bf16" else 4
+        lb = float(sh.batch * sh.seq * sh.hidden * e + sh.hidden * sh.heads * e + sh.batch * sh.heads * sh.seq * 5)
+        gbs = lb / (lin_ms * 1e-3) / 1e9
+        rooflines["gate_linear"] = {"bound": "hbm", "kernel": "ag_gate_linear_forward (not part of the step)",
+                                    "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                    "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                                    "algorithmic_bytes": lb, "ms": lin_ms}
     for k, r in rooflines.items():
         r["traffic"] = TRAFFIC.get((args.workload, k))
     head = "prefill" if run.has_prefill else "decode"

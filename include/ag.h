@@ -123,6 +123,28 @@ int ag_gate_forward(const ag_layer_desc *desc, const void *X, const void *Wq_g,
                     size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Step 1, local variant — the gate with MHA' replaced by one linear layer
+ * (Sec. 3.4, "Local or global?"; ablation setting (5)): a token's flag depends
+ * on its own hidden state only.
+ *   s = X W_lin                                       (n x h);
+ *   flag[t, i] = 1 iff Sigmoid(s[t, i] + gamma[i]) > tau   (strict),
+ * compared as s + gamma > log(tau / (1 - tau)) in float32, like ag_gate_forward.
+ * Uses desc->batch, seq, hidden, heads, tau, dtype; the gate_* fields are ignored.
+ * Needs no workspace.  Its flags feed ag_compact_kv and the later steps unchanged.
+ *
+ *   X      [B, n, d]                 in
+ *   W_lin  [d, h]                    in   ("in x out")
+ *   gamma  [h] float32 or NULL (= 0) in
+ *   scores [B, h, n] float32 or NULL out  s, head-major
+ *   flags  [B, h, n] uint8           out
+ * Returns AG_ERR_INVALID_ARG for missing or misaligned (16-byte) pointers or a
+ * tau outside (0, 1); AG_ERR_CUDA if a launch fails.
+ */
+int ag_gate_linear_forward(const ag_layer_desc *desc, const void *X, const void *W_lin,
+                           const float *gamma, float *scores, uint8_t *flags,
+                           void *cuda_stream);
+
+/*
  * Step 2 — selective caching (Sec. 3.3: k_i^(t), v_i^(t) are retained iff
  * AG(X)_i^(t) = 1).  For every slab s = (b, i):
  *   prefix[s, j] = #{t < j : flags[s, t] = 1}, j = 0..n  (prefix[s, n] = L_s);

@@ -21,7 +21,7 @@ AG_DEV_OVERFLOW = 1
 EXPORTS = (
     "ag_workspace_bytes", "ag_gate_forward", "ag_compact_kv", "ag_prefill_attn",
     "ag_decode_attn", "ag_cache_append", "ag_status_string", "ag_last_cuda_error",
-    "ag_decode_attn_noalloc", "ag_device_wait_timeouts",
+    "ag_decode_attn_noalloc", "ag_device_wait_timeouts", "ag_gate_linear_forward",
 )
 
 
@@ -66,6 +66,8 @@ def lib():
         L.ag_workspace_bytes.argtypes = [dp, i32]
         L.ag_gate_forward.restype = i32
         L.ag_gate_forward.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.ag_gate_linear_forward.restype = i32
+        L.ag_gate_linear_forward.argtypes = [dp, vp, vp, vp, vp, vp, vp]
         L.ag_compact_kv.restype = i32
         L.ag_compact_kv.argtypes = [dp, vp, vp, vp, cp, vp, vp, vp, vp, sz, vp]
         L.ag_prefill_attn.restype = i32
@@ -169,6 +171,11 @@ def ag_gate_forward(desc, X, Wq_g, Wk_g, Wv_g, Wo_g, gamma, scores, flags, ws, s
     return _check(lib().ag_gate_forward(ctypes.byref(desc), _ptr(X), _ptr(Wq_g), _ptr(Wk_g), _ptr(Wv_g),
                                         _ptr(Wo_g), _ptr(gamma), _ptr(scores), _ptr(flags), p, nbytes,
                                         _stream(stream)), "ag_gate_forward")
+
+
+def ag_gate_linear_forward(desc, X, W_lin, gamma, scores, flags, stream=None):
+    return _check(lib().ag_gate_linear_forward(ctypes.byref(desc), _ptr(X), _ptr(W_lin), _ptr(gamma), _ptr(scores),
+                                               _ptr(flags), _stream(stream)), "ag_gate_linear_forward")
 
 
 def ag_compact_kv(desc, K, V, flags, cache, prefix, idx, dev_status, ws, stream=None):

@@ -86,6 +86,17 @@ int ag_gate_forward(const ag_layer_desc *desc, const void *X, const void *Wq_g,
                      (cudaStream_t)cuda_stream);
 }
 
+int ag_gate_linear_forward(const ag_layer_desc *desc, const void *X, const void *W_lin,
+                           const float *gamma, float *scores, uint8_t *flags, void *cuda_stream) {
+  int st = check_desc(desc);
+  if (st) return st;
+  if (desc->hidden <= 0 || !(desc->tau > 0.f && desc->tau < 1.f)) return AG_ERR_INVALID_ARG;
+  if (!X || !W_lin || !flags) return AG_ERR_INVALID_ARG;
+  if (misaligned16(X) || misaligned16(W_lin) || misaligned16(flags) || misaligned16(scores) || misaligned16(gamma))
+    return AG_ERR_INVALID_ARG;
+  return launch_gate_linear(*desc, X, W_lin, gamma, scores, flags, (cudaStream_t)cuda_stream);
+}
+
 int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
                   const uint8_t *flags, ag_cache *cache, int32_t *prefix,
                   int32_t *idx, int32_t *dev_status, void *ws, size_t ws_bytes,
@@ -174,7 +185,8 @@ int ag_last_cuda_error(void) { return ag::g_last_cuda_error; }
 
 int ag_device_wait_timeouts(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return -1;
-  const int a = gemm_tc_wait_timeouts(), b = prefill_tc_wait_timeouts(), c = gate_attn_tc_wait_timeouts();
+  const int a = gemm_tc_wait_timeouts(), b = prefill_tc_wait_timeouts(),
+            c = gate_attn_tc_wait_timeouts() + gate_linear_wait_timeouts();
   return (a < 0 || b < 0 || c < 0) ? -1 : a + b + c;
 }
 

@@ -52,6 +52,10 @@ int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *
                         const void *Wo, const float *gamma, float logit_tau, float *scores, uint8_t *flags,
                         cudaStream_t st);
 int gate_attn_tc_wait_timeouts();
+// The local gate of Sec. 3.4: s = X W_lin and the threshold of Eq. 4.
+int launch_gate_linear(const ag_layer_desc &d, const void *X, const void *W, const float *gamma,
+                       float *scores, uint8_t *flags, cudaStream_t st);
+int gate_linear_wait_timeouts();
 int gemm_tc_wait_timeouts();
 
 size_t compact_workspace_bytes(const ag_layer_desc &d);

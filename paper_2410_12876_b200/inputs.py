@@ -81,6 +81,11 @@ def layer_weights(shape, seed, device="cpu"):
     }
 
 
+def linear_gate_weight(shape, seed, device="cpu"):
+    """W_lin [d, h] ~ N(0, 1/d) for the local gate (scores of O(1) for unit-variance hidden states)."""
+    return randn((shape.hidden, shape.heads), seed, device, shape.torch_dtype, 1.0 / math.sqrt(shape.hidden))
+
+
 def project_qkv(shape, X, W):
     """Upstream projection Q_i = X W^Q_i etc. -> three [B, h, n, D] tensors in
     the layer dtype.  float64 accumulate for the fp32 layer, float32 otherwise."""
