@@ -320,13 +320,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       l = l * alpha + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
       m = m_new;
 
-      // P V completions alternate between two barriers, so the wait that keeps this
-      // thread in step with their phases is for tile i - 2, long finished; only a
-      // rescale of O has to wait for the P V of tile i - 1 itself.
-      if (i >= 2) {
-        ok = mbar_wait(&pv_done[st], ((i - 2) >> 1) & 1);
-        if (!ok) break;
-      }
+      // Only a rescale of O has to wait for the P V of tile i - 1.  The parity wait is unambiguous
+      // although this thread has not watched every phase of that barrier: the P V of tile i - 3
+      // (the barrier's previous phase) completed before the Q K^T of tile i - 1 was issued, whose
+      // scores this thread has already used, and the P V of tile i + 1 cannot have been issued yet.
       if (rescale) {
         ok = mbar_wait(&pv_done[(i - 1) & 1], ((i - 1) >> 1) & 1);
         if (!ok) break;
