@@ -47,7 +47,7 @@ TRAFFIC = {
 }
 # kernels launched per call of the library
 # (decode: one cluster kernel up to DECODE_CLUSTER_MAX_SLABS slabs, else chunk pass + merge)
-LAUNCHES = {"gate": 3, "compact": 2, "prefill": 1, "decode": 2, "append": 1}
+LAUNCHES = {"gate": 3, "compact": 1, "prefill": 1, "decode": 2, "append": 1}
 DECODE_CLUSTER_MAX_SLABS = 64
 
 

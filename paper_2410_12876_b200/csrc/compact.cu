@@ -2,102 +2,117 @@
 // v_i^(t) are retained iff AG(X)_i^(t) = 1) and the conditional append of the
 // decoding stage (Sec. 3.1).
 //
-//   scan_flags_kernel   one CTA per slab: warp ballot + popc per 32-token
-//                       word, shuffle scan across the warps of the CTA,
-//                       running carry across 1024-token chunks.
-//   gather_rows_kernel  destination-ordered 16-byte-vector row moves: only
-//                       retained rows are read, every access is a full row.
+//   compact_kernel   one CTA per 256 tokens of a slab.  It counts the flags of the whole slab row
+//                    (a few KB, read as 16-byte vectors) to get the number of retained tokens
+//                    before its chunk and in the slab, ranks its own tokens by warp ballot +
+//                    popc, writes prefix and idx for them, and moves the retained rows of its
+//                    chunk: 16-byte-vector row moves, only retained rows are read, every access
+//                    is a full row.  One launch; no pass over the flags on its own.
 #include "ag_common.cuh"
 
 namespace ag {
 
-constexpr int kScanThreads = 1024;
+constexpr int kCompactThreads = 256;   // = tokens per CTA
 
-__global__ void __launch_bounds__(kScanThreads)
-scan_flags_kernel(const uint8_t *__restrict__ flags, int n, const int32_t *__restrict__ cap,
-                  int32_t *__restrict__ len, int32_t *__restrict__ prefix,
-                  int32_t *__restrict__ idx, int32_t *__restrict__ dev_status, int check_cap) {
-  const int slab = blockIdx.x;
+// Bytes of a 32-bit word that are not zero.
+__device__ __forceinline__ int nonzero_bytes(uint32_t w) { return __popc(__vcmpne4(w, 0u) & 0x01010101u); }
+
+// One row = D * sizeof(T) bytes = kVecs 16-byte vectors; a group of kVecs consecutive lanes moves
+// one row of K and one row of V.  kRowBytes = 0: count pass, no rows move.
+template <int kRowBytes>
+__global__ void __launch_bounds__(kCompactThreads)
+compact_kernel(const uint8_t *__restrict__ flags, int n, const int32_t *__restrict__ cap,
+               int32_t *__restrict__ len, int32_t *__restrict__ prefix, int32_t *__restrict__ idx,
+               int32_t *__restrict__ dev_status, const uint8_t *__restrict__ K,
+               const uint8_t *__restrict__ V, const int64_t *__restrict__ row_off,
+               uint8_t *__restrict__ k_rows, uint8_t *__restrict__ v_rows) {
+  const int slab = blockIdx.y, t0 = blockIdx.x * kCompactThreads;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint8_t *f = flags + (size_t)slab * n;
-  int32_t *pre = prefix + (size_t)slab * (n + 1);
-  int32_t *ix = idx + (size_t)slab * n;
-  __shared__ int warp_excl[32];
-  __shared__ int chunk_total;
-  int carry = 0;
-  for (int base = 0; base < n; base += kScanThreads) {
-    const int t = base + threadIdx.x;
-    const bool keep = (t < n) && (f[t] != 0);
-    const unsigned word = __ballot_sync(0xffffffffu, keep);
-    const int in_warp = __popc(word & ((1u << lane) - 1u));
-    if (lane == 0) warp_excl[warp] = __popc(word);
-    __syncthreads();
-    if (warp == 0) {
-      const int c = warp_excl[lane];
-      int inc = c;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        int v = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += v;
-      }
-      warp_excl[lane] = inc - c;
-      if (lane == 31) chunk_total = inc;
-    }
-    __syncthreads();
-    const int p = carry + warp_excl[warp] + in_warp;
-    if (t < n) {
-      pre[t] = p;
-      if (keep) ix[p] = t;
-    }
-    carry += chunk_total;
-    __syncthreads();
-  }
-  if (threadIdx.x == 0) {
-    pre[n] = carry;
-    if (check_cap && carry > cap[slab]) {
-      len[slab] = 0;
-      if (dev_status) atomicOr(dev_status, AG_DEV_OVERFLOW);
-    } else {
-      len[slab] = carry;
-    }
-  }
-}
+  __shared__ int red_before[kCompactThreads / 32], red_total[kCompactThreads / 32];
+  __shared__ int warp_excl[kCompactThreads / 32];
+  __shared__ int tok_list[kCompactThreads];
 
-// One row = D * sizeof(T) bytes = kVecs 16-byte vectors; a group of kVecs
-// consecutive lanes moves one row of K and one row of V.
-template <int kRowBytes>
-__global__ void __launch_bounds__(256)
-gather_rows_kernel(const uint8_t *__restrict__ K, const uint8_t *__restrict__ V, int n,
-                   const int32_t *__restrict__ idx, const int32_t *__restrict__ len,
-                   const int64_t *__restrict__ row_off, uint8_t *__restrict__ k_rows,
-                   uint8_t *__restrict__ v_rows, int rows_per_cta) {
-  constexpr int kVecs = kRowBytes / 16;
-  constexpr int kGroups = 256 / kVecs;
-  const int slab = blockIdx.y;
-  const int L = len[slab];
-  const int r0 = blockIdx.x * rows_per_cta;
-  if (r0 >= L) return;
-  const int r1 = min(L, r0 + rows_per_cta);
+  // retained tokens before this chunk, and in the slab
+  int before = 0, total = 0;
+  if ((n & 15) == 0) {                       // rows of the flag array start on 16-byte boundaries
+    const uint4 *fv = reinterpret_cast<const uint4 *>(f);
+    for (int x = threadIdx.x; x < n / 16; x += kCompactThreads) {
+      const uint4 w = ldg128(fv + x);
+      const int c = nonzero_bytes(w.x) + nonzero_bytes(w.y) + nonzero_bytes(w.z) + nonzero_bytes(w.w);
+      total += c;
+      if (x * 16 < t0) before += c;          // t0 is a multiple of 16: a vector lies on one side
+    }
+  } else {
+    for (int x = threadIdx.x; x < n; x += kCompactThreads) {
+      const int c = f[x] != 0;
+      total += c;
+      if (x < t0) before += c;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    before += __shfl_xor_sync(0xffffffffu, before, o);
+    total += __shfl_xor_sync(0xffffffffu, total, o);
+  }
+  // this chunk's tokens
+  const int t = t0 + threadIdx.x;
+  const bool keep = (t < n) && (f[t] != 0);
+  const unsigned word = __ballot_sync(0xffffffffu, keep);
+  const int in_warp = __popc(word & ((1u << lane) - 1u));
+  if (lane == 0) { red_before[warp] = before; red_total[warp] = total; warp_excl[warp] = __popc(word); }
+  __syncthreads();
+  before = 0; total = 0;
+  int excl = 0, count = 0;
+#pragma unroll
+  for (int w = 0; w < kCompactThreads / 32; ++w) {
+    before += red_before[w];
+    total += red_total[w];
+    if (w < warp) excl += warp_excl[w];
+    count += warp_excl[w];
+  }
+  const int local = excl + in_warp;          // rank within the chunk
+  const int p = before + local;              // rank within the slab
+  int32_t *pre = prefix + (size_t)slab * (n + 1);
+  if (t < n) {
+    pre[t] = p;
+    if (keep) {
+      idx[(size_t)slab * n + p] = t;
+      tok_list[local] = t;
+    }
+  }
+  const bool overflow = kRowBytes != 0 && total > cap[slab];
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    pre[n] = total;
+    len[slab] = overflow ? 0 : total;
+    if (overflow && dev_status) atomicOr(dev_status, AG_DEV_OVERFLOW);
+  }
+  if (kRowBytes == 0 || overflow) return;    // count pass, or a slab that does not fit: nothing moves
+  __syncthreads();
+
+  constexpr int kVecs = kRowBytes > 0 ? kRowBytes / 16 : 1;
+  constexpr int kGroups = kCompactThreads / kVecs;
   const int g = threadIdx.x / kVecs, v = threadIdx.x % kVecs;
-  const int32_t *ix = idx + (size_t)slab * n;
   const uint8_t *Ks = K + (size_t)slab * n * kRowBytes;
   const uint8_t *Vs = V + (size_t)slab * n * kRowBytes;
-  const size_t dst0 = (size_t)row_off[slab] * kRowBytes;
-  // two rows per group in flight
-  for (int r = r0 + g; r < r1; r += 2 * kGroups) {
-    const int ra = r, rb = r + kGroups;
-    const int ta = ix[ra];
-    const bool has_b = rb < r1;
-    const int tb = has_b ? ix[rb] : ta;
-    uint4 ka = ldg128_stream(Ks + (size_t)ta * kRowBytes + v * 16);
-    uint4 va = ldg128_stream(Vs + (size_t)ta * kRowBytes + v * 16);
-    uint4 kb = ldg128_stream(Ks + (size_t)tb * kRowBytes + v * 16);
-    uint4 vb = ldg128_stream(Vs + (size_t)tb * kRowBytes + v * 16);
-    *reinterpret_cast<uint4 *>(k_rows + dst0 + (size_t)ra * kRowBytes + v * 16) = ka;
-    *reinterpret_cast<uint4 *>(v_rows + dst0 + (size_t)ra * kRowBytes + v * 16) = va;
-    if (has_b) {
-      *reinterpret_cast<uint4 *>(k_rows + dst0 + (size_t)rb * kRowBytes + v * 16) = kb;
-      *reinterpret_cast<uint4 *>(v_rows + dst0 + (size_t)rb * kRowBytes + v * 16) = vb;
+  const size_t dst0 = ((size_t)row_off[slab] + before) * kRowBytes;
+  // kFlight rows of K and of V per group in flight
+  constexpr int kFlight = 2;
+  for (int j = g; j < count; j += kFlight * kGroups) {
+    uint4 kv[kFlight], vv[kFlight];
+#pragma unroll
+    for (int u = 0; u < kFlight; ++u) {
+      const int tu = tok_list[min(j + u * kGroups, count - 1)];
+      kv[u] = ldg128_stream(Ks + (size_t)tu * kRowBytes + v * 16);
+      vv[u] = ldg128_stream(Vs + (size_t)tu * kRowBytes + v * 16);
+    }
+#pragma unroll
+    for (int u = 0; u < kFlight; ++u) {
+      const int ju = j + u * kGroups;
+      if (ju < count) {
+        *reinterpret_cast<uint4 *>(k_rows + dst0 + (size_t)ju * kRowBytes + v * 16) = kv[u];
+        *reinterpret_cast<uint4 *>(v_rows + dst0 + (size_t)ju * kRowBytes + v * 16) = vv[u];
+      }
     }
   }
 }
@@ -144,26 +159,23 @@ int launch_compact(const ag_layer_desc &d, const void *K, const void *V, const u
                    void *ws, cudaStream_t st) {
   const int slabs = d.batch * d.heads;
   int32_t *ix = idx ? idx : static_cast<int32_t *>(ws);
-  scan_flags_kernel<<<slabs, kScanThreads, 0, st>>>(flags, d.seq, c.cap, c.len, prefix, ix,
-                                                    dev_status, K != nullptr);
-  AG_LAUNCH_CHECK();
-  if (!K) return AG_OK;
-  const int rb = row_bytes(d);
-  const int rows_per_cta = 128;
-  dim3 grid((d.seq + rows_per_cta - 1) / rows_per_cta, slabs);
+  dim3 grid((d.seq + kCompactThreads - 1) / kCompactThreads, slabs);
   auto Kb = static_cast<const uint8_t *>(K);
   auto Vb = static_cast<const uint8_t *>(V);
   auto kr = static_cast<uint8_t *>(c.k_rows);
   auto vr = static_cast<uint8_t *>(c.v_rows);
-  switch (rb) {
+  switch (K ? row_bytes(d) : 0) {
+    case 0:
+      compact_kernel<0><<<grid, kCompactThreads, 0, st>>>(flags, d.seq, c.cap, c.len, prefix, ix, dev_status, Kb, Vb, c.row_off, kr, vr);
+      break;
     case 128:
-      gather_rows_kernel<128><<<grid, 256, 0, st>>>(Kb, Vb, d.seq, ix, c.len, c.row_off, kr, vr, rows_per_cta);
+      compact_kernel<128><<<grid, kCompactThreads, 0, st>>>(flags, d.seq, c.cap, c.len, prefix, ix, dev_status, Kb, Vb, c.row_off, kr, vr);
       break;
     case 256:
-      gather_rows_kernel<256><<<grid, 256, 0, st>>>(Kb, Vb, d.seq, ix, c.len, c.row_off, kr, vr, rows_per_cta);
+      compact_kernel<256><<<grid, kCompactThreads, 0, st>>>(flags, d.seq, c.cap, c.len, prefix, ix, dev_status, Kb, Vb, c.row_off, kr, vr);
       break;
     case 512:
-      gather_rows_kernel<512><<<grid, 256, 0, st>>>(Kb, Vb, d.seq, ix, c.len, c.row_off, kr, vr, rows_per_cta);
+      compact_kernel<512><<<grid, kCompactThreads, 0, st>>>(flags, d.seq, c.cap, c.len, prefix, ix, dev_status, Kb, Vb, c.row_off, kr, vr);
       break;
     default:
       return AG_ERR_UNSUPPORTED;
