@@ -46,8 +46,8 @@ TRAFFIC = {
     ("decode_ragged", "decode"): 2.3530e9 + 7.1e6,       # decode_partial_kernel<bf16,128>
 }
 # kernels launched per call of the library
-# (decode: one cluster kernel up to DECODE_CLUSTER_MAX_SLABS slabs, else chunk pass + merge)
-LAUNCHES = {"gate": 3, "compact": 1, "prefill": 1, "decode": 2, "append": 1}
+# (decode step, attention + append: one cluster kernel up to DECODE_CLUSTER_MAX_SLABS slabs, else chunk pass + merge)
+LAUNCHES = {"gate": 3, "compact": 1, "prefill": 1, "decode": 2}
 DECODE_CLUSTER_MAX_SLABS = 64
 
 
@@ -239,8 +239,8 @@ class LayerRun:
     def decode(self, s):
         ag = self.ag
         q, kn, vn, fn = self.dq[s]
-        ag.ag_decode_attn(self.desc, q, kn, vn, self.cache, 0.0, self.o, self.ws[ag.AG_CALL_DECODE])
-        ag.ag_cache_append(self.desc, kn, vn, fn, self.cache, self.status)
+        # attention + conditional append of the step in one call
+        ag.ag_decode_step(self.desc, q, kn, vn, fn, self.cache, 0.0, self.o, self.status, self.ws[ag.AG_CALL_DECODE])
 
     def step(self, ev=None):
         """One pass; ev (optional) = dict of lists of (start, end) CUDA events per call."""
@@ -290,7 +290,7 @@ class LayerRun:
     def launches_per_step(self):
         return self.layers * ((LAUNCHES["gate"] if self.has_gate else 0) +
                               (LAUNCHES["compact"] + LAUNCHES["prefill"] if self.has_prefill else 0) +
-                              self.decode_steps * (self.decode_launches() + LAUNCHES["append"]))
+                              self.decode_steps * self.decode_launches())
 
     def decode_launches(self):
         slabs = self.shape.batch * self.shape.heads
@@ -462,7 +462,7 @@ def run_ours(args, rank, world, dev):
     dec_bytes = work["decode_bytes"]
     dec_ms = per_call_ms["decode"] / run.decode_steps
     dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
-    rooflines["decode"] = {"bound": "hbm", "kernel": "ag_decode_attn + ag_cache_append", "achieved": dec_gbs,
+    rooflines["decode"] = {"bound": "hbm", "kernel": "ag_decode_step", "achieved": dec_gbs,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"],
                            "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": dec_bytes,
                            "ms": dec_ms}

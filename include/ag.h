@@ -10,6 +10,8 @@
  *   ag_prefill_attn   Softmax(QK^T/sqrt(d_k) - INF(1-M_i))V    Eq. 2 with M_i of Eq. 5
  *   ag_decode_attn    one query over the retained cache + self Sec. 3.1 (decoding stage), Eq. 5 (j = t)
  *   ag_cache_append   concatenate the new k, v to the cache    Sec. 3.1 (decoding stage)
+ *   ag_decode_step    the two above in one call                Sec. 3.1 (decoding stage)
+ *   ag_gate_linear_forward  the local gate, s = X W_lin        Sec. 3.4 ("Local or global?")
  *
  * Conventions common to every call
  * --------------------------------
@@ -214,6 +216,23 @@ int ag_decode_attn(const ag_layer_desc *desc, const void *q, const void *k_new,
 int ag_cache_append(const ag_layer_desc *desc, const void *k_new,
                     const void *v_new, const uint8_t *flag_new, ag_cache *cache,
                     int32_t *dev_status, void *cuda_stream);
+
+/*
+ * Steps 4a + 4b in one call (Sec. 3.1, decoding stage): the attention of
+ * ag_decode_attn over the cache as it stands, then the conditional append of
+ * ag_cache_append, carried by the same kernels (the slab's rows and length are
+ * read before the new row goes in, so o is exactly what ag_decode_attn gives
+ * and the cache ends exactly as ag_cache_append leaves it).  One decode step
+ * of a layer is one such call; it saves a launch per step.
+ *
+ *   q, k_new, v_new [B, h, D]  in      flag_new [B, h] uint8  in
+ *   o [B, h, D]  out                   dev_status int32 or NULL  in/out
+ * Workspace and errors as for ag_decode_attn (AG_CALL_DECODE).
+ */
+int ag_decode_step(const ag_layer_desc *desc, const void *q, const void *k_new,
+                   const void *v_new, const uint8_t *flag_new, ag_cache *cache,
+                   float softmax_scale, void *o, int32_t *dev_status, void *ws,
+                   size_t ws_bytes, void *cuda_stream);
 
 /*
  * ag_decode_attn without any caller-supplied scratch.  The paper has no

@@ -21,7 +21,7 @@ AG_DEV_OVERFLOW = 1
 EXPORTS = (
     "ag_workspace_bytes", "ag_gate_forward", "ag_compact_kv", "ag_prefill_attn",
     "ag_decode_attn", "ag_cache_append", "ag_status_string", "ag_last_cuda_error",
-    "ag_decode_attn_noalloc", "ag_device_wait_timeouts", "ag_gate_linear_forward",
+    "ag_decode_attn_noalloc", "ag_device_wait_timeouts", "ag_gate_linear_forward", "ag_decode_step",
 )
 
 
@@ -74,6 +74,8 @@ def lib():
         L.ag_prefill_attn.argtypes = [dp, vp, vp, vp, vp, cp, vp, f32, vp, vp, sz, vp]
         L.ag_decode_attn.restype = i32
         L.ag_decode_attn.argtypes = [dp, vp, vp, vp, cp, f32, vp, vp, sz, vp]
+        L.ag_decode_step.restype = i32
+        L.ag_decode_step.argtypes = [dp, vp, vp, vp, vp, cp, f32, vp, vp, vp, sz, vp]
         L.ag_decode_attn_noalloc.restype = i32
         L.ag_decode_attn_noalloc.argtypes = [dp, vp, vp, vp, cp, f32, vp, vp]
         L.ag_cache_append.restype = i32
@@ -207,6 +209,13 @@ def ag_decode_attn_noalloc(desc, q, k_new, v_new, cache, softmax_scale, o, strea
     return _check(lib().ag_decode_attn_noalloc(ctypes.byref(desc), _ptr(q), _ptr(k_new), _ptr(v_new),
                                                ctypes.byref(cache.struct), float(softmax_scale), _ptr(o),
                                                _stream(stream)), "ag_decode_attn_noalloc")
+
+
+def ag_decode_step(desc, q, k_new, v_new, flag_new, cache, softmax_scale, o, dev_status, ws, stream=None):
+    p, nbytes = _ws(ws)
+    return _check(lib().ag_decode_step(ctypes.byref(desc), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(flag_new),
+                                       ctypes.byref(cache.struct), float(softmax_scale), _ptr(o), _ptr(dev_status),
+                                       p, nbytes, _stream(stream)), "ag_decode_step")
 
 
 def ag_cache_append(desc, k_new, v_new, flag_new, cache, dev_status, stream=None):

@@ -156,6 +156,24 @@ int ag_decode_attn(const ag_layer_desc *desc, const void *q, const void *k_new,
                        (cudaStream_t)cuda_stream);
 }
 
+int ag_decode_step(const ag_layer_desc *desc, const void *q, const void *k_new, const void *v_new,
+                   const uint8_t *flag_new, ag_cache *cache, float softmax_scale, void *o,
+                   int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream) {
+  int st = check_desc(desc);
+  if (st) return st;
+  if (!q || !k_new || !v_new || !flag_new || !o) return AG_ERR_INVALID_ARG;
+  st = check_cache(cache);
+  if (st) return st;
+  if (misaligned16(q) || misaligned16(k_new) || misaligned16(v_new) || misaligned16(o))
+    return AG_ERR_INVALID_ARG;
+  if (!(softmax_scale >= 0.f) || isinf(softmax_scale)) return AG_ERR_INVALID_ARG;
+  st = check_ws(decode_workspace_bytes(*desc), ws, ws_bytes);
+  if (st) return st;
+  float scale = softmax_scale == 0.f ? 1.0f / sqrtf((float)desc->head_dim) : softmax_scale;
+  return launch_decode_step(*desc, q, k_new, v_new, flag_new, *cache, scale, o, dev_status, ws,
+                            (cudaStream_t)cuda_stream);
+}
+
 int ag_cache_append(const ag_layer_desc *desc, const void *k_new, const void *v_new,
                     const uint8_t *flag_new, ag_cache *cache, int32_t *dev_status,
                     void *cuda_stream) {

@@ -78,6 +78,9 @@ size_t decode_workspace_bytes(const ag_layer_desc &d);
 int launch_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
                   const ag_cache &c, float scale, void *o, void *ws, size_t ws_bytes,
                   cudaStream_t st);
+int launch_decode_step(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
+                       const uint8_t *flag_new, const ag_cache &c, float scale, void *o,
+                       int32_t *dev_status, void *ws, cudaStream_t st);
 int launch_append(const ag_layer_desc &d, const void *k_new, const void *v_new,
                   const uint8_t *flag_new, const ag_cache &c, int32_t *dev_status,
                   cudaStream_t st);

@@ -26,6 +26,35 @@ constexpr int kUnroll = 8;         // rows in flight per lane group (x2: K and V
 constexpr int kClusterMaxSlabs = 64;    // up to here one cluster per slab; beyond, split-K through the workspace
 constexpr int kClusterThreads = 512;    // 256 rows in flight per CTA of a cluster (bf16, D = 128)
 
+// The conditional append of the decoding stage (Sec. 3.1 with the gate's flag for the new token),
+// for kernels that carry it with the attention of the same step: flag_new = NULL means no append.
+struct AppendArgs {
+  const uint8_t *flag_new;   // [slabs] or NULL
+  const int32_t *cap;
+  int32_t *len;
+  void *k_rows, *v_rows;
+  int32_t *dev_status;
+};
+// Called by the threads [0, row vectors) of ONE CTA per slab, after every read of len[slab] and
+// of the slab's rows by this launch has completed.  L = the length those reads saw.
+template <typename T, int D>
+__device__ __forceinline__ void append_new_row(const AppendArgs &ap, int slab, int L, int64_t row0,
+                                               const T *__restrict__ k_new, const T *__restrict__ v_new) {
+  constexpr int kVecs = D * (int)sizeof(T) / 16;
+  if (ap.flag_new == nullptr || ap.flag_new[slab] == 0 || (int)threadIdx.x >= kVecs) return;
+  if (L >= ap.cap[slab]) {
+    if (threadIdx.x == 0 && ap.dev_status) atomicOr(ap.dev_status, AG_DEV_OVERFLOW);
+    return;
+  }
+  const size_t dst = ((size_t)row0 + L) * D * sizeof(T) + threadIdx.x * 16;
+  const size_t src = (size_t)slab * D * sizeof(T) + threadIdx.x * 16;
+  *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(ap.k_rows) + dst) =
+      *reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(k_new) + src);
+  *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(ap.v_rows) + dst) =
+      *reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(v_new) + src);
+  if (threadIdx.x == 0) ap.len[slab] = L + 1;
+}
+
 // Rows [r_begin, r_end) of one slab, streamed by a whole CTA of kThreads threads: thread (g, v) =
 // (row group, 16-byte slice of the row) ends with its group's running maximum m, sum l and slice
 // of o (log2 domain).
@@ -144,9 +173,12 @@ __global__ void __launch_bounds__(D)
 decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
                       const T *__restrict__ v_new, const int32_t *__restrict__ len,
                       float scale_log2, int chunk_rows, const float *__restrict__ part_o,
-                      const float *__restrict__ part_ml, T *__restrict__ o) {
+                      const float *__restrict__ part_ml, T *__restrict__ o,
+                      const int64_t *__restrict__ row_off, const AppendArgs ap) {
   const int slab = blockIdx.x, d = threadIdx.x;
   const int L = len[slab];
+  // the chunk pass, the only reader of the slab's rows, has completed: the new row may go in
+  append_new_row<T, D>(ap, slab, L, row_off[slab], k_new, v_new);
   const int n_chunks = (L + chunk_rows - 1) / chunk_rows;
   __shared__ float red[D / 32];
   float a = Elem<T>::load(q + (size_t)slab * D + d) * Elem<T>::load(k_new + (size_t)slab * D + d);
@@ -184,7 +216,7 @@ __global__ void __launch_bounds__(kThreads)
 decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, const T *__restrict__ v_new,
                       const T *__restrict__ k_rows, const T *__restrict__ v_rows,
                       const int64_t *__restrict__ row_off, const int32_t *__restrict__ len,
-                      float scale_log2, T *__restrict__ out) {
+                      float scale_log2, T *__restrict__ out, const AppendArgs ap) {
   namespace cg = cooperative_groups;
   constexpr int kEpl = Elem<T>::kPerVec;
   constexpr int kLanes = D / kEpl;
@@ -239,6 +271,8 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
     cta_ml[1] = lc;
   }
   cluster.sync();
+  // every CTA of the cluster has read the length and its rows: the new row may go in
+  if (rank == 0) append_new_row<T, D>(ap, slab, L, row_off[slab], k_new, v_new);
   if (rank == 0 && threadIdx.x < D) {
     const int d = threadIdx.x;
     float s_self = 0.f;
@@ -272,7 +306,8 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
 
 template <typename T, int D, int kThreads>
 static int launch_decode_cluster(int slabs, const void *q, const void *k_new, const void *v_new,
-                                 const ag_cache &c, float scale_log2, void *o, cudaStream_t st) {
+                                 const ag_cache &c, float scale_log2, void *o, const AppendArgs &ap,
+                                 cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(kClusterSize, slabs);
   cfg.blockDim = dim3(kThreads);
@@ -286,7 +321,7 @@ static int launch_decode_cluster(int slabs, const void *q, const void *k_new, co
   AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_cluster_kernel<T, D, kThreads>, static_cast<const T *>(q),
                                  static_cast<const T *>(k_new), static_cast<const T *>(v_new),
                                  static_cast<const T *>(c.k_rows), static_cast<const T *>(c.v_rows),
-                                 c.row_off, c.len, scale_log2, static_cast<T *>(o)));
+                                 c.row_off, c.len, scale_log2, static_cast<T *>(o), ap));
   return AG_OK;
 }
 
@@ -297,11 +332,11 @@ size_t decode_workspace_bytes(const ag_layer_desc &d) {
 
 template <typename T, int D>
 static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
-                      const ag_cache &c, float scale, void *o, void *ws, cudaStream_t st) {
+                      const ag_cache &c, float scale, void *o, void *ws, const AppendArgs &ap, cudaStream_t st) {
   const int slabs = d.batch * d.heads;
   const float scale_log2 = scale * 1.4426950408889634f;
   if (slabs <= kClusterMaxSlabs)
-    return launch_decode_cluster<T, D, kClusterThreads>(slabs, q, k_new, v_new, c, scale_log2, o, st);
+    return launch_decode_cluster<T, D, kClusterThreads>(slabs, q, k_new, v_new, c, scale_log2, o, ap, st);
   int chunk_rows = (c.max_cap + kMaxSplits - 1) / kMaxSplits;
   chunk_rows = (chunk_rows + 127) / 128 * 128;   // whole iterations of the partial kernel (bf16, D = 128)
   const int n_chunks = c.max_cap > 0 ? (c.max_cap + chunk_rows - 1) / chunk_rows : 0;
@@ -316,19 +351,35 @@ static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, 
   }
   decode_combine_kernel<T, D><<<slabs, D, 0, st>>>(
       static_cast<const T *>(q), static_cast<const T *>(k_new), static_cast<const T *>(v_new),
-      c.len, scale_log2, chunk_rows, part_o, part_ml, static_cast<T *>(o));
+      c.len, scale_log2, chunk_rows, part_o, part_ml, static_cast<T *>(o), c.row_off, ap);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
 
+static int dispatch_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
+                           const ag_cache &c, float scale, void *o, void *ws, const AppendArgs &ap,
+                           cudaStream_t st) {
+  if (d.dtype == AG_F32) {
+    if (d.head_dim == 64) return run_decode<float, 64>(d, q, k_new, v_new, c, scale, o, ws, ap, st);
+    return run_decode<float, 128>(d, q, k_new, v_new, c, scale, o, ws, ap, st);
+  }
+  if (d.head_dim == 64) return run_decode<__nv_bfloat16, 64>(d, q, k_new, v_new, c, scale, o, ws, ap, st);
+  return run_decode<__nv_bfloat16, 128>(d, q, k_new, v_new, c, scale, o, ws, ap, st);
+}
+
 int launch_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
                   const ag_cache &c, float scale, void *o, void *ws, size_t, cudaStream_t st) {
-  if (d.dtype == AG_F32) {
-    if (d.head_dim == 64) return run_decode<float, 64>(d, q, k_new, v_new, c, scale, o, ws, st);
-    return run_decode<float, 128>(d, q, k_new, v_new, c, scale, o, ws, st);
-  }
-  if (d.head_dim == 64) return run_decode<__nv_bfloat16, 64>(d, q, k_new, v_new, c, scale, o, ws, st);
-  return run_decode<__nv_bfloat16, 128>(d, q, k_new, v_new, c, scale, o, ws, st);
+  return dispatch_decode(d, q, k_new, v_new, c, scale, o, ws, AppendArgs{}, st);
+}
+
+// Attention of the step and the conditional append in the same launches.
+int launch_decode_step(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
+                       const uint8_t *flag_new, const ag_cache &c, float scale, void *o,
+                       int32_t *dev_status, void *ws, cudaStream_t st) {
+  AppendArgs ap;
+  ap.flag_new = flag_new; ap.cap = c.cap; ap.len = c.len;
+  ap.k_rows = c.k_rows; ap.v_rows = c.v_rows; ap.dev_status = dev_status;
+  return dispatch_decode(d, q, k_new, v_new, c, scale, o, ws, ap, st);
 }
 
 // ---------------------------------------------------------------------------

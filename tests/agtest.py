@@ -116,13 +116,17 @@ def gpu_prefill(shape, Q, K, V, flags, cache, prefix, scale=0.0):
     return O
 
 
-def gpu_decode_step(shape, q, kn, vn, fn, cache, status, ws=None, scale=0.0):
+def gpu_decode_step(shape, q, kn, vn, fn, cache, status, ws=None, scale=0.0, fused=False):
+    """One decode step: ag_decode_attn + ag_cache_append, or ag_decode_step (both in one call)."""
     desc = ag.make_desc(shape)
     if ws is None:
         ws = ag.workspace(desc, ag.AG_CALL_DECODE)
     o = torch.full_like(q, float("nan"))
-    ag.ag_decode_attn(desc, q, kn, vn, cache, scale, o, ws)
-    ag.ag_cache_append(desc, kn, vn, fn, cache, status)
+    if fused:
+        ag.ag_decode_step(desc, q, kn, vn, fn, cache, scale, o, status, ws)
+    else:
+        ag.ag_decode_attn(desc, q, kn, vn, cache, scale, o, ws)
+        ag.ag_cache_append(desc, kn, vn, fn, cache, status)
     return o
 
 

@@ -106,7 +106,7 @@ def test_deep_layer_pattern():
     for step in range(steps):
         q, kn, vn, fn = inputs.decode_inputs(shape, seed + 500, step, DEV, keep_new=0.1)
         fn[:, torch.from_numpy(empty).to(DEV)] = 0
-        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status)
+        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status, fused=True)
         T.check_close(T.f64(o), orc.decode_attention(T.f64(q), T.f64(kn), T.f64(vn), ocache), "bf16", f"decode {step}")
         for i in empty:
             assert torch.equal(o[0, i], vn[0, i])                      # empty slab: o = v_new

@@ -207,8 +207,9 @@ def test_tiny_layer_end_to_end():
         assert int(status.item()) == 0
 
 
+@pytest.mark.parametrize("fused", [False, True], ids=["two_calls", "one_call"])
 @pytest.mark.parametrize("name", ["bf16", "bf16_d64", "f32_d128"])
-def test_decode_and_append(name):
+def test_decode_and_append(name, fused):
     shape = SHAPES[name].with_(seq=700)
     Q, K, V = inputs.qkv_gaussian(shape, 400, DEV)
     flags = _flag_patterns(shape, 410)
@@ -219,7 +220,7 @@ def test_decode_and_append(name):
     ocache = orc.compact_kv(T.f64(K), T.f64(V), flags.cpu().numpy())
     for step in range(steps):
         q, kn, vn, fn = inputs.decode_inputs(shape, 420, step, DEV, keep_new=0.5)
-        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status)
+        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status, fused=fused)
         o_ref = orc.decode_attention(T.f64(q), T.f64(kn), T.f64(vn), ocache)
         T.check_close(T.f64(o), o_ref, shape.dtype, f"decode step {step}")
         orc.cache_append(ocache, T.f64(kn), T.f64(vn), fn.cpu().numpy())
@@ -252,7 +253,8 @@ def test_decode_long_slabs_many_chunks():
 @pytest.mark.parametrize("shape", [LayerShape(9, 300, 256, 8, 128, 2, 128, "bf16"),
                                    LayerShape(17, 150, 128, 4, 64, 1, 64, "f32")],
                          ids=["bf16_72slabs", "f32_d64_68slabs"])
-def test_decode_many_slabs_takes_the_workspace_form(shape):
+@pytest.mark.parametrize("fused", [False, True], ids=["two_calls", "one_call"])
+def test_decode_many_slabs_takes_the_workspace_form(shape, fused):
     """More slabs than the one-cluster-per-slab form serves: chunk pass + merge through the
     workspace, at a size the oracle checks in full; ragged and empty slabs included."""
     Q, K, V = inputs.qkv_gaussian(shape, 470, DEV)
@@ -267,7 +269,7 @@ def test_decode_many_slabs_takes_the_workspace_form(shape):
     ocache = orc.compact_kv(T.f64(K), T.f64(V), f)
     for step in range(steps):
         q, kn, vn, fn = inputs.decode_inputs(shape, 472, step, DEV, keep_new=0.5)
-        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status)
+        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status, fused=fused)
         o_ref = orc.decode_attention(T.f64(q), T.f64(kn), T.f64(vn), ocache)
         T.check_close(T.f64(o), o_ref, shape.dtype, f"decode step {step}")
         orc.cache_append(ocache, T.f64(kn), T.f64(vn), fn.cpu().numpy())
@@ -275,18 +277,19 @@ def test_decode_many_slabs_takes_the_workspace_form(shape):
     assert int(status.item()) == 0
 
 
-def test_decode_empty_cache_returns_own_value_and_full_slab_reports_overflow():
+@pytest.mark.parametrize("fused", [False, True], ids=["two_calls", "one_call"])
+def test_decode_empty_cache_returns_own_value_and_full_slab_reports_overflow(fused):
     shape = SMALL_BF16.with_(seq=64)
     Q, K, V = inputs.qkv_gaussian(shape, 500, DEV)
     flags = torch.zeros(shape.batch, shape.heads, shape.seq, dtype=torch.uint8, device=DEV)
     cap = [1] * (shape.batch * shape.heads)
     cache, prefix, idx, status = T.gpu_compact(shape, K, V, flags, cap=cap)
     q, kn, vn, fn = inputs.decode_inputs(shape, 510, 0, DEV, keep_new=1.0)
-    o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status)
+    o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status, fused=fused)
     assert torch.equal(o, vn)                                   # L = 0: only the self term
     assert int(status.item()) == 0 and cache.len.cpu().tolist() == cap
     q2, kn2, vn2, fn2 = inputs.decode_inputs(shape, 510, 1, DEV, keep_new=1.0)
-    o2 = T.gpu_decode_step(shape, q2, kn2, vn2, fn2, cache, status)
+    o2 = T.gpu_decode_step(shape, q2, kn2, vn2, fn2, cache, status, fused=fused)
     assert int(status.item()) & ag.AG_DEV_OVERFLOW                # slabs are full: write skipped
     assert cache.len.cpu().tolist() == cap
     assert torch.equal(cache.k_rows, kn.reshape(-1, shape.head_dim))
