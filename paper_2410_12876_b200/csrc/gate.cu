@@ -126,9 +126,11 @@ gate_out_kernel(const float *__restrict__ H, const T *__restrict__ Wo,
 
 size_t gate_workspace_bytes(const ag_layer_desc &d) {
   const size_t rows = (size_t)d.batch * d.seq, GD = (size_t)d.gate_heads * d.gate_head_dim;
-  size_t bytes = align_up(rows * 3 * GD * sizeof(float), 256) + align_up(rows * GD * sizeof(float), 256);
-  if (gate_attn_tc_supported(d)) bytes += gate_attn_partial_bytes(d);
-  return bytes;
+  // [Q' | K' | V'] (float32, or the bf16 hi and lo halves), then H' (CUDA-core path) or the split-K
+  // partials of MHA' (tensor-core path, where H' stays on chip)
+  const size_t qkv = align_up(rows * 3 * GD * sizeof(float), 256);
+  if (d.dtype == AG_BF16 && gate_attn_tc_supported(d)) return qkv + gate_attn_partial_bytes(d);
+  return qkv + align_up(rows * GD * sizeof(float), 256);
 }
 
 template <typename T>
@@ -146,7 +148,7 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
     void *lo = static_cast<char *>(ws) + (size_t)M * 3 * GD * sizeof(__nv_bfloat16);
     int rc = launch_gate_proj_tc(X, Wq, Wk, Wv, nullptr, hi, lo, M, d.hidden, GD, st);
     if (rc) return rc;
-    void *partials = reinterpret_cast<char *>(hcat) + align_up((size_t)M * GD * sizeof(float), 256);
+    void *partials = hcat;                           // H' stays on chip: the partials take its place
     // the merge of the split-K partials carries the output layer and the threshold with it
     return launch_gate_attn_tc(d, hi, lo, partials, Wo, gamma, logit_tau, scores, flags, st);
   } else {

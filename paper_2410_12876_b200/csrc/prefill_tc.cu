@@ -31,17 +31,15 @@ constexpr int kPfPanel = 128 * 128;                   // [128 rows][64 bf16] = 1
 constexpr int kPfTile = 2 * kPfPanel;                 // 32 KB
 constexpr float kRescaleThreshold = 8.f;              // log2 units
 
-// Geometry for key tiles of BN cache rows.  BN = 64: two CTAs per SM (256 TMEM columns each);
-// BN = 128: one CTA per SM (384 of 512 columns used).  TMEM: S0 [0,BN) S1 [BN,2BN), each
-// overwritten in place by its P (bf16 pairs); O [2BN, 2BN+128).
-template <int BN> struct PfCfg {
-  static constexpr int kKvPanel = BN * 128;           // [BN rows][64 bf16]
-  static constexpr int kKvTile = 2 * kKvPanel;
-  static constexpr int kKvBuf = 2 * kKvTile;          // two stages; >= one 32 KB dense tile
-  static constexpr int kSmemBytes = kPfTile + 2 * kKvBuf + 1024 + 256;
-  static constexpr uint32_t kColO = 2 * BN, kTmemCols = BN == 64 ? 256 : 512;
-  static constexpr int kCtasPerSm = BN == 64 ? 2 : 1;
-};
+// Key tiles of 64 cache rows; two CTAs per SM (256 TMEM columns, 97 KB of shared memory each).
+// 128-row tiles with one CTA per SM measured slower on 4096-token heads (131 us against 100 us).
+constexpr int kPfBN = 64;
+constexpr int kPfKvPanel = kPfBN * 128;               // [64 rows][64 bf16] = 8 KB
+constexpr int kPfKvTile = 2 * kPfKvPanel;             // 16 KB
+constexpr int kPfKvBuf = 2 * kPfKvTile;               // two stages = one 32 KB dense tile
+constexpr int kPfSmemBytes = kPfTile + 2 * kPfKvBuf + 1024 + 256;
+constexpr uint32_t kColS = 0, kColO = 2 * kPfBN, kTmemCols = 256;
+constexpr int kPfCtasPerSm = 2;
 
 struct PrefillTcArgs {
   const int32_t *prefix;            // [slabs, n + 1]
@@ -67,21 +65,17 @@ __device__ __forceinline__ uint32_t tile_chunk_offset(int row, int chunk) {
 // CTA's own 128 rows, of which only the diagonal (q_j . k_j) is read.  Last,
 // the dense V tile is brought in for the self term of the output, and the O
 // tile leaves through shared memory with one TMA store.
-template <int BN>
-__global__ void __launch_bounds__(kPfThreads, PfCfg<BN>::kCtasPerSm)
+__global__ void __launch_bounds__(kPfThreads, kPfCtasPerSm)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKd,
                   const __grid_constant__ CUtensorMap tmVd, const __grid_constant__ CUtensorMap tmO,
                   const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const PrefillTcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  using Cfg = PfCfg<BN>;
-  constexpr int kPfBN = BN, kPfKvPanel = Cfg::kKvPanel, kPfKvTile = Cfg::kKvTile;
-  constexpr uint32_t kColS = 0, kColO = Cfg::kColO, kTmemCols = Cfg::kTmemCols;
   uint8_t *sQ = smem;
   uint8_t *sK = sQ + kPfTile;                      // two stages, or one 128-row dense tile
-  uint8_t *sV = sK + Cfg::kKvBuf;
-  uint64_t *bars = reinterpret_cast<uint64_t *>(sV + Cfg::kKvBuf);
+  uint8_t *sV = sK + kPfKvBuf;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(sV + kPfKvBuf);
   uint64_t *q_full = bars;
   uint64_t *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;   // [2] each
   uint64_t *s_full = bars + 9;                     // [2]
@@ -101,7 +95,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int max_bound = pre[j_last];               // keys any row of this tile may see
   const int n_kv = (max_bound + kPfBN - 1) / kPfBN;
   const int row0 = (int)a.row_off[slab];
-  static_assert(BN == 64, "the self tile below spans exactly the two V stages");
+  static_assert(kPfKvBuf == kPfTile, "the self tile below spans exactly the two V stages");
   // uses of K stage 0 / 1 before the dense V tile: even / odd cache tiles
   const int k0_uses = (n_kv + 1) / 2, k1_uses = n_kv / 2;
 
@@ -279,11 +273,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const int nvalid = min(max(bound - i * kPfBN, 0), kPfBN);
       const uint32_t tS = tm_lane + kColS + st * kPfBN;
 
-      uint32_t r[BN];
-      if (BN == 64) tmem_ld_x64_sync(tS, r); else tmem_ld_x128_sync(tS, r);
+      uint32_t r[kPfBN];
+      tmem_ld_x64_sync(tS, r);
       if (nvalid < kPfBN) {
 #pragma unroll
-        for (int e = 0; e < BN; ++e)
+        for (int e = 0; e < kPfBN; ++e)
           if (e >= nvalid) r[e] = 0xff800000u;        // -inf: weight 0 below
       }
       // eight independent chains instead of one long dependency
@@ -291,7 +285,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
       for (int q = 0; q < 8; ++q) mx[q] = __uint_as_float(r[q]);
 #pragma unroll
-      for (int e = 8; e < BN; e += 8)
+      for (int e = 8; e < kPfBN; e += 8)
 #pragma unroll
         for (int q = 0; q < 8; ++q) mx[q] = fmaxf(mx[q], __uint_as_float(r[e + q]));
       float tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
@@ -306,7 +300,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       // p = 2^(s - m) as bf16 pairs, written over the columns S occupied
       float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < BN / 16; ++c) {
+      for (int c = 0; c < kPfBN / 16; ++c) {
         uint32_t pk[8];
 #pragma unroll
         for (int e = 0; e < 16; e += 2) {
@@ -344,16 +338,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       if ((i + 1) * kPfBN > L) {
         ok = mbar_wait(&v_full[st], ((i >> 1) + (st == 0 ? 1 : 0)) & 1);
         if (!ok) break;
-        // BN = 64: two threads per row, one panel each; BN = 128: one thread per row, both panels
-        const int vr = BN == 64 ? tid >> 1 : tid;
+        const int vr = tid >> 1;                      // two threads per row, one panel each
         if (i * kPfBN + vr >= L) {
           uint4 z = make_uint4(0, 0, 0, 0);
-          uint8_t *v0 = sV + st * kPfKvTile + (BN == 64 ? (tid & 1) * kPfKvPanel : 0) + vr * 128;
+          uint8_t *v0 = sV + st * kPfKvTile + (tid & 1) * kPfKvPanel + vr * 128;
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            *reinterpret_cast<uint4 *>(v0 + c * 16) = z;
-            if (BN == 128) *reinterpret_cast<uint4 *>(v0 + kPfKvPanel + c * 16) = z;
-          }
+          for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4 *>(v0 + c * 16) = z;
         }
         fence_proxy_async_smem();
       }
@@ -411,10 +401,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
-// Cache rows per key tile.  64 (two CTAs per SM) measured faster than 128 (one CTA per SM) on
-// 4096-token heads: 100 us against 131 us; the softmax threads, not the tensor core, set the pace.
-constexpr int kPrefillKeyTile = 64;
-
 bool prefill_tc_supported(const ag_layer_desc &d, const ag_cache &c) {
   return d.dtype == AG_BF16 && d.head_dim == 128 && c.pool_rows < ((int64_t)1 << 31) &&
          (int64_t)d.batch * d.heads * ((d.seq + kPfBM - 1) / kPfBM) < ((int64_t)1 << 31);
@@ -431,18 +417,16 @@ int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, cons
   if ((rc = make_tmap_3d_bf16(&tmO, O, slabs, d.seq, kPfD, kPfBM, 64))) return rc;
   // an empty pool still needs a valid map: describe one row of the dense K / V instead (never read)
   const bool empty = c.pool_rows == 0;
-  constexpr int BN = kPrefillKeyTile;
-  rc = make_tmap_2d_bf16(&tmK, empty ? K : c.k_rows, empty ? 1 : (uint64_t)c.pool_rows, kPfD, kPfD * 2, BN, 64);
+  rc = make_tmap_2d_bf16(&tmK, empty ? K : c.k_rows, empty ? 1 : (uint64_t)c.pool_rows, kPfD, kPfD * 2, kPfBN, 64);
   if (rc) return rc;
-  rc = make_tmap_2d_bf16(&tmV, empty ? V : c.v_rows, empty ? 1 : (uint64_t)c.pool_rows, kPfD, kPfD * 2, BN, 64);
+  rc = make_tmap_2d_bf16(&tmV, empty ? V : c.v_rows, empty ? 1 : (uint64_t)c.pool_rows, kPfD, kPfD * 2, kPfBN, 64);
   if (rc) return rc;
   PrefillTcArgs a;
   a.prefix = prefix; a.row_off = c.row_off; a.len = c.len;
   a.n = d.seq; a.n_qtiles = (d.seq + kPfBM - 1) / kPfBM; a.slabs = slabs;
   a.scale_log2 = scale * 1.4426950408889634f;
-  auto kern = prefill_tc_kernel<BN>;
-  AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PfCfg<BN>::kSmemBytes));
-  kern<<<a.n_qtiles * slabs, kPfThreads, PfCfg<BN>::kSmemBytes, st>>>(tmQ, tmKd, tmVd, tmO, tmK, tmV, a);
+  AG_CUDA_TRY(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes));
+  prefill_tc_kernel<<<a.n_qtiles * slabs, kPfThreads, kPfSmemBytes, st>>>(tmQ, tmKd, tmVd, tmO, tmK, tmV, a);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
