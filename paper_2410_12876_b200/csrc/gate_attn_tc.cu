@@ -40,14 +40,20 @@ constexpr int kGaSmemBytes = 2 * kGaTile + 4 * kGaKvStage + 1024 + 256;   // Q +
 constexpr uint32_t kGaColS = 0, kGaColO = 256, kGaColPhi = 384, kGaColPlo = 448, kGaTmemCols = 512;
 constexpr float kGaRescaleThreshold = 8.f;
 
+constexpr int kGaMaxSeg = 256;       // segments at most (one per SM)
+constexpr int kGaPieceCost = 3;      // set-up + epilogue of a piece, in half tile steps
+
 struct GateAttnArgs {
   float *part_o;            // [items, 128, 128] un-normalised partial outputs
   float *part_ml;           // [items, 128, 2]   running max (log2 units) and sum per row
   int n, n_qtiles, gate_heads, problems, GD, causal;
   int steps_per_prob;       // (query tile, key tile) steps of one (sequence, head)
   int total_steps;          // over all problems
-  int seg_steps;            // steps per segment (even: a piece starts on a 128-key boundary, so its
-                            // first tile holds a key every row of the query tile may see)
+  int n_seg;                // segments (= CTAs of the attention kernel)
+  // Segment s covers steps [seg_begin[s], seg_begin[s + 1]) of the list.  Every boundary is even: a
+  // piece starts on a 128-key boundary, so its first tile holds a key every row of the query tile
+  // may see.  Segments are cut to equal cost, a piece counting as much as kGaPieceCost / 2 steps.
+  int seg_begin[kGaMaxSeg + 1];
   float scale_log2;
 };
 
@@ -81,6 +87,15 @@ __device__ inline GaPiece ga_piece(const GateAttnArgs &a, int x, int x_end) {
   p.n_kv = min(x_end, tile_end) - x;
   return p;
 }
+// Segment that holds global step x.
+__device__ inline int ga_segment_of(const GateAttnArgs &a, int x) {
+  int lo = 0, hi = a.n_seg - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (a.seg_begin[mid] <= x) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
 // Partial slot of the piece of query tile (prob, qt) that lies in segment seg: consecutive pieces
 // differ in the query tile, the segment or both, so the sum is unique and grows along the list.
 __host__ __device__ inline int ga_slot(int prob, int qt, int n_qtiles, int seg) {
@@ -90,7 +105,7 @@ __host__ __device__ inline int ga_slot(int prob, int qt, int n_qtiles, int seg) 
 __global__ void __launch_bounds__(kGaThreads, 1)
 gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_constant__ CUtensorMap tmLo,
                     const __grid_constant__ CUtensorMap tmHiKv, const __grid_constant__ CUtensorMap tmLoKv,
-                    const GateAttnArgs a) {
+                    const __grid_constant__ GateAttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *sQ = smem;                    // [hi | lo]
@@ -107,8 +122,8 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
   // This CTA's segment of the step list.  Every role walks its pieces with the same arithmetic;
   // tiles are numbered t = 0, 1, ... across the pieces (stage and S buffer t & 1, in their use
   // number t >> 1; P and the P V barrier in their use number t), pieces pc = 0, 1, ...
-  const int x_begin = blockIdx.x * a.seg_steps;
-  const int x_end = min(a.total_steps, x_begin + a.seg_steps);
+  const int x_begin = a.seg_begin[blockIdx.x];
+  const int x_end = a.seg_begin[blockIdx.x + 1];
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
@@ -374,7 +389,7 @@ bool gate_attn_tc_supported(const ag_layer_desc &d) {
 constexpr int kMoTokens = 16, kMoThreads = kMoTokens * 32;
 template <typename T>
 __global__ void __launch_bounds__(kMoThreads)
-gate_merge_out_kernel(const GateAttnArgs a, const T *__restrict__ Wo, const float *__restrict__ gamma,
+gate_merge_out_kernel(const __grid_constant__ GateAttnArgs a, const T *__restrict__ Wo, const float *__restrict__ gamma,
                       float logit_tau, int h, float *__restrict__ scores, uint8_t *__restrict__ flags) {
   extern __shared__ __align__(16) unsigned char mo_smem[];
   float *Hs = reinterpret_cast<float *>(mo_smem);                                   // [16][GD]
@@ -391,7 +406,7 @@ gate_merge_out_kernel(const GateAttnArgs a, const T *__restrict__ Wo, const floa
       const int prob = b * a.gate_heads + g;
       // the query tile's steps [x0, x1) of the list lie in segments seg0 .. seg1, one piece in each
       const int x0 = prob * a.steps_per_prob + y0, x1 = prob * a.steps_per_prob + y1;
-      const int seg0 = x0 / a.seg_steps, ns = (x1 - 1) / a.seg_steps - seg0 + 1;
+      const int seg0 = ga_segment_of(a, x0), ns = ga_segment_of(a, x1 - 1) - seg0 + 1;
       const size_t row0 = (size_t)ga_slot(prob, qt, a.n_qtiles, seg0) * kGaBM + r;   // + s * 128 per piece
       float mmax = -INFINITY;
       for (int s = lane; s < ns; s += 32) mmax = fmaxf(mmax, a.part_ml[(row0 + (size_t)s * kGaBM) * 2]);
@@ -456,11 +471,39 @@ gate_merge_out_kernel(const GateAttnArgs a, const T *__restrict__ Wo, const floa
   }
 }
 
-// Segments: one per SM (at most kGaMaxSeg) when there is that much work, of an even number of steps.
-constexpr int kGaMaxSeg = 256;
+// Cuts the step list into at most `n_target` segments of about equal cost (2 per tile step,
+// kGaPieceCost per piece) and writes their boundaries; returns the number of segments.
+static int cut_segments(int problems, int nq, int causal, int n_target, int target, int *seg_begin) {
+  int n = 0, cur = 0, x = 0;
+  seg_begin[n++] = 0;
+  for (int prob = 0; prob < problems; ++prob)
+    for (int qt = 0; qt < nq; ++qt) {
+      int r = ga_key_tiles(qt, nq, causal);
+      while (r > 0) {
+        if (cur > 0 && cur + kGaPieceCost + 4 > target) {      // not even a two-tile piece fits: new segment
+          if (n >= n_target) return n_target + 1;
+          seg_begin[n++] = x;
+          cur = 0;
+        }
+        cur += kGaPieceCost;
+        int fit = ((target - cur) / 2) & ~1;
+        if (fit < 2) fit = 2;
+        const int take = r < fit ? r : fit;
+        cur += 2 * take; x += take; r -= take;
+        if (r > 0) {                                           // segment full inside the query tile
+          if (n >= n_target) return n_target + 1;
+          seg_begin[n++] = x;
+          cur = 0;
+        }
+      }
+    }
+  seg_begin[n] = x;
+  return n;                                                    // seg_begin[0 .. n]
+}
+
 struct GateAttnPlan {
-  int steps_per_prob, total_steps, seg_steps, n_seg;
-  size_t slots;
+  int steps_per_prob, total_steps, n_seg;
+  int seg_begin[kGaMaxSeg + 1];
 };
 static int gate_attn_plan(const ag_layer_desc &d, GateAttnPlan &p) {
   static int sm_count[64] = {0};                     // per device, read once
@@ -475,14 +518,18 @@ static int gate_attn_plan(const ag_layer_desc &d, GateAttnPlan &p) {
   const int nq = (d.seq + kGaBM - 1) / kGaBM, problems = d.batch * d.gate_heads;
   const long long per = d.gate_causal ? (long long)nq * (nq + 1) : 2LL * nq * nq;
   const long long total = per * problems;
-  if (total >= (1LL << 30)) return AG_ERR_UNSUPPORTED;
-  long long seg = (total + sm_count[dev] - 1) / sm_count[dev];
-  seg = (seg + 1) & ~1LL;
+  if (total >= (1LL << 28)) return AG_ERR_UNSUPPORTED;
   p.steps_per_prob = (int)per;
   p.total_steps = (int)total;
-  p.seg_steps = (int)seg;
-  p.n_seg = (int)((total + seg - 1) / seg);
-  p.slots = (size_t)problems * nq + p.n_seg;
+  const int n_target = sm_count[dev];
+  // cost per segment: raised until the cuts fit into n_target segments
+  long long target = (2 * total + (long long)kGaPieceCost * ((long long)problems * nq + n_target) + n_target - 1) / n_target;
+  if (target < kGaPieceCost + 4) target = kGaPieceCost + 4;
+  for (;;) {
+    p.n_seg = cut_segments(problems, nq, d.gate_causal, n_target, (int)target, p.seg_begin);
+    if (p.n_seg <= n_target) break;
+    target += 1 + target / 64;
+  }
   return AG_OK;
 }
 
@@ -508,9 +555,10 @@ int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *
   GateAttnArgs a;
   a.n = d.seq; a.n_qtiles = (d.seq + kGaBM - 1) / kGaBM;
   a.gate_heads = d.gate_heads; a.problems = d.batch * d.gate_heads; a.GD = GD; a.causal = d.gate_causal;
-  GateAttnPlan plan;
+  static thread_local GateAttnPlan plan;             // 1 KB of boundaries: not on the stack of every call
   if ((rc = gate_attn_plan(d, plan))) return rc;
-  a.steps_per_prob = plan.steps_per_prob; a.total_steps = plan.total_steps; a.seg_steps = plan.seg_steps;
+  a.steps_per_prob = plan.steps_per_prob; a.total_steps = plan.total_steps; a.n_seg = plan.n_seg;
+  for (int i = 0; i <= plan.n_seg; ++i) a.seg_begin[i] = plan.seg_begin[i];
   const size_t slots = (size_t)a.problems * a.n_qtiles + kGaMaxSeg;
   a.part_o = static_cast<float *>(partials);
   a.part_ml = reinterpret_cast<float *>(static_cast<char *>(partials) +
