@@ -383,9 +383,9 @@ bool gate_attn_tc_supported(const ag_layer_desc &d) {
 //   H'[t, g * 128 + c] = sum_s w_s O_s[r, c] / sum_s w_s l_s,  w_s = 2^(m_s - max_s m_s)
 //   s[t, i] = H'[t, :] Wo_g[:, i];  flag = s + gamma_i > logit(tau)
 // One CTA = 16 tokens, one warp per token.  A warp merges the token's row of every gate head
-// (a lane per four columns: every access is one 512-byte row) into shared memory; then four
-// warps take four tokens each, a lane per head, in rounds of 32 heads, against a [GD][32]
-// slice of Wo staged in shared memory.  H' never goes to global memory.
+// (a lane per four columns: every access is one 512-byte row) into shared memory; then warp w
+// takes four tokens and a quarter of the reduction, a lane per head, in rounds of 32 heads,
+// against a [GD][32] slice of Wo staged in shared memory.  H' never goes to global memory.
 constexpr int kMoTokens = 16, kMoThreads = kMoTokens * 32;
 template <typename T>
 __global__ void __launch_bounds__(kMoThreads)
@@ -394,6 +394,7 @@ gate_merge_out_kernel(const __grid_constant__ GateAttnArgs a, const T *__restric
   extern __shared__ __align__(16) unsigned char mo_smem[];
   float *Hs = reinterpret_cast<float *>(mo_smem);                                   // [16][GD]
   T *Ws = reinterpret_cast<T *>(mo_smem + sizeof(float) * kMoTokens * a.GD);       // [GD][32]
+  float *red = reinterpret_cast<float *>(mo_smem + sizeof(float) * kMoTokens * a.GD + sizeof(T) * a.GD * 32);  // [4][16][32]
   const int tiles_per_seq = (a.n + kMoTokens - 1) / kMoTokens;
   const int b = blockIdx.x / tiles_per_seq, t0 = (blockIdx.x % tiles_per_seq) * kMoTokens;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -402,46 +403,80 @@ gate_merge_out_kernel(const __grid_constant__ GateAttnArgs a, const T *__restric
   if (t < a.n) {
     const int qt = t / kGaBM, r = t % kGaBM;
     const int y0 = ga_first_step(qt, a.n_qtiles, a.causal), y1 = y0 + ga_key_tiles(qt, a.n_qtiles, a.causal);
-    for (int g = 0; g < a.gate_heads; ++g) {
-      const int prob = b * a.gate_heads + g;
-      // the query tile's steps [x0, x1) of the list lie in segments seg0 .. seg1, one piece in each
-      const int x0 = prob * a.steps_per_prob + y0, x1 = prob * a.steps_per_prob + y1;
-      const int seg0 = ga_segment_of(a, x0), ns = ga_segment_of(a, x1 - 1) - seg0 + 1;
-      const size_t row0 = (size_t)ga_slot(prob, qt, a.n_qtiles, seg0) * kGaBM + r;   // + s * 128 per piece
-      float mmax = -INFINITY;
-      for (int s = lane; s < ns; s += 32) mmax = fmaxf(mmax, a.part_ml[(row0 + (size_t)s * kGaBM) * 2]);
+    // four gate heads at a time, so that their loads are in flight together
+    for (int g0 = 0; g0 < a.gate_heads; g0 += 4) {
+      size_t row0[4];
+      int ns[4];
+      float mmax[4];
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      float lsum = 0.f;
-#pragma unroll 4
-      for (int s = 0; s < ns; ++s) {
-        const float2 ml = *reinterpret_cast<const float2 *>(a.part_ml + (row0 + (size_t)s * kGaBM) * 2);
-        const float4 o = *reinterpret_cast<const float4 *>(a.part_o + (row0 + (size_t)s * kGaBM) * kGaD + lane * 4);
-        const float w = fast_exp2(ml.x - mmax);
-        acc.x = fmaf(w, o.x, acc.x); acc.y = fmaf(w, o.y, acc.y);
-        acc.z = fmaf(w, o.z, acc.z); acc.w = fmaf(w, o.w, acc.w);
-        lsum = fmaf(w, ml.y, lsum);
+      for (int u = 0; u < 4; ++u) {
+        const int prob = b * a.gate_heads + min(g0 + u, a.gate_heads - 1);
+        // the query tile's steps [x0, x1) of the list lie in segments seg0 .. seg1, one piece in each
+        const int x0 = prob * a.steps_per_prob + y0, x1 = prob * a.steps_per_prob + y1;
+        const int seg0 = ga_segment_of(a, x0);
+        ns[u] = ga_segment_of(a, x1 - 1) - seg0 + 1;
+        row0[u] = (size_t)ga_slot(prob, qt, a.n_qtiles, seg0) * kGaBM + r;   // + s * 128 per piece
+        mmax[u] = -INFINITY;
+        for (int s = lane; s < ns[u]; s += 32) mmax[u] = fmaxf(mmax[u], a.part_ml[(row0[u] + (size_t)s * kGaBM) * 2]);
       }
-      const float inv = 1.f / lsum;
-      *reinterpret_cast<float4 *>(hrow + g * kGaD + lane * 4) =
-          make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) mmax[u] = fmaxf(mmax[u], __shfl_xor_sync(0xffffffffu, mmax[u], off));
+      float4 acc[4];
+      float lsum[4];
+      int ns_max = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { acc[u] = make_float4(0.f, 0.f, 0.f, 0.f); lsum[u] = 0.f; ns_max = max(ns_max, ns[u]); }
+      for (int s = 0; s < ns_max; ++s) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (s < ns[u]) {
+            const float2 ml = *reinterpret_cast<const float2 *>(a.part_ml + (row0[u] + (size_t)s * kGaBM) * 2);
+            const float4 o = *reinterpret_cast<const float4 *>(a.part_o + (row0[u] + (size_t)s * kGaBM) * kGaD + lane * 4);
+            const float w = fast_exp2(ml.x - mmax[u]);
+            acc[u].x = fmaf(w, o.x, acc[u].x); acc[u].y = fmaf(w, o.y, acc[u].y);
+            acc[u].z = fmaf(w, o.z, acc[u].z); acc[u].w = fmaf(w, o.w, acc[u].w);
+            lsum[u] = fmaf(w, ml.y, lsum[u]);
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (g0 + u < a.gate_heads) {
+          const float inv = 1.f / lsum[u];
+          *reinterpret_cast<float4 *>(hrow + (g0 + u) * kGaD + lane * 4) =
+              make_float4(acc[u].x * inv, acc[u].y * inv, acc[u].z * inv, acc[u].w * inv);
+        }
+      }
     }
   }
   for (int i0 = 0; i0 < h; i0 += 32) {
     __syncthreads();                                 // H' rows complete; previous slice of Wo consumed
-    for (int x = threadIdx.x; x < a.GD * 32; x += kMoThreads) {
-      const int c = x >> 5, i = i0 + (x & 31);
-      Ws[x] = i < h ? Wo[(size_t)c * h + i] : T(0.f);
+    if (sizeof(T) == 2 && (h & 7) == 0) {            // 16-byte pieces of the rows of Wo
+      for (int x = threadIdx.x; x < a.GD * 4; x += kMoThreads) {
+        const int c = x >> 2, i = i0 + (x & 3) * 8;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (i < h) v = ldg128(Wo + (size_t)c * h + i);
+        *reinterpret_cast<uint4 *>(Ws + c * 32 + (x & 3) * 8) = v;
+      }
+    } else {
+      for (int x = threadIdx.x; x < a.GD * 32; x += kMoThreads) {
+        const int c = x >> 5, i = i0 + (x & 31);
+        Ws[x] = i < h ? Wo[(size_t)c * h + i] : T(0.f);
+      }
     }
     __syncthreads();
-    if (warp < kMoTokens / 4) {
-      // warp w: tokens 4 w .. 4 w + 3 against head `lane`; per four steps of the reduction four
-      // broadcast float4 of H' and four values of Wo feed sixteen FMAs
+    {
+      // warp w: tokens 4 (w & 3) .. + 3 against head `lane` over a quarter of the reduction,
+      // c in [cq, cq + 1) GD / 4; per four steps four broadcast float4 of H' and four values of Wo
+      // feed sixteen FMAs.  The quarters are added in a fixed order below.
+      const int tq = warp & 3, cq = warp >> 2;
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
-      const float *h4 = Hs + warp * 4 * a.GD;
-#pragma unroll 2
-      for (int c = 0; c < a.GD; c += 4) {
+      const float *h4 = Hs + tq * 4 * a.GD;
+      const int c_begin = cq * (a.GD / 4), c_end = c_begin + a.GD / 4;    // GD is a multiple of 128
+#pragma unroll 4
+      for (int c = c_begin; c < c_end; c += 4) {
         float w[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) w[k] = Elem<T>::load(Ws + (c + k) * 32 + lane);
@@ -454,18 +489,19 @@ gate_merge_out_kernel(const __grid_constant__ GateAttnArgs a, const T *__restric
           acc[q] = fmaf(x.w, w[3], acc[q]);
         }
       }
-      const int i = i0 + lane;
-      if (i < h) {
-        const float gm = gamma ? gamma[i] : 0.f;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int tt = t0 + warp * 4 + q;
-          if (tt < a.n) {
-            const size_t o = ((size_t)b * h + i) * a.n + tt;
-            if (scores) scores[o] = acc[q];
-            flags[o] = (acc[q] + gm) > logit_tau ? 1 : 0;
-          }
-        }
+      for (int q = 0; q < 4; ++q) red[(cq * kMoTokens + tq * 4 + q) * 32 + lane] = acc[q];
+    }
+    __syncthreads();
+    {
+      // thread (token = warp, head = lane): the four quarters in order
+      const float *rp = red + warp * 32 + lane;
+      const float sc = ((rp[0] + rp[kMoTokens * 32]) + rp[2 * kMoTokens * 32]) + rp[3 * kMoTokens * 32];
+      const int i = i0 + lane;
+      if (i < h && t < a.n) {
+        const size_t o = ((size_t)b * h + i) * a.n + t;
+        if (scores) scores[o] = sc;
+        flags[o] = (sc + (gamma ? gamma[i] : 0.f)) > logit_tau ? 1 : 0;
       }
     }
   }
@@ -567,7 +603,7 @@ int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *
   AG_CUDA_TRY(cudaFuncSetAttribute(gate_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGaSmemBytes));
   gate_attn_tc_kernel<<<(unsigned)plan.n_seg, kGaThreads, kGaSmemBytes, st>>>(tmHi, tmLo, tmHiKv, tmLoKv, a);
   AG_LAUNCH_CHECK();
-  const size_t mo_smem = sizeof(float) * kMoTokens * GD + sizeof(__nv_bfloat16) * GD * 32;
+  const size_t mo_smem = sizeof(float) * kMoTokens * GD + sizeof(__nv_bfloat16) * GD * 32 + sizeof(float) * 4 * kMoTokens * 32;
   auto mo = gate_merge_out_kernel<__nv_bfloat16>;
   AG_CUDA_TRY(cudaFuncSetAttribute(mo, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mo_smem));
   const int blocks = d.batch * ((d.seq + kMoTokens - 1) / kMoTokens);
