@@ -400,9 +400,24 @@ gate_merge_out_kernel(const __grid_constant__ GateAttnArgs a, const T *__restric
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = t0 + warp;
   float *hrow = Hs + warp * a.GD;
+  // The CTA's 16 tokens lie in one query tile: which segments hold its pieces is looked up once per
+  // gate head (a binary search over the boundaries in constant memory), by one thread each.
+  int *seg_first = reinterpret_cast<int *>(red);     // [gate_heads] first segment, then [gate_heads] piece count
+  {
+    const int qt = t0 / kGaBM;
+    const int y0 = ga_first_step(qt, a.n_qtiles, a.causal), y1 = y0 + ga_key_tiles(qt, a.n_qtiles, a.causal);
+    for (int g = threadIdx.x; g < a.gate_heads; g += kMoThreads) {
+      const int prob = b * a.gate_heads + g;
+      // the query tile's steps [x0, x1) of the list lie in segments seg0 .. seg1, one piece in each
+      const int x0 = prob * a.steps_per_prob + y0, x1 = prob * a.steps_per_prob + y1;
+      const int seg0 = ga_segment_of(a, x0);
+      seg_first[g] = seg0;
+      seg_first[a.gate_heads + g] = ga_segment_of(a, x1 - 1) - seg0 + 1;
+    }
+  }
+  __syncthreads();
   if (t < a.n) {
     const int qt = t / kGaBM, r = t % kGaBM;
-    const int y0 = ga_first_step(qt, a.n_qtiles, a.causal), y1 = y0 + ga_key_tiles(qt, a.n_qtiles, a.causal);
     // four gate heads at a time, so that their loads are in flight together
     for (int g0 = 0; g0 < a.gate_heads; g0 += 4) {
       size_t row0[4];
@@ -410,12 +425,9 @@ gate_merge_out_kernel(const __grid_constant__ GateAttnArgs a, const T *__restric
       float mmax[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const int prob = b * a.gate_heads + min(g0 + u, a.gate_heads - 1);
-        // the query tile's steps [x0, x1) of the list lie in segments seg0 .. seg1, one piece in each
-        const int x0 = prob * a.steps_per_prob + y0, x1 = prob * a.steps_per_prob + y1;
-        const int seg0 = ga_segment_of(a, x0);
-        ns[u] = ga_segment_of(a, x1 - 1) - seg0 + 1;
-        row0[u] = (size_t)ga_slot(prob, qt, a.n_qtiles, seg0) * kGaBM + r;   // + s * 128 per piece
+        const int g = min(g0 + u, a.gate_heads - 1), prob = b * a.gate_heads + g;
+        ns[u] = seg_first[a.gate_heads + g];
+        row0[u] = (size_t)ga_slot(prob, qt, a.n_qtiles, seg_first[g]) * kGaBM + r;   // + s * 128 per piece
         mmax[u] = -INFINITY;
         for (int s = lane; s < ns[u]; s += 32) mmax[u] = fmaxf(mmax[u], a.part_ml[(row0[u] + (size_t)s * kGaBM) * 2]);
       }
