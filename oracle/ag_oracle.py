@@ -128,6 +128,27 @@ def attention_gate(X, Wq_g, Wk_g, Wv_g, Wo_g, gate_heads, gamma, tau, causal=Tru
     return s, gate_flags(s, gamma, tau)
 
 
+def ragged_gate(X, seq_lens, gate_fn):
+    """A batch of sequences of different lengths, padded to a common n (the paper
+    treats one sequence; sequences of a batch are independent).  Sequence b is
+    its first seq_lens[b] tokens: the gate runs on exactly those (gate_fn maps
+    [1, len, d] -> (scores, flags), e.g. a closure over attention_gate or
+    linear_gate), the padding positions get score 0 and flag 0 (evicted), so
+    nothing downstream ever retains them."""
+    X = _as_f64(X)
+    B, n = X.shape[0], X.shape[1]
+    scores = flags = None
+    for b in range(B):
+        L = int(seq_lens[b])
+        s, f = gate_fn(X[b:b + 1, :L])
+        if scores is None:
+            scores = np.zeros((B, s.shape[1], n), dtype=F64)
+            flags = np.zeros((B, s.shape[1], n), dtype=np.uint8)
+        scores[b, :, :L] = s[0]
+        flags[b, :, :L] = f[0]
+    return scores, flags
+
+
 # --------------------------------------------------------------------------
 # Step 2: selective caching.  Sec. 3.3, sentence after Eq. 4: k_i^(t), v_i^(t)
 # are retained iff AG(X)_i^(t) = 1.

@@ -158,3 +158,31 @@ def test_linear_gate_flags_follow_eq4():
     s, f = orc.linear_gate(X, W, gamma, tau)
     want = 1.0 / (1.0 + np.exp(-(s + gamma[None, :, None]))) > tau
     assert np.array_equal(f, want.astype(np.uint8)) and f.dtype == np.uint8
+
+
+# ---- batches of sequences of different lengths (padding is never retained)
+
+def test_ragged_gate_padding_is_evicted_and_never_seen():
+    """Whatever sits in the padding, the valid tokens score as their sequence alone does, in the
+    causal and in the bidirectional reading of MHA', and every padding flag is 0."""
+    n, d, hg, Dg, h = 9, 6, 2, 4, 3
+    X = _w((2, n, d), 60)
+    Wq, Wk, Wv = (_w((d, hg * Dg), 61 + k, 0.5) for k in range(3))
+    Wo = _w((hg * Dg, h), 64, 0.5)
+    lens = [n, 4]
+    for causal in (True, False):
+        fn = lambda x: orc.attention_gate(x, Wq, Wk, Wv, Wo, hg, gamma=0.1, tau=0.5, causal=causal)
+        s, f = orc.ragged_gate(X, lens, fn)
+        X2 = X.copy()
+        X2[1, 4:] = 1e3                                        # garbage in the padding
+        s2, f2 = orc.ragged_gate(X2, lens, fn)
+        assert np.array_equal(s, s2) and np.array_equal(f, f2)
+        assert np.all(f[1, :, 4:] == 0) and np.all(s[1, :, 4:] == 0)
+        alone_s, alone_f = fn(X[1:2, :4])
+        assert np.array_equal(s[1, :, :4], alone_s[0]) and np.array_equal(f[1, :, :4], alone_f[0])
+        full_s, full_f = fn(X[0:1])
+        assert np.array_equal(s[0], full_s[0]) and np.array_equal(f[0], full_f[0])
+    # the bidirectional reading does depend on the length: a full-length run differs on the valid part
+    s_full, _ = orc.attention_gate(X, Wq, Wk, Wv, Wo, hg, gamma=0.1, tau=0.5, causal=False)
+    s_rag, _ = orc.ragged_gate(X, lens, lambda x: orc.attention_gate(x, Wq, Wk, Wv, Wo, hg, 0.1, 0.5, causal=False))
+    assert not np.allclose(s_full[1, :, :4], s_rag[1, :, :4])
