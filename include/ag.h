@@ -78,6 +78,14 @@ typedef struct {
   int32_t gate_causal;   /* 1: MHA' uses the lower-triangular decoder mask;
                             0: every token of MHA' sees the whole sequence  */
   int32_t dtype;         /* ag_dtype                                       */
+  const int32_t *seq_lens; /* NULL, or DEVICE pointer to B lengths, 1 <= seq_lens[b] <= n:
+                            sequence b is its first seq_lens[b] tokens, the rest
+                            of its n positions is padding.  Read by the two gate
+                            calls only: a valid token's score is what its sequence
+                            alone would give (the bidirectional MHA' sees seq_lens[b]
+                            keys), and every padding position gets flag 0, so it is
+                            never cached and never attended to; scores and attention
+                            outputs at padding positions are unspecified.            */
 } ag_layer_desc;
 
 /* Ragged per-(sequence, head) cache of retained keys and values.  The struct

@@ -37,6 +37,7 @@ class ag_layer_desc(ctypes.Structure):
         ("heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
         ("gate_heads", ctypes.c_int32), ("gate_head_dim", ctypes.c_int32),
         ("tau", ctypes.c_float), ("gate_causal", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("seq_lens", ctypes.c_void_p),
     ]
 
 
@@ -90,11 +91,15 @@ def lib():
     return _lib
 
 
-def make_desc(shape):
-    """ag_layer_desc from an object with the LayerShape fields."""
+def make_desc(shape, seq_lens=None):
+    """ag_layer_desc from an object with the LayerShape fields; seq_lens: optional int32 device
+    tensor [batch] of sequence lengths (the caller keeps it alive while the descriptor is used)."""
+    if seq_lens is not None:
+        assert seq_lens.dtype == torch.int32 and seq_lens.is_cuda and seq_lens.numel() == shape.batch
     return ag_layer_desc(shape.batch, shape.seq, shape.hidden, shape.heads, shape.head_dim,
                          shape.gate_heads, shape.gate_head_dim, float(shape.tau),
-                         int(shape.gate_causal), AG_F32 if shape.dtype == "f32" else AG_BF16)
+                         int(shape.gate_causal), AG_F32 if shape.dtype == "f32" else AG_BF16,
+                         None if seq_lens is None else seq_lens.data_ptr())
 
 
 def _ptr(t):

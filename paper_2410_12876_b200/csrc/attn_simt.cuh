@@ -31,6 +31,8 @@ struct SimtAttnArgs {
   const void *k_rows, *v_rows;         // compacted cache pools
   const int64_t *row_off;
   const int32_t *prefix;               // [problems, n + 1]
+  // kGateFull only: [batch] keys each sequence has (the rest is padding), or NULL = n
+  const int32_t *seq_lens;
 };
 
 constexpr int kSimtBM = 64, kSimtBN = 64, kSimtThreads = 256;
@@ -70,6 +72,7 @@ simt_attn_kernel(const SimtAttnArgs a) {
     kp_row = D; vp_row = D;
   }
   const int32_t *pre = MODE == kPrefill ? a.prefix + (size_t)prob * (a.n + 1) : nullptr;
+  const int n_keys = (MODE == kGateFull && a.seq_lens) ? a.seq_lens[prob / a.inner] : a.n;
 
   // Q tile -> shared (rows past n are clamped; they are never stored)
   for (int x = tid; x < kSimtBM * kVecPerRow; x += kSimtThreads) {
@@ -88,11 +91,11 @@ simt_attn_kernel(const SimtAttnArgs a) {
     const int j = j0 + ty * 4 + r;
     valid[r] = j < a.n;
     const int jc = min(j, a.n - 1);
-    bound[r] = MODE == kGateCausal ? jc + 1 : (MODE == kGateFull ? a.n : pre[jc]);
+    bound[r] = MODE == kGateCausal ? jc + 1 : (MODE == kGateFull ? n_keys : pre[jc]);
     if (!valid[r]) bound[r] = 0;
   }
   const int j_last = min(j0 + kSimtBM, a.n) - 1;
-  const int max_bound = MODE == kGateCausal ? j_last + 1 : (MODE == kGateFull ? a.n : pre[j_last]);
+  const int max_bound = MODE == kGateCausal ? j_last + 1 : (MODE == kGateFull ? n_keys : pre[j_last]);
   const int n_tiles = (max_bound + kSimtBN - 1) / kSimtBN;
 
   float m[4], l[4], o[4][kOC][4];

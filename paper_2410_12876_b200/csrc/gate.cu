@@ -83,7 +83,7 @@ template <typename T>
 __global__ void __launch_bounds__(kOutThreads)
 gate_out_kernel(const float *__restrict__ H, const T *__restrict__ Wo,
                 const float *__restrict__ gamma, float logit_tau, int B, int n, int GD, int h,
-                float *__restrict__ scores, uint8_t *__restrict__ flags) {
+                const int32_t *__restrict__ seq_lens, float *__restrict__ scores, uint8_t *__restrict__ flags) {
   extern __shared__ __align__(16) unsigned char sh_raw[];
   float *Hs = reinterpret_cast<float *>(sh_raw);                       // [16][GD]
   T *Ws = reinterpret_cast<T *>(sh_raw + sizeof(float) * kOutTokens * GD);   // [GD][32]
@@ -116,8 +116,9 @@ gate_out_kernel(const float *__restrict__ H, const T *__restrict__ Wo,
         const int tt = warp * 4 + q;
         if (tt < nt) {
           const size_t o = ((size_t)b * h + i) * n + t0 + tt;
+          const bool padding = seq_lens && t0 + tt >= seq_lens[b];
           if (scores) scores[o] = acc[q];
-          flags[o] = (acc[q] + gm) > logit_tau ? 1 : 0;
+          flags[o] = !padding && (acc[q] + gm) > logit_tau ? 1 : 0;
         }
       }
     }
@@ -170,6 +171,7 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
     a.q_row = a.k_row = a.v_row = 3 * GD;
     a.o_batch = (long long)d.seq * GD; a.o_inner = Dg; a.o_row = GD;
     a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)Dg));
+    a.seq_lens = d.seq_lens;
     const int problems = d.batch * d.gate_heads;
     int rc;
     if (Dg == 64)
@@ -186,7 +188,7 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
   AG_CUDA_TRY(cudaFuncSetAttribute(out_kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)out_smem));
   const int blocks = d.batch * ((d.seq + kOutTokens - 1) / kOutTokens);
   out_kern<<<blocks, kOutThreads, out_smem, st>>>(hcat, static_cast<const T *>(Wo), gamma, logit_tau,
-                                                 d.batch, d.seq, GD, d.heads, scores, flags);
+                                                 d.batch, d.seq, GD, d.heads, d.seq_lens, scores, flags);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }

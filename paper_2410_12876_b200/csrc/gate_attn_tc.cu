@@ -44,6 +44,7 @@ constexpr int kGaMaxSeg = 256;       // segments at most (one per SM)
 constexpr int kGaPieceCost = 3;      // set-up + epilogue of a piece, in half tile steps
 
 struct GateAttnArgs {
+  const int32_t *seq_lens;  // [B] or NULL: tokens past seq_lens[b] are padding
   float *part_o;            // [items, 128, 128] un-normalised partial outputs
   float *part_ml;           // [items, 128, 2]   running max (log2 units) and sum per row
   int n, n_qtiles, gate_heads, problems, GD, causal;
@@ -262,7 +263,9 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
     const int j = pz.qt * kGaBM + row;
     const bool valid = j < a.n;
     const int jc = min(j, a.n - 1);
-    const int bound = a.causal ? jc + 1 : a.n;       // keys below bound are visible
+    // keys below bound are visible (bidirectional: the sequence's own tokens, not its padding)
+    const int seq_len = a.seq_lens ? a.seq_lens[pz.prob / a.gate_heads] : a.n;
+    const int bound = a.causal ? jc + 1 : seq_len;
     float m = -INFINITY, l = 0.f;
 
     for (int i = 0; i < n_kv && ok; ++i) {
@@ -291,14 +294,17 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
       float tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
                          fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
       tmax *= a.scale_log2;
-      // the first tile of an item always holds a key visible to every row (key 0, or a tile
-      // wholly before the query tile), so m is finite from here on
+      // The first tile of a piece holds a key visible to every row (key 0, or a tile wholly before
+      // the query tile) - unless the sequence is shorter than its padded length and the bidirectional
+      // MHA' has no key in this piece at all: m then stays -inf, every weight is 0, and the piece's
+      // partial (m = -inf, l = 0, O = 0) drops out of the merge.
       float m_new;
       if (i == 0) m_new = tmax;
       else m_new = (tmax > m + kGaRescaleThreshold) ? tmax : m;
       const bool rescale = (i > 0) && __any_sync(0xffffffffu, m_new != m);
-      const float alpha = (i == 0) ? 0.f : fast_exp2(m - m_new);
+      const float alpha = (i == 0 || m == -INFINITY) ? 0.f : fast_exp2(m - m_new);
       l *= alpha;
+      const float m_exp = m_new == -INFINITY ? 0.f : m_new;    // exponent offset: keeps -inf - (-inf) out
 
       if (i > 0) {
         ok = mbar_wait(pv_done, (t - 1) & 1);
@@ -322,8 +328,8 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
         uint32_t ph[8], pl[8];
 #pragma unroll
         for (int e = 0; e < 16; e += 2) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e]), a.scale_log2, -m_new));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e + 1]), a.scale_log2, -m_new));
+          const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e]), a.scale_log2, -m_exp));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e + 1]), a.scale_log2, -m_exp));
           rs[(e >> 1) & 3] += p0 + p1;
           float h0, l0, h1, l1;
           split_bf16(p0, h0, l0);
@@ -512,8 +518,9 @@ gate_merge_out_kernel(const __grid_constant__ GateAttnArgs a, const T *__restric
       const int i = i0 + lane;
       if (i < h && t < a.n) {
         const size_t o = ((size_t)b * h + i) * a.n + t;
+        const bool padding = a.seq_lens && t >= a.seq_lens[b];
         if (scores) scores[o] = sc;
-        flags[o] = (sc + (gamma ? gamma[i] : 0.f)) > logit_tau ? 1 : 0;
+        flags[o] = !padding && (sc + (gamma ? gamma[i] : 0.f)) > logit_tau ? 1 : 0;
       }
     }
   }
@@ -601,6 +608,7 @@ int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *
   if ((rc = make_tmap_3d_bf16(&tmHiKv, qkv_hi, d.batch, d.seq, 3 * GD, kGaBN, 64))) return rc;
   if ((rc = make_tmap_3d_bf16(&tmLoKv, qkv_lo, d.batch, d.seq, 3 * GD, kGaBN, 64))) return rc;
   GateAttnArgs a;
+  a.seq_lens = d.seq_lens;
   a.n = d.seq; a.n_qtiles = (d.seq + kGaBM - 1) / kGaBM;
   a.gate_heads = d.gate_heads; a.problems = d.batch * d.gate_heads; a.GD = GD; a.causal = d.gate_causal;
   static thread_local GateAttnPlan plan;             // 1 KB of boundaries: not on the stack of every call

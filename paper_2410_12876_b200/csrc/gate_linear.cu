@@ -35,6 +35,7 @@ constexpr int kGlSmemBytes = kGlStages * kGlStageBytes + kGlPartBytes + 1024 /*a
 constexpr uint32_t kGlTmemCols = 64;
 
 struct GateLinearArgs {
+  const int32_t *seq_lens;   // [B] or NULL: tokens past seq_lens[b] are padding (flag 0)
   const float *gamma;
   float *scores;
   uint8_t *flags;
@@ -138,6 +139,7 @@ gate_linear_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     const int tok = m0 + r_in;
     if (tok < a.M) {
       const int b = tok / a.n, t = tok % a.n;
+      const bool padding = a.seq_lens && t >= a.seq_lens[b];
       float s[N];
 #pragma unroll
       for (int i = 0; i < N; ++i) s[i] = 0.f;
@@ -151,7 +153,7 @@ gate_linear_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         if (i < a.h) {
           const size_t o = ((size_t)b * a.h + i) * a.n + t;   // lanes = consecutive tokens: coalesced
           if (a.scores) a.scores[o] = s[i];
-          a.flags[o] = (s[i] + (a.gamma ? a.gamma[i] : 0.f)) > a.logit_tau ? 1 : 0;
+          a.flags[o] = !padding && (s[i] + (a.gamma ? a.gamma[i] : 0.f)) > a.logit_tau ? 1 : 0;
         }
       }
     }
@@ -166,8 +168,8 @@ gate_linear_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
 template <typename T>
 __global__ void __launch_bounds__(256)
 gate_linear_simt_kernel(const T *__restrict__ X, const T *__restrict__ W, const float *__restrict__ gamma,
-                        float logit_tau, int M, int n, int d, int h, float *__restrict__ scores,
-                        uint8_t *__restrict__ flags) {
+                        float logit_tau, int M, int n, int d, int h, const int32_t *__restrict__ seq_lens,
+                        float *__restrict__ scores, uint8_t *__restrict__ flags) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tok = blockIdx.x * 8 + warp;
   if (tok >= M) return;
@@ -195,7 +197,7 @@ gate_linear_simt_kernel(const T *__restrict__ X, const T *__restrict__ W, const 
         if (i < h) {
           const size_t o = ((size_t)b * h + i) * n + t;
           if (scores) scores[o] = acc[e];
-          flags[o] = (acc[e] + (gamma ? gamma[i] : 0.f)) > logit_tau ? 1 : 0;
+          flags[o] = !(seq_lens && t >= seq_lens[b]) && (acc[e] + (gamma ? gamma[i] : 0.f)) > logit_tau ? 1 : 0;
         }
       }
     }
@@ -235,7 +237,7 @@ static int run_gate_linear_tc(const ag_layer_desc &d, const void *X, const void 
 int launch_gate_linear(const ag_layer_desc &d, const void *X, const void *W, const float *gamma,
                        float *scores, uint8_t *flags, cudaStream_t st) {
   GateLinearArgs a;
-  a.gamma = gamma; a.scores = scores; a.flags = flags;
+  a.seq_lens = d.seq_lens; a.gamma = gamma; a.scores = scores; a.flags = flags;
   a.M = d.batch * d.seq; a.n = d.seq; a.h = d.heads;
   a.kb_total = (d.hidden + kGlBK - 1) / kGlBK; a.kb_per_cta = a.kb_total;
   a.logit_tau = (float)log((double)d.tau / (1.0 - (double)d.tau));
@@ -248,11 +250,11 @@ int launch_gate_linear(const ag_layer_desc &d, const void *X, const void *W, con
   const int blocks = (a.M + 7) / 8;
   if (d.dtype == AG_F32)
     gate_linear_simt_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(W),
-                                                          gamma, a.logit_tau, a.M, a.n, d.hidden, d.heads, scores, flags);
+                                                          gamma, a.logit_tau, a.M, a.n, d.hidden, d.heads, d.seq_lens, scores, flags);
   else
     gate_linear_simt_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(
         static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(W), gamma, a.logit_tau, a.M, a.n,
-        d.hidden, d.heads, scores, flags);
+        d.hidden, d.heads, d.seq_lens, scores, flags);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
