@@ -214,13 +214,24 @@ def prefill_head(Q_i, K_i, V_i, flags_i, scale=None, rows=None):
     return A @ V_i
 
 
+def kv_head_of(i, h, h_kv):
+    """Grouped-query attention: h query heads share h_kv key/value heads, consecutive query heads
+    in groups of h / h_kv (the paper's Mistral runs; h_kv = h is ordinary multi-head attention).
+    The cache, and therefore the flag, belongs to the key/value head."""
+    assert h % h_kv == 0
+    return i // (h // h_kv)
+
+
 def prefill_attention(Q, K, V, flags, scale=None):
-    """All heads of all sequences: [B, h, n, D] -> [B, h, n, D] float64."""
+    """All heads of all sequences: Q [B, h, n, D], K, V [B, h_kv, n, D], flags [B, h_kv, n]
+    -> [B, h, n, D] float64.  Query head i reads key/value head kv_head_of(i) and its flags."""
     B, h, n, D = np.asarray(Q).shape
+    h_kv = np.asarray(K).shape[1]
     O = np.empty((B, h, n, D), dtype=F64)
     for b in range(B):
         for i in range(h):
-            O[b, i] = prefill_head(Q[b, i], K[b, i], V[b, i], flags[b, i], scale)
+            g = kv_head_of(i, h, h_kv)
+            O[b, i] = prefill_head(Q[b, i], K[b, g], V[b, g], flags[b, g], scale)
     return O
 
 
@@ -244,14 +255,17 @@ def decode_head(q, k_new, v_new, k_cache, v_cache, scale=None):
 
 
 def decode_attention(q, k_new, v_new, cache, scale=None):
-    """q, k_new, v_new [B, h, D]; cache as returned by compact_kv -> [B, h, D]."""
+    """q [B, h, D]; k_new, v_new [B, h_kv, D]; cache as returned by compact_kv (one slab per
+    key/value head) -> [B, h, D].  Query head i reads slab kv_head_of(i)."""
     q = np.asarray(q)
     B, h, D = q.shape
+    h_kv = np.asarray(k_new).shape[1]
     o = np.empty((B, h, D), dtype=F64)
     for b in range(B):
         for i in range(h):
-            c = cache[b][i]
-            o[b, i] = decode_head(q[b, i], k_new[b, i], v_new[b, i], c["k"], c["v"], scale)
+            g = kv_head_of(i, h, h_kv)
+            c = cache[b][g]
+            o[b, i] = decode_head(q[b, i], k_new[b, g], v_new[b, g], c["k"], c["v"], scale)
     return o
 
 

@@ -29,6 +29,11 @@ class LayerShape:
     dtype: str = "bf16"        # "f32" | "bf16"
     tau: float = 0.5
     gate_causal: int = 1
+    kv_heads: int = 0          # key/value heads (grouped-query attention); 0 = one per query head
+
+    @property
+    def kvh(self):
+        return self.kv_heads if self.kv_heads > 0 else self.heads
 
     @property
     def torch_dtype(self):
@@ -69,15 +74,16 @@ def hidden_states(shape, seed, device="cpu"):
 def layer_weights(shape, seed, device="cpu"):
     """All projection weights ~ N(0, 0.02), stored "in x out"."""
     d, hD, gD = shape.hidden, shape.heads * shape.head_dim, shape.gate_heads * shape.gate_head_dim
+    kD = shape.kvh * shape.head_dim
     dt = shape.torch_dtype
     return {
         "Wq": randn((d, hD), seed + 1, device, dt, 0.02),
-        "Wk": randn((d, hD), seed + 2, device, dt, 0.02),
-        "Wv": randn((d, hD), seed + 3, device, dt, 0.02),
+        "Wk": randn((d, kD), seed + 2, device, dt, 0.02),
+        "Wv": randn((d, kD), seed + 3, device, dt, 0.02),
         "Wq_g": randn((d, gD), seed + 4, device, dt, 0.02),
         "Wk_g": randn((d, gD), seed + 5, device, dt, 0.02),
         "Wv_g": randn((d, gD), seed + 6, device, dt, 0.02),
-        "Wo_g": randn((gD, shape.heads), seed + 7, device, dt, 0.02),
+        "Wo_g": randn((gD, shape.kvh), seed + 7, device, dt, 0.02),      # one flag column per key/value head
     }
 
 
@@ -87,21 +93,23 @@ def linear_gate_weight(shape, seed, device="cpu"):
 
 
 def project_qkv(shape, X, W):
-    """Upstream projection Q_i = X W^Q_i etc. -> three [B, h, n, D] tensors in
+    """Upstream projection Q_i = X W^Q_i etc. -> Q [B, h, n, D], K, V [B, h_kv, n, D] in
     the layer dtype.  float64 accumulate for the fp32 layer, float32 otherwise."""
     acc = torch.float64 if shape.dtype == "f32" else torch.float32
     out = []
     for name in ("Wq", "Wk", "Wv"):
         y = (X.to(acc) @ W[name].to(acc)).to(shape.torch_dtype)
-        y = y.view(shape.batch, shape.seq, shape.heads, shape.head_dim).permute(0, 2, 1, 3)
+        heads = shape.heads if name == "Wq" else shape.kvh
+        y = y.view(shape.batch, shape.seq, heads, shape.head_dim).permute(0, 2, 1, 3)
         out.append(y.contiguous())
     return out
 
 
 def qkv_gaussian(shape, seed, device="cpu", std=1.0):
     """Q, K, V ~ N(0, std^2) directly (workloads that give no hidden size)."""
-    s = (shape.batch, shape.heads, shape.seq, shape.head_dim)
-    return [randn(s, seed + k, device, shape.torch_dtype, std) for k in range(3)]
+    sq = (shape.batch, shape.heads, shape.seq, shape.head_dim)
+    skv = (shape.batch, shape.kvh, shape.seq, shape.head_dim)
+    return [randn(sq if k == 0 else skv, seed + k, device, shape.torch_dtype, std) for k in range(3)]
 
 
 def keep_targets_uniform(heads, seed, lo=0.3, hi=0.8):
@@ -174,16 +182,17 @@ def slab_layout(cap):
 
 
 def decode_inputs(shape, seed, step, device="cpu", keep_new=0.5):
-    """q, k_new, v_new [B, h, D] ~ N(0, 1) and flag_new [B, h] for one step."""
+    """q [B, h, D], k_new, v_new [B, h_kv, D] ~ N(0, 1) and flag_new [B, h_kv] for one step."""
     s = (shape.batch, shape.heads, shape.head_dim)
+    skv = (shape.batch, shape.kvh, shape.head_dim)
     base = seed + 10 * step
     q = randn(s, base + 1, device, shape.torch_dtype)
-    k = randn(s, base + 2, device, shape.torch_dtype)
-    v = randn(s, base + 3, device, shape.torch_dtype)
+    k = randn(skv, base + 2, device, shape.torch_dtype)
+    v = randn(skv, base + 3, device, shape.torch_dtype)
     if keep_new >= 1.0:
-        f = torch.ones(shape.batch, shape.heads, dtype=torch.uint8)
+        f = torch.ones(shape.batch, shape.kvh, dtype=torch.uint8)
     else:
-        f = bernoulli_flags((shape.batch, shape.heads), keep_new, base + 4)
+        f = bernoulli_flags((shape.batch, shape.kvh), keep_new, base + 4)
     return q, k, v, f.to(device)
 
 

@@ -169,3 +169,30 @@ def test_pins_catch_a_planted_mistake(monkeypatch):
         want = _attend_set(Q[j], K, V, _visible_set(f, j), 1.0 / math.sqrt(D))
         bad |= np.max(np.abs(O[j] - want)) > 1e-9
     assert bad
+
+
+# ---- grouped-query attention: query heads in groups share a key/value head and its flags
+
+def test_grouped_query_prefill_and_decode_equal_shared_heads_written_out():
+    """h = 6 query heads over h_kv = 2 key/value heads give exactly what ordinary multi-head
+    attention gives when each key/value head (and its flags, and its cache slab) is written out
+    once per query head of its group."""
+    rng = np.random.default_rng(70)
+    B, h, h_kv, n, D = 2, 6, 2, 9, 4
+    Q = rng.standard_normal((B, h, n, D))
+    K = rng.standard_normal((B, h_kv, n, D))
+    V = rng.standard_normal((B, h_kv, n, D))
+    f = (rng.random((B, h_kv, n)) < 0.5).astype(np.uint8)
+    rep = lambda a: np.repeat(a, h // h_kv, axis=1)
+    assert [orc.kv_head_of(i, h, h_kv) for i in range(h)] == [0, 0, 0, 1, 1, 1]
+    assert np.array_equal(orc.prefill_attention(Q, K, V, f), orc.prefill_attention(Q, rep(K), rep(V), rep(f)))
+    q = rng.standard_normal((B, h, D))
+    kn, vn = rng.standard_normal((B, h_kv, D)), rng.standard_normal((B, h_kv, D))
+    o = orc.decode_attention(q, kn, vn, orc.compact_kv(K, V, f))
+    o_rep = orc.decode_attention(q, rep(kn), rep(vn), orc.compact_kv(rep(K), rep(V), rep(f)))
+    assert np.array_equal(o, o_rep)
+    # and query heads of one group really differ only through q
+    Q2 = Q.copy()
+    Q2[:, 1] = Q2[:, 0]
+    O2 = orc.prefill_attention(Q2, K, V, f)
+    assert np.array_equal(O2[:, 0], O2[:, 1])
