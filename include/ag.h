@@ -86,6 +86,12 @@ typedef struct {
                             keys), and every padding position gets flag 0, so it is
                             never cached and never attended to; scores and attention
                             outputs at padding positions are unspecified.            */
+  int32_t kv_heads;      /* 0 (= heads), or the number of key/value heads of grouped-query
+                            attention: heads must be a multiple; query head i reads
+                            key/value head i / (heads / kv_heads).  K, V, k_new, v_new,
+                            flags, flag_new, scores, prefix, idx and the cache slabs then
+                            have kv_heads where the comments below say h; Q, q, O, o keep
+                            h; Wo_g and W_lin have kv_heads columns.                  */
 } ag_layer_desc;
 
 /* Ragged per-(sequence, head) cache of retained keys and values.  The struct

@@ -37,7 +37,7 @@ class ag_layer_desc(ctypes.Structure):
         ("heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
         ("gate_heads", ctypes.c_int32), ("gate_head_dim", ctypes.c_int32),
         ("tau", ctypes.c_float), ("gate_causal", ctypes.c_int32), ("dtype", ctypes.c_int32),
-        ("seq_lens", ctypes.c_void_p),
+        ("seq_lens", ctypes.c_void_p), ("kv_heads", ctypes.c_int32),
     ]
 
 
@@ -99,7 +99,7 @@ def make_desc(shape, seq_lens=None):
     return ag_layer_desc(shape.batch, shape.seq, shape.hidden, shape.heads, shape.head_dim,
                          shape.gate_heads, shape.gate_head_dim, float(shape.tau),
                          int(shape.gate_causal), AG_F32 if shape.dtype == "f32" else AG_BF16,
-                         None if seq_lens is None else seq_lens.data_ptr())
+                         None if seq_lens is None else seq_lens.data_ptr(), int(getattr(shape, "kv_heads", 0)))
 
 
 def _ptr(t):

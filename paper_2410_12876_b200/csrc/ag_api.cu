@@ -17,6 +17,7 @@ static int check_desc(const ag_layer_desc *d) {
   if (d->dtype != AG_F32 && d->dtype != AG_BF16) return AG_ERR_INVALID_ARG;
   if (!dim_ok(d->head_dim)) return AG_ERR_UNSUPPORTED;
   if ((int64_t)d->batch * d->heads > (int64_t)1 << 24) return AG_ERR_UNSUPPORTED;
+  if (d->kv_heads < 0 || (d->kv_heads > 0 && d->heads % d->kv_heads != 0)) return AG_ERR_INVALID_ARG;
   return AG_OK;
 }
 

@@ -23,6 +23,8 @@ void set_last_cuda_error(int e);
 #define AG_LAUNCH_CHECK() AG_CUDA_TRY(cudaGetLastError())
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+// Key/value heads of the layer (grouped-query attention), = heads when the field is 0.
+inline int kv_heads_of(const ag_layer_desc &d) { return d.kv_heads > 0 ? d.kv_heads : d.heads; }
 // Launch attribute that lets a kernel overlap its set-up with the tail of its predecessor (the
 // kernel itself starts with pdl_wait()).
 inline cudaLaunchAttribute pdl_attribute() {

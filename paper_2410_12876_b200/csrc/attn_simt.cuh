@@ -22,6 +22,7 @@ struct SimtAttnArgs {
   void *O;
   int n;                      // query rows per problem
   int inner;                  // problems per batch element (h' or h)
+  int kv_group;               // kPrefill: query heads per key/value head (0 or 1 = one each)
   long long q_batch, q_inner, q_row;   // element strides
   long long k_batch, k_inner, k_row;   // gate: K/V rows inside the packed projection
   long long v_batch, v_inner, v_row;
@@ -62,16 +63,19 @@ simt_attn_kernel(const SimtAttnArgs a) {
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
 
   const TIn *Qp = static_cast<const TIn *>(a.Q) + b * a.q_batch + i * a.q_inner;
-  const TIn *Kd = static_cast<const TIn *>(a.K) + b * a.k_batch + i * a.k_inner;
-  const TIn *Vd = static_cast<const TIn *>(a.V) + b * a.v_batch + i * a.v_inner;
+  // grouped-query attention: query head i reads key/value head ik, cache slab prob_kv
+  const int group = a.kv_group > 1 ? a.kv_group : 1;
+  const int ik = i / group, prob_kv = b * (a.inner / group) + ik;
+  const TIn *Kd = static_cast<const TIn *>(a.K) + b * a.k_batch + ik * a.k_inner;
+  const TIn *Vd = static_cast<const TIn *>(a.V) + b * a.v_batch + ik * a.v_inner;
   const TIn *Kp = Kd, *Vp = Vd;
   long long kp_row = a.k_row, vp_row = a.v_row;
   if (MODE == kPrefill) {
-    Kp = static_cast<const TIn *>(a.k_rows) + a.row_off[prob] * (long long)D;
-    Vp = static_cast<const TIn *>(a.v_rows) + a.row_off[prob] * (long long)D;
+    Kp = static_cast<const TIn *>(a.k_rows) + a.row_off[prob_kv] * (long long)D;
+    Vp = static_cast<const TIn *>(a.v_rows) + a.row_off[prob_kv] * (long long)D;
     kp_row = D; vp_row = D;
   }
-  const int32_t *pre = MODE == kPrefill ? a.prefix + (size_t)prob * (a.n + 1) : nullptr;
+  const int32_t *pre = MODE == kPrefill ? a.prefix + (size_t)prob_kv * (a.n + 1) : nullptr;
   const int n_keys = (MODE == kGateFull && a.seq_lens) ? a.seq_lens[prob / a.inner] : a.n;
 
   // Q tile -> shared (rows past n are clamped; they are never stored)

@@ -151,13 +151,13 @@ static int row_bytes(const ag_layer_desc &d) {
 
 size_t compact_workspace_bytes(const ag_layer_desc &d) {
   // room for idx when the caller does not want it back
-  return align_up((size_t)d.batch * d.heads * d.seq * sizeof(int32_t), 256);
+  return align_up((size_t)d.batch * kv_heads_of(d) * d.seq * sizeof(int32_t), 256);
 }
 
 int launch_compact(const ag_layer_desc &d, const void *K, const void *V, const uint8_t *flags,
                    const ag_cache &c, int32_t *prefix, int32_t *idx, int32_t *dev_status,
                    void *ws, cudaStream_t st) {
-  const int slabs = d.batch * d.heads;
+  const int slabs = d.batch * kv_heads_of(d);
   int32_t *ix = idx ? idx : static_cast<int32_t *>(ws);
   dim3 grid((d.seq + kCompactThreads - 1) / kCompactThreads, slabs);
   auto Kb = static_cast<const uint8_t *>(K);
@@ -187,7 +187,7 @@ int launch_compact(const ag_layer_desc &d, const void *K, const void *V, const u
 int launch_append(const ag_layer_desc &d, const void *k_new, const void *v_new,
                   const uint8_t *flag_new, const ag_cache &c, int32_t *dev_status,
                   cudaStream_t st) {
-  const int slabs = d.batch * d.heads;
+  const int slabs = d.batch * kv_heads_of(d);
   const int rb = row_bytes(d);
   auto kn = static_cast<const uint8_t *>(k_new);
   auto vn = static_cast<const uint8_t *>(v_new);

@@ -26,6 +26,15 @@ constexpr int kUnroll = 8;         // rows in flight per lane group (x2: K and V
 constexpr int kClusterMaxSlabs = 64;    // up to here one cluster per slab; beyond, split-K through the workspace
 constexpr int kClusterThreads = 512;    // 256 rows in flight per CTA of a cluster (bf16, D = 128)
 
+// Grouped-query attention: slab s = (sequence, query head) of q and o reads the cache slab, k_new
+// and v_new of its key/value head.
+struct HeadMap {
+  int heads, kv_heads;
+  __device__ __forceinline__ int kv_slab(int slab) const {
+    return (slab / heads) * kv_heads + (slab % heads) / (heads / kv_heads);
+  }
+};
+
 // The conditional append of the decoding stage (Sec. 3.1 with the gate's flag for the new token),
 // for kernels that carry it with the attention of the same step: flag_new = NULL means no append.
 struct AppendArgs {
@@ -129,18 +138,19 @@ __global__ void __launch_bounds__(kPartThreads)
 decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
                       const T *__restrict__ v_rows, const int64_t *__restrict__ row_off,
                       const int32_t *__restrict__ len, float scale_log2, int chunk_rows,
-                      float *__restrict__ part_o, float *__restrict__ part_ml) {
+                      float *__restrict__ part_o, float *__restrict__ part_ml, const HeadMap hm) {
   constexpr int kEpl = Elem<T>::kPerVec;
   constexpr int kLanes = D / kEpl;
   constexpr int kGroups = kPartThreads / kLanes;
   const int slab = blockIdx.y, chunk = blockIdx.x;
-  const int L = len[slab];
+  const int kv = hm.kv_slab(slab);
+  const int L = len[kv];
   const int r_begin = chunk * chunk_rows;
   if (r_begin >= L) return;
   const int r_end = min(L, r_begin + chunk_rows);
   const int g = threadIdx.x / kLanes, v = threadIdx.x % kLanes;
   float m, l, o[kEpl];
-  decode_stream_rows<T, D, kPartThreads>(q, k_rows, v_rows, row_off[slab], slab, r_begin, r_end, scale_log2, m, l, o);
+  decode_stream_rows<T, D, kPartThreads>(q, k_rows, v_rows, row_off[kv], slab, r_begin, r_end, scale_log2, m, l, o);
 
   __shared__ float sm_m[kGroups], sm_l[kGroups];
   __shared__ float sm_o[kGroups][D];
@@ -174,14 +184,16 @@ decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
                       const T *__restrict__ v_new, const int32_t *__restrict__ len,
                       float scale_log2, int chunk_rows, const float *__restrict__ part_o,
                       const float *__restrict__ part_ml, T *__restrict__ o,
-                      const int64_t *__restrict__ row_off, const AppendArgs ap) {
+                      const int64_t *__restrict__ row_off, const AppendArgs ap, const HeadMap hm) {
   const int slab = blockIdx.x, d = threadIdx.x;
-  const int L = len[slab];
+  const int kv = hm.kv_slab(slab);
+  const int L = len[kv];
   // the chunk pass, the only reader of the slab's rows, has completed: the new row may go in
-  append_new_row<T, D>(ap, slab, L, row_off[slab], k_new, v_new);
+  // (never asked for when query heads share a slab: another head's CTA may still be reading its length)
+  append_new_row<T, D>(ap, kv, L, row_off[kv], k_new, v_new);
   const int n_chunks = (L + chunk_rows - 1) / chunk_rows;
   __shared__ float red[D / 32];
-  float a = Elem<T>::load(q + (size_t)slab * D + d) * Elem<T>::load(k_new + (size_t)slab * D + d);
+  float a = Elem<T>::load(q + (size_t)slab * D + d) * Elem<T>::load(k_new + (size_t)kv * D + d);
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
   if ((d & 31) == 0) red[d >> 5] = a;
@@ -194,7 +206,7 @@ decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
   float m = s_self;
   for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, pml[2 * c]);
   const float w_self = exp2f(s_self - m);
-  float acc = w_self * Elem<T>::load(v_new + (size_t)slab * D + d);
+  float acc = w_self * Elem<T>::load(v_new + (size_t)kv * D + d);
   float l = w_self;
   const float *po = part_o + (size_t)slab * kMaxSplits * D + d;
   for (int c = 0; c < n_chunks; ++c) {
@@ -216,16 +228,17 @@ __global__ void __launch_bounds__(kThreads)
 decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, const T *__restrict__ v_new,
                       const T *__restrict__ k_rows, const T *__restrict__ v_rows,
                       const int64_t *__restrict__ row_off, const int32_t *__restrict__ len,
-                      float scale_log2, T *__restrict__ out, const AppendArgs ap) {
+                      float scale_log2, T *__restrict__ out, const AppendArgs ap, const HeadMap hm) {
   namespace cg = cooperative_groups;
   constexpr int kEpl = Elem<T>::kPerVec;
   constexpr int kLanes = D / kEpl;
   constexpr int kGroups = kThreads / kLanes;
   cg::cluster_group cluster = cg::this_cluster();
   const int slab = blockIdx.y, rank = (int)cluster.block_rank();
+  const int kv = hm.kv_slab(slab);
   pdl_launch_dependents();
   pdl_wait();
-  const int L = len[slab];
+  const int L = len[kv];
   const int per = ((L + kClusterSize - 1) / kClusterSize + kGroups - 1) / kGroups * kGroups;
   const int r_begin = min(L, rank * per), r_end = min(L, r_begin + per);
   const int g = threadIdx.x / kLanes, v = threadIdx.x % kLanes;
@@ -239,10 +252,10 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
   // self score q . k_new: only the first CTA needs it; its loads are in flight with the stream's
   float prod = 0.f;
   if (rank == 0 && threadIdx.x < D)
-    prod = Elem<T>::load(q + (size_t)slab * D + threadIdx.x) * Elem<T>::load(k_new + (size_t)slab * D + threadIdx.x);
+    prod = Elem<T>::load(q + (size_t)slab * D + threadIdx.x) * Elem<T>::load(k_new + (size_t)kv * D + threadIdx.x);
 
   float m, l, o[kEpl];
-  decode_stream_rows<T, D, kThreads>(q, k_rows, v_rows, row_off[slab], slab, r_begin, r_end, scale_log2, m, l, o);
+  decode_stream_rows<T, D, kThreads>(q, k_rows, v_rows, row_off[kv], slab, r_begin, r_end, scale_log2, m, l, o);
 
   if (v == 0) { sm_m[g] = m; sm_l[g] = l; }
 #pragma unroll
@@ -272,7 +285,8 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
   }
   cluster.sync();
   // every CTA of the cluster has read the length and its rows: the new row may go in
-  if (rank == 0) append_new_row<T, D>(ap, slab, L, row_off[slab], k_new, v_new);
+  // (never asked for when query heads share a slab: another head's cluster may still be reading its length)
+  if (rank == 0) append_new_row<T, D>(ap, kv, L, row_off[kv], k_new, v_new);
   if (rank == 0 && threadIdx.x < D) {
     const int d = threadIdx.x;
     float s_self = 0.f;
@@ -291,7 +305,7 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
 #pragma unroll
     for (int r = 0; r < kClusterSize; ++r) mm = fmaxf(mm, mr[r]);
     const float w_self = exp2f(s_self - mm);
-    float acc = w_self * Elem<T>::load(v_new + (size_t)slab * D + d);
+    float acc = w_self * Elem<T>::load(v_new + (size_t)kv * D + d);
     float lsum = w_self;
 #pragma unroll
     for (int r = 0; r < kClusterSize; ++r) {
@@ -307,7 +321,7 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
 template <typename T, int D, int kThreads>
 static int launch_decode_cluster(int slabs, const void *q, const void *k_new, const void *v_new,
                                  const ag_cache &c, float scale_log2, void *o, const AppendArgs &ap,
-                                 cudaStream_t st) {
+                                 const HeadMap &hm, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(kClusterSize, slabs);
   cfg.blockDim = dim3(kThreads);
@@ -321,7 +335,7 @@ static int launch_decode_cluster(int slabs, const void *q, const void *k_new, co
   AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_cluster_kernel<T, D, kThreads>, static_cast<const T *>(q),
                                  static_cast<const T *>(k_new), static_cast<const T *>(v_new),
                                  static_cast<const T *>(c.k_rows), static_cast<const T *>(c.v_rows),
-                                 c.row_off, c.len, scale_log2, static_cast<T *>(o), ap));
+                                 c.row_off, c.len, scale_log2, static_cast<T *>(o), ap, hm));
   return AG_OK;
 }
 
@@ -333,10 +347,11 @@ size_t decode_workspace_bytes(const ag_layer_desc &d) {
 template <typename T, int D>
 static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
                       const ag_cache &c, float scale, void *o, void *ws, const AppendArgs &ap, cudaStream_t st) {
-  const int slabs = d.batch * d.heads;
+  const int slabs = d.batch * d.heads;              // one per (sequence, query head)
+  const HeadMap hm{d.heads, kv_heads_of(d)};
   const float scale_log2 = scale * 1.4426950408889634f;
   if (slabs <= kClusterMaxSlabs)
-    return launch_decode_cluster<T, D, kClusterThreads>(slabs, q, k_new, v_new, c, scale_log2, o, ap, st);
+    return launch_decode_cluster<T, D, kClusterThreads>(slabs, q, k_new, v_new, c, scale_log2, o, ap, hm, st);
   int chunk_rows = (c.max_cap + kMaxSplits - 1) / kMaxSplits;
   chunk_rows = (chunk_rows + 127) / 128 * 128;   // whole iterations of the partial kernel (bf16, D = 128)
   const int n_chunks = c.max_cap > 0 ? (c.max_cap + chunk_rows - 1) / chunk_rows : 0;
@@ -346,12 +361,12 @@ static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, 
     dim3 grid(n_chunks, slabs);
     decode_partial_kernel<T, D><<<grid, kPartThreads, 0, st>>>(
         static_cast<const T *>(q), static_cast<const T *>(c.k_rows),
-        static_cast<const T *>(c.v_rows), c.row_off, c.len, scale_log2, chunk_rows, part_o, part_ml);
+        static_cast<const T *>(c.v_rows), c.row_off, c.len, scale_log2, chunk_rows, part_o, part_ml, hm);
     AG_LAUNCH_CHECK();
   }
   decode_combine_kernel<T, D><<<slabs, D, 0, st>>>(
       static_cast<const T *>(q), static_cast<const T *>(k_new), static_cast<const T *>(v_new),
-      c.len, scale_log2, chunk_rows, part_o, part_ml, static_cast<T *>(o), c.row_off, ap);
+      c.len, scale_log2, chunk_rows, part_o, part_ml, static_cast<T *>(o), c.row_off, ap, hm);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
@@ -376,6 +391,12 @@ int launch_decode(const ag_layer_desc &d, const void *q, const void *k_new, cons
 int launch_decode_step(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
                        const uint8_t *flag_new, const ag_cache &c, float scale, void *o,
                        int32_t *dev_status, void *ws, cudaStream_t st) {
+  if (kv_heads_of(d) != d.heads) {
+    // query heads share a slab: the append waits for all of them, in a launch of its own
+    int rc = dispatch_decode(d, q, k_new, v_new, c, scale, o, ws, AppendArgs{}, st);
+    if (rc) return rc;
+    return launch_append(d, k_new, v_new, flag_new, c, dev_status, st);
+  }
   AppendArgs ap;
   ap.flag_new = flag_new; ap.cap = c.cap; ap.len = c.len;
   ap.k_rows = c.k_rows; ap.v_rows = c.v_rows; ap.dev_status = dev_status;

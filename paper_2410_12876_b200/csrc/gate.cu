@@ -188,7 +188,7 @@ static int run_gate(const ag_layer_desc &d, const void *X, const void *Wq, const
   AG_CUDA_TRY(cudaFuncSetAttribute(out_kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)out_smem));
   const int blocks = d.batch * ((d.seq + kOutTokens - 1) / kOutTokens);
   out_kern<<<blocks, kOutThreads, out_smem, st>>>(hcat, static_cast<const T *>(Wo), gamma, logit_tau,
-                                                 d.batch, d.seq, GD, d.heads, d.seq_lens, scores, flags);
+                                                 d.batch, d.seq, GD, kv_heads_of(d), d.seq_lens, scores, flags);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }

@@ -627,7 +627,7 @@ int launch_gate_attn_tc(const ag_layer_desc &d, const void *qkv_hi, const void *
   auto mo = gate_merge_out_kernel<__nv_bfloat16>;
   AG_CUDA_TRY(cudaFuncSetAttribute(mo, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mo_smem));
   const int blocks = d.batch * ((d.seq + kMoTokens - 1) / kMoTokens);
-  mo<<<blocks, kMoThreads, mo_smem, st>>>(a, static_cast<const __nv_bfloat16 *>(Wo), gamma, logit_tau, d.heads,
+  mo<<<blocks, kMoThreads, mo_smem, st>>>(a, static_cast<const __nv_bfloat16 *>(Wo), gamma, logit_tau, kv_heads_of(d),
                                           scores, flags);
   AG_LAUNCH_CHECK();
   return AG_OK;

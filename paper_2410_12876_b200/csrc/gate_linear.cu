@@ -211,7 +211,7 @@ static int run_gate_linear_tc(const ag_layer_desc &d, const void *X, const void 
   CUtensorMap tmX, tmW;
   int rc = make_tmap_2d_bf16(&tmX, X, a.M, d.hidden, (uint64_t)d.hidden * 2, kGlBM, kGlBK);
   if (rc) return rc;
-  rc = make_tmap_2d_bf16(&tmW, W, d.hidden, d.heads, (uint64_t)d.heads * 2, kGlBK, 64);
+  rc = make_tmap_2d_bf16(&tmW, W, d.hidden, kv_heads_of(d), (uint64_t)kv_heads_of(d) * 2, kGlBK, 64);
   if (rc) return rc;
   // split d over a cluster until about one CTA per SM streams X (at least four k blocks each)
   const int m_tiles = (a.M + kGlBM - 1) / kGlBM;
@@ -238,23 +238,23 @@ int launch_gate_linear(const ag_layer_desc &d, const void *X, const void *W, con
                        float *scores, uint8_t *flags, cudaStream_t st) {
   GateLinearArgs a;
   a.seq_lens = d.seq_lens; a.gamma = gamma; a.scores = scores; a.flags = flags;
-  a.M = d.batch * d.seq; a.n = d.seq; a.h = d.heads;
+  a.M = d.batch * d.seq; a.n = d.seq; a.h = kv_heads_of(d);
   a.kb_total = (d.hidden + kGlBK - 1) / kGlBK; a.kb_per_cta = a.kb_total;
   a.logit_tau = (float)log((double)d.tau / (1.0 - (double)d.tau));
-  const bool tc = d.dtype == AG_BF16 && d.heads <= kGlMaxN && d.heads % 8 == 0 && d.hidden % 8 == 0 &&
+  const bool tc = d.dtype == AG_BF16 && kv_heads_of(d) <= kGlMaxN && kv_heads_of(d) % 8 == 0 && d.hidden % 8 == 0 &&
                   (int64_t)d.batch * d.seq < ((int64_t)1 << 31) - kGlBM && (a.M + kGlBM - 1) / kGlBM <= 65535;
   if (tc) {
-    if (d.heads <= 32) return run_gate_linear_tc<32>(d, X, W, a, st);
+    if (kv_heads_of(d) <= 32) return run_gate_linear_tc<32>(d, X, W, a, st);
     return run_gate_linear_tc<64>(d, X, W, a, st);
   }
   const int blocks = (a.M + 7) / 8;
   if (d.dtype == AG_F32)
     gate_linear_simt_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float *>(X), static_cast<const float *>(W),
-                                                          gamma, a.logit_tau, a.M, a.n, d.hidden, d.heads, d.seq_lens, scores, flags);
+                                                          gamma, a.logit_tau, a.M, a.n, d.hidden, kv_heads_of(d), d.seq_lens, scores, flags);
   else
     gate_linear_simt_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(
         static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(W), gamma, a.logit_tau, a.M, a.n,
-        d.hidden, d.heads, d.seq_lens, scores, flags);
+        d.hidden, kv_heads_of(d), d.seq_lens, scores, flags);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }

@@ -17,9 +17,10 @@ static int run_prefill_simt(const ag_layer_desc &d, const void *Q, const void *K
                             cudaStream_t st) {
   SimtAttnArgs a{};
   a.Q = Q; a.K = K; a.V = V; a.O = O;
-  a.n = d.seq; a.inner = d.heads;
+  a.n = d.seq; a.inner = d.heads; a.kv_group = d.heads / kv_heads_of(d);
   const long long head = (long long)d.seq * D, batch = head * d.heads;
-  a.q_batch = a.k_batch = a.v_batch = a.o_batch = batch;
+  a.q_batch = a.o_batch = batch;
+  a.k_batch = a.v_batch = head * kv_heads_of(d);
   a.q_inner = a.k_inner = a.v_inner = a.o_inner = head;
   a.q_row = a.k_row = a.v_row = a.o_row = D;
   a.scale_log2 = scale * 1.4426950408889634f;

@@ -45,7 +45,8 @@ struct PrefillTcArgs {
   const int32_t *prefix;            // [slabs, n + 1]
   const int64_t *row_off;
   const int32_t *len;
-  int n, n_qtiles, slabs;
+  int n, n_qtiles, slabs;           // slabs: (sequence, query head) pairs
+  int heads, kv_heads;              // query heads share key/value heads in groups of heads / kv_heads
   float scale_log2;
 };
 
@@ -88,13 +89,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // heaviest query tiles first
   const int qt = a.n_qtiles - 1 - (int)(blockIdx.x / a.slabs);
-  const int slab = blockIdx.x % a.slabs;
+  const int slab = blockIdx.x % a.slabs;           // Q and O live here
+  // K, V, the flags' prefix counts and the cache belong to the key/value head (grouped-query attention)
+  const int kv_slab = (slab / a.heads) * a.kv_heads + (slab % a.heads) / (a.heads / a.kv_heads);
   const int j0 = qt * kPfBM;
   const int j_last = min(j0 + kPfBM, a.n) - 1;
-  const int32_t *pre = a.prefix + (size_t)slab * (a.n + 1);
+  const int32_t *pre = a.prefix + (size_t)kv_slab * (a.n + 1);
   const int max_bound = pre[j_last];               // keys any row of this tile may see
   const int n_kv = (max_bound + kPfBN - 1) / kPfBN;
-  const int row0 = (int)a.row_off[slab];
+  const int row0 = (int)a.row_off[kv_slab];
   static_assert(kPfKvBuf == kPfTile, "the self tile below spans exactly the two V stages");
   // uses of K stage 0 / 1 before the dense V tile: even / odd cache tiles
   const int k0_uses = (n_kv + 1) / 2, k1_uses = n_kv / 2;
@@ -133,8 +136,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // self tile: dense K rows j0 .. j0 + 127 across both V stages, which no P V needs before
         // the first softmax is done; the first cache tiles of K load alongside it
         mbar_arrive_expect_tx(&v_full[0], kPfTile);
-        tma_load_3d(sV, &tmKd, &v_full[0], 0, j0, slab);
-        tma_load_3d(sV + kPfPanel, &tmKd, &v_full[0], 64, j0, slab);
+        tma_load_3d(sV, &tmKd, &v_full[0], 0, j0, kv_slab);
+        tma_load_3d(sV + kPfPanel, &tmKd, &v_full[0], 64, j0, kv_slab);
         for (int i = 0; i < n_kv && ok; ++i) {
           const int st = i & 1;
           const int y = row0 + i * kPfBN;
@@ -155,8 +158,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       if (ok && k1_uses > 0) ok = mbar_wait(&k_empty[1], (k1_uses & 1) ^ 1);
       if (ok) {
         mbar_arrive_expect_tx(&k_full[0], kPfTile);
-        tma_load_3d(sK, &tmVd, &k_full[0], 0, j0, slab);
-        tma_load_3d(sK + kPfPanel, &tmVd, &k_full[0], 64, j0, slab);
+        tma_load_3d(sK, &tmVd, &k_full[0], 0, j0, kv_slab);
+        tma_load_3d(sK + kPfPanel, &tmVd, &k_full[0], 64, j0, kv_slab);
       }
     }
   } else if (warp == 1) {
@@ -247,7 +250,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int j = j0 + row;
     const bool valid = j < a.n;
     const int bound = valid ? pre[j] : 0;
-    const int L = a.len[slab];
+    const int L = a.len[kv_slab];
     const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
     float m = 0.f, self2 = 0.f, l = 1.f;
     bool ok = true;
@@ -412,8 +415,9 @@ int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, cons
   CUtensorMap tmQ, tmKd, tmVd, tmO, tmK, tmV;
   int rc;
   if ((rc = make_tmap_3d_bf16(&tmQ, Q, slabs, d.seq, kPfD, kPfBM, 64))) return rc;
-  if ((rc = make_tmap_3d_bf16(&tmKd, K, slabs, d.seq, kPfD, kPfBM, 64))) return rc;
-  if ((rc = make_tmap_3d_bf16(&tmVd, V, slabs, d.seq, kPfD, kPfBM, 64))) return rc;
+  const int kv_slabs = d.batch * kv_heads_of(d);
+  if ((rc = make_tmap_3d_bf16(&tmKd, K, kv_slabs, d.seq, kPfD, kPfBM, 64))) return rc;
+  if ((rc = make_tmap_3d_bf16(&tmVd, V, kv_slabs, d.seq, kPfD, kPfBM, 64))) return rc;
   if ((rc = make_tmap_3d_bf16(&tmO, O, slabs, d.seq, kPfD, kPfBM, 64))) return rc;
   // an empty pool still needs a valid map: describe one row of the dense K / V instead (never read)
   const bool empty = c.pool_rows == 0;
@@ -424,6 +428,7 @@ int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, cons
   PrefillTcArgs a;
   a.prefix = prefix; a.row_off = c.row_off; a.len = c.len;
   a.n = d.seq; a.n_qtiles = (d.seq + kPfBM - 1) / kPfBM; a.slabs = slabs;
+  a.heads = d.heads; a.kv_heads = kv_heads_of(d);
   a.scale_log2 = scale * 1.4426950408889634f;
   AG_CUDA_TRY(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes));
   prefill_tc_kernel<<<a.n_qtiles * slabs, kPfThreads, kPfSmemBytes, st>>>(tmQ, tmKd, tmVd, tmO, tmK, tmV, a);

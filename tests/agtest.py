@@ -45,7 +45,7 @@ def check_close(got, want, dtype, what=""):
 def gpu_gate(shape, X, W, gamma, want_scores=True):
     desc = ag.make_desc(shape)
     dev = X.device
-    B, h, n = shape.batch, shape.heads, shape.seq
+    B, h, n = shape.batch, shape.kvh, shape.seq              # one flag column per key/value head
     scores = torch.empty(B, h, n, dtype=torch.float32, device=dev) if want_scores else None
     flags = torch.full((B, h, n), 7, dtype=torch.uint8, device=dev)
     ws = ag.workspace(desc, ag.AG_CALL_GATE)
@@ -64,7 +64,7 @@ def check_flags(shape, flags_gpu, scores_ref, flags_ref, gamma):
     """Bit-exact outside the band |s + gamma - logit(tau)| < FLAG_BAND;
     returns the fraction of (head, token) pairs inside the band."""
     tau = float(np.float32(shape.tau))
-    g = np.zeros(shape.heads) if gamma is None else f64(gamma)
+    g = np.zeros(shape.kvh) if gamma is None else f64(gamma)
     dist = np.abs(scores_ref + g[None, :, None] - math.log(tau / (1 - tau)))
     outside = dist >= FLAG_BAND
     fg = flags_gpu.cpu().numpy()
@@ -76,7 +76,7 @@ def check_flags(shape, flags_gpu, scores_ref, flags_ref, gamma):
 def gpu_compact(shape, K, V, flags, cap=None, want_idx=True):
     desc = ag.make_desc(shape)
     dev = flags.device
-    B, h, n = shape.batch, shape.heads, shape.seq
+    B, h, n = shape.batch, shape.kvh, shape.seq              # one cache slab per key/value head
     if cap is None:
         cap = [n] * (B * h)
     cache = ag.RaggedCache.allocate(shape, cap, dev)
@@ -99,8 +99,8 @@ def check_compaction(shape, K, V, flags, cache, prefix, idx):
     kr, vr = bits(cache.k_rows), bits(cache.v_rows)
     off = cache.row_off.cpu().numpy()
     for b in range(shape.batch):
-        for i in range(shape.heads):
-            s = b * shape.heads + i
+        for i in range(shape.kvh):
+            s = b * shape.kvh + i
             c = ocache[b][i]
             assert np.array_equal(pre[b, i], orc.exclusive_counts(fl[b, i]))
             if ix is not None:
@@ -139,8 +139,8 @@ def gpu_cache_as_lists(cache, shape):
     out = []
     for b in range(shape.batch):
         row = []
-        for i in range(shape.heads):
-            s = b * shape.heads + i
+        for i in range(shape.kvh):
+            s = b * shape.kvh + i
             row.append({"k": kr[off[s]:off[s] + L[s]].copy(), "v": vr[off[s]:off[s] + L[s]].copy()})
         out.append(row)
     return out
