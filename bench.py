@@ -36,6 +36,7 @@ WORKLOADS = {
     "deep_layer": (inputs.DEEP_LAYER, 16, "deep-layer pattern, batch 1 x seq 16384: 24 heads keep ~10%, 8 heads keep nothing"),
     "stack7b": (inputs.STACK7B, 16, "32 AG-gated layers back to back, batch 8 x seq 4096; per-layer mean eviction rising from 10% to 90%"),
     "decode_ragged": (inputs.DECODE_RAGGED, 16, "ragged decode, batch 32 x 32 heads, retained lengths U[0.2,0.9] x 8192, keep-new Bernoulli(0.5)"),
+    "decode_ragged_gqa": (inputs.DECODE_RAGGED_GQA, 16, "ragged decode with grouped-query attention, batch 32 x 32 query heads over 8 key/value heads, retained lengths U[0.2,0.9] x 8192"),
 }
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None for workloads that were not captured).  To be reset to
@@ -162,7 +163,7 @@ class LayerRun:
         self.use_graph, self.graph = True, None
         self.has_gate = name in ("prefill7b", "tiny", "stack7b")
         self.layers = 32 if name == "stack7b" else 1
-        self.has_prefill = name != "decode_ragged"
+        self.has_prefill = name not in ("decode_ragged", "decode_ragged_gqa")
         if self.has_gate:
             self.X = inputs.hidden_states(sh, seed, dev)
             self.W = inputs.layer_weights(sh, seed + 10, dev)
@@ -184,7 +185,7 @@ class LayerRun:
             self.cache = ag.RaggedCache.allocate(sh, [n + self.decode_steps] * (B * h), dev)
         else:
             # the cache is the input: tight slabs of seeded random length, filled with N(0, 1)
-            self.L0 = inputs.ragged_lengths(B * h, n, seed + 30)
+            self.L0 = inputs.ragged_lengths(B * sh.kvh, n, seed + 30)       # one slab per key/value head
             self.cache = ag.RaggedCache.allocate(sh, (self.L0.astype(np.int64) + 256).tolist(), dev)
             for t, sd in ((self.cache.k_rows, seed + 31), (self.cache.v_rows, seed + 32)):
                 step_rows = 1 << 20

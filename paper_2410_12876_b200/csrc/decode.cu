@@ -177,6 +177,116 @@ decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
   }
 }
 
+// Grouped-query form of the chunk pass: one CTA streams a chunk of a KEY/VALUE slab once for the
+// G query heads that share it (G = 2 or 4; rows in flight per lane group halved to make room for
+// G running softmaxes per thread) and leaves one triple per query head, where
+// decode_combine_kernel expects it.
+constexpr int kUnrollGqa = 4;
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kPartThreads)
+decode_partial_gqa_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
+                          const T *__restrict__ v_rows, const int64_t *__restrict__ row_off,
+                          const int32_t *__restrict__ len, float scale_log2, int chunk_rows,
+                          float *__restrict__ part_o, float *__restrict__ part_ml, int kv_heads) {
+  constexpr int kEpl = Elem<T>::kPerVec;
+  constexpr int kLanes = D / kEpl;
+  constexpr int kGroups = kPartThreads / kLanes;
+  const int kv = blockIdx.y, chunk = blockIdx.x;
+  const int slab0 = (kv / kv_heads) * kv_heads * G + (kv % kv_heads) * G;   // first query slab of the group
+  const int L = len[kv];
+  const int r_begin = chunk * chunk_rows;
+  if (r_begin >= L) return;
+  const int r_end = min(L, r_begin + chunk_rows);
+  const int g = threadIdx.x / kLanes, v = threadIdx.x % kLanes;
+
+  float qf[G][kEpl], o[G][kEpl], m[G], l[G];
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    Elem<T>::unpack(ldg128(q + (size_t)(slab0 + h) * D + v * kEpl), qf[h]);
+    m[h] = -INFINITY; l[h] = 0.f;
+#pragma unroll
+    for (int e = 0; e < kEpl; ++e) { qf[h][e] *= scale_log2; o[h][e] = 0.f; }
+  }
+  const T *Kb = k_rows + (size_t)row_off[kv] * D + v * kEpl;
+  const T *Vb = v_rows + (size_t)row_off[kv] * D + v * kEpl;
+
+  // uniform trip count (the shuffles need whole warps); rows past r_end are clamped and get weight 0
+  for (int r0 = r_begin; r0 < r_end; r0 += kUnrollGqa * kGroups) {
+    const int r = r0 + g;
+    uint4 kv4[kUnrollGqa], vv4[kUnrollGqa];
+#pragma unroll
+    for (int u = 0; u < kUnrollGqa; ++u) {
+      const int ru = min(r + u * kGroups, r_end - 1);
+      kv4[u] = ldg128_stream(Kb + (size_t)ru * D);
+      vv4[u] = ldg128_stream(Vb + (size_t)ru * D);
+    }
+    float sc[kUnrollGqa][G];
+#pragma unroll
+    for (int u = 0; u < kUnrollGqa; ++u) {
+      float kf[kEpl];
+      Elem<T>::unpack(kv4[u], kf);
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        float a = 0.f;
+#pragma unroll
+        for (int e = 0; e < kEpl; ++e) a = fmaf(qf[h][e], kf[e], a);
+#pragma unroll
+        for (int off = kLanes / 2; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+        sc[u][h] = (r + u * kGroups < r_end) ? a : -INFINITY;
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      float m_new = m[h];
+#pragma unroll
+      for (int u = 0; u < kUnrollGqa; ++u) m_new = fmaxf(m_new, sc[u][h]);
+      const float alpha = (m_new == -INFINITY) ? 1.f : exp2f(m[h] - m_new);
+      l[h] *= alpha;
+#pragma unroll
+      for (int e = 0; e < kEpl; ++e) o[h][e] *= alpha;
+#pragma unroll
+      for (int u = 0; u < kUnrollGqa; ++u) {
+        const float p = (sc[u][h] == -INFINITY) ? 0.f : exp2f(sc[u][h] - m_new);
+        l[h] += p;
+        float vf[kEpl];
+        Elem<T>::unpack(vv4[u], vf);
+#pragma unroll
+        for (int e = 0; e < kEpl; ++e) o[h][e] = fmaf(p, vf[e], o[h][e]);
+      }
+      m[h] = m_new;
+    }
+  }
+
+  __shared__ float sm_m[G][kGroups], sm_l[G][kGroups];
+  __shared__ float sm_o[kGroups][D];
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    __syncthreads();                                 // sm_o of the previous head has been read
+    if (v == 0) { sm_m[h][g] = m[h]; sm_l[h][g] = l[h]; }
+#pragma unroll
+    for (int e = 0; e < kEpl; ++e) sm_o[g][v * kEpl + e] = o[h][e];
+    __syncthreads();
+    float mc = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < kGroups; ++i) mc = fmaxf(mc, sm_m[h][i]);
+    const size_t slot = (size_t)(slab0 + h) * kMaxSplits + chunk;
+    for (int d = threadIdx.x; d < D; d += kPartThreads) {
+      float acc = 0.f;
+#pragma unroll
+      for (int i = 0; i < kGroups; ++i)
+        acc = fmaf(sm_m[h][i] == -INFINITY ? 0.f : exp2f(sm_m[h][i] - mc), sm_o[i][d], acc);
+      part_o[slot * D + d] = acc;
+    }
+    if (threadIdx.x == 0) {
+      float lc = 0.f;
+#pragma unroll
+      for (int i = 0; i < kGroups; ++i) lc = fmaf(sm_m[h][i] == -INFINITY ? 0.f : exp2f(sm_m[h][i] - mc), sm_l[h][i], lc);
+      part_ml[slot * 2 + 0] = mc;
+      part_ml[slot * 2 + 1] = lc;
+    }
+  }
+}
+
 // One CTA of D threads per slab: thread d owns output dimension d.
 template <typename T, int D>
 __global__ void __launch_bounds__(D)
@@ -357,7 +467,20 @@ static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, 
   const int n_chunks = c.max_cap > 0 ? (c.max_cap + chunk_rows - 1) / chunk_rows : 0;
   float *part_o = static_cast<float *>(ws);
   float *part_ml = part_o + (size_t)slabs * kMaxSplits * D;
-  if (n_chunks > 0) {
+  const int group = hm.heads / hm.kv_heads;
+  if (n_chunks > 0 && (group == 2 || group == 4)) {
+    // grouped-query attention: the rows of a key/value slab are read once for its query heads
+    dim3 grid(n_chunks, d.batch * hm.kv_heads);
+    auto qp = static_cast<const T *>(q);
+    auto kr = static_cast<const T *>(c.k_rows), vr = static_cast<const T *>(c.v_rows);
+    if (group == 2)
+      decode_partial_gqa_kernel<T, D, 2><<<grid, kPartThreads, 0, st>>>(qp, kr, vr, c.row_off, c.len, scale_log2,
+                                                                         chunk_rows, part_o, part_ml, hm.kv_heads);
+    else
+      decode_partial_gqa_kernel<T, D, 4><<<grid, kPartThreads, 0, st>>>(qp, kr, vr, c.row_off, c.len, scale_log2,
+                                                                         chunk_rows, part_o, part_ml, hm.kv_heads);
+    AG_LAUNCH_CHECK();
+  } else if (n_chunks > 0) {
     dim3 grid(n_chunks, slabs);
     decode_partial_kernel<T, D><<<grid, kPartThreads, 0, st>>>(
         static_cast<const T *>(q), static_cast<const T *>(c.k_rows),

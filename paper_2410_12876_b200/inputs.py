@@ -50,6 +50,8 @@ PREFILL7B = LayerShape(1, 4096, 4096, 32, 128, 4, 128, "bf16")
 DECODE_RAGGED = LayerShape(32, 8192, 4096, 32, 128, 4, 128, "bf16")
 DEEP_LAYER = LayerShape(1, 16384, 4096, 32, 128, 4, 128, "bf16")
 STACK7B = LayerShape(8, 4096, 4096, 32, 128, 4, 128, "bf16")
+# grouped-query variant of the ragged decode shape (Mistral-7B-like: 32 query heads over 8 key/value heads)
+DECODE_RAGGED_GQA = LayerShape(32, 8192, 4096, 32, 128, 4, 128, "bf16", kv_heads=8)
 
 
 def _gen(seed, device):
