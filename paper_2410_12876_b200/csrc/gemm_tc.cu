@@ -2,7 +2,9 @@
 // the accumulator in tensor memory, operands staged by TMA), used for the gate's
 // projection [Q' | K' | V'] = X [Wq_g | Wk_g | Wv_g] (Sec. 3.3, MHA').
 //
-// One CTA computes a 128 x BN tile of the packed output.  Warp 0 drives TMA,
+// One CTA computes a 128 x BN tile of the packed output - or, for the tiles of a last wave that
+// would fill less than half of the SMs, one half of it (each such tile goes to two CTAs of
+// BN / 2 columns, so that the wave ends in about half the time).  Warp 0 drives TMA,
 // warp 1 owns TMEM and issues the MMAs, warps 2..5 drain the accumulator: the
 // float32 form straight to global memory, the hi / lo bf16 form through the
 // (by then free) operand stages and TMA stores, which write whole 128-byte lines.
@@ -33,7 +35,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                     const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
                     const __grid_constant__ CUtensorMap tmChi, const __grid_constant__ CUtensorMap tmClo,
-                    float *__restrict__ C, bool split, int M, int K, int GD) {
+                    float *__restrict__ C, bool split, int M, int K, int GD, int n_tiles_n, int halved_from) {
   using Cfg = GemmTcCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -43,8 +45,13 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.y * kTcBM;
-  const int n0 = blockIdx.x * BN;              // column in the packed [3 * GD] output
+  // CTAs below halved_from take whole tiles (row-major over the tile grid), the rest half tiles
+  const int cta = blockIdx.x;
+  const bool halved = cta >= halved_from;
+  const int tile = halved ? halved_from + ((cta - halved_from) >> 1) : cta;
+  const int bn = halved ? BN / 2 : BN;         // columns of this CTA (a multiple of 64)
+  const int m0 = (tile / n_tiles_n) * kTcBM;
+  const int n0 = (tile % n_tiles_n) * BN + (halved ? ((cta - halved_from) & 1) * (BN / 2) : 0);   // in the packed [3 * GD] output
   const int which = n0 / GD, nw = n0 % GD;     // BN divides GD: a tile never straddles two weights
   const CUtensorMap *tmB = which == 0 ? &tmB0 : (which == 1 ? &tmB1 : &tmB2);
   const int num_kb = (K + kTcBK - 1) / kTcBK;
@@ -72,16 +79,15 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const uint32_t ph = (kb / Cfg::kStages) & 1;
         if (!mbar_wait(&empty[s], ph ^ 1)) break;
         uint8_t *a = smem + s * Cfg::kStageBytes, *b = a + Cfg::kABytes;
-        mbar_arrive_expect_tx(&full[s], Cfg::kStageBytes);
+        mbar_arrive_expect_tx(&full[s], Cfg::kABytes + (bn / 64) * Cfg::kPanelBytes);
         tma_load_2d(a, &tmA, &full[s], kb * kTcBK, m0);
-#pragma unroll
-        for (int p = 0; p < BN / 64; ++p)
+        for (int p = 0; p < bn / 64; ++p)
           tma_load_2d(b + p * Cfg::kPanelBytes, tmB, &full[s], nw + p * 64, kb * kTcBK);
       }
     }
   } else if (warp == 1) {
     // every lane runs the control flow (operands stay warp-uniform); one elected lane issues
-    constexpr uint32_t idesc = idesc_bf16_f32(kTcBM, BN, false, true);
+    const uint32_t idesc = idesc_bf16_f32(kTcBM, bn, false, true);
     const uint64_t da0 = desc_kmajor_sw128(smem_u32(smem));
     const uint64_t db0 = desc_mnmajor_sw128(smem_u32(smem) + Cfg::kABytes, Cfg::kPanelBytes);
     const uint32_t a_lo0 = (uint32_t)da0, a_hi = (uint32_t)(da0 >> 32);
@@ -121,7 +127,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int r_in = quad * 32 + lane;
       uint8_t *stage_lo = smem + (BN / 64) * kTcBM * 128;
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = 0; c < bn; c += 32) {
         uint32_t r[32];
         tmem_ld_x32_sync(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
         const uint32_t panel = (uint32_t)(c >> 6) * kTcBM * 128 + r_in * 128;
@@ -145,8 +151,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       fence_proxy_async_smem();
       named_barrier_sync(1, 128);
       if (threadIdx.x == 64) {
-#pragma unroll
-        for (int p = 0; p < BN / 64; ++p) {            // rows past M are dropped by the tensor map
+        for (int p = 0; p < bn / 64; ++p) {            // rows past M are dropped by the tensor map
           tma_store_2d(&tmChi, smem + p * kTcBM * 128, n0 + p * 64, m0);
           tma_store_2d(&tmClo, stage_lo + p * kTcBM * 128, n0 + p * 64, m0);
         }
@@ -156,7 +161,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     } else if (ok && num_kb > 0) {
       const size_t crow = (size_t)row * 3 * GD + n0;
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = 0; c < bn; c += 32) {
         uint32_t r[32];
         tmem_ld_x32_sync(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
         if (row < M) {
@@ -243,8 +248,19 @@ static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void
   }
   auto kern = gemm_bf16_tc_kernel<BN>;
   AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-  dim3 grid(3 * GD / BN, (M + kTcBM - 1) / kTcBM);
-  kern<<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(tmA, tmB[0], tmB[1], tmB[2], tmC[0], tmC[1], C, Chi != nullptr, M, K, GD);
+  const int n_tiles_n = 3 * GD / BN, n_tiles = n_tiles_n * ((M + kTcBM - 1) / kTcBM);
+  // tiles of a last wave that would fill at most half of the SMs are halved
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, v = 0;
+    sms = (cudaGetDevice(&dev) == cudaSuccess &&
+           cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) ? v : 148;
+  }
+  const int tail = n_tiles % sms;
+  const int halved_from = (BN >= 128 && tail > 0 && 2 * tail <= sms) ? n_tiles - tail : n_tiles;
+  const int ctas = halved_from + 2 * (n_tiles - halved_from);
+  kern<<<ctas, kTcThreads, Cfg::kSmemBytes, st>>>(tmA, tmB[0], tmB[1], tmB[2], tmC[0], tmC[1], C, Chi != nullptr, M, K,
+                                                  GD, n_tiles_n, halved_from);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
