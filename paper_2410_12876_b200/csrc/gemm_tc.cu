@@ -21,22 +21,25 @@ using namespace umma;
 
 constexpr int kTcBM = 128, kTcBK = 64, kTcThreads = 192;
 
-template <int BN> struct GemmTcCfg {
-  static constexpr int kStages = BN == 256 ? 4 : 6;
-  static constexpr int kABytes = kTcBM * kTcBK * 2;          // 16 KB
+// MT: 128-row sub-tiles of A per CTA (1 or 2; two share every B stage, a third less traffic per FLOP).
+template <int BN, int MT> struct GemmTcCfg {
+  static constexpr int kStages = BN == 256 ? (MT == 2 ? 3 : 4) : 6;
+  static constexpr int kABytes = MT * kTcBM * kTcBK * 2;     // 16 KB per sub-tile
   static constexpr int kPanelBytes = kTcBK * 64 * 2;         // [64 k][64 n] = 8 KB
   static constexpr int kBBytes = (BN / 64) * kPanelBytes;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
 };
 
-template <int BN>
+template <int BN, int MT>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                     const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
                     const __grid_constant__ CUtensorMap tmChi, const __grid_constant__ CUtensorMap tmClo,
                     float *__restrict__ C, bool split, int M, int K, int GD, int n_tiles_n, int halved_from) {
-  using Cfg = GemmTcCfg<BN>;
+  using Cfg = GemmTcCfg<BN, MT>;
+  constexpr uint32_t kTmemCols = MT * BN;
+  static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "TMEM columns: a power of two");
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t *full = reinterpret_cast<uint64_t *>(smem + Cfg::kStages * Cfg::kStageBytes);
@@ -50,7 +53,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const bool halved = cta >= halved_from;
   const int tile = halved ? halved_from + ((cta - halved_from) >> 1) : cta;
   const int bn = halved ? BN / 2 : BN;         // columns of this CTA (a multiple of 64)
-  const int m0 = (tile / n_tiles_n) * kTcBM;
+  const int m0 = (tile / n_tiles_n) * (MT * kTcBM);
   const int n0 = (tile % n_tiles_n) * BN + (halved ? ((cta - halved_from) & 1) * (BN / 2) : 0);   // in the packed [3 * GD] output
   const int which = n0 / GD, nw = n0 % GD;     // BN divides GD: a tile never straddles two weights
   const CUtensorMap *tmB = which == 0 ? &tmB0 : (which == 1 ? &tmB1 : &tmB2);
@@ -64,7 +67,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     prefetch_tensormap(tmB);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, BN);
+    tmem_alloc(tmem_slot, kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before_sync();
@@ -80,7 +83,9 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (!mbar_wait(&empty[s], ph ^ 1)) break;
         uint8_t *a = smem + s * Cfg::kStageBytes, *b = a + Cfg::kABytes;
         mbar_arrive_expect_tx(&full[s], Cfg::kABytes + (bn / 64) * Cfg::kPanelBytes);
-        tma_load_2d(a, &tmA, &full[s], kb * kTcBK, m0);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)              // rows past M are filled with zeros
+          tma_load_2d(a + mt * (kTcBM * kTcBK * 2), &tmA, &full[s], kb * kTcBK, m0 + mt * kTcBM);
         for (int p = 0; p < bn / 64; ++p)
           tma_load_2d(b + p * Cfg::kPanelBytes, tmB, &full[s], nw + p * 64, kb * kTcBK);
       }
@@ -104,7 +109,10 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
         for (int k = 0; k < kTcBK / 16; ++k) {
           // 16 elements of K: 32 bytes along a K-major row; 16 k-rows (2048 B) of an MN-major panel
-          mma_ss_lohi(tmem_acc, a_lo + ((k * 32) >> 4), a_hi, b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+            mma_ss_lohi(tmem_acc + mt * BN, a_lo + ((mt * kTcBM * kTcBK * 2 + k * 32) >> 4), a_hi,
+                        b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
         }
         mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
       }
@@ -115,9 +123,12 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   } else {
     // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32)
     const int quad = warp & 3;
-    const int row = m0 + quad * 32 + lane;
     const bool ok = mbar_wait(acc_full, 0);
     tc_fence_after_sync();
+#pragma unroll 1
+    for (int mt = 0; mt < MT; ++mt) {
+    const int row = m0 + mt * kTcBM + quad * 32 + lane;
+    const uint32_t tmem_sub = tmem_acc + mt * BN;
     if (ok && num_kb > 0 && split) {
       // x = hi + lo in bf16 pairs, for consumers that rebuild float32 precision from three
       // products.  Every MMA has completed, so every stage has been read: the tile is staged
@@ -129,7 +140,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll 1
       for (int c = 0; c < bn; c += 32) {
         uint32_t r[32];
-        tmem_ld_x32_sync(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
+        tmem_ld_x32_sync(tmem_sub + ((uint32_t)(quad * 32) << 16) + c, r);
         const uint32_t panel = (uint32_t)(c >> 6) * kTcBM * 128 + r_in * 128;
 #pragma unroll
         for (int e = 0; e < 32; e += 8) {
@@ -152,18 +163,19 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       named_barrier_sync(1, 128);
       if (threadIdx.x == 64) {
         for (int p = 0; p < bn / 64; ++p) {            // rows past M are dropped by the tensor map
-          tma_store_2d(&tmChi, smem + p * kTcBM * 128, n0 + p * 64, m0);
-          tma_store_2d(&tmClo, stage_lo + p * kTcBM * 128, n0 + p * 64, m0);
+          tma_store_2d(&tmChi, smem + p * kTcBM * 128, n0 + p * 64, m0 + mt * kTcBM);
+          tma_store_2d(&tmClo, stage_lo + p * kTcBM * 128, n0 + p * 64, m0 + mt * kTcBM);
         }
         tma_store_commit();
         tma_store_wait_read();
       }
+      if (MT > 1) named_barrier_sync(1, 128);          // the staging area is free for the next sub-tile
     } else if (ok && num_kb > 0) {
       const size_t crow = (size_t)row * 3 * GD + n0;
 #pragma unroll 1
       for (int c = 0; c < bn; c += 32) {
         uint32_t r[32];
-        tmem_ld_x32_sync(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
+        tmem_ld_x32_sync(tmem_sub + ((uint32_t)(quad * 32) << 16) + c, r);
         if (row < M) {
 #pragma unroll
           for (int e = 0; e < 32; e += 4)
@@ -171,10 +183,11 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
     }
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_acc, BN);
+  if (warp == 1) tmem_dealloc(tmem_acc, kTmemCols);
 }
 
 // ------------------------------------------------------------ tensor maps
@@ -226,10 +239,20 @@ int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t planes, uint6
 }
 
 // ----------------------------------------------------------------- launch
-template <int BN>
+static int gemm_sm_count() {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, v = 0;
+    sms = (cudaGetDevice(&dev) == cudaSuccess &&
+           cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) ? v : 148;
+  }
+  return sms;
+}
+
+template <int BN, int MT>
 static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C,
                        __nv_bfloat16 *Chi, __nv_bfloat16 *Clo, int M, int K, int GD, cudaStream_t st) {
-  using Cfg = GemmTcCfg<BN>;
+  using Cfg = GemmTcCfg<BN, MT>;
   CUtensorMap tmA, tmB[3];
   int rc = make_tmap_2d_bf16(&tmA, X, M, K, (uint64_t)K * 2, kTcBM, kTcBK);
   if (rc) return rc;
@@ -246,18 +269,13 @@ static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void
              : make_tmap_2d_bf16(&tmC[i], outs[i], 1, GD, (uint64_t)GD * 2, 1, 64);
     if (rc) return rc;
   }
-  auto kern = gemm_bf16_tc_kernel<BN>;
+  auto kern = gemm_bf16_tc_kernel<BN, MT>;
   AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-  const int n_tiles_n = 3 * GD / BN, n_tiles = n_tiles_n * ((M + kTcBM - 1) / kTcBM);
+  const int n_tiles_n = 3 * GD / BN, n_tiles = n_tiles_n * ((M + MT * kTcBM - 1) / (MT * kTcBM));
   // tiles of a last wave that would fill at most half of the SMs are halved
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0, v = 0;
-    sms = (cudaGetDevice(&dev) == cudaSuccess &&
-           cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) ? v : 148;
-  }
+  const int sms = gemm_sm_count();
   const int tail = n_tiles % sms;
-  const int halved_from = (BN >= 128 && tail > 0 && 2 * tail <= sms) ? n_tiles - tail : n_tiles;
+  const int halved_from = (BN >= 128 && tail > 0 && 2 * tail <= sms) ? n_tiles - tail : n_tiles;   // (any MT)
   const int ctas = halved_from + 2 * (n_tiles - halved_from);
   kern<<<ctas, kTcThreads, Cfg::kSmemBytes, st>>>(tmA, tmB[0], tmB[1], tmB[2], tmC[0], tmC[1], C, Chi != nullptr, M, K,
                                                   GD, n_tiles_n, halved_from);
@@ -270,8 +288,14 @@ bool gate_proj_tc_supported(int K, int GD) { return GD % 128 == 0 && K % 8 == 0;
 int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, void *Chi,
                         void *Clo, int M, int K, int GD, cudaStream_t st) {
   auto hi = static_cast<__nv_bfloat16 *>(Chi), lo = static_cast<__nv_bfloat16 *>(Clo);
-  if (GD % 256 == 0) return run_gemm_tc<256>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
-  return run_gemm_tc<128>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
+  if (GD % 256 == 0) {
+    // more than one wave of 128 x 256 tiles: 256 x 256 tiles, whose two row sub-tiles share every
+    // stage of W (a third less operand traffic per FLOP; the kernel is bound by feeding the SMs)
+    const long long tiles128 = (long long)(3 * GD / 256) * ((M + kTcBM - 1) / kTcBM);
+    if (tiles128 > gemm_sm_count()) return run_gemm_tc<256, 2>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
+    return run_gemm_tc<256, 1>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
+  }
+  return run_gemm_tc<128, 1>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
 }
 
 int gemm_tc_wait_timeouts() {
