@@ -149,6 +149,28 @@ def ragged_gate(X, seq_lens, gate_fn):
     return scores, flags
 
 
+def previous_layer_flags(gate_fns, first_gated, shape):
+    """Eviction guided by the previous layer (Sec. 4.4, ablation settings (4-1) and
+    (4-2)): layer l evicts by the flags that layer l-1's AG module computes from
+    layer l-1's hidden states, so a layer's gate no longer has to finish before
+    that layer's attention starts.  Layers before `first_gated` (1 in setting
+    (4-1), 2 in (4-2)) evict nothing: their flags are all 1.
+
+    gate_fns[l]() returns (scores, flags) of layer l's AG module applied to layer
+    l's own hidden states; shape = (B, h, n) of a flag tensor.  Returns the list
+    of flag tensors the layers' attention uses, one per layer.  The last layer's
+    own gate has no consumer and is not evaluated."""
+    if first_gated < 1:
+        raise ValueError("the first layer has no previous layer to take flags from")
+    used = []
+    for l in range(len(gate_fns)):
+        if l < first_gated:
+            used.append(np.ones(shape, dtype=np.uint8))
+        else:
+            used.append(gate_fns[l - 1]()[1])
+    return used
+
+
 # --------------------------------------------------------------------------
 # Step 2: selective caching.  Sec. 3.3, sentence after Eq. 4: k_i^(t), v_i^(t)
 # are retained iff AG(X)_i^(t) = 1.

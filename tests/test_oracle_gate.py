@@ -186,3 +186,56 @@ def test_ragged_gate_padding_is_evicted_and_never_seen():
     s_full, _ = orc.attention_gate(X, Wq, Wk, Wv, Wo, hg, gamma=0.1, tau=0.5, causal=False)
     s_rag, _ = orc.ragged_gate(X, lens, lambda x: orc.attention_gate(x, Wq, Wk, Wv, Wo, hg, 0.1, 0.5, causal=False))
     assert not np.allclose(s_full[1, :, :4], s_rag[1, :, :4])
+
+
+# ---- eviction guided by the previous layer (Sec. 4.4, settings (4-1) and (4-2)) ----
+def _const_gate(keep, shape):
+    """A gate whose answer is known without computing anything: W^{O'} = 0 gives score 0, so
+    Sigmoid(gamma) > tau keeps every token (gamma large) or none (gamma very negative)."""
+    B, h, n = shape
+    rng = np.random.default_rng(5)
+    X = rng.standard_normal((B, n, 8))
+    Wq, Wk, Wv = (rng.standard_normal((8, 4)) for _ in range(3))
+    gamma = np.full(h, 20.0 if keep else -20.0)
+    return lambda: orc.attention_gate(X, Wq, Wk, Wv, np.zeros((4, h)), 2, gamma, 0.5)
+
+
+@pytest.mark.parametrize("first_gated", [1, 2])
+def test_previous_layer_flags_take_the_module_of_the_layer_before(first_gated):
+    shape = (2, 3, 6)
+    keeps = [False, True, False, False, True]          # what layer l's own module answers
+    used = orc.previous_layer_flags([_const_gate(k, shape) for k in keeps], first_gated, shape)
+    assert len(used) == len(keeps)
+    for l, f in enumerate(used):
+        assert f.shape == shape and f.dtype == np.uint8
+        expect = 1 if l < first_gated else int(keeps[l - 1])
+        assert (f == expect).all(), (l, first_gated)
+
+
+def test_previous_layer_flags_take_the_hidden_states_of_the_layer_before():
+    # one shared local gate with positive weights: a layer's flags are the sign of ITS hidden states
+    shape = (1, 2, 5)
+    W = np.ones((4, 2))
+    signs = [+1.0, -1.0, -1.0, +1.0]
+    Xs = [s * np.ones((1, 5, 4)) for s in signs]
+    gates = [lambda X=X: orc.linear_gate(X, W, np.zeros(2), 0.5) for X in Xs]
+    used = orc.previous_layer_flags(gates, 1, shape)
+    assert [int(f.all()) for f in used] == [1, 1, 0, 0]
+    assert [int(f.any()) for f in used] == [1, 1, 0, 0]
+
+
+def test_previous_layer_flags_unevicted_layers_are_plain_causal_attention():
+    shape = (1, 2, 7)
+    used = orc.previous_layer_flags([_const_gate(False, shape)] * 2, 1, shape)
+    rng = np.random.default_rng(11)
+    Q, K, V = (rng.standard_normal((1, 2, 7, 4)) for _ in range(3))
+    O = orc.prefill_attention(Q, K, V, used[0])
+    ref = torch.nn.functional.scaled_dot_product_attention(*(torch.from_numpy(t) for t in (Q, K, V)), is_causal=True)
+    np.testing.assert_allclose(O, ref.numpy(), rtol=1e-10, atol=1e-12)
+    # and the layer after it, guided by a module that evicts everything, sees only the diagonal
+    np.testing.assert_allclose(orc.prefill_attention(Q, K, V, used[1]), V, rtol=1e-12, atol=1e-12)
+
+
+def test_previous_layer_flags_need_a_previous_layer():
+    with pytest.raises(ValueError):
+        orc.previous_layer_flags([_const_gate(True, (1, 1, 2))], 0, (1, 1, 2))
