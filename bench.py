@@ -35,6 +35,9 @@ WORKLOADS = {
     "tiny": (inputs.TINY, 16, "fp32 correctness layer, batch 1 x seq 128, ~50% keep"),
     "deep_layer": (inputs.DEEP_LAYER, 16, "deep-layer pattern, batch 1 x seq 16384: 24 heads keep ~10%, 8 heads keep nothing"),
     "stack7b": (inputs.STACK7B, 16, "32 AG-gated layers back to back, batch 8 x seq 4096; per-layer mean eviction rising from 10% to 90%"),
+    "stack7b_prev": (inputs.STACK7B, 16, "the stack7b layers with eviction guided by the previous layer (ablation setting 4-1): "
+                                         "layer l runs under the flags of layer l-1's gate, the first layer evicts nothing, "
+                                         "each gate pass runs on a second stream beside its layer's attention"),
     "decode_ragged": (inputs.DECODE_RAGGED, 16, "ragged decode, batch 32 x 32 heads, retained lengths U[0.2,0.9] x 8192, keep-new Bernoulli(0.5)"),
     "decode_ragged_gqa": (inputs.DECODE_RAGGED_GQA, 16, "ragged decode with grouped-query attention, batch 32 x 32 query heads over 8 key/value heads, retained lengths U[0.2,0.9] x 8192"),
 }
@@ -161,8 +164,9 @@ class LayerRun:
         B, h, n, D = sh.batch, sh.heads, sh.seq, sh.head_dim
         self.name = name
         self.use_graph, self.graph = True, None
-        self.has_gate = name in ("prefill7b", "tiny", "stack7b")
-        self.layers = 32 if name == "stack7b" else 1
+        self.has_gate = name in ("prefill7b", "tiny", "stack7b", "stack7b_prev")
+        self.layers = 32 if name.startswith("stack7b") else 1
+        self.first_gated = 1 if name == "stack7b_prev" else 0      # 0: every layer evicts by its own gate
         self.has_prefill = name not in ("decode_ragged", "decode_ragged_gqa")
         if self.has_gate:
             self.X = inputs.hidden_states(sh, seed, dev)
@@ -179,6 +183,7 @@ class LayerRun:
         if self.has_prefill:
             self.scores = torch.empty(B, h, n, dtype=torch.float32, device=dev)
             self.flags = torch.empty(B, h, n, dtype=torch.uint8, device=dev)
+            self.cur_flags = self.flags                             # what compaction and prefill run under
             self.prefix = torch.empty(B, h, n + 1, dtype=torch.int32, device=dev)
             self.O = torch.empty_like(self.Q)
             # dense-capacity slabs: n rows + the decode steps of one pass
@@ -201,7 +206,7 @@ class LayerRun:
         self.gamma = None
         if self.has_gate:
             self.gate()
-            if name == "stack7b":
+            if self.layers > 1:
                 # the layers share X and the weights (inputs, not the timed work); what differs per
                 # layer is the keep rate, i.e. gamma: mean eviction 10 % (first) ... 90 % (last)
                 self.gammas = [inputs.calibrate_gamma(self.scores, inputs.keep_targets_layer(h, seed + 20, l), sh.tau).to(dev)
@@ -216,10 +221,10 @@ class LayerRun:
             for q in self.dq:
                 q[3][:, torch.from_numpy(empty).to(dev)] = 0     # fully evicted heads stay empty
 
-    def gate(self):
+    def gate(self, flags_out=None):
         W, ag = self.W, self.ag
         ag.ag_gate_forward(self.desc, self.X, W["Wq_g"], W["Wk_g"], W["Wv_g"], W["Wo_g"], self.gamma,
-                           self.scores, self.flags, self.ws[ag.AG_CALL_GATE])
+                           self.scores, self.flags if flags_out is None else flags_out, self.ws[ag.AG_CALL_GATE])
 
     def gate_linear(self):
         """The local gate (Sec. 3.4): same X, one [d, h] weight; timed on its own, not part of a step."""
@@ -230,12 +235,12 @@ class LayerRun:
 
     def compact(self):
         ag = self.ag
-        ag.ag_compact_kv(self.desc, self.K, self.V, self.flags, self.cache, self.prefix, None, self.status,
+        ag.ag_compact_kv(self.desc, self.K, self.V, self.cur_flags, self.cache, self.prefix, None, self.status,
                          self.ws[ag.AG_CALL_COMPACT])
 
     def prefill(self):
         ag = self.ag
-        ag.ag_prefill_attn(self.desc, self.Q, self.K, self.V, self.flags, self.cache, self.prefix, 0.0, self.O,
+        ag.ag_prefill_attn(self.desc, self.Q, self.K, self.V, self.cur_flags, self.cache, self.prefix, 0.0, self.O,
                            self.ws[ag.AG_CALL_PREFILL])
 
     def decode(self, s):
@@ -254,6 +259,8 @@ class LayerRun:
             fn(*a)
             e.record()
             ev[key].append((s, e))
+        if self.first_gated:
+            return self._step_guided_by_previous_layer(timed)
         for layer in range(self.layers):
             if self.has_gate:
                 self.gamma = self.gammas[layer]
@@ -264,6 +271,25 @@ class LayerRun:
             else:
                 self.cache.len.copy_(self.len0)      # every pass starts from the same cache
             timed("decode", self.decode_all)
+
+    def _step_guided_by_previous_layer(self, timed):
+        """Layer l runs under the flags of layer l-1's gate (Sec. 4.4, setting (4-1)); the gate passes
+        run on a second stream, each beside the compaction, prefill and decode of its own layer."""
+        if not hasattr(self, "schedule"):
+            from paper_2410_12876_b200.schedule import PreviousLayerGate
+            ones = torch.ones_like(self.flags)
+            self.schedule = PreviousLayerGate(self.first_gated, [self.flags, torch.empty_like(self.flags)], ones, self.dev)
+
+        def gate(layer, flags_out):
+            self.gamma = self.gammas[layer]
+            timed("gate", self.gate, flags_out)
+
+        def attend(layer, flags):
+            self.cur_flags = flags
+            timed("compact", self.compact)
+            timed("prefill", self.prefill)
+            timed("decode", self.decode_all)
+        self.schedule.run(self.layers, gate, attend)
 
     def decode_all(self):
         """All decode steps of a pass.  They are dozens of small launches, so they are
@@ -290,9 +316,9 @@ class LayerRun:
         return self.shape.batch * ((self.shape.seq if self.has_prefill else 0) + self.decode_steps) * self.layers
 
     def launches_per_step(self):
-        return self.layers * ((LAUNCHES["gate"] if self.has_gate else 0) +
-                              (LAUNCHES["compact"] + LAUNCHES["prefill"] if self.has_prefill else 0) +
-                              self.decode_steps * self.decode_launches())
+        gates = (self.layers - self.first_gated) if self.has_gate else 0      # the last guided layer's gate has no consumer
+        return gates * LAUNCHES["gate"] + self.layers * (
+            (LAUNCHES["compact"] + LAUNCHES["prefill"] if self.has_prefill else 0) + self.decode_steps * self.decode_launches())
 
     def decode_launches(self):
         slabs = self.shape.batch * self.shape.heads
@@ -308,7 +334,13 @@ class LayerRun:
         appended = float(sum(q[3].to(torch.float64).sum().item() for q in self.dq))
         f_eff, kept = [], []
         for layer in range(self.layers):
-            if self.has_gate:
+            if self.first_gated:
+                if layer < self.first_gated:
+                    self.cur_flags = torch.ones_like(self.flags)
+                else:
+                    self.gamma, self.cur_flags = self.gammas[layer - 1], self.flags
+                    self.gate()
+            elif self.has_gate:
                 self.gamma = self.gammas[layer]
                 self.gate()
             if self.has_prefill:
