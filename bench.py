@@ -33,13 +33,13 @@ WORKLOADS = {
     # name: (shape, decode steps per step, description)
     "prefill7b": (inputs.PREFILL7B, 16, "Llama-2-7B-shaped AG-gated layer, batch 1 x seq 4096, keep rates U[0.3,0.8] per head"),
     "tiny": (inputs.TINY, 16, "fp32 correctness layer, batch 1 x seq 128, ~50% keep"),
-    "deep_layer": (inputs.DEEP_LAYER, 16, "deep-layer pattern, batch 1 x seq 16384: 24 heads keep ~10%, 8 heads keep nothing"),
-    "stack7b": (inputs.STACK7B, 16, "32 AG-gated layers back to back, batch 8 x seq 4096; per-layer mean eviction rising from 10% to 90%"),
-    "stack7b_prev": (inputs.STACK7B, 16, "the stack7b layers with eviction guided by the previous layer (ablation setting 4-1): "
+    "deep_layer": (inputs.DEEP_LAYER, 128, "deep-layer pattern, batch 1 x seq 16384: 24 heads keep ~10%, 8 heads keep nothing"),
+    "stack7b": (inputs.STACK7B, 256, "32 AG-gated layers back to back, batch 8 x seq 4096; per-layer mean eviction rising from 10% to 90%"),
+    "stack7b_prev": (inputs.STACK7B, 256, "the stack7b layers with eviction guided by the previous layer (ablation setting 4-1): "
                                          "layer l runs under the flags of layer l-1's gate, the first layer evicts nothing, "
                                          "each gate pass runs on a second stream beside its layer's attention"),
-    "decode_ragged": (inputs.DECODE_RAGGED, 16, "ragged decode, batch 32 x 32 heads, retained lengths U[0.2,0.9] x 8192, keep-new Bernoulli(0.5)"),
-    "decode_ragged_gqa": (inputs.DECODE_RAGGED_GQA, 16, "ragged decode with grouped-query attention, batch 32 x 32 query heads over 8 key/value heads, retained lengths U[0.2,0.9] x 8192"),
+    "decode_ragged": (inputs.DECODE_RAGGED, 256, "ragged decode, batch 32 x 32 heads, retained lengths U[0.2,0.9] x 8192, keep-new Bernoulli(0.5)"),
+    "decode_ragged_gqa": (inputs.DECODE_RAGGED_GQA, 256, "ragged decode with grouped-query attention, batch 32 x 32 query heads over 8 key/value heads, retained lengths U[0.2,0.9] x 8192"),
 }
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None for workloads that were not captured).  To be reset to
