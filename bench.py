@@ -199,8 +199,10 @@ class LayerRun:
                     t[r0:r1] = inputs.randn((r1 - r0, D), sd + r0, dev, sh.torch_dtype)
             self.len0 = torch.from_numpy(self.L0).to(dev)
             self.cache.len.copy_(self.len0)
-        self.dq = [inputs.decode_inputs(sh, seed + 500, s, dev, keep_new=0.1 if name == "deep_layer" else 0.5)
-                   for s in range(self.decode_steps)]
+        # new-token flags: Bernoulli(0.1) on the deep layer, every token kept in the stack (the paper's
+        # decode stage runs no gate), Bernoulli(0.5) elsewhere
+        keep_new = 0.1 if name == "deep_layer" else 1.0 if self.layers > 1 else 0.5
+        self.dq = [inputs.decode_inputs(sh, seed + 500, s, dev, keep_new=keep_new) for s in range(self.decode_steps)]
         self.o = torch.empty(B, h, D, dtype=sh.torch_dtype, device=dev)
         # gamma: per-head keep rate ~ U[0.3, 0.8], calibrated on the scores at gamma = 0
         self.gamma = None

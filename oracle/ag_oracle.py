@@ -189,19 +189,28 @@ def exclusive_counts(flags_i):
     return np.asarray([int(f[:j].sum()) for j in range(n + 1)], dtype=np.int64)
 
 
-def compact_kv(K, V, flags):
+def compact_kv(K, V, flags, window=1):
     """Ragged cache after prefill: cache[b][i] = dict(k=[L, D], v=[L, D],
     idx=[L]) holding exactly the retained tokens in ascending position.
-    K, V [B, h, n, D] are copied bit-for-bit (dtype preserved)."""
+    K, V [B, h, n, D] are copied bit-for-bit (dtype preserved).
+
+    With a recent-token window (Appendix, Table 6: the `window` most recent
+    tokens, the current one included, are visible whatever their flags) the
+    slab also remembers the last window - 1 tokens as a list "recent" of
+    (k, v, flag), oldest first: the next window - 1 queries still see them."""
     K = np.asarray(K)
     V = np.asarray(V)
-    B, h = flags.shape[0], flags.shape[1]
+    B, h, n = flags.shape
     cache = []
     for b in range(B):
         row = []
         for i in range(h):
             idx = retained_indices(flags[b, i])
-            row.append({"k": K[b, i][idx].copy(), "v": V[b, i][idx].copy(), "idx": idx})
+            c = {"k": K[b, i][idx].copy(), "v": V[b, i][idx].copy(), "idx": idx}
+            if window > 1:
+                c["recent"] = [(K[b, i][t].copy(), V[b, i][t].copy(), int(flags[b, i][t]))
+                               for t in range(max(0, n - (window - 1)), n)]
+            row.append(c)
         cache.append(row)
     return cache
 
@@ -209,19 +218,24 @@ def compact_kv(K, V, flags):
 # --------------------------------------------------------------------------
 # Step 3: prefill attention under the eviction mask.  Eq. 2 and Eq. 5.
 # --------------------------------------------------------------------------
-def eviction_mask(flags_i, rows=None):
+def eviction_mask(flags_i, rows=None, window=1):
     """M_i[j, t] of Eq. 5 for one head: 0 above the diagonal (j < t), 1 on it,
     AG(X)_i^(t) below it.  j indexes queries (rows), t keys (columns).
-    `rows` selects a subset of query positions; default all."""
+    `rows` selects a subset of query positions; default all.
+
+    window = number of recent tokens always retained, the current one included
+    (Appendix, Table 6: 1 in the method as published, "only the current token
+    is retained", 5 and 10 in settings (6-1), (6-2)): the diagonal widens to
+    the band 0 <= j - t < window."""
     f = np.asarray(flags_i).astype(np.int64)
     n = f.shape[0]
     j = (np.arange(n) if rows is None else np.asarray(rows, dtype=np.int64))[:, None]
     t = np.arange(n)[None, :]
     below = np.broadcast_to(f[None, :], (j.shape[0], n))
-    return np.where(j < t, 0, np.where(j == t, 1, below))
+    return np.where(j < t, 0, np.where(j - t < window, 1, below))
 
 
-def prefill_head(Q_i, K_i, V_i, flags_i, scale=None, rows=None):
+def prefill_head(Q_i, K_i, V_i, flags_i, scale=None, rows=None, window=1):
     """H_i = Softmax(Q K^T / sqrt(d_k) - INF (1 - M_i)) V for one head
     (Eq. 2) with M_i from Eq. 5.  Q_i, K_i, V_i [n, D] -> [len(rows), D]."""
     Q_i, K_i, V_i = map(_as_f64, (Q_i, K_i, V_i))
@@ -230,7 +244,7 @@ def prefill_head(Q_i, K_i, V_i, flags_i, scale=None, rows=None):
         scale = 1.0 / math.sqrt(D)
     Qs = Q_i if rows is None else Q_i[np.asarray(rows, dtype=np.int64)]
     S = (Qs @ K_i.T) * scale
-    M = eviction_mask(flags_i, rows)
+    M = eviction_mask(flags_i, rows, window)
     S = np.where(M == 1, S, -np.inf)
     A = softmax_rows(S)
     return A @ V_i
@@ -244,7 +258,7 @@ def kv_head_of(i, h, h_kv):
     return i // (h // h_kv)
 
 
-def prefill_attention(Q, K, V, flags, scale=None):
+def prefill_attention(Q, K, V, flags, scale=None, window=1):
     """All heads of all sequences: Q [B, h, n, D], K, V [B, h_kv, n, D], flags [B, h_kv, n]
     -> [B, h, n, D] float64.  Query head i reads key/value head kv_head_of(i) and its flags."""
     B, h, n, D = np.asarray(Q).shape
@@ -253,7 +267,7 @@ def prefill_attention(Q, K, V, flags, scale=None):
     for b in range(B):
         for i in range(h):
             g = kv_head_of(i, h, h_kv)
-            O[b, i] = prefill_head(Q[b, i], K[b, g], V[b, g], flags[b, g], scale)
+            O[b, i] = prefill_head(Q[b, i], K[b, g], V[b, g], flags[b, g], scale, window=window)
     return O
 
 
@@ -278,7 +292,9 @@ def decode_head(q, k_new, v_new, k_cache, v_cache, scale=None):
 
 def decode_attention(q, k_new, v_new, cache, scale=None):
     """q [B, h, D]; k_new, v_new [B, h_kv, D]; cache as returned by compact_kv (one slab per
-    key/value head) -> [B, h, D].  Query head i reads slab kv_head_of(i)."""
+    key/value head) -> [B, h, D].  Query head i reads slab kv_head_of(i).  A slab with a
+    recent-token window also shows the query its evicted recent tokens (the retained ones are
+    rows of the cache already)."""
     q = np.asarray(q)
     B, h, D = q.shape
     h_kv = np.asarray(k_new).shape[1]
@@ -287,13 +303,20 @@ def decode_attention(q, k_new, v_new, cache, scale=None):
         for i in range(h):
             g = kv_head_of(i, h, h_kv)
             c = cache[b][g]
-            o[b, i] = decode_head(q[b, i], k_new[b, g], v_new[b, g], c["k"], c["v"], scale)
+            kc, vc = c["k"], c["v"]
+            evicted = [(k, v) for k, v, f in c.get("recent", []) if f == 0]
+            if evicted:
+                kc = np.concatenate([_as_f64(kc).reshape(-1, D)] + [_as_f64(k)[None, :] for k, _ in evicted], axis=0)
+                vc = np.concatenate([_as_f64(vc).reshape(-1, D)] + [_as_f64(v)[None, :] for _, v in evicted], axis=0)
+            o[b, i] = decode_head(q[b, i], k_new[b, g], v_new[b, g], kc, vc, scale)
     return o
 
 
-def cache_append(cache, k_new, v_new, flag_new):
+def cache_append(cache, k_new, v_new, flag_new, window=1):
     """Append (k_new, v_new)[b, i] to slab (b, i) iff flag_new[b, i] = 1.
-    Bit-for-bit copy; mutates and returns `cache`."""
+    Bit-for-bit copy; mutates and returns `cache`.  With a recent-token window
+    the token also joins the slab's recent list, whose oldest entry leaves
+    once the list holds window - 1 tokens."""
     k_new = np.asarray(k_new)
     v_new = np.asarray(v_new)
     B, h = flag_new.shape
@@ -303,6 +326,9 @@ def cache_append(cache, k_new, v_new, flag_new):
                 c = cache[b][i]
                 c["k"] = np.concatenate([c["k"], k_new[b, i][None, :]], axis=0)
                 c["v"] = np.concatenate([c["v"], v_new[b, i][None, :]], axis=0)
+            if window > 1:
+                c = cache[b][i]
+                c["recent"] = (c.get("recent", []) + [(k_new[b, i].copy(), v_new[b, i].copy(), int(flag_new[b, i]))])[-(window - 1):]
     return cache
 
 

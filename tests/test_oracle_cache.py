@@ -3,6 +3,7 @@
 import math
 
 import numpy as np
+import pytest
 
 from oracle import ag_oracle as orc
 
@@ -85,3 +86,23 @@ def test_append_is_conditional_and_bit_exact():
     # a token whose flag evicts it still attended to itself in decode_attention
     # but never reaches the cache of later steps
     assert cache[0][1]["k"].shape[0] == 3
+
+
+@pytest.mark.parametrize("w,n", [(2, 17), (5, 17), (10, 17), (5, 3), (4, 0)])
+def test_window_decode_matches_longer_prefill(w, n):
+    # the same statement two ways: the band mask on n + m tokens, and the cache with its
+    # list of recent tokens carried through m decode steps (prompts shorter than the window too)
+    B, h, m, D = 2, 2, 12, 8
+    Q, K, V = (_rand((B, h, n + m, D), s) for s in (21, 22, 23))
+    flags = (np.random.default_rng(24).random((B, h, n + m)) < 0.4).astype(np.uint8)
+    full = orc.prefill_attention(Q, K, V, flags, window=w)
+    assert not np.allclose(full, orc.prefill_attention(Q, K, V, flags))          # the window matters here
+    cache = orc.compact_kv(K[:, :, :n], V[:, :, :n], flags[:, :, :n], window=w)
+    for s in range(m):
+        t = n + s
+        o = orc.decode_attention(Q[:, :, t], K[:, :, t], V[:, :, t], cache)
+        assert np.max(np.abs(o - full[:, :, t])) < 1e-12, s
+        orc.cache_append(cache, K[:, :, t], V[:, :, t], flags[:, :, t], window=w)
+        assert all(len(c["recent"]) == min(w - 1, t + 1) for row in cache for c in row)
+    # the window never changes what is cached for good
+    assert np.array_equal(orc.cache_lengths(cache), flags.sum(axis=2))

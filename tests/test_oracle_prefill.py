@@ -153,7 +153,7 @@ def test_rows_subset_and_scale():
 def test_pins_catch_a_planted_mistake(monkeypatch):
     # Plant "flag indexed by the query instead of the key" in the oracle and
     # check that the brute-force pin notices.
-    def wrong_mask(flags_i, rows=None):
+    def wrong_mask(flags_i, rows=None, window=1):
         f = np.asarray(flags_i).astype(np.int64)
         n = f.shape[0]
         j = (np.arange(n) if rows is None else np.asarray(rows))[:, None]
@@ -196,3 +196,52 @@ def test_grouped_query_prefill_and_decode_equal_shared_heads_written_out():
     Q2[:, 1] = Q2[:, 0]
     O2 = orc.prefill_attention(Q2, K, V, f)
     assert np.array_equal(O2[:, 0], O2[:, 1])
+
+
+# ---- recent-token window (Appendix, Table 6: the w most recent tokens are always visible) ----
+def _visible_set_window(flags, j, w):
+    return [t for t in range(j + 1) if j - t < w or flags[t] == 1]
+
+
+@pytest.mark.parametrize("n,w", [(6, 2), (7, 3), (7, 5), (5, 10)])
+def test_window_brute_force_every_flag_pattern(n, w):
+    D = 3
+    Q, K, V = (_rand((n, D), 40 + n + s) for s in (0, 1, 2))
+    scale = 1.0 / math.sqrt(D)
+    for pattern in itertools.product([0, 1], repeat=n):
+        f = np.asarray(pattern, dtype=np.uint8)
+        O = orc.prefill_head(Q, K, V, f, window=w)
+        for j in range(n):
+            want = _attend_set(Q[j], K, V, _visible_set_window(pattern, j, w), scale)
+            assert np.max(np.abs(O[j] - want)) < 1e-12, (pattern, j)
+
+
+def test_window_of_one_is_the_published_method_and_a_full_window_is_causal_attention():
+    n, D = 9, 4
+    Q, K, V = (_rand((n, D), 70 + s) for s in (0, 1, 2))
+    f = (np.random.default_rng(73).random(n) < 0.4).astype(np.uint8)
+    assert np.array_equal(orc.eviction_mask(f, window=1), orc.eviction_mask(f))
+    assert np.array_equal(orc.prefill_head(Q, K, V, f, window=1), orc.prefill_head(Q, K, V, f))
+    # a window that covers the whole prompt leaves nothing to evict: the flags drop out
+    causal = orc.prefill_head(Q, K, V, np.ones(n, dtype=np.uint8))
+    np.testing.assert_allclose(orc.prefill_head(Q, K, V, f, window=n), causal, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(orc.prefill_head(Q, K, V, np.zeros(n, dtype=np.uint8), window=n + 3), causal, rtol=0, atol=1e-13)
+
+
+def test_window_mask_entries_all_evicted_is_a_band():
+    M = orc.eviction_mask(np.zeros(6, dtype=np.uint8), window=3)
+    want = np.array([[1, 0, 0, 0, 0, 0],
+                     [1, 1, 0, 0, 0, 0],
+                     [1, 1, 1, 0, 0, 0],
+                     [0, 1, 1, 1, 0, 0],
+                     [0, 0, 1, 1, 1, 0],
+                     [0, 0, 0, 1, 1, 1]])
+    assert np.array_equal(M, want)
+    # all evicted, window 2, value rows one-hot and equal scores: the mean of the last two values
+    n = 5
+    O = orc.prefill_head(np.zeros((n, 2)), np.ones((n, 2)), np.eye(n), np.zeros(n, dtype=np.uint8), window=2)
+    want = np.zeros((n, n))
+    want[0, 0] = 1.0
+    for j in range(1, n):
+        want[j, j] = want[j, j - 1] = 0.5
+    np.testing.assert_allclose(O, want, rtol=0, atol=1e-15)
