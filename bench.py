@@ -154,10 +154,13 @@ class ClockSampler:
 class LayerRun:
     """Device buffers of one workload and the five calls of one step."""
 
-    def __init__(self, name, seed, dev):
+    def __init__(self, name, seed, dev, recent_window=0):
         from paper_2410_12876_b200 import binding as ag
         self.ag = ag
         self.shape, self.decode_steps, self.desc_text = WORKLOADS[name]
+        if recent_window > 1:
+            assert name not in ("decode_ragged", "decode_ragged_gqa"), "the window needs a prompt to fill its ring from"
+            self.shape = self.shape.with_(recent_window=recent_window)
         sh = self.shape
         self.dev = dev
         self.desc = ag.make_desc(sh)
@@ -319,8 +322,10 @@ class LayerRun:
 
     def launches_per_step(self):
         gates = (self.layers - self.first_gated) if self.has_gate else 0      # the last guided layer's gate has no consumer
+        window = 2 if self.shape.recent_window > 1 else 0      # the ring fill after compaction, the band pass after prefill
         return gates * LAUNCHES["gate"] + self.layers * (
-            (LAUNCHES["compact"] + LAUNCHES["prefill"] if self.has_prefill else 0) + self.decode_steps * self.decode_launches())
+            (LAUNCHES["compact"] + LAUNCHES["prefill"] + window if self.has_prefill else 0)
+            + self.decode_steps * self.decode_launches())
 
     def decode_launches(self):
         slabs = self.shape.batch * self.shape.heads
@@ -385,7 +390,7 @@ def flush_l2(buf):
 
 def run_ours(args, rank, world, dev):
     torch.cuda.set_device(dev)
-    run = LayerRun(args.workload, 2000 + 100 * rank, dev)
+    run = LayerRun(args.workload, 2000 + 100 * rank, dev, args.recent_window)
     run.use_graph = not args.no_graph
     l2buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     dist = None
@@ -553,6 +558,7 @@ def run_ours(args, rank, world, dev):
         "config": {"workload": args.workload, "description": run.desc_text, "batch": sh.batch, "seq": sh.seq,
                    "hidden": sh.hidden, "heads": sh.heads, "head_dim": sh.head_dim, "gate_heads": sh.gate_heads,
                    "gate_head_dim": sh.gate_head_dim, "decode_steps_per_step": run.decode_steps,
+                   "recent_window": max(1, sh.recent_window),
                    "mean_keep": float(run.flags.float().mean().item()) if run.has_prefill else None,
                    "l2": "flushed between steps (256 MiB write)", "replicas": world,
                    "decode_launch": "one CUDA graph per pass" if run.use_graph else "individual launches"},
@@ -656,6 +662,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="prefill7b", choices=list(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--recent-window", type=int, default=0,
+                    help="recent tokens always visible, the current one included (0 or 1: the method as published)")
     ap.add_argument("--no-graph", action="store_true", help="launch the decode steps one by one instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -92,6 +92,14 @@ typedef struct {
                             flags, flag_new, scores, prefix, idx and the cache slabs then
                             have kv_heads where the comments below say h; Q, q, O, o keep
                             h; Wo_g and W_lin have kv_heads columns.                  */
+  int32_t recent_window; /* 0 or 1: the method as published, a token always sees itself and
+                            otherwise only retained tokens (the diagonal of Eq. 5).
+                            w in 2..17: the w most recent tokens, the current one included,
+                            are visible whatever their flags (Appendix, Table 6, settings
+                            (6-1), (6-2): w = 5, 10); an evicted token leaves the attention
+                            of later tokens once it is w or more positions behind.  What is
+                            cached for good is unchanged.  The cache then needs its
+                            recent_* arrays; not combined with seq_lens (AG_ERR_UNSUPPORTED). */
 } ag_layer_desc;
 
 /* Ragged per-(sequence, head) cache of retained keys and values.  The struct
@@ -108,6 +116,15 @@ typedef struct {
   int32_t *len;      /* [B*h] rows in use (written by compact, append)      */
   int32_t max_cap;   /* host-known upper bound of every cap[s] (sizes the
                         decode grid; must be >= max_s cap[s])               */
+  /* Only with desc->recent_window = w > 1 (NULL otherwise): per slab a ring of the last
+   * R = w - 1 tokens, token number p in slot p % R.  ag_compact_kv fills it from the end of
+   * the prompt, ag_cache_append / ag_decode_step put every new token in (kept or not), and
+   * decode attention reads the slots marked live.                                          */
+  void *recent_k;       /* [B*h, R, head_dim] keys of the ring                              */
+  void *recent_v;       /* [B*h, R, head_dim] values                                        */
+  uint8_t *recent_live; /* [B*h, R] 1: the slot holds an EVICTED token that later tokens
+                           still see (a retained one is a row of the slab already)          */
+  int32_t *pos;         /* [B*h] tokens the slab has seen (prompt + appended or not)        */
 } ag_cache;
 
 /* Bits of the device status word written by ag_compact_kv / ag_cache_append. */
@@ -273,6 +290,8 @@ int ag_decode_step(const ag_layer_desc *desc, const void *q, const void *k_new,
  *  - The first call on each device looks up the array's device address (the
  *    device must be current, as for every call).  Make that first call
  *    outside any stream capture.
+ *  - A layer with desc->recent_window > 1 is refused with AG_ERR_UNSUPPORTED:
+ *    this entry does not read the ring of recent tokens.
  *  - All calls share the one array.  Its previous contents never matter (each
  *    call writes every partial result before reading it), but two calls that
  *    may overlap on the GPU — different streams, or different host threads

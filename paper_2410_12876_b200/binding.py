@@ -37,7 +37,7 @@ class ag_layer_desc(ctypes.Structure):
         ("heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
         ("gate_heads", ctypes.c_int32), ("gate_head_dim", ctypes.c_int32),
         ("tau", ctypes.c_float), ("gate_causal", ctypes.c_int32), ("dtype", ctypes.c_int32),
-        ("seq_lens", ctypes.c_void_p), ("kv_heads", ctypes.c_int32),
+        ("seq_lens", ctypes.c_void_p), ("kv_heads", ctypes.c_int32), ("recent_window", ctypes.c_int32),
     ]
 
 
@@ -46,6 +46,8 @@ class ag_cache(ctypes.Structure):
         ("k_rows", ctypes.c_void_p), ("v_rows", ctypes.c_void_p), ("pool_rows", ctypes.c_int64),
         ("row_off", ctypes.c_void_p), ("cap", ctypes.c_void_p), ("len", ctypes.c_void_p),
         ("max_cap", ctypes.c_int32),
+        ("recent_k", ctypes.c_void_p), ("recent_v", ctypes.c_void_p), ("recent_live", ctypes.c_void_p),
+        ("pos", ctypes.c_void_p),
     ]
 
 
@@ -99,7 +101,8 @@ def make_desc(shape, seq_lens=None):
     return ag_layer_desc(shape.batch, shape.seq, shape.hidden, shape.heads, shape.head_dim,
                          shape.gate_heads, shape.gate_head_dim, float(shape.tau),
                          int(shape.gate_causal), AG_F32 if shape.dtype == "f32" else AG_BF16,
-                         None if seq_lens is None else seq_lens.data_ptr(), int(getattr(shape, "kv_heads", 0)))
+                         None if seq_lens is None else seq_lens.data_ptr(), int(getattr(shape, "kv_heads", 0)),
+                         int(getattr(shape, "recent_window", 0)))
 
 
 def _ptr(t):
@@ -128,11 +131,14 @@ class RaggedCache:
     """Device buffers of a ragged retained-KV cache plus the host struct the
     C calls take.  Holds references so the tensors outlive the struct."""
 
-    def __init__(self, k_rows, v_rows, row_off, cap, length, max_cap):
+    def __init__(self, k_rows, v_rows, row_off, cap, length, max_cap, recent=None):
         self.k_rows, self.v_rows, self.row_off, self.cap, self.len = k_rows, v_rows, row_off, cap, length
         self.max_cap = int(max_cap)
+        # ring of the last recent_window - 1 tokens of every slab: (keys, values, live marks, tokens seen)
+        self.recent_k, self.recent_v, self.recent_live, self.pos = recent if recent is not None else (None,) * 4
         self.struct = ag_cache(_ptr(k_rows), _ptr(v_rows), int(k_rows.shape[0]), _ptr(row_off),
-                               _ptr(cap), _ptr(length), self.max_cap)
+                               _ptr(cap), _ptr(length), self.max_cap, _ptr(self.recent_k), _ptr(self.recent_v),
+                               _ptr(self.recent_live), _ptr(self.pos))
 
     @classmethod
     def allocate(cls, shape, cap, device="cuda"):
@@ -144,11 +150,17 @@ class RaggedCache:
         pool = int(cap.sum())
         k = torch.zeros(max(pool, 1), shape.head_dim, dtype=shape.torch_dtype, device=device)
         v = torch.zeros_like(k)
+        recent = None
+        R = int(getattr(shape, "recent_window", 0)) - 1
+        if R > 0:
+            rk = torch.zeros(cap.size, R, shape.head_dim, dtype=shape.torch_dtype, device=device)
+            recent = (rk, torch.zeros_like(rk), torch.zeros(cap.size, R, dtype=torch.uint8, device=device),
+                      torch.zeros(cap.size, dtype=torch.int32, device=device))
         return cls(k[:pool], v[:pool],
                    torch.from_numpy(off).to(device),
                    torch.from_numpy(cap.astype("int32")).to(device),
                    torch.zeros(cap.size, dtype=torch.int32, device=device),
-                   int(cap.max()) if cap.size else 0)
+                   int(cap.max()) if cap.size else 0, recent)
 
 
 def ag_status_string(status):

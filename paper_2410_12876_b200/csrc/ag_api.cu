@@ -18,6 +18,9 @@ static int check_desc(const ag_layer_desc *d) {
   if (!dim_ok(d->head_dim)) return AG_ERR_UNSUPPORTED;
   if ((int64_t)d->batch * d->heads > (int64_t)1 << 24) return AG_ERR_UNSUPPORTED;
   if (d->kv_heads < 0 || (d->kv_heads > 0 && d->heads % d->kv_heads != 0)) return AG_ERR_INVALID_ARG;
+  if (d->recent_window < 0) return AG_ERR_INVALID_ARG;
+  if (d->recent_window > kMaxRecent + 1) return AG_ERR_UNSUPPORTED;
+  if (recent_rows(*d) > 0 && d->seq_lens) return AG_ERR_UNSUPPORTED;
   return AG_OK;
 }
 
@@ -34,8 +37,13 @@ static int check_gate_desc(const ag_layer_desc *d) {
   return AG_OK;
 }
 
-static int check_cache(const ag_cache *c) {
+// need_recent: the call reads or writes the ring of recent tokens (compaction, decode, append).
+static int check_cache(const ag_cache *c, const ag_layer_desc *d = nullptr, bool need_recent = false) {
   if (!c) return AG_ERR_INVALID_ARG;
+  if (need_recent && d && recent_rows(*d) > 0) {
+    if (!c->recent_k || !c->recent_v || !c->recent_live || !c->pos) return AG_ERR_INVALID_ARG;
+    if (misaligned16(c->recent_k) || misaligned16(c->recent_v)) return AG_ERR_INVALID_ARG;
+  }
   if (!c->row_off || !c->cap || !c->len) return AG_ERR_INVALID_ARG;
   if (c->pool_rows < 0 || c->max_cap < 0) return AG_ERR_INVALID_ARG;
   if (c->pool_rows > 0 && (!c->k_rows || !c->v_rows)) return AG_ERR_INVALID_ARG;
@@ -106,7 +114,7 @@ int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
   if (st) return st;
   if (!flags || !prefix) return AG_ERR_INVALID_ARG;
   if ((K == nullptr) != (V == nullptr)) return AG_ERR_INVALID_ARG;
-  st = check_cache(cache);
+  st = check_cache(cache, desc, K != nullptr);
   if (st) return st;
   if (misaligned16(K) || misaligned16(V) || misaligned16(flags) || misaligned16(prefix) ||
       misaligned16(idx))
@@ -145,7 +153,7 @@ int ag_decode_attn(const ag_layer_desc *desc, const void *q, const void *k_new,
   int st = check_desc(desc);
   if (st) return st;
   if (!q || !k_new || !v_new || !o) return AG_ERR_INVALID_ARG;
-  st = check_cache(cache);
+  st = check_cache(cache, desc, true);
   if (st) return st;
   if (misaligned16(q) || misaligned16(k_new) || misaligned16(v_new) || misaligned16(o))
     return AG_ERR_INVALID_ARG;
@@ -163,7 +171,7 @@ int ag_decode_step(const ag_layer_desc *desc, const void *q, const void *k_new, 
   int st = check_desc(desc);
   if (st) return st;
   if (!q || !k_new || !v_new || !flag_new || !o) return AG_ERR_INVALID_ARG;
-  st = check_cache(cache);
+  st = check_cache(cache, desc, true);
   if (st) return st;
   if (misaligned16(q) || misaligned16(k_new) || misaligned16(v_new) || misaligned16(o))
     return AG_ERR_INVALID_ARG;
@@ -181,7 +189,7 @@ int ag_cache_append(const ag_layer_desc *desc, const void *k_new, const void *v_
   int st = check_desc(desc);
   if (st) return st;
   if (!k_new || !v_new || !flag_new) return AG_ERR_INVALID_ARG;
-  st = check_cache(cache);
+  st = check_cache(cache, desc, true);
   if (st) return st;
   if (misaligned16(k_new) || misaligned16(v_new)) return AG_ERR_INVALID_ARG;
   return launch_append(*desc, k_new, v_new, flag_new, *cache, dev_status,

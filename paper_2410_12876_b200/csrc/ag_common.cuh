@@ -33,6 +33,22 @@ inline cudaLaunchAttribute pdl_attribute() {
   at.val.programmaticStreamSerializationAllowed = 1;
   return at;
 }
+// Recent-token window: the ring of a slab holds the last recent_window - 1 tokens (0 = no ring).
+constexpr int kMaxRecent = 16;
+inline int recent_rows(const ag_layer_desc &d) { return d.recent_window > 1 ? d.recent_window - 1 : 0; }
+// The ring of a cache as the kernels take it (R = 0: the layer has no window, nothing is touched).
+struct RecentRing {
+  void *k, *v;        // [slabs, R, D]
+  uint8_t *live;      // [slabs, R]
+  int32_t *pos;       // [slabs]
+  int R;
+};
+inline RecentRing ring_of(const ag_layer_desc &d, const ag_cache &c) {
+  RecentRing r = {};
+  r.R = recent_rows(d);
+  if (r.R > 0) { r.k = c.recent_k; r.v = c.recent_v; r.live = c.recent_live; r.pos = c.pos; }
+  return r;
+}
 inline bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
 // Per-step launchers (defined in the kernel files, called from ag_api.cu).
@@ -72,8 +88,10 @@ int launch_prefill(const ag_layer_desc &d, const void *Q, const void *K, const v
 
 // Tensor-core (tcgen05) prefill attention for bf16, head_dim 128.
 bool prefill_tc_supported(const ag_layer_desc &d, const ag_cache &c);
+// lse (NULL or [slabs, n]): log2 of each row's softmax denominator, in the units of the scaled
+// scores times log2(e); -inf where a whole query tile had no retained key (O = v_j there).
 int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, const void *V, const ag_cache &c,
-                      const int32_t *prefix, float scale, void *O, cudaStream_t st);
+                      const int32_t *prefix, float scale, void *O, float *lse, cudaStream_t st);
 int prefill_tc_wait_timeouts();
 
 size_t decode_workspace_bytes(const ag_layer_desc &d);
@@ -117,6 +135,27 @@ template <> struct Elem<__nv_bfloat16> {
 // in the stream is still running.  It must call pdl_wait() before it touches global memory (the
 // predecessor has then completed, its writes visible); pdl_launch_dependents() lets the successor's
 // set-up begin.  Both are no-ops in a launch without the attribute.
+// Puts the new token of slab `slab` into its ring (recent-token window): slot = tokens seen % R,
+// marked live iff the token is NOT kept (a kept one is a row of the slab).  Called by kVecs
+// consecutive lanes of one warp (vec = 0 .. kVecs - 1, one 16-byte piece of the row each), after
+// every read of the ring by this launch.
+template <int kVecs>
+__device__ __forceinline__ void ring_put(const RecentRing &rg, int slab, int vec, const uint8_t *k_row,
+                                         const uint8_t *v_row, bool kept) {
+  const unsigned lane = threadIdx.x & 31u;
+  const unsigned mask = kVecs == 32 ? 0xffffffffu : (((1u << kVecs) - 1u) << (lane / kVecs * kVecs));
+  const int p = rg.pos[slab];
+  __syncwarp(mask);                                 // every lane has read pos before it moves
+  const int slot = p % rg.R;
+  const size_t dst = ((size_t)slab * rg.R + slot) * (kVecs * 16) + vec * 16;
+  *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(rg.k) + dst) = *reinterpret_cast<const uint4 *>(k_row + vec * 16);
+  *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(rg.v) + dst) = *reinterpret_cast<const uint4 *>(v_row + vec * 16);
+  if (vec == 0) {
+    rg.live[(size_t)slab * rg.R + slot] = kept ? 0 : 1;
+    rg.pos[slab] = p + 1;
+  }
+}
+
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

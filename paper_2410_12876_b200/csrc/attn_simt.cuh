@@ -32,6 +32,7 @@ struct SimtAttnArgs {
   const void *k_rows, *v_rows;         // compacted cache pools
   const int64_t *row_off;
   const int32_t *prefix;               // [problems, n + 1]
+  float *lse;                          // NULL, or [problems, n]: m + log2(l) of every row
   // kGateFull only: [batch] keys each sequence has (the rest is padding), or NULL = n
   const int32_t *seq_lens;
 };
@@ -224,6 +225,7 @@ simt_attn_kernel(const SimtAttnArgs a) {
     if (!valid[r]) continue;
     const int j = j0 + ty * 4 + r;
     const float inv = 1.f / l[r];
+    if (MODE == kPrefill && a.lse != nullptr && tx == 0) a.lse[(size_t)prob * a.n + j] = m[r] + log2f(l[r]);
 #pragma unroll
     for (int c = 0; c < kOC; ++c)
 #pragma unroll

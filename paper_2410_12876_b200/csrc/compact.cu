@@ -123,7 +123,7 @@ append_rows_kernel(const uint8_t *__restrict__ k_new, const uint8_t *__restrict_
                    const uint8_t *__restrict__ flag_new, int n_slabs,
                    const int64_t *__restrict__ row_off, const int32_t *__restrict__ cap,
                    int32_t *__restrict__ len, uint8_t *__restrict__ k_rows,
-                   uint8_t *__restrict__ v_rows, int32_t *__restrict__ dev_status) {
+                   uint8_t *__restrict__ v_rows, int32_t *__restrict__ dev_status, const RecentRing ring) {
   constexpr int kVecs = kRowBytes / 16;
   constexpr int kGroups = 256 / kVecs;
   const int slab = blockIdx.x * kGroups + threadIdx.x / kVecs;
@@ -143,6 +143,31 @@ append_rows_kernel(const uint8_t *__restrict__ k_new, const uint8_t *__restrict_
     if (v == 0) len[slab] = L + 1;
   }
   if (full && v == 0 && dev_status) atomicOr(dev_status, AG_DEV_OVERFLOW);
+  // recent-token window: kept or not, the token is one of the slab's recent tokens from now on
+  if (ring.R > 0 && slab < n_slabs)
+    ring_put<kVecs>(ring, slab, v, k_new + (size_t)slab * kRowBytes, v_new + (size_t)slab * kRowBytes, want);
+}
+
+// Recent-token window: after the prompt, the ring of a slab holds its last R tokens (token t in
+// slot t % R), the evicted ones marked live; a prompt shorter than R leaves the other slots dead.
+// One CTA per slab, thread (slot, 16-byte piece).
+template <int kRowBytes>
+__global__ void recent_fill_kernel(const uint8_t *__restrict__ K, const uint8_t *__restrict__ V,
+                                   const uint8_t *__restrict__ flags, int n, const RecentRing ring) {
+  constexpr int kVecs = kRowBytes / 16;
+  const int slab = blockIdx.x, slot = threadIdx.x / kVecs, v = threadIdx.x % kVecs;
+  if (slot >= ring.R) return;
+  // the last token whose number is slot modulo R, if the prompt has one
+  const bool have = slot <= n - 1;
+  const int t = have ? slot + (n - 1 - slot) / ring.R * ring.R : 0;
+  if (have) {
+    const size_t src = ((size_t)slab * n + t) * kRowBytes + v * 16;
+    const size_t dst = ((size_t)slab * ring.R + slot) * kRowBytes + v * 16;
+    *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(ring.k) + dst) = *reinterpret_cast<const uint4 *>(K + src);
+    *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(ring.v) + dst) = *reinterpret_cast<const uint4 *>(V + src);
+  }
+  if (v == 0) ring.live[(size_t)slab * ring.R + slot] = (have && flags[(size_t)slab * n + t] == 0) ? 1 : 0;
+  if (threadIdx.x == 0) ring.pos[slab] = n;
 }
 
 static int row_bytes(const ag_layer_desc &d) {
@@ -181,6 +206,16 @@ int launch_compact(const ag_layer_desc &d, const void *K, const void *V, const u
       return AG_ERR_UNSUPPORTED;
   }
   AG_LAUNCH_CHECK();
+  const RecentRing ring = ring_of(d, c);
+  if (K && ring.R > 0) {
+    const int threads = ring.R * (row_bytes(d) / 16);
+    switch (row_bytes(d)) {
+      case 128: recent_fill_kernel<128><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
+      case 256: recent_fill_kernel<256><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
+      default: recent_fill_kernel<512><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
+    }
+    AG_LAUNCH_CHECK();
+  }
   return AG_OK;
 }
 
@@ -202,15 +237,16 @@ int launch_append(const ag_layer_desc &d, const void *k_new, const void *v_new,
   cudaLaunchAttribute attr = pdl_attribute();
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
+  const RecentRing ring = ring_of(d, c);
   switch (rb) {
     case 128:
-      AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, append_rows_kernel<128>, kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status));
+      AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, append_rows_kernel<128>, kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status, ring));
       break;
     case 256:
-      AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, append_rows_kernel<256>, kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status));
+      AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, append_rows_kernel<256>, kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status, ring));
       break;
     case 512:
-      AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, append_rows_kernel<512>, kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status));
+      AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, append_rows_kernel<512>, kn, vn, flag_new, slabs, c.row_off, c.cap, c.len, kr, vr, dev_status, ring));
       break;
     default:
       return AG_ERR_UNSUPPORTED;

@@ -64,6 +64,24 @@ __device__ __forceinline__ void append_new_row(const AppendArgs &ap, int slab, i
   if (threadIdx.x == 0) ap.len[slab] = L + 1;
 }
 
+// Recent-token window: scores of the query against the ring of its key/value slab, by every warp
+// of the CTA: sm_s[r] = scale_log2 * q . k_r for a live slot (an evicted token the query still
+// sees), -inf otherwise.  The caller synchronises the CTA before reading sm_s.
+template <typename T, int D>
+__device__ __forceinline__ void ring_scores(const RecentRing &rg, int kv, const T *__restrict__ q_row,
+                                            float scale_log2, float *sm_s) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+  for (int r = warp; r < rg.R; r += n_warps) {
+    const T *kr = static_cast<const T *>(rg.k) + ((size_t)kv * rg.R + r) * D;
+    float a = 0.f;
+#pragma unroll
+    for (int d = lane; d < D; d += 32) a = fmaf(Elem<T>::load(q_row + d), Elem<T>::load(kr + d), a);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+    if (lane == 0) sm_s[r] = rg.live[(size_t)kv * rg.R + r] != 0 ? a * scale_log2 : -INFINITY;
+  }
+}
+
 // Rows [r_begin, r_end) of one slab, streamed by a whole CTA of kThreads threads: thread (g, v) =
 // (row group, 16-byte slice of the row) ends with its group's running maximum m, sum l and slice
 // of o (log2 domain).
@@ -294,7 +312,8 @@ decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
                       const T *__restrict__ v_new, const int32_t *__restrict__ len,
                       float scale_log2, int chunk_rows, const float *__restrict__ part_o,
                       const float *__restrict__ part_ml, T *__restrict__ o,
-                      const int64_t *__restrict__ row_off, const AppendArgs ap, const HeadMap hm) {
+                      const int64_t *__restrict__ row_off, const AppendArgs ap, const HeadMap hm,
+                      const RecentRing rg) {
   const int slab = blockIdx.x, d = threadIdx.x;
   const int kv = hm.kv_slab(slab);
   const int L = len[kv];
@@ -303,10 +322,12 @@ decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
   append_new_row<T, D>(ap, kv, L, row_off[kv], k_new, v_new);
   const int n_chunks = (L + chunk_rows - 1) / chunk_rows;
   __shared__ float red[D / 32];
+  __shared__ float ring_s[kMaxRecent];
   float a = Elem<T>::load(q + (size_t)slab * D + d) * Elem<T>::load(k_new + (size_t)kv * D + d);
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
   if ((d & 31) == 0) red[d >> 5] = a;
+  ring_scores<T, D>(rg, kv, q + (size_t)slab * D, scale_log2, ring_s);
   __syncthreads();
   float s_self = 0.f;
 #pragma unroll
@@ -315,6 +336,7 @@ decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
   const float *pml = part_ml + (size_t)slab * kMaxSplits * 2;
   float m = s_self;
   for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, pml[2 * c]);
+  for (int r = 0; r < rg.R; ++r) m = fmaxf(m, ring_s[r]);
   const float w_self = exp2f(s_self - m);
   float acc = w_self * Elem<T>::load(v_new + (size_t)kv * D + d);
   float l = w_self;
@@ -324,7 +346,22 @@ decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
     acc = fmaf(w, po[(size_t)c * D], acc);
     l = fmaf(w, pml[2 * c + 1], l);
   }
+  // the evicted tokens of the recent-token window
+  for (int r = 0; r < rg.R; ++r) {
+    if (ring_s[r] == -INFINITY) continue;
+    const float w = exp2f(ring_s[r] - m);
+    acc = fmaf(w, Elem<T>::load(static_cast<const T *>(rg.v) + ((size_t)kv * rg.R + r) * D + d), acc);
+    l += w;
+  }
   Elem<T>::store(o + (size_t)slab * D + d, acc / l);
+  if (rg.R > 0 && ap.flag_new != nullptr) {
+    // the step carries the append: the new token joins the ring once every thread has read it
+    constexpr int kVecs = D * (int)sizeof(T) / 16;
+    __syncthreads();
+    if (d < kVecs)
+      ring_put<kVecs>(rg, kv, d, reinterpret_cast<const uint8_t *>(k_new + (size_t)kv * D),
+                      reinterpret_cast<const uint8_t *>(v_new + (size_t)kv * D), ap.flag_new[kv] != 0);
+  }
 }
 
 // One cluster of kClusterSize CTAs per slab.  CTA `rank` reduces rows [rank, rank + 1) * per of
@@ -338,7 +375,8 @@ __global__ void __launch_bounds__(kThreads)
 decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, const T *__restrict__ v_new,
                       const T *__restrict__ k_rows, const T *__restrict__ v_rows,
                       const int64_t *__restrict__ row_off, const int32_t *__restrict__ len,
-                      float scale_log2, T *__restrict__ out, const AppendArgs ap, const HeadMap hm) {
+                      float scale_log2, T *__restrict__ out, const AppendArgs ap, const HeadMap hm,
+                      const RecentRing rg) {
   namespace cg = cooperative_groups;
   constexpr int kEpl = Elem<T>::kPerVec;
   constexpr int kLanes = D / kEpl;
@@ -358,6 +396,7 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
   __shared__ float cta_o[D];          // this CTA's triple, read by the first CTA of the cluster
   __shared__ float cta_ml[2];
   __shared__ float red[D / 32];
+  __shared__ float ring_s[kMaxRecent];
 
   // self score q . k_new: only the first CTA needs it; its loads are in flight with the stream's
   float prod = 0.f;
@@ -375,6 +414,7 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
     for (int off = 16; off > 0; off >>= 1) prod += __shfl_xor_sync(0xffffffffu, prod, off);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = prod;
   }
+  if (rank == 0) ring_scores<T, D>(rg, kv, q + (size_t)slab * D, scale_log2, ring_s);
   __syncthreads();
   float mc = -INFINITY;
 #pragma unroll
@@ -414,6 +454,7 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
     float mm = s_self;
 #pragma unroll
     for (int r = 0; r < kClusterSize; ++r) mm = fmaxf(mm, mr[r]);
+    for (int r = 0; r < rg.R; ++r) mm = fmaxf(mm, ring_s[r]);
     const float w_self = exp2f(s_self - mm);
     float acc = w_self * Elem<T>::load(v_new + (size_t)kv * D + d);
     float lsum = w_self;
@@ -423,7 +464,22 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
       acc = fmaf(w, orr[r], acc);
       lsum = fmaf(w, lr[r], lsum);
     }
+    // the evicted tokens of the recent-token window
+    for (int r = 0; r < rg.R; ++r) {
+      if (ring_s[r] == -INFINITY) continue;
+      const float w = exp2f(ring_s[r] - mm);
+      acc = fmaf(w, Elem<T>::load(static_cast<const T *>(rg.v) + ((size_t)kv * rg.R + r) * D + d), acc);
+      lsum += w;
+    }
     Elem<T>::store(out + (size_t)slab * D + d, acc / lsum);
+  }
+  if (rank == 0 && rg.R > 0 && ap.flag_new != nullptr) {
+    // the step carries the append: the new token joins the ring once every thread has read it
+    constexpr int kVecs = D * (int)sizeof(T) / 16;
+    __syncthreads();
+    if ((int)threadIdx.x < kVecs)
+      ring_put<kVecs>(rg, kv, threadIdx.x, reinterpret_cast<const uint8_t *>(k_new + (size_t)kv * D),
+                      reinterpret_cast<const uint8_t *>(v_new + (size_t)kv * D), ap.flag_new[kv] != 0);
   }
   cluster.sync();
 }
@@ -431,7 +487,7 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
 template <typename T, int D, int kThreads>
 static int launch_decode_cluster(int slabs, const void *q, const void *k_new, const void *v_new,
                                  const ag_cache &c, float scale_log2, void *o, const AppendArgs &ap,
-                                 const HeadMap &hm, cudaStream_t st) {
+                                 const HeadMap &hm, const RecentRing &rg, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(kClusterSize, slabs);
   cfg.blockDim = dim3(kThreads);
@@ -445,7 +501,7 @@ static int launch_decode_cluster(int slabs, const void *q, const void *k_new, co
   AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_cluster_kernel<T, D, kThreads>, static_cast<const T *>(q),
                                  static_cast<const T *>(k_new), static_cast<const T *>(v_new),
                                  static_cast<const T *>(c.k_rows), static_cast<const T *>(c.v_rows),
-                                 c.row_off, c.len, scale_log2, static_cast<T *>(o), ap, hm));
+                                 c.row_off, c.len, scale_log2, static_cast<T *>(o), ap, hm, rg));
   return AG_OK;
 }
 
@@ -459,9 +515,10 @@ static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, 
                       const ag_cache &c, float scale, void *o, void *ws, const AppendArgs &ap, cudaStream_t st) {
   const int slabs = d.batch * d.heads;              // one per (sequence, query head)
   const HeadMap hm{d.heads, kv_heads_of(d)};
+  const RecentRing rg = ring_of(d, c);
   const float scale_log2 = scale * 1.4426950408889634f;
   if (slabs <= kClusterMaxSlabs)
-    return launch_decode_cluster<T, D, kClusterThreads>(slabs, q, k_new, v_new, c, scale_log2, o, ap, hm, st);
+    return launch_decode_cluster<T, D, kClusterThreads>(slabs, q, k_new, v_new, c, scale_log2, o, ap, hm, rg, st);
   int chunk_rows = (c.max_cap + kMaxSplits - 1) / kMaxSplits;
   chunk_rows = (chunk_rows + 127) / 128 * 128;   // whole iterations of the partial kernel (bf16, D = 128)
   const int n_chunks = c.max_cap > 0 ? (c.max_cap + chunk_rows - 1) / chunk_rows : 0;
@@ -489,7 +546,7 @@ static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, 
   }
   decode_combine_kernel<T, D><<<slabs, D, 0, st>>>(
       static_cast<const T *>(q), static_cast<const T *>(k_new), static_cast<const T *>(v_new),
-      c.len, scale_log2, chunk_rows, part_o, part_ml, static_cast<T *>(o), c.row_off, ap, hm);
+      c.len, scale_log2, chunk_rows, part_o, part_ml, static_cast<T *>(o), c.row_off, ap, hm, rg);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
@@ -563,6 +620,8 @@ extern "C" int ag_decode_attn_noalloc(const ag_layer_desc *desc, const void *q, 
   if (desc->batch <= 0 || desc->heads <= 0 || desc->seq <= 0) return AG_ERR_INVALID_ARG;
   if (desc->dtype != AG_F32 && desc->dtype != AG_BF16) return AG_ERR_INVALID_ARG;
   if (desc->head_dim != 64 && desc->head_dim != 128) return AG_ERR_UNSUPPORTED;
+  if (desc->recent_window < 0) return AG_ERR_INVALID_ARG;
+  if (desc->recent_window > 1) return AG_ERR_UNSUPPORTED;     // this entry does not read the ring of recent tokens
   if (!cache->row_off || !cache->cap || !cache->len || cache->pool_rows < 0 || cache->max_cap < 0)
     return AG_ERR_INVALID_ARG;
   if (cache->pool_rows > 0 && (!cache->k_rows || !cache->v_rows)) return AG_ERR_INVALID_ARG;

@@ -48,6 +48,7 @@ struct PrefillTcArgs {
   int n, n_qtiles, slabs;           // slabs: (sequence, query head) pairs
   int heads, kv_heads;              // query heads share key/value heads in groups of heads / kv_heads
   float scale_log2;
+  float *lse;                       // NULL, or [slabs, n]: m + log2(l) of every row (see launch_prefill_tc)
 };
 
 // Byte offset of 16-byte chunk `chunk` (0..15) of row `row` inside a [128 x 128] bf16 tile stored
@@ -365,6 +366,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (ok) {
       const float w_self = fast_exp2(self2 - m);
       const float inv = 1.f / l;
+      if (a.lse != nullptr && valid) a.lse[(size_t)slab * a.n + j] = n_kv > 0 ? m + log2f(l) : -INFINITY;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         uint32_t r[32];
@@ -410,7 +412,7 @@ bool prefill_tc_supported(const ag_layer_desc &d, const ag_cache &c) {
 }
 
 int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, const void *V, const ag_cache &c,
-                      const int32_t *prefix, float scale, void *O, cudaStream_t st) {
+                      const int32_t *prefix, float scale, void *O, float *lse, cudaStream_t st) {
   const int slabs = d.batch * d.heads;
   CUtensorMap tmQ, tmKd, tmVd, tmO, tmK, tmV;
   int rc;
@@ -430,6 +432,7 @@ int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, cons
   a.n = d.seq; a.n_qtiles = (d.seq + kPfBM - 1) / kPfBM; a.slabs = slabs;
   a.heads = d.heads; a.kv_heads = kv_heads_of(d);
   a.scale_log2 = scale * 1.4426950408889634f;
+  a.lse = lse;
   AG_CUDA_TRY(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes));
   prefill_tc_kernel<<<a.n_qtiles * slabs, kPfThreads, kPfSmemBytes, st>>>(tmQ, tmKd, tmVd, tmO, tmK, tmV, a);
   AG_LAUNCH_CHECK();

@@ -30,6 +30,7 @@ class LayerShape:
     tau: float = 0.5
     gate_causal: int = 1
     kv_heads: int = 0          # key/value heads (grouped-query attention); 0 = one per query head
+    recent_window: int = 0     # recent tokens always visible, the current one included; 0 or 1 = itself only
 
     @property
     def kvh(self):

@@ -30,11 +30,13 @@ def test_every_declared_function_is_exported(lib):
 
 
 def test_struct_layout_matches_header():
-    assert ctypes.sizeof(ag.ag_layer_desc) == 56            # ten 4-byte fields, the seq_lens pointer, kv_heads
+    assert ctypes.sizeof(ag.ag_layer_desc) == 56            # ten 4-byte fields, the seq_lens pointer, kv_heads, recent_window
     assert ag.ag_layer_desc.seq_lens.offset == 40
     assert ag.ag_layer_desc.kv_heads.offset == 48
-    assert ctypes.sizeof(ag.ag_cache) == 56
+    assert ag.ag_layer_desc.recent_window.offset == 52
+    assert ctypes.sizeof(ag.ag_cache) == 88
     assert ag.ag_cache.max_cap.offset == 48
+    assert ag.ag_cache.recent_k.offset == 56 and ag.ag_cache.pos.offset == 80
 
 
 def test_workspace_sizes(lib):
