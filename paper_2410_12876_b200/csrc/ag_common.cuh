@@ -101,6 +101,12 @@ int launch_decode(const ag_layer_desc &d, const void *q, const void *k_new, cons
 int launch_decode_step(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
                        const uint8_t *flag_new, const ag_cache &c, float scale, void *o,
                        int32_t *dev_status, void *ws, cudaStream_t st);
+// Chunk pass of decode for grouped-query attention on the tensor cores (bf16, head_dim 128, groups
+// of 2..16 query heads): writes the (m, l, o) triples of every (query slab, chunk).
+bool decode_gqa_mma_supported(const ag_layer_desc &d);
+int launch_decode_partial_gqa_mma(const ag_layer_desc &d, const void *q, const ag_cache &c, float scale_log2,
+                                  int chunk_rows, int n_chunks, float *part_o, float *part_ml, int max_splits,
+                                  cudaStream_t st);
 int launch_append(const ag_layer_desc &d, const void *k_new, const void *v_new,
                   const uint8_t *flag_new, const ag_cache &c, int32_t *dev_status,
                   cudaStream_t st);

@@ -525,7 +525,11 @@ static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, 
   float *part_o = static_cast<float *>(ws);
   float *part_ml = part_o + (size_t)slabs * kMaxSplits * D;
   const int group = hm.heads / hm.kv_heads;
-  if (n_chunks > 0 && (group == 2 || group == 4)) {
+  if (n_chunks > 0 && decode_gqa_mma_supported(d)) {
+    // grouped-query attention, bf16: the group's heads are the rows of a tensor-core tile
+    int rc = launch_decode_partial_gqa_mma(d, q, c, scale_log2, chunk_rows, n_chunks, part_o, part_ml, kMaxSplits, st);
+    if (rc) return rc;
+  } else if (n_chunks > 0 && (group == 2 || group == 4)) {
     // grouped-query attention: the rows of a key/value slab are read once for its query heads
     dim3 grid(n_chunks, d.batch * hm.kv_heads);
     auto qp = static_cast<const T *>(q);

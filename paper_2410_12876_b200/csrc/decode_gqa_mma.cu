@@ -1,0 +1,259 @@
+// Chunk pass of decode attention for grouped-query attention on the tensor cores.
+//
+// The G query heads that share a key/value head meet the same rows of the slab, so one step of the
+// decoding stage (Sec. 3.1) is, per slab, the small dense contraction S = Q_g K^T (G x L x D) and
+// O = P V (G x D x L), not G matrix-vector products.  On CUDA cores that costs G dot products and G
+// weighted sums per row and the kernel ends up bound by arithmetic, not by HBM.  Here the G heads
+// are the rows of a 16-row MMA operand (the other rows are zero): warp-level m16n8k16 bf16 MMAs,
+// the shape that fits an M of 2..16 (a tcgen05 tile needs M >= 64).  The work is a stream of K/V
+// rows through shared memory and the kernel is bound by HBM.
+//
+// One CTA = one chunk of one key/value slab, as in the CUDA-core chunk pass; it leaves one
+// (m, l, o) triple per query head of the group where decode_combine_kernel expects it.  Rows go
+// global -> shared by 16-byte cp.async in tiles of 64 rows (K and V, three tiles in flight); each of
+// the four warps owns 16 rows of every tile and keeps its own running softmax; the warps' triples
+// are merged through shared memory at the end.
+#include "ag_common.cuh"
+
+namespace ag {
+
+constexpr int kGqD = 128;                 // head_dim (bf16)
+constexpr int kGqTile = 64;               // rows per tile
+constexpr int kGqWarps = 4, kGqThreads = kGqWarps * 32;
+constexpr int kGqStages = 3;
+constexpr int kGqRowBytes = kGqD * 2;
+constexpr int kGqTileBytes = kGqTile * kGqRowBytes;           // 16 KB
+constexpr int kGqSmemBytes = kGqStages * 2 * kGqTileBytes;    // 96 KB: two CTAs per SM
+constexpr int kGqMaxGroup = 16;
+
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void *gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (16 x 8, f32) += A (16 x 16, bf16, row-major fragments) * B (16 x 8, bf16, column-major fragments)
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+// Byte offset of 16-byte piece `piece` (0..15) of row `row` in a tile: pieces are XOR-ed with the
+// row number so that the eight rows one ldmatrix reads fall into different banks.
+__device__ __forceinline__ uint32_t gq_off(int row, int piece) {
+  return (uint32_t)(row * kGqRowBytes + ((piece ^ (row & 7)) << 4));
+}
+
+__global__ void __launch_bounds__(kGqThreads, 2)
+decode_partial_gqa_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_rows,
+                              const __nv_bfloat16 *__restrict__ v_rows, const int64_t *__restrict__ row_off,
+                              const int32_t *__restrict__ len, float scale_log2, int chunk_rows,
+                              float *__restrict__ part_o, float *__restrict__ part_ml, int kv_heads, int G,
+                              int max_splits) {
+  extern __shared__ __align__(128) uint8_t gq_smem[];
+  const int kv = blockIdx.y, chunk = blockIdx.x;
+  const int slab0 = (kv / kv_heads) * kv_heads * G + (kv % kv_heads) * G;     // first query slab of the group
+  const int L = len[kv];
+  const int r_begin = chunk * chunk_rows;
+  if (r_begin >= L) return;                                                    // the whole CTA, before any barrier
+  const int r_end = min(L, r_begin + chunk_rows);
+  const int n_tiles = (r_end - r_begin + kGqTile - 1) / kGqTile;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;                                       // fragment row, column pair
+  const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(gq_smem);
+  const uint8_t *Kg = reinterpret_cast<const uint8_t *>(k_rows) + (size_t)row_off[kv] * kGqRowBytes;
+  const uint8_t *Vg = reinterpret_cast<const uint8_t *>(v_rows) + (size_t)row_off[kv] * kGqRowBytes;
+
+  // tile i -> stage i % kGqStages; rows past r_end are clamped to the last valid row (weight 0 below)
+  auto load_tile = [&](int i) {
+    const uint32_t sk = smem0 + (i % kGqStages) * 2 * kGqTileBytes, sv = sk + kGqTileBytes;
+    const int r0 = r_begin + i * kGqTile;
+#pragma unroll
+    for (int x = 0; x < kGqTile * 16 / kGqThreads; ++x) {
+      const int idx = threadIdx.x + x * kGqThreads, r = idx >> 4, c = idx & 15;
+      const size_t src = (size_t)min(r0 + r, r_end - 1) * kGqRowBytes + c * 16;
+      cp_async16(sk + gq_off(r, c), Kg + src);
+      cp_async16(sv + gq_off(r, c), Vg + src);
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < kGqStages - 1; ++i) {
+    if (i < n_tiles) load_tile(i);
+    cp_async_commit();
+  }
+
+  // A fragments of Q: row g = query head g of the group (rows >= G are zero), 8 steps of 16 dims
+  uint32_t qa[kGqD / 16][4];
+#pragma unroll
+  for (int ks = 0; ks < kGqD / 16; ++ks) {
+    const uint32_t *qrow = reinterpret_cast<const uint32_t *>(q + (size_t)(slab0 + min(g, G - 1)) * kGqD);
+    const uint32_t lo = qrow[ks * 8 + t], hi = qrow[ks * 8 + 4 + t];
+    qa[ks][0] = g < G ? lo : 0u;
+    qa[ks][1] = 0u;                                     // rows 8..15: G <= 8 is all this kernel is asked for
+    qa[ks][2] = g < G ? hi : 0u;
+    qa[ks][3] = 0u;
+  }
+  const bool two_halves = G > 8;
+  if (two_halves) {
+#pragma unroll
+    for (int ks = 0; ks < kGqD / 16; ++ks) {
+      const uint32_t *qrow = reinterpret_cast<const uint32_t *>(q + (size_t)(slab0 + min(g + 8, G - 1)) * kGqD);
+      qa[ks][1] = g + 8 < G ? qrow[ks * 8 + t] : 0u;
+      qa[ks][3] = g + 8 < G ? qrow[ks * 8 + 4 + t] : 0u;
+    }
+  }
+
+  float o[kGqD / 8][4];
+#pragma unroll
+  for (int nt = 0; nt < kGqD / 8; ++nt)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) o[nt][e] = 0.f;
+  float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};       // rows g and g + 8
+
+  for (int i = 0; i < n_tiles; ++i) {
+    if (i + kGqStages - 1 < n_tiles) load_tile(i + kGqStages - 1);
+    cp_async_commit();
+    cp_async_wait<kGqStages - 1>();                             // tile i has landed (this thread's pieces)
+    __syncthreads();                                            // ... and everybody's
+    const uint32_t sk = smem0 + (i % kGqStages) * 2 * kGqTileBytes, sv = sk + kGqTileBytes;
+    const int key0 = r_begin + i * kGqTile + warp * 16;         // this warp's 16 rows of the tile
+
+    if (key0 < r_end) {
+      // S = Q K^T for 16 keys: two 8-key column tiles
+      float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int ks = 0; ks < kGqD / 16; ++ks) {
+        uint32_t b[4];
+        // matrices: (keys 0-7, dims lo), (keys 0-7, dims hi), (keys 8-15, dims lo), (keys 8-15, dims hi)
+        const int mi = lane >> 3, row = warp * 16 + (mi >> 1) * 8 + (lane & 7);
+        ldmatrix_x4(b, sk + gq_off(row, ks * 2 + (mi & 1)));
+        mma_16816(s0, qa[ks], b[0], b[1]);
+        mma_16816(s1, qa[ks], b[2], b[3]);
+      }
+      // online softmax of rows g (and g + 8): this thread holds keys 2t, 2t+1 of each column tile
+      uint32_t pa[4];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        float sv4[4] = {s0[2 * h], s0[2 * h + 1], s1[2 * h], s1[2 * h + 1]};
+        const int kcol[4] = {2 * t, 2 * t + 1, 8 + 2 * t, 9 + 2 * t};
+        float tmax = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          sv4[e] = (key0 + kcol[e] < r_end) ? sv4[e] * scale_log2 : -INFINITY;
+          tmax = fmaxf(tmax, sv4[e]);
+        }
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+        const float m_new = fmaxf(m[h], tmax);                  // finite: key0 < r_end, so column 0 is valid
+        const float alpha = exp2f(m[h] - m_new);                // m = -inf at first: 0
+        float p[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) p[e] = exp2f(sv4[e] - m_new);
+        const bool row_used = h == 0 ? g < G : g + 8 < G;       // unused rows: zero weights, not 2^(0 - m)
+        l[h] = l[h] * alpha + (row_used ? (p[0] + p[1]) + (p[2] + p[3]) : 0.f);
+        m[h] = m_new;
+        pa[h] = row_used ? pack2_bf16(p[0], p[1]) : 0u;
+        pa[2 + h] = row_used ? pack2_bf16(p[2], p[3]) : 0u;
+#pragma unroll
+        for (int nt = 0; nt < kGqD / 8; ++nt) {
+          o[nt][2 * h] *= alpha;
+          o[nt][2 * h + 1] *= alpha;
+        }
+      }
+      // O += P V: 16 keys x 128 dims, two 8-dim column tiles per ldmatrix
+#pragma unroll
+      for (int nt2 = 0; nt2 < kGqD / 16; ++nt2) {
+        uint32_t b[4];
+        // matrices: (keys 0-7, dims lo), (keys 8-15, dims lo), (keys 0-7, dims hi), (keys 8-15, dims hi)
+        const int mi = lane >> 3, row = warp * 16 + (mi & 1) * 8 + (lane & 7);
+        ldmatrix_x4_trans(b, sv + gq_off(row, nt2 * 2 + (mi >> 1)));
+        mma_16816(o[2 * nt2], pa, b[0], b[1]);
+        mma_16816(o[2 * nt2 + 1], pa, b[2], b[3]);
+      }
+    }
+    __syncthreads();                                            // the stage may be refilled
+  }
+  cp_async_wait<0>();
+
+  // merge the four warps' triples through shared memory (the tiles are no longer needed)
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    l[h] += __shfl_xor_sync(0xffffffffu, l[h], 1);
+    l[h] += __shfl_xor_sync(0xffffffffu, l[h], 2);
+  }
+  float *sm_o = reinterpret_cast<float *>(gq_smem);             // [warps][16][D]
+  float *sm_m = sm_o + kGqWarps * kGqMaxGroup * kGqD;           // [warps][16]
+  float *sm_l = sm_m + kGqWarps * kGqMaxGroup;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int row = g + 8 * h;
+    if (row < G) {
+#pragma unroll
+      for (int nt = 0; nt < kGqD / 8; ++nt) {
+        float *dst = sm_o + ((size_t)(warp * kGqMaxGroup + row)) * kGqD + nt * 8 + 2 * t;
+        dst[0] = o[nt][2 * h];
+        dst[1] = o[nt][2 * h + 1];
+      }
+      if (t == 0) {
+        sm_m[warp * kGqMaxGroup + row] = m[h];
+        sm_l[warp * kGqMaxGroup + row] = l[h];
+      }
+    }
+  }
+  __syncthreads();
+  const int d = threadIdx.x;                                    // kGqThreads == kGqD: one output dimension each
+  for (int h = 0; h < G; ++h) {
+    float mc = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kGqWarps; ++w) mc = fmaxf(mc, sm_m[w * kGqMaxGroup + h]);
+    float acc = 0.f, lc = 0.f;
+#pragma unroll
+    for (int w = 0; w < kGqWarps; ++w) {
+      const float mw = sm_m[w * kGqMaxGroup + h];
+      const float wgt = mw == -INFINITY ? 0.f : exp2f(mw - mc);
+      acc = fmaf(wgt, sm_o[((size_t)(w * kGqMaxGroup + h)) * kGqD + d], acc);
+      lc = fmaf(wgt, sm_l[w * kGqMaxGroup + h], lc);
+    }
+    const size_t slot = (size_t)(slab0 + h) * max_splits + chunk;
+    part_o[slot * kGqD + d] = acc;
+    if (d == 0) {
+      part_ml[slot * 2 + 0] = mc;
+      part_ml[slot * 2 + 1] = lc;
+    }
+  }
+}
+
+bool decode_gqa_mma_supported(const ag_layer_desc &d) {
+  const int group = d.heads / kv_heads_of(d);
+  return d.dtype == AG_BF16 && d.head_dim == kGqD && group >= 2 && group <= kGqMaxGroup;
+}
+
+int launch_decode_partial_gqa_mma(const ag_layer_desc &d, const void *q, const ag_cache &c, float scale_log2,
+                                  int chunk_rows, int n_chunks, float *part_o, float *part_ml, int max_splits,
+                                  cudaStream_t st) {
+  const int kvh = kv_heads_of(d);
+  AG_CUDA_TRY(cudaFuncSetAttribute(decode_partial_gqa_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   kGqSmemBytes));
+  dim3 grid(n_chunks, d.batch * kvh);
+  decode_partial_gqa_mma_kernel<<<grid, kGqThreads, kGqSmemBytes, st>>>(
+      static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(c.k_rows),
+      static_cast<const __nv_bfloat16 *>(c.v_rows), c.row_off, c.len, scale_log2, chunk_rows, part_o, part_ml,
+      kvh, d.heads / kvh, max_splits);
+  AG_LAUNCH_CHECK();
+  return AG_OK;
+}
+
+}  // namespace ag

@@ -73,3 +73,29 @@ def test_gqa_rejects_heads_that_do_not_divide():
         ag.ag_workspace_bytes(ag.make_desc(shape), ag.AG_CALL_DECODE) or ag.ag_decode_attn(
             ag.make_desc(shape), Q[:, :, 0].contiguous(), K[:, :, 0].contiguous(), V[:, :, 0].contiguous(),
             ag.RaggedCache.allocate(shape, [4] * 4, DEV), 0.0, torch.empty_like(Q[:, :, 0]), None)
+
+
+@pytest.mark.parametrize("heads,kv_heads", [(16, 8), (24, 8), (16, 4), (16, 2), (16, 1)],
+                         ids=["group2", "group3", "group4", "group8", "group16"])
+@pytest.mark.parametrize("n", [700, 65, 1])
+def test_gqa_decode_chunk_pass_on_tensor_cores(heads, kv_heads, n):
+    """bf16, head_dim 128, more than 64 query slabs: the group's heads are the rows of one MMA tile.
+    Slabs of every length from empty to full, several tiles and a ragged tail, caches that grow."""
+    shape = LayerShape(5, n, 256, heads, 128, 2, 128, "bf16", kv_heads=kv_heads)
+    B, hk = shape.batch, shape.kvh
+    Q, K, V = inputs.qkv_gaussian(shape, 950 + heads + kv_heads, DEV)
+    keep = np.linspace(0.0, 1.0, B * hk).reshape(B, hk, 1)        # slab 0 keeps nothing, the last one everything
+    f = (np.random.default_rng(951).random((B, hk, n)) < keep).astype(np.uint8)
+    f[-1, -1] = 1
+    fl = torch.from_numpy(f).to(DEV)
+    steps = 4
+    cache, prefix, idx, status = T.gpu_compact(shape, K, V, fl, cap=[n + steps] * (B * hk))
+    ocache = orc.compact_kv(T.f64(K), T.f64(V), f)
+    for fused in (False, True):
+        for step in range(steps // 2):
+            q, kn, vn, fn = inputs.decode_inputs(shape, 960 + 10 * fused, step, DEV, keep_new=0.6)
+            o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status, fused=fused)
+            T.check_close(T.f64(o), orc.decode_attention(T.f64(q), T.f64(kn), T.f64(vn), ocache), "bf16", f"decode {step}")
+            orc.cache_append(ocache, T.f64(kn), T.f64(vn), fn.cpu().numpy())
+    assert np.array_equal(cache.len.cpu().numpy(), orc.cache_lengths(ocache).reshape(-1))
+    assert int(status.item()) == 0
