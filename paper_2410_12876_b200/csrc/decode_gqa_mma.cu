@@ -10,20 +10,21 @@
 //
 // One CTA = one chunk of one key/value slab, as in the CUDA-core chunk pass; it leaves one
 // (m, l, o) triple per query head of the group where decode_combine_kernel expects it.  Rows go
-// global -> shared by 16-byte cp.async in tiles of 64 rows (K and V, three tiles in flight); each of
-// the four warps owns 16 rows of every tile and keeps its own running softmax; the warps' triples
-// are merged through shared memory at the end.
+// global -> shared by 16-byte cp.async in tiles of 64 rows (K and V; the next tile is in flight while
+// one is worked on, and three CTAs share an SM, which measured better than deeper rings in fewer
+// CTAs); each of the four warps owns 16 rows of every tile and keeps its own running softmax; the
+// warps' triples are merged through shared memory at the end.
 #include "ag_common.cuh"
 
 namespace ag {
 
 constexpr int kGqD = 128;                 // head_dim (bf16)
-constexpr int kGqTile = 64;               // rows per tile
 constexpr int kGqWarps = 4, kGqThreads = kGqWarps * 32;
-constexpr int kGqStages = 3;
+constexpr int kGqTile = kGqWarps * 16;    // rows per tile: 16 per warp
+constexpr int kGqStages = 2;
 constexpr int kGqRowBytes = kGqD * 2;
 constexpr int kGqTileBytes = kGqTile * kGqRowBytes;           // 16 KB
-constexpr int kGqSmemBytes = kGqStages * 2 * kGqTileBytes;    // 96 KB: two CTAs per SM
+constexpr int kGqSmemBytes = kGqStages * 2 * kGqTileBytes;    // 64 KB: three CTAs per SM
 constexpr int kGqMaxGroup = 16;
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void *gsrc) {
@@ -57,7 +58,7 @@ __device__ __forceinline__ uint32_t gq_off(int row, int piece) {
   return (uint32_t)(row * kGqRowBytes + ((piece ^ (row & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(kGqThreads, 2)
+__global__ void __launch_bounds__(kGqThreads, 3)
 decode_partial_gqa_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_rows,
                               const __nv_bfloat16 *__restrict__ v_rows, const int64_t *__restrict__ row_off,
                               const int32_t *__restrict__ len, float scale_log2, int chunk_rows,
@@ -214,8 +215,8 @@ decode_partial_gqa_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bf
     }
   }
   __syncthreads();
-  const int d = threadIdx.x;                                    // kGqThreads == kGqD: one output dimension each
-  for (int h = 0; h < G; ++h) {
+  for (int x = threadIdx.x; x < G * kGqD; x += kGqThreads) {     // one (head, output dimension) at a time
+    const int h = x / kGqD, d = x % kGqD;
     float mc = -INFINITY;
 #pragma unroll
     for (int w = 0; w < kGqWarps; ++w) mc = fmaxf(mc, sm_m[w * kGqMaxGroup + h]);
