@@ -93,6 +93,10 @@ bool prefill_tc_supported(const ag_layer_desc &d, const ag_cache &c);
 int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, const void *V, const ag_cache &c,
                       const int32_t *prefix, float scale, void *O, float *lse, cudaStream_t st);
 int prefill_tc_wait_timeouts();
+// Band pass of a recent-token window on the tensor cores (bf16, head_dim 128): extends every row of O
+// by the evicted tokens of its window, given the rows' log-sum-exp.
+int launch_prefill_band_mma(const ag_layer_desc &d, const void *Q, const void *K, const void *V,
+                            const uint8_t *flags, const float *lse, float scale, void *O, cudaStream_t st);
 
 size_t decode_workspace_bytes(const ag_layer_desc &d);
 int launch_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
@@ -141,6 +145,9 @@ template <> struct Elem<__nv_bfloat16> {
 // in the stream is still running.  It must call pdl_wait() before it touches global memory (the
 // predecessor has then completed, its writes visible); pdl_launch_dependents() lets the successor's
 // set-up begin.  Both are no-ops in a launch without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Puts the new token of slab `slab` into its ring (recent-token window): slot = tokens seen % R,
 // marked live iff the token is NOT kept (a kept one is a row of the slab).  Called by kVecs
 // consecutive lanes of one warp (vec = 0 .. kVecs - 1, one 16-byte piece of the row each), after
@@ -161,9 +168,6 @@ __device__ __forceinline__ void ring_put(const RecentRing &rg, int slab, int vec
     rg.pos[slab] = p + 1;
   }
 }
-
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ uint4 ldg128(const void *p) {
   return __ldg(reinterpret_cast<const uint4 *>(p));

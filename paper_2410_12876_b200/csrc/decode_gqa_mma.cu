@@ -15,6 +15,7 @@
 // CTAs); each of the four warps owns 16 rows of every tile and keeps its own running softmax; the
 // warps' triples are merged through shared memory at the end.
 #include "ag_common.cuh"
+#include "mma_sync.cuh"
 
 namespace ag {
 
@@ -26,37 +27,6 @@ constexpr int kGqRowBytes = kGqD * 2;
 constexpr int kGqTileBytes = kGqTile * kGqRowBytes;           // 16 KB
 constexpr int kGqSmemBytes = kGqStages * 2 * kGqTileBytes;    // 64 KB: three CTAs per SM
 constexpr int kGqMaxGroup = 16;
-
-__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void *gsrc) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-// D (16 x 8, f32) += A (16 x 16, bf16, row-major fragments) * B (16 x 8, bf16, column-major fragments)
-__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t *>(&v);
-}
-// Byte offset of 16-byte piece `piece` (0..15) of row `row` in a tile: pieces are XOR-ed with the
-// row number so that the eight rows one ldmatrix reads fall into different banks.
-__device__ __forceinline__ uint32_t gq_off(int row, int piece) {
-  return (uint32_t)(row * kGqRowBytes + ((piece ^ (row & 7)) << 4));
-}
 
 __global__ void __launch_bounds__(kGqThreads, 3)
 decode_partial_gqa_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_rows,
@@ -86,8 +56,8 @@ decode_partial_gqa_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bf
     for (int x = 0; x < kGqTile * 16 / kGqThreads; ++x) {
       const int idx = threadIdx.x + x * kGqThreads, r = idx >> 4, c = idx & 15;
       const size_t src = (size_t)min(r0 + r, r_end - 1) * kGqRowBytes + c * 16;
-      cp_async16(sk + gq_off(r, c), Kg + src);
-      cp_async16(sv + gq_off(r, c), Vg + src);
+      cp_async16(sk + tile256_off(r, c), Kg + src);
+      cp_async16(sv + tile256_off(r, c), Vg + src);
     }
   };
 #pragma unroll
@@ -140,7 +110,7 @@ decode_partial_gqa_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bf
         uint32_t b[4];
         // matrices: (keys 0-7, dims lo), (keys 0-7, dims hi), (keys 8-15, dims lo), (keys 8-15, dims hi)
         const int mi = lane >> 3, row = warp * 16 + (mi >> 1) * 8 + (lane & 7);
-        ldmatrix_x4(b, sk + gq_off(row, ks * 2 + (mi & 1)));
+        ldmatrix_x4(b, sk + tile256_off(row, ks * 2 + (mi & 1)));
         mma_16816(s0, qa[ks], b[0], b[1]);
         mma_16816(s1, qa[ks], b[2], b[3]);
       }
@@ -180,7 +150,7 @@ decode_partial_gqa_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bf
         uint32_t b[4];
         // matrices: (keys 0-7, dims lo), (keys 8-15, dims lo), (keys 0-7, dims hi), (keys 8-15, dims hi)
         const int mi = lane >> 3, row = warp * 16 + (mi & 1) * 8 + (lane & 7);
-        ldmatrix_x4_trans(b, sv + gq_off(row, nt2 * 2 + (mi >> 1)));
+        ldmatrix_x4_trans(b, sv + tile256_off(row, nt2 * 2 + (mi >> 1)));
         mma_16816(o[2 * nt2], pa, b[0], b[1]);
         mma_16816(o[2 * nt2 + 1], pa, b[2], b[3]);
       }

@@ -21,7 +21,8 @@ size_t prefill_workspace_bytes(const ag_layer_desc &d) {
 // scores of those tokens against the dense K, then the row's softmax is extended by them,
 //   O_j <- (2^(lse - M) O_j + sum_t 2^(s_t - M) v_t) / (2^(lse - M) + sum_t 2^(s_t - M)),
 // with lse the row's log-sum-exp from the attention kernel and M the larger of lse and max s_t.
-// Rows with no evicted token in their window are left untouched.
+// Rows with no evicted token in their window are left untouched.  CUDA-core form, for fp32 and
+// head_dim 64; bf16 with head_dim 128 takes prefill_band_mma_kernel.
 constexpr int kBandThreads = 256;
 template <typename T, int D>
 __global__ void __launch_bounds__(kBandThreads)
@@ -153,14 +154,16 @@ int launch_prefill(const ag_layer_desc &d, const void *Q, const void *K, const v
   if (prefill_tc_supported(d, c)) {
     int rc = launch_prefill_tc(d, Q, K, V, c, prefix, scale, O, lse, st);
     if (rc || !lse) return rc;
-    return run_prefill_band<__nv_bfloat16, 128>(d, Q, K, V, flags, lse, scale, O, st);
+    return launch_prefill_band_mma(d, Q, K, V, flags, lse, scale, O, st);
   }
   if (d.dtype == AG_F32) {
     if (d.head_dim == 64) return run_prefill<float, 64>(d, Q, K, V, flags, c, prefix, scale, O, lse, st);
     return run_prefill<float, 128>(d, Q, K, V, flags, c, prefix, scale, O, lse, st);
   }
   if (d.head_dim == 64) return run_prefill<__nv_bfloat16, 64>(d, Q, K, V, flags, c, prefix, scale, O, lse, st);
-  return run_prefill<__nv_bfloat16, 128>(d, Q, K, V, flags, c, prefix, scale, O, lse, st);
+  int rc = run_prefill_simt<__nv_bfloat16, 128>(d, Q, K, V, c, prefix, scale, O, lse, st);
+  if (rc || !lse) return rc;
+  return launch_prefill_band_mma(d, Q, K, V, flags, lse, scale, O, st);
 }
 
 }  // namespace ag
