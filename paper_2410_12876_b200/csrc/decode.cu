@@ -44,24 +44,27 @@ struct AppendArgs {
   void *k_rows, *v_rows;
   int32_t *dev_status;
 };
-// Called by the threads [0, row vectors) of ONE CTA per slab, after every read of len[slab] and
-// of the slab's rows by this launch has completed.  L = the length those reads saw.
+// Called by the threads [first, first + row vectors) of ONE CTA per slab (every thread may call, the
+// others return), after every read of len[slab] and of the slab's rows by this launch has
+// completed.  L = the length those reads saw.
 template <typename T, int D>
 __device__ __forceinline__ void append_new_row(const AppendArgs &ap, int slab, int L, int64_t row0,
-                                               const T *__restrict__ k_new, const T *__restrict__ v_new) {
+                                               const T *__restrict__ k_new, const T *__restrict__ v_new,
+                                               int first = 0) {
   constexpr int kVecs = D * (int)sizeof(T) / 16;
-  if (ap.flag_new == nullptr || ap.flag_new[slab] == 0 || (int)threadIdx.x >= kVecs) return;
+  const int vec = (int)threadIdx.x - first;
+  if (ap.flag_new == nullptr || vec < 0 || vec >= kVecs || ap.flag_new[slab] == 0) return;
   if (L >= ap.cap[slab]) {
-    if (threadIdx.x == 0 && ap.dev_status) atomicOr(ap.dev_status, AG_DEV_OVERFLOW);
+    if (vec == 0 && ap.dev_status) atomicOr(ap.dev_status, AG_DEV_OVERFLOW);
     return;
   }
-  const size_t dst = ((size_t)row0 + L) * D * sizeof(T) + threadIdx.x * 16;
-  const size_t src = (size_t)slab * D * sizeof(T) + threadIdx.x * 16;
+  const size_t dst = ((size_t)row0 + L) * D * sizeof(T) + vec * 16;
+  const size_t src = (size_t)slab * D * sizeof(T) + vec * 16;
   *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(ap.k_rows) + dst) =
       *reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(k_new) + src);
   *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(ap.v_rows) + dst) =
       *reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(v_new) + src);
-  if (threadIdx.x == 0) ap.len[slab] = L + 1;
+  if (vec == 0) ap.len[slab] = L + 1;
 }
 
 // Recent-token window: scores of the query against the ring of its key/value slab, by every warp
@@ -399,9 +402,12 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
   __shared__ float ring_s[kMaxRecent];
 
   // self score q . k_new: only the first CTA needs it; its loads are in flight with the stream's
-  float prod = 0.f;
-  if (rank == 0 && threadIdx.x < D)
+  // (and the new value, which the merge after the cluster barrier would otherwise wait for)
+  float prod = 0.f, v_self = 0.f;
+  if (rank == 0 && threadIdx.x < D) {
     prod = Elem<T>::load(q + (size_t)slab * D + threadIdx.x) * Elem<T>::load(k_new + (size_t)kv * D + threadIdx.x);
+    v_self = Elem<T>::load(v_new + (size_t)kv * D + threadIdx.x);
+  }
 
   float m, l, o[kEpl];
   decode_stream_rows<T, D, kThreads>(q, k_rows, v_rows, row_off[kv], slab, r_begin, r_end, scale_log2, m, l, o);
@@ -436,7 +442,8 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
   cluster.sync();
   // every CTA of the cluster has read the length and its rows: the new row may go in
   // (never asked for when query heads share a slab: another head's cluster may still be reading its length)
-  if (rank == 0) append_new_row<T, D>(ap, kv, L, row_off[kv], k_new, v_new);
+  // by threads that have no part in the merge below, so that the two run side by side
+  if (rank == 0) append_new_row<T, D>(ap, kv, L, row_off[kv], k_new, v_new, D);
   if (rank == 0 && threadIdx.x < D) {
     const int d = threadIdx.x;
     float s_self = 0.f;
@@ -456,7 +463,7 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
     for (int r = 0; r < kClusterSize; ++r) mm = fmaxf(mm, mr[r]);
     for (int r = 0; r < rg.R; ++r) mm = fmaxf(mm, ring_s[r]);
     const float w_self = exp2f(s_self - mm);
-    float acc = w_self * Elem<T>::load(v_new + (size_t)kv * D + d);
+    float acc = w_self * v_self;
     float lsum = w_self;
 #pragma unroll
     for (int r = 0; r < kClusterSize; ++r) {
