@@ -16,7 +16,10 @@
 #include <cooperative_groups.h>
 #include <math.h>
 
+#include <type_traits>
+
 #include "ag_common.cuh"
+#include "decode_mma_core.cuh"
 
 namespace ag {
 
@@ -491,6 +494,137 @@ decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
   cluster.sync();
 }
 
+// The cluster form for bf16, head_dim 128, with the rows streamed through shared memory and the
+// scores and weighted sums on warp-level MMAs (decode_mma_core.cuh; the query is row 0 of the 16-row
+// operand): per row a fraction of the instructions of the CUDA-core form, which at these sizes is
+// bound by instruction issue and by what one SM can take in, not by latency alone.  CTA `rank`
+// takes whole 64-row tiles; everything after the streaming is as in decode_cluster_kernel.
+// three stages: a CTA has few tiles and no neighbour to hide behind, so two of them are kept in flight
+constexpr int kCmStages = 3;
+__global__ void __launch_bounds__(kGqThreads, 2)
+decode_cluster_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_new,
+                          const __nv_bfloat16 *__restrict__ v_new, const __nv_bfloat16 *__restrict__ k_rows,
+                          const __nv_bfloat16 *__restrict__ v_rows, const int64_t *__restrict__ row_off,
+                          const int32_t *__restrict__ len, float scale_log2, __nv_bfloat16 *__restrict__ out,
+                          const AppendArgs ap, const HeadMap hm, const RecentRing rg) {
+  namespace cg = cooperative_groups;
+  using T = __nv_bfloat16;
+  constexpr int D = kGqD;
+  static_assert(kGqThreads == D, "one thread per output dimension in the merge");
+  extern __shared__ __align__(128) uint8_t gq_smem[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int slab = blockIdx.y, rank = (int)cluster.block_rank();
+  const int kv = hm.kv_slab(slab);
+  const int d = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int L = len[kv];
+  const int per = ((L + kClusterSize - 1) / kClusterSize + kGqTile - 1) / kGqTile * kGqTile;
+  const int r_begin = min(L, rank * per), r_end = min(L, r_begin + per);
+
+  __shared__ float cta_o[D];          // this CTA's triple, read by the first CTA of the cluster
+  __shared__ float cta_ml[2];
+  __shared__ float red[D / 32];
+  __shared__ float ring_s[kMaxRecent];
+
+  // self score q . k_new and the new value: only the first CTA needs them; in flight with the stream
+  float prod = 0.f, v_self = 0.f;
+  if (rank == 0) {
+    prod = Elem<T>::load(q + (size_t)slab * D + d) * Elem<T>::load(k_new + (size_t)kv * D + d);
+    v_self = Elem<T>::load(v_new + (size_t)kv * D + d);
+  }
+
+  if (r_begin < r_end) {              // the same for the whole CTA
+    const size_t row0 = (size_t)row_off[kv] * kGqRowBytes;
+    const GqWarpTriples w = gq_stream_rows<kCmStages>(gq_smem, q + (size_t)slab * D, 1,
+                                           reinterpret_cast<const uint8_t *>(k_rows) + row0,
+                                           reinterpret_cast<const uint8_t *>(v_rows) + row0, r_begin, r_end, scale_log2);
+    float acc, mc, lc;
+    gq_combine(w, 0, d, acc, mc, lc);
+    cta_o[d] = acc;
+    if (d == 0) { cta_ml[0] = mc; cta_ml[1] = lc; }
+  } else {
+    cta_o[d] = 0.f;
+    if (d == 0) { cta_ml[0] = -INFINITY; cta_ml[1] = 0.f; }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) prod += __shfl_xor_sync(0xffffffffu, prod, off);
+  if ((d & 31) == 0) red[d >> 5] = prod;
+  if (rank == 0) ring_scores<T, D>(rg, kv, q + (size_t)slab * D, scale_log2, ring_s);
+  cluster.sync();
+  // every CTA of the cluster has read the length and its rows: the new row may go in
+  // (never asked for when query heads share a slab: another head's cluster may still be reading its length)
+  if (rank == 0) append_new_row<T, D>(ap, kv, L, row_off[kv], k_new, v_new);
+  if (rank == 0) {
+    float s_self = 0.f;
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) s_self += red[i];
+    s_self *= scale_log2;
+    float mr[kClusterSize], lr[kClusterSize], orr[kClusterSize];
+#pragma unroll
+    for (int r = 0; r < kClusterSize; ++r) {
+      const float *ml = cluster.map_shared_rank(cta_ml, r);
+      mr[r] = ml[0];
+      lr[r] = ml[1];
+      orr[r] = cluster.map_shared_rank(cta_o, r)[d];
+    }
+    float mm = s_self;
+#pragma unroll
+    for (int r = 0; r < kClusterSize; ++r) mm = fmaxf(mm, mr[r]);
+    for (int r = 0; r < rg.R; ++r) mm = fmaxf(mm, ring_s[r]);
+    const float w_self = exp2f(s_self - mm);
+    float acc = w_self * v_self;
+    float lsum = w_self;
+#pragma unroll
+    for (int r = 0; r < kClusterSize; ++r) {
+      const float w = mr[r] == -INFINITY ? 0.f : exp2f(mr[r] - mm);
+      acc = fmaf(w, orr[r], acc);
+      lsum = fmaf(w, lr[r], lsum);
+    }
+    // the evicted tokens of the recent-token window
+    for (int r = 0; r < rg.R; ++r) {
+      if (ring_s[r] == -INFINITY) continue;
+      const float w = exp2f(ring_s[r] - mm);
+      acc = fmaf(w, Elem<T>::load(static_cast<const T *>(rg.v) + ((size_t)kv * rg.R + r) * D + d), acc);
+      lsum += w;
+    }
+    Elem<T>::store(out + (size_t)slab * D + d, acc / lsum);
+  }
+  if (rank == 0 && rg.R > 0 && ap.flag_new != nullptr) {
+    // the step carries the append: the new token joins the ring once every thread has read it
+    constexpr int kVecs = D * (int)sizeof(T) / 16;
+    __syncthreads();
+    if (d < kVecs)
+      ring_put<kVecs>(rg, kv, d, reinterpret_cast<const uint8_t *>(k_new + (size_t)kv * D),
+                      reinterpret_cast<const uint8_t *>(v_new + (size_t)kv * D), ap.flag_new[kv] != 0);
+  }
+  cluster.sync();
+}
+
+static int launch_decode_cluster_mma(int slabs, const void *q, const void *k_new, const void *v_new,
+                                     const ag_cache &c, float scale_log2, void *o, const AppendArgs &ap,
+                                     const HeadMap &hm, const RecentRing &rg, cudaStream_t st) {
+  using T = __nv_bfloat16;
+  AG_CUDA_TRY(cudaFuncSetAttribute(decode_cluster_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   gq_smem_bytes(kCmStages)));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kClusterSize, slabs);
+  cfg.blockDim = dim3(kGqThreads);
+  cfg.dynamicSmemBytes = gq_smem_bytes(kCmStages);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kClusterSize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1] = pdl_attribute();
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  AG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_cluster_mma_kernel, static_cast<const T *>(q),
+                                 static_cast<const T *>(k_new), static_cast<const T *>(v_new),
+                                 static_cast<const T *>(c.k_rows), static_cast<const T *>(c.v_rows),
+                                 c.row_off, c.len, scale_log2, static_cast<T *>(o), ap, hm, rg));
+  return AG_OK;
+}
+
 template <typename T, int D, int kThreads>
 static int launch_decode_cluster(int slabs, const void *q, const void *k_new, const void *v_new,
                                  const ag_cache &c, float scale_log2, void *o, const AppendArgs &ap,
@@ -524,6 +658,10 @@ static int run_decode(const ag_layer_desc &d, const void *q, const void *k_new, 
   const HeadMap hm{d.heads, kv_heads_of(d)};
   const RecentRing rg = ring_of(d, c);
   const float scale_log2 = scale * 1.4426950408889634f;
+  if constexpr (std::is_same_v<T, __nv_bfloat16> && D == kGqD) {
+    if (slabs <= kClusterMaxSlabs)
+      return launch_decode_cluster_mma(slabs, q, k_new, v_new, c, scale_log2, o, ap, hm, rg, st);
+  }
   if (slabs <= kClusterMaxSlabs)
     return launch_decode_cluster<T, D, kClusterThreads>(slabs, q, k_new, v_new, c, scale_log2, o, ap, hm, rg, st);
   int chunk_rows = (c.max_cap + kMaxSplits - 1) / kMaxSplits;
