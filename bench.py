@@ -46,7 +46,7 @@ WORKLOADS = {
 # None whenever the kernel changes after the capture.
 TRAFFIC = {
     ("prefill7b", "prefill"): 154.86e6 + 18.50e6,        # prefill_tc_kernel
-    ("prefill7b", "decode"): 41.21e6 + 0.03e6,           # decode_cluster_kernel<bf16,128,512>
+    ("prefill7b", "decode"): 41.22e6 + 0.01e6,           # decode_cluster_mma_kernel
     ("prefill7b", "compact"): 41.26e6 + 3.10e6,          # compact_kernel<256> (written rows still in L2 at kernel end)
     ("decode_ragged", "decode"): 2.3530e9 + 7.1e6,       # decode_partial_kernel<bf16,128>
 }
