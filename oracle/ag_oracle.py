@@ -215,6 +215,31 @@ def compact_kv(K, V, flags, window=1):
     return cache
 
 
+def project_kv(X, Wk, Wv, kv_heads):
+    """Keys and values of the layer from its hidden states, Eq. 2: K_i = X W^K_i,
+    V_i = X W^V_i, head i taking columns [i D, (i + 1) D) of the "in x out"
+    weight.  X [B, n, d], Wk, Wv [d, kv_heads * D] -> K, V [B, kv_heads, n, D]
+    in float64 (no rounding to a storage type)."""
+    X, Wk, Wv = _as_f64(X), _as_f64(Wk), _as_f64(Wv)
+    B, n, d = X.shape
+    D = Wk.shape[1] // kv_heads
+    K = np.empty((B, kv_heads, n, D), dtype=F64)
+    V = np.empty((B, kv_heads, n, D), dtype=F64)
+    for b in range(B):
+        for i in range(kv_heads):
+            K[b, i] = X[b] @ Wk[:, i * D:(i + 1) * D]
+            V[b, i] = X[b] @ Wv[:, i * D:(i + 1) * D]
+    return K, V
+
+
+def project_and_cache(X, Wk, Wv, flags):
+    """Eq. 2's projection followed by selective caching (Sec. 3.3): the dense
+    K, V [B, h, n, D] and the ragged cache of the retained rows, as
+    (K, V, compact_kv(K, V, flags))."""
+    K, V = project_kv(X, Wk, Wv, flags.shape[1])
+    return K, V, compact_kv(K, V, flags)
+
+
 # --------------------------------------------------------------------------
 # Step 3: prefill attention under the eviction mask.  Eq. 2 and Eq. 5.
 # --------------------------------------------------------------------------
