@@ -12,6 +12,9 @@
  *   ag_cache_append   concatenate the new k, v to the cache    Sec. 3.1 (decoding stage)
  *   ag_decode_step    the two above in one call                Sec. 3.1 (decoding stage)
  *   ag_gate_linear_forward  the local gate, s = X W_lin        Sec. 3.4 ("Local or global?")
+ *   ag_kv_project_cache     K_i = X W^K_i, V_i = X W^V_i written
+ *                           to the dense K, V and, for retained
+ *                           tokens, straight into the cache     Eq. 2 + Sec. 3.3 (after Eq. 4)
  *
  * Conventions common to every call
  * --------------------------------
@@ -200,6 +203,36 @@ int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
                   const uint8_t *flags, ag_cache *cache, int32_t *prefix,
                   int32_t *idx, int32_t *dev_status, void *ws, size_t ws_bytes,
                   void *cuda_stream);
+
+/*
+ * Steps "project" + 2 in one call — the key/value projection of Eq. 2,
+ *   K_i = X W^K_i,  V_i = X W^V_i      (head i = columns [i D, (i + 1) D) of the weight),
+ * fused with selective caching (Sec. 3.3: k_i^(t), v_i^(t) are retained iff
+ * AG(X)_i^(t) = 1).  Each projected tile is rounded to the layer dtype once and
+ * written to both places the layer reads it from: the dense K, V (every token
+ * attends to its own key and value, the diagonal of Eq. 5) and, for retained
+ * tokens, cache row row_off[s] + prefix[s, t].  It replaces the copying pass of
+ * ag_compact_kv: the order of calls is gate -> ag_compact_kv with K = V = NULL
+ * (flags -> prefix, idx) -> this call -> ag_prefill_attn.
+ *
+ *   X       [B, n, d]             in
+ *   Wk, Wv  [d, h D]              in   ("in x out")
+ *   flags   [B, h, n] uint8       in
+ *   prefix  [B, h, n + 1] int32   in   (as the count pass wrote it)
+ *   cache   host struct           in/out: k_rows, v_rows of the retained tokens, len[s] = prefix[s, n]
+ *   K, V    [B, h, n, D]          out  dense projections (h = kv_heads for grouped-query attention)
+ *   dev_status  int32 or NULL     in/out
+ * A slab with prefix[s, n] > cap[s] gets no rows, len[s] = 0 and AG_DEV_OVERFLOW,
+ * as in ag_compact_kv.  The cache rows are bit copies of the dense K, V rows.
+ * Needs no workspace.  Kernel coverage: bfloat16, head_dim 128, n a multiple of
+ * 128, d a multiple of 8, no recent-token window; anything else returns
+ * AG_ERR_UNSUPPORTED (project with a GEMM of your own and call ag_compact_kv).
+ * AG_ERR_INVALID_ARG for missing or misaligned (16-byte) pointers.
+ */
+int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk,
+                        const void *Wv, const uint8_t *flags, const int32_t *prefix,
+                        ag_cache *cache, void *K, void *V, int32_t *dev_status,
+                        void *cuda_stream);
 
 /*
  * Step 3 — prefill attention under the eviction mask (Eq. 2 with Eq. 5):

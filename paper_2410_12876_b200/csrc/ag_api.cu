@@ -127,6 +127,23 @@ int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
                         (cudaStream_t)cuda_stream);
 }
 
+int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk, const void *Wv,
+                        const uint8_t *flags, const int32_t *prefix, ag_cache *cache, void *K, void *V,
+                        int32_t *dev_status, void *cuda_stream) {
+  int st = check_desc(desc);
+  if (st) return st;
+  if (desc->hidden <= 0) return AG_ERR_INVALID_ARG;
+  if (!X || !Wk || !Wv || !flags || !prefix || !K || !V) return AG_ERR_INVALID_ARG;
+  st = check_cache(cache);
+  if (st) return st;
+  if (misaligned16(X) || misaligned16(Wk) || misaligned16(Wv) || misaligned16(K) || misaligned16(V) ||
+      misaligned16(prefix))
+    return AG_ERR_INVALID_ARG;
+  if (!kv_proj_cache_supported(*desc)) return AG_ERR_UNSUPPORTED;
+  return launch_kv_proj_cache(*desc, X, Wk, Wv, flags, prefix, *cache, K, V, dev_status,
+                              (cudaStream_t)cuda_stream);
+}
+
 int ag_prefill_attn(const ag_layer_desc *desc, const void *Q, const void *K,
                     const void *V, const uint8_t *flags, const ag_cache *cache,
                     const int32_t *prefix, float softmax_scale, void *O, void *ws,
@@ -213,8 +230,8 @@ int ag_last_cuda_error(void) { return ag::g_last_cuda_error; }
 int ag_device_wait_timeouts(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return -1;
   const int a = gemm_tc_wait_timeouts(), b = prefill_tc_wait_timeouts(),
-            c = gate_attn_tc_wait_timeouts() + gate_linear_wait_timeouts();
-  return (a < 0 || b < 0 || c < 0) ? -1 : a + b + c;
+            c = gate_attn_tc_wait_timeouts() + gate_linear_wait_timeouts(), e = kv_proj_cache_wait_timeouts();
+  return (a < 0 || b < 0 || c < 0 || e < 0) ? -1 : a + b + c + e;
 }
 
 }  // extern "C"

@@ -1,0 +1,280 @@
+// Key/value projection fused with selective caching: K_i = X W^K_i, V_i = X W^V_i (Eq. 2) on the
+// 5th-generation tensor cores, with an epilogue that rounds each tile to bf16 once and sends it
+// to both places the layer reads it from: the dense K, V [B, h, n, D] (every token attends to its
+// own key, the diagonal of Eq. 5) and, for the tokens the gate retains (Sec. 3.3: k, v are kept
+// iff AG = 1), row row_off[s] + prefix[s, t] of the ragged cache.  The separate compaction pass
+// over K and V (a read of the retained rows and a launch) disappears; only the count pass that
+// turns flags into prefix stays.
+//
+// One CTA computes MT sub-tiles of 128 tokens x BN columns of the packed output [K | V]; a tile
+// lies in one weight and covers BN / 128 whole heads.  Warp 0 drives TMA, warp 1 owns tensor
+// memory and issues the MMAs, warps 2..5 drain the accumulator.  Main loop as in the gate's
+// projection GEMM (A = X K-major, B = W MN-major panels of [64 k][64 n], 128-byte swizzle).
+// Epilogue per sub-tile: the destination rows of its tokens are looked up while the MMAs run;
+// the tile is staged as bf16 over the (by then free) operand stages in the layout of a swizzled
+// TMA store, the dense copy leaves by TMA stores, and the retained rows are copied from the
+// same staging area, one 256-byte row per half-warp.
+#include "ag_common.cuh"
+#include "umma.cuh"
+
+namespace ag {
+
+using namespace umma;
+
+namespace {
+
+constexpr int kBM = 128, kBK = 64, kThreads = 192, kD = 128;
+
+template <int BN, int MT> struct KvCfg {
+  static constexpr int kStages = BN == 256 ? (MT == 2 ? 3 : 4) : 6;
+  static constexpr int kABytes = MT * kBM * kBK * 2;
+  static constexpr int kPanelBytes = kBK * 64 * 2;           // [64 k][64 n] = 8 KB
+  static constexpr int kBBytes = (BN / 64) * kPanelBytes;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kHeads = BN / kD;                     // heads per tile
+  static constexpr int kDstBytes = MT * kHeads * kBM * 8;    // destination row of every (sub-tile, head, token)
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + kDstBytes;
+};
+
+template <int BN, int MT>
+__global__ void __launch_bounds__(kThreads, 1)
+kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBk,
+                     const __grid_constant__ CUtensorMap tmBv, const __grid_constant__ CUtensorMap tmK,
+                     const __grid_constant__ CUtensorMap tmV, const uint8_t *__restrict__ flags,
+                     const int32_t *__restrict__ prefix, const int64_t *__restrict__ row_off,
+                     const int32_t *__restrict__ cap, int32_t *__restrict__ len, uint8_t *__restrict__ k_rows,
+                     uint8_t *__restrict__ v_rows, int32_t *__restrict__ dev_status, int M, int Kdim, int GD,
+                     int n, int kv_heads, int n_tiles_n) {
+  using Cfg = KvCfg<BN, MT>;
+  constexpr uint32_t kTmemCols = MT * BN;
+  static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "TMEM columns: a power of two");
+  static_assert((BN / 64) * kBM * 128 <= Cfg::kStages * Cfg::kStageBytes, "staging fits the stages");
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + Cfg::kStages * Cfg::kStageBytes);
+  uint64_t *empty = full + Cfg::kStages;
+  uint64_t *acc_full = empty + Cfg::kStages;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  long long *dst_row = reinterpret_cast<long long *>(smem + Cfg::kStages * Cfg::kStageBytes + 256);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x;
+  const int m0 = (tile / n_tiles_n) * (MT * kBM);
+  const int n0 = (tile % n_tiles_n) * BN;        // in the packed [2 * GD] output
+  const int which = n0 / GD, nw = n0 % GD;       // BN divides GD: a tile lies in one weight
+  const CUtensorMap *tmB = which == 0 ? &tmBk : &tmBv;
+  const int num_kb = (Kdim + kBK - 1) / kBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    fence_barrier_init();
+    prefetch_tensormap(&tmA);
+    prefetch_tensormap(tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_acc = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % Cfg::kStages;
+        const uint32_t ph = (kb / Cfg::kStages) & 1;
+        if (!mbar_wait(&empty[s], ph ^ 1)) break;
+        uint8_t *a = smem + s * Cfg::kStageBytes, *b = a + Cfg::kABytes;
+        mbar_arrive_expect_tx(&full[s], Cfg::kStageBytes);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)              // rows past M are filled with zeros
+          tma_load_2d(a + mt * (kBM * kBK * 2), &tmA, &full[s], kb * kBK, m0 + mt * kBM);
+#pragma unroll
+        for (int p = 0; p < BN / 64; ++p)
+          tma_load_2d(b + p * Cfg::kPanelBytes, tmB, &full[s], nw + p * 64, kb * kBK);
+      }
+    }
+  } else if (warp == 1) {
+    // every lane runs the control flow (operands stay warp-uniform); one elected lane issues
+    const uint32_t idesc = idesc_bf16_f32(kBM, BN, false, true);
+    const uint64_t da0 = desc_kmajor_sw128(smem_u32(smem));
+    const uint64_t db0 = desc_mnmajor_sw128(smem_u32(smem) + Cfg::kABytes, Cfg::kPanelBytes);
+    const uint32_t a_lo0 = (uint32_t)da0, a_hi = (uint32_t)(da0 >> 32);
+    const uint32_t b_lo0 = (uint32_t)db0, b_hi = (uint32_t)(db0 >> 32);
+    bool ok = true;
+    for (int kb = 0; kb < num_kb && ok; ++kb) {
+      const int s = kb % Cfg::kStages;
+      const uint32_t ph = (kb / Cfg::kStages) & 1;
+      ok = mbar_wait(&full[s], ph);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t a_lo = a_lo0 + ((s * Cfg::kStageBytes) >> 4), b_lo = b_lo0 + ((s * Cfg::kStageBytes) >> 4);
+      if (elect_one()) {
+#pragma unroll
+        for (int k = 0; k < kBK / 16; ++k) {
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+            mma_ss_lohi(tmem_acc + mt * BN, a_lo + ((mt * kBM * kBK * 2 + k * 32) >> 4), a_hi,
+                        b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
+        }
+        mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
+      }
+      __syncwarp();
+    }
+    if (elect_one()) mma_commit(acc_full);   // accumulator complete (or unwinding)
+    __syncwarp();
+  } else {
+    // epilogue warps: warp w may touch TMEM lanes [32 * (w % 4), +32)
+    const int quad = warp & 3;
+    const int r_in = quad * 32 + lane;           // token of the sub-tile this thread drains
+    // Where each token of the tile goes in the ragged cache (-1: evicted, or its slab is too small),
+    // looked up while the MMAs run.  The CTAs of the key tiles that hold a sequence's first token
+    // also set the slab's length.
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      const int m_base = m0 + mt * kBM;
+      const int b = m_base / n, t = m_base % n + r_in;      // n is a multiple of 128: one sequence per sub-tile
+#pragma unroll
+      for (int hh = 0; hh < Cfg::kHeads; ++hh) {
+        long long d = -1;
+        if (m_base < M) {
+          const size_t slab = (size_t)b * kv_heads + nw / kD + hh;
+          const int32_t *pre = prefix + slab * (n + 1);
+          const int total = pre[n];
+          const bool fits = total <= cap[slab];
+          if (fits && flags[slab * n + t] != 0) d = row_off[slab] + pre[t];
+          if (t == 0 && which == 0) {
+            len[slab] = fits ? total : 0;
+            if (!fits && dev_status) atomicOr(dev_status, AG_DEV_OVERFLOW);
+          }
+        }
+        dst_row[(mt * Cfg::kHeads + hh) * kBM + r_in] = d;
+      }
+    }
+    const bool ok = mbar_wait(acc_full, 0);
+    tc_fence_after_sync();
+    const CUtensorMap *tmOut = which == 0 ? &tmK : &tmV;
+    uint8_t *rows_out = which == 0 ? k_rows : v_rows;
+    const int hw = (warp - 2) * 2 + (lane >> 4), l16 = lane & 15;   // half-warp 0..7, 16-byte piece of a row
+#pragma unroll 1
+    for (int mt = 0; mt < MT; ++mt) {
+      const int m_base = m0 + mt * kBM;
+      if (!ok || num_kb == 0 || m_base >= M) break;
+      const uint32_t tmem_sub = tmem_acc + mt * BN;
+      // bf16 tile as panels of [128 tokens][64 columns] (128-byte rows, 16-byte chunks XOR-swizzled by the row)
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 32) {
+        uint32_t r[32];
+        tmem_ld_x32_sync(tmem_sub + ((uint32_t)(quad * 32) << 16) + c, r);
+        const uint32_t panel = (uint32_t)(c >> 6) * kBM * 128 + r_in * 128;
+#pragma unroll
+        for (int e = 0; e < 32; e += 8) {
+          uint32_t h[4];
+#pragma unroll
+          for (int q = 0; q < 8; q += 2)
+            h[q >> 1] = pack_bf16x2(__uint_as_float(r[e + q]), __uint_as_float(r[e + q + 1]));
+          const uint32_t chunk = (uint32_t)(((c & 32) >> 3) + (e >> 3));
+          *reinterpret_cast<uint4 *>(smem + panel + ((chunk ^ (r_in & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
+        }
+      }
+      fence_proxy_async_smem();
+      named_barrier_sync(1, 128);
+      const int b = m_base / n, t0 = m_base % n;
+      if (threadIdx.x == 64) {
+#pragma unroll
+        for (int p = 0; p < BN / 64; ++p)
+          tma_store_3d(tmOut, smem + p * kBM * 128, (p & 1) * 64, t0, b * kv_heads + nw / kD + (p >> 1));
+        tma_store_commit();
+      }
+      // retained rows: half-warp per row, 16 bytes per lane
+#pragma unroll
+      for (int hh = 0; hh < Cfg::kHeads; ++hh) {
+        const long long *dr = dst_row + (mt * Cfg::kHeads + hh) * kBM;
+#pragma unroll 4
+        for (int r = hw; r < kBM; r += 8) {
+          const long long d = dr[r];
+          if (d >= 0) {
+            const uint32_t off = (uint32_t)(hh * 2 + (l16 >> 3)) * kBM * 128 + r * 128 + (((l16 & 7) ^ (r & 7)) << 4);
+            *reinterpret_cast<uint4 *>(rows_out + (size_t)d * (kD * 2) + l16 * 16) =
+                *reinterpret_cast<const uint4 *>(smem + off);
+          }
+        }
+      }
+      if (MT > 1) {
+        if (threadIdx.x == 64) tma_store_wait_read();
+        named_barrier_sync(1, 128);          // the staging area is free for the next sub-tile
+      }
+    }
+    if (threadIdx.x == 64) tma_store_wait_read();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_acc, kTmemCols);
+}
+
+int sm_count() {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, v = 0;
+    sms = (cudaGetDevice(&dev) == cudaSuccess &&
+           cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) ? v : 148;
+  }
+  return sms;
+}
+
+template <int BN, int MT>
+int run(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, const uint8_t *flags,
+        const int32_t *prefix, const ag_cache &c, void *K, void *V, int32_t *dev_status, cudaStream_t st) {
+  using Cfg = KvCfg<BN, MT>;
+  const int hk = kv_heads_of(d), GD = hk * kD, M = d.batch * d.seq, Kdim = d.hidden;
+  CUtensorMap tmA, tmBk, tmBv, tmK, tmV;
+  int rc = make_tmap_2d_bf16(&tmA, X, M, Kdim, (uint64_t)Kdim * 2, kBM, kBK);
+  if (rc) return rc;
+  rc = make_tmap_2d_bf16(&tmBk, Wk, Kdim, GD, (uint64_t)GD * 2, kBK, 64);
+  if (rc) return rc;
+  rc = make_tmap_2d_bf16(&tmBv, Wv, Kdim, GD, (uint64_t)GD * 2, kBK, 64);
+  if (rc) return rc;
+  rc = make_tmap_3d_bf16(&tmK, K, (uint64_t)d.batch * hk, d.seq, kD, kBM, 64);
+  if (rc) return rc;
+  rc = make_tmap_3d_bf16(&tmV, V, (uint64_t)d.batch * hk, d.seq, kD, kBM, 64);
+  if (rc) return rc;
+  auto kern = kv_proj_cache_kernel<BN, MT>;
+  AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+  const int n_tiles_n = 2 * GD / BN, n_tiles = n_tiles_n * ((M + MT * kBM - 1) / (MT * kBM));
+  kern<<<n_tiles, kThreads, Cfg::kSmemBytes, st>>>(tmA, tmBk, tmBv, tmK, tmV, flags, prefix, c.row_off, c.cap, c.len,
+                                                   static_cast<uint8_t *>(c.k_rows), static_cast<uint8_t *>(c.v_rows),
+                                                   dev_status, M, Kdim, GD, d.seq, hk, n_tiles_n);
+  AG_LAUNCH_CHECK();
+  return AG_OK;
+}
+
+}  // namespace
+
+bool kv_proj_cache_supported(const ag_layer_desc &d) {
+  return d.dtype == AG_BF16 && d.head_dim == kD && d.seq % kBM == 0 && d.hidden > 0 && d.hidden % 8 == 0 &&
+         recent_rows(d) == 0 && (int64_t)d.batch * d.seq < ((int64_t)1 << 31);
+}
+
+int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, const uint8_t *flags,
+                         const int32_t *prefix, const ag_cache &c, void *K, void *V, int32_t *dev_status,
+                         cudaStream_t st) {
+  const int hk = kv_heads_of(d);
+  const long long tiles128 = (long long)(2 * hk * kD / 128) * (d.batch * (long long)d.seq / kBM);
+  if (hk % 2 == 0) {
+    // more than one wave: 256-token tiles, whose two sub-tiles share every stage of W
+    if (tiles128 > 2 * sm_count()) return run<256, 2>(d, X, Wk, Wv, flags, prefix, c, K, V, dev_status, st);
+    return run<256, 1>(d, X, Wk, Wv, flags, prefix, c, K, V, dev_status, st);
+  }
+  return run<128, 1>(d, X, Wk, Wv, flags, prefix, c, K, V, dev_status, st);
+}
+
+int kv_proj_cache_wait_timeouts() {
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, umma::g_wait_expired, sizeof(int)) != cudaSuccess) return -1;
+  return v;
+}
+
+}  // namespace ag

@@ -1,0 +1,188 @@
+"""Parity of ag_kv_project_cache with the oracle: the key/value projection of Eq. 2 whose
+epilogue writes the retained rows straight into the ragged cache (Sec. 3.3).
+
+The dense K, V are compared with the oracle's float64 projection element by element (one
+rounding to bfloat16 plus float32 summation error); lengths and the positions of the cached
+rows are bit-exact against the oracle's cache (a cached row must be the bit pattern of the
+dense row at the oracle's r-th retained position); at the full layer size the dense outputs
+are compared on sampled (head, token) rows the oracle computes one by one."""
+import numpy as np
+import pytest
+import torch
+
+import agtest as T
+from oracle import ag_oracle as orc
+from paper_2410_12876_b200 import binding as ag
+from paper_2410_12876_b200 import inputs
+from paper_2410_12876_b200.inputs import LayerShape
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    T.ensure_built()
+
+
+def _close_to_rounded(got, ref, what):
+    """|got - ref| <= half a bfloat16 ulp of ref (2^-8 |ref| bounds it) + float32 summation slack."""
+    got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, what
+    if got.size == 0:
+        return
+    assert np.all(np.isfinite(got)), what
+    excess = np.abs(got - ref) - (2.0 ** -8 * np.abs(ref) + 1e-5)
+    assert np.max(excess) <= 0, f"{what}: {np.max(excess):.3e} beyond one rounding"
+
+
+def _flags(shape, seed):
+    """Per-head Bernoulli flags with rates spread over [0, 1]; head 0 keeps nothing, head 1 everything."""
+    rng = np.random.default_rng(seed)
+    B, h, n = shape.batch, shape.kvh, shape.seq
+    rate = rng.uniform(0.05, 0.95, size=(B, h, 1))
+    f = (rng.random((B, h, n)) < rate).astype(np.uint8)
+    f[:, 0] = 0
+    if h > 1:
+        f[:, 1] = 1
+    return f
+
+
+def gpu_project_cache(shape, X, W, flags, cap=None):
+    """Count pass (flags -> prefix, idx), then the fused projection."""
+    desc = ag.make_desc(shape)
+    B, h, n, D = shape.batch, shape.kvh, shape.seq, shape.head_dim
+    if cap is None:
+        cap = [n] * (B * h)
+    cache = ag.RaggedCache.allocate(shape, cap, DEV)
+    prefix = torch.full((B, h, n + 1), -1, dtype=torch.int32, device=DEV)
+    idx = torch.full((B, h, n), -1, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ag.ag_compact_kv(desc, None, None, flags, cache, prefix, idx, status, None)
+    cache.len.fill_(-7)                                    # the fused call sets the lengths itself
+    K = torch.full((B, h, n, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+    V = torch.full_like(K, float("nan"))
+    ag.ag_kv_project_cache(desc, X, W["Wk"], W["Wv"], flags, prefix, cache, K, V, status)
+    torch.cuda.synchronize()
+    return cache, prefix, idx, status, K, V
+
+
+def _check(shape, seed, cap=None):
+    X = inputs.hidden_states(shape, seed, DEV)
+    W = inputs.layer_weights(shape, seed + 10, DEV)
+    fl = _flags(shape, seed + 20)
+    flags = torch.from_numpy(fl).to(DEV)
+    cache, prefix, idx, status, K, V = gpu_project_cache(shape, X, W, flags, cap)
+    Kr, Vr, ocache = orc.project_and_cache(T.f64(X), T.f64(W["Wk"]), T.f64(W["Wv"]), fl)
+    _close_to_rounded(T.f64(K), Kr, "dense K")
+    _close_to_rounded(T.f64(V), Vr, "dense V")
+    L = orc.cache_lengths(ocache).reshape(-1)
+    capv = cache.cap.cpu().numpy()
+    fits = L <= capv
+    assert np.array_equal(cache.len.cpu().numpy(), np.where(fits, L, 0))
+    assert int(status.item()) == (0 if fits.all() else ag.AG_DEV_OVERFLOW)
+    kd, vd = T.bits(K), T.bits(V)
+    kr, vr = T.bits(cache.k_rows), T.bits(cache.v_rows)
+    off = cache.row_off.cpu().numpy()
+    for b in range(shape.batch):
+        for i in range(shape.kvh):
+            s = b * shape.kvh + i
+            pos = ocache[b][i]["idx"]                      # the oracle's retained positions
+            if fits[s]:
+                assert np.array_equal(kr[off[s]:off[s] + L[s]], kd[b, i][pos]), (b, i)
+                assert np.array_equal(vr[off[s]:off[s] + L[s]], vd[b, i][pos]), (b, i)
+                _close_to_rounded(T.f64(cache.k_rows[off[s]:off[s] + L[s]]), ocache[b][i]["k"], "cached keys")
+                _close_to_rounded(T.f64(cache.v_rows[off[s]:off[s] + L[s]]), ocache[b][i]["v"], "cached values")
+                # rows of the slab past its length were not written
+                assert not kr[off[s] + L[s]:off[s] + capv[s]].any()
+            else:
+                assert not kr[off[s]:off[s] + capv[s]].any() and not vr[off[s]:off[s] + capv[s]].any()
+    assert ag.ag_device_wait_timeouts() == 0
+    return cache, prefix, K, V, fl
+
+
+# (batch, seq, hidden, heads, head_dim, gate_heads, gate_head_dim, dtype)
+CASES = {
+    "two_heads_per_tile": LayerShape(2, 256, 512, 4, 128, 2, 128, "bf16"),
+    "k_tail": LayerShape(1, 384, 520, 4, 128, 2, 128, "bf16"),                 # hidden not a multiple of 64
+    "odd_heads": LayerShape(2, 128, 256, 3, 128, 1, 128, "bf16"),              # one head per tile
+    "two_subtiles": LayerShape(1, 1280, 256, 16, 128, 2, 128, "bf16"),         # 256-token tiles
+    "two_subtiles_odd_rows": LayerShape(1, 1152, 192, 18, 128, 2, 128, "bf16"),  # last tile has one sub-tile
+    "subtiles_of_two_sequences": LayerShape(3, 384, 128, 20, 128, 2, 128, "bf16"),
+    "grouped_query": LayerShape(2, 256, 256, 8, 128, 2, 128, "bf16", kv_heads=2),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_projection_and_cache(name):
+    _check(CASES[name], 900)
+
+
+def test_slab_too_small_is_skipped_and_reported():
+    shape = CASES["two_heads_per_tile"]
+    cap = [shape.seq] * (shape.batch * shape.kvh)
+    cap[1] = 17                                            # head 1 keeps every token
+    cap[5] = shape.seq - 1
+    _check(shape, 910, cap)
+
+
+def test_feeds_prefill_and_decode():
+    """gate flags -> count pass -> fused projection -> prefill attention and a decode step, against the
+    oracle run on the projected K, V the library wrote."""
+    shape = LayerShape(1, 512, 512, 4, 128, 2, 128, "bf16")
+    cache, prefix, K, V, fl = _check(shape, 920)
+    Q = inputs.randn((1, 4, 512, 128), 921, DEV, torch.bfloat16)
+    flags = torch.from_numpy(fl).to(DEV)
+    O = T.gpu_prefill(shape, Q, K, V, flags, cache, prefix)
+    ref = orc.prefill_attention(T.f64(Q), T.f64(K), T.f64(V), fl)
+    T.check_close(T.f64(O), ref, "bf16", "prefill after the fused projection")
+    q, kn, vn, fn = inputs.decode_inputs(shape, 922, 0, DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status, fused=True)
+    oc = orc.compact_kv(T.f64(K), T.f64(V), fl)
+    ref = orc.decode_attention(T.f64(q), T.f64(kn), T.f64(vn), oc)
+    T.check_close(T.f64(o), ref, "bf16", "decode after the fused projection")
+
+
+def test_full_size_layer_sampled():
+    """The 7B-shaped layer in the launch configuration bench.py times: sampled dense rows against the
+    oracle, lengths and every cached row against the flags."""
+    shape = inputs.PREFILL7B
+    X = inputs.hidden_states(shape, 2000, DEV)
+    W = inputs.layer_weights(shape, 2010, DEV)
+    fl = _flags(shape, 930)
+    flags = torch.from_numpy(fl).to(DEV)
+    cache, prefix, idx, status, K, V = gpu_project_cache(shape, X, W, flags)
+    assert int(status.item()) == 0
+    L = fl.sum(axis=2, dtype=np.int64).reshape(-1)
+    assert np.array_equal(cache.len.cpu().numpy(), L)
+    Xf, Wk, Wv = T.f64(X)[0], T.f64(W["Wk"]), T.f64(W["Wv"])
+    rng = np.random.default_rng(931)
+    D = shape.head_dim
+    for i in range(shape.heads):
+        rows = np.unique(np.concatenate([[0, 127, 128, shape.seq - 1], rng.integers(0, shape.seq, 12)]))
+        _close_to_rounded(T.f64(K[0, i][torch.from_numpy(rows).to(DEV)]), Xf[rows] @ Wk[:, i * D:(i + 1) * D], "K")
+        _close_to_rounded(T.f64(V[0, i][torch.from_numpy(rows).to(DEV)]), Xf[rows] @ Wv[:, i * D:(i + 1) * D], "V")
+    off = cache.row_off.cpu().numpy()
+    kd, vd, kr, vr = T.bits(K), T.bits(V), T.bits(cache.k_rows), T.bits(cache.v_rows)
+    for i in range(shape.heads):
+        pos = np.flatnonzero(fl[0, i])
+        assert np.array_equal(kr[off[i]:off[i] + L[i]], kd[0, i][pos])
+        assert np.array_equal(vr[off[i]:off[i] + L[i]], vd[0, i][pos])
+    assert ag.ag_device_wait_timeouts() == 0
+
+
+def test_rejects_what_it_has_no_kernel_for():
+    shape = CASES["two_heads_per_tile"]
+    X = inputs.hidden_states(shape, 1, DEV)
+    W = inputs.layer_weights(shape, 2, DEV)
+    flags = torch.ones(shape.batch, shape.kvh, shape.seq, dtype=torch.uint8, device=DEV)
+    cache, prefix, idx, status, K, V = gpu_project_cache(shape, X, W, flags)
+    for bad in (shape.with_(seq=200), shape.with_(head_dim=64), shape.with_(dtype="f32"), shape.with_(hidden=516),
+                shape.with_(recent_window=5)):
+        with pytest.raises(ag.AgError) as e:
+            ag.ag_kv_project_cache(ag.make_desc(bad), X, W["Wk"], W["Wv"], flags, prefix, cache, K, V, status)
+        assert e.value.status in (ag.AG_ERR_UNSUPPORTED, ag.AG_ERR_INVALID_ARG)
+    with pytest.raises(ag.AgError) as e:
+        ag.ag_kv_project_cache(ag.make_desc(shape), X, W["Wk"], None, flags, prefix, cache, K, V, status)
+    assert e.value.status == ag.AG_ERR_INVALID_ARG
