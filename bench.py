@@ -238,6 +238,18 @@ class LayerRun:
             self.flags_lin = torch.empty_like(self.flags)
         self.ag.ag_gate_linear_forward(self.desc, self.X, self.W_lin, None, self.scores, self.flags_lin)
 
+    def kv_project_cache(self):
+        """Eq. 2's key/value projection with the retained rows written straight into the cache (count
+        pass + ag_kv_project_cache): what a layer that owns its K/V projection runs in place of
+        projection + compaction; timed on its own, not part of a step."""
+        ag = self.ag
+        if not hasattr(self, "K2"):
+            self.K2, self.V2 = torch.empty_like(self.K), torch.empty_like(self.V)
+        ag.ag_compact_kv(self.desc, None, None, self.cur_flags, self.cache, self.prefix, None, self.status,
+                         self.ws[ag.AG_CALL_COMPACT])
+        ag.ag_kv_project_cache(self.desc, self.X, self.W["Wk"], self.W["Wv"], self.cur_flags, self.prefix, self.cache,
+                               self.K2, self.V2, self.status)
+
     def compact(self):
         ag = self.ag
         ag.ag_compact_kv(self.desc, self.K, self.V, self.cur_flags, self.cache, self.prefix, None, self.status,
@@ -546,6 +558,26 @@ def run_ours(args, rank, world, dev):
                                     "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                     "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
                                     "algorithmic_bytes": lb, "ms": lin_ms}
+        if sh.dtype == "bf16" and sh.head_dim == 128 and sh.seq % 128 == 0 and sh.recent_window <= 1 and run.layers == 1:
+            # the fused key/value projection, timed apart from the step like the local gate
+            kv_ev = []
+            for i in range(3 + min(args.steps, 20)):
+                flush_l2(l2buf)
+                s_, e_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                s_.record()
+                run.kv_project_cache()
+                e_.record()
+                if i >= 3:
+                    kv_ev.append((s_, e_))
+            torch.cuda.synchronize()
+            kv_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in kv_ev]))
+            kf = 2.0 * sh.batch * sh.seq * sh.hidden * 2 * sh.kvh * sh.head_dim
+            tf = kf / (kv_ms * 1e-3) / 1e12
+            rooflines["kv_project_cache"] = {"bound": "tensor",
+                                             "kernel": "count pass + ag_kv_project_cache (not part of the step)",
+                                             "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                             "frac": tf / peaks["bf16_tflops"], "traffic": None,
+                                             "peak_source": peaks["source"], "algorithmic_flops": kf, "ms": kv_ms}
     for k, r in rooflines.items():
         r["traffic"] = TRAFFIC.get((args.workload, k))
     head = "prefill" if run.has_prefill else "decode"

@@ -7,7 +7,9 @@
 // turns flags into prefix stays.
 //
 // One CTA computes MT sub-tiles of 128 tokens x BN columns of the packed output [K | V]; a tile
-// lies in one weight and covers BN / 128 whole heads.  Warp 0 drives TMA, warp 1 owns tensor
+// lies in one weight and covers BN / 128 whole heads.  With MT = 2 the tiles of a last wave that
+// would fill at most half of the SMs go to two CTAs of one sub-tile each, so that the wave ends
+// in half the time.  Warp 0 drives TMA, warp 1 owns tensor
 // memory and issues the MMAs, warps 2..5 drain the accumulator.  Main loop as in the gate's
 // projection GEMM (A = X K-major, B = W MN-major panels of [64 k][64 n], 128-byte swizzle).
 // Epilogue per sub-tile: the destination rows of its tokens are looked up while the MMAs run;
@@ -24,6 +26,7 @@ using namespace umma;
 namespace {
 
 constexpr int kBM = 128, kBK = 64, kThreads = 192, kD = 128;
+constexpr int kBandTiles = 16;   // row tiles per band of the tile order
 
 template <int BN, int MT> struct KvCfg {
   static constexpr int kStages = BN == 256 ? (MT == 2 ? 3 : 4) : 6;
@@ -44,7 +47,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                      const int32_t *__restrict__ prefix, const int64_t *__restrict__ row_off,
                      const int32_t *__restrict__ cap, int32_t *__restrict__ len, uint8_t *__restrict__ k_rows,
                      uint8_t *__restrict__ v_rows, int32_t *__restrict__ dev_status, int M, int Kdim, int GD,
-                     int n, int kv_heads, int n_tiles_n) {
+                     int n, int kv_heads, int n_tiles_m, int n_tiles_n, int split_from) {
   using Cfg = KvCfg<BN, MT>;
   constexpr uint32_t kTmemCols = MT * BN;
   static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "TMEM columns: a power of two");
@@ -58,9 +61,18 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   long long *dst_row = reinterpret_cast<long long *>(smem + Cfg::kStages * Cfg::kStageBytes + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x;
-  const int m0 = (tile / n_tiles_n) * (MT * kBM);
-  const int n0 = (tile % n_tiles_n) * BN;        // in the packed [2 * GD] output
+  // CTAs below split_from take whole tiles (row-major over the tile grid), the rest one sub-tile of a tile
+  const int cta = blockIdx.x;
+  const bool single = MT > 1 && cta >= split_from;
+  const int tile = single ? split_from + ((cta - split_from) >> 1) : cta;
+  const int mts = single ? 1 : MT;               // sub-tiles of this CTA
+  // tile order: bands of kBandTiles row tiles; inside a band the row tile runs fastest, so the CTAs in
+  // flight share a few column slices of W while the band's rows of X stay in L2
+  const int band = tile / (kBandTiles * n_tiles_n), in_band = tile % (kBandTiles * n_tiles_n);
+  const int band_rows = min(kBandTiles, n_tiles_m - band * kBandTiles);
+  const int tile_m = band * kBandTiles + in_band % band_rows, tile_n = in_band / band_rows;
+  const int m0 = tile_m * (MT * kBM) + (single ? ((cta - split_from) & 1) * kBM : 0);
+  const int n0 = tile_n * BN;                    // in the packed [2 * GD] output
   const int which = n0 / GD, nw = n0 % GD;       // BN divides GD: a tile lies in one weight
   const CUtensorMap *tmB = which == 0 ? &tmBk : &tmBv;
   const int num_kb = (Kdim + kBK - 1) / kBK;
@@ -88,10 +100,10 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const uint32_t ph = (kb / Cfg::kStages) & 1;
         if (!mbar_wait(&empty[s], ph ^ 1)) break;
         uint8_t *a = smem + s * Cfg::kStageBytes, *b = a + Cfg::kABytes;
-        mbar_arrive_expect_tx(&full[s], Cfg::kStageBytes);
+        mbar_arrive_expect_tx(&full[s], mts * (kBM * kBK * 2) + Cfg::kBBytes);
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)              // rows past M are filled with zeros
-          tma_load_2d(a + mt * (kBM * kBK * 2), &tmA, &full[s], kb * kBK, m0 + mt * kBM);
+          if (mt < mts) tma_load_2d(a + mt * (kBM * kBK * 2), &tmA, &full[s], kb * kBK, m0 + mt * kBM);
 #pragma unroll
         for (int p = 0; p < BN / 64; ++p)
           tma_load_2d(b + p * Cfg::kPanelBytes, tmB, &full[s], nw + p * 64, kb * kBK);
@@ -117,7 +129,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         for (int k = 0; k < kBK / 16; ++k) {
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt)
-            mma_ss_lohi(tmem_acc + mt * BN, a_lo + ((mt * kBM * kBK * 2 + k * 32) >> 4), a_hi,
+            if (mt < mts) mma_ss_lohi(tmem_acc + mt * BN, a_lo + ((mt * kBM * kBK * 2 + k * 32) >> 4), a_hi,
                         b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
         }
         mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
@@ -140,7 +152,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
       for (int hh = 0; hh < Cfg::kHeads; ++hh) {
         long long d = -1;
-        if (m_base < M) {
+        if (m_base < M && mt < mts) {
           const size_t slab = (size_t)b * kv_heads + nw / kD + hh;
           const int32_t *pre = prefix + slab * (n + 1);
           const int total = pre[n];
@@ -162,7 +174,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll 1
     for (int mt = 0; mt < MT; ++mt) {
       const int m_base = m0 + mt * kBM;
-      if (!ok || num_kb == 0 || m_base >= M) break;
+      if (!ok || num_kb == 0 || m_base >= M || mt >= mts) break;
       const uint32_t tmem_sub = tmem_acc + mt * BN;
       // bf16 tile as panels of [128 tokens][64 columns] (128-byte rows, 16-byte chunks XOR-swizzled by the row)
 #pragma unroll 1
@@ -203,7 +215,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           }
         }
       }
-      if (MT > 1) {
+      if (mt + 1 < mts) {
         if (threadIdx.x == 64) tma_store_wait_read();
         named_barrier_sync(1, 128);          // the staging area is free for the next sub-tile
       }
@@ -243,10 +255,13 @@ int run(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, c
   if (rc) return rc;
   auto kern = kv_proj_cache_kernel<BN, MT>;
   AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-  const int n_tiles_n = 2 * GD / BN, n_tiles = n_tiles_n * ((M + MT * kBM - 1) / (MT * kBM));
-  kern<<<n_tiles, kThreads, Cfg::kSmemBytes, st>>>(tmA, tmBk, tmBv, tmK, tmV, flags, prefix, c.row_off, c.cap, c.len,
+  const int n_tiles_n = 2 * GD / BN, n_tiles_m = (M + MT * kBM - 1) / (MT * kBM), n_tiles = n_tiles_n * n_tiles_m;
+  const int tail = n_tiles % sm_count();
+  const int split_from = (MT > 1 && tail > 0 && 2 * tail <= sm_count()) ? n_tiles - tail : n_tiles;
+  const int ctas = split_from + 2 * (n_tiles - split_from);
+  kern<<<ctas, kThreads, Cfg::kSmemBytes, st>>>(tmA, tmBk, tmBv, tmK, tmV, flags, prefix, c.row_off, c.cap, c.len,
                                                    static_cast<uint8_t *>(c.k_rows), static_cast<uint8_t *>(c.v_rows),
-                                                   dev_status, M, Kdim, GD, d.seq, hk, n_tiles_n);
+                                                   dev_status, M, Kdim, GD, d.seq, hk, n_tiles_m, n_tiles_n, split_from);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }

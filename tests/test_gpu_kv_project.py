@@ -109,6 +109,8 @@ CASES = {
     "two_subtiles": LayerShape(1, 1280, 256, 16, 128, 2, 128, "bf16"),         # 256-token tiles
     "two_subtiles_odd_rows": LayerShape(1, 1152, 192, 18, 128, 2, 128, "bf16"),  # last tile has one sub-tile
     "subtiles_of_two_sequences": LayerShape(3, 384, 128, 20, 128, 2, 128, "bf16"),
+    "split_last_wave": LayerShape(1, 2560, 128, 16, 128, 2, 128, "bf16"),      # 160 tiles on 148 SMs: 12 are split
+    "split_last_wave_odd_rows": LayerShape(1, 2432, 128, 16, 128, 2, 128, "bf16"),
     "grouped_query": LayerShape(2, 256, 256, 8, 128, 2, 128, "bf16", kv_heads=2),
 }
 
