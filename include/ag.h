@@ -205,34 +205,36 @@ int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
                   void *cuda_stream);
 
 /*
- * Steps "project" + 2 in one call — the key/value projection of Eq. 2,
+ * Step 2 fused with the projection that feeds it — the key/value projection of Eq. 2,
  *   K_i = X W^K_i,  V_i = X W^V_i      (head i = columns [i D, (i + 1) D) of the weight),
- * fused with selective caching (Sec. 3.3: k_i^(t), v_i^(t) are retained iff
- * AG(X)_i^(t) = 1).  Each projected tile is rounded to the layer dtype once and
- * written to both places the layer reads it from: the dense K, V (every token
- * attends to its own key and value, the diagonal of Eq. 5) and, for retained
- * tokens, cache row row_off[s] + prefix[s, t].  It replaces the copying pass of
- * ag_compact_kv: the order of calls is gate -> ag_compact_kv with K = V = NULL
- * (flags -> prefix, idx) -> this call -> ag_prefill_attn.
+ * and selective caching (Sec. 3.3: k_i^(t), v_i^(t) are retained iff
+ * AG(X)_i^(t) = 1) in one call.  Each projected tile is rounded to the layer
+ * dtype once and written to both places the layer reads it from: the dense K, V
+ * (every token attends to its own key and value, the diagonal of Eq. 5) and,
+ * for retained tokens, cache row row_off[s] + prefix[s, t].  prefix, idx and
+ * len are computed from the flags as ag_compact_kv computes them.  A layer that
+ * owns its key/value projection calls gate -> this call -> ag_prefill_attn, and
+ * ag_compact_kv not at all.
  *
  *   X       [B, n, d]             in
  *   Wk, Wv  [d, h D]              in   ("in x out")
  *   flags   [B, h, n] uint8       in
- *   prefix  [B, h, n + 1] int32   in   (as the count pass wrote it)
- *   cache   host struct           in/out: k_rows, v_rows of the retained tokens, len[s] = prefix[s, n]
+ *   cache   host struct           in/out: k_rows, v_rows of the retained tokens, len[s] = L_s
+ *   prefix  [B, h, n + 1] int32   out  exclusive counts of the flags, prefix[s, n] = L_s
+ *   idx     [B, h, n] int32 or NULL  out  (entries r >= L_s are left untouched)
  *   K, V    [B, h, n, D]          out  dense projections (h = kv_heads for grouped-query attention)
  *   dev_status  int32 or NULL     in/out
- * A slab with prefix[s, n] > cap[s] gets no rows, len[s] = 0 and AG_DEV_OVERFLOW,
- * as in ag_compact_kv.  The cache rows are bit copies of the dense K, V rows.
+ * A slab with L_s > cap[s] gets no rows, len[s] = 0 and AG_DEV_OVERFLOW, as in
+ * ag_compact_kv.  The cache rows are bit copies of the dense K, V rows.
  * Needs no workspace.  Kernel coverage: bfloat16, head_dim 128, n a multiple of
  * 128, d a multiple of 8, no recent-token window; anything else returns
  * AG_ERR_UNSUPPORTED (project with a GEMM of your own and call ag_compact_kv).
  * AG_ERR_INVALID_ARG for missing or misaligned (16-byte) pointers.
  */
 int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk,
-                        const void *Wv, const uint8_t *flags, const int32_t *prefix,
-                        ag_cache *cache, void *K, void *V, int32_t *dev_status,
-                        void *cuda_stream);
+                        const void *Wv, const uint8_t *flags, ag_cache *cache,
+                        int32_t *prefix, int32_t *idx, void *K, void *V,
+                        int32_t *dev_status, void *cuda_stream);
 
 /*
  * Step 3 — prefill attention under the eviction mask (Eq. 2 with Eq. 5):

@@ -75,7 +75,7 @@ def lib():
         L.ag_compact_kv.restype = i32
         L.ag_compact_kv.argtypes = [dp, vp, vp, vp, cp, vp, vp, vp, vp, sz, vp]
         L.ag_kv_project_cache.restype = i32
-        L.ag_kv_project_cache.argtypes = [dp, vp, vp, vp, vp, vp, cp, vp, vp, vp, vp]
+        L.ag_kv_project_cache.argtypes = [dp, vp, vp, vp, vp, cp, vp, vp, vp, vp, vp, vp]
         L.ag_prefill_attn.restype = i32
         L.ag_prefill_attn.argtypes = [dp, vp, vp, vp, vp, cp, vp, f32, vp, vp, sz, vp]
         L.ag_decode_attn.restype = i32
@@ -207,9 +207,9 @@ def ag_compact_kv(desc, K, V, flags, cache, prefix, idx, dev_status, ws, stream=
                                       _ptr(dev_status), p, nbytes, _stream(stream)), "ag_compact_kv")
 
 
-def ag_kv_project_cache(desc, X, Wk, Wv, flags, prefix, cache, K, V, dev_status, stream=None):
+def ag_kv_project_cache(desc, X, Wk, Wv, flags, cache, prefix, idx, K, V, dev_status, stream=None):
     return _check(lib().ag_kv_project_cache(ctypes.byref(desc), _ptr(X), _ptr(Wk), _ptr(Wv), _ptr(flags),
-                                            _ptr(prefix), ctypes.byref(cache.struct), _ptr(K), _ptr(V),
+                                            ctypes.byref(cache.struct), _ptr(prefix), _ptr(idx), _ptr(K), _ptr(V),
                                             _ptr(dev_status), _stream(stream)), "ag_kv_project_cache")
 
 

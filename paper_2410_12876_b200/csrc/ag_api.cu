@@ -128,7 +128,7 @@ int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
 }
 
 int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk, const void *Wv,
-                        const uint8_t *flags, const int32_t *prefix, ag_cache *cache, void *K, void *V,
+                        const uint8_t *flags, ag_cache *cache, int32_t *prefix, int32_t *idx, void *K, void *V,
                         int32_t *dev_status, void *cuda_stream) {
   int st = check_desc(desc);
   if (st) return st;
@@ -137,10 +137,10 @@ int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk
   st = check_cache(cache);
   if (st) return st;
   if (misaligned16(X) || misaligned16(Wk) || misaligned16(Wv) || misaligned16(K) || misaligned16(V) ||
-      misaligned16(prefix))
+      misaligned16(flags) || misaligned16(prefix) || misaligned16(idx))
     return AG_ERR_INVALID_ARG;
   if (!kv_proj_cache_supported(*desc)) return AG_ERR_UNSUPPORTED;
-  return launch_kv_proj_cache(*desc, X, Wk, Wv, flags, prefix, *cache, K, V, dev_status,
+  return launch_kv_proj_cache(*desc, X, Wk, Wv, flags, *cache, prefix, idx, K, V, dev_status,
                               (cudaStream_t)cuda_stream);
 }
 

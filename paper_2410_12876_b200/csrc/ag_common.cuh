@@ -85,7 +85,7 @@ int launch_compact(const ag_layer_desc &d, const void *K, const void *V, const u
 // ragged cache (bf16, head_dim 128, seq a multiple of 128).
 bool kv_proj_cache_supported(const ag_layer_desc &d);
 int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, const uint8_t *flags,
-                         const int32_t *prefix, const ag_cache &c, void *K, void *V, int32_t *dev_status,
+                         const ag_cache &c, int32_t *prefix, int32_t *idx, void *K, void *V, int32_t *dev_status,
                          cudaStream_t st);
 int kv_proj_cache_wait_timeouts();
 

@@ -2,9 +2,9 @@
 // 5th-generation tensor cores, with an epilogue that rounds each tile to bf16 once and sends it
 // to both places the layer reads it from: the dense K, V [B, h, n, D] (every token attends to its
 // own key, the diagonal of Eq. 5) and, for the tokens the gate retains (Sec. 3.3: k, v are kept
-// iff AG = 1), row row_off[s] + prefix[s, t] of the ragged cache.  The separate compaction pass
-// over K and V (a read of the retained rows and a launch) disappears; only the count pass that
-// turns flags into prefix stays.
+// iff AG = 1), row row_off[s] + prefix[s, t] of the ragged cache.  The compaction pass over K and
+// V (a read of the retained rows and a launch) disappears: the ranks prefix[s, t] are counted
+// from the flags by the epilogue warps while the MMAs run.
 //
 // One CTA computes MT sub-tiles of 128 tokens x BN columns of the packed output [K | V]; a tile
 // lies in one weight and covers BN / 128 whole heads.  With MT = 2 the tiles of a last wave that
@@ -12,7 +12,7 @@
 // in half the time.  Warp 0 drives TMA, warp 1 owns tensor
 // memory and issues the MMAs, warps 2..5 drain the accumulator.  Main loop as in the gate's
 // projection GEMM (A = X K-major, B = W MN-major panels of [64 k][64 n], 128-byte swizzle).
-// Epilogue per sub-tile: the destination rows of its tokens are looked up while the MMAs run;
+// Epilogue per sub-tile: the destination rows of its tokens are computed while the MMAs run;
 // the tile is staged as bf16 over the (by then free) operand stages in the layout of a swizzled
 // TMA store, the dense copy leaves by TMA stores, and the retained rows are copied from the
 // same staging area, one 256-byte row per half-warp.
@@ -28,6 +28,9 @@ namespace {
 constexpr int kBM = 128, kBK = 64, kThreads = 192, kD = 128;
 constexpr int kBandTiles = 16;   // row tiles per band of the tile order
 
+// Bytes of a 32-bit word that are not zero.
+__device__ __forceinline__ int nonzero_bytes(uint32_t w) { return __popc(__vcmpne4(w, 0u) & 0x01010101u); }
+
 template <int BN, int MT> struct KvCfg {
   static constexpr int kStages = BN == 256 ? (MT == 2 ? 3 : 4) : 6;
   static constexpr int kABytes = MT * kBM * kBK * 2;
@@ -36,7 +39,7 @@ template <int BN, int MT> struct KvCfg {
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kHeads = BN / kD;                     // heads per tile
   static constexpr int kDstBytes = MT * kHeads * kBM * 8;    // destination row of every (sub-tile, head, token)
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + kDstBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + kDstBytes + 64 /*counts*/;
 };
 
 template <int BN, int MT>
@@ -44,7 +47,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBk,
                      const __grid_constant__ CUtensorMap tmBv, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, const uint8_t *__restrict__ flags,
-                     const int32_t *__restrict__ prefix, const int64_t *__restrict__ row_off,
+                     int32_t *__restrict__ prefix, int32_t *__restrict__ idx, const int64_t *__restrict__ row_off,
                      const int32_t *__restrict__ cap, int32_t *__restrict__ len, uint8_t *__restrict__ k_rows,
                      uint8_t *__restrict__ v_rows, int32_t *__restrict__ dev_status, int M, int Kdim, int GD,
                      int n, int kv_heads, int n_tiles_m, int n_tiles_n, int split_from) {
@@ -59,6 +62,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   uint64_t *acc_full = empty + Cfg::kStages;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
   long long *dst_row = reinterpret_cast<long long *>(smem + Cfg::kStages * Cfg::kStageBytes + 256);
+  int *red = reinterpret_cast<int *>(smem + Cfg::kStages * Cfg::kStageBytes + 256 + Cfg::kDstBytes);   // 12 ints
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // CTAs below split_from take whole tiles (row-major over the tile grid), the rest one sub-tile of a tile
@@ -142,25 +146,57 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     // epilogue warps: warp w may touch TMEM lanes [32 * (w % 4), +32)
     const int quad = warp & 3;
     const int r_in = quad * 32 + lane;           // token of the sub-tile this thread drains
-    // Where each token of the tile goes in the ragged cache (-1: evicted, or its slab is too small),
-    // looked up while the MMAs run.  The CTAs of the key tiles that hold a sequence's first token
-    // also set the slab's length.
+    // While the MMAs run: the rank of every token of the tile among the retained tokens of its slab
+    // (the slab's flag row is a few KB: counted whole, as 16-byte vectors, for the number retained
+    // before the tile and in the slab; the tile's own tokens ranked by warp ballot + popc), hence its
+    // row in the ragged cache (-1: evicted, or the slab is too small).  The key tiles also write
+    // prefix (and idx), and the one that holds a sequence's first token the slab's length.
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
       const int m_base = m0 + mt * kBM;
-      const int b = m_base / n, t = m_base % n + r_in;      // n is a multiple of 128: one sequence per sub-tile
+      const int b = m_base / n, t0 = m_base % n, t = t0 + r_in;   // n is a multiple of 128: one sequence per sub-tile
 #pragma unroll
       for (int hh = 0; hh < Cfg::kHeads; ++hh) {
         long long d = -1;
-        if (m_base < M && mt < mts) {
+        if (m_base < M && mt < mts) {                             // the same for all 128 threads
           const size_t slab = (size_t)b * kv_heads + nw / kD + hh;
-          const int32_t *pre = prefix + slab * (n + 1);
-          const int total = pre[n];
+          const uint8_t *f = flags + slab * n;
+          const uint4 *fv = reinterpret_cast<const uint4 *>(f);
+          int before = 0, total = 0;
+          for (int x = r_in; x < n / 16; x += kBM) {
+            const uint4 w = ldg128(fv + x);
+            const int c = nonzero_bytes(w.x) + nonzero_bytes(w.y) + nonzero_bytes(w.z) + nonzero_bytes(w.w);
+            total += c;
+            if (x * 16 < t0) before += c;                         // t0 is a multiple of 16: a vector lies on one side
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            before += __shfl_xor_sync(0xffffffffu, before, o);
+            total += __shfl_xor_sync(0xffffffffu, total, o);
+          }
+          const bool keep = f[t] != 0;
+          const unsigned word = __ballot_sync(0xffffffffu, keep);
+          const int in_warp = __popc(word & ((1u << lane) - 1u));
+          if (lane == 0) { red[quad] = before; red[4 + quad] = total; red[8 + quad] = __popc(word); }
+          named_barrier_sync(2, 128);
+          before = red[0] + red[1] + red[2] + red[3];
+          total = red[4] + red[5] + red[6] + red[7];
+          int excl = 0;
+#pragma unroll
+          for (int q = 0; q < 3; ++q) excl += q < quad ? red[8 + q] : 0;
+          named_barrier_sync(2, 128);                             // red is free for the next head
+          const int p = before + excl + in_warp;                  // rank within the slab
           const bool fits = total <= cap[slab];
-          if (fits && flags[slab * n + t] != 0) d = row_off[slab] + pre[t];
-          if (t == 0 && which == 0) {
-            len[slab] = fits ? total : 0;
-            if (!fits && dev_status) atomicOr(dev_status, AG_DEV_OVERFLOW);
+          if (fits && keep) d = row_off[slab] + p;
+          if (which == 0) {
+            int32_t *pre = prefix + slab * (n + 1);
+            pre[t] = p;
+            if (keep && idx) idx[slab * n + p] = t;
+            if (t == 0) {
+              pre[n] = total;
+              len[slab] = fits ? total : 0;
+              if (!fits && dev_status) atomicOr(dev_status, AG_DEV_OVERFLOW);
+            }
           }
         }
         dst_row[(mt * Cfg::kHeads + hh) * kBM + r_in] = d;
@@ -239,7 +275,7 @@ int sm_count() {
 
 template <int BN, int MT>
 int run(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, const uint8_t *flags,
-        const int32_t *prefix, const ag_cache &c, void *K, void *V, int32_t *dev_status, cudaStream_t st) {
+        const ag_cache &c, int32_t *prefix, int32_t *idx, void *K, void *V, int32_t *dev_status, cudaStream_t st) {
   using Cfg = KvCfg<BN, MT>;
   const int hk = kv_heads_of(d), GD = hk * kD, M = d.batch * d.seq, Kdim = d.hidden;
   CUtensorMap tmA, tmBk, tmBv, tmK, tmV;
@@ -259,7 +295,7 @@ int run(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, c
   const int tail = n_tiles % sm_count();
   const int split_from = (MT > 1 && tail > 0 && 2 * tail <= sm_count()) ? n_tiles - tail : n_tiles;
   const int ctas = split_from + 2 * (n_tiles - split_from);
-  kern<<<ctas, kThreads, Cfg::kSmemBytes, st>>>(tmA, tmBk, tmBv, tmK, tmV, flags, prefix, c.row_off, c.cap, c.len,
+  kern<<<ctas, kThreads, Cfg::kSmemBytes, st>>>(tmA, tmBk, tmBv, tmK, tmV, flags, prefix, idx, c.row_off, c.cap, c.len,
                                                    static_cast<uint8_t *>(c.k_rows), static_cast<uint8_t *>(c.v_rows),
                                                    dev_status, M, Kdim, GD, d.seq, hk, n_tiles_m, n_tiles_n, split_from);
   AG_LAUNCH_CHECK();
@@ -274,16 +310,16 @@ bool kv_proj_cache_supported(const ag_layer_desc &d) {
 }
 
 int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, const uint8_t *flags,
-                         const int32_t *prefix, const ag_cache &c, void *K, void *V, int32_t *dev_status,
+                         const ag_cache &c, int32_t *prefix, int32_t *idx, void *K, void *V, int32_t *dev_status,
                          cudaStream_t st) {
   const int hk = kv_heads_of(d);
   const long long tiles128 = (long long)(2 * hk * kD / 128) * (d.batch * (long long)d.seq / kBM);
   if (hk % 2 == 0) {
     // more than one wave: 256-token tiles, whose two sub-tiles share every stage of W
-    if (tiles128 > 2 * sm_count()) return run<256, 2>(d, X, Wk, Wv, flags, prefix, c, K, V, dev_status, st);
-    return run<256, 1>(d, X, Wk, Wv, flags, prefix, c, K, V, dev_status, st);
+    if (tiles128 > 2 * sm_count()) return run<256, 2>(d, X, Wk, Wv, flags, c, prefix, idx, K, V, dev_status, st);
+    return run<256, 1>(d, X, Wk, Wv, flags, c, prefix, idx, K, V, dev_status, st);
   }
-  return run<128, 1>(d, X, Wk, Wv, flags, prefix, c, K, V, dev_status, st);
+  return run<128, 1>(d, X, Wk, Wv, flags, c, prefix, idx, K, V, dev_status, st);
 }
 
 int kv_proj_cache_wait_timeouts() {

@@ -49,7 +49,7 @@ def _flags(shape, seed):
 
 
 def gpu_project_cache(shape, X, W, flags, cap=None):
-    """Count pass (flags -> prefix, idx), then the fused projection."""
+    """The fused projection on buffers that hold nothing of a previous call."""
     desc = ag.make_desc(shape)
     B, h, n, D = shape.batch, shape.kvh, shape.seq, shape.head_dim
     if cap is None:
@@ -58,11 +58,10 @@ def gpu_project_cache(shape, X, W, flags, cap=None):
     prefix = torch.full((B, h, n + 1), -1, dtype=torch.int32, device=DEV)
     idx = torch.full((B, h, n), -1, dtype=torch.int32, device=DEV)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    ag.ag_compact_kv(desc, None, None, flags, cache, prefix, idx, status, None)
-    cache.len.fill_(-7)                                    # the fused call sets the lengths itself
+    cache.len.fill_(-7)                                    # the call sets the lengths itself
     K = torch.full((B, h, n, D), float("nan"), dtype=torch.bfloat16, device=DEV)
     V = torch.full_like(K, float("nan"))
-    ag.ag_kv_project_cache(desc, X, W["Wk"], W["Wv"], flags, prefix, cache, K, V, status)
+    ag.ag_kv_project_cache(desc, X, W["Wk"], W["Wv"], flags, cache, prefix, idx, K, V, status)
     torch.cuda.synchronize()
     return cache, prefix, idx, status, K, V
 
@@ -84,10 +83,13 @@ def _check(shape, seed, cap=None):
     kd, vd = T.bits(K), T.bits(V)
     kr, vr = T.bits(cache.k_rows), T.bits(cache.v_rows)
     off = cache.row_off.cpu().numpy()
+    pre, ix = prefix.cpu().numpy(), idx.cpu().numpy()
     for b in range(shape.batch):
         for i in range(shape.kvh):
             s = b * shape.kvh + i
             pos = ocache[b][i]["idx"]                      # the oracle's retained positions
+            assert np.array_equal(pre[b, i], orc.exclusive_counts(fl[b, i])), (b, i)
+            assert np.array_equal(ix[b, i, :L[s]], pos) and np.all(ix[b, i, L[s]:] == -1), (b, i)
             if fits[s]:
                 assert np.array_equal(kr[off[s]:off[s] + L[s]], kd[b, i][pos]), (b, i)
                 assert np.array_equal(vr[off[s]:off[s] + L[s]], vd[b, i][pos]), (b, i)
@@ -129,7 +131,7 @@ def test_slab_too_small_is_skipped_and_reported():
 
 
 def test_feeds_prefill_and_decode():
-    """gate flags -> count pass -> fused projection -> prefill attention and a decode step, against the
+    """flags -> fused projection -> prefill attention and a decode step, against the
     oracle run on the projected K, V the library wrote."""
     shape = LayerShape(1, 512, 512, 4, 128, 2, 128, "bf16")
     cache, prefix, K, V, fl = _check(shape, 920)
@@ -158,6 +160,8 @@ def test_full_size_layer_sampled():
     assert int(status.item()) == 0
     L = fl.sum(axis=2, dtype=np.int64).reshape(-1)
     assert np.array_equal(cache.len.cpu().numpy(), L)
+    want = np.concatenate([np.zeros((1, shape.heads, 1), dtype=np.int64), np.cumsum(fl, axis=2, dtype=np.int64)], axis=2)
+    assert np.array_equal(prefix.cpu().numpy(), want)
     Xf, Wk, Wv = T.f64(X)[0], T.f64(W["Wk"]), T.f64(W["Wv"])
     rng = np.random.default_rng(931)
     D = shape.head_dim
@@ -183,8 +187,8 @@ def test_rejects_what_it_has_no_kernel_for():
     for bad in (shape.with_(seq=200), shape.with_(head_dim=64), shape.with_(dtype="f32"), shape.with_(hidden=516),
                 shape.with_(recent_window=5)):
         with pytest.raises(ag.AgError) as e:
-            ag.ag_kv_project_cache(ag.make_desc(bad), X, W["Wk"], W["Wv"], flags, prefix, cache, K, V, status)
+            ag.ag_kv_project_cache(ag.make_desc(bad), X, W["Wk"], W["Wv"], flags, cache, prefix, idx, K, V, status)
         assert e.value.status in (ag.AG_ERR_UNSUPPORTED, ag.AG_ERR_INVALID_ARG)
     with pytest.raises(ag.AgError) as e:
-        ag.ag_kv_project_cache(ag.make_desc(shape), X, W["Wk"], None, flags, prefix, cache, K, V, status)
+        ag.ag_kv_project_cache(ag.make_desc(shape), X, W["Wk"], None, flags, cache, prefix, idx, K, V, status)
     assert e.value.status == ag.AG_ERR_INVALID_ARG
