@@ -10,7 +10,7 @@
 // lies in one weight and covers BN / 128 whole heads.  With MT = 2 the tiles of a last wave that
 // would fill at most half of the SMs go to two CTAs of one sub-tile each, so that the wave ends
 // in half the time.  Warp 0 drives TMA, warp 1 owns tensor
-// memory and issues the MMAs, warps 2..5 drain the accumulator.  Main loop as in the gate's
+// memory and issues the MMAs, warps 2..9 drain the accumulator (two per quarter of its lanes).  Main loop as in the gate's
 // projection GEMM (A = X K-major, B = W MN-major panels of [64 k][64 n], 128-byte swizzle).
 // Epilogue per sub-tile: the destination rows of its tokens are computed while the MMAs run;
 // the tile is staged as bf16 over the (by then free) operand stages in the layout of a swizzled
@@ -25,7 +25,7 @@ using namespace umma;
 
 namespace {
 
-constexpr int kBM = 128, kBK = 64, kThreads = 192, kD = 128;
+constexpr int kBM = 128, kBK = 64, kThreads = 320, kD = 128;   // warps: TMA, MMA, 8 x epilogue
 constexpr int kBandTiles = 16;   // row tiles per band of the tile order
 
 // Bytes of a 32-bit word that are not zero.
@@ -54,7 +54,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   using Cfg = KvCfg<BN, MT>;
   constexpr uint32_t kTmemCols = MT * BN;
   static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "TMEM columns: a power of two");
-  static_assert((BN / 64) * kBM * 128 <= Cfg::kStages * Cfg::kStageBytes, "staging fits the stages");
+  static_assert(MT * (BN / 64) * kBM * 128 <= Cfg::kStages * Cfg::kStageBytes, "staging fits the stages");
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t *full = reinterpret_cast<uint64_t *>(smem + Cfg::kStages * Cfg::kStageBytes);
@@ -143,8 +143,9 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     if (elect_one()) mma_commit(acc_full);   // accumulator complete (or unwinding)
     __syncwarp();
   } else {
-    // epilogue warps: warp w may touch TMEM lanes [32 * (w % 4), +32)
-    const int quad = warp & 3;
+    // epilogue warps: warp w may touch TMEM lanes [32 * (w % 4), +32); warps 2..5 drain the first
+    // half of a sub-tile's columns, warps 6..9 the second
+    const int quad = warp & 3, half = (warp - 2) >> 2;
     const int r_in = quad * 32 + lane;           // token of the sub-tile this thread drains
     // While the MMAs run: the rank of every token of the tile among the retained tokens of its slab
     // (the slab's flag row is a few KB: counted whole, as 16-byte vectors, for the number retained
@@ -152,7 +153,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     // row in the ragged cache (-1: evicted, or the slab is too small).  The key tiles also write
     // prefix (and idx), and the one that holds a sequence's first token the slab's length.
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
+    for (int mt = 0; mt < (half == 0 ? MT : 0); ++mt) {           // warps 2..5 only
       const int m_base = m0 + mt * kBM;
       const int b = m_base / n, t0 = m_base % n, t = t0 + r_in;   // n is a multiple of 128: one sequence per sub-tile
 #pragma unroll
@@ -206,15 +207,17 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     tc_fence_after_sync();
     const CUtensorMap *tmOut = which == 0 ? &tmK : &tmV;
     uint8_t *rows_out = which == 0 ? k_rows : v_rows;
-    const int hw = (warp - 2) * 2 + (lane >> 4), l16 = lane & 15;   // half-warp 0..7, 16-byte piece of a row
+    const int hw = (warp - 2) * 2 + (lane >> 4), l16 = lane & 15;   // half-warp 0..15, 16-byte piece of a row
 #pragma unroll 1
     for (int mt = 0; mt < MT; ++mt) {
       const int m_base = m0 + mt * kBM;
       if (!ok || num_kb == 0 || m_base >= M || mt >= mts) break;
       const uint32_t tmem_sub = tmem_acc + mt * BN;
-      // bf16 tile as panels of [128 tokens][64 columns] (128-byte rows, 16-byte chunks XOR-swizzled by the row)
+      // bf16 tile as panels of [128 tokens][64 columns] (128-byte rows, 16-byte chunks XOR-swizzled by the
+      // row); each sub-tile has a staging area of its own, so the second is drained while the first leaves
+      uint8_t *stg = smem + mt * (BN / 64) * kBM * 128;
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
         uint32_t r[32];
         tmem_ld_x32_sync(tmem_sub + ((uint32_t)(quad * 32) << 16) + c, r);
         const uint32_t panel = (uint32_t)(c >> 6) * kBM * 128 + r_in * 128;
@@ -225,16 +228,16 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           for (int q = 0; q < 8; q += 2)
             h[q >> 1] = pack_bf16x2(__uint_as_float(r[e + q]), __uint_as_float(r[e + q + 1]));
           const uint32_t chunk = (uint32_t)(((c & 32) >> 3) + (e >> 3));
-          *reinterpret_cast<uint4 *>(smem + panel + ((chunk ^ (r_in & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
+          *reinterpret_cast<uint4 *>(stg + panel + ((chunk ^ (r_in & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
         }
       }
       fence_proxy_async_smem();
-      named_barrier_sync(1, 128);
+      named_barrier_sync(1, 256);                  // the tile is staged (and dst_row written, first time round)
       const int b = m_base / n, t0 = m_base % n;
       if (threadIdx.x == 64) {
 #pragma unroll
         for (int p = 0; p < BN / 64; ++p)
-          tma_store_3d(tmOut, smem + p * kBM * 128, (p & 1) * 64, t0, b * kv_heads + nw / kD + (p >> 1));
+          tma_store_3d(tmOut, stg + p * kBM * 128, (p & 1) * 64, t0, b * kv_heads + nw / kD + (p >> 1));
         tma_store_commit();
       }
       // retained rows: half-warp per row, 16 bytes per lane
@@ -242,18 +245,14 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       for (int hh = 0; hh < Cfg::kHeads; ++hh) {
         const long long *dr = dst_row + (mt * Cfg::kHeads + hh) * kBM;
 #pragma unroll 4
-        for (int r = hw; r < kBM; r += 8) {
+        for (int r = hw; r < kBM; r += 16) {
           const long long d = dr[r];
           if (d >= 0) {
             const uint32_t off = (uint32_t)(hh * 2 + (l16 >> 3)) * kBM * 128 + r * 128 + (((l16 & 7) ^ (r & 7)) << 4);
             *reinterpret_cast<uint4 *>(rows_out + (size_t)d * (kD * 2) + l16 * 16) =
-                *reinterpret_cast<const uint4 *>(smem + off);
+                *reinterpret_cast<const uint4 *>(stg + off);
           }
         }
-      }
-      if (mt + 1 < mts) {
-        if (threadIdx.x == 64) tma_store_wait_read();
-        named_barrier_sync(1, 128);          // the staging area is free for the next sub-tile
       }
     }
     if (threadIdx.x == 64) tma_store_wait_read();
