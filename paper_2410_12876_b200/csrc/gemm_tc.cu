@@ -2,7 +2,7 @@
 // the accumulator in tensor memory, operands staged by TMA), used for the gate's
 // projection [Q' | K' | V'] = X [Wq_g | Wk_g | Wv_g] (Sec. 3.3, MHA').
 //
-// One CTA computes a 128 x BN tile of the packed output - or, for the tiles of a last wave that
+// One CTA computes MT (1 or 2) sub-tiles of 128 rows x BN columns (BN = 128, 192 or 256) of the packed output - or, for the tiles of a last wave that
 // would fill less than half of the SMs, one half of it (each such tile goes to two CTAs of
 // BN / 2 columns, so that the wave ends in about half the time).  Warp 0 drives TMA,
 // warp 1 owns TMEM and issues the MMAs, warps 2..5 drain the accumulator: the
@@ -23,7 +23,8 @@ constexpr int kTcBM = 128, kTcBK = 64, kTcThreads = 192;
 
 // MT: 128-row sub-tiles of A per CTA (1 or 2; two share every B stage, a third less traffic per FLOP).
 template <int BN, int MT> struct GemmTcCfg {
-  static constexpr int kStages = BN == 256 ? (MT == 2 ? 3 : 4) : 6;
+  static constexpr int kStages = BN == 256 ? (MT == 2 ? 3 : 4) : BN == 192 ? 4 : 6;
+  static constexpr int kAccCols = BN > 128 ? 256 : 128;      // TMEM columns between the sub-tiles' accumulators
   static constexpr int kABytes = MT * kTcBM * kTcBK * 2;     // 16 KB per sub-tile
   static constexpr int kPanelBytes = kTcBK * 64 * 2;         // [64 k][64 n] = 8 KB
   static constexpr int kBBytes = (BN / 64) * kPanelBytes;
@@ -38,7 +39,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const __grid_constant__ CUtensorMap tmChi, const __grid_constant__ CUtensorMap tmClo,
                     float *__restrict__ C, bool split, int M, int K, int GD, int n_tiles_n, int halved_from) {
   using Cfg = GemmTcCfg<BN, MT>;
-  constexpr uint32_t kTmemCols = MT * BN;
+  constexpr uint32_t kTmemCols = MT * Cfg::kAccCols;
   static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "TMEM columns: a power of two");
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -55,8 +56,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int bn = halved ? BN / 2 : BN;         // columns of this CTA (a multiple of 64)
   const int m0 = (tile / n_tiles_n) * (MT * kTcBM);
   const int n0 = (tile % n_tiles_n) * BN + (halved ? ((cta - halved_from) & 1) * (BN / 2) : 0);   // in the packed [3 * GD] output
-  const int which = n0 / GD, nw = n0 % GD;     // BN divides GD: a tile never straddles two weights
-  const CUtensorMap *tmB = which == 0 ? &tmB0 : (which == 1 ? &tmB1 : &tmB2);
+  // a 64-column panel of B lies in one weight (64 divides GD); a tile may straddle two
   const int num_kb = (K + kTcBK - 1) / kTcBK;
 
   if (threadIdx.x == 0) {
@@ -64,7 +64,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     mbar_init(acc_full, 1);
     fence_barrier_init();
     prefetch_tensormap(&tmA);
-    prefetch_tensormap(tmB);
+    prefetch_tensormap(&tmB0);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, kTmemCols);
@@ -86,8 +86,11 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)              // rows past M are filled with zeros
           tma_load_2d(a + mt * (kTcBM * kTcBK * 2), &tmA, &full[s], kb * kTcBK, m0 + mt * kTcBM);
-        for (int p = 0; p < bn / 64; ++p)
-          tma_load_2d(b + p * Cfg::kPanelBytes, tmB, &full[s], nw + p * 64, kb * kTcBK);
+        for (int p = 0; p < bn / 64; ++p) {
+          const int col = n0 + p * 64, which = col / GD;
+          tma_load_2d(b + p * Cfg::kPanelBytes, which == 0 ? &tmB0 : (which == 1 ? &tmB1 : &tmB2), &full[s],
+                      col % GD, kb * kTcBK);
+        }
       }
     }
   } else if (warp == 1) {
@@ -111,7 +114,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           // 16 elements of K: 32 bytes along a K-major row; 16 k-rows (2048 B) of an MN-major panel
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt)
-            mma_ss_lohi(tmem_acc + mt * BN, a_lo + ((mt * kTcBM * kTcBK * 2 + k * 32) >> 4), a_hi,
+            mma_ss_lohi(tmem_acc + mt * Cfg::kAccCols, a_lo + ((mt * kTcBM * kTcBK * 2 + k * 32) >> 4), a_hi,
                         b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
         }
         mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
@@ -128,7 +131,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll 1
     for (int mt = 0; mt < MT; ++mt) {
     const int row = m0 + mt * kTcBM + quad * 32 + lane;
-    const uint32_t tmem_sub = tmem_acc + mt * BN;
+    const uint32_t tmem_sub = tmem_acc + mt * Cfg::kAccCols;
     if (ok && num_kb > 0 && split) {
       // x = hi + lo in bf16 pairs, for consumers that rebuild float32 precision from three
       // products.  Every MMA has completed, so every stage has been read: the tile is staged
@@ -275,7 +278,7 @@ static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void
   // tiles of a last wave that would fill at most half of the SMs are halved
   const int sms = gemm_sm_count();
   const int tail = n_tiles % sms;
-  const int halved_from = (BN >= 128 && tail > 0 && 2 * tail <= sms) ? n_tiles - tail : n_tiles;   // (any MT)
+  const int halved_from = (BN % 128 == 0 && tail > 0 && 2 * tail <= sms) ? n_tiles - tail : n_tiles;   // (any MT)
   const int ctas = halved_from + 2 * (n_tiles - halved_from);
   kern<<<ctas, kTcThreads, Cfg::kSmemBytes, st>>>(tmA, tmB[0], tmB[1], tmB[2], tmC[0], tmC[1], C, Chi != nullptr, M, K,
                                                   GD, n_tiles_n, halved_from);
@@ -285,6 +288,12 @@ static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void
 
 bool gate_proj_tc_supported(int K, int GD) { return GD % 128 == 0 && K % 8 == 0; }
 
+// Rounds of CTAs x columns per tile: what the slowest SM computes, in units of 128 rows x 1 column x MT.
+static long long makespan(long long tiles, int bn) {
+  const int sms = gemm_sm_count();
+  return (tiles + sms - 1) / sms * bn;
+}
+
 int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, void *Chi,
                         void *Clo, int M, int K, int GD, cudaStream_t st) {
   auto hi = static_cast<__nv_bfloat16 *>(Chi), lo = static_cast<__nv_bfloat16 *>(Clo);
@@ -292,7 +301,14 @@ int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const voi
     // more than one wave of 128 x 256 tiles: 256 x 256 tiles, whose two row sub-tiles share every
     // stage of W (a third less operand traffic per FLOP; the kernel is bound by feeding the SMs)
     const long long tiles128 = (long long)(3 * GD / 256) * ((M + kTcBM - 1) / kTcBM);
-    if (tiles128 > gemm_sm_count()) return run_gemm_tc<256, 2>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
+    if (tiles128 > gemm_sm_count()) {
+      // 256-row tiles of 256 or of 192 columns, whichever leaves the slowest SM less to do (the
+      // 7B-shaped layer: 96 tiles of 256 x 256 fill 96 of 148 SMs, 128 tiles of 256 x 192 fill 128)
+      const long long row_tiles = (M + 2 * kTcBM - 1) / (2 * kTcBM);
+      if (makespan(row_tiles * (3 * GD / 192), 192) < makespan(row_tiles * (3 * GD / 256), 256))
+        return run_gemm_tc<192, 2>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
+      return run_gemm_tc<256, 2>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
+    }
     return run_gemm_tc<256, 1>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
   }
   return run_gemm_tc<128, 1>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
