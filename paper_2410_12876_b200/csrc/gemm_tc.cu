@@ -288,12 +288,6 @@ static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void
 
 bool gate_proj_tc_supported(int K, int GD) { return GD % 128 == 0 && K % 8 == 0; }
 
-// Rounds of CTAs x columns per tile: what the slowest SM computes, in units of 128 rows x 1 column x MT.
-static long long makespan(long long tiles, int bn) {
-  const int sms = gemm_sm_count();
-  return (tiles + sms - 1) / sms * bn;
-}
-
 int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, void *Chi,
                         void *Clo, int M, int K, int GD, cudaStream_t st) {
   auto hi = static_cast<__nv_bfloat16 *>(Chi), lo = static_cast<__nv_bfloat16 *>(Clo);
@@ -302,10 +296,11 @@ int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const voi
     // stage of W (a third less operand traffic per FLOP; the kernel is bound by feeding the SMs)
     const long long tiles128 = (long long)(3 * GD / 256) * ((M + kTcBM - 1) / kTcBM);
     if (tiles128 > gemm_sm_count()) {
-      // 256-row tiles of 256 or of 192 columns, whichever leaves the slowest SM less to do (the
-      // 7B-shaped layer: 96 tiles of 256 x 256 fill 96 of 148 SMs, 128 tiles of 256 x 192 fill 128)
+      // one round either way: 192-column tiles put more SMs to work (the 7B-shaped layer: 128 tiles
+      // of 256 x 192 instead of 96 of 256 x 256).  The time of a tile hardly depends on its width (the
+      // operand loads, not the MMAs, set it), so with several rounds the fewer, wider tiles stay.
       const long long row_tiles = (M + 2 * kTcBM - 1) / (2 * kTcBM);
-      if (makespan(row_tiles * (3 * GD / 192), 192) < makespan(row_tiles * (3 * GD / 256), 256))
+      if (GD % 64 == 0 && row_tiles * (3 * GD / 192) <= gemm_sm_count())
         return run_gemm_tc<192, 2>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
       return run_gemm_tc<256, 2>(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
     }
