@@ -48,6 +48,7 @@ TRAFFIC = {
     ("prefill7b", "prefill"): 154.86e6 + 18.50e6,        # prefill_tc_kernel
     ("prefill7b", "decode"): 41.22e6 + 0.01e6,           # decode_cluster_mma_kernel
     ("prefill7b", "compact"): 41.26e6 + 3.10e6,          # compact_kernel<256> (written rows still in L2 at kernel end)
+    ("prefill7b", "kv_project_cache"): 171.96e6 + 80.44e6,   # kv_proj_cache_kernel<256, 2>
     ("decode_ragged", "decode"): 2.3530e9 + 7.1e6,       # decode_partial_kernel<bf16,128>
 }
 # kernels launched per call of the library
@@ -167,6 +168,7 @@ class LayerRun:
         B, h, n, D = sh.batch, sh.heads, sh.seq, sh.head_dim
         self.name = name
         self.use_graph, self.graph = True, None
+        self._groups = {}
         self.has_gate = name in ("prefill7b", "tiny", "stack7b", "stack7b_prev")
         self.layers = 32 if name.startswith("stack7b") else 1
         self.first_gated = 1 if name == "stack7b_prev" else 0      # 0: every layer evicts by its own gate
@@ -248,13 +250,32 @@ class LayerRun:
         ag.ag_kv_project_cache(self.desc, self.X, self.W["Wk"], self.W["Wv"], self.cur_flags, self.cache, self.prefix,
                                None, self.K2, self.V2, self.status)
 
-    def compact(self):
+    def _group(self, g):
+        """Descriptor and cache view of the heads g = (first, last + 1) of a batch-1 layer (the calls
+        of a layer work on any subset of its heads: every (sequence, head) is independent)."""
+        if g not in self._groups:
+            assert self.shape.batch == 1 and self.shape.kv_heads == 0 and self.shape.recent_window <= 1
+            ag, c = self.ag, self.cache
+            view = ag.RaggedCache(c.k_rows, c.v_rows, c.row_off[g[0]:g[1]], c.cap[g[0]:g[1]], c.len[g[0]:g[1]], c.max_cap)
+            self._groups[g] = (ag.make_desc(self.shape.with_(heads=g[1] - g[0])), view)
+        return self._groups[g]
+
+    def compact(self, g=None):
         ag = self.ag
+        if g is not None:
+            desc, cache = self._group(g)
+            return ag.ag_compact_kv(desc, self.K[:, g[0]:g[1]], self.V[:, g[0]:g[1]], self.cur_flags[:, g[0]:g[1]], cache,
+                                    self.prefix[:, g[0]:g[1]], None, self.status, self.ws[ag.AG_CALL_COMPACT])
         ag.ag_compact_kv(self.desc, self.K, self.V, self.cur_flags, self.cache, self.prefix, None, self.status,
                          self.ws[ag.AG_CALL_COMPACT])
 
-    def prefill(self):
+    def prefill(self, g=None):
         ag = self.ag
+        if g is not None:
+            desc, cache = self._group(g)
+            return ag.ag_prefill_attn(desc, self.Q[:, g[0]:g[1]], self.K[:, g[0]:g[1]], self.V[:, g[0]:g[1]],
+                                      self.cur_flags[:, g[0]:g[1]], cache, self.prefix[:, g[0]:g[1]], 0.0,
+                                      self.O[:, g[0]:g[1]], self.ws[ag.AG_CALL_PREFILL])
         ag.ag_prefill_attn(self.desc, self.Q, self.K, self.V, self.cur_flags, self.cache, self.prefix, 0.0, self.O,
                            self.ws[ag.AG_CALL_PREFILL])
 
@@ -453,13 +474,18 @@ def run_ours(args, rank, world, dev):
     d2h = sum(t.numel() * t.element_size() for t in host_out)
     e2e_steps = max(1, min(args.steps, 10))
     # One layer with a gate: the copies run on their own streams, each call waits only for the inputs
-    # it reads (X -> gate; K, V -> compaction; Q -> prefill; the decode tokens -> decode), and the flags
-    # go back to the host while attention runs.  Other workloads: copy in, step, copy out, in order.
+    # it reads (X -> gate; a head group's K, V, Q -> its compaction and prefill; the decode tokens ->
+    # decode), and the flags and each group's O go back to the host while later groups come in.
+    # Other workloads: copy in, step, copy out, in order.
     overlap = run.has_gate and run.has_prefill and run.layers == 1
     if overlap:
         main = torch.cuda.current_stream()
         s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
         n_dq = len(dev_in) - 4
+        # head groups of the pipelined copies: the heads of a sequence are contiguous only when batch = 1
+        n_groups = 4 if (sh.batch == 1 and sh.kv_heads == 0 and sh.heads % 4 == 0 and sh.recent_window <= 1) else 1
+        groups = [(g * sh.heads // n_groups, (g + 1) * sh.heads // n_groups) for g in range(n_groups)]
+    O_step = run.O.clone() if run.has_prefill else None      # what the device-resident steps produced
     barrier()
     t_e2e = 0.0
     for _ in range(e2e_steps):
@@ -469,11 +495,15 @@ def run_ours(args, rank, world, dev):
         if overlap:
             s_in.wait_stream(main)
             s_out.wait_stream(main)
-            ready = []                                       # events: X, (K, V), Q, decode inputs
+            ready = []                                       # events: X, one per head group (its K, V, Q), decode inputs
             with torch.cuda.stream(s_in):
-                for group in ([0], [2, 3], [1], list(range(4, 4 + n_dq))):
-                    for i in group:
-                        dev_in[i].copy_(host_in[i], non_blocking=True)
+                for group in ([(0, None)], *[[(2, g), (3, g), (1, g)] for g in groups],
+                              [(i, None) for i in range(4, 4 + n_dq)]):
+                    for i, g in group:
+                        if g is None:
+                            dev_in[i].copy_(host_in[i], non_blocking=True)
+                        else:
+                            dev_in[i][:, g[0]:g[1]].copy_(host_in[i][:, g[0]:g[1]], non_blocking=True)
                     ev_ = torch.cuda.Event()
                     ev_.record(s_in)
                     ready.append(ev_)
@@ -483,13 +513,16 @@ def run_ours(args, rank, world, dev):
             with torch.cuda.stream(s_out):
                 s_out.wait_event(flags_done)
                 host_out[1].copy_(run.flags, non_blocking=True)
-            main.wait_event(ready[1]); run.compact()
-            main.wait_event(ready[2]); run.prefill()
-            o_done = torch.cuda.Event(); o_done.record(main)
-            with torch.cuda.stream(s_out):
-                s_out.wait_event(o_done)
-                host_out[0].copy_(run.O, non_blocking=True)
-            main.wait_event(ready[3]); run.decode_all()
+            for gi, g in enumerate(groups):
+                # compaction and prefill attention of a head group as soon as its K, V, Q are in; its O
+                # goes back while the next groups are still coming in (the link carries both directions)
+                main.wait_event(ready[1 + gi])
+                run.compact(g); run.prefill(g)
+                o_done = torch.cuda.Event(); o_done.record(main)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(o_done)
+                    host_out[0][:, g[0]:g[1]].copy_(run.O[:, g[0]:g[1]], non_blocking=True)
+            main.wait_event(ready[-1]); run.decode_all()
             host_out[2].copy_(run.o, non_blocking=True)
             main.wait_stream(s_out)
         else:
@@ -502,6 +535,8 @@ def run_ours(args, rank, world, dev):
         e.synchronize()
         t_e2e += s.elapsed_time(e)
     barrier()
+    if O_step is not None:
+        assert torch.equal(host_out[0], O_step.cpu()), "the end-to-end pass and the device-resident step disagree"
 
     total_ms, t_e2e = max_over_ranks([total_ms, t_e2e], dist, dev)
     if rank != 0:
