@@ -32,6 +32,8 @@ UNIT = "tokens/s"
 WORKLOADS = {
     # name: (shape, decode steps per step, description)
     "prefill7b": (inputs.PREFILL7B, 16, "Llama-2-7B-shaped AG-gated layer, batch 1 x seq 4096, keep rates U[0.3,0.8] per head"),
+    "prefill7b_proj": (inputs.PREFILL7B, 16, "the prefill7b layer owning its key/value projection: K, V = X [Wk | Wv] are computed in the "
+                                             "step and the retained rows go straight into the cache (ag_kv_project_cache in place of ag_compact_kv)"),
     "tiny": (inputs.TINY, 16, "fp32 correctness layer, batch 1 x seq 128, ~50% keep"),
     "deep_layer": (inputs.DEEP_LAYER, 128, "deep-layer pattern, batch 1 x seq 16384: 24 heads keep ~10%, 8 heads keep nothing"),
     "stack7b": (inputs.STACK7B, 256, "32 AG-gated layers back to back, batch 8 x seq 4096; per-layer mean eviction rising from 10% to 90%"),
@@ -49,6 +51,9 @@ TRAFFIC = {
     ("prefill7b", "decode"): 41.22e6 + 0.01e6,           # decode_cluster_mma_kernel
     ("prefill7b", "compact"): 41.26e6 + 3.10e6,          # compact_kernel<256> (written rows still in L2 at kernel end)
     ("prefill7b", "kv_project_cache"): 171.96e6 + 80.44e6,   # kv_proj_cache_kernel<256, 2>
+    ("prefill7b_proj", "project"): 171.96e6 + 80.44e6,
+    ("prefill7b_proj", "prefill"): 154.86e6 + 18.50e6,
+    ("prefill7b_proj", "decode"): 41.22e6 + 0.01e6,
     ("decode_ragged", "decode"): 2.3530e9 + 7.1e6,       # decode_partial_kernel<bf16,128>
 }
 # kernels launched per call of the library
@@ -169,7 +174,8 @@ class LayerRun:
         self.name = name
         self.use_graph, self.graph = True, None
         self._groups = {}
-        self.has_gate = name in ("prefill7b", "tiny", "stack7b", "stack7b_prev")
+        self.has_gate = name in ("prefill7b", "prefill7b_proj", "tiny", "stack7b", "stack7b_prev")
+        self.project = name == "prefill7b_proj"                     # K, V are computed in the step
         self.layers = 32 if name.startswith("stack7b") else 1
         self.first_gated = 1 if name == "stack7b_prev" else 0      # 0: every layer evicts by its own gate
         self.has_prefill = name not in ("decode_ragged", "decode_ragged_gqa")
@@ -177,6 +183,8 @@ class LayerRun:
             self.X = inputs.hidden_states(sh, seed, dev)
             self.W = inputs.layer_weights(sh, seed + 10, dev)
             self.Q, self.K, self.V = inputs.project_qkv(sh, self.X, self.W)
+            if self.project:
+                self.K2, self.V2 = self.K, self.V                  # the step writes them itself
         elif self.has_prefill:
             self.Q, self.K, self.V = inputs.qkv_gaussian(sh, seed, dev)
         else:
@@ -301,7 +309,10 @@ class LayerRun:
             if self.has_gate:
                 self.gamma = self.gammas[layer]
                 timed("gate", self.gate)
-            if self.has_prefill:
+            if self.project:
+                timed("project", self.kv_project_cache)
+                timed("prefill", self.prefill)
+            elif self.has_prefill:
                 timed("compact", self.compact)
                 timed("prefill", self.prefill)
             else:
@@ -440,7 +451,7 @@ def run_ours(args, rank, world, dev):
     sampler = ClockSampler(torch.cuda.current_device())
     if rank == 0:
         sampler.start()
-    ev = {k: [] for k in ("gate", "compact", "prefill", "decode")}
+    ev = {k: [] for k in ("gate", "compact", "project", "prefill", "decode")}
     step_ev = []
     barrier()
     for _ in range(args.steps):
@@ -460,7 +471,9 @@ def run_ours(args, rank, world, dev):
 
     # end to end: pinned host inputs in, results out, through the same calls
     sh = run.shape
-    if run.has_gate:
+    if run.project:
+        dev_in = [run.X, run.Q]                              # K and V are made on the device
+    elif run.has_gate:
         dev_in = [run.X, run.Q, run.K, run.V]
     elif run.has_prefill:
         dev_in = [run.Q, run.K, run.V, run.flags]
@@ -478,7 +491,10 @@ def run_ours(args, rank, world, dev):
     # decode), and the flags and each group's O go back to the host while later groups come in.
     # Other workloads: copy in, step, copy out, in order.
     overlap = run.has_gate and run.has_prefill and run.layers == 1
-    if overlap:
+    if overlap and run.project:
+        main = torch.cuda.current_stream()
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    elif overlap:
         main = torch.cuda.current_stream()
         s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
         n_dq = len(dev_in) - 4
@@ -492,7 +508,34 @@ def run_ours(args, rank, world, dev):
         flush_l2(l2buf)
         s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s.record()
-        if overlap:
+        if overlap and run.project:
+            # X -> gate and the key/value projection; Q -> prefill; the decode tokens -> decode
+            s_in.wait_stream(main)
+            s_out.wait_stream(main)
+            ready = []
+            with torch.cuda.stream(s_in):
+                for group in ([0], [1], list(range(2, len(dev_in)))):
+                    for i in group:
+                        dev_in[i].copy_(host_in[i], non_blocking=True)
+                    ev_ = torch.cuda.Event()
+                    ev_.record(s_in)
+                    ready.append(ev_)
+            run.gamma = run.gammas[0]
+            main.wait_event(ready[0]); run.gate()
+            flags_done = torch.cuda.Event(); flags_done.record(main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(flags_done)
+                host_out[1].copy_(run.flags, non_blocking=True)
+            run.kv_project_cache()
+            main.wait_event(ready[1]); run.prefill()
+            o_done = torch.cuda.Event(); o_done.record(main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(o_done)
+                host_out[0].copy_(run.O, non_blocking=True)
+            main.wait_event(ready[2]); run.decode_all()
+            host_out[2].copy_(run.o, non_blocking=True)
+            main.wait_stream(s_out)
+        elif overlap:
             s_in.wait_stream(main)
             s_out.wait_stream(main)
             ready = []                                       # events: X, one per head group (its K, V, Q), decode inputs
@@ -561,11 +604,19 @@ def run_ours(args, rank, world, dev):
                                 "ms": per_call_ms["prefill"]}
         e = 2 if sh.dtype == "bf16" else 4
         kept = work["kept_rows"]
-        cb = 2.0 * (2.0 * kept * sh.head_dim * e) + sh.batch * sh.heads * sh.seq * 9.0
-        gbs = cb / (per_call_ms["compact"] * 1e-3) / 1e9
-        rooflines["compact"] = {"bound": "hbm", "kernel": "ag_compact_kv", "achieved": gbs, "peak": peaks["hbm_gbs"],
-                                "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
-                                "peak_source": peaks["source"], "algorithmic_bytes": cb, "ms": per_call_ms["compact"]}
+        if "compact" in per_call_ms:
+            cb = 2.0 * (2.0 * kept * sh.head_dim * e) + sh.batch * sh.heads * sh.seq * 9.0
+            gbs = cb / (per_call_ms["compact"] * 1e-3) / 1e9
+            rooflines["compact"] = {"bound": "hbm", "kernel": "ag_compact_kv", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                                    "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                                    "peak_source": peaks["source"], "algorithmic_bytes": cb, "ms": per_call_ms["compact"]}
+        if "project" in per_call_ms:
+            kf = 2.0 * sh.batch * sh.seq * sh.hidden * 2 * sh.kvh * sh.head_dim
+            tf = kf / (per_call_ms["project"] * 1e-3) / 1e12
+            rooflines["project"] = {"bound": "tensor", "kernel": "ag_kv_project_cache", "achieved": tf,
+                                    "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
+                                    "traffic": None, "peak_source": peaks["source"], "algorithmic_flops": kf,
+                                    "ms": per_call_ms["project"]}
     if run.has_gate:
         gf = run.gate_flops()
         tf = gf / (per_call_ms["gate"] * 1e-3) / 1e12
@@ -591,7 +642,8 @@ def run_ours(args, rank, world, dev):
                                     "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                     "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
                                     "algorithmic_bytes": lb, "ms": lin_ms}
-        if sh.dtype == "bf16" and sh.head_dim == 128 and sh.seq % 128 == 0 and sh.recent_window <= 1 and run.layers == 1:
+        if (sh.dtype == "bf16" and sh.head_dim == 128 and sh.seq % 128 == 0 and sh.recent_window <= 1 and run.layers == 1
+                and not run.project):
             # the fused key/value projection, timed apart from the step like the local gate
             kv_ev = []
             for i in range(3 + min(args.steps, 20)):
@@ -638,7 +690,7 @@ def run_ours(args, rank, world, dev):
         "decode_tokens_per_s": sh.batch * run.decode_steps / (per_call_ms["decode"] * 1e-3),
     }
     if run.has_prefill:
-        pre_ms = sum(per_call_ms.get(k, 0.0) for k in ("gate", "compact", "prefill"))
+        pre_ms = sum(per_call_ms.get(k, 0.0) for k in ("gate", "compact", "project", "prefill"))
         out["prefill_tokens_per_s"] = sh.batch * sh.seq / (pre_ms * 1e-3)
     return out, run
 
@@ -672,6 +724,8 @@ def oracle_sample(name, seed, n_heads_sample=2, decode_steps=2):
     t_gate += time.perf_counter() - t0
     fl = flags[:, :hs]
     t0 = time.perf_counter()
+    if name == "prefill7b_proj":                 # the layer owns its key/value projection (Eq. 2)
+        Kd, Vd = orc.project_kv(Xd, f64(Wsub["Wk"]), f64(Wsub["Wv"]), hs)
     cache = orc.compact_kv(Kd, Vd, fl)
     O = orc.prefill_attention(Qd, Kd, Vd, fl)
     t_heads = time.perf_counter() - t0
@@ -756,7 +810,7 @@ def main():
     res = run_ours(args, rank, world, torch.device("cuda", local))
     if rank == 0:
         out, run = res
-        if not args.no_cpu_baseline and world == 1 and args.workload in ("prefill7b", "tiny"):
+        if not args.no_cpu_baseline and world == 1 and args.workload in ("prefill7b", "prefill7b_proj", "tiny"):
             cb = oracle_sample(args.workload, 2000, n_heads_sample=WORKLOADS[args.workload][0].heads, decode_steps=16)
             cb.pop("est_step_s", None)
             out["cpu_baseline"] = cb
