@@ -517,6 +517,9 @@ decode_cluster_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat
   const int kv = hm.kv_slab(slab);
   const int d = threadIdx.x;
   pdl_launch_dependents();
+  // the slab's first row never changes once the cache is laid out: read ahead of the wait for the
+  // preceding kernel, so that only the length is on the critical path after it
+  const int64_t slab_row0 = row_off[kv];
   pdl_wait();
   const int L = len[kv];
   const int per = ((L + kClusterSize - 1) / kClusterSize + kGqTile - 1) / kGqTile * kGqTile;
@@ -535,7 +538,7 @@ decode_cluster_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat
   }
 
   if (r_begin < r_end) {              // the same for the whole CTA
-    const size_t row0 = (size_t)row_off[kv] * kGqRowBytes;
+    const size_t row0 = (size_t)slab_row0 * kGqRowBytes;
     const GqWarpTriples w = gq_stream_rows<kCmStages>(gq_smem, q + (size_t)slab * D, 1,
                                            reinterpret_cast<const uint8_t *>(k_rows) + row0,
                                            reinterpret_cast<const uint8_t *>(v_rows) + row0, r_begin, r_end, scale_log2);
@@ -554,7 +557,7 @@ decode_cluster_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat
   cluster.sync();
   // every CTA of the cluster has read the length and its rows: the new row may go in
   // (never asked for when query heads share a slab: another head's cluster may still be reading its length)
-  if (rank == 0) append_new_row<T, D>(ap, kv, L, row_off[kv], k_new, v_new);
+  if (rank == 0) append_new_row<T, D>(ap, kv, L, slab_row0, k_new, v_new);
   if (rank == 0) {
     float s_self = 0.f;
 #pragma unroll
