@@ -232,6 +232,21 @@ def project_kv(X, Wk, Wv, kv_heads):
     return K, V
 
 
+def project_q(X, Wq, heads):
+    """Queries of the layer, Eq. 2: Q_i = X W^Q_i, head i taking columns
+    [i D, (i + 1) D) of the "in x out" weight.  X [B, n, d], Wq [d, heads * D]
+    -> Q [B, heads, n, D] in float64."""
+    X, Wq = _as_f64(X), _as_f64(Wq)
+    B, n, d = X.shape
+    D = Wq.shape[1] // heads
+    Q = np.empty((B, heads, n, D), dtype=F64)
+    for b in range(B):
+        for i in range(heads):
+            for t in range(n):
+                Q[b, i, t] = X[b, t] @ Wq[:, i * D:(i + 1) * D]
+    return Q
+
+
 def project_and_cache(X, Wk, Wv, flags):
     """Eq. 2's projection followed by selective caching (Sec. 3.3): the dense
     K, V [B, h, n, D] and the ragged cache of the retained rows, as

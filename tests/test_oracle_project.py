@@ -73,3 +73,23 @@ def test_cache_holds_the_projected_rows_of_the_retained_tokens():
             for r, t in enumerate(kept):
                 assert np.allclose(cache[b][i]["k"][r], X[b, t] @ Wk[:, i * 4:(i + 1) * 4], rtol=0, atol=1e-12)
                 assert np.allclose(cache[b][i]["v"][r], X[b, t] @ Wv[:, i * 4:(i + 1) * 4], rtol=0, atol=1e-12)
+
+
+def test_queries_unit_rows_loops_and_library():
+    d, h, D = 6, 3, 2
+    rng = np.random.default_rng(5)
+    Wq = rng.standard_normal((d, h * D))
+    Q = orc.project_q(np.eye(d)[None], Wq, h)             # token c = e_c  =>  Q_i[c] = row c of W^Q_i
+    for i in range(h):
+        assert np.array_equal(Q[0, i], Wq[:, i * D:(i + 1) * D])
+    X = rng.standard_normal((2, 5, d))
+    Q = orc.project_q(X, Wq, h)
+    for b in range(2):
+        for i in range(h):
+            for t in range(5):
+                for c in range(D):
+                    assert abs(Q[b, i, t, c] - sum(X[b, t, a] * Wq[a, i * D + c] for a in range(d))) < 1e-12
+    assert np.allclose(Q, np.einsum("bnd,dhc->bhnc", X, Wq.reshape(d, h, D)), rtol=0, atol=1e-12)
+    # with the same weight, queries are what the key projection gives for as many heads
+    K, _ = orc.project_kv(X, Wq, Wq, h)
+    assert np.allclose(Q, K, rtol=0, atol=1e-12)
