@@ -15,6 +15,7 @@
  *   ag_kv_project_cache     K_i = X W^K_i, V_i = X W^V_i written
  *                           to the dense K, V and, for retained
  *                           tokens, straight into the cache     Eq. 2 + Sec. 3.3 (after Eq. 4)
+ *   ag_qkv_project_cache    the same with Q_i = X W^Q_i         Eq. 2
  *
  * Conventions common to every call
  * --------------------------------
@@ -235,6 +236,22 @@ int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk
                         const void *Wv, const uint8_t *flags, ag_cache *cache,
                         int32_t *prefix, int32_t *idx, void *K, void *V,
                         int32_t *dev_status, void *cuda_stream);
+
+/*
+ * ag_kv_project_cache with the query projection of Eq. 2, Q_i = X W^Q_i, in the
+ * same launch: the whole Q, K, V projection of the layer runs inside the path.
+ * Queries take no part in eviction: Q goes to its dense tensor only.
+ *
+ *   Wq      [d, heads D]          in   ("in x out")
+ *   Q       [B, heads, n, D]      out
+ * Everything else (arguments, results, kernel coverage, errors) as for
+ * ag_kv_project_cache; with grouped-query attention Q has desc->heads heads and
+ * K, V, flags, prefix, idx and the cache desc->kv_heads.
+ */
+int ag_qkv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wq,
+                         const void *Wk, const void *Wv, const uint8_t *flags,
+                         ag_cache *cache, int32_t *prefix, int32_t *idx, void *Q,
+                         void *K, void *V, int32_t *dev_status, void *cuda_stream);
 
 /*
  * Step 3 — prefill attention under the eviction mask (Eq. 2 with Eq. 5):

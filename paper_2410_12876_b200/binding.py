@@ -22,7 +22,7 @@ EXPORTS = (
     "ag_workspace_bytes", "ag_gate_forward", "ag_compact_kv", "ag_prefill_attn",
     "ag_decode_attn", "ag_cache_append", "ag_status_string", "ag_last_cuda_error",
     "ag_decode_attn_noalloc", "ag_device_wait_timeouts", "ag_gate_linear_forward", "ag_decode_step",
-    "ag_kv_project_cache",
+    "ag_kv_project_cache", "ag_qkv_project_cache",
 )
 
 
@@ -76,6 +76,8 @@ def lib():
         L.ag_compact_kv.argtypes = [dp, vp, vp, vp, cp, vp, vp, vp, vp, sz, vp]
         L.ag_kv_project_cache.restype = i32
         L.ag_kv_project_cache.argtypes = [dp, vp, vp, vp, vp, cp, vp, vp, vp, vp, vp, vp]
+        L.ag_qkv_project_cache.restype = i32
+        L.ag_qkv_project_cache.argtypes = [dp, vp, vp, vp, vp, vp, cp, vp, vp, vp, vp, vp, vp, vp]
         L.ag_prefill_attn.restype = i32
         L.ag_prefill_attn.argtypes = [dp, vp, vp, vp, vp, cp, vp, f32, vp, vp, sz, vp]
         L.ag_decode_attn.restype = i32
@@ -211,6 +213,12 @@ def ag_kv_project_cache(desc, X, Wk, Wv, flags, cache, prefix, idx, K, V, dev_st
     return _check(lib().ag_kv_project_cache(ctypes.byref(desc), _ptr(X), _ptr(Wk), _ptr(Wv), _ptr(flags),
                                             ctypes.byref(cache.struct), _ptr(prefix), _ptr(idx), _ptr(K), _ptr(V),
                                             _ptr(dev_status), _stream(stream)), "ag_kv_project_cache")
+
+
+def ag_qkv_project_cache(desc, X, Wq, Wk, Wv, flags, cache, prefix, idx, Q, K, V, dev_status, stream=None):
+    return _check(lib().ag_qkv_project_cache(ctypes.byref(desc), _ptr(X), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(flags),
+                                             ctypes.byref(cache.struct), _ptr(prefix), _ptr(idx), _ptr(Q), _ptr(K),
+                                             _ptr(V), _ptr(dev_status), _stream(stream)), "ag_qkv_project_cache")
 
 
 def ag_prefill_attn(desc, Q, K, V, flags, cache, prefix, softmax_scale, O, ws, stream=None):

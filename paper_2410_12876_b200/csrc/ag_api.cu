@@ -140,7 +140,24 @@ int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk
       misaligned16(flags) || misaligned16(prefix) || misaligned16(idx))
     return AG_ERR_INVALID_ARG;
   if (!kv_proj_cache_supported(*desc)) return AG_ERR_UNSUPPORTED;
-  return launch_kv_proj_cache(*desc, X, Wk, Wv, flags, *cache, prefix, idx, K, V, dev_status,
+  return launch_kv_proj_cache(*desc, X, nullptr, Wk, Wv, flags, *cache, prefix, idx, nullptr, K, V, dev_status,
+                              (cudaStream_t)cuda_stream);
+}
+
+int ag_qkv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wq, const void *Wk, const void *Wv,
+                         const uint8_t *flags, ag_cache *cache, int32_t *prefix, int32_t *idx, void *Q, void *K,
+                         void *V, int32_t *dev_status, void *cuda_stream) {
+  int st = check_desc(desc);
+  if (st) return st;
+  if (desc->hidden <= 0) return AG_ERR_INVALID_ARG;
+  if (!X || !Wq || !Wk || !Wv || !flags || !prefix || !Q || !K || !V) return AG_ERR_INVALID_ARG;
+  st = check_cache(cache);
+  if (st) return st;
+  if (misaligned16(X) || misaligned16(Wq) || misaligned16(Wk) || misaligned16(Wv) || misaligned16(Q) ||
+      misaligned16(K) || misaligned16(V) || misaligned16(flags) || misaligned16(prefix) || misaligned16(idx))
+    return AG_ERR_INVALID_ARG;
+  if (!kv_proj_cache_supported(*desc)) return AG_ERR_UNSUPPORTED;
+  return launch_kv_proj_cache(*desc, X, Wq, Wk, Wv, flags, *cache, prefix, idx, Q, K, V, dev_status,
                               (cudaStream_t)cuda_stream);
 }
 

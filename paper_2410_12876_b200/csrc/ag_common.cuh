@@ -84,9 +84,10 @@ int launch_compact(const ag_layer_desc &d, const void *K, const void *V, const u
 // Key/value projection (Eq. 2) on the tensor cores with the retained rows written straight into the
 // ragged cache (bf16, head_dim 128, seq a multiple of 128).
 bool kv_proj_cache_supported(const ag_layer_desc &d);
-int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, const uint8_t *flags,
-                         const ag_cache &c, int32_t *prefix, int32_t *idx, void *K, void *V, int32_t *dev_status,
-                         cudaStream_t st);
+// Wq, Q: NULL, or the query projection Q = X Wq rides in the same launch (dense output only).
+int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, const void *Wv,
+                         const uint8_t *flags, const ag_cache &c, int32_t *prefix, int32_t *idx, void *Q, void *K,
+                         void *V, int32_t *dev_status, cudaStream_t st);
 int kv_proj_cache_wait_timeouts();
 
 size_t prefill_workspace_bytes(const ag_layer_desc &d);

@@ -1,4 +1,5 @@
-// Key/value projection fused with selective caching: K_i = X W^K_i, V_i = X W^V_i (Eq. 2) on the
+// Key/value (and, optionally, query) projection fused with selective caching: K_i = X W^K_i, V_i = X W^V_i
+// (and Q_i = X W^Q_i, which goes to its dense tensor only) (Eq. 2) on the
 // 5th-generation tensor cores, with an epilogue that rounds each tile to bf16 once and sends it
 // to both places the layer reads it from: the dense K, V [B, h, n, D] (every token attends to its
 // own key, the diagonal of Eq. 5) and, for the tokens the gate retains (Sec. 3.3: k, v are kept
@@ -45,12 +46,13 @@ template <int BN, int MT> struct KvCfg {
 template <int BN, int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBk,
-                     const __grid_constant__ CUtensorMap tmBv, const __grid_constant__ CUtensorMap tmK,
-                     const __grid_constant__ CUtensorMap tmV, const uint8_t *__restrict__ flags,
+                     const __grid_constant__ CUtensorMap tmBv, const __grid_constant__ CUtensorMap tmBq,
+                     const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                     const __grid_constant__ CUtensorMap tmQ, const uint8_t *__restrict__ flags,
                      int32_t *__restrict__ prefix, int32_t *__restrict__ idx, const int64_t *__restrict__ row_off,
                      const int32_t *__restrict__ cap, int32_t *__restrict__ len, uint8_t *__restrict__ k_rows,
                      uint8_t *__restrict__ v_rows, int32_t *__restrict__ dev_status, int M, int Kdim, int GD,
-                     int n, int kv_heads, int n_tiles_m, int n_tiles_n, int split_from) {
+                     int n, int kv_heads, int heads, int n_tiles_m, int n_tiles_n, int split_from) {
   using Cfg = KvCfg<BN, MT>;
   constexpr uint32_t kTmemCols = MT * BN;
   static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "TMEM columns: a power of two");
@@ -76,9 +78,13 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   const int band_rows = min(kBandTiles, n_tiles_m - band * kBandTiles);
   const int tile_m = band * kBandTiles + in_band % band_rows, tile_n = in_band / band_rows;
   const int m0 = tile_m * (MT * kBM) + (single ? ((cta - split_from) & 1) * kBM : 0);
-  const int n0 = tile_n * BN;                    // in the packed [2 * GD] output
-  const int which = n0 / GD, nw = n0 % GD;       // BN divides GD: a tile lies in one weight
-  const CUtensorMap *tmB = which == 0 ? &tmBk : &tmBv;
+  const int n0 = tile_n * BN;                    // in the packed output [K | V | Q] (GD, GD and heads * D columns)
+  // BN divides the width of every weight: a tile lies in one weight.  which: 0 keys, 1 values, 2 queries
+  // (queries go to their dense tensor only: no flags, no cache)
+  const int which = n0 < GD ? 0 : (n0 < 2 * GD ? 1 : 2);
+  const int nw = n0 - min(which, 2) * GD;
+  const CUtensorMap *tmB = which == 0 ? &tmBk : (which == 1 ? &tmBv : &tmBq);
+  const int out_heads = which == 2 ? heads : kv_heads;
   const int num_kb = (Kdim + kBK - 1) / kBK;
 
   if (threadIdx.x == 0) {
@@ -159,7 +165,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
       for (int hh = 0; hh < Cfg::kHeads; ++hh) {
         long long d = -1;
-        if (m_base < M && mt < mts) {                             // the same for all 128 threads
+        if (m_base < M && mt < mts && which != 2) {               // the same for all 128 threads
           const size_t slab = (size_t)b * kv_heads + nw / kD + hh;
           const uint8_t *f = flags + slab * n;
           const uint4 *fv = reinterpret_cast<const uint4 *>(f);
@@ -205,7 +211,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
     const bool ok = mbar_wait(acc_full, 0);
     tc_fence_after_sync();
-    const CUtensorMap *tmOut = which == 0 ? &tmK : &tmV;
+    const CUtensorMap *tmOut = which == 0 ? &tmK : (which == 1 ? &tmV : &tmQ);
     uint8_t *rows_out = which == 0 ? k_rows : v_rows;
     const int hw = (warp - 2) * 2 + (lane >> 4), l16 = lane & 15;   // half-warp 0..15, 16-byte piece of a row
 #pragma unroll 1
@@ -237,12 +243,12 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       if (threadIdx.x == 64) {
 #pragma unroll
         for (int p = 0; p < BN / 64; ++p)
-          tma_store_3d(tmOut, stg + p * kBM * 128, (p & 1) * 64, t0, b * kv_heads + nw / kD + (p >> 1));
+          tma_store_3d(tmOut, stg + p * kBM * 128, (p & 1) * 64, t0, b * out_heads + nw / kD + (p >> 1));
         tma_store_commit();
       }
       // retained rows: half-warp per row, 16 bytes per lane
 #pragma unroll
-      for (int hh = 0; hh < Cfg::kHeads; ++hh) {
+      for (int hh = 0; hh < (which != 2 ? Cfg::kHeads : 0); ++hh) {
         const long long *dr = dst_row + (mt * Cfg::kHeads + hh) * kBM;
 #pragma unroll 4
         for (int r = hw; r < kBM; r += 16) {
@@ -273,11 +279,13 @@ int sm_count() {
 }
 
 template <int BN, int MT>
-int run(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, const uint8_t *flags,
-        const ag_cache &c, int32_t *prefix, int32_t *idx, void *K, void *V, int32_t *dev_status, cudaStream_t st) {
+int run(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, const void *Wv, const uint8_t *flags,
+        const ag_cache &c, int32_t *prefix, int32_t *idx, void *Q, void *K, void *V, int32_t *dev_status,
+        cudaStream_t st) {
   using Cfg = KvCfg<BN, MT>;
   const int hk = kv_heads_of(d), GD = hk * kD, M = d.batch * d.seq, Kdim = d.hidden;
-  CUtensorMap tmA, tmBk, tmBv, tmK, tmV;
+  const int QD = Wq ? d.heads * kD : 0;          // query columns of the packed output (0: keys and values only)
+  CUtensorMap tmA, tmBk, tmBv, tmBq, tmK, tmV, tmQ;
   int rc = make_tmap_2d_bf16(&tmA, X, M, Kdim, (uint64_t)Kdim * 2, kBM, kBK);
   if (rc) return rc;
   rc = make_tmap_2d_bf16(&tmBk, Wk, Kdim, GD, (uint64_t)GD * 2, kBK, 64);
@@ -288,15 +296,23 @@ int run(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, c
   if (rc) return rc;
   rc = make_tmap_3d_bf16(&tmV, V, (uint64_t)d.batch * hk, d.seq, kD, kBM, 64);
   if (rc) return rc;
+  tmBq = tmBk;                                   // stand-ins when there is no query projection
+  tmQ = tmK;
+  if (Wq) {
+    rc = make_tmap_2d_bf16(&tmBq, Wq, Kdim, QD, (uint64_t)QD * 2, kBK, 64);
+    if (rc) return rc;
+    rc = make_tmap_3d_bf16(&tmQ, Q, (uint64_t)d.batch * d.heads, d.seq, kD, kBM, 64);
+    if (rc) return rc;
+  }
   auto kern = kv_proj_cache_kernel<BN, MT>;
   AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-  const int n_tiles_n = 2 * GD / BN, n_tiles_m = (M + MT * kBM - 1) / (MT * kBM), n_tiles = n_tiles_n * n_tiles_m;
+  const int n_tiles_n = (2 * GD + QD) / BN, n_tiles_m = (M + MT * kBM - 1) / (MT * kBM), n_tiles = n_tiles_n * n_tiles_m;
   const int tail = n_tiles % sm_count();
   const int split_from = (MT > 1 && tail > 0 && 2 * tail <= sm_count()) ? n_tiles - tail : n_tiles;
   const int ctas = split_from + 2 * (n_tiles - split_from);
-  kern<<<ctas, kThreads, Cfg::kSmemBytes, st>>>(tmA, tmBk, tmBv, tmK, tmV, flags, prefix, idx, c.row_off, c.cap, c.len,
+  kern<<<ctas, kThreads, Cfg::kSmemBytes, st>>>(tmA, tmBk, tmBv, tmBq, tmK, tmV, tmQ, flags, prefix, idx, c.row_off, c.cap, c.len,
                                                    static_cast<uint8_t *>(c.k_rows), static_cast<uint8_t *>(c.v_rows),
-                                                   dev_status, M, Kdim, GD, d.seq, hk, n_tiles_m, n_tiles_n, split_from);
+                                                   dev_status, M, Kdim, GD, d.seq, hk, d.heads, n_tiles_m, n_tiles_n, split_from);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
@@ -308,17 +324,17 @@ bool kv_proj_cache_supported(const ag_layer_desc &d) {
          recent_rows(d) == 0 && (int64_t)d.batch * d.seq < ((int64_t)1 << 31);
 }
 
-int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wk, const void *Wv, const uint8_t *flags,
-                         const ag_cache &c, int32_t *prefix, int32_t *idx, void *K, void *V, int32_t *dev_status,
-                         cudaStream_t st) {
-  const int hk = kv_heads_of(d);
-  const long long tiles128 = (long long)(2 * hk * kD / 128) * (d.batch * (long long)d.seq / kBM);
-  if (hk % 2 == 0) {
+int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, const void *Wv,
+                         const uint8_t *flags, const ag_cache &c, int32_t *prefix, int32_t *idx, void *Q, void *K,
+                         void *V, int32_t *dev_status, cudaStream_t st) {
+  const int hk = kv_heads_of(d), hq = Wq ? d.heads : 0;
+  const long long tiles128 = (long long)(2 * hk + hq) * (d.batch * (long long)d.seq / kBM);
+  if (hk % 2 == 0 && hq % 2 == 0) {
     // more than one wave: 256-token tiles, whose two sub-tiles share every stage of W
-    if (tiles128 > 2 * sm_count()) return run<256, 2>(d, X, Wk, Wv, flags, c, prefix, idx, K, V, dev_status, st);
-    return run<256, 1>(d, X, Wk, Wv, flags, c, prefix, idx, K, V, dev_status, st);
+    if (tiles128 > 2 * sm_count()) return run<256, 2>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
+    return run<256, 1>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
   }
-  return run<128, 1>(d, X, Wk, Wv, flags, c, prefix, idx, K, V, dev_status, st);
+  return run<128, 1>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
 }
 
 int kv_proj_cache_wait_timeouts() {

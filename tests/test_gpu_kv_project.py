@@ -48,8 +48,9 @@ def _flags(shape, seed):
     return f
 
 
-def gpu_project_cache(shape, X, W, flags, cap=None):
-    """The fused projection on buffers that hold nothing of a previous call."""
+def gpu_project_cache(shape, X, W, flags, cap=None, with_q=False):
+    """The fused projection on buffers that hold nothing of a previous call; with_q: the call that
+    projects the queries too (Q is then the last item returned)."""
     desc = ag.make_desc(shape)
     B, h, n, D = shape.batch, shape.kvh, shape.seq, shape.head_dim
     if cap is None:
@@ -61,17 +62,24 @@ def gpu_project_cache(shape, X, W, flags, cap=None):
     cache.len.fill_(-7)                                    # the call sets the lengths itself
     K = torch.full((B, h, n, D), float("nan"), dtype=torch.bfloat16, device=DEV)
     V = torch.full_like(K, float("nan"))
+    if with_q:
+        Q = torch.full((B, shape.heads, n, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+        ag.ag_qkv_project_cache(desc, X, W["Wq"], W["Wk"], W["Wv"], flags, cache, prefix, idx, Q, K, V, status)
+        torch.cuda.synchronize()
+        return cache, prefix, idx, status, K, V, Q
     ag.ag_kv_project_cache(desc, X, W["Wk"], W["Wv"], flags, cache, prefix, idx, K, V, status)
     torch.cuda.synchronize()
     return cache, prefix, idx, status, K, V
 
 
-def _check(shape, seed, cap=None):
+def _check(shape, seed, cap=None, with_q=False):
     X = inputs.hidden_states(shape, seed, DEV)
     W = inputs.layer_weights(shape, seed + 10, DEV)
     fl = _flags(shape, seed + 20)
     flags = torch.from_numpy(fl).to(DEV)
-    cache, prefix, idx, status, K, V = gpu_project_cache(shape, X, W, flags, cap)
+    cache, prefix, idx, status, K, V, *rest = gpu_project_cache(shape, X, W, flags, cap, with_q)
+    if with_q:
+        _close_to_rounded(T.f64(rest[0]), orc.project_q(T.f64(X), T.f64(W["Wq"]), shape.heads), "dense Q")
     Kr, Vr, ocache = orc.project_and_cache(T.f64(X), T.f64(W["Wk"]), T.f64(W["Wv"]), fl)
     _close_to_rounded(T.f64(K), Kr, "dense K")
     _close_to_rounded(T.f64(V), Vr, "dense V")
@@ -120,6 +128,13 @@ CASES = {
 @pytest.mark.parametrize("name", list(CASES))
 def test_projection_and_cache(name):
     _check(CASES[name], 900)
+
+
+@pytest.mark.parametrize("name", ["two_heads_per_tile", "k_tail", "odd_heads", "subtiles_of_two_sequences",
+                                  "split_last_wave_odd_rows", "grouped_query"])
+def test_projection_with_queries(name):
+    """ag_qkv_project_cache: Q against the oracle's query projection, K, V and the cache as without it."""
+    _check(CASES[name], 940, with_q=True)
 
 
 def test_slab_too_small_is_skipped_and_reported():
@@ -191,4 +206,7 @@ def test_rejects_what_it_has_no_kernel_for():
         assert e.value.status in (ag.AG_ERR_UNSUPPORTED, ag.AG_ERR_INVALID_ARG)
     with pytest.raises(ag.AgError) as e:
         ag.ag_kv_project_cache(ag.make_desc(shape), X, W["Wk"], None, flags, cache, prefix, idx, K, V, status)
+    assert e.value.status == ag.AG_ERR_INVALID_ARG
+    with pytest.raises(ag.AgError) as e:
+        ag.ag_qkv_project_cache(ag.make_desc(shape), X, None, W["Wk"], W["Wv"], flags, cache, prefix, idx, K, K, V, status)
     assert e.value.status == ag.AG_ERR_INVALID_ARG
