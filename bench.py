@@ -32,8 +32,8 @@ UNIT = "tokens/s"
 WORKLOADS = {
     # name: (shape, decode steps per step, description)
     "prefill7b": (inputs.PREFILL7B, 16, "Llama-2-7B-shaped AG-gated layer, batch 1 x seq 4096, keep rates U[0.3,0.8] per head"),
-    "prefill7b_proj": (inputs.PREFILL7B, 16, "the prefill7b layer owning its key/value projection: K, V = X [Wk | Wv] are computed in the "
-                                             "step and the retained rows go straight into the cache (ag_kv_project_cache in place of ag_compact_kv)"),
+    "prefill7b_proj": (inputs.PREFILL7B, 16, "the prefill7b layer owning its projection: Q, K, V = X [Wq | Wk | Wv] are computed in the "
+                                             "step and the retained rows go straight into the cache (ag_qkv_project_cache in place of ag_compact_kv)"),
     "tiny": (inputs.TINY, 16, "fp32 correctness layer, batch 1 x seq 128, ~50% keep"),
     "deep_layer": (inputs.DEEP_LAYER, 128, "deep-layer pattern, batch 1 x seq 16384: 24 heads keep ~10%, 8 heads keep nothing"),
     "stack7b": (inputs.STACK7B, 256, "32 AG-gated layers back to back, batch 8 x seq 4096; per-layer mean eviction rising from 10% to 90%"),
@@ -51,7 +51,6 @@ TRAFFIC = {
     ("prefill7b", "decode"): 41.22e6 + 0.003e6,          # decode_cluster_mma_kernel
     ("prefill7b", "compact"): 41.26e6 + 3.10e6,          # compact_kernel<256> (written rows still in L2 at kernel end)
     ("prefill7b", "kv_project_cache"): 171.96e6 + 80.44e6,   # kv_proj_cache_kernel<256, 2>
-    ("prefill7b_proj", "project"): 171.96e6 + 80.44e6,
     ("prefill7b_proj", "prefill"): 154.86e6 + 18.50e6,
     ("prefill7b_proj", "decode"): 41.22e6 + 0.003e6,
     ("decode_ragged", "decode"): 2.3530e9 + 7.1e6,       # decode_partial_kernel<bf16,128>
@@ -175,7 +174,7 @@ class LayerRun:
         self.use_graph, self.graph = True, None
         self._groups = {}
         self.has_gate = name in ("prefill7b", "prefill7b_proj", "tiny", "stack7b", "stack7b_prev")
-        self.project = name == "prefill7b_proj"                     # K, V are computed in the step
+        self.project = name == "prefill7b_proj"                     # Q, K, V are computed in the step
         self.layers = 32 if name.startswith("stack7b") else 1
         self.first_gated = 1 if name == "stack7b_prev" else 0      # 0: every layer evicts by its own gate
         self.has_prefill = name not in ("decode_ragged", "decode_ragged_gqa")
@@ -255,6 +254,9 @@ class LayerRun:
         ag = self.ag
         if not hasattr(self, "K2"):
             self.K2, self.V2 = torch.empty_like(self.K), torch.empty_like(self.V)
+        if self.project:           # the layer owns its whole Q, K, V projection
+            return ag.ag_qkv_project_cache(self.desc, self.X, self.W["Wq"], self.W["Wk"], self.W["Wv"], self.cur_flags,
+                                           self.cache, self.prefix, None, self.Q, self.K2, self.V2, self.status)
         ag.ag_kv_project_cache(self.desc, self.X, self.W["Wk"], self.W["Wv"], self.cur_flags, self.cache, self.prefix,
                                None, self.K2, self.V2, self.status)
 
@@ -472,7 +474,7 @@ def run_ours(args, rank, world, dev):
     # end to end: pinned host inputs in, results out, through the same calls
     sh = run.shape
     if run.project:
-        dev_in = [run.X, run.Q]                              # K and V are made on the device
+        dev_in = [run.X]                                     # Q, K and V are made on the device
     elif run.has_gate:
         dev_in = [run.X, run.Q, run.K, run.V]
     elif run.has_prefill:
@@ -509,12 +511,12 @@ def run_ours(args, rank, world, dev):
         s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s.record()
         if overlap and run.project:
-            # X -> gate and the key/value projection; Q -> prefill; the decode tokens -> decode
+            # X -> gate, the projection and prefill; the decode tokens -> decode
             s_in.wait_stream(main)
             s_out.wait_stream(main)
             ready = []
             with torch.cuda.stream(s_in):
-                for group in ([0], [1], list(range(2, len(dev_in)))):
+                for group in ([0], list(range(1, len(dev_in)))):
                     for i in group:
                         dev_in[i].copy_(host_in[i], non_blocking=True)
                     ev_ = torch.cuda.Event()
@@ -527,12 +529,12 @@ def run_ours(args, rank, world, dev):
                 s_out.wait_event(flags_done)
                 host_out[1].copy_(run.flags, non_blocking=True)
             run.kv_project_cache()
-            main.wait_event(ready[1]); run.prefill()
+            run.prefill()
             o_done = torch.cuda.Event(); o_done.record(main)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(o_done)
                 host_out[0].copy_(run.O, non_blocking=True)
-            main.wait_event(ready[2]); run.decode_all()
+            main.wait_event(ready[1]); run.decode_all()
             host_out[2].copy_(run.o, non_blocking=True)
             main.wait_stream(s_out)
         elif overlap:
@@ -611,9 +613,9 @@ def run_ours(args, rank, world, dev):
                                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
                                     "peak_source": peaks["source"], "algorithmic_bytes": cb, "ms": per_call_ms["compact"]}
         if "project" in per_call_ms:
-            kf = 2.0 * sh.batch * sh.seq * sh.hidden * 2 * sh.kvh * sh.head_dim
+            kf = 2.0 * sh.batch * sh.seq * sh.hidden * (2 * sh.kvh + sh.heads) * sh.head_dim
             tf = kf / (per_call_ms["project"] * 1e-3) / 1e12
-            rooflines["project"] = {"bound": "tensor", "kernel": "ag_kv_project_cache", "achieved": tf,
+            rooflines["project"] = {"bound": "tensor", "kernel": "ag_qkv_project_cache", "achieved": tf,
                                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
                                     "traffic": None, "peak_source": peaks["source"], "algorithmic_flops": kf,
                                     "ms": per_call_ms["project"]}
@@ -724,7 +726,8 @@ def oracle_sample(name, seed, n_heads_sample=2, decode_steps=2):
     t_gate += time.perf_counter() - t0
     fl = flags[:, :hs]
     t0 = time.perf_counter()
-    if name == "prefill7b_proj":                 # the layer owns its key/value projection (Eq. 2)
+    if name == "prefill7b_proj":                 # the layer owns its projection (Eq. 2)
+        Qd = orc.project_q(Xd, f64(Wsub["Wq"]), hs)
         Kd, Vd = orc.project_kv(Xd, f64(Wsub["Wk"]), f64(Wsub["Wv"]), hs)
     cache = orc.compact_kv(Kd, Vd, fl)
     O = orc.prefill_attention(Qd, Kd, Vd, fl)
