@@ -295,16 +295,25 @@ class LayerRun:
         # attention + conditional append of the step in one call
         ag.ag_decode_step(self.desc, q, kn, vn, fn, self.cache, 0.0, self.o, self.status, self.ws[ag.AG_CALL_DECODE])
 
-    def step(self, ev=None):
-        """One pass; ev (optional) = dict of lists of (start, end) CUDA events per call."""
+    def step(self, ev=None, start=None):
+        """One pass; ev (optional) = dict of lists of (start, end) CUDA events per call.  The calls of a
+        pass run back to back on one stream, so the end mark of a call is the start mark of the next
+        (start = the event the caller recorded just before the pass): one event per call."""
+        chain = not self.first_gated                 # the guided stack runs its gates on a second stream
+        prev = [start if chain else None]
+
         def timed(key, fn, *a):
             if ev is None:
                 return fn(*a)
-            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            s.record()
+            s = prev[0]
+            if s is None:
+                s = torch.cuda.Event(enable_timing=True)
+                s.record()
             fn(*a)
+            e = torch.cuda.Event(enable_timing=True)
             e.record()
             ev[key].append((s, e))
+            prev[0] = e if chain else None
         if self.first_gated:
             return self._step_guided_by_previous_layer(timed)
         for layer in range(self.layers):
@@ -460,7 +469,7 @@ def run_ours(args, rank, world, dev):
         flush_l2(l2buf)
         s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s.record()
-        run.step(ev)
+        run.step(ev, s)
         e.record()
         step_ev.append((s, e))
     barrier()
