@@ -510,7 +510,9 @@ def run_ours(args, rank, world, dev):
         s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
         n_dq = len(dev_in) - 4
         # head groups of the pipelined copies: the heads of a sequence are contiguous only when batch = 1
-        n_groups = 4 if (sh.batch == 1 and sh.kv_heads == 0 and sh.heads % 4 == 0 and sh.recent_window <= 1) else 1
+        hg = sh.heads // 4                       # heads per group; every group's slices must start on 16-byte boundaries
+        n_groups = 4 if (sh.batch == 1 and sh.kv_heads == 0 and sh.heads % 4 == 0 and sh.recent_window <= 1
+                         and (hg * (sh.seq + 1) * 4) % 16 == 0 and (hg * sh.seq) % 16 == 0) else 1
         groups = [(g * sh.heads // n_groups, (g + 1) * sh.heads // n_groups) for g in range(n_groups)]
     O_step = run.O.clone() if run.has_prefill else None      # what the device-resident steps produced
     barrier()
@@ -571,7 +573,8 @@ def run_ours(args, rank, world, dev):
                 # compaction and prefill attention of a head group as soon as its K, V, Q are in; its O
                 # goes back while the next groups are still coming in (the link carries both directions)
                 main.wait_event(ready[1 + gi])
-                run.compact(g); run.prefill(g)
+                gg = g if n_groups > 1 else None
+                run.compact(gg); run.prefill(gg)
                 o_done = torch.cuda.Event(); o_done.record(main)
                 with torch.cuda.stream(s_out):
                     s_out.wait_event(o_done)
