@@ -97,7 +97,7 @@ compact_kernel(const uint8_t *__restrict__ flags, int n, const int32_t *__restri
   const uint8_t *Vs = V + (size_t)slab * n * kRowBytes;
   const size_t dst0 = ((size_t)row_off[slab] + before) * kRowBytes;
   // kFlight rows of K and of V per group in flight
-  constexpr int kFlight = 2;
+  constexpr int kFlight = 4;
   for (int j = g; j < count; j += kFlight * kGroups) {
     uint4 kv[kFlight], vv[kFlight];
 #pragma unroll
