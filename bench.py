@@ -49,8 +49,8 @@ WORKLOADS = {
 TRAFFIC = {
     ("prefill7b", "prefill"): 154.86e6 + 18.50e6,        # prefill_tc_kernel
     ("prefill7b", "decode"): 41.22e6 + 0.003e6,          # decode_cluster_mma_kernel
-    ("prefill7b", "compact"): 41.26e6 + 3.10e6,          # compact_kernel<256> (written rows still in L2 at kernel end)
-    ("prefill7b", "kv_project_cache"): 171.96e6 + 80.44e6,   # kv_proj_cache_kernel<256, 2>
+    ("prefill7b", "compact"): 41.26e6 + 2.46e6,          # compact_kernel<256> (written rows still in L2 at kernel end)
+    ("prefill7b", "kv_project_cache"): 179.50e6 + 82.40e6,   # kv_proj_cache_kernel<256, 2>
     ("prefill7b_proj", "prefill"): 154.86e6 + 18.50e6,
     ("prefill7b_proj", "decode"): 41.22e6 + 0.003e6,
     ("decode_ragged", "decode"): 2.3530e9 + 7.1e6,       # decode_partial_kernel<bf16,128>
