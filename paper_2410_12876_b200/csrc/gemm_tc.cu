@@ -5,7 +5,7 @@
 // One CTA computes MT (1 or 2) sub-tiles of 128 rows x BN columns (BN = 128, 192 or 256) of the packed output - or, for the tiles of a last wave that
 // would fill less than half of the SMs, one half of it (each such tile goes to two CTAs of
 // BN / 2 columns, so that the wave ends in about half the time).  Warp 0 drives TMA,
-// warp 1 owns TMEM and issues the MMAs, warps 2..5 drain the accumulator: the
+// warp 1 owns TMEM and issues the MMAs, warps 2..9 drain the accumulator (two per quarter of its lanes): the
 // float32 form straight to global memory, the hi / lo bf16 form through the
 // (by then free) operand stages and TMA stores, which write whole 128-byte lines.
 //   A = X   [M, K]  row-major  -> K-major operand, 128-byte swizzled rows
@@ -19,7 +19,7 @@ namespace ag {
 
 using namespace umma;
 
-constexpr int kTcBM = 128, kTcBK = 64, kTcThreads = 192;
+constexpr int kTcBM = 128, kTcBK = 64, kTcThreads = 320;   // warps: TMA, MMA, 8 x epilogue
 
 // MT: 128-row sub-tiles of A per CTA (1 or 2; two share every B stage, a third less traffic per FLOP).
 template <int BN, int MT> struct GemmTcCfg {
@@ -124,8 +124,10 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (elect_one()) mma_commit(acc_full);   // accumulator complete (or unwinding)
     __syncwarp();
   } else {
-    // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32)
-    const int quad = warp & 3;
+    // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32); warps 2..5 drain the first half of
+    // the tile's columns, warps 6..9 the second
+    const int quad = warp & 3, half = (warp - 2) >> 2;
+    const int c_begin = half * (bn / 2), c_end = c_begin + bn / 2;      // bn / 2 is a multiple of 32
     const bool ok = mbar_wait(acc_full, 0);
     tc_fence_after_sync();
 #pragma unroll 1
@@ -141,7 +143,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int r_in = quad * 32 + lane;
       uint8_t *stage_lo = smem + (BN / 64) * kTcBM * 128;
 #pragma unroll 1
-      for (int c = 0; c < bn; c += 32) {
+      for (int c = c_begin; c < c_end; c += 32) {
         uint32_t r[32];
         tmem_ld_x32_sync(tmem_sub + ((uint32_t)(quad * 32) << 16) + c, r);
         const uint32_t panel = (uint32_t)(c >> 6) * kTcBM * 128 + r_in * 128;
@@ -163,7 +165,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
       fence_proxy_async_smem();
-      named_barrier_sync(1, 128);
+      named_barrier_sync(1, 256);
       if (threadIdx.x == 64) {
         for (int p = 0; p < bn / 64; ++p) {            // rows past M are dropped by the tensor map
           tma_store_2d(&tmChi, smem + p * kTcBM * 128, n0 + p * 64, m0 + mt * kTcBM);
@@ -172,11 +174,11 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         tma_store_commit();
         tma_store_wait_read();
       }
-      if (MT > 1) named_barrier_sync(1, 128);          // the staging area is free for the next sub-tile
+      if (MT > 1) named_barrier_sync(1, 256);          // the staging area is free for the next sub-tile
     } else if (ok && num_kb > 0) {
       const size_t crow = (size_t)row * 3 * GD + n0;
 #pragma unroll 1
-      for (int c = 0; c < bn; c += 32) {
+      for (int c = c_begin; c < c_end; c += 32) {
         uint32_t r[32];
         tmem_ld_x32_sync(tmem_sub + ((uint32_t)(quad * 32) << 16) + c, r);
         if (row < M) {
