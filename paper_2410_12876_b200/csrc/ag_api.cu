@@ -134,7 +134,7 @@ int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk
   if (st) return st;
   if (desc->hidden <= 0) return AG_ERR_INVALID_ARG;
   if (!X || !Wk || !Wv || !flags || !prefix || !K || !V) return AG_ERR_INVALID_ARG;
-  st = check_cache(cache);
+  st = check_cache(cache, desc, true);
   if (st) return st;
   if (misaligned16(X) || misaligned16(Wk) || misaligned16(Wv) || misaligned16(K) || misaligned16(V) ||
       misaligned16(flags) || misaligned16(prefix) || misaligned16(idx))
@@ -151,7 +151,7 @@ int ag_qkv_project_cache(const ag_layer_desc *desc, const void *X, const void *W
   if (st) return st;
   if (desc->hidden <= 0) return AG_ERR_INVALID_ARG;
   if (!X || !Wq || !Wk || !Wv || !flags || !prefix || !Q || !K || !V) return AG_ERR_INVALID_ARG;
-  st = check_cache(cache);
+  st = check_cache(cache, desc, true);
   if (st) return st;
   if (misaligned16(X) || misaligned16(Wq) || misaligned16(Wk) || misaligned16(Wv) || misaligned16(Q) ||
       misaligned16(K) || misaligned16(V) || misaligned16(flags) || misaligned16(prefix) || misaligned16(idx))

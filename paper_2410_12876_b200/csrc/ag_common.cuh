@@ -90,6 +90,10 @@ int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wq, 
                          void *V, int32_t *dev_status, cudaStream_t st);
 int kv_proj_cache_wait_timeouts();
 
+// Fills the ring of a recent-token window (no-op without one) from the dense K, V of the prompt.
+int launch_recent_fill(const ag_layer_desc &d, const void *K, const void *V, const uint8_t *flags, const ag_cache &c,
+                       cudaStream_t st);
+
 size_t prefill_workspace_bytes(const ag_layer_desc &d);
 int launch_prefill(const ag_layer_desc &d, const void *Q, const void *K, const void *V,
                    const uint8_t *flags, const ag_cache &c, const int32_t *prefix, float scale,

@@ -207,15 +207,25 @@ int launch_compact(const ag_layer_desc &d, const void *K, const void *V, const u
   }
   AG_LAUNCH_CHECK();
   const RecentRing ring = ring_of(d, c);
-  if (K && ring.R > 0) {
-    const int threads = ring.R * (row_bytes(d) / 16);
-    switch (row_bytes(d)) {
-      case 128: recent_fill_kernel<128><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
-      case 256: recent_fill_kernel<256><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
-      default: recent_fill_kernel<512><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
-    }
-    AG_LAUNCH_CHECK();
+  if (K && ring.R > 0) return launch_recent_fill(d, K, V, flags, c, st);
+  return AG_OK;
+}
+
+// Ring of a recent-token window from the dense K, V of the prompt (one more small launch).
+int launch_recent_fill(const ag_layer_desc &d, const void *K, const void *V, const uint8_t *flags, const ag_cache &c,
+                       cudaStream_t st) {
+  const RecentRing ring = ring_of(d, c);
+  if (ring.R == 0) return AG_OK;
+  const int slabs = d.batch * kv_heads_of(d);
+  auto Kb = static_cast<const uint8_t *>(K);
+  auto Vb = static_cast<const uint8_t *>(V);
+  const int threads = ring.R * (row_bytes(d) / 16);
+  switch (row_bytes(d)) {
+    case 128: recent_fill_kernel<128><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
+    case 256: recent_fill_kernel<256><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
+    default: recent_fill_kernel<512><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
   }
+  AG_LAUNCH_CHECK();
   return AG_OK;
 }
 

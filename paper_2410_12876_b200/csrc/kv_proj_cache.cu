@@ -321,7 +321,7 @@ int run(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, c
 
 bool kv_proj_cache_supported(const ag_layer_desc &d) {
   return d.dtype == AG_BF16 && d.head_dim == kD && d.seq % kBM == 0 && d.hidden > 0 && d.hidden % 8 == 0 &&
-         recent_rows(d) == 0 && (int64_t)d.batch * d.seq < ((int64_t)1 << 31);
+         (int64_t)d.batch * d.seq < ((int64_t)1 << 31);
 }
 
 int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, const void *Wv,
@@ -329,12 +329,17 @@ int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wq, 
                          void *V, int32_t *dev_status, cudaStream_t st) {
   const int hk = kv_heads_of(d), hq = Wq ? d.heads : 0;
   const long long tiles128 = (long long)(2 * hk + hq) * (d.batch * (long long)d.seq / kBM);
+  int rc;
   if (hk % 2 == 0 && hq % 2 == 0) {
     // more than one wave: 256-token tiles, whose two sub-tiles share every stage of W
-    if (tiles128 > 2 * sm_count()) return run<256, 2>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
-    return run<256, 1>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
+    if (tiles128 > 2 * sm_count()) rc = run<256, 2>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
+    else rc = run<256, 1>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
+  } else {
+    rc = run<128, 1>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
   }
-  return run<128, 1>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
+  if (rc) return rc;
+  // recent-token window: the ring takes the prompt's last tokens from the dense K, V just written
+  return launch_recent_fill(d, K, V, flags, c, st);
 }
 
 int kv_proj_cache_wait_timeouts() {

@@ -163,6 +163,36 @@ def test_feeds_prefill_and_decode():
     T.check_close(T.f64(o), ref, "bf16", "decode after the fused projection")
 
 
+@pytest.mark.parametrize("w", [5, 10])
+def test_recent_window_ring_filled_by_the_projection(w):
+    """With a recent-token window the call leaves the ring as compaction leaves it: ring contents against
+    the oracle's list, then prefill under the band mask and decode steps that read and move the ring."""
+    shape = LayerShape(2, 256, 256, 4, 128, 2, 128, "bf16", recent_window=w)
+    R = w - 1
+    X = inputs.hidden_states(shape, 950 + w, DEV)
+    W = inputs.layer_weights(shape, 960 + w, DEV)
+    fl = _flags(shape, 970 + w)
+    flags = torch.from_numpy(fl).to(DEV)
+    steps = w + 2
+    cache, prefix, idx, status, K, V, Q = gpu_project_cache(shape, X, W, flags, [shape.seq + steps] * 8, with_q=True)
+    obits = orc.compact_kv(T.bits(K), T.bits(V), fl, window=w)          # the oracle's ring of the rows the call wrote
+    live = cache.recent_live.cpu().numpy()
+    rk = T.bits(cache.recent_k)
+    got = [sorted(rk[s, r].tobytes() for r in range(R) if live[s, r]) for s in range(live.shape[0])]
+    want = [sorted(np.ascontiguousarray(k).tobytes() for k, _, f in c["recent"] if f == 0) for row in obits for c in row]
+    assert got == want
+    assert np.array_equal(cache.pos.cpu().numpy(), np.full(8, shape.seq))
+    O = T.gpu_prefill(shape, Q, K, V, flags, cache, prefix)
+    T.check_close(T.f64(O), orc.prefill_attention(T.f64(Q), T.f64(K), T.f64(V), fl, window=w), "bf16", "prefill")
+    ocache = orc.compact_kv(T.f64(K), T.f64(V), fl, window=w)
+    for s in range(steps):
+        q, kn, vn, fn = inputs.decode_inputs(shape, 980 + w, s, DEV, keep_new=0.4)
+        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status, fused=True)
+        T.check_close(T.f64(o), orc.decode_attention(T.f64(q), T.f64(kn), T.f64(vn), ocache), "bf16", f"decode {s}")
+        orc.cache_append(ocache, T.f64(kn), T.f64(vn), fn.cpu().numpy(), window=w)
+    assert int(status.item()) == 0
+
+
 def test_full_size_layer_sampled():
     """The 7B-shaped layer in the launch configuration bench.py times: sampled dense rows against the
     oracle, lengths and every cached row against the flags."""
@@ -200,7 +230,7 @@ def test_rejects_what_it_has_no_kernel_for():
     flags = torch.ones(shape.batch, shape.kvh, shape.seq, dtype=torch.uint8, device=DEV)
     cache, prefix, idx, status, K, V = gpu_project_cache(shape, X, W, flags)
     for bad in (shape.with_(seq=200), shape.with_(head_dim=64), shape.with_(dtype="f32"), shape.with_(hidden=516),
-                shape.with_(recent_window=5)):
+                shape.with_(recent_window=5)):              # the last one: a window, and a cache without a ring
         with pytest.raises(ag.AgError) as e:
             ag.ag_kv_project_cache(ag.make_desc(bad), X, W["Wk"], W["Wv"], flags, cache, prefix, idx, K, V, status)
         assert e.value.status in (ag.AG_ERR_UNSUPPORTED, ag.AG_ERR_INVALID_ARG)
