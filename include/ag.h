@@ -229,9 +229,9 @@ int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
  * ag_compact_kv.  The cache rows are bit copies of the dense K, V rows.
  * With a recent-token window the ring of the cache is filled from the dense K, V,
  * as ag_compact_kv fills it.
- * Needs no workspace.  Kernel coverage: bfloat16, head_dim 128, n a multiple of
- * 128, d a multiple of 8; anything else returns AG_ERR_UNSUPPORTED (project
- * with a GEMM of your own and call ag_compact_kv).
+ * Needs no workspace.  Kernel coverage: bfloat16, head_dim 128, d a multiple of 8,
+ * and n a multiple of 128 unless batch = 1 (any n); anything else returns
+ * AG_ERR_UNSUPPORTED (project with a GEMM of your own and call ag_compact_kv).
  * AG_ERR_INVALID_ARG for missing or misaligned (16-byte) pointers.
  */
 int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk,

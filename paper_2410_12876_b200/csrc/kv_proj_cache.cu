@@ -161,27 +161,38 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
     for (int mt = 0; mt < (half == 0 ? MT : 0); ++mt) {           // warps 2..5 only
       const int m_base = m0 + mt * kBM;
-      const int b = m_base / n, t0 = m_base % n, t = t0 + r_in;   // n is a multiple of 128: one sequence per sub-tile
+      // one sequence per sub-tile: n is a multiple of 128, or there is a single sequence (whose last
+      // sub-tile may reach past its end: those rows are skipped here and dropped by the TMA stores)
+      const int b = m_base / n, t0 = m_base % n, t = t0 + r_in;
 #pragma unroll
       for (int hh = 0; hh < Cfg::kHeads; ++hh) {
         long long d = -1;
         if (m_base < M && mt < mts && which != 2) {               // the same for all 128 threads
           const size_t slab = (size_t)b * kv_heads + nw / kD + hh;
           const uint8_t *f = flags + slab * n;
-          const uint4 *fv = reinterpret_cast<const uint4 *>(f);
           int before = 0, total = 0;
-          for (int x = r_in; x < n / 16; x += kBM) {
-            const uint4 w = ldg128(fv + x);
-            const int c = nonzero_bytes(w.x) + nonzero_bytes(w.y) + nonzero_bytes(w.z) + nonzero_bytes(w.w);
-            total += c;
-            if (x * 16 < t0) before += c;                         // t0 is a multiple of 16: a vector lies on one side
+          if ((n & 15) == 0) {                                      // flag rows start on 16-byte boundaries
+            const uint4 *fv = reinterpret_cast<const uint4 *>(f);
+            for (int x = r_in; x < n / 16; x += kBM) {
+              const uint4 w = ldg128(fv + x);
+              const int c = nonzero_bytes(w.x) + nonzero_bytes(w.y) + nonzero_bytes(w.z) + nonzero_bytes(w.w);
+              total += c;
+              if (x * 16 < t0) before += c;                         // t0 is a multiple of 16: a vector lies on one side
+            }
+          } else {
+            for (int x = r_in; x < n; x += kBM) {
+              const int c = f[x] != 0;
+              total += c;
+              if (x < t0) before += c;
+            }
           }
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) {
             before += __shfl_xor_sync(0xffffffffu, before, o);
             total += __shfl_xor_sync(0xffffffffu, total, o);
           }
-          const bool keep = f[t] != 0;
+          const bool in_seq = t < n;                                // a single sequence may end inside its last sub-tile
+          const bool keep = in_seq && f[t] != 0;
           const unsigned word = __ballot_sync(0xffffffffu, keep);
           const int in_warp = __popc(word & ((1u << lane) - 1u));
           if (lane == 0) { red[quad] = before; red[4 + quad] = total; red[8 + quad] = __popc(word); }
@@ -195,7 +206,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           const int p = before + excl + in_warp;                  // rank within the slab
           const bool fits = total <= cap[slab];
           if (fits && keep) d = row_off[slab] + p;
-          if (which == 0) {
+          if (which == 0 && in_seq) {
             int32_t *pre = prefix + slab * (n + 1);
             pre[t] = p;
             if (keep && idx) idx[slab * n + p] = t;
@@ -320,7 +331,7 @@ int run(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, c
 }  // namespace
 
 bool kv_proj_cache_supported(const ag_layer_desc &d) {
-  return d.dtype == AG_BF16 && d.head_dim == kD && d.seq % kBM == 0 && d.hidden > 0 && d.hidden % 8 == 0 &&
+  return d.dtype == AG_BF16 && d.head_dim == kD && (d.seq % kBM == 0 || d.batch == 1) && d.hidden > 0 && d.hidden % 8 == 0 &&
          (int64_t)d.batch * d.seq < ((int64_t)1 << 31);
 }
 

@@ -122,6 +122,9 @@ CASES = {
     "split_last_wave": LayerShape(1, 2560, 128, 16, 128, 2, 128, "bf16"),      # 160 tiles on 148 SMs: 12 are split
     "split_last_wave_odd_rows": LayerShape(1, 2432, 128, 16, 128, 2, 128, "bf16"),
     "grouped_query": LayerShape(2, 256, 256, 8, 128, 2, 128, "bf16", kv_heads=2),
+    "one_sequence_ragged_end": LayerShape(1, 333, 256, 4, 128, 2, 128, "bf16"),      # n not a multiple of 16
+    "one_sequence_short": LayerShape(1, 48, 128, 6, 128, 2, 128, "bf16"),            # less than one tile
+    "one_sequence_long_ragged": LayerShape(1, 2500, 128, 16, 128, 2, 128, "bf16"),   # split last wave, ragged end
 }
 
 
@@ -131,7 +134,7 @@ def test_projection_and_cache(name):
 
 
 @pytest.mark.parametrize("name", ["two_heads_per_tile", "k_tail", "odd_heads", "subtiles_of_two_sequences",
-                                  "split_last_wave_odd_rows", "grouped_query"])
+                                  "split_last_wave_odd_rows", "grouped_query", "one_sequence_ragged_end"])
 def test_projection_with_queries(name):
     """ag_qkv_project_cache: Q against the oracle's query projection, K, V and the cache as without it."""
     _check(CASES[name], 940, with_q=True)
@@ -229,7 +232,8 @@ def test_rejects_what_it_has_no_kernel_for():
     W = inputs.layer_weights(shape, 2, DEV)
     flags = torch.ones(shape.batch, shape.kvh, shape.seq, dtype=torch.uint8, device=DEV)
     cache, prefix, idx, status, K, V = gpu_project_cache(shape, X, W, flags)
-    for bad in (shape.with_(seq=200), shape.with_(head_dim=64), shape.with_(dtype="f32"), shape.with_(hidden=516),
+    for bad in (shape.with_(seq=200), shape.with_(head_dim=64),             # seq 200 with batch 2: sub-tiles would straddle sequences
+                shape.with_(dtype="f32"), shape.with_(hidden=516),
                 shape.with_(recent_window=5)):              # the last one: a window, and a cache without a ring
         with pytest.raises(ag.AgError) as e:
             ag.ag_kv_project_cache(ag.make_desc(bad), X, W["Wk"], W["Wv"], flags, cache, prefix, idx, K, V, status)
