@@ -94,6 +94,26 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert lib.ag_decode_attn(byref(d), p, p, p, byref(c), float("inf"), p, p, 1 << 30, None) == ag.AG_ERR_INVALID_ARG
 
 
+def test_projection_calls_reject_on_the_host(lib):
+    """ag_kv_project_cache / ag_qkv_project_cache: argument checks and kernel coverage, nothing launched."""
+    p = 4096
+    byref = ctypes.byref
+    c = _cache_struct()
+    ok = ag.make_desc(inputs.LayerShape(2, 256, 512, 4, 128, 2, 128, "bf16"))
+    kv = lambda d, X=p, Wk=p, Wv=p, fl=p, pre=p, K=p, V=p: lib.ag_kv_project_cache(
+        byref(d), X, Wk, Wv, fl, byref(c), pre, None, K, V, None, None)
+    assert kv(ok, X=None) == ag.AG_ERR_INVALID_ARG
+    assert kv(ok, V=None) == ag.AG_ERR_INVALID_ARG
+    assert kv(ok, pre=None) == ag.AG_ERR_INVALID_ARG
+    assert kv(ok, Wk=p + 2) == ag.AG_ERR_INVALID_ARG
+    assert kv(ag.make_desc(inputs.TINY)) == ag.AG_ERR_UNSUPPORTED                                      # float32, head_dim 64
+    assert kv(ag.make_desc(inputs.LayerShape(2, 200, 512, 4, 128, 2, 128, "bf16"))) == ag.AG_ERR_UNSUPPORTED   # two sequences, n % 128 != 0
+    assert kv(ag.make_desc(inputs.LayerShape(2, 256, 516, 4, 128, 2, 128, "bf16"))) == ag.AG_ERR_UNSUPPORTED   # rows of X not 16-byte multiples
+    assert kv(ag.make_desc(inputs.LayerShape(2, 256, 512, 4, 128, 2, 128, "bf16", recent_window=5))) == ag.AG_ERR_INVALID_ARG  # no ring
+    assert lib.ag_qkv_project_cache(byref(ok), p, None, p, p, p, byref(c), p, None, p, p, p, None, None) == ag.AG_ERR_INVALID_ARG
+    assert lib.ag_qkv_project_cache(byref(ok), p, p, p, p, p, byref(c), p, None, None, p, p, None, None) == ag.AG_ERR_INVALID_ARG
+
+
 def test_binding_raises_with_status(lib):
     d = ag.make_desc(inputs.TINY.with_(gate_heads=7))
     with pytest.raises(ag.AgError) as e:
