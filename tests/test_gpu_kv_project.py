@@ -122,6 +122,8 @@ CASES = {
     "split_last_wave": LayerShape(1, 2560, 128, 16, 128, 2, 128, "bf16"),      # 160 tiles on 148 SMs: 12 are split
     "split_last_wave_odd_rows": LayerShape(1, 2432, 128, 16, 128, 2, 128, "bf16"),
     "grouped_query": LayerShape(2, 256, 256, 8, 128, 2, 128, "bf16", kv_heads=2),
+    "three_bands_of_row_tiles": LayerShape(1, 4864, 128, 2, 128, 1, 128, "bf16"),    # 38 row tiles: bands of 16, 16, 6
+    "two_bands_of_256_row_tiles": LayerShape(2, 2432, 128, 8, 128, 2, 128, "bf16"),  # 19 row tiles: bands of 16 and 3, split last wave
     "one_sequence_ragged_end": LayerShape(1, 333, 256, 4, 128, 2, 128, "bf16"),      # n not a multiple of 16
     "one_sequence_short": LayerShape(1, 48, 128, 6, 128, 2, 128, "bf16"),            # less than one tile
     "one_sequence_long_ragged": LayerShape(1, 2500, 128, 16, 128, 2, 128, "bf16"),   # split last wave, ragged end
