@@ -198,27 +198,31 @@ def test_recent_window_ring_filled_by_the_projection(w):
     assert int(status.item()) == 0
 
 
-def test_full_size_layer_sampled():
-    """The 7B-shaped layer in the launch configuration bench.py times: sampled dense rows against the
-    oracle, lengths and every cached row against the flags."""
+@pytest.mark.parametrize("with_q", [False, True])
+def test_full_size_layer_sampled(with_q):
+    """The 7B-shaped layer in the launch configurations bench.py times (keys and values; queries, keys and
+    values): sampled dense rows against the oracle, lengths and every cached row against the flags."""
     shape = inputs.PREFILL7B
     X = inputs.hidden_states(shape, 2000, DEV)
     W = inputs.layer_weights(shape, 2010, DEV)
     fl = _flags(shape, 930)
     flags = torch.from_numpy(fl).to(DEV)
-    cache, prefix, idx, status, K, V = gpu_project_cache(shape, X, W, flags)
+    cache, prefix, idx, status, K, V, Q = gpu_project_cache(shape, X, W, flags, with_q=with_q)[:7] if with_q else \
+        (*gpu_project_cache(shape, X, W, flags), None)
     assert int(status.item()) == 0
     L = fl.sum(axis=2, dtype=np.int64).reshape(-1)
     assert np.array_equal(cache.len.cpu().numpy(), L)
     want = np.concatenate([np.zeros((1, shape.heads, 1), dtype=np.int64), np.cumsum(fl, axis=2, dtype=np.int64)], axis=2)
     assert np.array_equal(prefix.cpu().numpy(), want)
-    Xf, Wk, Wv = T.f64(X)[0], T.f64(W["Wk"]), T.f64(W["Wv"])
+    Xf, Wk, Wv, Wq = T.f64(X)[0], T.f64(W["Wk"]), T.f64(W["Wv"]), T.f64(W["Wq"])
     rng = np.random.default_rng(931)
     D = shape.head_dim
     for i in range(shape.heads):
         rows = np.unique(np.concatenate([[0, 127, 128, shape.seq - 1], rng.integers(0, shape.seq, 12)]))
         _close_to_rounded(T.f64(K[0, i][torch.from_numpy(rows).to(DEV)]), Xf[rows] @ Wk[:, i * D:(i + 1) * D], "K")
         _close_to_rounded(T.f64(V[0, i][torch.from_numpy(rows).to(DEV)]), Xf[rows] @ Wv[:, i * D:(i + 1) * D], "V")
+        if with_q:
+            _close_to_rounded(T.f64(Q[0, i][torch.from_numpy(rows).to(DEV)]), Xf[rows] @ Wq[:, i * D:(i + 1) * D], "Q")
     off = cache.row_off.cpu().numpy()
     kd, vd, kr, vr = T.bits(K), T.bits(V), T.bits(cache.k_rows), T.bits(cache.v_rows)
     for i in range(shape.heads):
