@@ -11,7 +11,7 @@ void set_last_cuda_error(int e) { g_last_cuda_error = e; }
 static bool dim_ok(int d) { return d == 64 || d == 128; }
 
 // Checks of the fields every call uses.
-static int check_desc(const ag_layer_desc *d) {
+int check_desc(const ag_layer_desc *d) {
   if (!d) return AG_ERR_INVALID_ARG;
   if (d->batch <= 0 || d->seq <= 0 || d->heads <= 0) return AG_ERR_INVALID_ARG;
   if (d->dtype != AG_F32 && d->dtype != AG_BF16) return AG_ERR_INVALID_ARG;
@@ -38,7 +38,7 @@ static int check_gate_desc(const ag_layer_desc *d) {
 }
 
 // need_recent: the call reads or writes the ring of recent tokens (compaction, decode, append).
-static int check_cache(const ag_cache *c, const ag_layer_desc *d = nullptr, bool need_recent = false) {
+int check_cache(const ag_cache *c, const ag_layer_desc *d, bool need_recent) {
   if (!c) return AG_ERR_INVALID_ARG;
   if (need_recent && d && recent_rows(*d) > 0) {
     if (!c->recent_k || !c->recent_v || !c->recent_live || !c->pos) return AG_ERR_INVALID_ARG;

@@ -51,6 +51,12 @@ inline RecentRing ring_of(const ag_layer_desc &d, const ag_cache &c) {
 }
 inline bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
+// Host-side argument checks shared by every entry point (ag_api.cu): the descriptor fields all calls
+// use (sizes, dtype, head_dim, the key/value head grouping, the recent-token window) and the cache
+// struct (need_recent: the call reads or writes the ring of recent tokens).
+int check_desc(const ag_layer_desc *d);
+int check_cache(const ag_cache *c, const ag_layer_desc *d = nullptr, bool need_recent = false);
+
 // Per-step launchers (defined in the kernel files, called from ag_api.cu).
 size_t gate_workspace_bytes(const ag_layer_desc &d);
 int launch_gate(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk,

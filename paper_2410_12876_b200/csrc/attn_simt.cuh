@@ -32,6 +32,7 @@ struct SimtAttnArgs {
   const void *k_rows, *v_rows;         // compacted cache pools
   const int64_t *row_off;
   const int32_t *prefix;               // [problems, n + 1]
+  const int32_t *len;                  // [problems] valid rows of each slab: a row bound never exceeds it
   float *lse;                          // NULL, or [problems, n]: m + log2(l) of every row
   // kGateFull only: [batch] keys each sequence has (the rest is padding), or NULL = n
   const int32_t *seq_lens;
@@ -77,6 +78,9 @@ simt_attn_kernel(const SimtAttnArgs a) {
     kp_row = D; vp_row = D;
   }
   const int32_t *pre = MODE == kPrefill ? a.prefix + (size_t)prob_kv * (a.n + 1) : nullptr;
+  // a slab that overflowed at compaction holds no rows (len = 0) although its prefix counts are
+  // full: its queries then see themselves only, and no read leaves the slab
+  const int slab_len = MODE == kPrefill ? a.len[prob_kv] : 0;
   const int n_keys = (MODE == kGateFull && a.seq_lens) ? a.seq_lens[prob / a.inner] : a.n;
 
   // Q tile -> shared (rows past n are clamped; they are never stored)
@@ -96,11 +100,11 @@ simt_attn_kernel(const SimtAttnArgs a) {
     const int j = j0 + ty * 4 + r;
     valid[r] = j < a.n;
     const int jc = min(j, a.n - 1);
-    bound[r] = MODE == kGateCausal ? jc + 1 : (MODE == kGateFull ? n_keys : pre[jc]);
+    bound[r] = MODE == kGateCausal ? jc + 1 : (MODE == kGateFull ? n_keys : min(pre[jc], slab_len));
     if (!valid[r]) bound[r] = 0;
   }
   const int j_last = min(j0 + kSimtBM, a.n) - 1;
-  const int max_bound = MODE == kGateCausal ? j_last + 1 : (MODE == kGateFull ? n_keys : pre[j_last]);
+  const int max_bound = MODE == kGateCausal ? j_last + 1 : (MODE == kGateFull ? n_keys : min(pre[j_last], slab_len));
   const int n_tiles = (max_bound + kSimtBN - 1) / kSimtBN;
 
   float m[4], l[4], o[4][kOC][4];

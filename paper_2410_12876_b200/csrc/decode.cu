@@ -315,7 +315,7 @@ decode_partial_gqa_kernel(const T *__restrict__ q, const T *__restrict__ k_rows,
 template <typename T, int D>
 __global__ void __launch_bounds__(D)
 decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
-                      const T *__restrict__ v_new, const int32_t *__restrict__ len,
+                      const T *__restrict__ v_new, const int32_t *len,
                       float scale_log2, int chunk_rows, const float *__restrict__ part_o,
                       const float *__restrict__ part_ml, T *__restrict__ o,
                       const int64_t *__restrict__ row_off, const AppendArgs ap, const HeadMap hm,
@@ -323,9 +323,6 @@ decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
   const int slab = blockIdx.x, d = threadIdx.x;
   const int kv = hm.kv_slab(slab);
   const int L = len[kv];
-  // the chunk pass, the only reader of the slab's rows, has completed: the new row may go in
-  // (never asked for when query heads share a slab: another head's CTA may still be reading its length)
-  append_new_row<T, D>(ap, kv, L, row_off[kv], k_new, v_new);
   const int n_chunks = (L + chunk_rows - 1) / chunk_rows;
   __shared__ float red[D / 32];
   __shared__ float ring_s[kMaxRecent];
@@ -335,6 +332,10 @@ decode_combine_kernel(const T *__restrict__ q, const T *__restrict__ k_new,
   if ((d & 31) == 0) red[d >> 5] = a;
   ring_scores<T, D>(rg, kv, q + (size_t)slab * D, scale_log2, ring_s);
   __syncthreads();
+  // Every thread of the CTA has read the slab's length (above the barrier), and the chunk pass, the
+  // only reader of the slab's rows, has completed: the new row may go in and the length may move.
+  // (Never asked for when query heads share a slab: another head's CTA may still be reading its length.)
+  append_new_row<T, D>(ap, kv, L, row_off[kv], k_new, v_new);
   float s_self = 0.f;
 #pragma unroll
   for (int i = 0; i < D / 32; ++i) s_self += red[i];
@@ -380,7 +381,7 @@ template <typename T, int D, int kThreads>
 __global__ void __launch_bounds__(kThreads)
 decode_cluster_kernel(const T *__restrict__ q, const T *__restrict__ k_new, const T *__restrict__ v_new,
                       const T *__restrict__ k_rows, const T *__restrict__ v_rows,
-                      const int64_t *__restrict__ row_off, const int32_t *__restrict__ len,
+                      const int64_t *__restrict__ row_off, const int32_t *len,
                       float scale_log2, T *__restrict__ out, const AppendArgs ap, const HeadMap hm,
                       const RecentRing rg) {
   namespace cg = cooperative_groups;
@@ -505,7 +506,7 @@ __global__ void __launch_bounds__(kGqThreads, 2)
 decode_cluster_mma_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_new,
                           const __nv_bfloat16 *__restrict__ v_new, const __nv_bfloat16 *__restrict__ k_rows,
                           const __nv_bfloat16 *__restrict__ v_rows, const int64_t *__restrict__ row_off,
-                          const int32_t *__restrict__ len, float scale_log2, __nv_bfloat16 *__restrict__ out,
+                          const int32_t *len, float scale_log2, __nv_bfloat16 *__restrict__ out,
                           const AppendArgs ap, const HeadMap hm, const RecentRing rg) {
   namespace cg = cooperative_groups;
   using T = __nv_bfloat16;
@@ -768,25 +769,19 @@ extern "C" int ag_decode_attn_noalloc(const ag_layer_desc *desc, const void *q, 
                                       const void *v_new, const ag_cache *cache, float softmax_scale,
                                       void *o, void *cuda_stream) {
   using namespace ag;
-  if (!desc || !cache || !q || !k_new || !v_new || !o) return AG_ERR_INVALID_ARG;
-  if (desc->batch <= 0 || desc->heads <= 0 || desc->seq <= 0) return AG_ERR_INVALID_ARG;
-  if (desc->dtype != AG_F32 && desc->dtype != AG_BF16) return AG_ERR_INVALID_ARG;
-  if (desc->head_dim != 64 && desc->head_dim != 128) return AG_ERR_UNSUPPORTED;
-  if (desc->recent_window < 0) return AG_ERR_INVALID_ARG;
+  // the same host-side checks as ag_decode_attn, before anything is launched
+  int st = check_desc(desc);
+  if (st) return st;
+  if (!q || !k_new || !v_new || !o) return AG_ERR_INVALID_ARG;
   if (desc->recent_window > 1) return AG_ERR_UNSUPPORTED;     // this entry does not read the ring of recent tokens
-  if (!cache->row_off || !cache->cap || !cache->len || cache->pool_rows < 0 || cache->max_cap < 0)
-    return AG_ERR_INVALID_ARG;
-  if (cache->pool_rows > 0 && (!cache->k_rows || !cache->v_rows)) return AG_ERR_INVALID_ARG;
-  if (cache->max_cap > cache->pool_rows) return AG_ERR_CAPACITY;
-  if (misaligned16(q) || misaligned16(k_new) || misaligned16(v_new) || misaligned16(o) ||
-      misaligned16(cache->k_rows) || misaligned16(cache->v_rows))
-    return AG_ERR_INVALID_ARG;
+  st = check_cache(cache, desc, false);
+  if (st) return st;
+  if (misaligned16(q) || misaligned16(k_new) || misaligned16(v_new) || misaligned16(o)) return AG_ERR_INVALID_ARG;
   if (!(softmax_scale >= 0.f) || isinf(softmax_scale)) return AG_ERR_INVALID_ARG;
   // the fixed array bounds the problem size: refuse anything that would not fit
-  if ((int64_t)desc->batch * desc->heads > ((int64_t)1 << 24)) return AG_ERR_CAPACITY;
   if (decode_workspace_bytes(*desc) > kNoAllocScratchBytes) return AG_ERR_CAPACITY;
   void *scratch = nullptr;
-  int st = noalloc_scratch_ptr(&scratch);
+  st = noalloc_scratch_ptr(&scratch);
   if (st) return st;
   const float scale = softmax_scale == 0.f ? 1.0f / sqrtf((float)desc->head_dim) : softmax_scale;
   // Nothing in the scratch has to start at zero: every partial the merge step

@@ -47,6 +47,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   uint64_t *empty = full + Cfg::kStages;
   uint64_t *acc_full = empty + Cfg::kStages;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  int *gave_up = reinterpret_cast<int *>(tmem_slot + 1);   // set by an epilogue thread whose wait for the accumulator expired
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // CTAs below halved_from take whole tiles (row-major over the tile grid), the rest half tiles
@@ -62,6 +63,7 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(acc_full, 1);
+    *gave_up = 0;
     fence_barrier_init();
     prefetch_tensormap(&tmA);
     prefetch_tensormap(&tmB0);
@@ -128,7 +130,10 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // the tile's columns, warps 6..9 the second
     const int quad = warp & 3, half = (warp - 2) >> 2;
     const int c_begin = half * (bn / 2), c_end = c_begin + bn / 2;      // bn / 2 is a multiple of 32
-    const bool ok = mbar_wait(acc_full, 0);
+    // all eight warps agree on whether the accumulator arrived before any of them enters the barriers below
+    if (!mbar_wait(acc_full, 0)) *gave_up = 1;
+    named_barrier_sync(1, 256);
+    const bool ok = *gave_up == 0;
     tc_fence_after_sync();
 #pragma unroll 1
     for (int mt = 0; mt < MT; ++mt) {

@@ -65,6 +65,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
   long long *dst_row = reinterpret_cast<long long *>(smem + Cfg::kStages * Cfg::kStageBytes + 256);
   int *red = reinterpret_cast<int *>(smem + Cfg::kStages * Cfg::kStageBytes + 256 + Cfg::kDstBytes);   // 12 ints
+  int *gave_up = red + 12;                       // set by an epilogue thread whose wait for the accumulator expired
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // CTAs below split_from take whole tiles (row-major over the tile grid), the rest one sub-tile of a tile
@@ -90,6 +91,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(acc_full, 1);
+    *gave_up = 0;
     fence_barrier_init();
     prefetch_tensormap(&tmA);
     prefetch_tensormap(tmB);
@@ -220,7 +222,12 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         dst_row[(mt * Cfg::kHeads + hh) * kBM + r_in] = d;
       }
     }
-    const bool ok = mbar_wait(acc_full, 0);
+    // the eight warps start this wait at different times (warps 2..5 rank the tile's tokens first): if it
+    // expires for some of them only, all of them must still agree to leave, or the barriers below would
+    // wait for threads that have gone
+    if (!mbar_wait(acc_full, 0)) *gave_up = 1;
+    named_barrier_sync(1, 256);
+    const bool ok = *gave_up == 0;
     tc_fence_after_sync();
     const CUtensorMap *tmOut = which == 0 ? &tmK : (which == 1 ? &tmV : &tmQ);
     uint8_t *rows_out = which == 0 ? k_rows : v_rows;

@@ -96,7 +96,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int j0 = qt * kPfBM;
   const int j_last = min(j0 + kPfBM, a.n) - 1;
   const int32_t *pre = a.prefix + (size_t)kv_slab * (a.n + 1);
-  const int max_bound = pre[j_last];               // keys any row of this tile may see
+  // keys any row of this tile may see; never past the slab's valid rows (a slab that overflowed at
+  // compaction has len = 0 under full prefix counts: its queries see themselves only)
+  const int max_bound = min(pre[j_last], a.len[kv_slab]);
   const int n_kv = (max_bound + kPfBN - 1) / kPfBN;
   const int row0 = (int)a.row_off[kv_slab];
   static_assert(kPfKvBuf == kPfTile, "the self tile below spans exactly the two V stages");
@@ -250,8 +252,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int tid = threadIdx.x - 64;                // 0..127
     const int j = j0 + row;
     const bool valid = j < a.n;
-    const int bound = valid ? pre[j] : 0;
     const int L = a.len[kv_slab];
+    const int bound = valid ? min(pre[j], L) : 0;
     const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
     float m = 0.f, self2 = 0.f, l = 1.f;
     bool ok = true;

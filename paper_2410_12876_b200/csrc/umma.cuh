@@ -2,9 +2,9 @@
 // tensor-core kernels use: mbarriers, TMA tile loads, tensor memory (TMEM)
 // allocation, tcgen05.mma issue/commit and TMEM loads/stores.
 //
-// Every wait is bounded: a wait that does not complete within kWaitCycles sets
-// g_wait_expired and returns false so that the kernel can unwind (release TMEM,
-// return) instead of spinning forever.
+// Every wait is bounded: a wait that does not complete within kWaitCycles counts itself in
+// g_wait_expired, marks its own launch as giving up and returns false so that the kernel can
+// unwind (release TMEM, return) instead of spinning forever.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -14,9 +14,20 @@
 namespace ag {
 namespace umma {
 
-// Counts waits that gave up in the kernels of this translation unit (each .cu
-// that includes this header has its own copy and reports it to the host).
+// Counts waits that gave up in the kernels of this translation unit since the library was loaded
+// (each .cu that includes this header has its own copy and reports it to the host).  Never reset:
+// a caller compares the count before and after the launches it cares about.
 static __device__ int g_wait_expired = 0;
+// The launch (its %gridid, unique per launch in a context) in which a wait last expired.  The other
+// waits of THAT launch give up quickly, so that a stuck launch drains in one time-out instead of one
+// per CTA; a later launch has another id and waits normally.
+static __device__ unsigned long long g_abort_grid = ~0ull;
+
+__device__ __forceinline__ unsigned long long this_grid_id() {
+  unsigned long long id;
+  asm volatile("mov.u64 %0, %%gridid;" : "=l"(id));
+  return id;
+}
 
 constexpr long long kWaitCycles = 4000000000LL;   // ~2 s at 2 GHz
 
@@ -60,21 +71,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait for the phase with the given parity to complete.  The poll loop
-// touches nothing but the barrier; the clock and the give-up flag are looked at
-// once every 1024 polls.  Once any wait of this translation unit has expired,
-// every later wait that blocks that long gives up too, so that a stuck launch
-// drains quickly instead of CTA by CTA.
+// touches nothing but the barrier; the clock and the give-up mark are looked at
+// once every 1024 polls.  Once a wait of this launch has expired, every other wait
+// of the same launch that blocks that long gives up too.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   uint32_t polls = 0;
   long long t0 = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++polls & 1023u) == 0) {
-      if (*reinterpret_cast<volatile int *>(&g_wait_expired) != 0) return false;
+      if (*reinterpret_cast<volatile unsigned long long *>(&g_abort_grid) == this_grid_id()) return false;
       const long long now = clock64();
       if (t0 == 0) t0 = now;
       else if (now - t0 > kWaitCycles) {
         atomicAdd(&g_wait_expired, 1);
+        atomicExch(&g_abort_grid, this_grid_id());
         return false;
       }
     }

@@ -115,6 +115,21 @@ def qkv_gaussian(shape, seed, device="cpu", std=1.0):
     return [randn(sq if k == 0 else skv, seed + k, device, shape.torch_dtype, std) for k in range(3)]
 
 
+def stack_layer_seed(seed, layer):
+    """Seed base of layer `layer` of a stack: every layer has its own hidden states and weights."""
+    return int(seed) + 1000 * (int(layer) + 1)
+
+
+def stack_layer_inputs(shape, seed, layer, device="cpu"):
+    """Hidden states X_l ~ N(0, 1), weights ~ N(0, 0.02) and the upstream projections Q, K, V of one
+    layer of a stack, all seeded by the layer's number."""
+    base = stack_layer_seed(seed, layer)
+    X = hidden_states(shape, base, device)
+    W = layer_weights(shape, base + 10, device)
+    Q, K, V = project_qkv(shape, X, W)
+    return X, W, Q, K, V
+
+
 def keep_targets_uniform(heads, seed, lo=0.3, hi=0.8):
     """Per-head target keep rate ~ U[lo, hi]."""
     return np.random.default_rng(seed).uniform(lo, hi, size=heads)

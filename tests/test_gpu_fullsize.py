@@ -59,8 +59,11 @@ def test_prefill7b_layer():
     scores, flags = T.gpu_gate(shape, X, W, gamma)
     err = np.max(np.abs(T.f64(scores) - s_ref))
     assert err < 1e-4, err
+    # what carries flag parity is the score check above (every score within 1e-4 of the oracle's); the
+    # bit-exact comparison leaves out only the scores closer than 1e-3 to the threshold
     excluded = T.check_flags(shape, flags, s_ref, f_ref, gamma)
-    assert excluded < 0.1, excluded
+    print(f"prefill7b: max score error {err:.2e}, {100 * excluded:.3f} % of the flags inside the threshold band")
+    assert excluded < 0.05, excluded
     assert np.max(np.abs(f_ref.mean(axis=(0, 2)) - keep)) < 0.01
     # downstream calls run on the oracle's flags
     fl = torch.from_numpy(f_ref).to(DEV)
@@ -159,3 +162,88 @@ def test_ragged_decode():
         assert np.array_equal(T.f64(cache.k_rows[off[s]:off[s] + n_s]), ocache[int(s)]["k"])
         assert np.array_equal(T.f64(cache.v_rows[off[s]:off[s] + n_s]), ocache[int(s)]["v"])
     assert int(status.item()) == 0
+
+
+def test_gate_projection_in_256_row_tiles():
+    """A gate projection of more than one wave of tiles (5120 rows x 1536 columns): the GEMM then
+    takes 256 x 256 tiles over several waves with a halved last wave, the form the batch-8 stack
+    runs.  Small hidden size, so that the oracle evaluates every score of both sequences."""
+    shape = inputs.LayerShape(2, 2560, 128, 8, 128, 4, 128, "bf16")
+    seed = 5200
+    X = inputs.hidden_states(shape, seed, DEV)
+    W = inputs.layer_weights(shape, seed + 10, DEV)
+    W["Wo_g"] = inputs.randn(tuple(W["Wo_g"].shape), seed + 17, DEV, shape.torch_dtype, 0.5)
+    keep = inputs.keep_targets_uniform(shape.heads, seed + 20)
+    s0, _ = T.oracle_gate(shape, X, W, None)
+    gamma = inputs.calibrate_gamma(torch.from_numpy(s0), keep, shape.tau).to(DEV)
+    s_ref, f_ref = T.oracle_gate(shape, X, W, gamma)
+    for causal in (1, 0):
+        sh = shape.with_(gate_causal=causal)
+        if causal == 0:
+            s_ref, f_ref = T.oracle_gate(sh, X, W, gamma)
+        scores, flags = T.gpu_gate(sh, X, W, gamma)
+        err = np.max(np.abs(T.f64(scores) - s_ref))
+        assert err < 1e-4, (causal, err)
+        excluded = T.check_flags(sh, flags, s_ref, np.ascontiguousarray(f_ref), gamma)
+        print(f"gate {shape.batch} x {shape.seq}, causal={causal}: max score error {err:.2e}, "
+              f"{100 * excluded:.3f} % of the flags inside the threshold band")
+        assert excluded < 0.05, excluded
+    assert ag.ag_device_wait_timeouts() == 0
+
+
+@pytest.mark.parametrize("layer", [0, 10, 21, 31])
+def test_stack7b_layer(layer):
+    """One layer of the 32-layer stack at its size (batch 8 x 4096 tokens, its own hidden states,
+    weights and keep rates): the whole batch runs on the GPU in the launch configuration the stack
+    benchmark times; the oracle evaluates sequence 0 - every gate score and flag, compaction bit for
+    bit, sampled prefill rows of every head, four decode steps."""
+    shape = inputs.STACK7B
+    seed = 5000
+    B, h, n = shape.batch, shape.heads, shape.seq
+    X, W, Q, K, V = inputs.stack_layer_inputs(shape, seed, layer, DEV)
+    one = shape.with_(batch=1)
+    keep = inputs.keep_targets_layer(h, seed + 20, layer)
+    s0, _ = T.oracle_gate(one, X[:1], W, None)
+    gamma = inputs.calibrate_gamma(torch.from_numpy(s0), keep, shape.tau).to(DEV)
+    s_ref, f_ref = T.oracle_gate(one, X[:1], W, gamma)
+    f_ref = np.ascontiguousarray(f_ref)
+    scores, flags = T.gpu_gate(shape, X, W, gamma)
+    err = np.max(np.abs(T.f64(scores[:1]) - s_ref))
+    assert err < 1e-4, err
+    excluded = T.check_flags(one, flags[:1], s_ref, f_ref, gamma)
+    print(f"stack layer {layer}: max score error {err:.2e}, {100 * excluded:.3f} % of the flags inside the band, "
+          f"keep {f_ref.mean():.3f}")
+    assert excluded < 0.05, excluded
+    assert np.max(np.abs(f_ref.mean(axis=(0, 2)) - keep)) < 0.01
+    # the other sequences keep about what sequence 0 keeps (same weights, same gamma)
+    got_keep = flags.float().mean(dim=(1, 2)).cpu().numpy()
+    assert np.max(np.abs(got_keep - got_keep[0])) < 0.05, got_keep
+    # downstream: sequence 0 under the oracle's flags, the others under the GPU's
+    fl = flags.clone()
+    fl[0] = torch.from_numpy(f_ref[0]).to(DEV)
+    steps = 4
+    cache, prefix, idx, status = T.gpu_compact(shape, K, V, fl, cap=[n + steps] * (B * h))
+    T.check_compaction(one, K[:1], V[:1], fl[:1], _first_sequence(cache, h), prefix[:1], idx[:1])
+    f_all = fl.cpu().numpy()
+    assert np.array_equal(cache.len.cpu().numpy(), f_all.reshape(B * h, n).sum(axis=1))
+    assert torch.equal(prefix[:, :, -1].reshape(-1), cache.len)
+    O = T.gpu_prefill(shape, Q, K, V, fl, cache, prefix)
+    assert torch.isfinite(O.float()).all()
+    _check_prefill_rows(one, Q[:1], K[:1], V[:1], f_ref, O[:1], range(h), 192, 13 + layer)
+    ocache = orc.compact_kv(T.f64(K[:1]), T.f64(V[:1]), f_ref)
+    ws = ag.workspace(ag.make_desc(shape), ag.AG_CALL_DECODE)
+    for step in range(steps):
+        q, kn, vn, fn = inputs.decode_inputs(shape, seed + 500 + layer, step, DEV, keep_new=1.0)
+        o = T.gpu_decode_step(shape, q, kn, vn, fn, cache, status, ws=ws, fused=True)
+        assert torch.isfinite(o.float()).all()
+        T.check_close(T.f64(o[:1]), orc.decode_attention(T.f64(q[:1]), T.f64(kn[:1]), T.f64(vn[:1]), ocache),
+                      "bf16", f"layer {layer} decode {step}")
+        orc.cache_append(ocache, T.f64(kn[:1]), T.f64(vn[:1]), fn[:1].cpu().numpy())
+    assert np.array_equal(cache.len.cpu().numpy()[:h], orc.cache_lengths(ocache).reshape(-1))
+    assert int(status.item()) == 0 and ag.ag_device_wait_timeouts() == 0
+
+
+def _first_sequence(cache, heads):
+    """View of the slabs of sequence 0 of a device cache (same pools, first `heads` slabs)."""
+    return ag.RaggedCache(cache.k_rows, cache.v_rows, cache.row_off[:heads], cache.cap[:heads], cache.len[:heads],
+                          cache.max_cap)

@@ -128,6 +128,34 @@ def test_compaction_overflow_is_reported_not_written():
     assert torch.count_nonzero(cache.k_rows[off[1]:off[1] + 10]) == 0
 
 
+@pytest.mark.parametrize("name", ["bf16", "bf16_d64", "f32_d128"])
+def test_prefill_after_an_overflow_stays_inside_the_slab(name):
+    """The LAST slab of the pool is too small for its retained tokens: compaction leaves it empty
+    (len = 0, overflow bit) while its prefix counts stay full.  Prefill attention must then see the
+    slab as empty - each of its queries attends to itself only, O = V exactly - read nothing past the
+    end of the pool, and leave the other slabs as the oracle has them."""
+    shape = SHAPES[name].with_(batch=1, seq=300)
+    h, n = shape.heads, shape.seq
+    Q, K, V = inputs.qkv_gaussian(shape, 240, DEV)
+    f = inputs.bernoulli_flags((1, h, n), 0.5, 241).numpy()
+    L = f.reshape(h, n).sum(axis=1)
+    cap = L.copy()
+    cap[-1] = L[-1] - 1                                          # one row short
+    flags = torch.from_numpy(f).to(DEV)
+    cache, prefix, idx, status = T.gpu_compact(shape, K, V, flags, cap=cap.tolist())
+    assert int(status.item()) & ag.AG_DEV_OVERFLOW
+    want_len = L.copy()
+    want_len[-1] = 0
+    assert cache.len.cpu().tolist() == want_len.tolist()
+    O = T.gpu_prefill(shape, Q, K, V, flags, cache, prefix)
+    assert torch.equal(O[0, h - 1], V[0, h - 1])                 # the emptied slab: the diagonal only
+    # the oracle's view: that head evicts everything, the others are untouched
+    f_seen = f.copy()
+    f_seen[0, h - 1] = 0
+    O_ref = orc.prefill_attention(T.f64(Q), T.f64(K), T.f64(V), f_seen)
+    T.check_close(T.f64(O), O_ref, shape.dtype, "prefill after an overflow")
+
+
 @pytest.mark.parametrize("name", list(SHAPES))
 def test_prefill_attention(name):
     shape = SHAPES[name]
@@ -297,6 +325,30 @@ def test_decode_empty_cache_returns_own_value_and_full_slab_reports_overflow(fus
                for b in range(shape.batch)]
     o2_ref = orc.decode_attention(T.f64(q2), T.f64(kn2), T.f64(vn2), one_row)
     T.check_close(T.f64(o2), o2_ref, "bf16", "decode over one row")
+
+
+@pytest.mark.parametrize("name", ["bf16", "f32_d128"])
+def test_decode_from_a_cache_snapshot_repeats_bit_for_bit(name):
+    """The cache after prefill is the whole state of a layer: copied aside, restored and decoded from
+    again, it gives the same outputs and the same cache, bit for bit."""
+    shape = SHAPES[name].with_(seq=500)
+    Q, K, V = inputs.qkv_gaussian(shape, 620, DEV)
+    flags = _flag_patterns(shape, 621)
+    steps = 16
+    cap = [shape.seq + steps] * (shape.batch * shape.heads)
+    cache, prefix, idx, status = T.gpu_compact(shape, K, V, flags, cap=cap)
+    snap = (cache.k_rows.clone(), cache.v_rows.clone(), cache.len.clone())
+    runs = []
+    for _ in range(2):
+        cache.k_rows.copy_(snap[0]); cache.v_rows.copy_(snap[1]); cache.len.copy_(snap[2])
+        outs = []
+        for step in range(steps):
+            q, kn, vn, fn = inputs.decode_inputs(shape, 630, step, DEV, keep_new=0.5)
+            outs.append(T.gpu_decode_step(shape, q, kn, vn, fn, cache, status, fused=True))
+        runs.append(outs + [cache.k_rows.clone(), cache.v_rows.clone(), cache.len.clone()])
+    for a, b in zip(*runs):
+        assert torch.equal(a, b)
+    assert int(status.item()) == 0
 
 
 def test_results_are_bitwise_repeatable():
