@@ -59,6 +59,8 @@ TRAFFIC = {
 # (decode step, attention + append: one cluster kernel up to DECODE_CLUSTER_MAX_SLABS slabs, else chunk pass + merge)
 LAUNCHES = {"gate": 3, "compact": 1, "prefill": 1, "decode": 2}
 DECODE_CLUSTER_MAX_SLABS = 64
+L2_BYTES = 126e6
+MIN_TIMED_S = 0.6     # a run's timed region lasts at least about this long
 
 
 def _peaks():
@@ -171,14 +173,18 @@ class LayerRun:
         self.desc = ag.make_desc(sh)
         B, h, n, D = sh.batch, sh.heads, sh.seq, sh.head_dim
         self.name = name
-        self.use_graph, self.graph = True, None
+        self.use_graph = True
         self._groups = {}
         self.has_gate = name in ("prefill7b", "prefill7b_proj", "tiny", "stack7b", "stack7b_prev")
         self.project = name == "prefill7b_proj"                     # Q, K, V are computed in the step
         self.layers = 32 if name.startswith("stack7b") else 1
         self.first_gated = 1 if name == "stack7b_prev" else 0      # 0: every layer evicts by its own gate
         self.has_prefill = name not in ("decode_ragged", "decode_ragged_gqa")
-        if self.has_gate:
+        if self.has_gate and self.layers > 1:
+            # every layer of a stack has its own hidden states X_l, weights and upstream Q, K, V
+            self.layer_in = [inputs.stack_layer_inputs(sh, seed, l, dev) for l in range(self.layers)]
+            self.X, self.W, self.Q, self.K, self.V = self.layer_in[0]
+        elif self.has_gate:
             self.X = inputs.hidden_states(sh, seed, dev)
             self.W = inputs.layer_weights(sh, seed + 10, dev)
             self.Q, self.K, self.V = inputs.project_qkv(sh, self.X, self.W)
@@ -214,18 +220,30 @@ class LayerRun:
         # new-token flags: Bernoulli(0.1) on the deep layer, every token kept in the stack (the paper's
         # decode stage runs no gate), Bernoulli(0.5) elsewhere
         keep_new = 0.1 if name == "deep_layer" else 1.0 if self.layers > 1 else 0.5
-        self.dq = [inputs.decode_inputs(sh, seed + 500, s, dev, keep_new=keep_new) for s in range(self.decode_steps)]
+        # decode tokens: one list of steps per layer (a stack's layers each decode their own)
+        self.dqs = [[inputs.decode_inputs(sh, inputs.stack_layer_seed(seed, l) + 500 if self.layers > 1 else seed + 500,
+                                          s, dev, keep_new=keep_new) for s in range(self.decode_steps)]
+                    for l in range(self.layers)]
+        self.dq = self.dqs[0]
+        self.layer = 0
+        self.graphs = {}
         self.o = torch.empty(B, h, D, dtype=sh.torch_dtype, device=dev)
         # gamma: per-head keep rate ~ U[0.3, 0.8], calibrated on the scores at gamma = 0
         self.gamma = None
         if self.has_gate:
-            self.gate()
             if self.layers > 1:
-                # the layers share X and the weights (inputs, not the timed work); what differs per
-                # layer is the keep rate, i.e. gamma: mean eviction 10 % (first) ... 90 % (last)
-                self.gammas = [inputs.calibrate_gamma(self.scores, inputs.keep_targets_layer(h, seed + 20, l), sh.tau).to(dev)
-                               for l in range(self.layers)]
+                # per layer: mean eviction 10 % (first) ... 90 % (last), gamma calibrated on the layer's
+                # own scores at gamma = 0
+                self.gammas = []
+                for l in range(self.layers):
+                    self.set_layer(l)
+                    self.gamma = None
+                    self.gate()
+                    self.gammas.append(inputs.calibrate_gamma(self.scores, inputs.keep_targets_layer(h, seed + 20, l),
+                                                              sh.tau).to(dev))
+                self.set_layer(0)
             else:
+                self.gate()
                 keep = inputs.keep_targets_uniform(h, seed + 20) if name != "tiny" else [0.5] * h
                 self.gammas = [inputs.calibrate_gamma(self.scores, keep, sh.tau).to(dev)]
             self.gamma = self.gammas[0]
@@ -234,6 +252,13 @@ class LayerRun:
             self.flags.copy_(f.to(dev))
             for q in self.dq:
                 q[3][:, torch.from_numpy(empty).to(dev)] = 0     # fully evicted heads stay empty
+
+    def set_layer(self, layer):
+        """Point the calls at the inputs of layer `layer` (a stack; a single layer has only layer 0)."""
+        self.layer = layer
+        self.dq = self.dqs[layer]
+        if self.layers > 1 and self.has_gate:
+            self.X, self.W, self.Q, self.K, self.V = self.layer_in[layer]
 
     def gate(self, flags_out=None):
         W, ag = self.W, self.ag
@@ -317,6 +342,7 @@ class LayerRun:
         if self.first_gated:
             return self._step_guided_by_previous_layer(timed)
         for layer in range(self.layers):
+            self.set_layer(layer)
             if self.has_gate:
                 self.gamma = self.gammas[layer]
                 timed("gate", self.gate)
@@ -339,10 +365,15 @@ class LayerRun:
             self.schedule = PreviousLayerGate(self.first_gated, [self.flags, torch.empty_like(self.flags)], ones, self.dev)
 
         def gate(layer, flags_out):
+            # the module of layer `layer` on that layer's hidden states; its flags guide layer + 1
+            keep = (self.layer, self.X, self.W)
+            self.X, self.W = self.layer_in[layer][0], self.layer_in[layer][1]
             self.gamma = self.gammas[layer]
             timed("gate", self.gate, flags_out)
+            self.layer, self.X, self.W = keep
 
         def attend(layer, flags):
+            self.set_layer(layer)
             self.cur_flags = flags
             timed("compact", self.compact)
             timed("prefill", self.prefill)
@@ -356,7 +387,7 @@ class LayerRun:
             for s in range(self.decode_steps):
                 self.decode(s)
             return
-        if self.graph is None:
+        if self.layer not in self.graphs:
             len_before = self.cache.len.clone()
             for s in range(self.decode_steps):       # warm-up outside capture
                 self.decode(s)
@@ -367,8 +398,8 @@ class LayerRun:
                 for s in range(self.decode_steps):
                     self.decode(s)
             self.cache.len.copy_(len_before)         # capture does not run the kernels
-            self.graph = g
-        self.graph.replay()
+            self.graphs[self.layer] = g
+        self.graphs[self.layer].replay()
 
     def tokens_per_step(self):
         return self.shape.batch * ((self.shape.seq if self.has_prefill else 0) + self.decode_steps) * self.layers
@@ -391,15 +422,18 @@ class LayerRun:
         K and V, plus q, k_new, v_new, o; lengths grow linearly over the decode steps)."""
         e = 2 if self.shape.dtype == "bf16" else 4
         D, slabs = self.shape.head_dim, self.shape.batch * self.shape.heads
-        appended = float(sum(q[3].to(torch.float64).sum().item() for q in self.dq))
+        appended = float(np.mean([sum(q[3].to(torch.float64).sum().item() for q in dq) for dq in self.dqs]))
         f_eff, kept = [], []
         for layer in range(self.layers):
+            self.set_layer(layer)
             if self.first_gated:
                 if layer < self.first_gated:
                     self.cur_flags = torch.ones_like(self.flags)
                 else:
                     self.gamma, self.cur_flags = self.gammas[layer - 1], self.flags
+                    self.X, self.W = self.layer_in[layer - 1][0], self.layer_in[layer - 1][1]
                     self.gate()
+                    self.set_layer(layer)
             elif self.has_gate:
                 self.gamma = self.gammas[layer]
                 self.gate()
@@ -441,6 +475,118 @@ def flush_l2(buf):
     buf.zero_()
 
 
+CALLS = ("gate", "compact", "project", "prefill", "decode")
+
+
+def timed_passes(run, n_passes, l2buf):
+    """n_passes passes of the whole path, each bracketed by CUDA events on the launching stream with
+    the L2 flushed (outside the events) before it.  Returns (total ms, mean ms per call)."""
+    ev = {k: [] for k in CALLS}
+    pass_ev = []
+    for _ in range(n_passes):
+        flush_l2(l2buf)
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        run.step(ev, s)
+        e.record()
+        pass_ev.append((s, e))
+    torch.cuda.synchronize()
+    total_ms = sum(s.elapsed_time(e) for s, e in pass_ev)
+    per_call_ms = {k: float(np.mean([s.elapsed_time(e) for s, e in v])) * len(v) / n_passes / run.layers
+                   for k, v in ev.items() if v}
+    return total_ms, per_call_ms
+
+
+def rooflines_of(run, per_call_ms, peaks, workload):
+    """Achieved rate of every call of a pass against its bound: algorithmic work of the call (from the
+    flags / lengths the run produced) over its CUDA-event time (mean per layer)."""
+    sh = run.shape
+    e = 2 if sh.dtype == "bf16" else 4
+    out = {}
+    work = run.work_per_call()
+
+    def entry(bound, kernel, amount, ms, key):
+        unit, peak = ("TFLOP/s", peaks["bf16_tflops"]) if bound == "tensor" else ("GB/s", peaks["hbm_gbs"])
+        rate = amount / (ms * 1e-3) / (1e12 if bound == "tensor" else 1e9)
+        r = {"bound": bound, "kernel": kernel, "achieved": rate, "peak": peak, "unit": unit, "frac": rate / peak,
+             "traffic": TRAFFIC.get((workload, key)), "peak_source": peaks["source"], "ms": ms, "workload": workload}
+        r["algorithmic_flops" if bound == "tensor" else "algorithmic_bytes"] = amount
+        return r
+
+    dec_ms = per_call_ms["decode"] / run.decode_steps
+    out["decode"] = entry("hbm", "ag_decode_step", work["decode_bytes"], dec_ms, "decode")
+    if work["decode_bytes"] < L2_BYTES:
+        # the cache of the step fits in L2 and has just been written by compaction and read by prefill:
+        # the replayed decode steps stream it from L2, and a few microseconds per step do not depend on
+        # its length at all.  The rate is reported, but it is no measurement of HBM bandwidth.
+        out["decode"]["bound"] = "l2/latency"
+        out["decode"]["note"] = ("cache of %.0f MB per step stays in L2 (126 MB): rate against the HBM copy peak for "
+                                 "scale only; the HBM-bound decode figure is the decode_ragged workload's"
+                                 % (work["decode_bytes"] / 1e6))
+    if run.has_prefill:
+        out["prefill"] = entry("tensor", "ag_prefill_attn", work["prefill_flops"], per_call_ms["prefill"], "prefill")
+        if "compact" in per_call_ms:
+            cb = 2.0 * (2.0 * work["kept_rows"] * sh.head_dim * e) + sh.batch * sh.heads * sh.seq * 9.0
+            out["compact"] = entry("hbm", "ag_compact_kv", cb, per_call_ms["compact"], "compact")
+        if "project" in per_call_ms:
+            kf = 2.0 * sh.batch * sh.seq * sh.hidden * (2 * sh.kvh + sh.heads) * sh.head_dim
+            out["project"] = entry("tensor", "ag_qkv_project_cache", kf, per_call_ms["project"], "project")
+    if run.has_gate:
+        out["gate"] = entry("tensor", "ag_gate_forward", run.gate_flops(), per_call_ms["gate"], "gate")
+    return out
+
+
+def timed_alone(fn, n, l2buf):
+    """Mean CUDA-event time (ms) of n calls of fn, L2 flushed before each, after 3 warm-up calls."""
+    evs = []
+    for i in range(3 + n):
+        flush_l2(l2buf)
+        s_, e_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s_.record()
+        fn()
+        e_.record()
+        if i >= 3:
+            evs.append((s_, e_))
+    torch.cuda.synchronize()
+    return float(np.mean([a_.elapsed_time(b_) for a_, b_ in evs]))
+
+
+def near_threshold_fractions(run):
+    """Share of the (head, token) gate scores that lie within 1e-3 of the threshold, in the two units
+    the tolerance can be read in: score units |s + gamma - logit(tau)| < 1e-3 (what the parity tests
+    exclude from the bit-exact flag comparison) and probability units |Sigmoid(s + gamma) - tau| < 1e-3.
+    Counted on the scores the last gate pass of the run produced."""
+    tau = float(run.shape.tau)
+    z = run.scores.double() + run.gamma.double().view(1, -1, 1)
+    logit = float(np.log(tau / (1.0 - tau)))
+    return {"score_units": float(((z - logit).abs() < 1e-3).double().mean().item()),
+            "probability_units": float(((torch.sigmoid(z) - tau).abs() < 1e-3).double().mean().item())}
+
+
+# The other full-size workloads, timed briefly after the headline workload in the default invocation:
+# name -> (warm-up passes, timed passes).  One pass of decode_ragged is 256 graph-replayed decode steps
+# over 2.4 GB of cache each; one of deep_layer is compaction + prefill of 16384 tokens + 128 decode
+# steps; one of stack7b is 32 layers of gate + compaction + prefill + 256 decode steps at batch 8.
+EXTRA_WORKLOADS = {"decode_ragged": (1, 3), "deep_layer": (3, 20), "stack7b": (1, 2)}
+
+
+def measure_extra(name, dev, l2buf, peaks):
+    warm, passes = EXTRA_WORKLOADS[name]
+    run = LayerRun(name, 2000, dev)
+    for _ in range(warm):
+        run.step()
+    torch.cuda.synchronize()
+    total_ms, per_call_ms = timed_passes(run, passes, l2buf)
+    assert int(run.status.item()) == 0, "device reported a cache overflow"
+    roofs = rooflines_of(run, per_call_ms, peaks, name)
+    info = {"ms_per_pass": total_ms / passes, "passes": passes, "tokens_per_s": run.tokens_per_step() * passes / (total_ms * 1e-3),
+            "per_call_ms_per_layer": per_call_ms, "launches": run.launches_per_step() * passes,
+            "mean_keep": float(run.flags.float().mean().item()) if run.has_prefill else None}
+    del run
+    torch.cuda.empty_cache()
+    return roofs, info
+
+
 def run_ours(args, rank, world, dev):
     torch.cuda.set_device(dev)
     run = LayerRun(args.workload, 2000 + 100 * rank, dev, args.recent_window)
@@ -459,30 +605,29 @@ def run_ours(args, rank, world, dev):
     for _ in range(args.warmup):
         run.step()
     barrier()
+    # A step is `passes` passes of the whole path over the batch, enough of them that the timed region
+    # (steps x passes) lasts about MIN_TIMED_S: a few milliseconds of work would leave the clock
+    # sampler, and whoever watches the GPU from outside, with a sample or two.
+    t_probe, _ = timed_passes(run, 2, l2buf)
+    est_pass_ms, = max_over_ranks([t_probe / 2], dist, dev)
+    passes = args.passes if args.passes > 0 else max(1, int(np.ceil(MIN_TIMED_S * 1e3 / (args.steps * est_pass_ms))))
     sampler = ClockSampler(torch.cuda.current_device())
     if rank == 0:
         sampler.start()
-    ev = {k: [] for k in ("gate", "compact", "project", "prefill", "decode")}
-    step_ev = []
     barrier()
-    for _ in range(args.steps):
-        flush_l2(l2buf)
-        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s.record()
-        run.step(ev, s)
-        e.record()
-        step_ev.append((s, e))
+    total_ms, per_call_ms = timed_passes(run, args.steps * passes, l2buf)
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    total_ms = sum(s.elapsed_time(e) for s, e in step_ev)
-    per_call_ms = {k: float(np.mean([s.elapsed_time(e) for s, e in v])) for k, v in ev.items() if v}
     assert int(run.status.item()) == 0, "device reported a cache overflow"
     timeouts = run.ag.ag_device_wait_timeouts()
     assert timeouts == 0, f"{timeouts} bounded device waits expired"
 
     # end to end: pinned host inputs in, results out, through the same calls
     sh = run.shape
-    if run.project:
+    stack = run.layers > 1 and run.has_gate
+    if stack:
+        dev_in = [t for (X, W, Q, K, V), dq in zip(run.layer_in, run.dqs) for t in [X, Q, K, V] + [u for q in dq for u in q]]
+    elif run.project:
         dev_in = [run.X]                                     # Q, K and V are made on the device
     elif run.has_gate:
         dev_in = [run.X, run.Q, run.K, run.V]
@@ -490,13 +635,14 @@ def run_ours(args, rank, world, dev):
         dev_in = [run.Q, run.K, run.V, run.flags]
     else:
         dev_in = []
-    dev_in += [t for q in run.dq for t in q]
+    if not stack:
+        dev_in += [t for q in run.dq for t in q]
     dev_out = ([run.O, run.flags] if run.has_prefill else []) + [run.o]
     host_in = [t.detach().cpu().pin_memory() for t in dev_in]
     host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in dev_out]
     h2d = sum(t.numel() * t.element_size() for t in host_in)
     d2h = sum(t.numel() * t.element_size() for t in host_out)
-    e2e_steps = max(1, min(args.steps, 10))
+    e2e_steps = max(1, min(args.steps, 10 if not stack else 1))
     # One layer with a gate: the copies run on their own streams, each call waits only for the inputs
     # it reads (X -> gate; a head group's K, V, Q -> its compaction and prefill; the decode tokens ->
     # decode), and the flags and each group's O go back to the host while later groups come in.
@@ -600,103 +746,50 @@ def run_ours(args, rank, world, dev):
         return None
     tokens = run.tokens_per_step() * world
     peaks = _peaks()
-    rooflines = {}
-    work = run.work_per_call()
-    dec_bytes = work["decode_bytes"]
-    dec_ms = per_call_ms["decode"] / run.decode_steps
-    dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
-    rooflines["decode"] = {"bound": "hbm", "kernel": "ag_decode_step", "achieved": dec_gbs,
-                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"],
-                           "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": dec_bytes,
-                           "ms": dec_ms}
-    if run.has_prefill:
-        f_eff = work["prefill_flops"]
-        tf = f_eff / (per_call_ms["prefill"] * 1e-3) / 1e12
-        rooflines["prefill"] = {"bound": "tensor", "kernel": "ag_prefill_attn", "achieved": tf,
-                                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
-                                "traffic": None, "peak_source": peaks["source"], "algorithmic_flops": f_eff,
-                                "ms": per_call_ms["prefill"]}
-        e = 2 if sh.dtype == "bf16" else 4
-        kept = work["kept_rows"]
-        if "compact" in per_call_ms:
-            cb = 2.0 * (2.0 * kept * sh.head_dim * e) + sh.batch * sh.heads * sh.seq * 9.0
-            gbs = cb / (per_call_ms["compact"] * 1e-3) / 1e9
-            rooflines["compact"] = {"bound": "hbm", "kernel": "ag_compact_kv", "achieved": gbs, "peak": peaks["hbm_gbs"],
-                                    "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
-                                    "peak_source": peaks["source"], "algorithmic_bytes": cb, "ms": per_call_ms["compact"]}
-        if "project" in per_call_ms:
-            kf = 2.0 * sh.batch * sh.seq * sh.hidden * (2 * sh.kvh + sh.heads) * sh.head_dim
-            tf = kf / (per_call_ms["project"] * 1e-3) / 1e12
-            rooflines["project"] = {"bound": "tensor", "kernel": "ag_qkv_project_cache", "achieved": tf,
-                                    "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
-                                    "traffic": None, "peak_source": peaks["source"], "algorithmic_flops": kf,
-                                    "ms": per_call_ms["project"]}
-    if run.has_gate:
-        gf = run.gate_flops()
-        tf = gf / (per_call_ms["gate"] * 1e-3) / 1e12
-        rooflines["gate"] = {"bound": "tensor", "kernel": "ag_gate_forward", "achieved": tf, "peak": peaks["bf16_tflops"],
-                             "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "traffic": None,
-                             "peak_source": peaks["source"], "algorithmic_flops": gf, "ms": per_call_ms["gate"]}
+    rooflines = rooflines_of(run, per_call_ms, peaks, args.workload)
+    if run.has_gate and run.layers == 1:
         # the local gate variant, timed apart from the step (L2 flushed before each call)
-        lin_ev = []
-        for i in range(3 + min(args.steps, 20)):
-            flush_l2(l2buf)
-            s_, e_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            s_.record()
-            run.gate_linear()
-            e_.record()
-            if i >= 3:
-                lin_ev.append((s_, e_))
-        torch.cuda.synchronize()
-        lin_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in lin_ev]))
+        lin_ms = timed_alone(run.gate_linear, min(args.steps, 20), l2buf)
         e = 2 if sh.dtype == "bf16" else 4
         lb = float(sh.batch * sh.seq * sh.hidden * e + sh.hidden * sh.heads * e + sh.batch * sh.heads * sh.seq * 5)
         gbs = lb / (lin_ms * 1e-3) / 1e9
         rooflines["gate_linear"] = {"bound": "hbm", "kernel": "ag_gate_linear_forward (not part of the step)",
                                     "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                     "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
-                                    "algorithmic_bytes": lb, "ms": lin_ms}
-        if (sh.dtype == "bf16" and sh.head_dim == 128 and sh.seq % 128 == 0 and sh.recent_window <= 1 and run.layers == 1
+                                    "algorithmic_bytes": lb, "ms": lin_ms, "workload": args.workload}
+        if (sh.dtype == "bf16" and sh.head_dim == 128 and sh.seq % 128 == 0 and sh.recent_window <= 1
                 and not run.project):
             # the fused key/value projection, timed apart from the step like the local gate
-            kv_ev = []
-            for i in range(3 + min(args.steps, 20)):
-                flush_l2(l2buf)
-                s_, e_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                s_.record()
-                run.kv_project_cache()
-                e_.record()
-                if i >= 3:
-                    kv_ev.append((s_, e_))
-            torch.cuda.synchronize()
-            kv_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in kv_ev]))
+            kv_ms = timed_alone(run.kv_project_cache, min(args.steps, 20), l2buf)
             kf = 2.0 * sh.batch * sh.seq * sh.hidden * 2 * sh.kvh * sh.head_dim
             tf = kf / (kv_ms * 1e-3) / 1e12
             rooflines["kv_project_cache"] = {"bound": "tensor",
                                              "kernel": "ag_kv_project_cache (not part of the step)",
                                              "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                                             "frac": tf / peaks["bf16_tflops"], "traffic": None,
-                                             "peak_source": peaks["source"], "algorithmic_flops": kf, "ms": kv_ms}
-    for k, r in rooflines.items():
-        r["traffic"] = TRAFFIC.get((args.workload, k))
+                                             "frac": tf / peaks["bf16_tflops"],
+                                             "traffic": TRAFFIC.get((args.workload, "kv_project_cache")),
+                                             "peak_source": peaks["source"], "algorithmic_flops": kf, "ms": kv_ms,
+                                             "workload": args.workload}
     head = "prefill" if run.has_prefill else "decode"
-    ms_step = total_ms / args.steps
+    n_timed = args.steps * passes
+    ms_pass = total_ms / n_timed
     out = {
-        "metric": METRIC, "value": aggregate_value(run.tokens_per_step(), world, args.steps, total_ms), "unit": UNIT,
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+        "metric": METRIC, "value": aggregate_value(run.tokens_per_step(), world, n_timed, total_ms), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if sh.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "description": run.desc_text, "batch": sh.batch, "seq": sh.seq,
-                   "hidden": sh.hidden, "heads": sh.heads, "head_dim": sh.head_dim, "gate_heads": sh.gate_heads,
-                   "gate_head_dim": sh.gate_head_dim, "decode_steps_per_step": run.decode_steps,
+        "config": config_of(args.workload, sh, run.decode_steps, run.desc_text),
+        "timing": {"passes_per_step": passes, "ms_per_pass": ms_pass,
+                   "step": f"{passes} passes of the whole path over the batch, L2 flushed before each pass (outside its events)",
                    "recent_window": max(1, sh.recent_window),
                    "mean_keep": float(run.flags.float().mean().item()) if run.has_prefill else None,
-                   "l2": "flushed between steps (256 MiB write)", "replicas": world,
+                   "near_threshold": near_threshold_fractions(run) if run.has_gate else None,
+                   "replicas": world,
                    "decode_launch": "one CUDA graph per pass" if run.use_graph else "individual launches"},
         "clocks": clocks,
         "e2e": {"value": tokens * e2e_steps / (t_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": run.launches_per_step() * args.steps,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "passes_per_step": 1},
+        "gpu_launches": run.launches_per_step() * n_timed,
         "roofline": rooflines[head],
         "rooflines": rooflines,
         "per_call_ms": per_call_ms,
@@ -706,6 +799,15 @@ def run_ours(args, rank, world, dev):
     if run.has_prefill:
         pre_ms = sum(per_call_ms.get(k, 0.0) for k in ("gate", "compact", "project", "prefill"))
         out["prefill_tokens_per_s"] = sh.batch * sh.seq / (pre_ms * 1e-3)
+    if args.workload == "prefill7b" and world == 1 and not args.no_extra and args.recent_window <= 1:
+        # the other full-size workloads, briefly: their rooflines ride in the same line
+        out["workloads"] = {}
+        del host_in, host_out
+        for name in EXTRA_WORKLOADS:
+            roofs, info = measure_extra(name, dev, l2buf, peaks)
+            out["workloads"][name] = info
+            for k, r in roofs.items():
+                rooflines[f"{name}.{k}"] = r
     return out, run
 
 
@@ -759,7 +861,7 @@ def oracle_sample(name, seed, n_heads_sample=2, decode_steps=2):
         cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     except Exception:
         cores = len(os.sched_getaffinity(0))
-    return {"value": tokens / est, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+    return {"value": tokens / est, "unit": UNIT, "cores": int(cores), "kind": "oracle", "sample_s": t_gate + t_heads + t_dec,
             "sample": f"full gate + {hs} of {shape.heads} heads of compaction/prefill + {ds} of {dsteps} decode steps, "
                       f"scaled to the whole step (gate {t_gate:.2f}s, heads {t_heads:.2f}s, decode {t_dec:.3f}s)",
             "est_step_s": est}
@@ -771,11 +873,13 @@ def run_reference(args, rank, world):
     shape, dsteps, text = WORKLOADS[args.workload]
     # each step is one bounded oracle sample (seconds of CPU work); the number of samples is capped so
     # that the whole run stays within a few minutes whatever --steps asks for
-    vals, t_start, budget_s = [], time.perf_counter(), 150.0
+    vals, walls, t_start, budget_s = [], [], time.perf_counter(), 150.0
     for k in range(args.warmup + args.steps):
+        t_k = time.perf_counter()
         r = oracle_sample(args.workload, 2000, n_heads_sample=1, decode_steps=1)
         if k >= args.warmup:
             vals.append(r)
+            walls.append(r["sample_s"])
         per = (time.perf_counter() - t_start) / (k + 1)
         if vals and time.perf_counter() - t_start + per > budget_s:
             break
@@ -785,13 +889,36 @@ def run_reference(args, rank, world):
     base = dict(vals[-1])
     base["value"] = v
     base.pop("est_step_s", None)
+    base.pop("sample_s", None)
+    # ms_per_step is the measured time of one step of THIS arm (one bounded sample); `value` is the
+    # whole-layer rate that sample extrapolates to (est_layer_ms)
     return {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": world, "steps": len(vals),
             "steps_requested": args.steps,
-            "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": float(np.mean(walls)) * 1e3, "est_layer_ms": est * 1e3,
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "description": text},
+            "config": config_of(args.workload, shape, dsteps, text),
             "cpu_baseline": base,
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def config_of(workload, sh, decode_steps, text):
+    """The keys of `config` both arms print alike."""
+    return {"workload": workload, "description": text, "batch": sh.batch, "seq": sh.seq, "hidden": sh.hidden,
+            "heads": sh.heads, "head_dim": sh.head_dim, "gate_heads": sh.gate_heads, "gate_head_dim": sh.gate_head_dim,
+            "decode_steps_per_pass": decode_steps,
+            "l2": "GPU arm: flushed before every pass (256 MiB write, outside the pass's events); the CPU arm has no GPU cache"}
+
+
+def replica_command(n_gpus, argv, port):
+    """The command line that runs this script as n_gpus replicas, one process per GPU, on this node."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+
+
+def spawn_replicas(n_gpus, argv):
+    port = 29500 + os.getpid() % 2000
+    return subprocess.call(replica_command(n_gpus, argv, port))
 
 
 def main():
@@ -805,8 +932,15 @@ def main():
     ap.add_argument("--recent-window", type=int, default=0,
                     help="recent tokens always visible, the current one included (0 or 1: the method as published)")
     ap.add_argument("--no-graph", action="store_true", help="launch the decode steps one by one instead of replaying a CUDA graph")
+    ap.add_argument("--passes", type=int, default=0,
+                    help="passes of the whole path per step (0: as many as make the timed region last about 0.6 s)")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the brief measurements of the other full-size workloads after the headline one")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started by hand with --gpus N: become N replicas, one process per GPU
+        raise SystemExit(spawn_replicas(args.gpus, sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -834,6 +968,7 @@ def main():
         if not args.no_cpu_baseline and world == 1 and args.workload in ("prefill7b", "prefill7b_proj", "tiny"):
             cb = oracle_sample(args.workload, 2000, n_heads_sample=WORKLOADS[args.workload][0].heads, decode_steps=16)
             cb.pop("est_step_s", None)
+            cb.pop("sample_s", None)
             out["cpu_baseline"] = cb
         print(json.dumps(out))
     if world > 1:

@@ -45,3 +45,14 @@ def test_oracle_timing_leg_on_the_tiny_workload():
     r = bench.oracle_sample("tiny", 2000, n_heads_sample=4, decode_steps=2)
     assert r["kind"] == "oracle" and r["unit"] == "tokens/s" and r["value"] > 0 and r["cores"] >= 1
     assert "gate" in r["sample"]
+
+
+def test_gpus_flag_turns_into_one_process_per_gpu():
+    """`bench.py --gpus N` started by hand (no WORLD_SIZE in the environment) re-launches itself as N
+    replicas on this node, rendezvous on 127.0.0.1, with its own arguments passed through."""
+    import bench
+    cmd = bench.replica_command(4, ["--gpus", "4", "--steps", "5"], 29611)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"]
+    assert "--nproc-per-node=4" in cmd and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[cmd.index("--master-port") + 1] == "29611"
+    assert cmd[-5].endswith("bench.py") and cmd[-4:] == ["--gpus", "4", "--steps", "5"]
