@@ -16,6 +16,7 @@ Layouts (same as the C boundary):
     Wq_g/Wk_g/Wv_g  [d, h' * D']     AG projections, row-major "in x out"
     Wo_g            [h' * D', h]     AG output projection (Sec. 3.3, W^{O'})
     Q, K, V, O      [B, h, n, D]
+    Wo              [h * D, d]       output projection of Eq. 1 (W^O)
     scores          [B, h, n]        MHA'(X) transposed to head-major
     flags           [B, h, n] uint8  1 = retain, 0 = evict
 
@@ -23,7 +24,8 @@ Pins (see tests/test_oracle_*.py): all-keep == textbook causal attention,
 all-evict == O[j] = V[j], brute force over explicit visible-key sets for all
 2^n flag patterns at tiny n, uniform-attention closed forms, gate closed
 forms (Wo'=0, identical rows, n=1), causality of MHA', prefill/decode
-consistency.  What remains unpinned: the paper prints no worked numeric
+consistency; the output projection of Eq. 1 by W^O = identity (pure concatenation),
+written-out loops, a library contraction and its locality in heads and tokens.  What remains unpinned: the paper prints no worked numeric
 example and does not say whether MHA' is causal; "parity unpinned" applies to
 that choice of reading only (both readings are implemented).
 """
@@ -245,6 +247,24 @@ def project_q(X, Wq, heads):
             for t in range(n):
                 Q[b, i, t] = X[b, t] @ Wq[:, i * D:(i + 1) * D]
     return Q
+
+
+def mha_output(H, Wo, X_res=None):
+    """The layer's output, Eq. 1: MHA(X) = [H_1(X), ..., H_h(X)] W^O, the heads' outputs concatenated
+    along the feature axis (head i in columns [i D, (i + 1) D)) and multiplied by W^O in R^{h D x d}.
+    H [B, h, n, D] (the O of prefill attention), Wo [h D, d] -> [B, n, d] in float64.
+    With X_res [B, n, d] the Transformer's skip connection is added: X_res + MHA(X) (the paper's Eq. 1
+    stops at MHA(X); a stack of attention layers feeds this sum to the next layer)."""
+    H, Wo = _as_f64(H), _as_f64(Wo)
+    B, h, n, D = H.shape
+    Y = np.zeros((B, n, Wo.shape[1]), dtype=F64)
+    for b in range(B):
+        for t in range(n):
+            concat = np.concatenate([H[b, i, t] for i in range(h)])      # [h D]
+            Y[b, t] = concat @ Wo
+    if X_res is not None:
+        Y = Y + _as_f64(X_res)
+    return Y
 
 
 def project_and_cache(X, Wk, Wv, flags):
