@@ -16,6 +16,7 @@
  *                           to the dense K, V and, for retained
  *                           tokens, straight into the cache     Eq. 2 + Sec. 3.3 (after Eq. 4)
  *   ag_qkv_project_cache    the same with Q_i = X W^Q_i         Eq. 2
+ *   ag_out_project          [H_1 .. H_h] W^O (+ skip connection) Eq. 1
  *
  * Conventions common to every call
  * --------------------------------
@@ -272,6 +273,28 @@ int ag_prefill_attn(const ag_layer_desc *desc, const void *Q, const void *K,
                     const void *V, const uint8_t *flags, const ag_cache *cache,
                     const int32_t *prefix, float softmax_scale, void *O,
                     void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Downstream of step 3 — the layer's output, Eq. 1: MHA(X) = [H_1(X), ..., H_h(X)] W^O, the
+ * heads' outputs concatenated along the feature axis (head i in columns [i D, (i + 1) D)) and
+ * projected by W^O in R^{h D x d}; with X_res, the Transformer's skip connection is added in the
+ * same pass:
+ *   Y[b, t, :] = X_res[b, t, :] + sum_i O[b, i, t, :] Wo[i D : (i + 1) D, :].
+ * The paper stops at Eq. 1; the skip connection is what feeds a layer's output to the next layer
+ * in a stack of attention layers (no normalisation, no feed-forward block in between).
+ * Float32 accumulation, one rounding to the layer dtype.  Uses desc->batch, seq, heads, head_dim,
+ * hidden, dtype.  Needs no workspace.
+ *
+ *   O      [B, h, n, D]          in   (as ag_prefill_attn writes it; h = desc->heads)
+ *   Wo     [h D, d]              in   ("in x out")
+ *   X_res  [B, n, d] or NULL     in   skip connection (NULL: Y = MHA(X))
+ *   Y      [B, n, d]             out  must not be X_res or O
+ * Tensor-core coverage: bfloat16, head_dim 128, d a multiple of 128, and n a multiple of 128
+ * unless batch = 1; other shapes run on CUDA cores (B n <= 65535), else AG_ERR_UNSUPPORTED.
+ * AG_ERR_INVALID_ARG for missing or misaligned (16-byte) pointers.
+ */
+int ag_out_project(const ag_layer_desc *desc, const void *O, const void *Wo, const void *X_res,
+                   void *Y, void *cuda_stream);
 
 /*
  * Step 4a — one decode query per (sequence, head) (Sec. 3.1 decoding stage;

@@ -22,7 +22,7 @@ EXPORTS = (
     "ag_workspace_bytes", "ag_gate_forward", "ag_compact_kv", "ag_prefill_attn",
     "ag_decode_attn", "ag_cache_append", "ag_status_string", "ag_last_cuda_error",
     "ag_decode_attn_noalloc", "ag_device_wait_timeouts", "ag_gate_linear_forward", "ag_decode_step",
-    "ag_kv_project_cache", "ag_qkv_project_cache",
+    "ag_kv_project_cache", "ag_qkv_project_cache", "ag_out_project",
 )
 
 
@@ -78,6 +78,8 @@ def lib():
         L.ag_kv_project_cache.argtypes = [dp, vp, vp, vp, vp, cp, vp, vp, vp, vp, vp, vp]
         L.ag_qkv_project_cache.restype = i32
         L.ag_qkv_project_cache.argtypes = [dp, vp, vp, vp, vp, vp, cp, vp, vp, vp, vp, vp, vp, vp]
+        L.ag_out_project.restype = i32
+        L.ag_out_project.argtypes = [dp, vp, vp, vp, vp, vp]
         L.ag_prefill_attn.restype = i32
         L.ag_prefill_attn.argtypes = [dp, vp, vp, vp, vp, cp, vp, f32, vp, vp, sz, vp]
         L.ag_decode_attn.restype = i32
@@ -226,6 +228,11 @@ def ag_prefill_attn(desc, Q, K, V, flags, cache, prefix, softmax_scale, O, ws, s
     return _check(lib().ag_prefill_attn(ctypes.byref(desc), _ptr(Q), _ptr(K), _ptr(V), _ptr(flags),
                                         ctypes.byref(cache.struct), _ptr(prefix), float(softmax_scale),
                                         _ptr(O), p, nbytes, _stream(stream)), "ag_prefill_attn")
+
+
+def ag_out_project(desc, O, Wo, X_res, Y, stream=None):
+    return _check(lib().ag_out_project(ctypes.byref(desc), _ptr(O), _ptr(Wo), _ptr(X_res), _ptr(Y), _stream(stream)),
+                  "ag_out_project")
 
 
 def ag_decode_attn(desc, q, k_new, v_new, cache, softmax_scale, o, ws, stream=None):

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libag.so")
-SOURCES = ["ag_api.cu", "gate.cu", "gemm_tc.cu", "gate_attn_tc.cu", "gate_linear.cu", "compact.cu", "prefill.cu", "prefill_tc.cu", "decode.cu", "decode_gqa_mma.cu", "prefill_band_mma.cu", "kv_proj_cache.cu"]
+SOURCES = ["ag_api.cu", "gate.cu", "gemm_tc.cu", "gate_attn_tc.cu", "gate_linear.cu", "compact.cu", "prefill.cu", "prefill_tc.cu", "decode.cu", "decode_gqa_mma.cu", "prefill_band_mma.cu", "kv_proj_cache.cu", "out_proj.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 NVCC_FLAGS = [*ARCH, "-lineinfo", "-O3", "-std=c++17", "--use_fast_math", "-Xcompiler", "-fPIC",
               "-cudart", "static"]

@@ -181,6 +181,18 @@ int ag_prefill_attn(const ag_layer_desc *desc, const void *Q, const void *K,
                         (cudaStream_t)cuda_stream);
 }
 
+int ag_out_project(const ag_layer_desc *desc, const void *O, const void *Wo, const void *X_res, void *Y,
+                   void *cuda_stream) {
+  int st = check_desc(desc);
+  if (st) return st;
+  if (desc->hidden <= 0) return AG_ERR_INVALID_ARG;
+  if (!O || !Wo || !Y) return AG_ERR_INVALID_ARG;
+  if (misaligned16(O) || misaligned16(Wo) || misaligned16(X_res) || misaligned16(Y)) return AG_ERR_INVALID_ARG;
+  if (Y == X_res || Y == O) return AG_ERR_INVALID_ARG;
+  if (desc->hidden % 8 != 0) return AG_ERR_UNSUPPORTED;
+  return launch_out_proj(*desc, O, Wo, X_res, Y, (cudaStream_t)cuda_stream);
+}
+
 int ag_decode_attn(const ag_layer_desc *desc, const void *q, const void *k_new,
                    const void *v_new, const ag_cache *cache, float softmax_scale,
                    void *o, void *ws, size_t ws_bytes, void *cuda_stream) {
@@ -247,8 +259,9 @@ int ag_last_cuda_error(void) { return ag::g_last_cuda_error; }
 int ag_device_wait_timeouts(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return -1;
   const int a = gemm_tc_wait_timeouts(), b = prefill_tc_wait_timeouts(),
-            c = gate_attn_tc_wait_timeouts() + gate_linear_wait_timeouts(), e = kv_proj_cache_wait_timeouts();
-  return (a < 0 || b < 0 || c < 0 || e < 0) ? -1 : a + b + c + e;
+            c = gate_attn_tc_wait_timeouts() + gate_linear_wait_timeouts(), e = kv_proj_cache_wait_timeouts(),
+            f = out_proj_wait_timeouts();
+  return (a < 0 || b < 0 || c < 0 || e < 0 || f < 0) ? -1 : a + b + c + e + f;
 }
 
 }  // extern "C"

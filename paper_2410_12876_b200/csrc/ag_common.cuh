@@ -117,6 +117,11 @@ int prefill_tc_wait_timeouts();
 int launch_prefill_band_mma(const ag_layer_desc &d, const void *Q, const void *K, const void *V,
                             const uint8_t *flags, const float *lse, float scale, void *O, cudaStream_t st);
 
+// Output projection of Eq. 1 with the skip connection: Y = X_res + [H_1 .. H_h] Wo (tensor cores for
+// bf16, head_dim 128; CUDA cores otherwise).
+int launch_out_proj(const ag_layer_desc &d, const void *O, const void *Wo, const void *X_res, void *Y, cudaStream_t st);
+int out_proj_wait_timeouts();
+
 size_t decode_workspace_bytes(const ag_layer_desc &d);
 int launch_decode(const ag_layer_desc &d, const void *q, const void *k_new, const void *v_new,
                   const ag_cache &c, float scale, void *o, void *ws, size_t ws_bytes,

@@ -90,6 +90,13 @@ def layer_weights(shape, seed, device="cpu"):
     }
 
 
+def output_weight(shape, seed, device="cpu", n_layers=1):
+    """W^O [h D, d] of Eq. 1 ~ N(0, 0.02 / sqrt(2 n_layers)): with the skip connection of a stack of
+    n_layers layers and nothing that normalises between them, the hidden states keep their scale."""
+    return randn((shape.heads * shape.head_dim, shape.hidden), seed, device, shape.torch_dtype,
+                 0.02 / math.sqrt(2.0 * n_layers))
+
+
 def linear_gate_weight(shape, seed, device="cpu"):
     """W_lin [d, h] ~ N(0, 1/d) for the local gate (scores of O(1) for unit-variance hidden states)."""
     return randn((shape.hidden, shape.heads), seed, device, shape.torch_dtype, 1.0 / math.sqrt(shape.hidden))
