@@ -40,6 +40,9 @@ WORKLOADS = {
     "stack7b_prev": (inputs.STACK7B, 256, "the stack7b layers with eviction guided by the previous layer (ablation setting 4-1): "
                                          "layer l runs under the flags of layer l-1's gate, the first layer evicts nothing, "
                                          "each gate pass runs on a second stream beside its layer's attention"),
+    "stack7b_chain": (inputs.STACK7B, 256, "32 chained AG-gated layers, batch 8 x seq 4096: every layer projects its Q, K, V from the "
+                                          "hidden states the previous layer produced, X_{l+1} = X_l + [H_1 .. H_h] W^O (no normalisation, "
+                                          "no feed-forward block in between); per-layer mean eviction rising from 10% to 90%"),
     "decode_ragged": (inputs.DECODE_RAGGED, 256, "ragged decode, batch 32 x 32 heads, retained lengths U[0.2,0.9] x 8192, keep-new Bernoulli(0.5)"),
     "decode_ragged_gqa": (inputs.DECODE_RAGGED_GQA, 256, "ragged decode with grouped-query attention, batch 32 x 32 query heads over 8 key/value heads, retained lengths U[0.2,0.9] x 8192"),
 }
@@ -175,12 +178,28 @@ class LayerRun:
         self.name = name
         self.use_graph = True
         self._groups = {}
-        self.has_gate = name in ("prefill7b", "prefill7b_proj", "tiny", "stack7b", "stack7b_prev")
-        self.project = name == "prefill7b_proj"                     # Q, K, V are computed in the step
+        self.has_gate = name in ("prefill7b", "prefill7b_proj", "tiny", "stack7b", "stack7b_prev", "stack7b_chain")
+        self.chain = name == "stack7b_chain"                        # layer l + 1 runs on layer l's output
+        self.project = name == "prefill7b_proj" or self.chain       # Q, K, V are computed in the step
         self.layers = 32 if name.startswith("stack7b") else 1
         self.first_gated = 1 if name == "stack7b_prev" else 0      # 0: every layer evicts by its own gate
         self.has_prefill = name not in ("decode_ragged", "decode_ragged_gqa")
-        if self.has_gate and self.layers > 1:
+        if self.chain:
+            # one X_0; every layer has its own weights (Wq, Wk, Wv, Wo and the gate's); the hidden states
+            # of the later layers are produced by the stack itself, in two buffers used in turn
+            self.X0 = inputs.hidden_states(sh, seed, dev)
+            self.Xbuf = [torch.empty_like(self.X0), torch.empty_like(self.X0)]
+            self.Ws = []
+            for l in range(self.layers):
+                W = inputs.layer_weights(sh, inputs.stack_layer_seed(seed, l) + 10, dev)
+                W["Wo"] = inputs.output_weight(sh, inputs.stack_layer_seed(seed, l) + 30, dev, self.layers)
+                self.Ws.append(W)
+            self.X, self.W = self.X0, self.Ws[0]
+            self.Q = torch.empty(B, h, n, D, dtype=sh.torch_dtype, device=dev)
+            self.K = torch.empty(B, sh.kvh, n, D, dtype=sh.torch_dtype, device=dev)
+            self.V = torch.empty_like(self.K)
+            self.K2, self.V2 = self.K, self.V
+        elif self.has_gate and self.layers > 1:
             # every layer of a stack has its own hidden states X_l, weights and upstream Q, K, V
             self.layer_in = [inputs.stack_layer_inputs(sh, seed, l, dev) for l in range(self.layers)]
             self.X, self.W, self.Q, self.K, self.V = self.layer_in[0]
@@ -230,7 +249,23 @@ class LayerRun:
         self.o = torch.empty(B, h, D, dtype=sh.torch_dtype, device=dev)
         # gamma: per-head keep rate ~ U[0.3, 0.8], calibrated on the scores at gamma = 0
         self.gamma = None
-        if self.has_gate:
+        if self.chain:
+            # gamma of layer l is calibrated on the hidden states the stack itself hands to layer l
+            self.gammas = []
+            for l in range(self.layers):
+                self.set_layer(l)
+                self.gamma = None
+                self.gate()
+                self.gammas.append(inputs.calibrate_gamma(self.scores, inputs.keep_targets_layer(h, seed + 20, l),
+                                                          sh.tau).to(dev))
+                self.gamma = self.gammas[l]
+                self.gate()
+                self.kv_project_cache()
+                self.prefill()
+                self.out_project()
+            self.set_layer(0)
+            self.gamma = self.gammas[0]
+        elif self.has_gate:
             if self.layers > 1:
                 # per layer: mean eviction 10 % (first) ... 90 % (last), gamma calibrated on the layer's
                 # own scores at gamma = 0
@@ -257,8 +292,16 @@ class LayerRun:
         """Point the calls at the inputs of layer `layer` (a stack; a single layer has only layer 0)."""
         self.layer = layer
         self.dq = self.dqs[layer]
-        if self.layers > 1 and self.has_gate:
+        if self.chain:
+            self.X = self.X0 if layer == 0 else self.Xbuf[(layer - 1) % 2]
+            self.X_next = self.Xbuf[layer % 2]
+            self.W = self.Ws[layer]
+        elif self.layers > 1 and self.has_gate:
             self.X, self.W, self.Q, self.K, self.V = self.layer_in[layer]
+
+    def out_project(self):
+        """The layer's output (Eq. 1) with the skip connection: the next layer's hidden states."""
+        self.ag.ag_out_project(self.desc, self.O, self.W["Wo"], self.X, self.X_next)
 
     def gate(self, flags_out=None):
         W, ag = self.W, self.ag
@@ -349,6 +392,8 @@ class LayerRun:
             if self.project:
                 timed("project", self.kv_project_cache)
                 timed("prefill", self.prefill)
+                if self.chain:
+                    timed("out_project", self.out_project)
             elif self.has_prefill:
                 timed("compact", self.compact)
                 timed("prefill", self.prefill)
@@ -408,7 +453,7 @@ class LayerRun:
         gates = (self.layers - self.first_gated) if self.has_gate else 0      # the last guided layer's gate has no consumer
         window = 2 if self.shape.recent_window > 1 else 0      # the ring fill after compaction, the band pass after prefill
         return gates * LAUNCHES["gate"] + self.layers * (
-            (LAUNCHES["compact"] + LAUNCHES["prefill"] + window if self.has_prefill else 0)
+            (LAUNCHES["compact"] + LAUNCHES["prefill"] + window + (1 if self.chain else 0) if self.has_prefill else 0)
             + self.decode_steps * self.decode_launches())
 
     def decode_launches(self):
@@ -438,7 +483,13 @@ class LayerRun:
                 self.gamma = self.gammas[layer]
                 self.gate()
             if self.has_prefill:
-                self.compact()
+                if self.project:
+                    self.kv_project_cache()
+                else:
+                    self.compact()
+                if self.chain:
+                    self.prefill()
+                    self.out_project()
                 P = self.prefix[:, :, :-1].to(torch.float64)
                 f_eff.append(float(4.0 * D * (P.sum() + P.numel())))
                 kept.append(float(self.prefix[:, :, -1].to(torch.float64).sum().item()))
@@ -475,7 +526,7 @@ def flush_l2(buf):
     buf.zero_()
 
 
-CALLS = ("gate", "compact", "project", "prefill", "decode")
+CALLS = ("gate", "compact", "project", "prefill", "out_project", "decode")
 
 
 def timed_passes(run, n_passes, l2buf):
@@ -531,6 +582,9 @@ def rooflines_of(run, per_call_ms, peaks, workload):
         if "project" in per_call_ms:
             kf = 2.0 * sh.batch * sh.seq * sh.hidden * (2 * sh.kvh + sh.heads) * sh.head_dim
             out["project"] = entry("tensor", "ag_qkv_project_cache", kf, per_call_ms["project"], "project")
+        if "out_project" in per_call_ms:
+            of = 2.0 * sh.batch * sh.seq * sh.heads * sh.head_dim * sh.hidden
+            out["out_project"] = entry("tensor", "ag_out_project", of, per_call_ms["out_project"], "out_project")
     if run.has_gate:
         out["gate"] = entry("tensor", "ag_gate_forward", run.gate_flops(), per_call_ms["gate"], "gate")
     return out
@@ -625,7 +679,9 @@ def run_ours(args, rank, world, dev):
     # end to end: pinned host inputs in, results out, through the same calls
     sh = run.shape
     stack = run.layers > 1 and run.has_gate
-    if stack:
+    if run.chain:
+        dev_in = [run.X0] + [u for dq in run.dqs for q in dq for u in q]
+    elif stack:
         dev_in = [t for (X, W, Q, K, V), dq in zip(run.layer_in, run.dqs) for t in [X, Q, K, V] + [u for q in dq for u in q]]
     elif run.project:
         dev_in = [run.X]                                     # Q, K and V are made on the device
@@ -648,6 +704,10 @@ def run_ours(args, rank, world, dev):
     # decode), and the flags and each group's O go back to the host while later groups come in.
     # Other workloads: copy in, step, copy out, in order.
     overlap = run.has_gate and run.has_prefill and run.layers == 1
+    if run.chain:
+        dev_out.append(run.Xbuf[(run.layers - 1) % 2])      # the stack's final hidden states
+        host_out.append(torch.empty(run.X0.shape, dtype=run.X0.dtype).pin_memory())
+        d2h = sum(t.numel() * t.element_size() for t in host_out)
     if overlap and run.project:
         main = torch.cuda.current_stream()
         s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
@@ -797,7 +857,7 @@ def run_ours(args, rank, world, dev):
         "decode_tokens_per_s": sh.batch * run.decode_steps / (per_call_ms["decode"] * 1e-3),
     }
     if run.has_prefill:
-        pre_ms = sum(per_call_ms.get(k, 0.0) for k in ("gate", "compact", "project", "prefill"))
+        pre_ms = sum(per_call_ms.get(k, 0.0) for k in ("gate", "compact", "project", "prefill", "out_project"))
         out["prefill_tokens_per_s"] = sh.batch * sh.seq / (pre_ms * 1e-3)
     if args.workload == "prefill7b" and world == 1 and not args.no_extra and args.recent_window <= 1:
         # the other full-size workloads, briefly: their rooflines ride in the same line

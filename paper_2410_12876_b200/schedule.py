@@ -56,3 +56,47 @@ class PreviousLayerGate:
         done = torch.cuda.Event()
         done.record(self.gate_stream)
         main.wait_event(done)
+
+
+class ChainedLayerBuffers:
+    """Device buffers one layer of a chained stack works in (shared by all layers of the stack: a
+    layer's Q, K, V, O, flags and cache are dead once its output has been projected, except for the
+    cache when decode steps follow)."""
+
+    def __init__(self, ag, shape, extra_rows=0, device="cuda"):
+        import torch as _t
+        B, h, hk, n, D = shape.batch, shape.heads, shape.kvh, shape.seq, shape.head_dim
+        dt = shape.torch_dtype
+        self.desc = ag.make_desc(shape)
+        self.scores = _t.empty(B, hk, n, dtype=_t.float32, device=device)
+        self.flags = _t.empty(B, hk, n, dtype=_t.uint8, device=device)
+        self.prefix = _t.empty(B, hk, n + 1, dtype=_t.int32, device=device)
+        self.Q = _t.empty(B, h, n, D, dtype=dt, device=device)
+        self.K = _t.empty(B, hk, n, D, dtype=dt, device=device)
+        self.V = _t.empty(B, hk, n, D, dtype=dt, device=device)
+        self.O = _t.empty(B, h, n, D, dtype=dt, device=device)
+        self.cache = ag.RaggedCache.allocate(shape, [n + extra_rows] * (B * hk), device)
+        self.status = _t.zeros(1, dtype=_t.int32, device=device)
+        self.ws_gate = ag.workspace(self.desc, ag.AG_CALL_GATE, device)
+        self.ws_prefill = ag.workspace(self.desc, ag.AG_CALL_PREFILL, device)
+
+
+def chained_layer(ag, buf, X, W, gamma, X_next, after=None):
+    """Enqueues one layer of a chained stack of attention layers on the current stream: the gate on
+    the layer's hidden states X (Sec. 3.3), the Q, K, V projection of Eq. 2 that writes the retained
+    rows into the cache, prefill attention under the eviction mask (Eq. 5), and the output
+    projection of Eq. 1 with the skip connection, X_next = X + [H_1 .. H_h] W^O: the next layer's
+    hidden states.  Nothing normalises and no feed-forward block sits between two layers.
+    W: dict with Wq, Wk, Wv, Wo and the gate's Wq_g, Wk_g, Wv_g, Wo_g.  after (optional) is called
+    between the layer's calls with the name of the call just enqueued (for timing marks)."""
+    mark = after if after is not None else (lambda name: None)
+    ag.ag_gate_forward(buf.desc, X, W["Wq_g"], W["Wk_g"], W["Wv_g"], W["Wo_g"], gamma, buf.scores, buf.flags,
+                       buf.ws_gate)
+    mark("gate")
+    ag.ag_qkv_project_cache(buf.desc, X, W["Wq"], W["Wk"], W["Wv"], buf.flags, buf.cache, buf.prefix, None, buf.Q,
+                            buf.K, buf.V, buf.status)
+    mark("project")
+    ag.ag_prefill_attn(buf.desc, buf.Q, buf.K, buf.V, buf.flags, buf.cache, buf.prefix, 0.0, buf.O, buf.ws_prefill)
+    mark("prefill")
+    ag.ag_out_project(buf.desc, buf.O, W["Wo"], X, X_next)
+    mark("out_project")
