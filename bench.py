@@ -806,6 +806,7 @@ def run_ours(args, rank, world, dev):
         return None
     tokens = run.tokens_per_step() * world
     peaks = _peaks()
+    near = near_threshold_fractions(run) if run.has_gate else None     # on the scores of the step's own gate pass
     rooflines = rooflines_of(run, per_call_ms, peaks, args.workload)
     if run.has_gate and run.layers == 1:
         # the local gate variant, timed apart from the step (L2 flushed before each call)
@@ -843,7 +844,7 @@ def run_ours(args, rank, world, dev):
                    "step": f"{passes} passes of the whole path over the batch, L2 flushed before each pass (outside its events)",
                    "recent_window": max(1, sh.recent_window),
                    "mean_keep": float(run.flags.float().mean().item()) if run.has_prefill else None,
-                   "near_threshold": near_threshold_fractions(run) if run.has_gate else None,
+                   "near_threshold": near,
                    "replicas": world,
                    "decode_launch": "one CUDA graph per pass" if run.use_graph else "individual launches"},
         "clocks": clocks,
