@@ -286,16 +286,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int e = 0; e < kPfBN; ++e)
           if (e >= nvalid) r[e] = 0xff800000u;        // -inf: weight 0 below
       }
-      // eight independent chains instead of one long dependency
+      // eight independent chains instead of one long dependency, two elements per instruction
       float mx[8];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) mx[q] = __uint_as_float(r[q]);
+      for (int q = 0; q < 8; ++q) mx[q] = max3_f32(__uint_as_float(r[q]), __uint_as_float(r[q + 8]), __uint_as_float(r[q + 16]));
 #pragma unroll
-      for (int e = 8; e < kPfBN; e += 8)
+      for (int e = 24; e + 8 < kPfBN; e += 16)
 #pragma unroll
-        for (int q = 0; q < 8; ++q) mx[q] = fmaxf(mx[q], __uint_as_float(r[e + q]));
-      float tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+        for (int q = 0; q < 8; ++q) mx[q] = max3_f32(mx[q], __uint_as_float(r[e + q]), __uint_as_float(r[e + q + 8]));
+#pragma unroll
+      for (int q = 0; q < 8; ++q) mx[q] = fmaxf(mx[q], __uint_as_float(r[kPfBN - 8 + q]));
+      float tmax = max3_f32(max3_f32(mx[0], mx[1], mx[2]), max3_f32(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]));
       tmax *= a.scale_log2;                           // scale > 0: max commutes; -inf stays -inf
       float m_new;
       if (i == 0) m_new = fmaxf(m, tmax);
@@ -303,21 +304,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const bool rescale = (i > 0) && __any_sync(0xffffffffu, m_new != m);
       const float alpha = fast_exp2(m - m_new);
 
-      // p = 2^(s - m) as bf16 pairs, written over the columns S occupied
-      float rs[4] = {0.f, 0.f, 0.f, 0.f};
+      // p = 2^(s - m) as bf16 pairs, written over the columns S occupied; the scaling and the row
+      // sums two elements per instruction
+      float rs[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      const float neg_m = -m_new;
 #pragma unroll
       for (int c = 0; c < kPfBN / 16; ++c) {
         uint32_t pk[8];
 #pragma unroll
         for (int e = 0; e < 16; e += 2) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e]), a.scale_log2, -m_new));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(r[c * 16 + e + 1]), a.scale_log2, -m_new));
-          rs[(e >> 1) & 3] += p0 + p1;
+          float t0, t1;
+          fma_f32x2(t0, t1, __uint_as_float(r[c * 16 + e]), __uint_as_float(r[c * 16 + e + 1]), a.scale_log2,
+                    a.scale_log2, neg_m, neg_m);
+          const float p0 = fast_exp2(t0), p1 = fast_exp2(t1);
+          const int k = ((e >> 1) & 3) * 2;
+          add_f32x2(rs[k], rs[k + 1], rs[k], rs[k + 1], p0, p1);
           pk[e >> 1] = pack_bf16x2(p0, p1);
         }
         tmem_st_x8(tS + c * 8, pk);
       }
-      l = l * alpha + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
+      l = l * alpha + (((rs[0] + rs[1]) + (rs[2] + rs[3])) + ((rs[4] + rs[5]) + (rs[6] + rs[7])));
       m = m_new;
 
       // Only a rescale of O has to wait for the P V of tile i - 1.  The parity wait is unambiguous
