@@ -90,7 +90,10 @@ typedef struct {
                             alone would give (the bidirectional MHA' sees seq_lens[b]
                             keys), and every padding position gets flag 0, so it is
                             never cached and never attended to; scores and attention
-                            outputs at padding positions are unspecified.            */
+                            outputs at padding positions are unspecified.  With a
+                            recent-token window, ag_compact_kv and ag_kv_project_cache
+                            read it too: the ring takes the last tokens of each
+                            sequence's own prompt.                                   */
   int32_t kv_heads;      /* 0 (= heads), or the number of key/value heads of grouped-query
                             attention: heads must be a multiple; query head i reads
                             key/value head i / (heads / kv_heads).  K, V, k_new, v_new,
@@ -104,7 +107,7 @@ typedef struct {
                             (6-1), (6-2): w = 5, 10); an evicted token leaves the attention
                             of later tokens once it is w or more positions behind.  What is
                             cached for good is unchanged.  The cache then needs its
-                            recent_* arrays; not combined with seq_lens (AG_ERR_UNSUPPORTED). */
+                            recent_* arrays.                                           */
 } ag_layer_desc;
 
 /* Ragged per-(sequence, head) cache of retained keys and values.  The struct
@@ -230,9 +233,9 @@ int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
  * ag_compact_kv.  The cache rows are bit copies of the dense K, V rows.
  * With a recent-token window the ring of the cache is filled from the dense K, V,
  * as ag_compact_kv fills it.
- * Needs no workspace.  Kernel coverage: bfloat16, head_dim 128, d a multiple of 8,
- * and n a multiple of 128 unless batch = 1 (any n); anything else returns
- * AG_ERR_UNSUPPORTED (project with a GEMM of your own and call ag_compact_kv).
+ * Needs no workspace.  Kernel coverage: bfloat16, head_dim 128, d a multiple of 8
+ * (any batch, any n); anything else returns AG_ERR_UNSUPPORTED (project with a
+ * GEMM of your own and call ag_compact_kv).
  * AG_ERR_INVALID_ARG for missing or misaligned (16-byte) pointers.
  */
 int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk,
@@ -289,8 +292,8 @@ int ag_prefill_attn(const ag_layer_desc *desc, const void *Q, const void *K,
  *   Wo     [h D, d]              in   ("in x out")
  *   X_res  [B, n, d] or NULL     in   skip connection (NULL: Y = MHA(X))
  *   Y      [B, n, d]             out  must not be X_res or O
- * Tensor-core coverage: bfloat16, head_dim 128, d a multiple of 128, and n a multiple of 128
- * unless batch = 1; other shapes run on CUDA cores (B n <= 65535), else AG_ERR_UNSUPPORTED.
+ * Tensor-core coverage: bfloat16, head_dim 128, d a multiple of 128; other shapes run on
+ * CUDA cores (B n <= 65535), else AG_ERR_UNSUPPORTED.
  * AG_ERR_INVALID_ARG for missing or misaligned (16-byte) pointers.
  */
 int ag_out_project(const ag_layer_desc *desc, const void *O, const void *Wo, const void *X_res,

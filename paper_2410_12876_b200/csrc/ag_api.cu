@@ -1,6 +1,7 @@
 // C boundary of the AG-gated attention layer: argument checks and dispatch.
 // Every check that can be made on the host is made here, before any launch.
 #include <math.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include "ag_common.cuh"
 
@@ -20,7 +21,6 @@ int check_desc(const ag_layer_desc *d) {
   if (d->kv_heads < 0 || (d->kv_heads > 0 && d->heads % d->kv_heads != 0)) return AG_ERR_INVALID_ARG;
   if (d->recent_window < 0) return AG_ERR_INVALID_ARG;
   if (d->recent_window > kMaxRecent + 1) return AG_ERR_UNSUPPORTED;
-  if (recent_rows(*d) > 0 && d->seq_lens) return AG_ERR_UNSUPPORTED;
   return AG_OK;
 }
 
@@ -62,6 +62,15 @@ static int check_ws(size_t need, void *ws, size_t ws_bytes) {
 
 using namespace ag;
 
+namespace {
+// A named range around every call of the boundary, for timelines: the header-only NVTX layer does
+// nothing (one predictable branch) unless a profiler has attached itself to the process.
+struct CallRange {
+  explicit CallRange(const char *name) { nvtxRangePushA(name); }
+  ~CallRange() { nvtxRangePop(); }
+};
+}  // namespace
+
 extern "C" {
 
 size_t ag_workspace_bytes(const ag_layer_desc *desc, int which) {
@@ -83,6 +92,7 @@ int ag_gate_forward(const ag_layer_desc *desc, const void *X, const void *Wq_g,
                     const void *Wk_g, const void *Wv_g, const void *Wo_g,
                     const float *gamma, float *scores, uint8_t *flags, void *ws,
                     size_t ws_bytes, void *cuda_stream) {
+  CallRange range_("ag_gate_forward");
   int st = check_gate_desc(desc);
   if (st) return st;
   if (!X || !Wq_g || !Wk_g || !Wv_g || !Wo_g || !flags) return AG_ERR_INVALID_ARG;
@@ -97,6 +107,7 @@ int ag_gate_forward(const ag_layer_desc *desc, const void *X, const void *Wq_g,
 
 int ag_gate_linear_forward(const ag_layer_desc *desc, const void *X, const void *W_lin,
                            const float *gamma, float *scores, uint8_t *flags, void *cuda_stream) {
+  CallRange range_("ag_gate_linear_forward");
   int st = check_desc(desc);
   if (st) return st;
   if (desc->hidden <= 0 || !(desc->tau > 0.f && desc->tau < 1.f)) return AG_ERR_INVALID_ARG;
@@ -110,6 +121,7 @@ int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
                   const uint8_t *flags, ag_cache *cache, int32_t *prefix,
                   int32_t *idx, int32_t *dev_status, void *ws, size_t ws_bytes,
                   void *cuda_stream) {
+  CallRange range_("ag_compact_kv");
   int st = check_desc(desc);
   if (st) return st;
   if (!flags || !prefix) return AG_ERR_INVALID_ARG;
@@ -130,6 +142,7 @@ int ag_compact_kv(const ag_layer_desc *desc, const void *K, const void *V,
 int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk, const void *Wv,
                         const uint8_t *flags, ag_cache *cache, int32_t *prefix, int32_t *idx, void *K, void *V,
                         int32_t *dev_status, void *cuda_stream) {
+  CallRange range_("ag_kv_project_cache");
   int st = check_desc(desc);
   if (st) return st;
   if (desc->hidden <= 0) return AG_ERR_INVALID_ARG;
@@ -147,6 +160,7 @@ int ag_kv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wk
 int ag_qkv_project_cache(const ag_layer_desc *desc, const void *X, const void *Wq, const void *Wk, const void *Wv,
                          const uint8_t *flags, ag_cache *cache, int32_t *prefix, int32_t *idx, void *Q, void *K,
                          void *V, int32_t *dev_status, void *cuda_stream) {
+  CallRange range_("ag_qkv_project_cache");
   int st = check_desc(desc);
   if (st) return st;
   if (desc->hidden <= 0) return AG_ERR_INVALID_ARG;
@@ -165,6 +179,7 @@ int ag_prefill_attn(const ag_layer_desc *desc, const void *Q, const void *K,
                     const void *V, const uint8_t *flags, const ag_cache *cache,
                     const int32_t *prefix, float softmax_scale, void *O, void *ws,
                     size_t ws_bytes, void *cuda_stream) {
+  CallRange range_("ag_prefill_attn");
   int st = check_desc(desc);
   if (st) return st;
   if (!Q || !K || !V || !flags || !prefix || !O) return AG_ERR_INVALID_ARG;
@@ -183,6 +198,7 @@ int ag_prefill_attn(const ag_layer_desc *desc, const void *Q, const void *K,
 
 int ag_out_project(const ag_layer_desc *desc, const void *O, const void *Wo, const void *X_res, void *Y,
                    void *cuda_stream) {
+  CallRange range_("ag_out_project");
   int st = check_desc(desc);
   if (st) return st;
   if (desc->hidden <= 0) return AG_ERR_INVALID_ARG;
@@ -196,6 +212,7 @@ int ag_out_project(const ag_layer_desc *desc, const void *O, const void *Wo, con
 int ag_decode_attn(const ag_layer_desc *desc, const void *q, const void *k_new,
                    const void *v_new, const ag_cache *cache, float softmax_scale,
                    void *o, void *ws, size_t ws_bytes, void *cuda_stream) {
+  CallRange range_("ag_decode_attn");
   int st = check_desc(desc);
   if (st) return st;
   if (!q || !k_new || !v_new || !o) return AG_ERR_INVALID_ARG;
@@ -214,6 +231,7 @@ int ag_decode_attn(const ag_layer_desc *desc, const void *q, const void *k_new,
 int ag_decode_step(const ag_layer_desc *desc, const void *q, const void *k_new, const void *v_new,
                    const uint8_t *flag_new, ag_cache *cache, float softmax_scale, void *o,
                    int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream) {
+  CallRange range_("ag_decode_step");
   int st = check_desc(desc);
   if (st) return st;
   if (!q || !k_new || !v_new || !flag_new || !o) return AG_ERR_INVALID_ARG;
@@ -232,6 +250,7 @@ int ag_decode_step(const ag_layer_desc *desc, const void *q, const void *k_new, 
 int ag_cache_append(const ag_layer_desc *desc, const void *k_new, const void *v_new,
                     const uint8_t *flag_new, ag_cache *cache, int32_t *dev_status,
                     void *cuda_stream) {
+  CallRange range_("ag_cache_append");
   int st = check_desc(desc);
   if (st) return st;
   if (!k_new || !v_new || !flag_new) return AG_ERR_INVALID_ARG;

@@ -88,7 +88,7 @@ int launch_compact(const ag_layer_desc &d, const void *K, const void *V, const u
                    void *ws, cudaStream_t st);
 
 // Key/value projection (Eq. 2) on the tensor cores with the retained rows written straight into the
-// ragged cache (bf16, head_dim 128, seq a multiple of 128).
+// ragged cache (bf16, head_dim 128).
 bool kv_proj_cache_supported(const ag_layer_desc &d);
 // Wq, Q: NULL, or the query projection Q = X Wq rides in the same launch (dense output only).
 int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, const void *Wv,

@@ -150,16 +150,19 @@ append_rows_kernel(const uint8_t *__restrict__ k_new, const uint8_t *__restrict_
 
 // Recent-token window: after the prompt, the ring of a slab holds its last R tokens (token t in
 // slot t % R), the evicted ones marked live; a prompt shorter than R leaves the other slots dead.
+// With per-sequence lengths the prompt of a slab is the first seq_lens[b] of its n positions.
 // One CTA per slab, thread (slot, 16-byte piece).
 template <int kRowBytes>
 __global__ void recent_fill_kernel(const uint8_t *__restrict__ K, const uint8_t *__restrict__ V,
-                                   const uint8_t *__restrict__ flags, int n, const RecentRing ring) {
+                                   const uint8_t *__restrict__ flags, int n, const int32_t *__restrict__ seq_lens,
+                                   int kv_heads, const RecentRing ring) {
   constexpr int kVecs = kRowBytes / 16;
   const int slab = blockIdx.x, slot = threadIdx.x / kVecs, v = threadIdx.x % kVecs;
   if (slot >= ring.R) return;
+  const int len = seq_lens ? min(max(seq_lens[slab / kv_heads], 0), n) : n;   // tokens of this slab's prompt
   // the last token whose number is slot modulo R, if the prompt has one
-  const bool have = slot <= n - 1;
-  const int t = have ? slot + (n - 1 - slot) / ring.R * ring.R : 0;
+  const bool have = slot <= len - 1;
+  const int t = have ? slot + (len - 1 - slot) / ring.R * ring.R : 0;
   if (have) {
     const size_t src = ((size_t)slab * n + t) * kRowBytes + v * 16;
     const size_t dst = ((size_t)slab * ring.R + slot) * kRowBytes + v * 16;
@@ -167,7 +170,7 @@ __global__ void recent_fill_kernel(const uint8_t *__restrict__ K, const uint8_t 
     *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(ring.v) + dst) = *reinterpret_cast<const uint4 *>(V + src);
   }
   if (v == 0) ring.live[(size_t)slab * ring.R + slot] = (have && flags[(size_t)slab * n + t] == 0) ? 1 : 0;
-  if (threadIdx.x == 0) ring.pos[slab] = n;
+  if (threadIdx.x == 0) ring.pos[slab] = len;
 }
 
 static int row_bytes(const ag_layer_desc &d) {
@@ -221,9 +224,9 @@ int launch_recent_fill(const ag_layer_desc &d, const void *K, const void *V, con
   auto Vb = static_cast<const uint8_t *>(V);
   const int threads = ring.R * (row_bytes(d) / 16);
   switch (row_bytes(d)) {
-    case 128: recent_fill_kernel<128><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
-    case 256: recent_fill_kernel<256><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
-    default: recent_fill_kernel<512><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, ring); break;
+    case 128: recent_fill_kernel<128><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, d.seq_lens, kv_heads_of(d), ring); break;
+    case 256: recent_fill_kernel<256><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, d.seq_lens, kv_heads_of(d), ring); break;
+    default: recent_fill_kernel<512><<<slabs, threads, 0, st>>>(Kb, Vb, flags, d.seq, d.seq_lens, kv_heads_of(d), ring); break;
   }
   AG_LAUNCH_CHECK();
   return AG_OK;

@@ -15,6 +15,7 @@
 // to the workspace and decode_combine_kernel merges them.
 #include <cooperative_groups.h>
 #include <math.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <type_traits>
 
@@ -769,6 +770,8 @@ extern "C" int ag_decode_attn_noalloc(const ag_layer_desc *desc, const void *q, 
                                       const void *v_new, const ag_cache *cache, float softmax_scale,
                                       void *o, void *cuda_stream) {
   using namespace ag;
+  nvtxRangePushA("ag_decode_attn_noalloc");          // (does nothing unless a profiler is attached)
+  struct Pop { ~Pop() { nvtxRangePop(); } } pop_;
   // the same host-side checks as ag_decode_attn, before anything is launched
   int st = check_desc(desc);
   if (st) return st;

@@ -51,7 +51,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                      const __grid_constant__ CUtensorMap tmQ, const uint8_t *__restrict__ flags,
                      int32_t *__restrict__ prefix, int32_t *__restrict__ idx, const int64_t *__restrict__ row_off,
                      const int32_t *__restrict__ cap, int32_t *__restrict__ len, uint8_t *__restrict__ k_rows,
-                     uint8_t *__restrict__ v_rows, int32_t *__restrict__ dev_status, int M, int Kdim, int GD,
+                     uint8_t *__restrict__ v_rows, int32_t *__restrict__ dev_status, int n_sub, int tps, int Kdim, int GD,
                      int n, int kv_heads, int heads, int n_tiles_m, int n_tiles_n, int split_from) {
   using Cfg = KvCfg<BN, MT>;
   constexpr uint32_t kTmemCols = MT * BN;
@@ -78,7 +78,10 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   const int band = tile / (kBandTiles * n_tiles_n), in_band = tile % (kBandTiles * n_tiles_n);
   const int band_rows = min(kBandTiles, n_tiles_m - band * kBandTiles);
   const int tile_m = band * kBandTiles + in_band % band_rows, tile_n = in_band / band_rows;
-  const int m0 = tile_m * (MT * kBM) + (single ? ((cta - split_from) & 1) * kBM : 0);
+  // Rows are counted in sub-tiles of 128 tokens laid out per sequence: sequence b owns sub-tiles
+  // [b tps, (b + 1) tps), the last of which may reach past the sequence's end (those rows are zeros on
+  // the way in, take no rank, and are dropped by the stores), so a sub-tile never spans two sequences.
+  const int sub0 = tile_m * MT + (single ? ((cta - split_from) & 1) : 0);
   const int n0 = tile_n * BN;                    // in the packed output [K | V | Q] (GD, GD and heads * D columns)
   // BN divides the width of every weight: a tile lies in one weight.  which: 0 keys, 1 values, 2 queries
   // (queries go to their dense tensor only: no flags, no cache)
@@ -114,8 +117,9 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         uint8_t *a = smem + s * Cfg::kStageBytes, *b = a + Cfg::kABytes;
         mbar_arrive_expect_tx(&full[s], mts * (kBM * kBK * 2) + Cfg::kBBytes);
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt)              // rows past M are filled with zeros
-          if (mt < mts) tma_load_2d(a + mt * (kBM * kBK * 2), &tmA, &full[s], kb * kBK, m0 + mt * kBM);
+        for (int mt = 0; mt < MT; ++mt)              // rows past the sequence (or past the batch) are filled with zeros
+          if (mt < mts)
+            tma_load_3d(a + mt * (kBM * kBK * 2), &tmA, &full[s], kb * kBK, ((sub0 + mt) % tps) * kBM, (sub0 + mt) / tps);
 #pragma unroll
         for (int p = 0; p < BN / 64; ++p)
           tma_load_2d(b + p * Cfg::kPanelBytes, tmB, &full[s], nw + p * 64, kb * kBK);
@@ -162,14 +166,12 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     // prefix (and idx), and the one that holds a sequence's first token the slab's length.
 #pragma unroll
     for (int mt = 0; mt < (half == 0 ? MT : 0); ++mt) {           // warps 2..5 only
-      const int m_base = m0 + mt * kBM;
-      // one sequence per sub-tile: n is a multiple of 128, or there is a single sequence (whose last
-      // sub-tile may reach past its end: those rows are skipped here and dropped by the TMA stores)
-      const int b = m_base / n, t0 = m_base % n, t = t0 + r_in;
+      const int sub = sub0 + mt;
+      const int b = sub / tps, t0 = (sub % tps) * kBM, t = t0 + r_in;
 #pragma unroll
       for (int hh = 0; hh < Cfg::kHeads; ++hh) {
         long long d = -1;
-        if (m_base < M && mt < mts && which != 2) {               // the same for all 128 threads
+        if (sub < n_sub && mt < mts && which != 2) {                // the same for all 128 threads
           const size_t slab = (size_t)b * kv_heads + nw / kD + hh;
           const uint8_t *f = flags + slab * n;
           int before = 0, total = 0;
@@ -234,8 +236,8 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const int hw = (warp - 2) * 2 + (lane >> 4), l16 = lane & 15;   // half-warp 0..15, 16-byte piece of a row
 #pragma unroll 1
     for (int mt = 0; mt < MT; ++mt) {
-      const int m_base = m0 + mt * kBM;
-      if (!ok || num_kb == 0 || m_base >= M || mt >= mts) break;
+      const int sub = sub0 + mt;
+      if (!ok || num_kb == 0 || sub >= n_sub || mt >= mts) break;
       const uint32_t tmem_sub = tmem_acc + mt * BN;
       // bf16 tile as panels of [128 tokens][64 columns] (128-byte rows, 16-byte chunks XOR-swizzled by the
       // row); each sub-tile has a staging area of its own, so the second is drained while the first leaves
@@ -257,7 +259,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       }
       fence_proxy_async_smem();
       named_barrier_sync(1, 256);                  // the tile is staged (and dst_row written, first time round)
-      const int b = m_base / n, t0 = m_base % n;
+      const int b = sub / tps, t0 = (sub % tps) * kBM;
       if (threadIdx.x == 64) {
 #pragma unroll
         for (int p = 0; p < BN / 64; ++p)
@@ -301,10 +303,11 @@ int run(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, c
         const ag_cache &c, int32_t *prefix, int32_t *idx, void *Q, void *K, void *V, int32_t *dev_status,
         cudaStream_t st) {
   using Cfg = KvCfg<BN, MT>;
-  const int hk = kv_heads_of(d), GD = hk * kD, M = d.batch * d.seq, Kdim = d.hidden;
+  const int hk = kv_heads_of(d), GD = hk * kD, Kdim = d.hidden;
+  const int tps = (d.seq + kBM - 1) / kBM, n_sub = d.batch * tps;   // sub-tiles of 128 tokens per sequence, in all
   const int QD = Wq ? d.heads * kD : 0;          // query columns of the packed output (0: keys and values only)
   CUtensorMap tmA, tmBk, tmBv, tmBq, tmK, tmV, tmQ;
-  int rc = make_tmap_2d_bf16(&tmA, X, M, Kdim, (uint64_t)Kdim * 2, kBM, kBK);
+  int rc = make_tmap_3d_bf16(&tmA, X, d.batch, d.seq, Kdim, kBM, kBK);
   if (rc) return rc;
   rc = make_tmap_2d_bf16(&tmBk, Wk, Kdim, GD, (uint64_t)GD * 2, kBK, 64);
   if (rc) return rc;
@@ -324,13 +327,13 @@ int run(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, c
   }
   auto kern = kv_proj_cache_kernel<BN, MT>;
   AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-  const int n_tiles_n = (2 * GD + QD) / BN, n_tiles_m = (M + MT * kBM - 1) / (MT * kBM), n_tiles = n_tiles_n * n_tiles_m;
+  const int n_tiles_n = (2 * GD + QD) / BN, n_tiles_m = (n_sub + MT - 1) / MT, n_tiles = n_tiles_n * n_tiles_m;
   const int tail = n_tiles % sm_count();
   const int split_from = (MT > 1 && tail > 0 && 2 * tail <= sm_count()) ? n_tiles - tail : n_tiles;
   const int ctas = split_from + 2 * (n_tiles - split_from);
   kern<<<ctas, kThreads, Cfg::kSmemBytes, st>>>(tmA, tmBk, tmBv, tmBq, tmK, tmV, tmQ, flags, prefix, idx, c.row_off, c.cap, c.len,
                                                    static_cast<uint8_t *>(c.k_rows), static_cast<uint8_t *>(c.v_rows),
-                                                   dev_status, M, Kdim, GD, d.seq, hk, d.heads, n_tiles_m, n_tiles_n, split_from);
+                                                   dev_status, n_sub, tps, Kdim, GD, d.seq, hk, d.heads, n_tiles_m, n_tiles_n, split_from);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
@@ -338,15 +341,15 @@ int run(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, c
 }  // namespace
 
 bool kv_proj_cache_supported(const ag_layer_desc &d) {
-  return d.dtype == AG_BF16 && d.head_dim == kD && (d.seq % kBM == 0 || d.batch == 1) && d.hidden > 0 && d.hidden % 8 == 0 &&
-         (int64_t)d.batch * d.seq < ((int64_t)1 << 31);
+  return d.dtype == AG_BF16 && d.head_dim == kD && d.hidden > 0 && d.hidden % 8 == 0 &&
+         (int64_t)d.batch * (d.seq + kBM) < ((int64_t)1 << 31);
 }
 
 int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, const void *Wv,
                          const uint8_t *flags, const ag_cache &c, int32_t *prefix, int32_t *idx, void *Q, void *K,
                          void *V, int32_t *dev_status, cudaStream_t st) {
   const int hk = kv_heads_of(d), hq = Wq ? d.heads : 0;
-  const long long tiles128 = (long long)(2 * hk + hq) * (d.batch * (long long)d.seq / kBM);
+  const long long tiles128 = (long long)(2 * hk + hq) * d.batch * ((d.seq + kBM - 1) / kBM);
   int rc;
   if (hk % 2 == 0 && hq % 2 == 0) {
     // more than one wave: 256-token tiles, whose two sub-tiles share every stage of W

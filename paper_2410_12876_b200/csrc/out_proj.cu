@@ -40,8 +40,8 @@ template <int BN, int MT> struct OpCfg {
 template <int BN, int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmW,
-                   const __grid_constant__ CUtensorMap tmY, const __nv_bfloat16 *__restrict__ X_res, int M, int n,
-                   int heads, int d, int n_tiles_m, int n_tiles_n, int split_from) {
+                   const __grid_constant__ CUtensorMap tmY, const __nv_bfloat16 *__restrict__ X_res, int n_sub, int tps,
+                   int n, int heads, int d, int n_tiles_m, int n_tiles_n, int split_from) {
   using Cfg = OpCfg<BN, MT>;
   constexpr uint32_t kTmemCols = MT * BN;
   static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "TMEM columns: a power of two");
@@ -63,7 +63,10 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
   const int band = tile / (kBandTiles * n_tiles_n), in_band = tile % (kBandTiles * n_tiles_n);
   const int band_rows = min(kBandTiles, n_tiles_m - band * kBandTiles);
   const int tile_m = band * kBandTiles + in_band % band_rows, tile_n = in_band / band_rows;
-  const int m0 = tile_m * (MT * kBM) + (single ? ((cta - split_from) & 1) * kBM : 0);
+  // Rows are counted in sub-tiles of 128 tokens laid out per sequence: sequence b owns sub-tiles
+  // [b tps, (b + 1) tps), the last of which may reach past the sequence's end (zeros on the way in,
+  // dropped on the way out), so a sub-tile never spans two sequences.
+  const int sub0 = tile_m * MT + (single ? ((cta - split_from) & 1) : 0);
   const int n0 = tile_n * BN;
   const int num_kb = heads * (kD / kBK);         // K = h D, 64 at a time: two blocks per head
 
@@ -97,9 +100,8 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
           if (mt < mts) {
-            // a sub-tile of 128 tokens lies in one sequence (n is a multiple of 128, or there is one
-            // sequence); tokens past its end, and whole sub-tiles past M, are filled with zeros
-            const int m_base = m0 + mt * kBM, b_seq = m_base / n, t0 = m_base % n;
+            // tokens past the sequence's end, and whole sub-tiles past the batch, are filled with zeros
+            const int sub = sub0 + mt, b_seq = sub / tps, t0 = (sub % tps) * kBM;
             tma_load_3d(a + mt * (kBM * kBK * 2), &tmO, &full[s], col, t0, b_seq * heads + head);
           }
         }
@@ -146,14 +148,15 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
     // this thread's piece of the skip connection for the first sub-tile, fetched while the MMAs run
     uint4 res[kChunks][4];
     auto fetch_residual = [&](int mt) {
-      const int row = m0 + mt * kBM + r_in;
-      const bool have = X_res != nullptr && row < M && mt < mts;
+      const int sub = sub0 + mt, t = (sub % tps) * kBM + r_in;
+      const bool have = X_res != nullptr && sub < n_sub && t < n && mt < mts;
+      const size_t row = (size_t)(sub / tps) * n + t;
 #pragma unroll
       for (int ci = 0; ci < kChunks; ++ci) {
         const int c = half * (BN / 2) + ci * 32;
 #pragma unroll
         for (int q = 0; q < 4; ++q)
-          res[ci][q] = have ? ldg128_stream(X_res + (size_t)row * d + n0 + c + q * 8) : make_uint4(0, 0, 0, 0);
+          res[ci][q] = have ? ldg128_stream(X_res + row * d + n0 + c + q * 8) : make_uint4(0, 0, 0, 0);
       }
     };
     fetch_residual(0);
@@ -164,8 +167,8 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
     tc_fence_after_sync();
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
-      const int m_base = m0 + mt * kBM;
-      if (!ok || m_base >= M || mt >= mts) break;           // the same for all 256 threads
+      const int sub = sub0 + mt;
+      if (!ok || sub >= n_sub || mt >= mts) break;          // the same for all 256 threads
       const uint32_t tmem_sub = tmem_acc + mt * BN;
       // bf16 tile as panels of [128 tokens][64 columns] (128-byte rows, 16-byte chunks XOR-swizzled by the
       // row); each sub-tile has a staging area of its own, so the second is drained while the first leaves
@@ -193,8 +196,8 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
       named_barrier_sync(1, 256);                  // the tile is staged
       if (threadIdx.x == 64) {
 #pragma unroll
-        for (int p = 0; p < BN / 64; ++p)          // rows past M are dropped by the tensor map
-          tma_store_2d(&tmY, stg + p * kBM * 128, n0 + p * 64, m_base);
+        for (int p = 0; p < BN / 64; ++p)          // rows past the sequence's end are dropped by the tensor map
+          tma_store_3d(&tmY, stg + p * kBM * 128, n0 + p * 64, (sub % tps) * kBM, sub / tps);
         tma_store_commit();
       }
     }
@@ -218,22 +221,23 @@ int sm_count() {
 template <int BN, int MT>
 int run_tc(const ag_layer_desc &dsc, const void *O, const void *Wo, const void *X_res, void *Y, cudaStream_t st) {
   using Cfg = OpCfg<BN, MT>;
-  const int M = dsc.batch * dsc.seq, d = dsc.hidden, Kdim = dsc.heads * kD;
+  const int d = dsc.hidden, Kdim = dsc.heads * kD;
+  const int tps = (dsc.seq + kBM - 1) / kBM, n_sub = dsc.batch * tps;   // sub-tiles of 128 tokens per sequence, in all
   CUtensorMap tmO, tmW, tmY;
   int rc = make_tmap_3d_bf16(&tmO, O, (uint64_t)dsc.batch * dsc.heads, dsc.seq, kD, kBM, kBK);
   if (rc) return rc;
   rc = make_tmap_2d_bf16(&tmW, Wo, Kdim, d, (uint64_t)d * 2, kBK, 64);
   if (rc) return rc;
-  rc = make_tmap_2d_bf16(&tmY, Y, M, d, (uint64_t)d * 2, kBM, 64);
+  rc = make_tmap_3d_bf16(&tmY, Y, dsc.batch, dsc.seq, d, kBM, 64);
   if (rc) return rc;
   auto kern = out_proj_tc_kernel<BN, MT>;
   AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-  const int n_tiles_n = d / BN, n_tiles_m = (M + MT * kBM - 1) / (MT * kBM), n_tiles = n_tiles_n * n_tiles_m;
+  const int n_tiles_n = d / BN, n_tiles_m = (n_sub + MT - 1) / MT, n_tiles = n_tiles_n * n_tiles_m;
   const int tail = n_tiles % sm_count();
   const int split_from = (MT > 1 && tail > 0 && 2 * tail <= sm_count()) ? n_tiles - tail : n_tiles;
   const int ctas = split_from + 2 * (n_tiles - split_from);
-  kern<<<ctas, kThreads, Cfg::kSmemBytes, st>>>(tmO, tmW, tmY, static_cast<const __nv_bfloat16 *>(X_res), M, dsc.seq,
-                                                   dsc.heads, d, n_tiles_m, n_tiles_n, split_from);
+  kern<<<ctas, kThreads, Cfg::kSmemBytes, st>>>(tmO, tmW, tmY, static_cast<const __nv_bfloat16 *>(X_res), n_sub, tps,
+                                                   dsc.seq, dsc.heads, d, n_tiles_m, n_tiles_n, split_from);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
@@ -270,13 +274,13 @@ int run_simt(const ag_layer_desc &dsc, const void *O, const void *Wo, const void
 }  // namespace
 
 bool out_proj_tc_supported(const ag_layer_desc &d) {
-  return d.dtype == AG_BF16 && d.head_dim == kD && d.hidden % 128 == 0 && (d.seq % kBM == 0 || d.batch == 1) &&
-         (int64_t)d.batch * d.seq < ((int64_t)1 << 31);
+  return d.dtype == AG_BF16 && d.head_dim == kD && d.hidden % 128 == 0 &&
+         (int64_t)d.batch * (d.seq + kBM) < ((int64_t)1 << 31);
 }
 
 int launch_out_proj(const ag_layer_desc &d, const void *O, const void *Wo, const void *X_res, void *Y, cudaStream_t st) {
   if (out_proj_tc_supported(d)) {
-    const long long tiles128 = (long long)(d.hidden / 128) * ((d.batch * (long long)d.seq + kBM - 1) / kBM);
+    const long long tiles128 = (long long)(d.hidden / 128) * d.batch * ((d.seq + kBM - 1) / kBM);
     if (d.hidden % 256 == 0) {
       // more than one wave: 256-token tiles, whose two sub-tiles share every stage of W^O
       if (tiles128 > 2 * sm_count()) return run_tc<256, 2>(d, O, Wo, X_res, Y, st);

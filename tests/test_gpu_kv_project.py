@@ -127,6 +127,8 @@ CASES = {
     "one_sequence_ragged_end": LayerShape(1, 333, 256, 4, 128, 2, 128, "bf16"),      # n not a multiple of 16
     "one_sequence_short": LayerShape(1, 48, 128, 6, 128, 2, 128, "bf16"),            # less than one tile
     "one_sequence_long_ragged": LayerShape(1, 2500, 128, 16, 128, 2, 128, "bf16"),   # split last wave, ragged end
+    "batch_ragged_end": LayerShape(3, 200, 256, 4, 128, 2, 128, "bf16"),             # every sequence ends inside its last sub-tile
+    "batch_ragged_two_subtiles": LayerShape(5, 333, 128, 20, 128, 2, 128, "bf16"),   # 256-token tiles whose sub-tiles belong to two sequences, ragged ends
 }
 
 
@@ -136,7 +138,8 @@ def test_projection_and_cache(name):
 
 
 @pytest.mark.parametrize("name", ["two_heads_per_tile", "k_tail", "odd_heads", "subtiles_of_two_sequences",
-                                  "split_last_wave_odd_rows", "grouped_query", "one_sequence_ragged_end"])
+                                  "split_last_wave_odd_rows", "grouped_query", "one_sequence_ragged_end",
+                                  "batch_ragged_end", "batch_ragged_two_subtiles"])
 def test_projection_with_queries(name):
     """ag_qkv_project_cache: Q against the oracle's query projection, K, V and the cache as without it."""
     _check(CASES[name], 940, with_q=True)
@@ -238,8 +241,7 @@ def test_rejects_what_it_has_no_kernel_for():
     W = inputs.layer_weights(shape, 2, DEV)
     flags = torch.ones(shape.batch, shape.kvh, shape.seq, dtype=torch.uint8, device=DEV)
     cache, prefix, idx, status, K, V = gpu_project_cache(shape, X, W, flags)
-    for bad in (shape.with_(seq=200), shape.with_(head_dim=64),             # seq 200 with batch 2: sub-tiles would straddle sequences
-                shape.with_(dtype="f32"), shape.with_(hidden=516),
+    for bad in (shape.with_(head_dim=64), shape.with_(dtype="f32"), shape.with_(hidden=516),
                 shape.with_(recent_window=5)):              # the last one: a window, and a cache without a ring
         with pytest.raises(ag.AgError) as e:
             ag.ag_kv_project_cache(ag.make_desc(bad), X, W["Wk"], W["Wv"], flags, cache, prefix, idx, K, V, status)

@@ -4,7 +4,7 @@ MHA(X) = [H_1 .. H_h] W^O, with the skip connection of a stack of layers added i
 Every output element is compared with the oracle's float64 value: it may differ by one rounding
 to the layer dtype plus float32 summation error.  The shapes take every tile form of the
 tensor-core kernel (one or two 128-token sub-tiles per CTA, 256- and 128-column tiles, a split last
-wave, a single sequence that ends inside its last sub-tile, sub-tiles of two sequences in one tile)
+wave, sequences that end inside their last sub-tile, sub-tiles of two sequences in one tile)
 and the CUDA-core form (float32, head_dim 64, a width the tiles do not divide)."""
 import ctypes
 
@@ -46,7 +46,8 @@ SHAPES = {
     "cuda_cores_f32": inputs.TINY,
     "cuda_cores_bf16_d64": LayerShape(2, 150, 256, 4, 64, 2, 64, "bf16"),
     "cuda_cores_odd_width": LayerShape(2, 100, 200, 2, 128, 1, 128, "bf16"),
-    "cuda_cores_ragged_batch": LayerShape(3, 100, 256, 2, 128, 1, 128, "bf16"),       # n not a multiple of 128, batch > 1
+    "batch_ragged_end": LayerShape(3, 100, 256, 2, 128, 1, 128, "bf16"),              # every sequence ends inside its only sub-tile
+    "batch_ragged_two_subtiles": LayerShape(21, 200, 2048, 8, 128, 2, 128, "bf16"),   # two sub-tiles per CTA, ragged ends
 }
 
 

@@ -140,13 +140,51 @@ def test_window_argument_checks():
     with pytest.raises(ag.AgError) as e:                       # a window needs the cache's ring
         compact(ag.make_desc(base.with_(recent_window=5)), no_ring)
     assert e.value.status == ag.AG_ERR_INVALID_ARG
-    lens = torch.full((B,), n, dtype=torch.int32, device=DEV)
-    with pytest.raises(ag.AgError) as e:                       # not combined with per-sequence lengths
-        compact(ag.make_desc(base.with_(recent_window=5), seq_lens=lens), with_ring)
-    assert e.value.status == ag.AG_ERR_UNSUPPORTED
     q, kn, vn, _ = inputs.decode_inputs(base, 7820, 0, DEV)
     o = torch.empty_like(q)
     with pytest.raises(ag.AgError) as e:                       # the no-allocation entry does not read the ring
         ag.ag_decode_attn_noalloc(ag.make_desc(base.with_(recent_window=5)), q, kn, vn, with_ring, 0.0, o)
     assert e.value.status == ag.AG_ERR_UNSUPPORTED
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("w", [5, 10])
+def test_window_with_per_sequence_lengths(w):
+    """A ragged batch under a recent-token window: the ring of a sequence takes the last tokens of
+    its own prompt, and every valid row of prefill and of the decode steps equals what the sequence
+    alone gives (the oracle runs each sequence on its own, without padding)."""
+    shape = LayerShape(3, 300, 256, 4, 128, 2, 128, "bf16", recent_window=w)
+    B, h, n = shape.batch, shape.heads, shape.seq
+    lens = np.array([300, 7, 131], dtype=np.int32)              # full, shorter than the window, ragged
+    lens_dev = torch.from_numpy(lens).to(DEV)
+    Q, K, V = inputs.qkv_gaussian(shape, 7900 + w, DEV)
+    f = inputs.bernoulli_flags((B, h, n), 0.5, 7910 + w).numpy()
+    for b, L in enumerate(lens):
+        f[b, :, L:] = 0                                        # what the gate calls guarantee for padding
+    fl = torch.from_numpy(f).to(DEV)
+    desc = ag.make_desc(shape, lens_dev)
+    steps = w + 2
+    cache = ag.RaggedCache.allocate(shape, [n + steps] * (B * h), DEV)
+    prefix = torch.empty(B, h, n + 1, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ag.ag_compact_kv(desc, K, V, fl, cache, prefix, None, status, ag.workspace(desc, ag.AG_CALL_COMPACT))
+    O = torch.full_like(Q, float("nan"))
+    ag.ag_prefill_attn(desc, Q, K, V, fl, cache, prefix, 0.0, O, ag.workspace(desc, ag.AG_CALL_PREFILL))
+    torch.cuda.synchronize()
+    assert cache.pos.cpu().tolist() == np.repeat(lens, h).tolist()
+    Qf, Kf, Vf = T.f64(Q), T.f64(K), T.f64(V)
+    alone = []
+    for b, L in enumerate(lens):
+        ref = orc.prefill_attention(Qf[b:b + 1, :, :L], Kf[b:b + 1, :, :L], Vf[b:b + 1, :, :L], f[b:b + 1, :, :L], window=w)
+        T.check_close(T.f64(O)[b, :, :L], ref[0], "bf16", f"prefill of sequence {b}")
+        alone.append(orc.compact_kv(Kf[b:b + 1, :, :L], Vf[b:b + 1, :, :L], f[b:b + 1, :, :L], window=w))
+    ws = ag.workspace(desc, ag.AG_CALL_DECODE)
+    for step in range(steps):
+        q, kn, vn, fn = inputs.decode_inputs(shape, 7920 + w, step, DEV, keep_new=0.5)
+        o = torch.full_like(q, float("nan"))
+        ag.ag_decode_step(desc, q, kn, vn, fn, cache, 0.0, o, status, ws)
+        for b in range(B):
+            ref = orc.decode_attention(T.f64(q[b:b + 1]), T.f64(kn[b:b + 1]), T.f64(vn[b:b + 1]), alone[b])
+            T.check_close(T.f64(o[b:b + 1]), ref, "bf16", f"decode step {step}, sequence {b}")
+            orc.cache_append(alone[b], T.f64(kn[b:b + 1]), T.f64(vn[b:b + 1]), fn[b:b + 1].cpu().numpy(), window=w)
+    assert int(status.item()) == 0
