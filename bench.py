@@ -40,6 +40,8 @@ WORKLOADS = {
     "stack7b_prev": (inputs.STACK7B, 256, "the stack7b layers with eviction guided by the previous layer (ablation setting 4-1): "
                                          "layer l runs under the flags of layer l-1's gate, the first layer evicts nothing, "
                                          "each gate pass runs on a second stream beside its layer's attention"),
+    "prefill7b_out": (inputs.PREFILL7B, 16, "the prefill7b layer from hidden states to hidden states: gate, Q, K, V projection into the cache, "
+                                           "prefill attention, output projection with the skip connection (Eq. 1), 16 decode steps"),
     "stack7b_chain": (inputs.STACK7B, 256, "32 chained AG-gated layers, batch 8 x seq 4096: every layer projects its Q, K, V from the "
                                           "hidden states the previous layer produced, X_{l+1} = X_l + [H_1 .. H_h] W^O (no normalisation, "
                                           "no feed-forward block in between); per-layer mean eviction rising from 10% to 90%"),
@@ -178,8 +180,8 @@ class LayerRun:
         self.name = name
         self.use_graph = True
         self._groups = {}
-        self.has_gate = name in ("prefill7b", "prefill7b_proj", "tiny", "stack7b", "stack7b_prev", "stack7b_chain")
-        self.chain = name == "stack7b_chain"                        # layer l + 1 runs on layer l's output
+        self.has_gate = name in ("prefill7b", "prefill7b_proj", "prefill7b_out", "tiny", "stack7b", "stack7b_prev", "stack7b_chain")
+        self.chain = name in ("stack7b_chain", "prefill7b_out")     # layer l + 1 runs on layer l's output
         self.project = name == "prefill7b_proj" or self.chain       # Q, K, V are computed in the step
         self.layers = 32 if name.startswith("stack7b") else 1
         self.first_gated = 1 if name == "stack7b_prev" else 0      # 0: every layer evicts by its own gate
@@ -256,8 +258,8 @@ class LayerRun:
                 self.set_layer(l)
                 self.gamma = None
                 self.gate()
-                self.gammas.append(inputs.calibrate_gamma(self.scores, inputs.keep_targets_layer(h, seed + 20, l),
-                                                          sh.tau).to(dev))
+                keep = inputs.keep_targets_layer(h, seed + 20, l) if self.layers > 1 else inputs.keep_targets_uniform(h, seed + 20)
+                self.gammas.append(inputs.calibrate_gamma(self.scores, keep, sh.tau).to(dev))
                 self.gamma = self.gammas[l]
                 self.gate()
                 self.kv_project_cache()
@@ -691,7 +693,7 @@ def run_ours(args, rank, world, dev):
         dev_in = [run.Q, run.K, run.V, run.flags]
     else:
         dev_in = []
-    if not stack:
+    if not stack and not run.chain:
         dev_in += [t for q in run.dq for t in q]
     dev_out = ([run.O, run.flags] if run.has_prefill else []) + [run.o]
     host_in = [t.detach().cpu().pin_memory() for t in dev_in]
@@ -747,12 +749,17 @@ def run_ours(args, rank, world, dev):
                 host_out[1].copy_(run.flags, non_blocking=True)
             run.kv_project_cache()
             run.prefill()
+            if run.chain:
+                run.set_layer(0)
+                run.out_project()
             o_done = torch.cuda.Event(); o_done.record(main)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(o_done)
                 host_out[0].copy_(run.O, non_blocking=True)
             main.wait_event(ready[1]); run.decode_all()
             host_out[2].copy_(run.o, non_blocking=True)
+            if run.chain:
+                host_out[3].copy_(run.Xbuf[0], non_blocking=True)     # the layer's output hidden states
             main.wait_stream(s_out)
         elif overlap:
             s_in.wait_stream(main)

@@ -93,7 +93,8 @@ typedef struct {
                             outputs at padding positions are unspecified.  With a
                             recent-token window, ag_compact_kv and ag_kv_project_cache
                             read it too: the ring takes the last tokens of each
-                            sequence's own prompt.                                   */
+                            sequence's own prompt.  ag_prefill_attn skips the query
+                            tiles that hold padding only.                            */
   int32_t kv_heads;      /* 0 (= heads), or the number of key/value heads of grouped-query
                             attention: heads must be a multiple; query head i reads
                             key/value head i / (heads / kv_heads).  K, V, k_new, v_new,

@@ -34,7 +34,8 @@ struct SimtAttnArgs {
   const int32_t *prefix;               // [problems, n + 1]
   const int32_t *len;                  // [problems] valid rows of each slab: a row bound never exceeds it
   float *lse;                          // NULL, or [problems, n]: m + log2(l) of every row
-  // kGateFull only: [batch] keys each sequence has (the rest is padding), or NULL = n
+  // [batch] tokens each sequence has (the rest is padding), or NULL = n: the keys of kGateFull, and
+  // the query tiles kPrefill has to compute
   const int32_t *seq_lens;
 };
 
@@ -82,6 +83,8 @@ simt_attn_kernel(const SimtAttnArgs a) {
   // full: its queries then see themselves only, and no read leaves the slab
   const int slab_len = MODE == kPrefill ? a.len[prob_kv] : 0;
   const int n_keys = (MODE == kGateFull && a.seq_lens) ? a.seq_lens[prob / a.inner] : a.n;
+  // prefill: a query tile past its sequence's end holds padding only (outputs unspecified): nothing to do
+  if (MODE == kPrefill && a.seq_lens && j0 >= a.seq_lens[prob / a.inner]) return;
 
   // Q tile -> shared (rows past n are clamped; they are never stored)
   for (int x = tid; x < kSimtBM * kVecPerRow; x += kSimtThreads) {

@@ -134,6 +134,7 @@ static int run_prefill_simt(const ag_layer_desc &d, const void *Q, const void *K
   a.q_row = a.k_row = a.v_row = a.o_row = D;
   a.scale_log2 = scale * 1.4426950408889634f;
   a.k_rows = c.k_rows; a.v_rows = c.v_rows; a.row_off = c.row_off; a.prefix = prefix; a.len = c.len;
+  a.seq_lens = d.seq_lens;
   a.lse = lse;
   return launch_simt_attn<T, T, D, kPrefill>(a, d.batch * d.heads, st);
 }

@@ -49,6 +49,7 @@ struct PrefillTcArgs {
   int heads, kv_heads;              // query heads share key/value heads in groups of heads / kv_heads
   float scale_log2;
   float *lse;                       // NULL, or [slabs, n]: m + log2(l) of every row (see launch_prefill_tc)
+  const int32_t *seq_lens;          // NULL, or [batch]: a query tile that holds padding only is skipped
 };
 
 // Byte offset of 16-byte chunk `chunk` (0..15) of row `row` inside a [128 x 128] bf16 tile stored
@@ -91,6 +92,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   // heaviest query tiles first
   const int qt = a.n_qtiles - 1 - (int)(blockIdx.x / a.slabs);
   const int slab = blockIdx.x % a.slabs;           // Q and O live here
+  // a query tile past its sequence's end holds padding only: its outputs are unspecified, nothing to do
+  if (a.seq_lens != nullptr && qt * kPfBM >= a.seq_lens[slab / a.heads]) return;
   // K, V, the flags' prefix counts and the cache belong to the key/value head (grouped-query attention)
   const int kv_slab = (slab / a.heads) * a.kv_heads + (slab % a.heads) / (a.heads / a.kv_heads);
   const int j0 = qt * kPfBM;
@@ -441,6 +444,7 @@ int launch_prefill_tc(const ag_layer_desc &d, const void *Q, const void *K, cons
   a.heads = d.heads; a.kv_heads = kv_heads_of(d);
   a.scale_log2 = scale * 1.4426950408889634f;
   a.lse = lse;
+  a.seq_lens = d.seq_lens;
   AG_CUDA_TRY(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes));
   prefill_tc_kernel<<<a.n_qtiles * slabs, kPfThreads, kPfSmemBytes, st>>>(tmQ, tmKd, tmVd, tmO, tmK, tmV, a);
   AG_LAUNCH_CHECK();

@@ -97,6 +97,12 @@ def test_ragged_batch_through_the_layer():
     cache, prefix, idx, status = T.gpu_compact(shape, K, V, fl, cap=[n + 1] * (B * h))
     T.check_compaction(shape, K, V, fl, cache, prefix, idx)
     O = T.gpu_prefill(shape, Q, K, V, fl, cache, prefix)
+    # the same call told the lengths (it then skips the query tiles that hold padding only): the valid rows are the same bits
+    desc_l = ag.make_desc(shape, torch.from_numpy(lens).to(DEV))
+    O_l = torch.full_like(Q, float("nan"))
+    ag.ag_prefill_attn(desc_l, Q, K, V, fl, cache, prefix, 0.0, O_l, ag.workspace(desc_l, ag.AG_CALL_PREFILL))
+    for b, L in enumerate(lens):
+        assert torch.equal(O_l[b, :, :L], O[b, :, :L])
     Qf, Kf, Vf = T.f64(Q), T.f64(K), T.f64(V)
     for b, L in enumerate(lens):
         alone = orc.prefill_attention(Qf[b:b + 1, :, :L], Kf[b:b + 1, :, :L], Vf[b:b + 1, :, :L], f[b:b + 1, :, :L])
