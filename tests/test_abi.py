@@ -107,7 +107,7 @@ def test_projection_calls_reject_on_the_host(lib):
     assert kv(ok, pre=None) == ag.AG_ERR_INVALID_ARG
     assert kv(ok, Wk=p + 2) == ag.AG_ERR_INVALID_ARG
     assert kv(ag.make_desc(inputs.TINY)) == ag.AG_ERR_UNSUPPORTED                                      # float32, head_dim 64
-    assert kv(ag.make_desc(inputs.LayerShape(2, 200, 512, 4, 128, 2, 128, "bf16"))) == ag.AG_ERR_UNSUPPORTED   # two sequences, n % 128 != 0
+    assert kv(ag.make_desc(inputs.LayerShape(2, 256, 516, 4, 128, 2, 128, "bf16"))) == ag.AG_ERR_UNSUPPORTED   # hidden not a multiple of 8
     assert kv(ag.make_desc(inputs.LayerShape(2, 256, 516, 4, 128, 2, 128, "bf16"))) == ag.AG_ERR_UNSUPPORTED   # rows of X not 16-byte multiples
     assert kv(ag.make_desc(inputs.LayerShape(2, 256, 512, 4, 128, 2, 128, "bf16", recent_window=5))) == ag.AG_ERR_INVALID_ARG  # no ring
     assert lib.ag_qkv_project_cache(byref(ok), p, None, p, p, p, byref(c), p, None, p, p, p, None, None) == ag.AG_ERR_INVALID_ARG
