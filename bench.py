@@ -52,12 +52,18 @@ WORKLOADS = {
 # captures summarised under profiles/ (None for workloads that were not captured).  To be reset to
 # None whenever the kernel changes after the capture.
 TRAFFIC = {
-    ("prefill7b", "prefill"): 154.86e6 + 18.50e6,        # prefill_tc_kernel
+    ("prefill7b", "prefill"): 155.20e6 + 17.45e6,        # prefill_tc_kernel
     ("prefill7b", "decode"): 41.22e6 + 0.003e6,          # decode_cluster_mma_kernel
     ("prefill7b", "compact"): 41.26e6 + 2.46e6,          # compact_kernel<256> (written rows still in L2 at kernel end)
     ("prefill7b", "kv_project_cache"): 179.50e6 + 82.40e6,   # kv_proj_cache_kernel<256, 2>
-    ("prefill7b_proj", "prefill"): 154.86e6 + 18.50e6,
+    ("prefill7b_proj", "prefill"): 155.20e6 + 17.45e6,
     ("prefill7b_proj", "decode"): 41.22e6 + 0.003e6,
+    ("prefill7b_proj", "project"): 246.71e6 + 121.11e6,  # kv_proj_cache_kernel<256, 2> with the query projection
+    ("prefill7b_out", "prefill"): 155.20e6 + 17.45e6,
+    ("prefill7b_out", "project"): 246.71e6 + 121.11e6,
+    ("prefill7b_out", "out_project"): 122.83e6 + 14.84e6,    # out_proj_tc_kernel<256, 2>
+    ("deep_layer", "prefill"): 364.64e6 + 106.70e6,      # prefill_tc_kernel
+    ("deep_layer", "compact"): 20.48e6 + 0.34e6,         # compact_kernel<256>
     ("decode_ragged", "decode"): 2.3530e9 + 7.1e6,       # decode_partial_kernel<bf16,128>
 }
 # kernels launched per call of the library
