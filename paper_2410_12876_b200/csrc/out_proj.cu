@@ -14,7 +14,8 @@
 // column slices of W^O while the band's rows of O stay in L2); the tiles of a last wave that would
 // fill at most half of the SMs go to two CTAs of one sub-tile each.
 //
-// out_proj_simt_kernel is the CUDA-core form for float32 layers, head_dim 64 and shapes the tiles
+// out_proj_pair_kernel is the same GEMM on CTA pairs (cta_group::2), used when there are many waves of
+// tiles.  out_proj_simt_kernel is the CUDA-core form for float32 layers, head_dim 64 and shapes the tiles
 // do not cover.
 #include "ag_common.cuh"
 #include "umma.cuh"
@@ -208,6 +209,181 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
   if (warp == 1) tmem_dealloc(tmem_acc, kTmemCols);
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same GEMM on CTA pairs (cta_group::2): two CTAs on neighbouring SMs compute a 512-token x
+// 256-column tile with shared MMAs of M = 256.  Each CTA holds two 128-token sub-tiles of A (its
+// own 256 tokens) and ONE HALF of every W^O stage (128 of the 256 columns); an MMA reads A from
+// both CTAs and half of B from each.  Per 64-deep k-block a CTA takes in 32 KB of A + 16 KB of B
+// for 8.4 MFLOP, against 32 + 32 KB for the single-CTA tile: the operand loads, which pace that
+// kernel, shrink by a quarter.  Loads are plain TMA loads (no multicast) that report to the
+// leader's barrier; the leader (even CTA) issues the MMAs; a commit frees a stage in both CTAs.
+constexpr int kPairBN = 256, kPairMT = 2, kPairStages = 4;
+constexpr int kPairABytes = kPairMT * kBM * kBK * 2;                 // 32 KB: this CTA's two sub-tiles
+constexpr int kPairBBytes = (kPairBN / 2 / 64) * (kBK * 64 * 2);     // 16 KB: this CTA's half of the W^O stage
+constexpr int kPairStageBytes = kPairABytes + kPairBBytes;           // 48 KB
+constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + 256;
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+out_proj_pair_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmW,
+                     const __grid_constant__ CUtensorMap tmY, const __nv_bfloat16 *__restrict__ X_res, int n_sub, int tps,
+                     int n, int heads, int d, int n_tiles_m, int n_tiles_n) {
+  constexpr int BN = kPairBN, MT = kPairMT;
+  constexpr uint32_t kTmemCols = MT * BN;          // 512: two accumulators of 128 rows x 256 columns per CTA
+  static_assert(MT * (BN / 64) * kBM * 128 <= kPairStages * kPairStageBytes, "staging fits the stages");
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + kPairStages * kPairStageBytes);   // used in the leader only
+  uint64_t *empty = full + kPairStages;            // one set per CTA: a commit arrives on both
+  uint64_t *acc_full = empty + kPairStages;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  int *gave_up = reinterpret_cast<int *>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();         // 0: leader
+  const int tile = blockIdx.x >> 1;
+  const int band = tile / (kBandTiles * n_tiles_n), in_band = tile % (kBandTiles * n_tiles_n);
+  const int band_rows = min(kBandTiles, n_tiles_m - band * kBandTiles);
+  const int tile_m = band * kBandTiles + in_band % band_rows, tile_n = in_band / band_rows;
+  const int sub0 = tile_m * (2 * MT) + (int)rank * MT;   // this CTA's first sub-tile of 128 tokens
+  const int n0 = tile_n * BN;
+  const int num_kb = heads * (kD / kBK);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPairStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    *gave_up = 0;
+    fence_barrier_init();
+    prefetch_tensormap(&tmO);
+    prefetch_tensormap(&tmW);
+    prefetch_tensormap(&tmY);
+  }
+  __syncthreads();
+  if (warp == 1) {                                 // the same warp of both CTAs, the same arguments
+    tmem_alloc_pair(tmem_slot, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  cluster_arrive_wait();                           // both CTAs' barriers are initialised, tensor memory is allocated
+  tc_fence_after_sync();
+  const uint32_t tmem_acc = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % kPairStages;
+        const uint32_t ph = (kb / kPairStages) & 1;
+        if (!mbar_wait(&empty[s], ph ^ 1)) break;  // this CTA's copy: the MMAs that read the stage (in both CTAs) are done
+        uint8_t *a = smem + s * kPairStageBytes, *b = a + kPairABytes;
+        // the leader's barrier counts the bytes of both CTAs
+        if (rank == 0) mbar_arrive_expect_tx(&full[s], 2 * kPairStageBytes);
+        const uint32_t bar = mapa_shared(smem_u32(&full[s]), 0);
+        const int head = kb / (kD / kBK), col = (kb % (kD / kBK)) * kBK;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          // tokens past the sequence's end, and whole sub-tiles past the batch, are filled with zeros
+          const int sub = sub0 + mt, b_seq = sub / tps, t0 = (sub % tps) * kBM;
+          tma_load_3d_pair(a + mt * (kBM * kBK * 2), &tmO, bar, col, t0, b_seq * heads + head);
+        }
+#pragma unroll
+        for (int p = 0; p < BN / 2 / 64; ++p)      // this CTA's half of the tile's columns
+          tma_load_2d_pair(b + p * (kBK * 64 * 2), &tmW, bar, n0 + (int)rank * (BN / 2) + p * 64, kb * kBK);
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0) {
+      // every lane runs the control flow (operands stay warp-uniform); one elected lane issues
+      const uint32_t idesc = idesc_bf16_f32(2 * kBM, BN, false, true);
+      const uint64_t da0 = desc_kmajor_sw128(smem_u32(smem));
+      const uint64_t db0 = desc_mnmajor_sw128(smem_u32(smem) + kPairABytes, kBK * 64 * 2);
+      const uint32_t a_lo0 = (uint32_t)da0, a_hi = (uint32_t)(da0 >> 32);
+      const uint32_t b_lo0 = (uint32_t)db0, b_hi = (uint32_t)(db0 >> 32);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb && ok; ++kb) {
+        const int s = kb % kPairStages;
+        const uint32_t ph = (kb / kPairStages) & 1;
+        ok = mbar_wait(&full[s], ph);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t a_lo = a_lo0 + ((s * kPairStageBytes) >> 4), b_lo = b_lo0 + ((s * kPairStageBytes) >> 4);
+        if (elect_one()) {
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+              mma_ss_pair_lohi(tmem_acc + mt * BN, a_lo + ((mt * kBM * kBK * 2 + k * 32) >> 4), a_hi,
+                               b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
+          }
+          mma_commit_pair(&empty[s]);              // frees the stage in both CTAs once these MMAs have read it
+        }
+        __syncwarp();
+      }
+      if (elect_one()) mma_commit_pair(acc_full);  // accumulators complete (or unwinding), in both CTAs
+      __syncwarp();
+    }
+  } else {
+    const int quad = warp & 3, half = (warp - 2) >> 2;
+    const int r_in = quad * 32 + lane;
+    constexpr int kChunks = BN / 2 / 32;
+    uint4 res[kChunks][4];
+    auto fetch_residual = [&](int mt) {
+      const int sub = sub0 + mt, t = (sub % tps) * kBM + r_in;
+      const bool have = X_res != nullptr && sub < n_sub && t < n;
+      const size_t row = (size_t)(sub / tps) * n + t;
+#pragma unroll
+      for (int ci = 0; ci < kChunks; ++ci) {
+        const int c = half * (BN / 2) + ci * 32;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          res[ci][q] = have ? ldg128_stream(X_res + row * d + n0 + c + q * 8) : make_uint4(0, 0, 0, 0);
+      }
+    };
+    fetch_residual(0);
+    if (!mbar_wait(acc_full, 0)) *gave_up = 1;
+    named_barrier_sync(1, 256);
+    const bool ok = *gave_up == 0;
+    tc_fence_after_sync();
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      const int sub = sub0 + mt;
+      if (!ok || sub >= n_sub) break;              // the same for all 256 threads
+      const uint32_t tmem_sub = tmem_acc + mt * BN;
+      uint8_t *stg = smem + mt * (BN / 64) * kBM * 128;
+#pragma unroll
+      for (int ci = 0; ci < kChunks; ++ci) {
+        const int c = half * (BN / 2) + ci * 32;
+        uint32_t r[32];
+        tmem_ld_x32_sync(tmem_sub + ((uint32_t)(quad * 32) << 16) + c, r);
+        const uint32_t panel = (uint32_t)(c >> 6) * kBM * 128 + r_in * 128;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          float xf[8];
+          Elem<__nv_bfloat16>::unpack(res[ci][q], xf);
+          uint32_t h[4];
+#pragma unroll
+          for (int e = 0; e < 8; e += 2)
+            h[e >> 1] = pack_bf16x2(__uint_as_float(r[q * 8 + e]) + xf[e], __uint_as_float(r[q * 8 + e + 1]) + xf[e + 1]);
+          const uint32_t chunk = (uint32_t)(((c & 32) >> 3) + q);
+          *reinterpret_cast<uint4 *>(stg + panel + ((chunk ^ (r_in & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
+        }
+      }
+      if (mt + 1 < MT) fetch_residual(mt + 1);
+      fence_proxy_async_smem();
+      named_barrier_sync(1, 256);
+      if (threadIdx.x == 64) {
+#pragma unroll
+        for (int p = 0; p < BN / 64; ++p)
+          tma_store_3d(&tmY, stg + p * kBM * 128, n0 + p * 64, (sub % tps) * kBM, sub / tps);
+        tma_store_commit();
+      }
+    }
+    if (threadIdx.x == 64) tma_store_wait_read();
+  }
+  // neither CTA leaves (or frees tensor memory) while the other may still use its shared or tensor memory
+  tc_fence_before_sync();
+  cluster_arrive_wait();
+  if (warp == 1) tmem_dealloc_pair(tmem_acc, kTmemCols);
+}
+
 int sm_count() {
   static int sms = 0;
   if (sms == 0) {
@@ -261,6 +437,24 @@ out_proj_simt_kernel(const T *__restrict__ O, const T *__restrict__ Wo, const T 
   Elem<T>::store(Y + (size_t)tok * d + c, acc);
 }
 
+int run_pair(const ag_layer_desc &dsc, const void *O, const void *Wo, const void *X_res, void *Y, cudaStream_t st) {
+  const int d = dsc.hidden, Kdim = dsc.heads * kD;
+  const int tps = (dsc.seq + kBM - 1) / kBM, n_sub = dsc.batch * tps;
+  CUtensorMap tmO, tmW, tmY;
+  int rc = make_tmap_3d_bf16(&tmO, O, (uint64_t)dsc.batch * dsc.heads, dsc.seq, kD, kBM, kBK);
+  if (rc) return rc;
+  rc = make_tmap_2d_bf16(&tmW, Wo, Kdim, d, (uint64_t)d * 2, kBK, 64);
+  if (rc) return rc;
+  rc = make_tmap_3d_bf16(&tmY, Y, dsc.batch, dsc.seq, d, kBM, 64);
+  if (rc) return rc;
+  AG_CUDA_TRY(cudaFuncSetAttribute(out_proj_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes));
+  const int n_tiles_n = d / kPairBN, n_tiles_m = (n_sub + 2 * kPairMT - 1) / (2 * kPairMT);
+  out_proj_pair_kernel<<<2 * n_tiles_n * n_tiles_m, kThreads, kPairSmemBytes, st>>>(
+      tmO, tmW, tmY, static_cast<const __nv_bfloat16 *>(X_res), n_sub, tps, dsc.seq, dsc.heads, d, n_tiles_m, n_tiles_n);
+  AG_LAUNCH_CHECK();
+  return AG_OK;
+}
+
 template <typename T>
 int run_simt(const ag_layer_desc &dsc, const void *O, const void *Wo, const void *X_res, void *Y, cudaStream_t st) {
   dim3 grid((dsc.hidden + 255) / 256, dsc.batch * dsc.seq);
@@ -282,6 +476,9 @@ int launch_out_proj(const ag_layer_desc &d, const void *O, const void *Wo, const
   if (out_proj_tc_supported(d)) {
     const long long tiles128 = (long long)(d.hidden / 128) * d.batch * ((d.seq + kBM - 1) / kBM);
     if (d.hidden % 256 == 0) {
+      // many waves: 512 x 256 tiles on CTA pairs, each CTA loading half of every W^O stage (a quarter less
+      // operand traffic from L2 at the same speed; on a few waves the single-CTA tiles are 1-2 % faster)
+      if (tiles128 >= 8 * sm_count()) return run_pair(d, O, Wo, X_res, Y, st);
       // more than one wave: 256-token tiles, whose two sub-tiles share every stage of W^O
       if (tiles128 > 2 * sm_count()) return run_tc<256, 2>(d, O, Wo, X_res, Y, st);
       return run_tc<256, 1>(d, O, Wo, X_res, Y, st);

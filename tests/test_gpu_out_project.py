@@ -90,6 +90,40 @@ def test_layer_output_at_the_7b_shape_on_sampled_tokens():
     assert ag.ag_device_wait_timeouts() == 0
 
 
+@pytest.mark.gpu
+def test_layer_output_at_batch_8_on_cta_pairs():
+    """Batch 8 x 4096 tokens (the stack's layer): many waves of tiles, which run on CTA pairs (two CTAs
+    share each MMA, each loading half of every W^O stage); the oracle evaluates sampled tokens of
+    every sequence."""
+    shape = inputs.STACK7B
+    B, h, n, D, d = shape.batch, shape.heads, shape.seq, shape.head_dim, shape.hidden
+    O = inputs.randn((B, h, n, D), 8201, DEV, shape.torch_dtype)
+    Wo = inputs.output_weight(shape, 8202, DEV)
+    X = inputs.hidden_states(shape, 8203, DEV)
+    Y = torch.full((B, n, d), float("nan"), dtype=shape.torch_dtype, device=DEV)
+    ag.ag_out_project(ag.make_desc(shape), O, Wo, X, Y)
+    torch.cuda.synchronize()
+    assert torch.isfinite(Y.float()).all()
+    toks = np.unique(np.concatenate([[0, 127, 128, 255, 256, 383, 384, 511, 512, n - 1],
+                                     np.random.default_rng(4).integers(0, n, size=30)]))
+    ti = torch.from_numpy(toks).to(DEV)
+    ref = orc.mha_output(T.f64(O[:, :, ti]), T.f64(Wo), T.f64(X[:, ti]))
+    _close_to_rounded(T.f64(Y[:, ti]), ref, "bf16", "batch-8 layer on CTA pairs")
+    # a ragged variant of the same size class: sequences that end inside a sub-tile, on the same path
+    shape2 = LayerShape(80, 200, 2048, 8, 128, 2, 128, "bf16")
+    O2 = inputs.randn((80, 8, 200, 128), 8211, DEV, torch.bfloat16)
+    Wo2 = inputs.randn((1024, 2048), 8212, DEV, torch.bfloat16, 0.05)
+    X2 = inputs.hidden_states(shape2, 8213, DEV)
+    Y2 = torch.full((80, 200, 2048), float("nan"), dtype=torch.bfloat16, device=DEV)
+    ag.ag_out_project(ag.make_desc(shape2), O2, Wo2, X2, Y2)
+    torch.cuda.synchronize()
+    bsel = torch.tensor([0, 1, 2, 3, 40, 79], device=DEV)
+    ref2 = orc.mha_output(T.f64(O2[bsel]), T.f64(Wo2), T.f64(X2[bsel]))
+    _close_to_rounded(T.f64(Y2[bsel]), ref2, "bf16", "ragged batch on CTA pairs")
+    assert torch.isfinite(Y2.float()).all()
+    assert ag.ag_device_wait_timeouts() == 0
+
+
 def test_argument_checks_on_the_host():
     lib = ag.lib()
     p = 4096
