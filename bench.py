@@ -251,6 +251,24 @@ class LayerRun:
         self.dqs = [[inputs.decode_inputs(sh, inputs.stack_layer_seed(seed, l) + 500 if self.layers > 1 else seed + 500,
                                           s, dev, keep_new=keep_new) for s in range(self.decode_steps)]
                     for l in range(self.layers)]
+        # the decode tokens of a layer live in ONE device buffer (the tensors above become views of it), so that
+        # the end-to-end pass sends them with one copy instead of four small ones per step
+        self.dq_flat = []
+        for l, dq in enumerate(self.dqs):
+            sizes = [t.numel() * t.element_size() for q in dq for t in q]
+            offs = np.concatenate([[0], np.cumsum([(x + 255) // 256 * 256 for x in sizes])])
+            flat = torch.empty(int(offs[-1]), dtype=torch.uint8, device=dev)
+            views, k = [], 0
+            for q in dq:
+                step = []
+                for t in q:
+                    v = flat[int(offs[k]):int(offs[k]) + sizes[k]].view(t.dtype).view(t.shape)
+                    v.copy_(t)
+                    step.append(v)
+                    k += 1
+                views.append(tuple(step))
+            self.dqs[l] = views
+            self.dq_flat.append(flat)
         self.dq = self.dqs[0]
         self.layer = 0
         self.graphs = {}
@@ -688,9 +706,9 @@ def run_ours(args, rank, world, dev):
     sh = run.shape
     stack = run.layers > 1 and run.has_gate
     if run.chain:
-        dev_in = [run.X0] + [u for dq in run.dqs for q in dq for u in q]
+        dev_in = [run.X0] + run.dq_flat
     elif stack:
-        dev_in = [t for (X, W, Q, K, V), dq in zip(run.layer_in, run.dqs) for t in [X, Q, K, V] + [u for q in dq for u in q]]
+        dev_in = [t for (X, W, Q, K, V), flat in zip(run.layer_in, run.dq_flat) for t in [X, Q, K, V, flat]]
     elif run.project:
         dev_in = [run.X]                                     # Q, K and V are made on the device
     elif run.has_gate:
@@ -700,7 +718,7 @@ def run_ours(args, rank, world, dev):
     else:
         dev_in = []
     if not stack and not run.chain:
-        dev_in += [t for q in run.dq for t in q]
+        dev_in += run.dq_flat
     dev_out = ([run.O, run.flags] if run.has_prefill else []) + [run.o]
     host_in = [t.detach().cpu().pin_memory() for t in dev_in]
     host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in dev_out]
@@ -770,10 +788,10 @@ def run_ours(args, rank, world, dev):
         elif overlap:
             s_in.wait_stream(main)
             s_out.wait_stream(main)
-            ready = []                                       # events: X, one per head group (its K, V, Q), decode inputs
+            ready = []                                       # events: X, decode inputs (small), one per head group (its K, V, Q)
             with torch.cuda.stream(s_in):
-                for group in ([(0, None)], *[[(2, g), (3, g), (1, g)] for g in groups],
-                              [(i, None) for i in range(4, 4 + n_dq)]):
+                for group in ([(0, None)], [(i, None) for i in range(4, 4 + n_dq)],
+                              *[[(2, g), (3, g), (1, g)] for g in groups]):
                     for i, g in group:
                         if g is None:
                             dev_in[i].copy_(host_in[i], non_blocking=True)
@@ -791,14 +809,14 @@ def run_ours(args, rank, world, dev):
             for gi, g in enumerate(groups):
                 # compaction and prefill attention of a head group as soon as its K, V, Q are in; its O
                 # goes back while the next groups are still coming in (the link carries both directions)
-                main.wait_event(ready[1 + gi])
+                main.wait_event(ready[2 + gi])
                 gg = g if n_groups > 1 else None
                 run.compact(gg); run.prefill(gg)
                 o_done = torch.cuda.Event(); o_done.record(main)
                 with torch.cuda.stream(s_out):
                     s_out.wait_event(o_done)
                     host_out[0][:, g[0]:g[1]].copy_(run.O[:, g[0]:g[1]], non_blocking=True)
-            main.wait_event(ready[-1]); run.decode_all()
+            main.wait_event(ready[1]); run.decode_all()
             host_out[2].copy_(run.o, non_blocking=True)
             main.wait_stream(s_out)
         else:
