@@ -88,6 +88,11 @@ __device__ inline GaPiece ga_piece(const GateAttnArgs &a, int x, int x_end) {
   p.n_kv = min(x_end, tile_end) - x;
   return p;
 }
+// A piece whose query tile lies wholly in its sequence's padding: nothing to compute (every role
+// skips it the same way; the softmax role leaves an empty partial for the merge).
+__device__ inline bool ga_padding_only(const GateAttnArgs &a, const GaPiece &p) {
+  return a.seq_lens != nullptr && p.qt * kGaBM >= a.seq_lens[p.prob / a.gate_heads];
+}
 // Segment that holds global step x.
 __device__ inline int ga_segment_of(const GateAttnArgs &a, int x) {
   int lo = 0, hi = a.n_seg - 1;
@@ -154,8 +159,9 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
     if (lane == 0) {
       bool ok = true;
       int t = 0;
-      for (int x = x_begin, pc = 0; x < x_end && ok; ++pc) {
+      for (int x = x_begin, pc = 0; x < x_end && ok; ++pc) {      // pc counts the pieces that are computed
         const GaPiece pz = ga_piece(a, x, x_end);
+        if (ga_padding_only(a, pz)) { x += pz.n_kv; --pc; continue; }
         const int b = pz.prob / a.gate_heads, g = pz.prob % a.gate_heads, j0 = pz.qt * kGaBM;
         const int xq = g * kGaD, xk = a.GD + g * kGaD, xv = 2 * a.GD + g * kGaD;   // columns in [Q' | K' | V']
         ok = mbar_wait(q_empty, (pc & 1) ^ 1);       // the previous piece's last Q K^T has read Q
@@ -218,8 +224,10 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
     };
     bool ok = true;
     int t0 = 0;                                      // tile number of the piece's first tile
-    for (int x = x_begin, pc = 0; x < x_end && ok; ++pc) {
-      const int n_kv = ga_piece(a, x, x_end).n_kv;
+    for (int x = x_begin, pc = 0; x < x_end && ok; ++pc) {        // pc counts the pieces that are computed
+      const GaPiece pz = ga_piece(a, x, x_end);
+      const int n_kv = pz.n_kv;
+      if (ga_padding_only(a, pz)) { x += n_kv; --pc; continue; }
       ok = mbar_wait(q_full, pc & 1);
       ok = ok && issue_qk(t0, n_kv == 1);
       for (int i = 0; i < n_kv && ok; ++i) {
@@ -267,6 +275,18 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
     const int seq_len = a.seq_lens ? a.seq_lens[pz.prob / a.gate_heads] : a.n;
     const int bound = a.causal ? jc + 1 : seq_len;
     float m = -INFINITY, l = 0.f;
+    if (ga_padding_only(a, pz)) {
+      // padding only: an empty partial (weight 0 in the merge; the merge gives padding flag 0 anyway)
+      const size_t it = (size_t)ga_slot(pz.prob, pz.qt, a.n_qtiles, (int)blockIdx.x);
+      if (valid) {
+        float *op = a.part_o + (it * kGaBM + row) * kGaD;
+#pragma unroll 4
+        for (int e = 0; e < kGaD; e += 4) *reinterpret_cast<uint4 *>(op + e) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<float2 *>(a.part_ml + (it * kGaBM + row) * 2) = make_float2(m, l);
+      }
+      x += n_kv;
+      continue;
+    }
 
     for (int i = 0; i < n_kv && ok; ++i) {
       const int t = t0 + i;
