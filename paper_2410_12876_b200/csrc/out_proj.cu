@@ -8,15 +8,16 @@
 //
 // One CTA computes MT sub-tiles of 128 tokens x BN output columns.  Warp 0 drives TMA, warp 1 owns
 // tensor memory and issues the MMAs, warps 2..9 drain the accumulator (two per quarter of its
-// lanes): they fetch their rows of the skip connection into registers while the MMAs run, add them
-// to the float32 accumulator, round once to bf16, stage the tile over the freed operand stages and
-// send it off with TMA stores.  Tile order in bands of row tiles (the CTAs in flight share a few
-// column slices of W^O while the band's rows of O stay in L2); the tiles of a last wave that would
-// fill at most half of the SMs go to two CTAs of one sub-tile each.
+// lanes): they fetch their rows of the skip connection into registers while the MMAs run (slice by
+// slice, each released by the MMA warp, so that the fetch is neither one burst among the first
+// operand loads nor waited for at the end), add them to the float32 accumulator, round once to
+// bf16, stage the tile over the freed operand stages and send it off with TMA stores.  Tile order
+// in bands of row tiles (the CTAs in flight share a few column slices of W^O while the band's rows
+// of O stay in L2).
 //
-// out_proj_pair_kernel is the same GEMM on CTA pairs (cta_group::2), used when there are many waves of
-// tiles.  out_proj_simt_kernel is the CUDA-core form for float32 layers, head_dim 64 and shapes the tiles
-// do not cover.
+// out_proj_pair_kernel is the same GEMM on CTA pairs (cta_group::2), used when the tiles fill the
+// SMs more than once.  out_proj_simt_kernel is the CUDA-core form for float32 layers, head_dim 64
+// and shapes the tiles do not cover.
 #include "ag_common.cuh"
 #include "umma.cuh"
 
@@ -28,6 +29,10 @@ namespace {
 
 constexpr int kBM = 128, kBK = 64, kThreads = 320, kD = 128;   // warps: TMA, MMA, 8 x epilogue
 constexpr int kBandTiles = 16;
+// The skip connection is fetched by the epilogue warps in slices of 32 columns spread over the main loop: slice i
+// once the MMAs of k-block kMidKb + i * step are done.  Fetched as one burst (at the start, or when the
+// accumulator is complete) it competes with the operand loads or is waited for.
+constexpr int kMidKb = 4, kMaxSlices = 8;
 
 template <int BN, int MT> struct OpCfg {
   static constexpr int kStages = BN == 256 ? (MT == 2 ? 3 : 4) : 6;
@@ -42,7 +47,7 @@ template <int BN, int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmW,
                    const __grid_constant__ CUtensorMap tmY, const __nv_bfloat16 *__restrict__ X_res, int n_sub, int tps,
-                   int n, int heads, int d, int n_tiles_m, int n_tiles_n, int split_from) {
+                   int n, int heads, int d, int n_tiles_m, int n_tiles_n) {
   using Cfg = OpCfg<BN, MT>;
   constexpr uint32_t kTmemCols = MT * BN;
   static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "TMEM columns: a power of two");
@@ -52,28 +57,27 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
   uint64_t *full = reinterpret_cast<uint64_t *>(smem + Cfg::kStages * Cfg::kStageBytes);
   uint64_t *empty = full + Cfg::kStages;
   uint64_t *acc_full = empty + Cfg::kStages;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  uint64_t *sig = acc_full + 1;                   // kMaxSlices barriers that release the skip connection slice by slice
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sig + kMaxSlices);
   int *gave_up = reinterpret_cast<int *>(tmem_slot + 1);   // set by an epilogue thread whose wait for the accumulator expired
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // CTAs below split_from take whole tiles, the rest one sub-tile of a tile
-  const int cta = blockIdx.x;
-  const bool single = MT > 1 && cta >= split_from;
-  const int tile = single ? split_from + ((cta - split_from) >> 1) : cta;
-  const int mts = single ? 1 : MT;               // sub-tiles of this CTA
+  const int tile = blockIdx.x;
   const int band = tile / (kBandTiles * n_tiles_n), in_band = tile % (kBandTiles * n_tiles_n);
   const int band_rows = min(kBandTiles, n_tiles_m - band * kBandTiles);
   const int tile_m = band * kBandTiles + in_band % band_rows, tile_n = in_band / band_rows;
   // Rows are counted in sub-tiles of 128 tokens laid out per sequence: sequence b owns sub-tiles
   // [b tps, (b + 1) tps), the last of which may reach past the sequence's end (zeros on the way in,
   // dropped on the way out), so a sub-tile never spans two sequences.
-  const int sub0 = tile_m * MT + (single ? ((cta - split_from) & 1) : 0);
+  const int sub0 = tile_m * MT;
   const int n0 = tile_n * BN;
   const int num_kb = heads * (kD / kBK);         // K = h D, 64 at a time: two blocks per head
+  const int sig_step = max(0, (num_kb - kMidKb - 8) / kMaxSlices);   // slice i leaves after k-block kMidKb + i sig_step
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(acc_full, 1);
+    for (int i = 0; i < kMaxSlices; ++i) mbar_init(&sig[i], 1);
     *gave_up = 0;
     fence_barrier_init();
     prefetch_tensormap(&tmO);
@@ -96,15 +100,13 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
         const uint32_t ph = (kb / Cfg::kStages) & 1;
         if (!mbar_wait(&empty[s], ph ^ 1)) break;
         uint8_t *a = smem + s * Cfg::kStageBytes, *b = a + Cfg::kABytes;
-        mbar_arrive_expect_tx(&full[s], mts * (kBM * kBK * 2) + Cfg::kBBytes);
+        mbar_arrive_expect_tx(&full[s], Cfg::kStageBytes);
         const int head = kb / (kD / kBK), col = (kb % (kD / kBK)) * kBK;
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          if (mt < mts) {
-            // tokens past the sequence's end, and whole sub-tiles past the batch, are filled with zeros
-            const int sub = sub0 + mt, b_seq = sub / tps, t0 = (sub % tps) * kBM;
-            tma_load_3d(a + mt * (kBM * kBK * 2), &tmO, &full[s], col, t0, b_seq * heads + head);
-          }
+          // tokens past the sequence's end, and whole sub-tiles past the batch, are filled with zeros
+          const int sub = sub0 + mt, b_seq = sub / tps, t0 = (sub % tps) * kBM;
+          tma_load_3d(a + mt * (kBM * kBK * 2), &tmO, &full[s], col, t0, b_seq * heads + head);
         }
 #pragma unroll
         for (int p = 0; p < BN / 64; ++p)
@@ -119,6 +121,7 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
     const uint32_t a_lo0 = (uint32_t)da0, a_hi = (uint32_t)(da0 >> 32);
     const uint32_t b_lo0 = (uint32_t)db0, b_hi = (uint32_t)(db0 >> 32);
     bool ok = true;
+    int nsig = 0;
     for (int kb = 0; kb < num_kb && ok; ++kb) {
       const int s = kb % Cfg::kStages;
       const uint32_t ph = (kb / Cfg::kStages) & 1;
@@ -126,19 +129,26 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t a_lo = a_lo0 + ((s * Cfg::kStageBytes) >> 4), b_lo = b_lo0 + ((s * Cfg::kStageBytes) >> 4);
+      int upto = nsig;                     // slices of the skip connection released after this k-block
+      while (upto < kMaxSlices && kb >= min(num_kb - 1, kMidKb + upto * sig_step)) ++upto;
       if (elect_one()) {
 #pragma unroll
         for (int k = 0; k < kBK / 16; ++k) {
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt)
-            if (mt < mts) mma_ss_lohi(tmem_acc + mt * BN, a_lo + ((mt * kBM * kBK * 2 + k * 32) >> 4), a_hi,
+            mma_ss_lohi(tmem_acc + mt * BN, a_lo + ((mt * kBM * kBK * 2 + k * 32) >> 4), a_hi,
                         b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
         }
         mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
+        for (int i = nsig; i < upto; ++i) mma_commit(&sig[i]);
       }
+      nsig = upto;
       __syncwarp();
     }
-    if (elect_one()) mma_commit(acc_full);   // accumulator complete (or unwinding)
+    if (elect_one()) {
+      for (int i = nsig; i < kMaxSlices; ++i) mma_commit(&sig[i]);
+      mma_commit(acc_full);                  // accumulator complete (or unwinding)
+    }
     __syncwarp();
   } else {
     // epilogue warps: warp w may touch TMEM lanes [32 * (w % 4), +32); warps 2..5 drain the first
@@ -146,21 +156,27 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
     const int quad = warp & 3, half = (warp - 2) >> 2;
     const int r_in = quad * 32 + lane;           // token of the sub-tile this thread drains
     constexpr int kChunks = BN / 2 / 32;         // 32-column chunks per thread and sub-tile
-    // this thread's piece of the skip connection for the first sub-tile, fetched while the MMAs run
-    uint4 res[kChunks][4];
-    auto fetch_residual = [&](int mt) {
+    // this thread's pieces of the skip connection, fetched while the MMAs run
+    uint4 res[MT][kChunks][4];
+    auto fetch_residual = [&](int mt, int ci) {
       const int sub = sub0 + mt, t = (sub % tps) * kBM + r_in;
-      const bool have = X_res != nullptr && sub < n_sub && t < n && mt < mts;
+      const bool have = X_res != nullptr && sub < n_sub && t < n;
       const size_t row = (size_t)(sub / tps) * n + t;
+      const int c = half * (BN / 2) + ci * 32;
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        res[mt][ci][q] = have ? ldg128_stream(X_res + row * d + n0 + c + q * 8) : make_uint4(0, 0, 0, 0);
+    };
+    bool fetched = true;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
       for (int ci = 0; ci < kChunks; ++ci) {
-        const int c = half * (BN / 2) + ci * 32;
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-          res[ci][q] = have ? ldg128_stream(X_res + row * d + n0 + c + q * 8) : make_uint4(0, 0, 0, 0);
+        fetched = fetched && mbar_wait(&sig[mt * kChunks + ci], 0);
+        if (fetched) fetch_residual(mt, ci);
       }
-    };
-    fetch_residual(0);
+    }
+    if (!fetched) *gave_up = 1;
     // all eight warps agree on whether the accumulator arrived before any of them enters the barriers below
     if (!mbar_wait(acc_full, 0)) *gave_up = 1;
     named_barrier_sync(1, 256);
@@ -169,7 +185,7 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
       const int sub = sub0 + mt;
-      if (!ok || sub >= n_sub || mt >= mts) break;          // the same for all 256 threads
+      if (!ok || sub >= n_sub) break;              // the same for all 256 threads
       const uint32_t tmem_sub = tmem_acc + mt * BN;
       // bf16 tile as panels of [128 tokens][64 columns] (128-byte rows, 16-byte chunks XOR-swizzled by the
       // row); each sub-tile has a staging area of its own, so the second is drained while the first leaves
@@ -183,7 +199,7 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           float xf[8];
-          Elem<__nv_bfloat16>::unpack(res[ci][q], xf);
+          Elem<__nv_bfloat16>::unpack(res[mt][ci][q], xf);
           uint32_t h[4];
 #pragma unroll
           for (int e = 0; e < 8; e += 2)
@@ -192,7 +208,6 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
           *reinterpret_cast<uint4 *>(stg + panel + ((chunk ^ (r_in & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
         }
       }
-      if (mt + 1 < MT) fetch_residual(mt + 1);     // in flight while this sub-tile leaves
       fence_proxy_async_smem();
       named_barrier_sync(1, 256);                  // the tile is staged
       if (threadIdx.x == 64) {
@@ -235,7 +250,8 @@ out_proj_pair_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_const
   uint64_t *full = reinterpret_cast<uint64_t *>(smem + kPairStages * kPairStageBytes);   // used in the leader only
   uint64_t *empty = full + kPairStages;            // one set per CTA: a commit arrives on both
   uint64_t *acc_full = empty + kPairStages;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  uint64_t *sig = acc_full + 1;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sig + kMaxSlices);
   int *gave_up = reinterpret_cast<int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -247,10 +263,12 @@ out_proj_pair_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_const
   const int sub0 = tile_m * (2 * MT) + (int)rank * MT;   // this CTA's first sub-tile of 128 tokens
   const int n0 = tile_n * BN;
   const int num_kb = heads * (kD / kBK);
+  const int sig_step = max(0, (num_kb - kMidKb - 8) / kMaxSlices);   // slice i leaves after k-block kMidKb + i sig_step
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kPairStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(acc_full, 1);
+    for (int i = 0; i < kMaxSlices; ++i) mbar_init(&sig[i], 1);
     *gave_up = 0;
     fence_barrier_init();
     prefetch_tensormap(&tmO);
@@ -298,6 +316,7 @@ out_proj_pair_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_const
       const uint32_t a_lo0 = (uint32_t)da0, a_hi = (uint32_t)(da0 >> 32);
       const uint32_t b_lo0 = (uint32_t)db0, b_hi = (uint32_t)(db0 >> 32);
       bool ok = true;
+      int nsig = 0;
       for (int kb = 0; kb < num_kb && ok; ++kb) {
         const int s = kb % kPairStages;
         const uint32_t ph = (kb / kPairStages) & 1;
@@ -305,6 +324,8 @@ out_proj_pair_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_const
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t a_lo = a_lo0 + ((s * kPairStageBytes) >> 4), b_lo = b_lo0 + ((s * kPairStageBytes) >> 4);
+        int upto = nsig;
+        while (upto < kMaxSlices && kb >= min(num_kb - 1, kMidKb + upto * sig_step)) ++upto;
         if (elect_one()) {
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k) {
@@ -314,30 +335,41 @@ out_proj_pair_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_const
                                b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
           }
           mma_commit_pair(&empty[s]);              // frees the stage in both CTAs once these MMAs have read it
+          for (int i = nsig; i < upto; ++i) mma_commit_pair(&sig[i]);
         }
+        nsig = upto;
         __syncwarp();
       }
-      if (elect_one()) mma_commit_pair(acc_full);  // accumulators complete (or unwinding), in both CTAs
+      if (elect_one()) {
+        for (int i = nsig; i < kMaxSlices; ++i) mma_commit_pair(&sig[i]);
+        mma_commit_pair(acc_full);               // accumulators complete (or unwinding), in both CTAs
+      }
       __syncwarp();
     }
   } else {
     const int quad = warp & 3, half = (warp - 2) >> 2;
     const int r_in = quad * 32 + lane;
     constexpr int kChunks = BN / 2 / 32;
-    uint4 res[kChunks][4];
-    auto fetch_residual = [&](int mt) {
+    uint4 res[MT][kChunks][4];
+    auto fetch_residual = [&](int mt, int ci) {
       const int sub = sub0 + mt, t = (sub % tps) * kBM + r_in;
       const bool have = X_res != nullptr && sub < n_sub && t < n;
       const size_t row = (size_t)(sub / tps) * n + t;
+      const int c = half * (BN / 2) + ci * 32;
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        res[mt][ci][q] = have ? ldg128_stream(X_res + row * d + n0 + c + q * 8) : make_uint4(0, 0, 0, 0);
+    };
+    bool fetched = true;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
       for (int ci = 0; ci < kChunks; ++ci) {
-        const int c = half * (BN / 2) + ci * 32;
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-          res[ci][q] = have ? ldg128_stream(X_res + row * d + n0 + c + q * 8) : make_uint4(0, 0, 0, 0);
+        fetched = fetched && mbar_wait(&sig[mt * kChunks + ci], 0);
+        if (fetched) fetch_residual(mt, ci);
       }
-    };
-    fetch_residual(0);
+    }
+    if (!fetched) *gave_up = 1;
     if (!mbar_wait(acc_full, 0)) *gave_up = 1;
     named_barrier_sync(1, 256);
     const bool ok = *gave_up == 0;
@@ -357,7 +389,7 @@ out_proj_pair_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_const
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           float xf[8];
-          Elem<__nv_bfloat16>::unpack(res[ci][q], xf);
+          Elem<__nv_bfloat16>::unpack(res[mt][ci][q], xf);
           uint32_t h[4];
 #pragma unroll
           for (int e = 0; e < 8; e += 2)
@@ -366,7 +398,6 @@ out_proj_pair_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_const
           *reinterpret_cast<uint4 *>(stg + panel + ((chunk ^ (r_in & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
         }
       }
-      if (mt + 1 < MT) fetch_residual(mt + 1);
       fence_proxy_async_smem();
       named_barrier_sync(1, 256);
       if (threadIdx.x == 64) {
@@ -409,11 +440,8 @@ int run_tc(const ag_layer_desc &dsc, const void *O, const void *Wo, const void *
   auto kern = out_proj_tc_kernel<BN, MT>;
   AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
   const int n_tiles_n = d / BN, n_tiles_m = (n_sub + MT - 1) / MT, n_tiles = n_tiles_n * n_tiles_m;
-  const int tail = n_tiles % sm_count();
-  const int split_from = (MT > 1 && tail > 0 && 2 * tail <= sm_count()) ? n_tiles - tail : n_tiles;
-  const int ctas = split_from + 2 * (n_tiles - split_from);
-  kern<<<ctas, kThreads, Cfg::kSmemBytes, st>>>(tmO, tmW, tmY, static_cast<const __nv_bfloat16 *>(X_res), n_sub, tps,
-                                                   dsc.seq, dsc.heads, d, n_tiles_m, n_tiles_n, split_from);
+  kern<<<n_tiles, kThreads, Cfg::kSmemBytes, st>>>(tmO, tmW, tmY, static_cast<const __nv_bfloat16 *>(X_res), n_sub, tps,
+                                                   dsc.seq, dsc.heads, d, n_tiles_m, n_tiles_n);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
@@ -476,11 +504,10 @@ int launch_out_proj(const ag_layer_desc &d, const void *O, const void *Wo, const
   if (out_proj_tc_supported(d)) {
     const long long tiles128 = (long long)(d.hidden / 128) * d.batch * ((d.seq + kBM - 1) / kBM);
     if (d.hidden % 256 == 0) {
-      // many waves: 512 x 256 tiles on CTA pairs, each CTA loading half of every W^O stage (a quarter less
-      // operand traffic from L2 at the same speed; on a few waves the single-CTA tiles are 1-2 % faster)
-      if (tiles128 >= 8 * sm_count()) return run_pair(d, O, Wo, X_res, Y, st);
-      // more than one wave: 256-token tiles, whose two sub-tiles share every stage of W^O
-      if (tiles128 > 2 * sm_count()) return run_tc<256, 2>(d, O, Wo, X_res, Y, st);
+      // more than one wave of 128 x 256 tiles: 512 x 256 tiles on CTA pairs, each CTA loading half of every W^O
+      // stage, which keeps the tensor pipe fed from shared memory (a single CTA on a 256 x 256 tile reads 12 KB of
+      // operands per MMA while TMA writes the next stage, more than shared memory's 128 B a clock)
+      if (tiles128 > 2 * sm_count()) return run_pair(d, O, Wo, X_res, Y, st);
       return run_tc<256, 1>(d, O, Wo, X_res, Y, st);
     }
     return run_tc<128, 1>(d, O, Wo, X_res, Y, st);
