@@ -55,13 +55,13 @@ TRAFFIC = {
     ("prefill7b", "prefill"): 155.20e6 + 17.45e6,        # prefill_tc_kernel
     ("prefill7b", "decode"): 41.22e6 + 0.003e6,          # decode_cluster_mma_kernel
     ("prefill7b", "compact"): 41.26e6 + 2.46e6,          # compact_kernel<256> (written rows still in L2 at kernel end)
-    ("prefill7b", "kv_project_cache"): 179.50e6 + 82.40e6,   # kv_proj_cache_kernel<256, 2>
+    ("prefill7b", "kv_project_cache"): 182.23e6 + 82.20e6,   # kv_proj_cache_pair_kernel
     ("prefill7b_proj", "prefill"): 155.20e6 + 17.45e6,
     ("prefill7b_proj", "decode"): 41.22e6 + 0.003e6,
-    ("prefill7b_proj", "project"): 246.71e6 + 121.11e6,  # kv_proj_cache_kernel<256, 2> with the query projection
+    ("prefill7b_proj", "project"): 251.70e6 + 121.58e6,  # kv_proj_cache_pair_kernel with the query projection
     ("prefill7b_out", "prefill"): 155.20e6 + 17.45e6,
-    ("prefill7b_out", "project"): 246.71e6 + 121.11e6,
-    ("prefill7b_out", "out_project"): 122.83e6 + 14.84e6,    # out_proj_tc_kernel<256, 2>
+    ("prefill7b_out", "project"): 251.70e6 + 121.58e6,
+    ("prefill7b_out", "out_project"): 132.63e6 + 16.75e6,    # out_proj_pair_kernel
     ("deep_layer", "prefill"): 364.64e6 + 106.70e6,      # prefill_tc_kernel
     ("deep_layer", "compact"): 20.48e6 + 0.34e6,         # compact_kernel<256>
     ("decode_ragged", "decode"): 2.3530e9 + 7.1e6,       # decode_partial_kernel<bf16,128>

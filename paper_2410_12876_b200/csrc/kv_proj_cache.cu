@@ -8,9 +8,8 @@
 // from the flags by the epilogue warps while the MMAs run.
 //
 // One CTA computes MT sub-tiles of 128 tokens x BN columns of the packed output [K | V]; a tile
-// lies in one weight and covers BN / 128 whole heads.  With MT = 2 the tiles of a last wave that
-// would fill at most half of the SMs go to two CTAs of one sub-tile each, so that the wave ends
-// in half the time.  Warp 0 drives TMA, warp 1 owns tensor
+// lies in one weight and covers BN / 128 whole heads.  Shapes whose tiles fill the SMs more than
+// once run on CTA pairs (kv_proj_cache_pair_kernel).  Warp 0 drives TMA, warp 1 owns tensor
 // memory and issues the MMAs, warps 2..9 drain the accumulator (two per quarter of its lanes).  Main loop as in the gate's
 // projection GEMM (A = X K-major, B = W MN-major panels of [64 k][64 n], 128-byte swizzle).
 // Epilogue per sub-tile: the destination rows of its tokens are computed while the MMAs run;
@@ -43,6 +42,161 @@ template <int BN, int MT> struct KvCfg {
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + kDstBytes + 64 /*counts*/;
 };
 
+// What the epilogue warps need besides the accumulator.
+struct KvEpilogue {
+  const CUtensorMap *tmK, *tmV, *tmQ;
+  const uint8_t *flags;
+  int32_t *prefix, *idx;
+  const int64_t *row_off;
+  const int32_t *cap;
+  int32_t *len;
+  uint8_t *k_rows, *v_rows;
+  int32_t *dev_status;
+  int n_sub, tps, n, kv_heads, heads;
+};
+
+// Warps 2..9 of a CTA: rank the tile's tokens while the MMAs run, then drain the CTA's mts sub-tiles
+// (first sub-tile sub0, columns [nw, nw + BN) of weight `which`) from tensor memory at tmem_acc.
+template <int BN, int MT>
+__device__ __forceinline__ void kv_epilogue(const KvEpilogue &e, uint8_t *smem, long long *dst_row, int *red, int *gave_up,
+                                            uint64_t *acc_full, uint32_t tmem_acc, int sub0, int mts, int which, int nw,
+                                            int num_kb, int warp, int lane) {
+  constexpr int kHeads = BN / kD;
+  const uint8_t *flags = e.flags;
+  int32_t *prefix = e.prefix, *idx = e.idx, *len = e.len, *dev_status = e.dev_status;
+  const int64_t *row_off = e.row_off;
+  const int32_t *cap = e.cap;
+  const int n_sub = e.n_sub, tps = e.tps, n = e.n, kv_heads = e.kv_heads;
+  const int out_heads = which == 2 ? e.heads : e.kv_heads;
+  // epilogue warps: warp w may touch TMEM lanes [32 * (w % 4), +32); warps 2..5 drain the first
+  // half of a sub-tile's columns, warps 6..9 the second
+  const int quad = warp & 3, half = (warp - 2) >> 2;
+  const int r_in = quad * 32 + lane;           // token of the sub-tile this thread drains
+  // While the MMAs run: the rank of every token of the tile among the retained tokens of its slab
+  // (the slab's flag row is a few KB: counted whole, as 16-byte vectors, for the number retained
+  // before the tile and in the slab; the tile's own tokens ranked by warp ballot + popc), hence its
+  // row in the ragged cache (-1: evicted, or the slab is too small).  The key tiles also write
+  // prefix (and idx), and the one that holds a sequence's first token the slab's length.
+#pragma unroll
+  for (int mt = 0; mt < (half == 0 ? MT : 0); ++mt) {           // warps 2..5 only
+    const int sub = sub0 + mt;
+    const int b = sub / tps, t0 = (sub % tps) * kBM, t = t0 + r_in;
+#pragma unroll
+    for (int hh = 0; hh < kHeads; ++hh) {
+      long long d = -1;
+      if (sub < n_sub && mt < mts && which != 2) {                // the same for all 128 threads
+        const size_t slab = (size_t)b * kv_heads + nw / kD + hh;
+        const uint8_t *f = flags + slab * n;
+        int before = 0, total = 0;
+        if ((n & 15) == 0) {                                      // flag rows start on 16-byte boundaries
+          const uint4 *fv = reinterpret_cast<const uint4 *>(f);
+          for (int x = r_in; x < n / 16; x += kBM) {
+            const uint4 w = ldg128(fv + x);
+            const int c = nonzero_bytes(w.x) + nonzero_bytes(w.y) + nonzero_bytes(w.z) + nonzero_bytes(w.w);
+            total += c;
+            if (x * 16 < t0) before += c;                         // t0 is a multiple of 16: a vector lies on one side
+          }
+        } else {
+          for (int x = r_in; x < n; x += kBM) {
+            const int c = f[x] != 0;
+            total += c;
+            if (x < t0) before += c;
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          before += __shfl_xor_sync(0xffffffffu, before, o);
+          total += __shfl_xor_sync(0xffffffffu, total, o);
+        }
+        const bool in_seq = t < n;                                // a single sequence may end inside its last sub-tile
+        const bool keep = in_seq && f[t] != 0;
+        const unsigned word = __ballot_sync(0xffffffffu, keep);
+        const int in_warp = __popc(word & ((1u << lane) - 1u));
+        if (lane == 0) { red[quad] = before; red[4 + quad] = total; red[8 + quad] = __popc(word); }
+        named_barrier_sync(2, 128);
+        before = red[0] + red[1] + red[2] + red[3];
+        total = red[4] + red[5] + red[6] + red[7];
+        int excl = 0;
+#pragma unroll
+        for (int q = 0; q < 3; ++q) excl += q < quad ? red[8 + q] : 0;
+        named_barrier_sync(2, 128);                             // red is free for the next head
+        const int p = before + excl + in_warp;                  // rank within the slab
+        const bool fits = total <= cap[slab];
+        if (fits && keep) d = row_off[slab] + p;
+        if (which == 0 && in_seq) {
+          int32_t *pre = prefix + slab * (n + 1);
+          pre[t] = p;
+          if (keep && idx) idx[slab * n + p] = t;
+          if (t == 0) {
+            pre[n] = total;
+            len[slab] = fits ? total : 0;
+            if (!fits && dev_status) atomicOr(dev_status, AG_DEV_OVERFLOW);
+          }
+        }
+      }
+      dst_row[(mt * kHeads + hh) * kBM + r_in] = d;
+    }
+  }
+  // the eight warps start this wait at different times (warps 2..5 rank the tile's tokens first): if it
+  // expires for some of them only, all of them must still agree to leave, or the barriers below would
+  // wait for threads that have gone
+  if (!mbar_wait(acc_full, 0)) *gave_up = 1;
+  named_barrier_sync(1, 256);
+  const bool ok = *gave_up == 0;
+  tc_fence_after_sync();
+  const CUtensorMap *tmOut = which == 0 ? e.tmK : (which == 1 ? e.tmV : e.tmQ);
+  uint8_t *rows_out = which == 0 ? e.k_rows : e.v_rows;
+  const int hw = (warp - 2) * 2 + (lane >> 4), l16 = lane & 15;   // half-warp 0..15, 16-byte piece of a row
+#pragma unroll 1
+  for (int mt = 0; mt < MT; ++mt) {
+    const int sub = sub0 + mt;
+    if (!ok || num_kb == 0 || sub >= n_sub || mt >= mts) break;
+    const uint32_t tmem_sub = tmem_acc + mt * BN;
+    // bf16 tile as panels of [128 tokens][64 columns] (128-byte rows, 16-byte chunks XOR-swizzled by the
+    // row); each sub-tile has a staging area of its own, so the second is drained while the first leaves
+    uint8_t *stg = smem + mt * (BN / 64) * kBM * 128;
+#pragma unroll 1
+    for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
+      uint32_t r[32];
+      tmem_ld_x32_sync(tmem_sub + ((uint32_t)(quad * 32) << 16) + c, r);
+      const uint32_t panel = (uint32_t)(c >> 6) * kBM * 128 + r_in * 128;
+#pragma unroll
+      for (int e = 0; e < 32; e += 8) {
+        uint32_t h[4];
+#pragma unroll
+        for (int q = 0; q < 8; q += 2)
+          h[q >> 1] = pack_bf16x2(__uint_as_float(r[e + q]), __uint_as_float(r[e + q + 1]));
+        const uint32_t chunk = (uint32_t)(((c & 32) >> 3) + (e >> 3));
+        *reinterpret_cast<uint4 *>(stg + panel + ((chunk ^ (r_in & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
+      }
+    }
+    fence_proxy_async_smem();
+    named_barrier_sync(1, 256);                  // the tile is staged (and dst_row written, first time round)
+    const int b = sub / tps, t0 = (sub % tps) * kBM;
+    if (threadIdx.x == 64) {
+#pragma unroll
+      for (int p = 0; p < BN / 64; ++p)
+        tma_store_3d(tmOut, stg + p * kBM * 128, (p & 1) * 64, t0, b * out_heads + nw / kD + (p >> 1));
+      tma_store_commit();
+    }
+    // retained rows: half-warp per row, 16 bytes per lane
+#pragma unroll
+    for (int hh = 0; hh < (which != 2 ? kHeads : 0); ++hh) {
+      const long long *dr = dst_row + (mt * kHeads + hh) * kBM;
+#pragma unroll 4
+      for (int r = hw; r < kBM; r += 16) {
+        const long long d = dr[r];
+        if (d >= 0) {
+          const uint32_t off = (uint32_t)(hh * 2 + (l16 >> 3)) * kBM * 128 + r * 128 + (((l16 & 7) ^ (r & 7)) << 4);
+          *reinterpret_cast<uint4 *>(rows_out + (size_t)d * (kD * 2) + l16 * 16) =
+              *reinterpret_cast<const uint4 *>(stg + off);
+        }
+      }
+    }
+  }
+  if (threadIdx.x == 64) tma_store_wait_read();
+}
+
 template <int BN, int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBk,
@@ -52,7 +206,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                      int32_t *__restrict__ prefix, int32_t *__restrict__ idx, const int64_t *__restrict__ row_off,
                      const int32_t *__restrict__ cap, int32_t *__restrict__ len, uint8_t *__restrict__ k_rows,
                      uint8_t *__restrict__ v_rows, int32_t *__restrict__ dev_status, int n_sub, int tps, int Kdim, int GD,
-                     int n, int kv_heads, int heads, int n_tiles_m, int n_tiles_n, int split_from) {
+                     int n, int kv_heads, int heads, int n_tiles_m, int n_tiles_n) {
   using Cfg = KvCfg<BN, MT>;
   constexpr uint32_t kTmemCols = MT * BN;
   static_assert(kTmemCols == 128 || kTmemCols == 256 || kTmemCols == 512, "TMEM columns: a power of two");
@@ -68,11 +222,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   int *gave_up = red + 12;                       // set by an epilogue thread whose wait for the accumulator expired
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // CTAs below split_from take whole tiles (row-major over the tile grid), the rest one sub-tile of a tile
-  const int cta = blockIdx.x;
-  const bool single = MT > 1 && cta >= split_from;
-  const int tile = single ? split_from + ((cta - split_from) >> 1) : cta;
-  const int mts = single ? 1 : MT;               // sub-tiles of this CTA
+  const int tile = blockIdx.x;
   // tile order: bands of kBandTiles row tiles; inside a band the row tile runs fastest, so the CTAs in
   // flight share a few column slices of W while the band's rows of X stay in L2
   const int band = tile / (kBandTiles * n_tiles_n), in_band = tile % (kBandTiles * n_tiles_n);
@@ -81,14 +231,13 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   // Rows are counted in sub-tiles of 128 tokens laid out per sequence: sequence b owns sub-tiles
   // [b tps, (b + 1) tps), the last of which may reach past the sequence's end (those rows are zeros on
   // the way in, take no rank, and are dropped by the stores), so a sub-tile never spans two sequences.
-  const int sub0 = tile_m * MT + (single ? ((cta - split_from) & 1) : 0);
+  const int sub0 = tile_m * MT;
   const int n0 = tile_n * BN;                    // in the packed output [K | V | Q] (GD, GD and heads * D columns)
   // BN divides the width of every weight: a tile lies in one weight.  which: 0 keys, 1 values, 2 queries
   // (queries go to their dense tensor only: no flags, no cache)
   const int which = n0 < GD ? 0 : (n0 < 2 * GD ? 1 : 2);
   const int nw = n0 - min(which, 2) * GD;
   const CUtensorMap *tmB = which == 0 ? &tmBk : (which == 1 ? &tmBv : &tmBq);
-  const int out_heads = which == 2 ? heads : kv_heads;
   const int num_kb = (Kdim + kBK - 1) / kBK;
 
   if (threadIdx.x == 0) {
@@ -115,11 +264,10 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const uint32_t ph = (kb / Cfg::kStages) & 1;
         if (!mbar_wait(&empty[s], ph ^ 1)) break;
         uint8_t *a = smem + s * Cfg::kStageBytes, *b = a + Cfg::kABytes;
-        mbar_arrive_expect_tx(&full[s], mts * (kBM * kBK * 2) + Cfg::kBBytes);
+        mbar_arrive_expect_tx(&full[s], Cfg::kStageBytes);
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)              // rows past the sequence (or past the batch) are filled with zeros
-          if (mt < mts)
-            tma_load_3d(a + mt * (kBM * kBK * 2), &tmA, &full[s], kb * kBK, ((sub0 + mt) % tps) * kBM, (sub0 + mt) / tps);
+          tma_load_3d(a + mt * (kBM * kBK * 2), &tmA, &full[s], kb * kBK, ((sub0 + mt) % tps) * kBM, (sub0 + mt) / tps);
 #pragma unroll
         for (int p = 0; p < BN / 64; ++p)
           tma_load_2d(b + p * Cfg::kPanelBytes, tmB, &full[s], nw + p * 64, kb * kBK);
@@ -145,7 +293,7 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         for (int k = 0; k < kBK / 16; ++k) {
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt)
-            if (mt < mts) mma_ss_lohi(tmem_acc + mt * BN, a_lo + ((mt * kBM * kBK * 2 + k * 32) >> 4), a_hi,
+            mma_ss_lohi(tmem_acc + mt * BN, a_lo + ((mt * kBM * kBK * 2 + k * 32) >> 4), a_hi,
                         b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
         }
         mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
@@ -155,137 +303,144 @@ kv_proj_cache_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     if (elect_one()) mma_commit(acc_full);   // accumulator complete (or unwinding)
     __syncwarp();
   } else {
-    // epilogue warps: warp w may touch TMEM lanes [32 * (w % 4), +32); warps 2..5 drain the first
-    // half of a sub-tile's columns, warps 6..9 the second
-    const int quad = warp & 3, half = (warp - 2) >> 2;
-    const int r_in = quad * 32 + lane;           // token of the sub-tile this thread drains
-    // While the MMAs run: the rank of every token of the tile among the retained tokens of its slab
-    // (the slab's flag row is a few KB: counted whole, as 16-byte vectors, for the number retained
-    // before the tile and in the slab; the tile's own tokens ranked by warp ballot + popc), hence its
-    // row in the ragged cache (-1: evicted, or the slab is too small).  The key tiles also write
-    // prefix (and idx), and the one that holds a sequence's first token the slab's length.
-#pragma unroll
-    for (int mt = 0; mt < (half == 0 ? MT : 0); ++mt) {           // warps 2..5 only
-      const int sub = sub0 + mt;
-      const int b = sub / tps, t0 = (sub % tps) * kBM, t = t0 + r_in;
-#pragma unroll
-      for (int hh = 0; hh < Cfg::kHeads; ++hh) {
-        long long d = -1;
-        if (sub < n_sub && mt < mts && which != 2) {                // the same for all 128 threads
-          const size_t slab = (size_t)b * kv_heads + nw / kD + hh;
-          const uint8_t *f = flags + slab * n;
-          int before = 0, total = 0;
-          if ((n & 15) == 0) {                                      // flag rows start on 16-byte boundaries
-            const uint4 *fv = reinterpret_cast<const uint4 *>(f);
-            for (int x = r_in; x < n / 16; x += kBM) {
-              const uint4 w = ldg128(fv + x);
-              const int c = nonzero_bytes(w.x) + nonzero_bytes(w.y) + nonzero_bytes(w.z) + nonzero_bytes(w.w);
-              total += c;
-              if (x * 16 < t0) before += c;                         // t0 is a multiple of 16: a vector lies on one side
-            }
-          } else {
-            for (int x = r_in; x < n; x += kBM) {
-              const int c = f[x] != 0;
-              total += c;
-              if (x < t0) before += c;
-            }
-          }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            before += __shfl_xor_sync(0xffffffffu, before, o);
-            total += __shfl_xor_sync(0xffffffffu, total, o);
-          }
-          const bool in_seq = t < n;                                // a single sequence may end inside its last sub-tile
-          const bool keep = in_seq && f[t] != 0;
-          const unsigned word = __ballot_sync(0xffffffffu, keep);
-          const int in_warp = __popc(word & ((1u << lane) - 1u));
-          if (lane == 0) { red[quad] = before; red[4 + quad] = total; red[8 + quad] = __popc(word); }
-          named_barrier_sync(2, 128);
-          before = red[0] + red[1] + red[2] + red[3];
-          total = red[4] + red[5] + red[6] + red[7];
-          int excl = 0;
-#pragma unroll
-          for (int q = 0; q < 3; ++q) excl += q < quad ? red[8 + q] : 0;
-          named_barrier_sync(2, 128);                             // red is free for the next head
-          const int p = before + excl + in_warp;                  // rank within the slab
-          const bool fits = total <= cap[slab];
-          if (fits && keep) d = row_off[slab] + p;
-          if (which == 0 && in_seq) {
-            int32_t *pre = prefix + slab * (n + 1);
-            pre[t] = p;
-            if (keep && idx) idx[slab * n + p] = t;
-            if (t == 0) {
-              pre[n] = total;
-              len[slab] = fits ? total : 0;
-              if (!fits && dev_status) atomicOr(dev_status, AG_DEV_OVERFLOW);
-            }
-          }
-        }
-        dst_row[(mt * Cfg::kHeads + hh) * kBM + r_in] = d;
-      }
-    }
-    // the eight warps start this wait at different times (warps 2..5 rank the tile's tokens first): if it
-    // expires for some of them only, all of them must still agree to leave, or the barriers below would
-    // wait for threads that have gone
-    if (!mbar_wait(acc_full, 0)) *gave_up = 1;
-    named_barrier_sync(1, 256);
-    const bool ok = *gave_up == 0;
-    tc_fence_after_sync();
-    const CUtensorMap *tmOut = which == 0 ? &tmK : (which == 1 ? &tmV : &tmQ);
-    uint8_t *rows_out = which == 0 ? k_rows : v_rows;
-    const int hw = (warp - 2) * 2 + (lane >> 4), l16 = lane & 15;   // half-warp 0..15, 16-byte piece of a row
-#pragma unroll 1
-    for (int mt = 0; mt < MT; ++mt) {
-      const int sub = sub0 + mt;
-      if (!ok || num_kb == 0 || sub >= n_sub || mt >= mts) break;
-      const uint32_t tmem_sub = tmem_acc + mt * BN;
-      // bf16 tile as panels of [128 tokens][64 columns] (128-byte rows, 16-byte chunks XOR-swizzled by the
-      // row); each sub-tile has a staging area of its own, so the second is drained while the first leaves
-      uint8_t *stg = smem + mt * (BN / 64) * kBM * 128;
-#pragma unroll 1
-      for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
-        uint32_t r[32];
-        tmem_ld_x32_sync(tmem_sub + ((uint32_t)(quad * 32) << 16) + c, r);
-        const uint32_t panel = (uint32_t)(c >> 6) * kBM * 128 + r_in * 128;
-#pragma unroll
-        for (int e = 0; e < 32; e += 8) {
-          uint32_t h[4];
-#pragma unroll
-          for (int q = 0; q < 8; q += 2)
-            h[q >> 1] = pack_bf16x2(__uint_as_float(r[e + q]), __uint_as_float(r[e + q + 1]));
-          const uint32_t chunk = (uint32_t)(((c & 32) >> 3) + (e >> 3));
-          *reinterpret_cast<uint4 *>(stg + panel + ((chunk ^ (r_in & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
-        }
-      }
-      fence_proxy_async_smem();
-      named_barrier_sync(1, 256);                  // the tile is staged (and dst_row written, first time round)
-      const int b = sub / tps, t0 = (sub % tps) * kBM;
-      if (threadIdx.x == 64) {
-#pragma unroll
-        for (int p = 0; p < BN / 64; ++p)
-          tma_store_3d(tmOut, stg + p * kBM * 128, (p & 1) * 64, t0, b * out_heads + nw / kD + (p >> 1));
-        tma_store_commit();
-      }
-      // retained rows: half-warp per row, 16 bytes per lane
-#pragma unroll
-      for (int hh = 0; hh < (which != 2 ? Cfg::kHeads : 0); ++hh) {
-        const long long *dr = dst_row + (mt * Cfg::kHeads + hh) * kBM;
-#pragma unroll 4
-        for (int r = hw; r < kBM; r += 16) {
-          const long long d = dr[r];
-          if (d >= 0) {
-            const uint32_t off = (uint32_t)(hh * 2 + (l16 >> 3)) * kBM * 128 + r * 128 + (((l16 & 7) ^ (r & 7)) << 4);
-            *reinterpret_cast<uint4 *>(rows_out + (size_t)d * (kD * 2) + l16 * 16) =
-                *reinterpret_cast<const uint4 *>(stg + off);
-          }
-        }
-      }
-    }
-    if (threadIdx.x == 64) tma_store_wait_read();
+    const KvEpilogue e{&tmK, &tmV, &tmQ, flags, prefix, idx, row_off, cap, len, k_rows, v_rows, dev_status, n_sub, tps, n, kv_heads, heads};
+    kv_epilogue<BN, MT>(e, smem, dst_row, red, gave_up, acc_full, tmem_acc, sub0, MT, which, nw, num_kb, warp, lane);
   }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_acc, kTmemCols);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same projection on CTA pairs (cta_group::2): a pair computes 512 tokens x 256 columns, each CTA
+// holding its own two sub-tiles of X and half of every stage of W, the leader issuing M = 256 MMAs
+// whose accumulators land in both CTAs' tensor memory.  A single CTA on a 256 x 256 tile reads 12 KB
+// of operands from shared memory per MMA while TMA writes the next stage, more than shared memory
+// moves in the MMA's 128 clocks; here it is 8 KB.  The pair tiles of a last wave that would fill at
+// most half of the SMs go to two pairs of 256 tokens each.
+constexpr int kPairBN = 256, kPairMT = 2, kPairStages = 4;
+constexpr int kPairABytes = kPairMT * kBM * kBK * 2;                 // 32 KB: this CTA's two sub-tiles of X
+constexpr int kPairBBytes = (kPairBN / 2 / 64) * (kBK * 64 * 2);     // 16 KB: this CTA's half of the stage of W
+constexpr int kPairBandTiles = 8;   // pair tiles of rows per band: the same 4096 tokens of A as a band of single-CTA tiles
+constexpr int kPairStageBytes = kPairABytes + kPairBBytes;           // 48 KB
+constexpr int kPairDstBytes = kPairMT * (kPairBN / kD) * kBM * 8;
+constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + 256 + kPairDstBytes + 64;
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+kv_proj_cache_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBk,
+                          const __grid_constant__ CUtensorMap tmBv, const __grid_constant__ CUtensorMap tmBq,
+                          const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                          const __grid_constant__ CUtensorMap tmQ, const uint8_t *__restrict__ flags,
+                          int32_t *__restrict__ prefix, int32_t *__restrict__ idx, const int64_t *__restrict__ row_off,
+                          const int32_t *__restrict__ cap, int32_t *__restrict__ len, uint8_t *__restrict__ k_rows,
+                          uint8_t *__restrict__ v_rows, int32_t *__restrict__ dev_status, int n_sub, int tps, int Kdim,
+                          int GD, int n, int kv_heads, int heads, int n_tiles_m, int n_tiles_n, int split_from) {
+  constexpr int BN = kPairBN, MT = kPairMT;
+  constexpr uint32_t kTmemCols = MT * BN;          // 512: two accumulators of 128 rows x 256 columns per CTA
+  static_assert(MT * (BN / 64) * kBM * 128 <= kPairStages * kPairStageBytes, "staging fits the stages");
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + kPairStages * kPairStageBytes);   // used in the leader only
+  uint64_t *empty = full + kPairStages;            // one set per CTA: a commit arrives on both
+  uint64_t *acc_full = empty + kPairStages;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  long long *dst_row = reinterpret_cast<long long *>(smem + kPairStages * kPairStageBytes + 256);
+  int *red = reinterpret_cast<int *>(smem + kPairStages * kPairStageBytes + 256 + kPairDstBytes);
+  int *gave_up = red + 12;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();         // 0: leader
+  // pairs below split_from take whole pair tiles, the rest one half (256 tokens) of a pair tile
+  const int pair = blockIdx.x >> 1;
+  const bool single = pair >= split_from;
+  const int tile = single ? split_from + ((pair - split_from) >> 1) : pair;
+  const int mts = single ? 1 : MT;                 // sub-tiles of each CTA
+  const int band = tile / (kPairBandTiles * n_tiles_n), in_band = tile % (kPairBandTiles * n_tiles_n);
+  const int band_rows = min(kPairBandTiles, n_tiles_m - band * kPairBandTiles);
+  const int tile_m = band * kPairBandTiles + in_band % band_rows, tile_n = in_band / band_rows;
+  const int sub0 = tile_m * (2 * MT) + (single ? ((pair - split_from) & 1) * 2 + (int)rank : (int)rank * MT);
+  const int n0 = tile_n * BN;
+  const int which = n0 < GD ? 0 : (n0 < 2 * GD ? 1 : 2);
+  const int nw = n0 - min(which, 2) * GD;
+  const CUtensorMap *tmB = which == 0 ? &tmBk : (which == 1 ? &tmBv : &tmBq);
+  const int num_kb = (Kdim + kBK - 1) / kBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPairStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    *gave_up = 0;
+    fence_barrier_init();
+    prefetch_tensormap(&tmA);
+    prefetch_tensormap(tmB);
+  }
+  __syncthreads();
+  if (warp == 1) {                                 // the same warp of both CTAs, the same arguments
+    tmem_alloc_pair(tmem_slot, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  cluster_arrive_wait();                           // both CTAs' barriers are initialised, tensor memory is allocated
+  tc_fence_after_sync();
+  const uint32_t tmem_acc = *tmem_slot;
+  const uint32_t stage_tx = (uint32_t)(mts * (kBM * kBK * 2) + kPairBBytes);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % kPairStages;
+        const uint32_t ph = (kb / kPairStages) & 1;
+        if (!mbar_wait(&empty[s], ph ^ 1)) break;  // this CTA's copy: the MMAs that read the stage (in both CTAs) are done
+        uint8_t *a = smem + s * kPairStageBytes, *b = a + kPairABytes;
+        if (rank == 0) mbar_arrive_expect_tx(&full[s], 2 * stage_tx);   // the leader's barrier counts both CTAs' bytes
+        const uint32_t bar = mapa_shared(smem_u32(&full[s]), 0);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)            // rows past the sequence (or past the batch) are filled with zeros
+          if (mt < mts)
+            tma_load_3d_pair(a + mt * (kBM * kBK * 2), &tmA, bar, kb * kBK, ((sub0 + mt) % tps) * kBM, (sub0 + mt) / tps);
+#pragma unroll
+        for (int p = 0; p < BN / 2 / 64; ++p)      // this CTA's half of the tile's columns
+          tma_load_2d_pair(b + p * (kBK * 64 * 2), tmB, bar, nw + (int)rank * (BN / 2) + p * 64, kb * kBK);
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0) {
+      // every lane runs the control flow (operands stay warp-uniform); one elected lane issues
+      const uint32_t idesc = idesc_bf16_f32(2 * kBM, BN, false, true);
+      const uint64_t da0 = desc_kmajor_sw128(smem_u32(smem));
+      const uint64_t db0 = desc_mnmajor_sw128(smem_u32(smem) + kPairABytes, kBK * 64 * 2);
+      const uint32_t a_lo0 = (uint32_t)da0, a_hi = (uint32_t)(da0 >> 32);
+      const uint32_t b_lo0 = (uint32_t)db0, b_hi = (uint32_t)(db0 >> 32);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb && ok; ++kb) {
+        const int s = kb % kPairStages;
+        const uint32_t ph = (kb / kPairStages) & 1;
+        ok = mbar_wait(&full[s], ph);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t a_lo = a_lo0 + ((s * kPairStageBytes) >> 4), b_lo = b_lo0 + ((s * kPairStageBytes) >> 4);
+        if (elect_one()) {
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+              if (mt < mts) mma_ss_pair_lohi(tmem_acc + mt * BN, a_lo + ((mt * kBM * kBK * 2 + k * 32) >> 4), a_hi,
+                                             b_lo + ((k * 2048) >> 4), b_hi, idesc, (kb | k) != 0);
+          }
+          mma_commit_pair(&empty[s]);              // frees the stage in both CTAs once these MMAs have read it
+        }
+        __syncwarp();
+      }
+      if (elect_one()) mma_commit_pair(acc_full);  // accumulators complete (or unwinding), in both CTAs
+      __syncwarp();
+    }
+  } else {
+    const KvEpilogue e{&tmK, &tmV, &tmQ, flags, prefix, idx, row_off, cap, len, k_rows, v_rows, dev_status, n_sub, tps, n, kv_heads, heads};
+    kv_epilogue<BN, MT>(e, smem, dst_row, red, gave_up, acc_full, tmem_acc, sub0, mts, which, nw, num_kb, warp, lane);
+  }
+  // neither CTA leaves (or frees tensor memory) while the other may still use its shared or tensor memory
+  tc_fence_before_sync();
+  cluster_arrive_wait();
+  if (warp == 1) tmem_dealloc_pair(tmem_acc, kTmemCols);
 }
 
 int sm_count() {
@@ -301,7 +456,7 @@ int sm_count() {
 template <int BN, int MT>
 int run(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, const void *Wv, const uint8_t *flags,
         const ag_cache &c, int32_t *prefix, int32_t *idx, void *Q, void *K, void *V, int32_t *dev_status,
-        cudaStream_t st) {
+        cudaStream_t st, bool pairs = false) {
   using Cfg = KvCfg<BN, MT>;
   const int hk = kv_heads_of(d), GD = hk * kD, Kdim = d.hidden;
   const int tps = (d.seq + kBM - 1) / kBM, n_sub = d.batch * tps;   // sub-tiles of 128 tokens per sequence, in all
@@ -325,15 +480,26 @@ int run(const ag_layer_desc &d, const void *X, const void *Wq, const void *Wk, c
     rc = make_tmap_3d_bf16(&tmQ, Q, (uint64_t)d.batch * d.heads, d.seq, kD, kBM, 64);
     if (rc) return rc;
   }
+  if (pairs) {
+    // 512 x 256 tiles on CTA pairs; the tiles of a last wave that would fill at most half of the pairs are halved
+    AG_CUDA_TRY(cudaFuncSetAttribute(kv_proj_cache_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes));
+    const int n_tiles_n = (2 * GD + QD) / kPairBN, n_tiles_m = (n_sub + 2 * kPairMT - 1) / (2 * kPairMT);
+    const int n_tiles = n_tiles_n * n_tiles_m, n_pairs = sm_count() / 2;
+    const int tail = n_tiles % n_pairs;
+    const int split_from = (tail > 0 && 2 * tail <= n_pairs) ? n_tiles - tail : n_tiles;
+    const int ctas = 2 * (split_from + 2 * (n_tiles - split_from));
+    kv_proj_cache_pair_kernel<<<ctas, kThreads, kPairSmemBytes, st>>>(
+        tmA, tmBk, tmBv, tmBq, tmK, tmV, tmQ, flags, prefix, idx, c.row_off, c.cap, c.len, static_cast<uint8_t *>(c.k_rows),
+        static_cast<uint8_t *>(c.v_rows), dev_status, n_sub, tps, Kdim, GD, d.seq, hk, d.heads, n_tiles_m, n_tiles_n, split_from);
+    AG_LAUNCH_CHECK();
+    return AG_OK;
+  }
   auto kern = kv_proj_cache_kernel<BN, MT>;
   AG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
   const int n_tiles_n = (2 * GD + QD) / BN, n_tiles_m = (n_sub + MT - 1) / MT, n_tiles = n_tiles_n * n_tiles_m;
-  const int tail = n_tiles % sm_count();
-  const int split_from = (MT > 1 && tail > 0 && 2 * tail <= sm_count()) ? n_tiles - tail : n_tiles;
-  const int ctas = split_from + 2 * (n_tiles - split_from);
-  kern<<<ctas, kThreads, Cfg::kSmemBytes, st>>>(tmA, tmBk, tmBv, tmBq, tmK, tmV, tmQ, flags, prefix, idx, c.row_off, c.cap, c.len,
+  kern<<<n_tiles, kThreads, Cfg::kSmemBytes, st>>>(tmA, tmBk, tmBv, tmBq, tmK, tmV, tmQ, flags, prefix, idx, c.row_off, c.cap, c.len,
                                                    static_cast<uint8_t *>(c.k_rows), static_cast<uint8_t *>(c.v_rows),
-                                                   dev_status, n_sub, tps, Kdim, GD, d.seq, hk, d.heads, n_tiles_m, n_tiles_n, split_from);
+                                                   dev_status, n_sub, tps, Kdim, GD, d.seq, hk, d.heads, n_tiles_m, n_tiles_n);
   AG_LAUNCH_CHECK();
   return AG_OK;
 }
@@ -352,8 +518,8 @@ int launch_kv_proj_cache(const ag_layer_desc &d, const void *X, const void *Wq, 
   const long long tiles128 = (long long)(2 * hk + hq) * d.batch * ((d.seq + kBM - 1) / kBM);
   int rc;
   if (hk % 2 == 0 && hq % 2 == 0) {
-    // more than one wave: 256-token tiles, whose two sub-tiles share every stage of W
-    if (tiles128 > 2 * sm_count()) rc = run<256, 2>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
+    // more than one wave: CTA pairs on 512 x 256 tiles
+    if (tiles128 > 2 * sm_count()) rc = run<256, 1>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st, true);
     else rc = run<256, 1>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);
   } else {
     rc = run<128, 1>(d, X, Wq, Wk, Wv, flags, c, prefix, idx, Q, K, V, dev_status, st);

@@ -235,6 +235,7 @@ out_proj_tc_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_constan
 constexpr int kPairBN = 256, kPairMT = 2, kPairStages = 4;
 constexpr int kPairABytes = kPairMT * kBM * kBK * 2;                 // 32 KB: this CTA's two sub-tiles
 constexpr int kPairBBytes = (kPairBN / 2 / 64) * (kBK * 64 * 2);     // 16 KB: this CTA's half of the W^O stage
+constexpr int kPairBandTiles = 8;   // pair tiles of rows per band: the same 4096 tokens of A as a band of single-CTA tiles
 constexpr int kPairStageBytes = kPairABytes + kPairBBytes;           // 48 KB
 constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + 256;
 
@@ -257,9 +258,9 @@ out_proj_pair_kernel(const __grid_constant__ CUtensorMap tmO, const __grid_const
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();         // 0: leader
   const int tile = blockIdx.x >> 1;
-  const int band = tile / (kBandTiles * n_tiles_n), in_band = tile % (kBandTiles * n_tiles_n);
-  const int band_rows = min(kBandTiles, n_tiles_m - band * kBandTiles);
-  const int tile_m = band * kBandTiles + in_band % band_rows, tile_n = in_band / band_rows;
+  const int band = tile / (kPairBandTiles * n_tiles_n), in_band = tile % (kPairBandTiles * n_tiles_n);
+  const int band_rows = min(kPairBandTiles, n_tiles_m - band * kPairBandTiles);
+  const int tile_m = band * kPairBandTiles + in_band % band_rows, tile_n = in_band / band_rows;
   const int sub0 = tile_m * (2 * MT) + (int)rank * MT;   // this CTA's first sub-tile of 128 tokens
   const int n0 = tile_n * BN;
   const int num_kb = heads * (kD / kBK);

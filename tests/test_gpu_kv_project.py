@@ -116,19 +116,20 @@ CASES = {
     "two_heads_per_tile": LayerShape(2, 256, 512, 4, 128, 2, 128, "bf16"),
     "k_tail": LayerShape(1, 384, 520, 4, 128, 2, 128, "bf16"),                 # hidden not a multiple of 64
     "odd_heads": LayerShape(2, 128, 256, 3, 128, 1, 128, "bf16"),              # one head per tile
-    "two_subtiles": LayerShape(1, 1280, 256, 16, 128, 2, 128, "bf16"),         # 256-token tiles
-    "two_subtiles_odd_rows": LayerShape(1, 1152, 192, 18, 128, 2, 128, "bf16"),  # last tile has one sub-tile
+    "two_subtiles": LayerShape(1, 1280, 256, 16, 128, 2, 128, "bf16"),         # CTA pairs; the last pair tile has two of four sub-tiles
+    "two_subtiles_odd_rows": LayerShape(1, 1152, 192, 18, 128, 2, 128, "bf16"),  # CTA pairs; nine sub-tiles: one CTA of the last pair has none
     "subtiles_of_two_sequences": LayerShape(3, 384, 128, 20, 128, 2, 128, "bf16"),
-    "split_last_wave": LayerShape(1, 2560, 128, 16, 128, 2, 128, "bf16"),      # 160 tiles on 148 SMs: 12 are split
+    "split_last_wave": LayerShape(1, 2560, 128, 16, 128, 2, 128, "bf16"),      # 80 pair tiles on 74 pairs: 6 are halved
     "split_last_wave_odd_rows": LayerShape(1, 2432, 128, 16, 128, 2, 128, "bf16"),
     "grouped_query": LayerShape(2, 256, 256, 8, 128, 2, 128, "bf16", kv_heads=2),
     "three_bands_of_row_tiles": LayerShape(1, 4864, 128, 2, 128, 1, 128, "bf16"),    # 38 row tiles: bands of 16, 16, 6
-    "two_bands_of_256_row_tiles": LayerShape(2, 2432, 128, 8, 128, 2, 128, "bf16"),  # 19 row tiles: bands of 16 and 3, split last wave
+    "two_sequences_of_19_subtiles": LayerShape(2, 2432, 128, 8, 128, 2, 128, "bf16"),  # 38 sub-tiles: 10 pair tiles of rows, the last half empty
+    "two_bands_of_pair_tiles": LayerShape(1, 8704, 128, 4, 128, 2, 128, "bf16"),     # 68 sub-tiles: bands of 16 pair tiles and 1
     "one_sequence_ragged_end": LayerShape(1, 333, 256, 4, 128, 2, 128, "bf16"),      # n not a multiple of 16
     "one_sequence_short": LayerShape(1, 48, 128, 6, 128, 2, 128, "bf16"),            # less than one tile
     "one_sequence_long_ragged": LayerShape(1, 2500, 128, 16, 128, 2, 128, "bf16"),   # split last wave, ragged end
     "batch_ragged_end": LayerShape(3, 200, 256, 4, 128, 2, 128, "bf16"),             # every sequence ends inside its last sub-tile
-    "batch_ragged_two_subtiles": LayerShape(5, 333, 128, 20, 128, 2, 128, "bf16"),   # 256-token tiles whose sub-tiles belong to two sequences, ragged ends
+    "batch_ragged_two_subtiles": LayerShape(5, 333, 128, 20, 128, 2, 128, "bf16"),   # pair tiles whose sub-tiles belong to several sequences, ragged ends, halved last wave
 }
 
 
