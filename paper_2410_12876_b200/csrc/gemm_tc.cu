@@ -200,6 +200,178 @@ gemm_bf16_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   if (warp == 1) tmem_dealloc(tmem_acc, kTmemCols);
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same GEMM on CTA pairs (cta_group::2): a pair computes 256 rows x 384 columns, each CTA holding
+// its 128 rows of X and half of every stage of W; the leader issues, per 16 elements of K, one MMA of
+// M = 256, N = 256 and one of N = 128 (384 = 3 x 128 divides the packed width 3 GD of every shape
+// this file covers).  Per 64-deep k-block the tensor cores read 56 KB of operands from each CTA's
+// shared memory while TMA writes 40 KB, under the 128 bytes a clock shared memory moves in the 768
+// clocks of MMA work; one CTA on a 256 x 192 tile (the same work) moves 136 KB and takes ~1,050.
+// The whole tile is staged at once over the operand stages (hi and lo: 192 KB of the 200).
+constexpr int kGpBN = 384, kGpStages = 5;
+constexpr int kGpABytes = kTcBM * kTcBK * 2;                      // 16 KB: this CTA's rows of X
+constexpr int kGpPanelBytes = kTcBK * 64 * 2;                     // [64 k][64 n] = 8 KB
+constexpr int kGpBBytes = (kGpBN / 2 / 64) * kGpPanelBytes;       // 24 KB: two panels of the N = 256 MMA, one of the N = 128
+constexpr int kGpStageBytes = kGpABytes + kGpBBytes;              // 40 KB
+constexpr int kGpSmemBytes = kGpStages * kGpStageBytes + 1024 + 256;
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTcThreads, 1)
+gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+                      const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
+                      const __grid_constant__ CUtensorMap tmChi, const __grid_constant__ CUtensorMap tmClo,
+                      float *__restrict__ C, bool split, int M, int K, int GD, int n_tiles_n) {
+  constexpr uint32_t kTmemCols = 512;              // 384 used: columns [0, 256) of the wide MMA, [256, 384) of the narrow
+  static_assert(2 * (kGpBN / 64) * kTcBM * 128 <= kGpStages * kGpStageBytes, "staging fits the stages");
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + kGpStages * kGpStageBytes);   // used in the leader only
+  uint64_t *empty = full + kGpStages;              // one set per CTA: a commit arrives on both
+  uint64_t *acc_full = empty + kGpStages;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  int *gave_up = reinterpret_cast<int *>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();         // 0: leader
+  const int tile = blockIdx.x >> 1;
+  const int m0 = (tile / n_tiles_n) * (2 * kTcBM) + (int)rank * kTcBM;   // this CTA's rows
+  const int n0 = (tile % n_tiles_n) * kGpBN;                              // in the packed [3 * GD] output
+  const int num_kb = (K + kTcBK - 1) / kTcBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kGpStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    *gave_up = 0;
+    fence_barrier_init();
+    prefetch_tensormap(&tmA);
+    prefetch_tensormap(&tmB0);
+  }
+  __syncthreads();
+  if (warp == 1) {                                 // the same warp of both CTAs, the same arguments
+    tmem_alloc_pair(tmem_slot, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  cluster_arrive_wait();                           // both CTAs' barriers are initialised, tensor memory is allocated
+  tc_fence_after_sync();
+  const uint32_t tmem_acc = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % kGpStages;
+        const uint32_t ph = (kb / kGpStages) & 1;
+        if (!mbar_wait(&empty[s], ph ^ 1)) break;  // this CTA's copy: the MMAs that read the stage (in both CTAs) are done
+        uint8_t *a = smem + s * kGpStageBytes, *b = a + kGpABytes;
+        if (rank == 0) mbar_arrive_expect_tx(&full[s], 2 * kGpStageBytes);   // the leader's barrier counts both CTAs' bytes
+        const uint32_t bar = mapa_shared(smem_u32(&full[s]), 0);
+        tma_load_2d_pair(a, &tmA, bar, kb * kTcBK, m0);                      // rows past M are filled with zeros
+#pragma unroll
+        for (int p = 0; p < 3; ++p) {
+          // this CTA's half of the wide MMA's columns (two panels), then of the narrow one's (one panel);
+          // a 64-column panel lies in one weight (64 divides GD)
+          const int col = n0 + (p < 2 ? (int)rank * 128 + p * 64 : 256 + (int)rank * 64), which = col / GD;
+          tma_load_2d_pair(b + p * kGpPanelBytes, which == 0 ? &tmB0 : (which == 1 ? &tmB1 : &tmB2), bar, col % GD,
+                           kb * kTcBK);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0) {
+      // every lane runs the control flow (operands stay warp-uniform); one elected lane issues
+      const uint32_t idesc_w = idesc_bf16_f32(2 * kTcBM, 256, false, true), idesc_n = idesc_bf16_f32(2 * kTcBM, 128, false, true);
+      const uint64_t da0 = desc_kmajor_sw128(smem_u32(smem));
+      const uint64_t db0 = desc_mnmajor_sw128(smem_u32(smem) + kGpABytes, kGpPanelBytes);
+      const uint32_t a_lo0 = (uint32_t)da0, a_hi = (uint32_t)(da0 >> 32);
+      const uint32_t b_lo0 = (uint32_t)db0, b_hi = (uint32_t)(db0 >> 32);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb && ok; ++kb) {
+        const int s = kb % kGpStages;
+        const uint32_t ph = (kb / kGpStages) & 1;
+        ok = mbar_wait(&full[s], ph);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t a_lo = a_lo0 + ((s * kGpStageBytes) >> 4), b_lo = b_lo0 + ((s * kGpStageBytes) >> 4);
+        if (elect_one()) {
+#pragma unroll
+          for (int k = 0; k < kTcBK / 16; ++k) {
+            // 16 elements of K: 32 bytes along a K-major row; 16 k-rows (2048 B) of an MN-major panel
+            mma_ss_pair_lohi(tmem_acc, a_lo + ((k * 32) >> 4), a_hi, b_lo + ((k * 2048) >> 4), b_hi, idesc_w, (kb | k) != 0);
+            mma_ss_pair_lohi(tmem_acc + 256, a_lo + ((k * 32) >> 4), a_hi, b_lo + ((2 * kGpPanelBytes + k * 2048) >> 4), b_hi,
+                             idesc_n, (kb | k) != 0);
+          }
+          mma_commit_pair(&empty[s]);              // frees the stage in both CTAs once these MMAs have read it
+        }
+        __syncwarp();
+      }
+      if (elect_one()) mma_commit_pair(acc_full);  // accumulators complete (or unwinding), in both CTAs
+      __syncwarp();
+    }
+  } else {
+    // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32); warps 2..5 drain columns [0, 192), warps 6..9 the rest
+    const int quad = warp & 3, half = (warp - 2) >> 2;
+    const int c_begin = half * (kGpBN / 2), c_end = c_begin + kGpBN / 2;
+    if (!mbar_wait(acc_full, 0)) *gave_up = 1;
+    named_barrier_sync(1, 256);
+    const bool ok = *gave_up == 0;
+    tc_fence_after_sync();
+    const int r_in = quad * 32 + lane, row = m0 + r_in;
+    if (ok && num_kb > 0 && split) {
+      // x = hi + lo in bf16 pairs.  Every MMA of both CTAs has completed, so every stage has been read: the
+      // tile is staged over them as panels of [128 rows][64 bf16] (128-byte rows, 16-byte chunks
+      // XOR-swizzled by the row): six hi panels, then six lo panels.
+      uint8_t *stage_lo = smem + (kGpBN / 64) * kTcBM * 128;
+#pragma unroll 1
+      for (int c = c_begin; c < c_end; c += 32) {
+        uint32_t r[32];
+        tmem_ld_x32_sync(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
+        const uint32_t panel = (uint32_t)(c >> 6) * kTcBM * 128 + r_in * 128;
+#pragma unroll
+        for (int e = 0; e < 32; e += 8) {
+          uint32_t h[4], l[4];
+#pragma unroll
+          for (int q = 0; q < 8; q += 2) {
+            float h0, l0, h1, l1;
+            split_bf16(__uint_as_float(r[e + q]), h0, l0);
+            split_bf16(__uint_as_float(r[e + q + 1]), h1, l1);
+            h[q >> 1] = pack_bf16x2(h0, h1);
+            l[q >> 1] = pack_bf16x2(l0, l1);
+          }
+          const uint32_t chunk = (uint32_t)(((c & 32) >> 3) + (e >> 3));          // 16-byte chunk within the 128-byte row
+          const uint32_t off = panel + ((chunk ^ (r_in & 7)) << 4);
+          *reinterpret_cast<uint4 *>(smem + off) = make_uint4(h[0], h[1], h[2], h[3]);
+          *reinterpret_cast<uint4 *>(stage_lo + off) = make_uint4(l[0], l[1], l[2], l[3]);
+        }
+      }
+      fence_proxy_async_smem();
+      named_barrier_sync(1, 256);
+      if (threadIdx.x == 64) {
+        for (int p = 0; p < kGpBN / 64; ++p) {         // rows past M are dropped by the tensor map
+          tma_store_2d(&tmChi, smem + p * kTcBM * 128, n0 + p * 64, m0);
+          tma_store_2d(&tmClo, stage_lo + p * kTcBM * 128, n0 + p * 64, m0);
+        }
+        tma_store_commit();
+        tma_store_wait_read();
+      }
+    } else if (ok && num_kb > 0) {
+      const size_t crow = (size_t)row * 3 * GD + n0;
+#pragma unroll 1
+      for (int c = c_begin; c < c_end; c += 32) {
+        uint32_t r[32];
+        tmem_ld_x32_sync(tmem_acc + ((uint32_t)(quad * 32) << 16) + c, r);
+        if (row < M) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 4)
+            *reinterpret_cast<uint4 *>(C + crow + c + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+        }
+      }
+    }
+  }
+  // neither CTA leaves (or frees tensor memory) while the other may still use its shared or tensor memory
+  tc_fence_before_sync();
+  cluster_arrive_wait();
+  if (warp == 1) tmem_dealloc_pair(tmem_acc, kTmemCols);
+}
+
 // ------------------------------------------------------------ tensor maps
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -293,11 +465,39 @@ static int run_gemm_tc(const void *X, const void *W0, const void *W1, const void
   return AG_OK;
 }
 
+static int run_gemm_pair(const void *X, const void *W0, const void *W1, const void *W2, float *C, __nv_bfloat16 *Chi,
+                         __nv_bfloat16 *Clo, int M, int K, int GD, cudaStream_t st) {
+  CUtensorMap tmA, tmB[3];
+  int rc = make_tmap_2d_bf16(&tmA, X, M, K, (uint64_t)K * 2, kTcBM, kTcBK);
+  if (rc) return rc;
+  const void *Ws[3] = {W0, W1, W2};
+  for (int i = 0; i < 3; ++i) {
+    rc = make_tmap_2d_bf16(&tmB[i], Ws[i], K, GD, (uint64_t)GD * 2, kTcBK, 64);
+    if (rc) return rc;
+  }
+  CUtensorMap tmC[2];
+  const void *outs[2] = {Chi ? (const void *)Chi : W0, Clo ? (const void *)Clo : W0};
+  for (int i = 0; i < 2; ++i) {
+    rc = Chi ? make_tmap_2d_bf16(&tmC[i], outs[i], M, 3 * (uint64_t)GD, 3 * (uint64_t)GD * 2, kTcBM, 64)
+             : make_tmap_2d_bf16(&tmC[i], outs[i], 1, GD, (uint64_t)GD * 2, 1, 64);
+    if (rc) return rc;
+  }
+  AG_CUDA_TRY(cudaFuncSetAttribute(gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGpSmemBytes));
+  const int n_tiles_n = 3 * GD / kGpBN, n_tiles_m = (M + 2 * kTcBM - 1) / (2 * kTcBM);
+  gemm_bf16_pair_kernel<<<2 * n_tiles_n * n_tiles_m, kTcThreads, kGpSmemBytes, st>>>(
+      tmA, tmB[0], tmB[1], tmB[2], tmC[0], tmC[1], C, Chi != nullptr, M, K, GD, n_tiles_n);
+  AG_LAUNCH_CHECK();
+  return AG_OK;
+}
+
 bool gate_proj_tc_supported(int K, int GD) { return GD % 128 == 0 && K % 8 == 0; }
 
 int launch_gate_proj_tc(const void *X, const void *W0, const void *W1, const void *W2, float *C, void *Chi,
                         void *Clo, int M, int K, int GD, cudaStream_t st) {
   auto hi = static_cast<__nv_bfloat16 *>(Chi), lo = static_cast<__nv_bfloat16 *>(Clo);
+  // at least half a wave of pair tiles (256 x 384): CTA pairs
+  if ((long long)(3 * GD / kGpBN) * ((M + 2 * kTcBM - 1) / (2 * kTcBM)) * 4 >= gemm_sm_count())
+    return run_gemm_pair(X, W0, W1, W2, C, hi, lo, M, K, GD, st);
   if (GD % 256 == 0) {
     // more than one wave of 128 x 256 tiles: 256 x 256 tiles, whose two row sub-tiles share every
     // stage of W (a third less operand traffic per FLOP; the kernel is bound by feeding the SMs)
