@@ -164,11 +164,13 @@ def test_ragged_decode():
     assert int(status.item()) == 0
 
 
-def test_gate_projection_in_256_row_tiles():
-    """A gate projection of more than one wave of tiles (5120 rows x 1536 columns): the GEMM then
-    takes 256 x 256 tiles over several waves with a halved last wave, the form the batch-8 stack
-    runs.  Small hidden size, so that the oracle evaluates every score of both sequences."""
-    shape = inputs.LayerShape(2, 2560, 128, 8, 128, 4, 128, "bf16")
+@pytest.mark.parametrize("batch,seq", [(2, 2560), (3, 1111)], ids=["whole_tiles", "ragged_rows"])
+def test_gate_projection_on_cta_pairs(batch, seq):
+    """A gate projection of more than half a wave of pair tiles (5120 or 3333 rows x 1536 columns):
+    the GEMM then runs 256 x 384 tiles on CTA pairs, the form the 7B-shaped layer and the batch-8
+    stack run; pair tiles straddle two weights, and with 3333 rows the last pair has 5 valid rows in
+    one CTA and none in the other.  Small hidden size, so that the oracle evaluates every score."""
+    shape = inputs.LayerShape(batch, seq, 128, 8, 128, 4, 128, "bf16")
     seed = 5200
     X = inputs.hidden_states(shape, seed, DEV)
     W = inputs.layer_weights(shape, seed + 10, DEV)
