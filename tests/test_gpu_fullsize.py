@@ -164,13 +164,15 @@ def test_ragged_decode():
     assert int(status.item()) == 0
 
 
-@pytest.mark.parametrize("batch,seq", [(2, 2560), (3, 1111)], ids=["whole_tiles", "ragged_rows"])
-def test_gate_projection_on_cta_pairs(batch, seq):
+@pytest.mark.parametrize("batch,seq,gh,gd", [(2, 2560, 4, 128), (3, 1111, 4, 128), (2, 1300, 8, 64)],
+                         ids=["whole_tiles", "ragged_rows", "float32_output"])
+def test_gate_projection_on_cta_pairs(batch, seq, gh, gd):
     """A gate projection of more than half a wave of pair tiles (5120 or 3333 rows x 1536 columns):
     the GEMM then runs 256 x 384 tiles on CTA pairs, the form the 7B-shaped layer and the batch-8
     stack run; pair tiles straddle two weights, and with 3333 rows the last pair has 5 valid rows in
-    one CTA and none in the other.  Small hidden size, so that the oracle evaluates every score."""
-    shape = inputs.LayerShape(batch, seq, 128, 8, 128, 4, 128, "bf16")
+    one CTA and none in the other.  With gate heads of 64 dimensions MHA' runs on CUDA cores and the
+    GEMM leaves float32 instead of hi / lo pairs.  Small hidden size, so that the oracle evaluates every score."""
+    shape = inputs.LayerShape(batch, seq, 128, 8 if gh < 8 else 16, 128, gh, gd, "bf16")
     seed = 5200
     X = inputs.hidden_states(shape, seed, DEV)
     W = inputs.layer_weights(shape, seed + 10, DEV)
