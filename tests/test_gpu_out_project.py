@@ -39,15 +39,17 @@ def _close_to_rounded(got, ref, dtype, what):
 SHAPES = {
     # name: (shape, what it reaches)
     "one_sub_tile_per_cta": LayerShape(2, 256, 512, 8, 128, 2, 128, "bf16"),          # 256-column tiles, MT = 1
-    "two_sequences_in_a_tile": LayerShape(21, 128, 2048, 8, 128, 2, 128, "bf16"),     # two sub-tiles per CTA, each of another sequence; the last tile has one
-    "split_last_wave": LayerShape(2, 2560, 2048, 4, 128, 2, 128, "bf16"),             # 160 tiles of 256 x 256: 148 + 12 split in two
+    "two_sequences_in_a_tile": LayerShape(21, 128, 2048, 8, 128, 2, 128, "bf16"),     # CTA pairs: four sub-tiles per pair tile, each of another sequence; the last pair tile has one
+    "split_last_wave": LayerShape(2, 2560, 2048, 4, 128, 2, 128, "bf16"),             # CTA pairs: 10 pair tiles of rows x 8 of columns
+    "pairs_one_head": LayerShape(3, 640, 2048, 1, 128, 1, 128, "bf16"),                # CTA pairs with two k-blocks only: fewer than the stages
+    "pairs_two_heads": LayerShape(3, 640, 2048, 2, 128, 1, 128, "bf16"),               # four k-blocks: every slice of the skip connection released at the last
     "single_sequence_ragged_end": LayerShape(1, 333, 512, 4, 128, 2, 128, "bf16"),    # the last sub-tile reaches past the sequence
     "columns_128": LayerShape(1, 300, 384, 3, 128, 1, 128, "bf16"),                   # 128-column tiles, odd head count
     "cuda_cores_f32": inputs.TINY,
     "cuda_cores_bf16_d64": LayerShape(2, 150, 256, 4, 64, 2, 64, "bf16"),
     "cuda_cores_odd_width": LayerShape(2, 100, 200, 2, 128, 1, 128, "bf16"),
     "batch_ragged_end": LayerShape(3, 100, 256, 2, 128, 1, 128, "bf16"),              # every sequence ends inside its only sub-tile
-    "batch_ragged_two_subtiles": LayerShape(21, 200, 2048, 8, 128, 2, 128, "bf16"),   # two sub-tiles per CTA, ragged ends
+    "batch_ragged_two_subtiles": LayerShape(21, 200, 2048, 8, 128, 2, 128, "bf16"),   # CTA pairs, ragged ends
 }
 
 
