@@ -21,7 +21,8 @@
 // (O, m, l); gate_merge_out_kernel combines the pieces of a query tile and
 // applies the gate's output layer and threshold.
 //
-// TMEM columns: S0 [0,128) S1 [128,256) O [256,384) Phi [384,448) Plo [448,512).
+// TMEM columns: S0 [0,64) S1 [128,192) O [256,384) Phi [384,448) Plo [448,512), each P half holding two
+// tiles' weights (32 columns per tile).
 #include "ag_common.cuh"
 #include "umma.cuh"
 
@@ -120,9 +121,12 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
   uint64_t *bars = reinterpret_cast<uint64_t *>(sV + 2 * kGaKvStage);
   uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;  // [2]
   uint64_t *s_full = bars + 9;           // [2]
-  uint64_t *p_ready = bars + 11, *pv_done = bars + 12;
-  uint64_t *q_empty = bars + 13, *o_free = bars + 14;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 15);
+  // p_ready[2], pv_done[2]: even / odd tiles.  P is double-buffered (32 of each half's 64 columns per tile), so
+  // the weights of tile t are written while the P V of tile t - 1 runs; a softmax warp may be a tile ahead
+  // of a slower one, never two (the scores of tile t + 2 exist only after every thread arrived for tile t).
+  uint64_t *p_ready = bars + 11, *pv_done = bars + 13;
+  uint64_t *q_empty = bars + 15, *o_free = bars + 16;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 17);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // This CTA's segment of the step list.  Every role walks its pieces with the same arithmetic;
@@ -138,8 +142,8 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
       mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
       mbar_init(&s_full[s], 1);
     }
-    mbar_init(p_ready, 128);
-    mbar_init(pv_done, 1);
+    mbar_init(&p_ready[0], 128); mbar_init(&p_ready[1], 128);
+    mbar_init(&pv_done[0], 1); mbar_init(&pv_done[1], 1);
     mbar_init(q_empty, 1);
     mbar_init(o_free, 128);
     fence_barrier_init();
@@ -235,7 +239,7 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
       if (i + 1 < n_kv) ok = issue_qk(t + 1, i + 2 == n_kv);
       if (!ok) break;
       const int st = t & 1;
-      if (!mbar_wait(p_ready, t & 1)) { ok = false; break; }
+      if (!mbar_wait(&p_ready[t & 1], (t >> 1) & 1)) { ok = false; break; }
       if (!mbar_wait(&v_full[st], (t >> 1) & 1)) { ok = false; break; }
       // the first P V of a piece overwrites O: the previous piece's epilogue must have read it
       if (i == 0 && pc > 0 && !mbar_wait(o_free, (pc - 1) & 1)) { ok = false; break; }
@@ -245,13 +249,13 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
         // Phi Vhi + Phi Vlo + Plo Vhi
 #pragma unroll
         for (int t = 0; t < 3; ++t) {
-          const uint32_t pa = tmem + (t == 2 ? kGaColPlo : kGaColPhi), va = vb + ((t == 1 ? kGaKvTile : 0) >> 4);
+          const uint32_t pa = tmem + (t == 2 ? kGaColPlo : kGaColPhi) + st * (kGaBN / 2), va = vb + ((t == 1 ? kGaKvTile : 0) >> 4);
 #pragma unroll
           for (int k = 0; k < kGaBN / 16; ++k)
             mma_ts_lohi(tmem + kGaColO, pa + k * 8, va + ((k * 2048) >> 4), v_hi, idesc_pv, (i | t | k) != 0);
         }
         mma_commit(&v_empty[st]);
-        mma_commit(pv_done);
+        mma_commit(&pv_done[st]);
       }
       __syncwarp();
       }
@@ -326,20 +330,26 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
       l *= alpha;
       const float m_exp = m_new == -INFINITY ? 0.f : m_new;    // exponent offset: keeps -inf - (-inf) out
 
-      if (i > 0) {
-        ok = mbar_wait(pv_done, (t - 1) & 1);
+      // Only a rescale of O has to wait for the P V of tile t - 1 (the next phase of that barrier is the P V of
+      // tile t + 1, which cannot have been issued yet: the parity is unambiguous)
+      if (rescale) {
+        ok = mbar_wait(&pv_done[(t - 1) & 1], ((t - 1) >> 1) & 1);
         if (!ok) break;
         tc_fence_after_sync();
-        if (rescale) {
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            uint32_t r[32];
-            tmem_ld_x32_sync(tm_lane + kGaColO + c * 32, r);
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld_x32_sync(tm_lane + kGaColO + c * 32, r);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-            tmem_st_x32(tm_lane + kGaColO + c * 32, r);
-          }
+          for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+          tmem_st_x32(tm_lane + kGaColO + c * 32, r);
         }
+      }
+      // this tile's P buffer was last read by the P V of tile t - 2
+      if (t >= 2) {
+        ok = mbar_wait(&pv_done[t & 1], ((t >> 1) & 1) ^ 1);
+        if (!ok) break;
+        tc_fence_after_sync();
       }
 
       float rs[4] = {0.f, 0.f, 0.f, 0.f};
@@ -357,19 +367,19 @@ gate_attn_tc_kernel(const __grid_constant__ CUtensorMap tmHi, const __grid_const
           ph[e >> 1] = pack_bf16x2(h0, h1);
           pl[e >> 1] = pack_bf16x2(l0, l1);
         }
-        tmem_st_x8(tm_lane + kGaColPhi + c * 8, ph);
-        tmem_st_x8(tm_lane + kGaColPlo + c * 8, pl);
+        tmem_st_x8(tm_lane + kGaColPhi + (t & 1) * (kGaBN / 2) + c * 8, ph);
+        tmem_st_x8(tm_lane + kGaColPlo + (t & 1) * (kGaBN / 2) + c * 8, pl);
       }
       const float rowsum = (rs[0] + rs[1]) + (rs[2] + rs[3]);
       l += rowsum;
       m = m_new;
       tmem_st_wait();
       tc_fence_before_sync();
-      mbar_arrive(p_ready);
+      mbar_arrive(&p_ready[t & 1]);
     }
 
     if (ok) {
-      ok = mbar_wait(pv_done, (t0 + n_kv - 1) & 1);
+      ok = mbar_wait(&pv_done[(t0 + n_kv - 1) & 1], ((t0 + n_kv - 1) >> 1) & 1);
       tc_fence_after_sync();
     }
     if (ok) {
